@@ -1,0 +1,251 @@
+/*
+ * dsp.h -- C ABI of the B200-native draft-and-verify core of DiffuSpec.
+ *
+ * One speculative step works on logits only (the two language models are the
+ * caller's): dsp_lattice_build turns the diffusion drafter's [B,L,V] block
+ * logits into the token lattice, dsp_cps_search picks one left-to-right path
+ * through it, dsp_verify checks that path against the target model's
+ * [B,Lt,V] logits, dsp_adl_update (host) sets the next draft length.
+ *
+ * Conventions
+ *  - Every function returns 0 (DSP_OK) or a negative dsp_status.  Argument
+ *    errors are detected on the host before anything is enqueued.
+ *  - Unless marked "host", every pointer is a DEVICE pointer to memory the
+ *    caller owns (inputs, outputs and the scratch workspace).  The library
+ *    allocates nothing and keeps no device state between calls.
+ *  - Device calls only enqueue work on `stream` (a cudaStream_t; NULL is the
+ *    legacy default stream) and never synchronise.  Outputs are valid once
+ *    the stream reaches the end of the call.  Two calls that share a
+ *    workspace must be ordered (same stream, or an event between them).
+ *  - Data-dependent conditions are reported per batch row in row_status[B]
+ *    (bit flags below), never as a return code.
+ *  - Tensors are row-major.  Logits have the vocabulary dimension contiguous;
+ *    stride_b / stride_l are in elements.  dtype is DSP_F32 or DSP_BF16.
+ *    Rows whose first element is 16-byte aligned are read with 128-bit loads;
+ *    any other layout takes an element-wise CUDA path (slower, same results).
+ *  - Positions, ranks and slots are 0-based (the paper counts from 1).
+ *  - -inf logits are legal (masked tokens).  NaN or +inf logits, or a row with
+ *    no finite logit, set DSP_ROW_NONFINITE_INPUT; that row's outputs are then
+ *    unspecified but in bounds.  Finite logits must exceed -1e37.
+ *  - The total order on tokens of one row is (logit descending, token id
+ *    ascending): the lowest id wins every tie (-0.0 and +0.0 are equal).
+ */
+#ifndef DSP_H_
+#define DSP_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef void *dsp_stream_t;   /* a cudaStream_t */
+
+enum dsp_status {
+    DSP_OK = 0,
+    DSP_ERR_INVALID_ARG = -1,   /* null pointer, non-positive size, bad stride ... */
+    DSP_ERR_UNSUPPORTED = -2,   /* dtype, K_max, W or L beyond the compiled limits */
+    DSP_ERR_WORKSPACE = -3,     /* workspace_bytes smaller than the query call's answer */
+    DSP_ERR_CUDA = -4           /* a CUDA runtime call failed; see dsp_last_cuda_error */
+};
+
+enum dsp_dtype { DSP_F32 = 0, DSP_BF16 = 1 };
+
+/* row_status bit flags */
+#define DSP_ROW_NONFINITE_INPUT 1u  /* NaN/+inf logit, or no finite logit, in a row of this batch row */
+#define DSP_ROW_ZERO_RESIDUAL   2u  /* residual mass was 0: replacement = target argmax */
+#define DSP_ROW_NO_BONUS_ROW    4u  /* whole path accepted and no target row path_len exists */
+#define DSP_ROW_EOS_ACCEPTED    8u  /* an accepted token is EOS: the caller terminates decoding */
+#define DSP_ROW_EOS_STOPPED     16u /* the path search stopped early at an EOS */
+
+#define DSP_MAX_K 32      /* largest K_max (per-position candidate cap M_max) */
+#define DSP_MAX_W 32      /* largest beam width */
+#define DSP_MAX_L 1024    /* largest draft length */
+
+const char *dsp_strerror(int32_t status);   /* host; static string */
+int32_t dsp_last_cuda_error(void);          /* host; the cudaError_t behind the last DSP_ERR_CUDA */
+int32_t dsp_version(void);                  /* host; ABI version, currently 1 */
+
+/* -------------------------------------------------------------------------
+ * Lattice build  (Sec. 3.2 "Lattice and pruning", Eq. 7; Alg. 1 stage 1;
+ *                 the generation-length signal of Eq. 9)
+ *
+ * For every row (b,l) of draft_logits, in one pass over its V logits:
+ *   lse      = log sum_v exp(x_v)                 (l^dlm(v) = x_v - lse)
+ *   entropy  = lse - sum_v x_v exp(x_v - lse)     (nats; -inf logits add 0)
+ *   the K = min(K_max, V) best tokens under the total order, -inf ones dropped
+ *   (at least one is kept), with their exact logits and log-probabilities;
+ *   cand_count = Eq. 7: the smallest m <= K whose cumulative full-vocabulary
+ *   probability reaches tau, K if none does.  Pruning is off unless
+ *   0 < tau <= 1.  If eos_id >= 0, EOS is not among the kept candidates and its
+ *   logit is finite, EOS is appended as one extra slot ("always keep EOS");
+ *   that slot is not counted in Eq. 7.
+ *   gen_len[b] = number of positions before the first whose best token is
+ *   eos_id (L if none, or if eos_id < 0)                          (Eq. 9)
+ *
+ * Inputs : draft_logits [B,L,V] (dtype), strides in elements.
+ * Outputs: cand_id    int32 [B,L,KC]   KC = K_max + (eos_id >= 0 ? 1 : 0);
+ *          cand_logit float [B,L,KC]   unused slots: id -1, logit -inf, logp -inf
+ *          cand_logp  float [B,L,KC]
+ *          cand_count int32 [B,L]
+ *          lse        float [B,L]      (nullable)
+ *          lse64      double[B,L]      the same value in double; dsp_cps_search
+ *                                      and dsp_verify read it
+ *          entropy    float [B,L]      (nullable)
+ *          gen_len    int32 [B]
+ *          row_status uint32[B]        overwritten
+ * workspace: at least dsp_lattice_workspace_bytes(...) bytes, 256-byte aligned;
+ *          contents need not be initialised and are garbage afterwards.
+ * Errors : INVALID_ARG (null required pointer, B<0, L<1, V<1, stride < V ...),
+ *          UNSUPPORTED (dtype, K_max outside 1..DSP_MAX_K, L > DSP_MAX_L),
+ *          WORKSPACE, CUDA.  B == 0 is a no-op returning DSP_OK.
+ */
+int32_t dsp_lattice_workspace_bytes(int32_t B, int32_t L, int32_t V, int32_t dtype,
+                                    int32_t K_max, size_t *bytes /* host, out */);
+
+int32_t dsp_lattice_build(const void *draft_logits, int32_t dtype,
+                          int32_t B, int32_t L, int32_t V,
+                          int64_t stride_b, int64_t stride_l,
+                          int32_t K_max, float tau, int32_t eos_id,
+                          int32_t *cand_id, float *cand_logit, float *cand_logp,
+                          int32_t *cand_count, float *lse, double *lse64, float *entropy,
+                          int32_t *gen_len, uint32_t *row_status,
+                          void *workspace, size_t workspace_bytes, dsp_stream_t stream);
+
+/* -------------------------------------------------------------------------
+ * Causal-consistency path search  (Sec. 3.2 "Scoring and search", Eq. 8;
+ *                                   Alg. 1 stage 2)
+ *
+ * Left-to-right beam search of width W over the lattice.  A path pi_1..pi_m
+ * scores  S(pi) = sum_i [ lambda * l^dlm_i(pi_i) + (1-lambda) * l^ng(pi_{i-1}, pi_i) ]
+ * with pi_0 = prev_token[b] (the last token of the prefix).  All live beams
+ * have equal depth, so they are ranked on the fp32 quantity
+ *   cum = sum_i step_i,  g = x - x_top1(i),
+ *   step = fl( fl(lambda*g) + fl((1-lambda)*n) ),  cum = fl(cum + step),
+ * (fl = round to fp32, no fused multiply-add, 1-lambda = fl(1 - lambda)), which
+ * differs from Eq. 8 by a term common to all beams; survivors are the best
+ * min(W, #expansions) under (cum descending, token id ascending, parent rank
+ * ascending).  The search stops after the first depth at which the rank-0
+ * survivor's new token is eos_id (row flag DSP_ROW_EOS_STOPPED).
+ *
+ * Causal proxy l^ng (the paper's n-gram model, here a caller-supplied bigram
+ * table of fp32 scores):
+ *   proxy_kind 0: hashed table of 2^table_log2 entries, 1 <= table_log2 <= 31.
+ *     With all arithmetic on uint32 modulo 2^32:
+ *       h = prev * 0x9E3779B1;  h ^= cur + hash_seed;  h *= 0x9E3779B1;
+ *       h ^= h >> 15;  h *= 0x9E3779B1;  h ^= h >> 13;
+ *       l^ng = proxy_table[h >> (32 - table_log2)]
+ *   proxy_kind 1: dense table [V,V]: l^ng = proxy_table[prev * V + cur].
+ *
+ * Inputs : cand_id, cand_logit, cand_count, lse64 as written by
+ *          dsp_lattice_build (KC = their last dimension); prev_token int32 [B].
+ * Outputs: path       int32 [B,L]   rank-0 path, -1 beyond path_len
+ *          path_slot  int32 [B,L]   candidate slot of each path token, -1 beyond
+ *          path_len   int32 [B]     m
+ *          path_score float [B]     Eq. 8 of the rank-0 path
+ *          beam_ids   int32 [B,W,L] (nullable) all survivors by rank, -1 padded
+ *          beam_score float [B,W]   (nullable) Eq. 8 per survivor, -inf if none
+ *          beam_cum   float [B,W]   (nullable) the ranking quantity, -inf if none
+ *          row_status uint32[B]     (nullable) flags OR-ed into existing content
+ * Errors : INVALID_ARG, UNSUPPORTED (W outside 1..DSP_MAX_W, KC > DSP_MAX_K+1,
+ *          L > DSP_MAX_L, proxy_kind), CUDA.
+ */
+int32_t dsp_cps_search(const int32_t *cand_id, const float *cand_logit,
+                       const double *lse64, const int32_t *cand_count,
+                       int32_t B, int32_t L, int32_t KC,
+                       const int32_t *prev_token,
+                       int32_t proxy_kind, const float *proxy_table, int32_t table_log2,
+                       uint32_t hash_seed, int32_t V,
+                       int32_t W, float lambda, int32_t eos_id,
+                       int32_t *path, int32_t *path_slot, int32_t *path_len, float *path_score,
+                       int32_t *beam_ids, float *beam_score, float *beam_cum,
+                       uint32_t *row_status, dsp_stream_t stream);
+
+/* -------------------------------------------------------------------------
+ * Verification  (Sec. 2: acceptance rule Eq. 1, residual resampling, accepted
+ *                length Eq. 2; Sec. 4: greedy = temperature 0; Alg. 1 stage 3;
+ *                the drafter probability q is the draft row's own softmax, the
+ *                left-to-right proxy of Eq. 6 under one refinement step)
+ *
+ * mode[b] == 0 (greedy): token i < m is accepted iff it equals the argmax of
+ *   target row i; the correction at the first rejection is that argmax.
+ * mode[b] != 0 (stochastic): ratio_i = p_i(y_i) / q_i(y_i) evaluated in
+ *   double; accepted iff u[b,i] < ratio_i; at the first rejection the
+ *   replacement is the inverse-CDF draw, in token-id order with the single
+ *   uniform u[b,L], from the residual max(0, p_i - q_i): the smallest v with
+ *   positive residual whose cumulative residual reaches u * (total residual).
+ *   A total of 0 gives the target argmax and DSP_ROW_ZERO_RESIDUAL.
+ * accepted_len[b] = index of the first rejection, or m = path_len[b].
+ * If all m are accepted and m < Lt, next_token is the bonus token from target
+ * row m (argmax, or the same inverse-CDF draw from p_m); if m == Lt it is -1
+ * and DSP_ROW_NO_BONUS_ROW is set.  An accepted EOS sets DSP_ROW_EOS_ACCEPTED.
+ *
+ * all_greedy != 0 promises that every row is greedy: mode, u, draft_logits,
+ * cand_logit, path_slot and draft_lse64 may then be NULL, no exponentials are
+ * evaluated and tgt_lse is not written.
+ *
+ * Inputs : target_logits [B,Lt,V], L <= Lt <= L+1; draft_logits [B,L,V] (same
+ *          dtype); path, path_slot, path_len from dsp_cps_search; cand_logit
+ *          [B,L,KC] and draft_lse64 [B,L] from dsp_lattice_build;
+ *          mode uint8 [B]; u float [B,L+1] in [0,1).
+ * Outputs: accepted_len int32 [B]; next_token int32 [B];
+ *          ratio      float [B,L]   (nullable) p/q at every i < m of a stochastic
+ *                                   row, -1 elsewhere
+ *          tgt_argmax int32 [B,Lt]  (nullable)
+ *          tgt_lse    float [B,Lt]  (nullable; only written if !all_greedy)
+ *          row_status uint32[B]     flags OR-ed into existing content
+ * workspace: at least dsp_verify_workspace_bytes(...) bytes, 256-byte aligned.
+ * Errors : INVALID_ARG, UNSUPPORTED, WORKSPACE, CUDA.
+ */
+int32_t dsp_verify_workspace_bytes(int32_t B, int32_t L, int32_t Lt, int32_t V, int32_t dtype,
+                                   size_t *bytes /* host, out */);
+
+int32_t dsp_verify(const void *target_logits, int32_t dtype,
+                   int32_t B, int32_t L, int32_t Lt, int32_t V,
+                   int64_t tstride_b, int64_t tstride_l,
+                   const void *draft_logits, int64_t dstride_b, int64_t dstride_l,
+                   const int32_t *path, const int32_t *path_slot, const int32_t *path_len,
+                   const float *cand_logit, const double *draft_lse64, int32_t KC,
+                   int32_t all_greedy, const uint8_t *mode, const float *u, int32_t eos_id,
+                   int32_t *accepted_len, int32_t *next_token, float *ratio,
+                   int32_t *tgt_argmax, float *tgt_lse, uint32_t *row_status,
+                   void *workspace, size_t workspace_bytes, dsp_stream_t stream);
+
+/* -------------------------------------------------------------------------
+ * Adaptive draft length  (Sec. 3.3, Eq. 9-11; Alg. 1 init and stage 4) -- host.
+ *
+ * State is plain data owned by the caller (copy it to checkpoint it).
+ *   init  : both moving averages 0, k = k_max.
+ *   update: ema = (1-rho)*ema + rho*signal for the batch means of gen_len and
+ *           accepted_len (batch 1 is the paper's setting), then
+ *           k = clip(ceil(ema_gen + delta * [ema_acc >= ema_gen]), k_min, k_max),
+ *           the ceiling first rounded up to a multiple of `granularity`
+ *           (1 = the paper's rule).  All arithmetic in double.
+ * accepted_len / gen_len are HOST pointers (the caller copies the two [B]
+ * arrays back; that copy is the step's only device-to-host traffic).
+ * Errors : INVALID_ARG (null pointer, B < 1, k_min < 1, k_min > k_max,
+ *          rho outside (0,1], delta < 0, granularity < 1).
+ */
+typedef struct dsp_adl_params {
+    int32_t k_min, k_max;
+    double delta;
+    double rho;
+    int32_t granularity;
+} dsp_adl_params;
+
+typedef struct dsp_adl_state {
+    double ema_gen, ema_acc;
+    int32_t k;        /* draft length for the next step */
+    int32_t steps;    /* updates so far */
+} dsp_adl_state;
+
+int32_t dsp_adl_init(dsp_adl_state *state, const dsp_adl_params *params);
+int32_t dsp_adl_update(dsp_adl_state *state, const dsp_adl_params *params,
+                       const int32_t *accepted_len, const int32_t *gen_len, int32_t B,
+                       int32_t *next_L /* host, out, nullable */);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* DSP_H_ */

@@ -1,0 +1,229 @@
+"""Thin ctypes binding of the C ABI in ``include/dsp.h`` (argument marshalling only).
+
+Functions carry the C entry points' names.  Tensors are torch CUDA tensors whose
+``data_ptr()`` is handed to the library; outputs and the scratch workspace are
+allocated here with torch (or passed in by the caller to reuse them) and the
+call is enqueued on torch's current stream.  There is no CPU fallback: if the
+CUDA library is missing or a call fails, an exception is raised.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from types import SimpleNamespace
+from typing import Optional
+
+import torch
+
+_PKG = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_PKG, "libdsp.so")
+
+DSP_OK, DSP_ERR_INVALID_ARG, DSP_ERR_UNSUPPORTED, DSP_ERR_WORKSPACE, DSP_ERR_CUDA = 0, -1, -2, -3, -4
+DSP_F32, DSP_BF16 = 0, 1
+ROW_NONFINITE_INPUT, ROW_ZERO_RESIDUAL, ROW_NO_BONUS_ROW, ROW_EOS_ACCEPTED, ROW_EOS_STOPPED = 1, 2, 4, 8, 16
+DSP_MAX_K, DSP_MAX_W, DSP_MAX_L = 32, 32, 1024
+
+EXPORTS = ["dsp_strerror", "dsp_last_cuda_error", "dsp_version", "dsp_lattice_workspace_bytes",
+           "dsp_lattice_build", "dsp_cps_search", "dsp_verify_workspace_bytes", "dsp_verify",
+           "dsp_adl_init", "dsp_adl_update"]
+
+
+class DspError(RuntimeError):
+    def __init__(self, fn: str, code: int):
+        msg = lib().dsp_strerror(code).decode()
+        if code == DSP_ERR_CUDA:
+            msg += " [cudaError %d]" % lib().dsp_last_cuda_error()
+        super().__init__("%s: %s (%d)" % (fn, msg, code))
+        self.code = code
+
+
+class AdlParams(C.Structure):
+    _fields_ = [("k_min", C.c_int32), ("k_max", C.c_int32), ("delta", C.c_double),
+                ("rho", C.c_double), ("granularity", C.c_int32)]
+
+
+class AdlState(C.Structure):
+    _fields_ = [("ema_gen", C.c_double), ("ema_acc", C.c_double), ("k", C.c_int32),
+                ("steps", C.c_int32)]
+
+
+_lib = None
+
+
+def lib():
+    """Load ``libdsp.so`` (built in-tree by ``paper_2510_02358_b200.build``); raises if absent."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise ImportError("CUDA library %s is not built; run paper_2510_02358_b200.build.build()"
+                              % LIB_PATH)
+        l = C.CDLL(LIB_PATH)
+        l.dsp_strerror.restype = C.c_char_p
+        l.dsp_strerror.argtypes = [C.c_int32]
+        for name in EXPORTS[1:]:
+            getattr(l, name).restype = C.c_int32
+        _lib = l
+    return _lib
+
+
+def _check(fn: str, code: int):
+    if code != DSP_OK:
+        raise DspError(fn, code)
+
+
+def _ptr(t: Optional[torch.Tensor]):
+    return C.c_void_p(0 if t is None else t.data_ptr())
+
+
+def _dtype(t: torch.Tensor) -> int:
+    if t.dtype == torch.float32:
+        return DSP_F32
+    if t.dtype == torch.bfloat16:
+        return DSP_BF16
+    raise DspError("dtype", DSP_ERR_UNSUPPORTED)
+
+
+def _stream(stream) -> C.c_void_p:
+    s = torch.cuda.current_stream() if stream is None else stream
+    return C.c_void_p(s.cuda_stream)
+
+
+def _logits3(t: torch.Tensor, name: str):
+    if t.dim() != 3 or not t.is_cuda or t.stride(2) != 1:
+        raise ValueError("%s must be a CUDA tensor [B, L, V] with a contiguous vocabulary dimension" % name)
+    return t.shape[0], t.shape[1], t.shape[2], t.stride(0), t.stride(1)
+
+
+def dsp_version() -> int:
+    return lib().dsp_version()
+
+
+def dsp_lattice_workspace_bytes(B: int, L: int, V: int, dtype: int, K_max: int) -> int:
+    n = C.c_size_t(0)
+    _check("dsp_lattice_workspace_bytes",
+           lib().dsp_lattice_workspace_bytes(B, L, V, dtype, K_max, C.byref(n)))
+    return n.value
+
+
+def dsp_verify_workspace_bytes(B: int, L: int, Lt: int, V: int, dtype: int) -> int:
+    n = C.c_size_t(0)
+    _check("dsp_verify_workspace_bytes", lib().dsp_verify_workspace_bytes(B, L, Lt, V, dtype, C.byref(n)))
+    return n.value
+
+
+def alloc_workspace(nbytes: int, device) -> torch.Tensor:
+    return torch.empty((max(nbytes, 256),), dtype=torch.uint8, device=device)
+
+
+def lattice_outputs(B: int, L: int, K_max: int, eos_id: int, device) -> SimpleNamespace:
+    KC = K_max + (1 if eos_id >= 0 else 0)
+    e = lambda shape, dt: torch.empty(shape, dtype=dt, device=device)
+    return SimpleNamespace(
+        cand_id=e((B, L, KC), torch.int32), cand_logit=e((B, L, KC), torch.float32),
+        cand_logp=e((B, L, KC), torch.float32), cand_count=e((B, L), torch.int32),
+        lse=e((B, L), torch.float32), lse64=e((B, L), torch.float64), entropy=e((B, L), torch.float32),
+        gen_len=e((B,), torch.int32), row_status=e((B,), torch.int32))
+
+
+def dsp_lattice_build(draft: torch.Tensor, K_max: int, tau: float = 0.0, eos_id: int = -1,
+                      out: Optional[SimpleNamespace] = None, workspace: Optional[torch.Tensor] = None,
+                      stream=None) -> SimpleNamespace:
+    B, L, V, sb, sl = _logits3(draft, "draft")
+    dt = _dtype(draft)
+    if out is None:
+        out = lattice_outputs(B, L, K_max, eos_id, draft.device)
+    if workspace is None:
+        workspace = alloc_workspace(dsp_lattice_workspace_bytes(B, L, V, dt, K_max), draft.device)
+    _check("dsp_lattice_build", lib().dsp_lattice_build(
+        _ptr(draft), dt, B, L, V, C.c_int64(sb), C.c_int64(sl), K_max, C.c_float(tau), eos_id,
+        _ptr(out.cand_id), _ptr(out.cand_logit), _ptr(out.cand_logp), _ptr(out.cand_count),
+        _ptr(out.lse), _ptr(out.lse64), _ptr(out.entropy), _ptr(out.gen_len), _ptr(out.row_status),
+        _ptr(workspace), C.c_size_t(workspace.numel()), _stream(stream)))
+    return out
+
+
+def cps_outputs(B: int, L: int, W: int, device, beams: bool = True) -> SimpleNamespace:
+    e = lambda shape, dt: torch.empty(shape, dtype=dt, device=device)
+    return SimpleNamespace(
+        path=e((B, L), torch.int32), path_slot=e((B, L), torch.int32), path_len=e((B,), torch.int32),
+        path_score=e((B,), torch.float32),
+        beam_ids=e((B, W, L), torch.int32) if beams else None,
+        beam_score=e((B, W), torch.float32) if beams else None,
+        beam_cum=e((B, W), torch.float32) if beams else None)
+
+
+def dsp_cps_search(lat: SimpleNamespace, prev_token: torch.Tensor, table: torch.Tensor, *, W: int,
+                   lam: float, eos_id: int = -1, proxy_kind: int = 0, table_log2: int = 0,
+                   hash_seed: int = 0, V: int = 1, out: Optional[SimpleNamespace] = None,
+                   row_status: Optional[torch.Tensor] = None, beams: bool = True,
+                   stream=None) -> SimpleNamespace:
+    B, L, KC = lat.cand_id.shape
+    if out is None:
+        out = cps_outputs(B, L, W, lat.cand_id.device, beams)
+    _check("dsp_cps_search", lib().dsp_cps_search(
+        _ptr(lat.cand_id), _ptr(lat.cand_logit), _ptr(lat.lse64), _ptr(lat.cand_count), B, L, KC,
+        _ptr(prev_token), proxy_kind, _ptr(table), table_log2, C.c_uint32(hash_seed & 0xFFFFFFFF), V,
+        W, C.c_float(lam), eos_id, _ptr(out.path), _ptr(out.path_slot), _ptr(out.path_len),
+        _ptr(out.path_score), _ptr(out.beam_ids), _ptr(out.beam_score), _ptr(out.beam_cum),
+        _ptr(row_status), _stream(stream)))
+    return out
+
+
+def verify_outputs(B: int, L: int, Lt: int, device) -> SimpleNamespace:
+    e = lambda shape, dt: torch.empty(shape, dtype=dt, device=device)
+    return SimpleNamespace(
+        accepted_len=e((B,), torch.int32), next_token=e((B,), torch.int32),
+        ratio=e((B, L), torch.float32), tgt_argmax=e((B, Lt), torch.int32),
+        tgt_lse=e((B, Lt), torch.float32))
+
+
+def dsp_verify(target: torch.Tensor, draft: Optional[torch.Tensor], cps: SimpleNamespace,
+               lat: Optional[SimpleNamespace], *, mode: Optional[torch.Tensor] = None,
+               u: Optional[torch.Tensor] = None, eos_id: int = -1, all_greedy: bool = False,
+               row_status: torch.Tensor, out: Optional[SimpleNamespace] = None,
+               workspace: Optional[torch.Tensor] = None, stream=None) -> SimpleNamespace:
+    B, Lt, V, tsb, tsl = _logits3(target, "target")
+    L = cps.path.shape[1]
+    dt = _dtype(target)
+    dsb = dsl = 0
+    if draft is not None:
+        Bd, Ld, Vd, dsb, dsl = _logits3(draft, "draft")
+        if (Bd, Ld, Vd) != (B, L, V) or draft.dtype != target.dtype:
+            raise ValueError("draft must be [B, L, V] with the target's dtype")
+    if out is None:
+        out = verify_outputs(B, L, Lt, target.device)
+    if workspace is None:
+        workspace = alloc_workspace(dsp_verify_workspace_bytes(B, L, Lt, V, dt), target.device)
+    KC = lat.cand_logit.shape[2] if lat is not None else 1
+    _check("dsp_verify", lib().dsp_verify(
+        _ptr(target), dt, B, L, Lt, V, C.c_int64(tsb), C.c_int64(tsl),
+        _ptr(draft), C.c_int64(dsb), C.c_int64(dsl),
+        _ptr(cps.path), _ptr(cps.path_slot), _ptr(cps.path_len),
+        _ptr(lat.cand_logit if lat is not None else None),
+        _ptr(lat.lse64 if lat is not None else None), KC,
+        1 if all_greedy else 0, _ptr(mode), _ptr(u), eos_id,
+        _ptr(out.accepted_len), _ptr(out.next_token), _ptr(out.ratio), _ptr(out.tgt_argmax),
+        _ptr(out.tgt_lse), _ptr(row_status), _ptr(workspace), C.c_size_t(workspace.numel()),
+        _stream(stream)))
+    return out
+
+
+def dsp_adl_init(k_min=20, k_max=30, delta=10.0, rho=0.5, granularity=1):
+    """Returns (state, params) for dsp_adl_update; the paper's defaults (Sec. 4)."""
+    p = AdlParams(int(k_min), int(k_max), float(delta), float(rho), int(granularity))
+    st = AdlState()
+    _check("dsp_adl_init", lib().dsp_adl_init(C.byref(st), C.byref(p)))
+    return st, p
+
+
+def dsp_adl_update(state: AdlState, params: AdlParams, accepted_len, gen_len) -> int:
+    """accepted_len / gen_len: host int32 tensors or sequences of equal length B."""
+    a = torch.as_tensor(accepted_len, dtype=torch.int32, device="cpu").contiguous().view(-1)
+    g = torch.as_tensor(gen_len, dtype=torch.int32, device="cpu").contiguous().view(-1)
+    if a.numel() != g.numel():
+        raise ValueError("accepted_len and gen_len must have the same length")
+    nxt = C.c_int32(0)
+    _check("dsp_adl_update", lib().dsp_adl_update(
+        C.byref(state), C.byref(params), C.c_void_p(a.data_ptr()), C.c_void_p(g.data_ptr()),
+        a.numel(), C.byref(nxt)))
+    return nxt.value

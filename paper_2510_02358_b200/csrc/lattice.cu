@@ -1,0 +1,263 @@
+// dsp_lattice_build: draft logits -> token lattice (Sec. 3.2 "Lattice and pruning", Eq. 7, Eq. 9).
+//
+// One kernel.  Each row (b,l) is cut into slices of whole tiles; one CTA streams one slice
+// once from HBM (log-sum-exp terms + exact top-K, see scan_core.cuh).  A row split over
+// several CTAs is finished by whichever CTA arrives last (atomic ticket): no CTA waits.
+// The CTA that finishes the last row of a batch row also writes gen_len and row_status.
+#include "scan_core.cuh"
+
+namespace dsp {
+
+struct LatticeArgs {
+    const void *logits;
+    int B, L, V;
+    long long stride_b, stride_l;
+    int K;          // min(K_max, V)
+    int K_max, KC;
+    float tau;
+    int eos_id;
+    int nslices, slice_elems;
+    int32_t *cand_id;
+    float *cand_logit, *cand_logp;
+    int32_t *cand_count;
+    float *lse;
+    double *lse64;
+    float *entropy;
+    int32_t *gen_len;
+    uint32_t *row_status;
+    // workspace
+    unsigned *row_ticket;     // [B*L]   zeroed per call
+    unsigned *b_ticket;       // [B]     zeroed per call
+    unsigned *b_status;       // [B]     zeroed per call
+    SlicePartial *partials;   // [B*L, nslices]
+    unsigned long long *keys; // [B*L, nslices, K]
+};
+
+struct LatticeWs {
+    size_t off_row_ticket, off_b_ticket, off_b_status, zero_bytes, off_partials, off_keys, total;
+};
+static LatticeWs lattice_ws_layout(int64_t B, int64_t L, int nslices, int K) {
+    LatticeWs w;
+    size_t o = 0;
+    w.off_row_ticket = o; o += align_up((size_t)(B * L) * 4, 256);
+    w.off_b_ticket = o;   o += align_up((size_t)B * 4, 256);
+    w.off_b_status = o;   o += align_up((size_t)B * 4, 256);
+    w.zero_bytes = o;
+    w.off_partials = o;   o += align_up((size_t)(B * L) * nslices * sizeof(SlicePartial), 256);
+    w.off_keys = o;       o += align_up((size_t)(B * L) * nslices * K * 8, 256);
+    w.total = o;
+    return w;
+}
+
+template <typename DT>
+__global__ void __launch_bounds__(kThreads, 4) lattice_kernel(const LatticeArgs a) {
+    __shared__ ScanSmem sm;
+    const int tid = threadIdx.x;
+    const long long row = blockIdx.x / a.nslices;
+    const int slice = blockIdx.x - (int)(row * a.nslices);
+    const int b = (int)(row / a.L), l = (int)(row - (long long)b * a.L);
+    const DT *rowp = reinterpret_cast<const DT *>(a.logits) + b * a.stride_b + l * a.stride_l;
+    const int s0 = slice * a.slice_elems;
+    const int s1 = min(a.V, s0 + a.slice_elems);
+
+    float c;
+    double S, T;
+    scan_slice<DT, true>(rowp, s0, s1, a.K, sm, c, S, T);
+
+    if (a.nslices > 1) {
+        SlicePartial *part = a.partials + row * a.nslices;
+        unsigned long long *keys = a.keys + (row * a.nslices + slice) * a.K;
+        const int nk = sm.cnt;
+        if (tid < nk) keys[tid] = sm.cand[tid];
+        if (tid == 0) {
+            part[slice].S = S; part[slice].T = T; part[slice].c = c; part[slice].nkeys = nk;
+        }
+        __threadfence();
+        __syncthreads();
+        if (tid == 0) sm.flag = (int)atomicAdd(&a.row_ticket[row], 1u);
+        __syncthreads();
+        if (sm.flag != a.nslices - 1) return;
+        __threadfence();
+        // last CTA of this row: gather every slice's keys and sums
+        if (tid == 0) sm.cnt = 0;
+        __syncthreads();
+        for (int s = 0; s < a.nslices; ++s) {
+            const int n = __ldcg(&part[s].nkeys);
+            const unsigned long long *ks = a.keys + (row * a.nslices + s) * a.K;
+            if (tid < n) sm.cand[s * a.K + tid] = __ldcg(&ks[tid]);
+            else if (tid < a.K) sm.cand[s * a.K + tid] = 0ull;     // below every real key
+        }
+        if (tid == 0) sm.cnt = a.nslices * a.K;
+        prune(sm, a.K);
+        if (tid == 0) {
+            int n = 0;                                  // drop the padding keys again
+            while (n < sm.cnt && sm.cand[n] != 0ull) ++n;
+            sm.cnt = n;
+            merge_partials(part, a.nslices, c, S, T);
+            sm.fin[0] = S; sm.fin[1] = T; sm.redc[0] = c;
+        }
+        __syncthreads();
+        S = sm.fin[0]; T = sm.fin[1]; c = sm.redc[0];
+    }
+
+    // ---- finalise the row: sm.cand[0..cnt) sorted best keys, (c,S,T) whole-row sums ----
+    const int nk = sm.cnt;
+    double lse, mean_x;
+    const bool ok = row_log_stats(c, S, T, lse, mean_x);
+    if (tid < nk) sm.pk[tid] = exp((double)key_value(sm.cand[tid]) - lse);
+    __syncthreads();
+    if (tid == 0) {
+        int count = nk;
+        if (a.tau > 0.f && a.tau <= 1.f && ok) {       // Eq. 7 on full-vocabulary probabilities
+            const double tau = (double)a.tau;
+            double cum = 0.0;
+            for (int k = 0; k < nk; ++k) {
+                cum += sm.pk[k];
+                if (cum >= tau) { count = k + 1; break; }
+            }
+        }
+        int eos_slot = -1;
+        float eos_x = 0.f;
+        if (a.eos_id >= 0 && a.eos_id < a.V) {          // always keep EOS
+            bool has = false;
+            for (int k = 0; k < count; ++k) has |= key_id(sm.cand[k]) == a.eos_id;
+            if (!has) {
+                eos_x = Elem<DT>::load1(rowp + a.eos_id);
+                if (eos_x > -CUDART_INF_F && eos_x < CUDART_INF_F) eos_slot = count;
+            }
+        }
+        sm.flag = count;
+        sm.overflow = eos_slot;
+        sm.thr_v = eos_x;
+        a.cand_count[row] = count + (eos_slot >= 0 ? 1 : 0);
+        if (a.lse) a.lse[row] = (float)lse;
+        a.lse64[row] = lse;
+        if (a.entropy) a.entropy[row] = (float)(lse - mean_x);
+        if (!ok) atomicOr(&a.b_status[b], DSP_ROW_NONFINITE_INPUT);
+    }
+    __syncthreads();
+    if (tid < a.KC) {
+        const int count = sm.flag, eos_slot = sm.overflow;
+        int id = -1;
+        float x = -CUDART_INF_F, lp = -CUDART_INF_F;
+        if (tid < count) {
+            id = key_id(sm.cand[tid]);
+            x = key_value(sm.cand[tid]);
+            lp = (float)((double)x - lse);
+        } else if (tid == eos_slot) {
+            id = a.eos_id;
+            x = sm.thr_v;
+            lp = (float)((double)x - lse);
+        }
+        const long long o = row * a.KC + tid;
+        a.cand_id[o] = id;
+        a.cand_logit[o] = x;
+        a.cand_logp[o] = lp;
+    }
+    // ---- last row of this batch row: generation length (Eq. 9) and status ----
+    __threadfence();
+    __syncthreads();
+    if (tid == 0) {
+        const unsigned t = atomicAdd(&a.b_ticket[b], 1u);
+        if (t == (unsigned)a.L - 1) {
+            __threadfence();
+            int g = a.L;
+            if (a.eos_id >= 0) {
+                for (int i = 0; i < a.L; ++i) {
+                    if (__ldcg(&a.cand_id[((long long)b * a.L + i) * a.KC]) == a.eos_id) { g = i; break; }
+                }
+            }
+            a.gen_len[b] = g;
+            a.row_status[b] = atomicOr(&a.b_status[b], 0u);
+        }
+    }
+}
+
+template <typename DT>
+static int32_t launch_lattice(LatticeArgs &a, void *workspace, size_t workspace_bytes, cudaStream_t st) {
+    const long long nrows = (long long)a.B * a.L;
+    const SlicePlan plan = plan_slices<DT>(nrows, a.V, 148 * 8);
+    a.nslices = plan.nslices;
+    a.slice_elems = plan.slice_elems;
+    const LatticeWs w = lattice_ws_layout(a.B, a.L, a.nslices, a.K);
+    if (workspace_bytes < w.total) return DSP_ERR_WORKSPACE;
+    char *ws = reinterpret_cast<char *>(workspace);
+    a.row_ticket = reinterpret_cast<unsigned *>(ws + w.off_row_ticket);
+    a.b_ticket = reinterpret_cast<unsigned *>(ws + w.off_b_ticket);
+    a.b_status = reinterpret_cast<unsigned *>(ws + w.off_b_status);
+    a.partials = reinterpret_cast<SlicePartial *>(ws + w.off_partials);
+    a.keys = reinterpret_cast<unsigned long long *>(ws + w.off_keys);
+    DSP_CUDA_TRY(cudaMemsetAsync(ws, 0, w.zero_bytes, st));
+    const long long nblocks = nrows * a.nslices;
+    if (nblocks > 0x7FFFFFFFLL) return DSP_ERR_UNSUPPORTED;
+    lattice_kernel<DT><<<(unsigned)nblocks, kThreads, 0, st>>>(a);
+    DSP_CUDA_TRY(cudaGetLastError());
+    return DSP_OK;
+}
+
+template <typename DT>
+static size_t lattice_ws_bytes(int B, int L, int V, int K) {
+    const SlicePlan plan = plan_slices<DT>((long long)B * L, V, 148 * 8);
+    return lattice_ws_layout(B, L, plan.nslices, K).total;
+}
+
+}  // namespace dsp
+
+using namespace dsp;
+
+static int32_t check_lattice_shape(int32_t B, int32_t L, int32_t V, int32_t dtype, int32_t K_max) {
+    if (B < 0 || L < 1 || V < 1) return DSP_ERR_INVALID_ARG;
+    if (dtype != DSP_F32 && dtype != DSP_BF16) return DSP_ERR_UNSUPPORTED;
+    if (K_max < 1 || K_max > DSP_MAX_K || L > DSP_MAX_L || V > (1 << 30)) return DSP_ERR_UNSUPPORTED;
+    return DSP_OK;
+}
+
+extern "C" int32_t dsp_lattice_workspace_bytes(int32_t B, int32_t L, int32_t V, int32_t dtype,
+                                               int32_t K_max, size_t *bytes) {
+    if (!bytes) return DSP_ERR_INVALID_ARG;
+    const int32_t rc = check_lattice_shape(B, L, V, dtype, K_max);
+    if (rc != DSP_OK) return rc;
+    const int K = K_max < V ? K_max : V;
+    const int Bq = B > 0 ? B : 1;
+    *bytes = dtype == DSP_BF16 ? lattice_ws_bytes<__nv_bfloat16>(Bq, L, V, K)
+                               : lattice_ws_bytes<float>(Bq, L, V, K);
+    return DSP_OK;
+}
+
+extern "C" int32_t dsp_lattice_build(const void *draft_logits, int32_t dtype,
+                                     int32_t B, int32_t L, int32_t V,
+                                     int64_t stride_b, int64_t stride_l,
+                                     int32_t K_max, float tau, int32_t eos_id,
+                                     int32_t *cand_id, float *cand_logit, float *cand_logp,
+                                     int32_t *cand_count, float *lse, double *lse64, float *entropy,
+                                     int32_t *gen_len, uint32_t *row_status,
+                                     void *workspace, size_t workspace_bytes, dsp_stream_t stream) {
+    const int32_t rc = check_lattice_shape(B, L, V, dtype, K_max);
+    if (rc != DSP_OK) return rc;
+    if (B == 0) return DSP_OK;
+    if (!draft_logits || !cand_id || !cand_logit || !cand_logp || !cand_count || !lse64 ||
+        !gen_len || !row_status || !workspace)
+        return DSP_ERR_INVALID_ARG;
+    if (stride_l < V || stride_b < 0 || (B > 1 && stride_b < (int64_t)(L - 1) * stride_l + V))
+        return DSP_ERR_INVALID_ARG;
+    if (tau != tau) return DSP_ERR_INVALID_ARG;
+    if ((reinterpret_cast<uintptr_t>(workspace) & 255) != 0) return DSP_ERR_INVALID_ARG;
+    const size_t es = dtype == DSP_BF16 ? 2 : 4;
+    if ((reinterpret_cast<uintptr_t>(draft_logits) & (es - 1)) != 0) return DSP_ERR_INVALID_ARG;
+
+    LatticeArgs a;
+    a.logits = draft_logits;
+    a.B = B; a.L = L; a.V = V;
+    a.stride_b = stride_b; a.stride_l = stride_l;
+    a.K = K_max < V ? K_max : V;
+    a.K_max = K_max;
+    a.KC = K_max + (eos_id >= 0 ? 1 : 0);
+    a.tau = tau;
+    a.eos_id = eos_id;
+    a.cand_id = cand_id; a.cand_logit = cand_logit; a.cand_logp = cand_logp;
+    a.cand_count = cand_count; a.lse = lse; a.lse64 = lse64; a.entropy = entropy;
+    a.gen_len = gen_len; a.row_status = row_status;
+    cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+    return dtype == DSP_BF16 ? launch_lattice<__nv_bfloat16>(a, workspace, workspace_bytes, st)
+                             : launch_lattice<float>(a, workspace, workspace_bytes, st);
+}

@@ -1,0 +1,485 @@
+// dsp_verify: verification of the chosen path against the target logits
+// (Sec. 2: Eq. 1 acceptance, residual resampling, Eq. 2 accepted length; greedy = temperature 0).
+//
+// Kernel 1 (target_kernel): every target row is streamed once (argmax; log-sum-exp terms only
+// for stochastic batch rows).  The CTA that finishes the last row of a batch row runs that
+// row's left-to-right acceptance scan and either writes the next token (greedy) or records
+// a sampling job (stochastic: residual at the first rejection, or bonus from row m).
+// Kernel 2 (residual_kernel): for each job, one more pass over ONE target row (and ONE draft
+// row): per-chunk sums of max(0, p - q) in token order; the CTA arriving last inverts the CDF.
+#include "scan_core.cuh"
+
+namespace dsp {
+
+struct SampleJob {
+    int trow;        // target row index b*Lt + i, or -1: no job
+    int drow;        // draft row index b*L + i, or -1: draw from p itself (bonus token)
+    float u;
+    int fallback;    // target argmax of that row (used when the residual mass is 0)
+};
+
+struct VerifyArgs {
+    const void *target;
+    const void *draft;
+    int B, L, Lt, V;
+    long long tstride_b, tstride_l, dstride_b, dstride_l;
+    const int32_t *path, *path_slot, *path_len;
+    const float *cand_logit;
+    const double *draft_lse64;
+    int KC;
+    int all_greedy;
+    const uint8_t *mode;
+    const float *u;
+    int eos_id;
+    int32_t *accepted_len, *next_token;
+    float *ratio;
+    int32_t *tgt_argmax;
+    float *tgt_lse;
+    uint32_t *row_status;
+    int nslices, slice_elems;
+    // workspace
+    unsigned *row_ticket;      // [B*Lt]  zeroed per call
+    unsigned *b_ticket;        // [B]     zeroed per call
+    unsigned *res_ticket;      // [B]     zeroed per call
+    unsigned *b_status;        // [B]     zeroed per call
+    SlicePartial *partials;    // [B*Lt, nslices]
+    unsigned long long *keys;  // [B*Lt, nslices]
+    int32_t *argmax;           // [B*Lt]
+    double *tlse64;            // [B*Lt]
+    SampleJob *jobs;           // [B]
+    double *chunk_sums;        // [B, nchunks]
+    int nchunks, res_slices, chunks_per_slice;
+};
+
+template <typename DT>
+__device__ __forceinline__ const DT *trow_ptr(const VerifyArgs &a, long long trow) {
+    const long long b = trow / a.Lt, i = trow - b * a.Lt;
+    return reinterpret_cast<const DT *>(a.target) + b * a.tstride_b + i * a.tstride_l;
+}
+template <typename DT>
+__device__ __forceinline__ const DT *drow_ptr(const VerifyArgs &a, long long drow) {
+    const long long b = drow / a.L, i = drow - b * a.L;
+    return reinterpret_cast<const DT *>(a.draft) + b * a.dstride_b + i * a.dstride_l;
+}
+
+// Left-to-right acceptance of batch row b by one warp (Eq. 1, Eq. 2).
+template <typename DT>
+__device__ void accept_row(const VerifyArgs &a, int b) {
+    const int lane = threadIdx.x & 31;
+    const int L = a.L, Lt = a.Lt;
+    const int m = max(0, min(__ldcg(&a.path_len[b]), L));
+    const bool stoch = !a.all_greedy && a.mode[b] != 0;
+    int acc = m;
+    bool eos_seen_before_acc = false;
+    for (int i0 = 0; i0 < L; i0 += 32) {
+        const int i = i0 + lane;
+        bool rej = false;
+        float rt_out = -1.f;
+        if (i < m) {
+            const int y = __ldcg(&a.path[(long long)b * L + i]);
+            if (!stoch) {
+                rej = y != __ldcg(&a.argmax[(long long)b * Lt + i]);
+            } else {
+                const int slot = __ldcg(&a.path_slot[(long long)b * L + i]);
+                const double xt = (double)Elem<DT>::load1(trow_ptr<DT>(a, (long long)b * Lt + i) + y);
+                const double xd = (double)__ldcg(&a.cand_logit[((long long)b * L + i) * a.KC + slot]);
+                const double lp = xt - __ldcg(&a.tlse64[(long long)b * Lt + i]);
+                const double lq = xd - __ldcg(&a.draft_lse64[(long long)b * L + i]);
+                const double rt = exp(lp - lq);
+                rej = !((double)a.u[(long long)b * (L + 1) + i] < rt);
+                rt_out = (float)rt;
+            }
+        }
+        if (a.ratio && i < L) a.ratio[(long long)b * L + i] = rt_out;
+        const unsigned bal = __ballot_sync(0xFFFFFFFFu, rej);
+        if (bal && acc == m) acc = i0 + __ffs(bal) - 1;
+    }
+    if (a.eos_id >= 0) {
+        for (int i0 = 0; i0 < acc; i0 += 32) {
+            const int i = i0 + lane;
+            const bool e = i < acc && __ldcg(&a.path[(long long)b * L + i]) == a.eos_id;
+            if (__ballot_sync(0xFFFFFFFFu, e)) eos_seen_before_acc = true;
+        }
+    }
+    if (lane == 0) {
+        unsigned status = atomicOr(&a.b_status[b], 0u);
+        if (eos_seen_before_acc) status |= DSP_ROW_EOS_ACCEPTED;
+        SampleJob job;
+        job.trow = -1; job.drow = -1; job.u = 0.f; job.fallback = -1;
+        int nt = -1;
+        const int at = acc < m ? acc : m;              // row the next token comes from
+        if (acc < m || m < Lt) {
+            const int am = __ldcg(&a.argmax[(long long)b * Lt + at]);
+            if (!stoch) {
+                nt = am;
+            } else {
+                job.trow = b * Lt + at;
+                job.drow = acc < m ? b * L + at : -1;
+                job.u = a.u[(long long)b * (L + 1) + L];
+                job.fallback = am;
+            }
+        } else {
+            status |= DSP_ROW_NO_BONUS_ROW;
+        }
+        a.accepted_len[b] = acc;
+        a.next_token[b] = nt;
+        if (!a.all_greedy) a.jobs[b] = job;
+        if (status) atomicOr(&a.row_status[b], status);
+    }
+}
+
+template <typename DT>
+__global__ void __launch_bounds__(kThreads, 4) target_kernel(const VerifyArgs a) {
+    __shared__ ScanSmem sm;
+    const int tid = threadIdx.x;
+    const long long row = blockIdx.x / a.nslices;
+    const int slice = blockIdx.x - (int)(row * a.nslices);
+    const int b = (int)(row / a.Lt);
+    const DT *rowp = trow_ptr<DT>(a, row);
+    const int s0 = slice * a.slice_elems;
+    const int s1 = min(a.V, s0 + a.slice_elems);
+    const bool sums = !a.all_greedy && a.mode[b] != 0;
+
+    float c;
+    double S, T;
+    if (sums) scan_slice<DT, true>(rowp, s0, s1, 1, sm, c, S, T);
+    else      scan_slice<DT, false>(rowp, s0, s1, 1, sm, c, S, T);
+
+    unsigned long long best = sm.cnt > 0 ? sm.cand[0] : 0ull;
+    if (a.nslices > 1) {
+        SlicePartial *part = a.partials + row * a.nslices;
+        unsigned long long *keys = a.keys + row * a.nslices;
+        if (tid == 0) {
+            keys[slice] = best;
+            part[slice].S = S; part[slice].T = T; part[slice].c = c; part[slice].nkeys = sm.cnt;
+            __threadfence();
+            sm.flag = (int)atomicAdd(&a.row_ticket[row], 1u);
+        }
+        __syncthreads();
+        if (sm.flag != a.nslices - 1) return;
+        __threadfence();
+        if (tid == 0) {
+            best = 0ull;
+            for (int s = 0; s < a.nslices; ++s) {
+                const unsigned long long k = __ldcg(&keys[s]);
+                best = k > best ? k : best;
+            }
+            if (sums) merge_partials(part, a.nslices, c, S, T);
+        }
+    }
+    if (tid == 0) {
+        const int am = best ? key_id(best) : 0;
+        a.argmax[row] = am;
+        if (a.tgt_argmax) a.tgt_argmax[row] = am;
+        bool ok = best != 0ull;
+        if (sums) {
+            double lse, mean_x;
+            ok = row_log_stats(c, S, T, lse, mean_x) && ok;
+            a.tlse64[row] = lse;
+            if (a.tgt_lse) a.tgt_lse[row] = (float)lse;
+        } else if (a.tgt_lse && !a.all_greedy) {
+            a.tgt_lse[row] = CUDART_NAN_F;             // greedy row of a mixed batch: not computed
+        }
+        if (!ok) atomicOr(&a.b_status[b], DSP_ROW_NONFINITE_INPUT);
+        __threadfence();
+        sm.flag = (int)atomicAdd(&a.b_ticket[b], 1u);
+    }
+    __syncthreads();
+    if (sm.flag != a.Lt - 1) return;
+    __threadfence();
+    if (tid < 32) accept_row<DT>(a, b);
+}
+
+// ---- residual / bonus sampling -------------------------------------------------------------
+
+// p(v) = 2^(x*kLog2e - c2) with c2 = lse*log2(e) split as hi + lo (lo folded into `corr`).
+struct RowProb {
+    float nchi;     // -c2_hi
+    float corr;     // 2^(-c2_lo)
+};
+__device__ __forceinline__ RowProb row_prob(double lse) {
+    const double c2 = lse / kLn2;
+    RowProb r;
+    const float hi = (float)c2;
+    r.nchi = -hi;
+    r.corr = (float)exp2(-(c2 - (double)hi));
+    return r;
+}
+__device__ __forceinline__ float prob(float x, const RowProb &r) {
+    return __fmul_rn(ex2_approx(fmaf(x, kLog2e, r.nchi)), r.corr);
+}
+__device__ __forceinline__ float residual(float xt, float xd, const RowProb &pt, const RowProb &pd, bool has_q) {
+    const float p = prob(xt, pt);
+    const float q = has_q ? prob(xd, pd) : 0.f;
+    const float r = __fsub_rn(p, q);
+    return r > 0.f ? r : 0.f;                  // NaN -> 0
+}
+
+template <typename DT>
+__global__ void __launch_bounds__(kThreads, 4) residual_kernel(const VerifyArgs a) {
+    constexpr int N = Elem<DT>::N;
+    constexpr int CE = 32 * N;                  // elements per chunk: one warp-wide vector load
+    __shared__ double s_scan[kThreads];
+    __shared__ double s_total;
+    __shared__ int s_found;
+    __shared__ int s_flag;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int b = blockIdx.x / a.res_slices;
+    const int rs = blockIdx.x - b * a.res_slices;
+    const SampleJob job = a.jobs[b];
+    if (job.trow < 0) return;
+    const bool has_q = job.drow >= 0;
+    const DT *tp = trow_ptr<DT>(a, job.trow);
+    const DT *dp = has_q ? drow_ptr<DT>(a, job.drow) : tp;
+    const bool aligned = ((reinterpret_cast<uintptr_t>(tp) | reinterpret_cast<uintptr_t>(dp)) & 15) == 0;
+    const RowProb pt = row_prob(a.tlse64[job.trow]);
+    const RowProb pd = has_q ? row_prob(a.draft_lse64[job.drow]) : pt;
+    double *sums = a.chunk_sums + (long long)b * a.nchunks;
+    const int V = a.V;
+
+    const int c0 = rs * a.chunks_per_slice, c1 = min(a.nchunks, c0 + a.chunks_per_slice);
+    for (int ch = c0 + warp; ch < c1; ch += kWarps) {
+        const int e0 = ch * CE + lane * N;
+        const uint4 vt = load_vec<DT>(tp, e0, V, aligned);
+        const uint4 vd = has_q ? load_vec<DT>(dp, e0, V, aligned) : vt;
+        float s = 0.f;
+#pragma unroll
+        for (int e = 0; e < N; ++e)
+            s = __fadd_rn(s, residual(Elem<DT>::get(vt, e), Elem<DT>::get(vd, e), pt, pd, has_q));
+        const double cs = warp_sum((double)s);
+        if (lane == 0) sums[ch] = cs;
+    }
+    __threadfence();
+    __syncthreads();
+    if (tid == 0) s_flag = (int)atomicAdd(&a.res_ticket[b], 1u);
+    __syncthreads();
+    if (s_flag != a.res_slices - 1) return;
+    __threadfence();
+
+    // ---- last CTA of this job: invert the CDF ----
+    const int per = (a.nchunks + kThreads - 1) / kThreads;     // consecutive chunks per thread
+    const int k0 = min(a.nchunks, tid * per), k1 = min(a.nchunks, k0 + per);
+    double mine = 0.0;
+    for (int k = k0; k < k1; ++k) mine += __ldcg(&sums[k]);
+    s_scan[tid] = mine;
+    if (tid == 0) s_found = 0x7FFFFFFF;
+    __syncthreads();
+    // exclusive prefix of the 256 thread sums (serial in thread 0: 256 adds, fixed order)
+    if (tid == 0) {
+        double run = 0.0;
+        for (int t = 0; t < kThreads; ++t) { const double x = s_scan[t]; s_scan[t] = run; run += x; }
+        s_total = run;
+    }
+    __syncthreads();
+    const double R = s_total;
+    if (!(R > 0.0)) {
+        if (tid == 0) {
+            a.next_token[b] = job.fallback;
+            atomicOr(&a.row_status[b], DSP_ROW_ZERO_RESIDUAL);
+        }
+        return;
+    }
+    const double thr = (double)job.u * R;
+    {
+        double run = s_scan[tid];
+        for (int k = k0; k < k1; ++k) {
+            const double cs = __ldcg(&sums[k]);
+            run += cs;
+            if (cs > 0.0 && run >= thr) { atomicMin(&s_found, k); break; }
+        }
+    }
+    __syncthreads();
+    int ch = s_found;
+    if (ch == 0x7FFFFFFF) {                     // rounding at the very top: last chunk with mass
+        if (tid == 0) {
+            int last = -1;
+            for (int k = a.nchunks - 1; k >= 0; --k)
+                if (__ldcg(&sums[k]) > 0.0) { last = k; break; }
+            s_found = last;
+        }
+        __syncthreads();
+        ch = s_found;
+    }
+    if (warp != 0) return;
+    // prefix of everything before chunk ch, in the same association as above
+    double before = 0.0;
+    {
+        const int owner = min(kThreads - 1, ch / per);
+        before = s_scan[owner];
+        for (int k = owner * per; k < ch; ++k) before += __ldcg(&sums[k]);
+    }
+    const int e0 = ch * CE + lane * N;
+    const uint4 vt = load_vec<DT>(tp, e0, V, aligned);
+    const uint4 vd = has_q ? load_vec<DT>(dp, e0, V, aligned) : vt;
+    float r[N];
+    float s = 0.f;
+#pragma unroll
+    for (int e = 0; e < N; ++e) {
+        r[e] = residual(Elem<DT>::get(vt, e), Elem<DT>::get(vd, e), pt, pd, has_q);
+        s = __fadd_rn(s, r[e]);
+    }
+    // exclusive prefix over lanes (double)
+    double incl = (double)s;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const double up = __shfl_up_sync(0xFFFFFFFFu, incl, o);
+        if (lane >= o) incl += up;
+    }
+    double run = before + (incl - (double)s);
+    int hit = -1, lastpos = -1;
+#pragma unroll
+    for (int e = 0; e < N; ++e) {
+        run += (double)r[e];
+        if (r[e] > 0.f && e0 + e < V) {
+            lastpos = e0 + e;
+            if (hit < 0 && run >= thr) hit = e0 + e;
+        }
+    }
+    const unsigned bal = __ballot_sync(0xFFFFFFFFu, hit >= 0);
+    int tok;
+    if (bal) {
+        tok = __shfl_sync(0xFFFFFFFFu, hit, __ffs(bal) - 1);
+    } else {
+        const unsigned bl = __ballot_sync(0xFFFFFFFFu, lastpos >= 0);
+        tok = bl ? __shfl_sync(0xFFFFFFFFu, lastpos, 31 - __clz(bl)) : job.fallback;
+    }
+    if (lane == 0) a.next_token[b] = tok;
+}
+
+struct VerifyWs {
+    size_t off_row_ticket, off_b_ticket, off_res_ticket, off_b_status, zero_bytes;
+    size_t off_partials, off_keys, off_argmax, off_tlse, off_jobs, off_chunks, total;
+};
+static VerifyWs verify_ws_layout(int64_t B, int64_t Lt, int nslices, int nchunks) {
+    VerifyWs w;
+    size_t o = 0;
+    w.off_row_ticket = o; o += align_up((size_t)(B * Lt) * 4, 256);
+    w.off_b_ticket = o;   o += align_up((size_t)B * 4, 256);
+    w.off_res_ticket = o; o += align_up((size_t)B * 4, 256);
+    w.off_b_status = o;   o += align_up((size_t)B * 4, 256);
+    w.zero_bytes = o;
+    w.off_partials = o;   o += align_up((size_t)(B * Lt) * nslices * sizeof(SlicePartial), 256);
+    w.off_keys = o;       o += align_up((size_t)(B * Lt) * nslices * 8, 256);
+    w.off_argmax = o;     o += align_up((size_t)(B * Lt) * 4, 256);
+    w.off_tlse = o;       o += align_up((size_t)(B * Lt) * 8, 256);
+    w.off_jobs = o;       o += align_up((size_t)B * sizeof(SampleJob), 256);
+    w.off_chunks = o;     o += align_up((size_t)B * nchunks * 8, 256);
+    w.total = o;
+    return w;
+}
+
+template <typename DT>
+static int nchunks_of(int V) { return (V + 32 * Elem<DT>::N - 1) / (32 * Elem<DT>::N); }
+
+template <typename DT>
+static size_t verify_ws_bytes(int B, int Lt, int V) {
+    const SlicePlan plan = plan_slices<DT>((long long)B * Lt, V, 148 * 8);
+    return verify_ws_layout(B, Lt, plan.nslices, nchunks_of<DT>(V)).total;
+}
+
+template <typename DT>
+static int32_t launch_verify(VerifyArgs &a, void *workspace, size_t workspace_bytes, cudaStream_t st) {
+    const long long nrows = (long long)a.B * a.Lt;
+    const SlicePlan plan = plan_slices<DT>(nrows, a.V, 148 * 8);
+    a.nslices = plan.nslices;
+    a.slice_elems = plan.slice_elems;
+    a.nchunks = nchunks_of<DT>(a.V);
+    const VerifyWs w = verify_ws_layout(a.B, a.Lt, a.nslices, a.nchunks);
+    if (workspace_bytes < w.total) return DSP_ERR_WORKSPACE;
+    char *ws = reinterpret_cast<char *>(workspace);
+    a.row_ticket = reinterpret_cast<unsigned *>(ws + w.off_row_ticket);
+    a.b_ticket = reinterpret_cast<unsigned *>(ws + w.off_b_ticket);
+    a.res_ticket = reinterpret_cast<unsigned *>(ws + w.off_res_ticket);
+    a.b_status = reinterpret_cast<unsigned *>(ws + w.off_b_status);
+    a.partials = reinterpret_cast<SlicePartial *>(ws + w.off_partials);
+    a.keys = reinterpret_cast<unsigned long long *>(ws + w.off_keys);
+    a.argmax = reinterpret_cast<int32_t *>(ws + w.off_argmax);
+    a.tlse64 = reinterpret_cast<double *>(ws + w.off_tlse);
+    a.jobs = reinterpret_cast<SampleJob *>(ws + w.off_jobs);
+    a.chunk_sums = reinterpret_cast<double *>(ws + w.off_chunks);
+    // residual pass: about 4 CTAs per SM over all jobs, at least one chunk per warp
+    int rsl = (148 * 4 + a.B - 1) / a.B;
+    const int max_rsl = (a.nchunks + kWarps - 1) / kWarps;
+    if (rsl > max_rsl) rsl = max_rsl;
+    if (rsl < 1) rsl = 1;
+    a.chunks_per_slice = (a.nchunks + rsl - 1) / rsl;
+    a.res_slices = (a.nchunks + a.chunks_per_slice - 1) / a.chunks_per_slice;
+
+    DSP_CUDA_TRY(cudaMemsetAsync(ws, 0, w.zero_bytes, st));
+    const long long nblocks = nrows * a.nslices;
+    if (nblocks > 0x7FFFFFFFLL) return DSP_ERR_UNSUPPORTED;
+    target_kernel<DT><<<(unsigned)nblocks, kThreads, 0, st>>>(a);
+    DSP_CUDA_TRY(cudaGetLastError());
+    if (!a.all_greedy) {
+        residual_kernel<DT><<<(unsigned)(a.B * a.res_slices), kThreads, 0, st>>>(a);
+        DSP_CUDA_TRY(cudaGetLastError());
+    }
+    return DSP_OK;
+}
+
+}  // namespace dsp
+
+using namespace dsp;
+
+static int32_t check_verify_shape(int32_t B, int32_t L, int32_t Lt, int32_t V, int32_t dtype) {
+    if (B < 0 || L < 1 || V < 1 || Lt < L || Lt > L + 1) return DSP_ERR_INVALID_ARG;
+    if (dtype != DSP_F32 && dtype != DSP_BF16) return DSP_ERR_UNSUPPORTED;
+    if (L > DSP_MAX_L || V > (1 << 30)) return DSP_ERR_UNSUPPORTED;
+    return DSP_OK;
+}
+
+extern "C" int32_t dsp_verify_workspace_bytes(int32_t B, int32_t L, int32_t Lt, int32_t V,
+                                              int32_t dtype, size_t *bytes) {
+    if (!bytes) return DSP_ERR_INVALID_ARG;
+    const int32_t rc = check_verify_shape(B, L, Lt, V, dtype);
+    if (rc != DSP_OK) return rc;
+    const int Bq = B > 0 ? B : 1;
+    *bytes = dtype == DSP_BF16 ? verify_ws_bytes<__nv_bfloat16>(Bq, Lt, V)
+                               : verify_ws_bytes<float>(Bq, Lt, V);
+    return DSP_OK;
+}
+
+extern "C" int32_t dsp_verify(const void *target_logits, int32_t dtype,
+                              int32_t B, int32_t L, int32_t Lt, int32_t V,
+                              int64_t tstride_b, int64_t tstride_l,
+                              const void *draft_logits, int64_t dstride_b, int64_t dstride_l,
+                              const int32_t *path, const int32_t *path_slot, const int32_t *path_len,
+                              const float *cand_logit, const double *draft_lse64, int32_t KC,
+                              int32_t all_greedy, const uint8_t *mode, const float *u, int32_t eos_id,
+                              int32_t *accepted_len, int32_t *next_token, float *ratio,
+                              int32_t *tgt_argmax, float *tgt_lse, uint32_t *row_status,
+                              void *workspace, size_t workspace_bytes, dsp_stream_t stream) {
+    const int32_t rc = check_verify_shape(B, L, Lt, V, dtype);
+    if (rc != DSP_OK) return rc;
+    if (B == 0) return DSP_OK;
+    if (!target_logits || !path || !path_len || !accepted_len || !next_token || !row_status || !workspace)
+        return DSP_ERR_INVALID_ARG;
+    if (!all_greedy) {
+        if (!draft_logits || !path_slot || !cand_logit || !draft_lse64 || !mode || !u)
+            return DSP_ERR_INVALID_ARG;
+        if (KC < 1 || KC > DSP_MAX_K + 1) return DSP_ERR_UNSUPPORTED;
+        if (dstride_l < V || dstride_b < 0 || (B > 1 && dstride_b < (int64_t)(L - 1) * dstride_l + V))
+            return DSP_ERR_INVALID_ARG;
+    }
+    if (tstride_l < V || tstride_b < 0 || (B > 1 && tstride_b < (int64_t)(Lt - 1) * tstride_l + V))
+        return DSP_ERR_INVALID_ARG;
+    if ((reinterpret_cast<uintptr_t>(workspace) & 255) != 0) return DSP_ERR_INVALID_ARG;
+    const size_t es = dtype == DSP_BF16 ? 2 : 4;
+    if ((reinterpret_cast<uintptr_t>(target_logits) & (es - 1)) != 0) return DSP_ERR_INVALID_ARG;
+    if (draft_logits && (reinterpret_cast<uintptr_t>(draft_logits) & (es - 1)) != 0)
+        return DSP_ERR_INVALID_ARG;
+
+    VerifyArgs a;
+    a.target = target_logits; a.draft = draft_logits;
+    a.B = B; a.L = L; a.Lt = Lt; a.V = V;
+    a.tstride_b = tstride_b; a.tstride_l = tstride_l;
+    a.dstride_b = dstride_b; a.dstride_l = dstride_l;
+    a.path = path; a.path_slot = path_slot; a.path_len = path_len;
+    a.cand_logit = cand_logit; a.draft_lse64 = draft_lse64; a.KC = KC;
+    a.all_greedy = all_greedy ? 1 : 0; a.mode = mode; a.u = u; a.eos_id = eos_id;
+    a.accepted_len = accepted_len; a.next_token = next_token; a.ratio = ratio;
+    a.tgt_argmax = tgt_argmax; a.tgt_lse = tgt_lse; a.row_status = row_status;
+    cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+    return dtype == DSP_BF16 ? launch_verify<__nv_bfloat16>(a, workspace, workspace_bytes, st)
+                             : launch_verify<float>(a, workspace, workspace_bytes, st);
+}

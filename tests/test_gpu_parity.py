@@ -1,0 +1,181 @@
+"""GPU parity: the CUDA path, called through the C ABI, against the CPU oracle on the same bytes."""
+import math
+
+import pytest
+import torch
+
+from paper_2510_02358_b200 import binding as dsp
+from paper_2510_02358_b200 import workloads as wl
+from parity import check_step, gpu_step
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda"
+
+
+def _to(inp, dev=DEV):
+    return {k: (v.to(dev) if isinstance(v, torch.Tensor) else v) for k, v in inp.items()}
+
+
+def _params(w):
+    return dict(K=w.K, W=w.W, tau=w.tau, lam=w.lam, eos_id=w.eos_id, all_greedy=(w.verify == "greedy"))
+
+
+# ---- the five workloads at sizes the oracle finishes in seconds (several tiles + ragged tail) ----
+SMALL = {
+    1: dict(B=2, L=8, V=32000),
+    2: dict(B=1, L=16, V=152064, eos_from=9),
+    3: dict(B=4, L=6, V=152064),
+    4: dict(B=6, L=8, V=50021),         # odd V: rows are not 16-byte aligned -> element-wise path
+    5: dict(B=3, L=5, V=256000),
+}
+
+
+@pytest.mark.parametrize("cid", [1, 2, 3, 4, 5])
+def test_workloads_small(cid):
+    w = wl.CONFIGS[cid].scaled(**SMALL[cid])
+    inp = wl.make_inputs(w, step=1, device=DEV)
+    g = gpu_step(inp, **_params(w))
+    rep = check_step(g, inp, **_params(w))
+    print(cid, rep)
+    assert rep["near_accept"] + rep["near_token"] + rep["near_tau"] <= 2
+
+
+# ---- the benchmark's own launch configuration at full size, oracle on sampled batch rows ----
+@pytest.mark.parametrize("cid,rows", [(1, None), (2, None), (3, [0, 7, 15]), (4, [0, 1, 33, 62, 63]),
+                                      (5, [0, 101, 255])])
+def test_workloads_full_size_sampled_rows(cid, rows):
+    w = wl.CONFIGS[cid]
+    if cid == 2:
+        w = w.scaled(eos_from=21)
+    inp = wl.make_inputs(w, step=0, device=DEV)
+    g = gpu_step(inp, **_params(w))
+    rep = check_step(g, inp, rows=rows, **_params(w))
+    print(cid, rep)
+    # properties that hold for every row at any size
+    m = g.cps.path_len
+    assert ((g.ver.accepted_len >= 0) & (g.ver.accepted_len <= m) & (m <= w.L)).all()
+    bc = g.cps.beam_cum
+    assert (bc[:, :-1] >= bc[:, 1:]).all()
+    assert (g.lat.cand_count >= 1).all() and (g.lat.cand_count <= w.K + (w.eos_id >= 0)).all()
+    assert torch.isfinite(g.lat.lse).all() and (g.lat.entropy > 0).all()
+    assert (g.lat.entropy <= math.log(w.V) + 1e-3).all()
+    if w.verify == "greedy":
+        am = g.ver.tgt_argmax
+        for b in range(w.B):
+            mm = int(m[b])
+            match = (g.cps.path[b, :mm] == am[b, :mm]).tolist()
+            assert int(g.ver.accepted_len[b]) == (match.index(False) if False in match else mm)
+    del inp
+    torch.cuda.empty_cache()
+
+
+# ---- edge shapes ----
+@pytest.mark.parametrize("B,L,V,K,W,dtype", [
+    (2, 3, 5, 8, 4, torch.float32),          # V < K
+    (1, 1, 1, 1, 1, torch.float32),          # one token
+    (3, 2, 37, 4, 3, torch.bfloat16),        # V not a multiple of 8
+    (2, 100, 300, 3, 2, torch.float32),      # long draft
+    (2, 4, 8200, 1, 1, torch.bfloat16),      # K = 1, W = 1, just over one tile
+    (2, 3, 4099, 32, 32, torch.float32),     # largest K and W
+    (5, 7, 1000, 15, 3, torch.bfloat16),     # the paper's defaults M_max = 15, beam 3
+])
+def test_edge_shapes(B, L, V, K, W, dtype):
+    inp = _to(wl.tiny_random(B, L, V, dtype=dtype, seed=B * 100 + L))
+    for tau, eos in ((0.0, -1), (0.8, V - 1)):
+        p = dict(K=K, W=W, tau=tau, lam=0.5, eos_id=eos)
+        rep = check_step(gpu_step(inp, **p), inp, **p)
+        assert rep["near_accept"] + rep["near_token"] + rep["near_tau"] <= 1
+
+
+def test_target_with_bonus_row_and_all_greedy():
+    B, L, V = 4, 5, 3000
+    inp = _to(wl.tiny_random(B, L, V, dtype=torch.bfloat16, seed=3))
+    extra = (inp["target"][:, :1].float() * 0.5).to(torch.bfloat16)
+    inp["target"] = torch.cat([inp["target"], extra], dim=1).contiguous()      # Lt = L + 1
+    inp["target"][:, :L] = inp["draft"]                                         # everything accepted
+    for ag in (False, True):
+        p = dict(K=4, W=4, lam=1.0, all_greedy=ag)
+        g = gpu_step(inp, **p)
+        check_step(g, inp, **p)
+        greedy = torch.ones(B, dtype=torch.bool) if ag else (inp["mode"].cpu() == 0)
+        assert (g.ver.accepted_len[greedy] == L).all() and (g.ver.next_token >= 0).all()
+
+
+def test_ties_everywhere_and_degenerate_rows():
+    B, L, V = 3, 2, 20000
+    base = wl.tiny_random(B, L, V, dtype=torch.bfloat16, seed=5)
+    d = base["draft"]
+    d[0] = 1.5                                            # uniform rows: every token ties
+    d[1, 0] = torch.arange(V, dtype=torch.float32).mul(1e-3).to(torch.bfloat16)   # ascending, many ties
+    d[1, 1] = torch.arange(V, 0, -1, dtype=torch.float32).mul(1e-3).to(torch.bfloat16)
+    d[2] = torch.round(d[2].float()).to(torch.bfloat16)   # few distinct values
+    base["target"] = (d.float() + 0.25 * torch.round(base["target"].float())).to(torch.bfloat16)
+    inp = _to(base)
+    p = dict(K=16, W=8, tau=0.0, lam=0.5)
+    g = gpu_step(inp, **p)
+    check_step(g, inp, **p)
+    assert g.lat.cand_id[0, 0].tolist() == list(range(16))
+
+
+def test_masked_logits_and_nonfinite_flags():
+    B, L, V = 4, 3, 9000
+    base = wl.tiny_random(B, L, V, dtype=torch.float32, seed=6)
+    ninf = -float("inf")
+    base["draft"][0, :, 100:] = ninf                      # 100 allowed tokens
+    base["target"][0, :, 100:] = ninf
+    base["draft"][1, 1, 5:] = ninf                        # fewer finite logits than K
+    base["draft"][2, 0, 77] = float("nan")
+    base["target"][3, 2, 5] = float("inf")
+    inp = _to(base)
+    p = dict(K=8, W=4, lam=0.5)
+    g = gpu_step(inp, **p)
+    check_step(g, inp, **p)
+    st = g.lat.row_status
+    assert st[2] & dsp.ROW_NONFINITE_INPUT and st[3] & dsp.ROW_NONFINITE_INPUT
+    assert not (st[0] & dsp.ROW_NONFINITE_INPUT) and not (st[1] & dsp.ROW_NONFINITE_INPUT)
+    assert g.lat.cand_count[1, 1].item() == 5
+
+
+def test_strided_and_offset_views():
+    B, L, V = 3, 4, 10000
+    base = wl.tiny_random(B, L, V + 24, dtype=torch.bfloat16, seed=8)
+    inp = _to(base)
+    full_d, full_t = inp["draft"], inp["target"]
+    for off in (0, 3, 8):                                 # 3: rows start 6 bytes off a 16-byte boundary
+        view_d, view_t = full_d[:, :, off:off + V], full_t[:, :, off:off + V]
+        assert not view_d.is_contiguous()
+        inp2 = dict(inp, draft=view_d.contiguous(), target=view_t.contiguous())
+        p = dict(K=8, W=8, lam=0.5)
+        g = gpu_step(inp, draft=view_d, target=view_t, **p)
+        check_step(g, inp2, **p)
+
+
+def test_run_to_run_determinism():
+    w = wl.CONFIGS[3].scaled(B=4, L=4, V=152064)
+    inp = wl.make_inputs(w, device=DEV)
+    a, b = gpu_step(inp, **_params(w)), gpu_step(inp, **_params(w))
+    for s in ("lat", "cps", "ver"):
+        for k, v in vars(getattr(a, s)).items():
+            assert torch.equal(v.view(torch.uint8), getattr(getattr(b, s), k).view(torch.uint8)), (s, k)
+
+
+def test_adl_closed_loop_matches_oracle():
+    """Configuration 2's loop: the draft length of each step comes from the controller."""
+    import oracle
+    w = wl.CONFIGS[2].scaled(V=20000, eos_id=19999)
+    st, prm = dsp.dsp_adl_init(**wl.ADL_C2)
+    ref = oracle.Adl(**wl.ADL_C2)
+    walk = wl.eos_walk(12)
+    seen = set()
+    for t, c in enumerate(walk):
+        L = st.k
+        assert L == ref.k and L in (8, 16, 24, 32)
+        seen.add(L)
+        ws = w.scaled(L=L, eos_from=c if c < L else -1)
+        inp = wl.make_inputs(ws, step=t, device=DEV)
+        g = gpu_step(inp, **_params(ws))
+        check_step(g, inp, **_params(ws))
+        nxt = dsp.dsp_adl_update(st, prm, g.ver.accepted_len, g.lat.gen_len)
+        assert nxt == ref.update(g.ver.accepted_len, g.lat.gen_len)
+        assert abs(st.ema_gen - ref.ema_gen) < 1e-12 and abs(st.ema_acc - ref.ema_acc) < 1e-12
+    assert len(seen) >= 2
