@@ -1,0 +1,416 @@
+#!/usr/bin/env python
+"""Benchmark of the draft-and-verify step (lattice build -> path search -> verify [-> ADL]).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--config 1..5] [--impl reference]
+
+One "step" is one pass of the whole hot path over one batch of seeded synthetic
+logits.  The headline workload is configuration 4 (B=64, L=32, V=152064, bf16,
+Eq. 7 pruning, mixed greedy/stochastic rows): 623 MB per logits tensor, far
+larger than L2, so every step streams from HBM.  Smaller configurations rotate
+over several input sets for the same reason.  Rank 0 prints ONE JSON line.
+
+Batch rows are independent, so with N GPUs every rank runs the same per-GPU
+workload on its own rows (weak scaling, no collective on the data path); the
+time is the maximum over ranks and the value the steps all ranks completed per
+second.
+
+--impl reference times the CPU oracle (plain C, as it stands) on a bounded
+sample of the same workload on this machine's host cores.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_2510_02358_b200 import workloads as wl  # noqa: E402
+
+L2_BYTES = 126 * 1024 * 1024
+HEADLINE = 4
+# DRAM bytes per launch of lattice_kernel from one ncu capture (see profiles/); None = not captured.
+NCU_TRAFFIC_BYTES = {}
+
+
+def measured_peak():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        return float(json.load(open(p))["hbm_gbs"]), "measured"
+    except Exception:
+        return 6650.0, "fallback"
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+         "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.f = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+        self.p = None
+        try:
+            self.p = subprocess.Popen(["nvidia-smi", "-i", str(gpu_index), "--query-gpu=" + self.Q,
+                                       "--format=csv,noheader,nounits", "-lms", "100"],
+                                      stdout=self.f, stderr=subprocess.DEVNULL)
+        except Exception:
+            self.p = None
+
+    def stop(self) -> dict:
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.p is None:
+            return out
+        self.p.terminate()
+        try:
+            self.p.wait(timeout=5)
+        except Exception:
+            self.p.kill()
+        self.f.flush()
+        self.f.seek(0)
+        sm, mx, power = [], [], []
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        seen = set()
+        for line in self.f.read().splitlines():
+            c = [x.strip() for x in line.split(",")]
+            if len(c) < 9:
+                continue
+            try:
+                sm.append(float(c[1])); mx.append(float(c[2])); power.append(float(c[3]))
+            except ValueError:
+                continue
+            for n, v in zip(names, c[5:9]):
+                if v.lower().startswith("active"):
+                    seen.add(n)
+        self.f.close()
+        os.unlink(self.f.name)
+        if sm:
+            out.update(sm_mhz=statistics.median(sm), sm_max_mhz=max(mx), samples=len(sm),
+                       power_w_max=max(power))
+        out["reasons"] = sorted(seen)
+        return out
+
+
+def params_of(w):
+    return dict(K=w.K, W=w.W, tau=w.tau, lam=w.lam, eos_id=w.eos_id)
+
+
+class GpuStep:
+    """Pre-allocated outputs and workspaces for one workload; ``run(inp)`` enqueues one step."""
+
+    def __init__(self, w, device):
+        from paper_2510_02358_b200 import binding as dsp
+        self.dsp, self.w, self.dev = dsp, w, device
+        dt = dsp.DSP_BF16 if w.dtype == torch.bfloat16 else dsp.DSP_F32
+        self.lat = dsp.lattice_outputs(w.B, w.L, w.K, w.eos_id, device)
+        self.cps = dsp.cps_outputs(w.B, w.L, w.W, device, beams=True)
+        self.ver = dsp.verify_outputs(w.B, w.L, w.Lt, device)
+        self.ws_l = dsp.alloc_workspace(dsp.dsp_lattice_workspace_bytes(w.B, w.L, w.V, dt, w.K), device)
+        self.ws_v = dsp.alloc_workspace(dsp.dsp_verify_workspace_bytes(w.B, w.L, w.Lt, w.V, dt), device)
+        self.all_greedy = w.verify == "greedy"
+        self.kernels_per_step = 3 if self.all_greedy else 4     # lattice, cps, target (+ residual)
+
+    def run(self, inp, ev=None):
+        dsp, w = self.dsp, self.w
+        if ev:
+            ev[0].record()
+        dsp.dsp_lattice_build(inp["draft"], w.K, w.tau, w.eos_id, out=self.lat, workspace=self.ws_l)
+        if ev:
+            ev[1].record()
+        dsp.dsp_cps_search(self.lat, inp["prev_token"], inp["table"], W=w.W, lam=w.lam, eos_id=w.eos_id,
+                           table_log2=inp["table_log2"], hash_seed=inp["hash_seed"], V=w.V,
+                           out=self.cps, row_status=self.lat.row_status)
+        if ev:
+            ev[2].record()
+        if self.all_greedy:
+            dsp.dsp_verify(inp["target"], None, self.cps, None, eos_id=w.eos_id, all_greedy=True,
+                           row_status=self.lat.row_status, out=self.ver, workspace=self.ws_v)
+        else:
+            dsp.dsp_verify(inp["target"], inp["draft"], self.cps, self.lat, mode=inp["mode"], u=inp["u"],
+                           eos_id=w.eos_id, row_status=self.lat.row_status, out=self.ver,
+                           workspace=self.ws_v)
+        if ev:
+            ev[3].record()
+
+
+def reduce_max_ms(ms: float, dist, device) -> float:
+    """Slowest rank's time (the job's time); identity on one rank."""
+    if dist is None:
+        return ms
+    t = torch.tensor([ms], device=device, dtype=torch.float64)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return t.item()
+
+
+def whole_job_steps_per_s(world: int, steps: int, ms: float) -> float:
+    """Every rank completes ``steps`` steps on its own batch rows in ``ms`` (max over ranks)."""
+    return world * steps / (ms * 1e-3)
+
+
+def rank_seed_base(rank: int) -> int:
+    """Each rank draws its own batch rows: disjoint seed ranges per rank."""
+    return rank * 1000
+
+
+def input_sets(w, device, seed_base=0):
+    step_bytes = wl.step_logits_bytes(w)
+    n = 1 if step_bytes > 4 * L2_BYTES else min(16, -(-4 * L2_BYTES // step_bytes))
+    return [wl.make_inputs(w, step=seed_base + i, device=device) for i in range(n)]
+
+
+def time_workload(w, device, steps, warmup, dist=None, stages=True, seed_base=0):
+    """Device-timed throughput of one workload; returns a dict of measurements."""
+    sets = input_sets(w, device, seed_base)
+    st = GpuStep(w, device)
+    for i in range(warmup):
+        st.run(sets[i % len(sets)])
+    torch.cuda.synchronize()
+    evs = [[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in range(steps)] if stages else None
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    if dist is not None:
+        dist.barrier()
+    torch.cuda.synchronize()
+    e0.record()
+    for i in range(steps):
+        st.run(sets[i % len(sets)], evs[i] if stages else None)
+    e1.record()
+    torch.cuda.synchronize()
+    if dist is not None:
+        dist.barrier()
+    ms = e0.elapsed_time(e1)
+    out = dict(ms_total=ms, ms_per_step=ms / steps, sets=len(sets), kernels_per_step=st.kernels_per_step)
+    if stages:
+        tl = [e[0].elapsed_time(e[1]) for e in evs]
+        tc = [e[1].elapsed_time(e[2]) for e in evs]
+        tv = [e[2].elapsed_time(e[3]) for e in evs]
+        out.update(ms_lattice=sum(tl) / steps, ms_cps=sum(tc) / steps, ms_verify=sum(tv) / steps,
+                   ms_lattice_min=min(tl), ms_verify_min=min(tv))
+    out["mean_accepted_len"] = st.ver.accepted_len.float().mean().item()
+    out["mean_path_len"] = st.cps.path_len.float().mean().item()
+    return out, st, sets
+
+
+def time_e2e(w, st, sets, device, steps):
+    """Same step through the public calls with HOST buffers: pinned logits are copied to the
+    device inside the timed region and the step's results are read back every step."""
+    inp = sets[0]
+    host = {k: inp[k].cpu().pin_memory() for k in ("draft", "target", "prev_token", "mode", "u")}
+    dev = {k: torch.empty_like(inp[k]) for k in host}
+    res_host = torch.empty((3, w.B), dtype=torch.int32).pin_memory()
+    h2d = sum(t.numel() * t.element_size() for t in host.values())
+    d2h = res_host.numel() * 4
+    staged = dict(inp)
+
+    def one():
+        for k in host:
+            dev[k].copy_(host[k], non_blocking=True)
+        staged.update(dev)
+        st.run(staged)
+        res_host[0].copy_(st.ver.accepted_len, non_blocking=True)
+        res_host[1].copy_(st.ver.next_token, non_blocking=True)
+        res_host[2].copy_(st.lat.gen_len, non_blocking=True)
+        torch.cuda.current_stream().synchronize()          # the caller needs the result to go on
+
+    one()
+    torch.cuda.synchronize()
+    t0 = time.perf_counter()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(steps):
+        one()
+    e1.record()
+    torch.cuda.synchronize()
+    wall = (time.perf_counter() - t0) * 1e3
+    ms = max(e0.elapsed_time(e1), wall)
+    return dict(value=steps / (ms / 1e3), unit="steps/s", h2d_bytes_per_step=h2d, d2h_bytes_per_step=d2h,
+                steps=steps, ms_per_step=ms / steps)
+
+
+def oracle_step(w, inp_cpu, rows):
+    """The oracle's whole step on the first ``rows`` batch rows; returns seconds."""
+    import oracle
+    sl = slice(0, rows)
+    d, t = inp_cpu["draft"][sl].contiguous(), inp_cpu["target"][sl].contiguous()
+    t0 = time.perf_counter()
+    lat = oracle.lattice_build(d, w.K, tau=w.tau, eos_id=w.eos_id)
+    cps = oracle.cps_search(lat.cand_id, lat.cand_logit, lat.lse64, lat.cand_count,
+                            inp_cpu["prev_token"][sl], inp_cpu["table"], W=w.W, lam=w.lam, eos_id=w.eos_id,
+                            table_log2=inp_cpu["table_log2"], hash_seed=inp_cpu["hash_seed"], V=w.V)
+    if w.verify == "greedy":
+        oracle.verify(t, None, cps.path, cps.path_len, None, None, eos_id=w.eos_id)
+    else:
+        oracle.verify(t, d, cps.path, cps.path_len, inp_cpu["mode"][sl], inp_cpu["u"][sl], eos_id=w.eos_id)
+    return time.perf_counter() - t0
+
+
+def cpu_inputs(inp, rows):
+    """CPU copies of the first ``rows`` batch rows of one input set."""
+    out = {}
+    for k, v in inp.items():
+        if isinstance(v, torch.Tensor):
+            out[k] = v.cpu() if k == "table" else v[:rows].cpu().contiguous()
+        else:
+            out[k] = v
+    return out
+
+
+def cpu_baseline(w, inp, budget_s=20.0):
+    """Oracle (kind=oracle) timed on a bounded sample of the workload's batch rows."""
+    import oracle
+    oracle.build()
+    cores = oracle.threads()
+    rows = min(w.B, max(1, cores))
+    t = oracle_step(w, cpu_inputs(inp, rows), rows)
+    if t < budget_s / 4 and rows < w.B:              # grow the sample while it stays cheap
+        grow = min(8.0, budget_s / 2 / max(t, 1e-3))
+        rows2 = min(w.B, max(rows, int(rows * grow) // cores * cores))
+        if rows2 > rows:
+            rows = rows2
+            t = oracle_step(w, cpu_inputs(inp, rows), rows)
+    step_s = t * w.B / rows
+    return dict(value=1.0 / step_s, unit="steps/s", cores=cores, kind="oracle",
+                sample="first %d of %d batch rows, one step, %.2f s of CPU wall-clock; scaled by B/rows"
+                       % (rows, w.B, t))
+
+
+def run_reference(args, rank, world):
+    if rank != 0:
+        return
+    import oracle
+    oracle.build()
+    w = wl.CONFIGS[args.config]
+    cores = oracle.threads()
+    rows = min(w.B, max(1, cores))
+    inp = wl.make_inputs(w.scaled(B=rows), step=0, device="cpu")
+    for _ in range(args.warmup):
+        oracle_step(w, inp, rows)
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        oracle_step(w, inp, rows)
+    t = (time.perf_counter() - t0) / args.steps
+    step_s = t * w.B / rows
+    val = 1.0 / step_s
+    sample = "each step = first %d of %d batch rows (same recipe and seed), scaled by B/rows" % (rows, w.B)
+    print(json.dumps({
+        "impl": "reference", "metric": "draft-verify steps/s", "value": val, "unit": "steps/s",
+        "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup, "ms_per_step": step_s * 1e3,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "f64", "data": "synthetic",
+        "config": {"workload": w.name, "B": w.B, "L": w.L, "V": w.V, "K": w.K, "W": w.W, "tau": w.tau,
+                   "verify": w.verify},
+        "cpu_baseline": {"value": val, "unit": "steps/s", "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": val, "unit": "steps/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--config", type=int, default=HEADLINE, choices=sorted(wl.CONFIGS))
+    ap.add_argument("--impl", default="dsp", choices=["dsp", "reference"])
+    ap.add_argument("--no-extras", action="store_true", help="skip the other four workloads and the CPU baseline")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "dsp" else args.warmup
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if args.impl == "reference":
+        run_reference(args, rank, world)
+        return
+
+    from paper_2510_02358_b200 import build
+    build.build()
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")
+    torch.cuda.set_device(local)
+    device = torch.device("cuda", local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist_mod
+        dist_mod.init_process_group("nccl", device_id=device)
+        dist = dist_mod
+
+    w = wl.CONFIGS[args.config]
+    sampler = ClockSampler(local) if rank == 0 else None
+    m, st, sets = time_workload(w, device, args.steps, args.warmup, dist, seed_base=rank_seed_base(rank))
+    clocks = sampler.stop() if sampler else None
+    ms = reduce_max_ms(m["ms_total"], dist, device)
+    e2e = time_e2e(w, st, sets, device, min(args.steps, 10))
+    if dist is not None:
+        e2e["ms_per_step"] = reduce_max_ms(e2e["ms_per_step"], dist, device)
+        e2e["value"] = whole_job_steps_per_s(world, 1, e2e["ms_per_step"])
+        e2e["h2d_bytes_per_step"] *= world
+        e2e["d2h_bytes_per_step"] *= world
+    if rank != 0:
+        if dist is not None:
+            dist.destroy_process_group()
+        return
+
+    peak, peak_kind = measured_peak()
+    tensor_bytes = w.logits_bytes
+    gbs_lat = tensor_bytes / (m["ms_lattice"] * 1e-3) / 1e9
+    gbs_ver = tensor_bytes / (m["ms_verify"] * 1e-3) / 1e9
+    gbs_both = 2 * tensor_bytes / ((m["ms_lattice"] + m["ms_verify"]) * 1e-3) / 1e9
+    line = {
+        "metric": "draft-verify steps/s", "value": whole_job_steps_per_s(world, args.steps, ms), "unit": "steps/s",
+        "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms / args.steps,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "f32", "data": "synthetic",
+        "config": {"workload": w.name, "B": w.B * world, "B_per_gpu": w.B, "L": w.L, "V": w.V,
+                   "logits_dtype": "bf16" if w.dtype == torch.bfloat16 else "f32", "K": w.K, "W": w.W,
+                   "tau": w.tau, "verify": w.verify, "parallelism": "batch rows sharded, no collective",
+                   "l2": "inputs larger than L2" if m["sets"] == 1 else "rotating %d input sets" % m["sets"]},
+        "logits_gbs": {"lattice_build": gbs_lat, "verify": gbs_ver, "lattice_plus_verify": gbs_both,
+                       "frac_of_8000": gbs_both / 8000.0, "frac_of_%s_copy_peak" % peak_kind: gbs_both / peak},
+        "stage_ms": {"lattice_build": m["ms_lattice"], "cps_search": m["ms_cps"], "verify": m["ms_verify"]},
+        "mean_accepted_len": m["mean_accepted_len"], "mean_path_len": m["mean_path_len"],
+        "roofline": {"bound": "hbm", "kernel": "lattice_kernel", "achieved": gbs_lat, "peak": peak,
+                     "peak_kind": "%s copy bandwidth" % peak_kind, "unit": "GB/s", "frac": gbs_lat / peak,
+                     "traffic": NCU_TRAFFIC_BYTES.get(w.cid),
+                     "algorithmic_bytes_per_launch": tensor_bytes},
+        "e2e": e2e,
+        "gpu_launches": m["kernels_per_step"] * args.steps,
+        "clocks": clocks,
+    }
+    if not args.no_extras and world == 1:
+        line["cpu_baseline"] = cpu_baseline(w, sets[0])
+        extras = {}
+        del st, sets
+        torch.cuda.empty_cache()
+        for cid in sorted(wl.CONFIGS):
+            if cid == args.config:
+                continue
+            variants = [wl.CONFIGS[cid]] if cid != 2 else [wl.CONFIGS[2].scaled(L=L, name="c2_L%d" % L)
+                                                             for L in (8, 16, 24, 32)]
+            for wv in variants:
+                n = 20 if cid == 5 else 200
+                mm, s2, i2 = time_workload(wv, device, n, 5)
+                tb = wv.logits_bytes
+                extras[wv.name] = {
+                    "steps_per_s": 1e3 / mm["ms_per_step"], "ms_per_step": mm["ms_per_step"],
+                    "stage_ms": {"lattice_build": mm["ms_lattice"], "cps_search": mm["ms_cps"],
+                                 "verify": mm["ms_verify"]},
+                    "logits_gbs": 2 * tb / ((mm["ms_lattice"] + mm["ms_verify"]) * 1e-3) / 1e9,
+                    "frac_of_8000": 2 * tb / ((mm["ms_lattice"] + mm["ms_verify"]) * 1e-3) / 1e9 / 8000.0,
+                    "input_sets": mm["sets"], "mean_accepted_len": mm["mean_accepted_len"]}
+                del s2, i2
+                torch.cuda.empty_cache()
+        line["workloads"] = extras
+    print(json.dumps(line))
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

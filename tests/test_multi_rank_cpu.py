@@ -1,0 +1,61 @@
+"""The benchmark's multi-rank plumbing on CPU: two gloo ranks, no GPU.
+
+Batch rows are independent, so ranks share nothing on the data path; what the ranks do
+exchange is the timing (maximum over ranks) and, in a sharded deployment, the per-row
+controller signals.  Both are exercised here with world_size 2.
+"""
+import os
+import sys
+
+import torch
+import torch.distributed as dist
+import torch.multiprocessing as mp
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def _worker(rank, world, port, out):
+    sys.path.insert(0, ROOT)
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port), RANK=str(rank), WORLD_SIZE=str(world))
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    import bench
+    import oracle
+    from paper_2510_02358_b200 import binding as dsp
+    from paper_2510_02358_b200 import workloads as wl
+    # timing: the job's time is the slowest rank's
+    ms = bench.reduce_max_ms(10.0 + 5.0 * rank, dist, torch.device("cpu"))
+    # each rank owns different batch rows of the same workload
+    w = wl.CONFIGS[3].scaled(B=2, L=3, V=512)
+    mine = wl.make_inputs(w, step=bench.rank_seed_base(rank))
+    lat = oracle.lattice_build(mine["draft"], w.K)
+    cps = oracle.cps_search(lat.cand_id, lat.cand_logit, lat.lse64, lat.cand_count, mine["prev_token"],
+                            mine["table"], W=w.W, lam=w.lam, table_log2=mine["table_log2"],
+                            hash_seed=mine["hash_seed"], V=w.V)
+    ver = oracle.verify(mine["target"], mine["draft"], cps.path, cps.path_len, mine["mode"], mine["u"])
+    # the controller needs the batch means over ALL rows: gather the two [B] int arrays
+    sig = torch.stack([ver.accepted_len, lat.gen_len]).int()
+    allsig = [torch.empty_like(sig) for _ in range(world)]
+    dist.all_gather(allsig, sig)
+    acc = torch.cat([s[0] for s in allsig])
+    gen = torch.cat([s[1] for s in allsig])
+    st, prm = dsp.dsp_adl_init(8, 32, 8.0, 0.5, 8)
+    k = dsp.dsp_adl_update(st, prm, acc, gen)
+    ks = [torch.zeros(1, dtype=torch.int32) for _ in range(world)]
+    dist.all_gather(ks, torch.tensor([k], dtype=torch.int32))
+    out[rank] = dict(ms=ms, k=[int(x) for x in ks], draft_sum=float(mine["draft"].float().sum()),
+                     value=bench.whole_job_steps_per_s(world, 20, ms))
+    dist.barrier()
+    dist.destroy_process_group()
+
+
+def test_two_ranks_gloo():
+    world = 2
+    port = 29500 + os.getpid() % 2000
+    mgr = mp.Manager()
+    out = mgr.dict()
+    mp.spawn(_worker, args=(world, port, out), nprocs=world, join=True)
+    r0, r1 = out[0], out[1]
+    assert r0["ms"] == r1["ms"] == 15.0                       # max over ranks
+    assert r0["value"] == r1["value"] == 2 * 20 / 0.015       # both ranks' steps over the slowest time
+    assert r0["k"] == r1["k"] and r0["k"][0] == r0["k"][1]    # every rank derives the same next length
+    assert r0["draft_sum"] != r1["draft_sum"]                 # different rows per rank
