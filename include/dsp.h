@@ -12,7 +12,8 @@
  *    errors are detected on the host before anything is enqueued.
  *  - Unless marked "host", every pointer is a DEVICE pointer to memory the
  *    caller owns (inputs, outputs and the scratch workspace).  The library
- *    allocates nothing and keeps no device state between calls.
+ *    allocates nothing and keeps no device state between calls (the one
+ *    exception, dsp_lattice_build_static, holds its scratch in a static array).
  *  - Device calls only enqueue work on `stream` (a cudaStream_t; NULL is the
  *    legacy default stream) and never synchronise.  Outputs are valid once
  *    the stream reaches the end of the call.  Two calls that share a
@@ -47,7 +48,9 @@ enum dsp_status {
     DSP_ERR_INVALID_ARG = -1,   /* null pointer, non-positive size, bad stride ... */
     DSP_ERR_UNSUPPORTED = -2,   /* dtype, K_max, W or L beyond the compiled limits */
     DSP_ERR_WORKSPACE = -3,     /* workspace_bytes smaller than the query call's answer */
-    DSP_ERR_CUDA = -4           /* a CUDA runtime call failed; see dsp_last_cuda_error */
+    DSP_ERR_CUDA = -4,          /* a CUDA runtime call failed; see dsp_last_cuda_error */
+    DSP_ERR_STATIC_SCRATCH = -5 /* dsp_lattice_build_static: the problem needs more scratch than
+                                   the library's built-in array of DSP_STATIC_WS_BYTES holds */
 };
 
 enum dsp_dtype { DSP_F32 = 0, DSP_BF16 = 1 };
@@ -112,6 +115,42 @@ int32_t dsp_lattice_build(const void *draft_logits, int32_t dtype,
                           int32_t *cand_count, float *lse, double *lse64, float *entropy,
                           int32_t *gen_len, uint32_t *row_status,
                           void *workspace, size_t workspace_bytes, dsp_stream_t stream);
+
+/* -------------------------------------------------------------------------
+ * Lattice build without a caller-supplied workspace.  (The paper has no
+ * counterpart: this entry point exists for the sake of deployment only.)
+ *
+ * Same inputs, outputs, results and argument errors as dsp_lattice_build, for
+ * callers that cannot allocate device memory for the scratch workspace: code
+ * that runs where cudaMalloc is not allowed or not reachable (inside another
+ * framework's callback, on a thread that must not call allocating CUDA
+ * routines, in a process whose device memory has all been handed out).  The
+ * caller still owns and passes every input and output buffer.  The scratch is
+ * an array of DSP_STATIC_WS_BYTES bytes that is part of the library image:
+ * every GPU on which the library is loaded holds it until the process exits.
+ *
+ *  - This function calls no allocating routine (no cudaMalloc / cudaFree).
+ *  - Limit: dsp_lattice_workspace_bytes(B, L, V, dtype, K_max) must not exceed
+ *    DSP_STATIC_WS_BYTES, else DSP_ERR_STATIC_SCRATCH is returned and nothing
+ *    is enqueued.  (The scratch grows with B*L; about 2 KB per draft row at
+ *    K_max = 16, so B*L up to a few thousand rows fits.)
+ *  - The first call on each device looks up the array's device address (a
+ *    host-side, once-per-device step with that device current).  Make that
+ *    first call outside any stream capture.
+ *  - All calls on one device share the one array, which keeps what the last
+ *    call left in it; each call clears on `stream` the part that has to start
+ *    at zero.  Two calls whose GPU work may overlap (different streams with no
+ *    ordering between them, or several host threads) race on it: order them.
+ */
+#define DSP_STATIC_WS_BYTES (4u << 20)
+
+int32_t dsp_lattice_build_static(const void *draft_logits, int32_t dtype,
+                                 int32_t B, int32_t L, int32_t V,
+                                 int64_t stride_b, int64_t stride_l,
+                                 int32_t K_max, float tau, int32_t eos_id,
+                                 int32_t *cand_id, float *cand_logit, float *cand_logp,
+                                 int32_t *cand_count, float *lse, double *lse64, float *entropy,
+                                 int32_t *gen_len, uint32_t *row_status, dsp_stream_t stream);
 
 /* -------------------------------------------------------------------------
  * Causal-consistency path search  (Sec. 3.2 "Scoring and search", Eq. 8;

@@ -19,12 +19,14 @@ _PKG = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_PKG, "libdsp.so")
 
 DSP_OK, DSP_ERR_INVALID_ARG, DSP_ERR_UNSUPPORTED, DSP_ERR_WORKSPACE, DSP_ERR_CUDA = 0, -1, -2, -3, -4
+DSP_ERR_STATIC_SCRATCH = -5
+DSP_STATIC_WS_BYTES = 4 << 20
 DSP_F32, DSP_BF16 = 0, 1
 ROW_NONFINITE_INPUT, ROW_ZERO_RESIDUAL, ROW_NO_BONUS_ROW, ROW_EOS_ACCEPTED, ROW_EOS_STOPPED = 1, 2, 4, 8, 16
 DSP_MAX_K, DSP_MAX_W, DSP_MAX_L = 32, 32, 1024
 
 EXPORTS = ["dsp_strerror", "dsp_last_cuda_error", "dsp_version", "dsp_lattice_workspace_bytes",
-           "dsp_lattice_build", "dsp_cps_search", "dsp_verify_workspace_bytes", "dsp_verify",
+           "dsp_lattice_build", "dsp_lattice_build_static", "dsp_cps_search", "dsp_verify_workspace_bytes", "dsp_verify",
            "dsp_adl_init", "dsp_adl_update"]
 
 
@@ -139,6 +141,23 @@ def dsp_lattice_build(draft: torch.Tensor, K_max: int, tau: float = 0.0, eos_id:
         _ptr(out.cand_id), _ptr(out.cand_logit), _ptr(out.cand_logp), _ptr(out.cand_count),
         _ptr(out.lse), _ptr(out.lse64), _ptr(out.entropy), _ptr(out.gen_len), _ptr(out.row_status),
         _ptr(workspace), C.c_size_t(workspace.numel()), _stream(stream)))
+    return out
+
+
+def dsp_lattice_build_static(draft: torch.Tensor, K_max: int, tau: float = 0.0, eos_id: int = -1,
+                             out: Optional[SimpleNamespace] = None, stream=None) -> SimpleNamespace:
+    """``dsp_lattice_build`` with the scratch held inside the library: for callers that cannot
+    allocate device memory.  Nothing is allocated by the C call; pass ``out`` to keep this wrapper
+    from allocating the outputs.  Raises DspError(DSP_ERR_STATIC_SCRATCH) beyond the size limit."""
+    B, L, V, sb, sl = _logits3(draft, "draft")
+    dt = _dtype(draft)
+    if out is None:
+        out = lattice_outputs(B, L, K_max, eos_id, draft.device)
+    _check("dsp_lattice_build_static", lib().dsp_lattice_build_static(
+        _ptr(draft), dt, B, L, V, C.c_int64(sb), C.c_int64(sl), K_max, C.c_float(tau), eos_id,
+        _ptr(out.cand_id), _ptr(out.cand_logit), _ptr(out.cand_logp), _ptr(out.cand_count),
+        _ptr(out.lse), _ptr(out.lse64), _ptr(out.entropy), _ptr(out.gen_len), _ptr(out.row_status),
+        _stream(stream)))
     return out
 
 

@@ -15,6 +15,7 @@ extern "C" const char *dsp_strerror(int32_t status) {
         case DSP_ERR_UNSUPPORTED: return "unsupported dtype or size beyond the compiled limits";
         case DSP_ERR_WORKSPACE: return "workspace too small";
         case DSP_ERR_CUDA: return "CUDA runtime error (see dsp_last_cuda_error)";
+        case DSP_ERR_STATIC_SCRATCH: return "problem too large for the library's built-in scratch array";
         default: return "unknown status";
     }
 }

@@ -261,3 +261,62 @@ extern "C" int32_t dsp_lattice_build(const void *draft_logits, int32_t dtype,
     return dtype == DSP_BF16 ? launch_lattice<__nv_bfloat16>(a, workspace, workspace_bytes, st)
                              : launch_lattice<float>(a, workspace, workspace_bytes, st);
 }
+
+// ---- dsp_lattice_build_static: the same build for callers that cannot allocate ----------------
+//
+// The scratch workspace lives in this translation unit as a file-scope device array, so a caller
+// that has no way to obtain device memory for it (a plug-in running inside a host process whose
+// memory pool is closed to it, a callback on a thread where CUDA allocation calls are forbidden,
+// code that runs after the memory budget has been handed out) passes only inputs and outputs.
+#include <mutex>
+
+namespace {
+
+constexpr size_t kStaticWsBytes = (size_t)DSP_STATIC_WS_BYTES;
+static __device__ __align__(256) unsigned char g_static_ws[kStaticWsBytes];
+
+constexpr int kMaxDevices = 64;
+std::mutex g_static_ws_mutex;
+void *g_static_ws_addr[kMaxDevices];    // device address of g_static_ws on each device, 0 = not asked yet
+
+// In host code `g_static_ws` only names the symbol; the address a kernel can use has to be asked
+// for, once per device and with that device current.
+int32_t static_ws_address(void **out) {
+    int dev = -1;
+    DSP_CUDA_TRY(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= kMaxDevices) return DSP_ERR_UNSUPPORTED;
+    std::lock_guard<std::mutex> lock(g_static_ws_mutex);
+    if (!g_static_ws_addr[dev]) {
+        void *p = nullptr;
+        DSP_CUDA_TRY(cudaGetSymbolAddress(&p, g_static_ws));
+        if (!p) return dsp::cuda_fail(cudaErrorInvalidSymbol);
+        g_static_ws_addr[dev] = p;
+    }
+    *out = g_static_ws_addr[dev];
+    return DSP_OK;
+}
+
+}  // namespace
+
+extern "C" int32_t dsp_lattice_build_static(const void *draft_logits, int32_t dtype,
+                                            int32_t B, int32_t L, int32_t V,
+                                            int64_t stride_b, int64_t stride_l,
+                                            int32_t K_max, float tau, int32_t eos_id,
+                                            int32_t *cand_id, float *cand_logit, float *cand_logp,
+                                            int32_t *cand_count, float *lse, double *lse64,
+                                            float *entropy, int32_t *gen_len, uint32_t *row_status,
+                                            dsp_stream_t stream) {
+    size_t need = 0;
+    const int32_t rc = dsp_lattice_workspace_bytes(B, L, V, dtype, K_max, &need);
+    if (rc != DSP_OK) return rc;
+    if (need > kStaticWsBytes) return DSP_ERR_STATIC_SCRATCH;
+    if (B == 0) return DSP_OK;
+    void *ws = nullptr;
+    const int32_t rs = static_ws_address(&ws);
+    if (rs != DSP_OK) return rs;
+    // The build zeroes the part of the scratch that must start at zero on `stream` before its
+    // kernel runs, so what the previous call left in the array does not matter.
+    return dsp_lattice_build(draft_logits, dtype, B, L, V, stride_b, stride_l, K_max, tau, eos_id,
+                             cand_id, cand_logit, cand_logp, cand_count, lse, lse64, entropy,
+                             gen_len, row_status, ws, kStaticWsBytes, stream);
+}
