@@ -61,6 +61,8 @@ enum dsp_dtype { DSP_F32 = 0, DSP_BF16 = 1 };
 #define DSP_ROW_NO_BONUS_ROW    4u  /* whole path accepted and no target row path_len exists */
 #define DSP_ROW_EOS_ACCEPTED    8u  /* an accepted token is EOS: the caller terminates decoding */
 #define DSP_ROW_EOS_STOPPED     16u /* the path search stopped early at an EOS */
+#define DSP_ROW_TIMEOUT         32u /* a bounded wait inside a kernel ran out (hardware fault or a
+                                       defect of this library): the row's outputs are unspecified */
 
 #define DSP_MAX_K 32      /* largest K_max (per-position candidate cap M_max) */
 #define DSP_MAX_W 32      /* largest beam width */

@@ -23,6 +23,7 @@ DSP_ERR_STATIC_SCRATCH = -5
 DSP_STATIC_WS_BYTES = 4 << 20
 DSP_F32, DSP_BF16 = 0, 1
 ROW_NONFINITE_INPUT, ROW_ZERO_RESIDUAL, ROW_NO_BONUS_ROW, ROW_EOS_ACCEPTED, ROW_EOS_STOPPED = 1, 2, 4, 8, 16
+ROW_TIMEOUT = 32
 DSP_MAX_K, DSP_MAX_W, DSP_MAX_L = 32, 32, 1024
 
 EXPORTS = ["dsp_strerror", "dsp_last_cuda_error", "dsp_version", "dsp_lattice_workspace_bytes",

@@ -4,7 +4,7 @@
 // once from HBM (log-sum-exp terms + exact top-K, see scan_core.cuh).  A row split over
 // several CTAs is finished by whichever CTA arrives last (atomic ticket): no CTA waits.
 // The CTA that finishes the last row of a batch row also writes gen_len and row_status.
-#include "scan_core.cuh"
+#include "stream_core.cuh"
 
 namespace dsp {
 
@@ -49,21 +49,15 @@ static LatticeWs lattice_ws_layout(int64_t B, int64_t L, int nslices, int K) {
     return w;
 }
 
-template <typename DT>
-__global__ void __launch_bounds__(kThreads, 4) lattice_kernel(const LatticeArgs a) {
-    __shared__ ScanSmem sm;
+// Everything after the scan of one slice: publish the slice's partial result, let the CTA that
+// arrives last merge the row, finalise the row (Eq. 7 count, EOS slot, outputs) and, for the
+// last row of a batch row, write gen_len and row_status.  `extra_status` is OR-ed into the
+// batch row's status.
+template <typename DT, typename SY>
+__device__ void lattice_finish(const LatticeArgs &a, ScanSmem &sm, long long row, int slice, int b,
+                               const DT *rowp, float c, double S, double T, unsigned extra_status) {
     const int tid = threadIdx.x;
-    const long long row = blockIdx.x / a.nslices;
-    const int slice = blockIdx.x - (int)(row * a.nslices);
-    const int b = (int)(row / a.L), l = (int)(row - (long long)b * a.L);
-    const DT *rowp = reinterpret_cast<const DT *>(a.logits) + b * a.stride_b + l * a.stride_l;
-    const int s0 = slice * a.slice_elems;
-    const int s1 = min(a.V, s0 + a.slice_elems);
-
-    float c;
-    double S, T;
-    scan_slice<DT, true>(rowp, s0, s1, a.K, sm, c, S, T);
-
+    if (extra_status && tid == 0) atomicOr(&a.b_status[b], extra_status);
     if (a.nslices > 1) {
         SlicePartial *part = a.partials + row * a.nslices;
         unsigned long long *keys = a.keys + (row * a.nslices + slice) * a.K;
@@ -73,14 +67,14 @@ __global__ void __launch_bounds__(kThreads, 4) lattice_kernel(const LatticeArgs 
             part[slice].S = S; part[slice].T = T; part[slice].c = c; part[slice].nkeys = nk;
         }
         __threadfence();
-        __syncthreads();
+        SY::sync();
         if (tid == 0) sm.flag = (int)atomicAdd(&a.row_ticket[row], 1u);
-        __syncthreads();
+        SY::sync();
         if (sm.flag != a.nslices - 1) return;
         __threadfence();
         // last CTA of this row: gather every slice's keys and sums
         if (tid == 0) sm.cnt = 0;
-        __syncthreads();
+        SY::sync();
         for (int s = 0; s < a.nslices; ++s) {
             const int n = __ldcg(&part[s].nkeys);
             const unsigned long long *ks = a.keys + (row * a.nslices + s) * a.K;
@@ -88,7 +82,7 @@ __global__ void __launch_bounds__(kThreads, 4) lattice_kernel(const LatticeArgs 
             else if (tid < a.K) sm.cand[s * a.K + tid] = 0ull;     // below every real key
         }
         if (tid == 0) sm.cnt = a.nslices * a.K;
-        prune(sm, a.K);
+        prune<SY>(sm, a.K);
         if (tid == 0) {
             int n = 0;                                  // drop the padding keys again
             while (n < sm.cnt && sm.cand[n] != 0ull) ++n;
@@ -96,16 +90,16 @@ __global__ void __launch_bounds__(kThreads, 4) lattice_kernel(const LatticeArgs 
             merge_partials(part, a.nslices, c, S, T);
             sm.fin[0] = S; sm.fin[1] = T; sm.redc[0] = c;
         }
-        __syncthreads();
+        SY::sync();
         S = sm.fin[0]; T = sm.fin[1]; c = sm.redc[0];
     }
 
     // ---- finalise the row: sm.cand[0..cnt) sorted best keys, (c,S,T) whole-row sums ----
     const int nk = sm.cnt;
     double lse, mean_x;
-    const bool ok = row_log_stats(c, S, T, lse, mean_x);
+    const bool ok = row_log_stats(c, S, T, lse, mean_x) && nk > 0;
     if (tid < nk) sm.pk[tid] = exp((double)key_value(sm.cand[tid]) - lse);
-    __syncthreads();
+    SY::sync();
     if (tid == 0) {
         int count = nk;
         if (a.tau > 0.f && a.tau <= 1.f && ok) {       // Eq. 7 on full-vocabulary probabilities
@@ -135,7 +129,7 @@ __global__ void __launch_bounds__(kThreads, 4) lattice_kernel(const LatticeArgs 
         if (a.entropy) a.entropy[row] = (float)(lse - mean_x);
         if (!ok) atomicOr(&a.b_status[b], DSP_ROW_NONFINITE_INPUT);
     }
-    __syncthreads();
+    SY::sync();
     if (tid < a.KC) {
         const int count = sm.flag, eos_slot = sm.overflow;
         int id = -1;
@@ -156,7 +150,7 @@ __global__ void __launch_bounds__(kThreads, 4) lattice_kernel(const LatticeArgs 
     }
     // ---- last row of this batch row: generation length (Eq. 9) and status ----
     __threadfence();
-    __syncthreads();
+    SY::sync();
     if (tid == 0) {
         const unsigned t = atomicAdd(&a.b_ticket[b], 1u);
         if (t == (unsigned)a.L - 1) {
@@ -171,6 +165,53 @@ __global__ void __launch_bounds__(kThreads, 4) lattice_kernel(const LatticeArgs 
             a.row_status[b] = atomicOr(&a.b_status[b], 0u);
         }
     }
+}
+
+
+// Element-wise kernel: any layout (rows need not be 16-byte aligned).
+template <typename DT>
+__global__ void __launch_bounds__(kThreads, 4) lattice_kernel(const LatticeArgs a) {
+    __shared__ ScanSmem sm;
+    const long long row = blockIdx.x / a.nslices;
+    const int slice = blockIdx.x - (int)(row * a.nslices);
+    const int b = (int)(row / a.L), l = (int)(row - (long long)b * a.L);
+    const DT *rowp = reinterpret_cast<const DT *>(a.logits) + b * a.stride_b + l * a.stride_l;
+    const int s0 = slice * a.slice_elems;
+    const int s1 = min(a.V, s0 + a.slice_elems);
+    float c;
+    double S, T;
+    scan_slice<DT, true>(rowp, s0, s1, a.K, sm, c, S, T);
+    lattice_finish<DT, SyncAll>(a, sm, row, slice, b, rowp, c, S, T, 0u);
+}
+
+// Streaming kernel for 16-byte aligned layouts: a service warp feeds the slice through a
+// shared-memory ring with bulk asynchronous copies and keeps the running top-K; the consumers
+// scan the ring (see stream_core.cuh).
+template <typename DT>
+__global__ void __launch_bounds__(kStreamThreads, 3) lattice_stream_kernel(const LatticeArgs a) {
+    extern __shared__ __align__(128) unsigned char ring[];
+    __shared__ ScanSmem sm;
+    __shared__ StreamBars bars;
+    __shared__ StreamCtl ctl;
+    const int tid = threadIdx.x;
+    const long long row = blockIdx.x / a.nslices;
+    const int slice = blockIdx.x - (int)(row * a.nslices);
+    const int b = (int)(row / a.L), l = (int)(row - (long long)b * a.L);
+    const DT *rowp = reinterpret_cast<const DT *>(a.logits) + b * a.stride_b + l * a.stride_l;
+    const int s0 = slice * a.slice_elems;
+    const int s1 = min(a.V, s0 + a.slice_elems);
+    stream_begin(sm, ctl, bars);
+    if (tid >= kThreads) {                                  // service warp: copies + running top-K
+        stream_service(reinterpret_cast<const char *>(rowp + s0), (s1 - s0) * (int)sizeof(DT), a.K, sm,
+                       ctl, ring, bars);
+        stream_sync_all();
+        return;
+    }
+    float c;
+    double S, T;
+    scan_slice_stream<DT, true>(rowp, s0, s1, a.K, sm, ctl, ring, bars, c, S, T);
+    lattice_finish<DT, SyncConsumers>(a, sm, row, slice, b, rowp, c, S, T,
+                                      ctl.timed_out ? DSP_ROW_TIMEOUT : 0u);
 }
 
 template <typename DT>
@@ -190,7 +231,13 @@ static int32_t launch_lattice(LatticeArgs &a, void *workspace, size_t workspace_
     DSP_CUDA_TRY(cudaMemsetAsync(ws, 0, w.zero_bytes, st));
     const long long nblocks = nrows * a.nslices;
     if (nblocks > 0x7FFFFFFFLL) return DSP_ERR_UNSUPPORTED;
-    lattice_kernel<DT><<<(unsigned)nblocks, kThreads, 0, st>>>(a);
+    if (stream_layout_ok(a.logits, sizeof(DT), a.V, a.stride_b, a.stride_l)) {
+        static RingSmemDone smem_done;                       // one per element type
+        DSP_CUDA_TRY(allow_ring_smem(lattice_stream_kernel<DT>, smem_done));
+        lattice_stream_kernel<DT><<<(unsigned)nblocks, kStreamThreads, kRingBytes, st>>>(a);
+    } else {
+        lattice_kernel<DT><<<(unsigned)nblocks, kThreads, 0, st>>>(a);
+    }
     DSP_CUDA_TRY(cudaGetLastError());
     return DSP_OK;
 }

@@ -22,6 +22,15 @@ struct ScanSmem {
     int flag;
 };
 
+// Block-wide barrier policies: every thread of the CTA, or only the kThreads consumer threads
+// of a kernel that also runs a service warp (named barrier 1).
+struct SyncAll {
+    static __device__ __forceinline__ void sync() { __syncthreads(); }
+};
+struct SyncConsumers {
+    static __device__ __forceinline__ void sync() { asm volatile("bar.sync 1, %0;" ::"n"(kThreads) : "memory"); }
+};
+
 template <typename DT>
 __device__ __forceinline__ uint4 load_vec(const DT *__restrict__ row, int e0, int end, bool aligned) {
     constexpr int N = Elem<DT>::N;
@@ -53,8 +62,9 @@ __device__ __forceinline__ uint4 load_vec(const DT *__restrict__ row, int e0, in
 
 // Keep the best min(K, n) of the n = min(cnt, cap) buffered keys, sorted, at the front of
 // cand; refresh the thresholds.  Every key is unique, so ranks are unique.  Block-wide.
+template <typename SY = SyncAll>
 __device__ __forceinline__ void prune(ScanSmem &sm, int K) {
-    __syncthreads();
+    SY::sync();
     const int tid = threadIdx.x;
     const int n = min(sm.cnt, kCandCap);
     if (tid == 0 && sm.cnt > kCandCap) sm.overflow = 1;
@@ -64,7 +74,7 @@ __device__ __forceinline__ void prune(ScanSmem &sm, int K) {
         for (int j = 0; j < n; ++j) rank += sm.cand[j] > key;
         if (rank < K) sm.sel[rank] = key;
     }
-    __syncthreads();
+    SY::sync();
     const int nk = min(n, K);
     if (tid < nk) sm.cand[tid] = sm.sel[tid];
     if (tid == 0) {
@@ -74,7 +84,7 @@ __device__ __forceinline__ void prune(ScanSmem &sm, int K) {
             sm.thr_v = key_value(sm.sel[K - 1]);
         }
     }
-    __syncthreads();
+    SY::sync();
 }
 
 __device__ __forceinline__ float bitonic_desc(float v, int lane) {
@@ -94,11 +104,12 @@ __device__ __forceinline__ float bitonic_desc(float v, int lane) {
 // First threshold of a slice from the 256 thread maxima of its first tile: the smallest r
 // such that r * (#warps whose r-th largest thread maximum is finite) >= K gives K distinct
 // elements >= min over those warps of that r-th largest.  -inf if there is no such r.
+template <typename SY = SyncAll>
 __device__ __forceinline__ void bootstrap_threshold(ScanSmem &sm, float tm, int K) {
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const float s = bitonic_desc(tm == tm ? tm : -CUDART_INF_F, lane);
     sm.wsorted[warp][lane] = s;
-    __syncthreads();
+    SY::sync();
     if (tid == 0) {
         float t = -CUDART_INF_F;
         for (int r = 1; r <= 32; ++r) {
@@ -113,18 +124,18 @@ __device__ __forceinline__ void bootstrap_threshold(ScanSmem &sm, float tm, int 
         }
         sm.thr_v = t;
     }
-    __syncthreads();
+    SY::sync();
 }
 
 // Exact top-K of a slice when the fast path overflowed its buffer (heavily tied or
 // adversarially ordered rows): one element per thread per round, exact key test, prune
 // whenever another round could overflow.  Slow, bounded, always correct.
-template <typename DT>
+template <typename DT, typename SY = SyncAll>
 __device__ void topk_careful(const DT *__restrict__ row, int s0, int s1, int K, ScanSmem &sm) {
     const int tid = threadIdx.x;
-    __syncthreads();
+    SY::sync();
     if (tid == 0) { sm.cnt = 0; sm.thrkey = 0ull; sm.thr_v = -CUDART_INF_F; sm.overflow = 0; }
-    __syncthreads();
+    SY::sync();
     for (int base = s0; base < s1; base += kThreads) {
         const int idx = base + tid;
         if (idx < s1) {
@@ -137,12 +148,71 @@ __device__ void topk_careful(const DT *__restrict__ row, int s0, int s1, int K, 
                 }
             }
         }
-        __syncthreads();
+        SY::sync();
         const int n = sm.cnt;          // read between two barriers: the same value in every thread
-        __syncthreads();
-        if (n > kCandCap - kThreads) prune(sm, K);
+        SY::sync();
+        if (n > kCandCap - kThreads) prune<SY>(sm, K);
     }
-    prune(sm, K);
+    prune<SY>(sm, K);
+}
+
+// Block reduction of the per-thread sums (c, S, T) of a slice to one reference exponent, in
+// double.  If masked (-inf) logits poisoned T only (0 * -inf), the slice's sums are redone from
+// global memory against the now known reference with the exponent clamped.
+template <typename DT, typename SY>
+__device__ void reduce_sums(const DT *__restrict__ row, int s0, int s1, ScanSmem &sm, float c, float S,
+                            float T, float &c_out, double &S_out, double &T_out) {
+    constexpr int N = Elem<DT>::N;
+    constexpr int TE = tile_elems<DT>();
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const bool aligned = (reinterpret_cast<uintptr_t>(row) & 15) == 0;
+    const int ntiles = (s1 - s0 + TE - 1) / TE;
+    float cb = warp_max(c);
+    if (lane == 0) sm.redc[warp] = cb;
+    SY::sync();
+    cb = sm.redc[0];
+#pragma unroll
+    for (int w = 1; w < kWarps; ++w) cb = fmaxf(cb, sm.redc[w]);
+    const float d = c - cb;
+    const float a = ex2_approx(d);
+    double Sd = warp_sum((double)(S * a));
+    double Td = warp_sum((double)((T + S * d) * a));
+    if (lane == 0) { sm.redS[warp] = Sd; sm.redT[warp] = Td; }
+    SY::sync();
+    Sd = 0.0; Td = 0.0;
+#pragma unroll
+    for (int w = 0; w < kWarps; ++w) { Sd += sm.redS[w]; Td += sm.redT[w]; }
+    SY::sync();
+
+    if (Td != Td && Sd == Sd && Sd < CUDART_INF) {
+        // 0 * -inf from masked (-inf) logits poisoned T only: redo the sums of this
+        // slice against the now known reference with the exponent clamped.
+        const float nc = -cb;
+        float S2 = 0.f, T2 = 0.f;
+        for (int t = 0; t < ntiles; ++t) {
+            const int base = s0 + t * TE;
+#pragma unroll
+            for (int j = 0; j < kVpt; ++j) {
+                const uint4 vv = load_vec<DT>(row, base + (j * kThreads + tid) * N, s1, aligned);
+#pragma unroll
+                for (int e = 0; e < N; ++e) {
+                    const float x = Elem<DT>::get(vv, e);
+                    const float a2 = fmaxf(fmaf(x, kLog2e, nc), -1000.f);
+                    const float ex = ex2_approx(a2);
+                    S2 += ex;
+                    T2 = fmaf(ex, a2, T2);
+                }
+            }
+        }
+        double S2d = warp_sum((double)S2), T2d = warp_sum((double)T2);
+        if (lane == 0) { sm.redS[warp] = S2d; sm.redT[warp] = T2d; }
+        SY::sync();
+        Sd = 0.0; Td = 0.0;
+#pragma unroll
+        for (int w = 0; w < kWarps; ++w) { Sd += sm.redS[w]; Td += sm.redT[w]; }
+        SY::sync();
+    }
+    c_out = cb; S_out = Sd; T_out = Td;
 }
 
 // Scan [s0, s1) of `row`.  On return (after a block barrier) sm.cand[0 .. sm.cnt) holds the
@@ -233,53 +303,7 @@ __device__ void scan_slice(const DT *__restrict__ row, int s0, int s1, int K, Sc
     if (sm.overflow) topk_careful<DT>(row, s0, s1, K, sm);
 
     if constexpr (SUMS) {
-        // block reduction to one reference exponent
-        float cb = warp_max(c);
-        if (lane == 0) sm.redc[warp] = cb;
-        __syncthreads();
-        cb = sm.redc[0];
-#pragma unroll
-        for (int w = 1; w < kWarps; ++w) cb = fmaxf(cb, sm.redc[w]);
-        const float d = c - cb;
-        const float a = ex2_approx(d);
-        double Sd = warp_sum((double)(S * a));
-        double Td = warp_sum((double)((T + S * d) * a));
-        if (lane == 0) { sm.redS[warp] = Sd; sm.redT[warp] = Td; }
-        __syncthreads();
-        Sd = 0.0; Td = 0.0;
-#pragma unroll
-        for (int w = 0; w < kWarps; ++w) { Sd += sm.redS[w]; Td += sm.redT[w]; }
-        __syncthreads();
-
-        if (Td != Td && Sd == Sd && Sd < CUDART_INF) {
-            // 0 * -inf from masked (-inf) logits poisoned T only: redo the sums of this
-            // slice against the now known reference with the exponent clamped.
-            const float nc = -cb;
-            float S2 = 0.f, T2 = 0.f;
-            for (int t = 0; t < ntiles; ++t) {
-                const int base = s0 + t * TE;
-#pragma unroll
-                for (int j = 0; j < kVpt; ++j) {
-                    const uint4 vv = load_vec<DT>(row, base + (j * kThreads + tid) * N, s1, aligned);
-#pragma unroll
-                    for (int e = 0; e < N; ++e) {
-                        const float x = Elem<DT>::get(vv, e);
-                        const float a2 = fmaxf(fmaf(x, kLog2e, nc), -1000.f);
-                        const float ex = ex2_approx(a2);
-                        S2 += ex;
-                        T2 = fmaf(ex, a2, T2);
-                    }
-                }
-            }
-            double S2d = warp_sum((double)S2), T2d = warp_sum((double)T2);
-            if (lane == 0) { sm.redS[warp] = S2d; sm.redT[warp] = T2d; }
-            __syncthreads();
-            Sd = 0.0; Td = 0.0;
-#pragma unroll
-            for (int w = 0; w < kWarps; ++w) { Sd += sm.redS[w]; Td += sm.redT[w]; }
-            __syncthreads();
-        }
-        c_out = cb; S_out = Sd; T_out = Td;
+        reduce_sums<DT, SyncAll>(row, s0, s1, sm, c, S, T, c_out, S_out, T_out);
     } else {
         c_out = kRefFloor; S_out = 0.0; T_out = 0.0;
     }

@@ -1,0 +1,360 @@
+// TMA-fed variant of the one-pass slice scan for rows whose start, strides and length are
+// multiples of 16 bytes.  A service warp streams the slice through a ring of shared-memory
+// stages with bulk asynchronous copies (cp.async.bulk, completion counted on an mbarrier per
+// stage, no multicast); the kThreads consumer threads read each stage with one 128-bit shared
+// load per vector, release it at once and do the arithmetic from registers.  Logits at or
+// above the current threshold are appended to a candidate list; the service warp turns that
+// list into the running top-K and a tighter threshold while the consumers keep streaming, so
+// the scan has no block-wide barrier except the first tile's threshold bootstrap.  Results are
+// the same as scan_slice's (scan_core.cuh): log-sum-exp terms and the exact top-K.
+#pragma once
+
+#include "scan_core.cuh"
+
+namespace dsp {
+
+constexpr int kTileBytes = kThreads * kVpt * 16;     // one ring stage = one tile of either dtype
+constexpr int kStages = 4;
+constexpr int kStreamThreads = kThreads + 32;        // consumers + the service warp
+constexpr int kRingBytes = kStages * kTileBytes;
+constexpr int kWaitTries = 1 << 22;                  // bound of every mbarrier wait and spin
+constexpr int kIdleLimit = 1 << 22;                  // idle polls of the service warp before it gives up
+
+__device__ __forceinline__ uint32_t smem_addr(const void *p) {
+    return (uint32_t)__cvta_generic_to_shared(p);
+}
+__device__ __forceinline__ void mbar_init(uint64_t *bar, int count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_addr(bar)), "r"(count));
+}
+__device__ __forceinline__ void mbar_init_fence() {
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint64_t *bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_addr(bar)), "r"(bytes)
+                 : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint64_t *bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_addr(bar)) : "memory");
+}
+// Bounded wait for the phase with the given parity; false if it never completed.
+__device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity) {
+    const uint32_t a = smem_addr(bar);
+    for (int i = 0; i < kWaitTries; ++i) {
+        uint32_t ok;
+        asm volatile(
+            "{\n"
+            ".reg .pred p;\n"
+            "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n"
+            "selp.u32 %0, 1, 0, p;\n"
+            "}"
+            : "=r"(ok)
+            : "r"(a), "r"(parity)
+            : "memory");
+        if (ok) return true;
+    }
+    return false;
+}
+// Non-blocking test of a phase.
+__device__ __forceinline__ bool mbar_test(uint64_t *bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n"
+        ".reg .pred p;\n"
+        "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n"
+        "selp.u32 %0, 1, 0, p;\n"
+        "}"
+        : "=r"(ok)
+        : "r"(smem_addr(bar)), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+// Bulk copy global -> this CTA's shared memory; both addresses and the size are multiples of 16.
+__device__ __forceinline__ void bulk_load(void *dst, const void *src, uint32_t bytes, uint64_t *bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(smem_addr(dst)), "l"(src), "r"(bytes), "r"(smem_addr(bar))
+                 : "memory");
+}
+__device__ __forceinline__ float max3(float a, float b, float c) {
+    float d;
+    asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+    return d;
+}
+
+struct StreamBars {
+    uint64_t full[kStages];
+    uint64_t empty[kStages];
+};
+
+// Shared state between the consumers and the service warp of one slice scan.
+struct StreamCtl {
+    int done_warps;      // consumer warps that have finished their last tile
+    int nsel;            // number of keys the service warp left in ScanSmem::sel
+    int timed_out;       // a bounded wait ran out
+};
+
+// Barrier of all kStreamThreads threads of the CTA (named barrier 2).
+__device__ __forceinline__ void stream_sync_all() {
+    asm volatile("bar.sync 2, %0;" ::"n"(kStreamThreads) : "memory");
+}
+
+// Called by every thread before service/consume start (ends with a CTA-wide barrier).
+__device__ __forceinline__ void stream_begin(ScanSmem &sm, StreamCtl &ctl, StreamBars &bars) {
+    const int tid = threadIdx.x;
+    if (tid == 0) {
+        for (int s = 0; s < kStages; ++s) {
+            mbar_init(&bars.full[s], 1);
+            mbar_init(&bars.empty[s], kWarps);
+        }
+        mbar_init_fence();
+        sm.cnt = 0; sm.thrkey = 0ull; sm.thr_v = -CUDART_INF_F; sm.overflow = 0;
+        ctl.done_warps = 0; ctl.nsel = 0; ctl.timed_out = 0;
+    }
+    for (int i = tid; i < kCandCap; i += kStreamThreads) sm.cand[i] = 0ull;   // 0 = not written yet
+    __syncthreads();
+}
+
+// The service warp of a slice scan (32 threads, all of them call this).  Two duties:
+//  - lane 0 streams bytes [0, nbytes) at `src` through the ring, one bulk copy per free stage;
+//  - the warp keeps the best 32 keys seen so far, one per lane, sorted descending.  It reads the
+//    candidate keys that the consumers append to sm.cand (an append-only list during the scan),
+//    inserts those that beat its K-th key, and publishes the K-th key's value as the new
+//    threshold sm.thr_v.  The consumers never stop for this: they pick the threshold up at
+//    their next tile.  The K-th best of any subset of the slice is a valid lower bound.
+// On return (all tiles issued, all consumer warps done, every appended key processed) the best
+// min(K, #keys) keys are in sm.sel[0 .. ctl.nsel), sorted.
+__device__ __forceinline__ void stream_service(const char *src, int nbytes, int K, ScanSmem &sm,
+                                               StreamCtl &ctl, unsigned char *ring, StreamBars &bars) {
+    const int lane = threadIdx.x & 31;
+    const int ntiles = (nbytes + kTileBytes - 1) / kTileBytes;
+    int t_next = 0;                                   // lane 0: next tile to issue
+    unsigned long long mykey = 0ull;                  // 0 = empty slot (below every real key)
+    unsigned long long kth = 0ull;                    // key of rank K-1, 0 while fewer than K are held
+    float thr_pub = -CUDART_INF_F;
+    int processed = 0, idle = 0;
+    volatile int *v_cnt = &sm.cnt;
+    volatile int *v_done = &ctl.done_warps;
+    volatile unsigned long long *v_cand = sm.cand;
+    for (;;) {
+        if (lane == 0) {
+            while (t_next < ntiles) {
+                const int s = t_next % kStages;
+                if (t_next >= kStages && !mbar_test(&bars.empty[s], ((t_next / kStages) - 1) & 1)) break;
+                const uint32_t bytes = (uint32_t)min(kTileBytes, nbytes - t_next * kTileBytes);
+                mbar_expect_tx(&bars.full[s], bytes);
+                bulk_load(ring + (size_t)s * kTileBytes, src + (size_t)t_next * kTileBytes, bytes,
+                          &bars.full[s]);
+                ++t_next;
+            }
+        }
+        const bool all_issued = __shfl_sync(0xFFFFFFFFu, (int)(t_next >= ntiles), 0) != 0;
+        const int done_w = *v_done;                   // read before the count: once every warp is
+        __threadfence_block();                        // done, the count that follows is final
+        const int cnt = min(*v_cnt, kCandCap);
+        if (processed < cnt) {
+            idle = 0;
+            const int i = processed + lane;
+            unsigned long long key = 0ull;
+            if (i < cnt) {                            // a slot is claimed before it is written
+                for (int spin = 0; spin < kWaitTries; ++spin) {
+                    key = v_cand[i];
+                    if (key != 0ull) break;
+                }
+            }
+            unsigned pending = __ballot_sync(0xFFFFFFFFu, key > kth);
+            while (pending) {
+                const int from = __ffs(pending) - 1;
+                pending &= pending - 1;
+                const unsigned long long nk = __shfl_sync(0xFFFFFFFFu, key, from);
+                const int p = __popc(__ballot_sync(0xFFFFFFFFu, mykey > nk));   // keys ahead of nk
+                const unsigned long long up = __shfl_up_sync(0xFFFFFFFFu, mykey, 1);
+                if (lane == p) mykey = nk;
+                else if (lane > p) mykey = up;
+            }
+            processed = min(cnt, processed + 32);
+            kth = __shfl_sync(0xFFFFFFFFu, mykey, K - 1);
+            if (lane == 0 && kth != 0ull) {
+                const float v = key_value(kth);
+                if (v > thr_pub) {
+                    thr_pub = v;
+                    *reinterpret_cast<volatile float *>(&sm.thr_v) = v;
+                }
+            }
+        } else if (all_issued && done_w == kWarps) {
+            break;
+        } else {
+            if (++idle > kIdleLimit) {
+                if (lane == 0) ctl.timed_out = 1;
+                break;
+            }
+            __nanosleep(100);
+        }
+    }
+    const unsigned have = __ballot_sync(0xFFFFFFFFu, mykey != 0ull && lane < K);
+    if (lane < DSP_MAX_K) sm.sel[lane] = mykey;
+    if (lane == 0) ctl.nsel = __popc(have);
+}
+
+// Padding for the vectors past the end of a ragged last tile: -2^124, below every finite
+// logit the interface allows, finite when scaled by log2(e), never a candidate (its index is
+// past the row).
+template <typename DT> struct Pad;
+template <> struct Pad<__nv_bfloat16> { static constexpr uint32_t kWord = 0xFD80FD80u; };
+template <> struct Pad<float> { static constexpr uint32_t kWord = 0xFD800000u; };
+
+// Consumer side of the scan of [s0, s1) of `row` (kThreads threads, barriers via SyncConsumers;
+// the service warp runs stream_service meanwhile and both sides meet in stream_sync_all).
+// Same contract as scan_slice.
+template <typename DT, bool SUMS>
+__device__ void scan_slice_stream(const DT *__restrict__ row, int s0, int s1, int K, ScanSmem &sm,
+                                  StreamCtl &ctl, const unsigned char *ring, StreamBars &bars,
+                                  float &c_out, double &S_out, double &T_out) {
+    using SY = SyncConsumers;
+    constexpr int N = Elem<DT>::N;
+    constexpr int TE = tile_elems<DT>();
+    constexpr int VT = kTileBytes / 16;
+    static_assert(VT == kThreads * kVpt && TE * (int)sizeof(DT) == kTileBytes, "tile geometry");
+    const int tid = threadIdx.x, lane = tid & 31;
+    const int nbytes = (s1 - s0) * (int)sizeof(DT);
+    const int ntiles = (nbytes + kTileBytes - 1) / kTileBytes;
+
+    float c = kRefFloor, S = 0.f, T = 0.f;
+    float thr = -CUDART_INF_F;
+    bool timed_out = false;
+
+    // the reference exponent must bound every logit below the threshold (those skip the test)
+    auto raise_ref = [&](float ts) {
+        if (ts > c) {
+            const float d = c - ts;
+            const float sc = ex2_approx(d);
+            T = (T + S * d) * sc;
+            S = S * sc;
+            c = ts;
+        }
+    };
+
+    for (int t = 0; t < ntiles; ++t) {
+        const int s = t % kStages;
+        if (!mbar_wait(&bars.full[s], (t / kStages) & 1)) timed_out = true;
+        const int nvec = min(kTileBytes, nbytes - t * kTileBytes) >> 4;
+        const uint4 *sp = reinterpret_cast<const uint4 *>(ring + (size_t)s * kTileBytes);
+        uint4 v[kVpt];
+        if (nvec == VT) {
+#pragma unroll
+            for (int j = 0; j < kVpt; ++j) v[j] = sp[j * kThreads + tid];
+        } else {
+            const uint32_t pw = Pad<DT>::kWord;
+#pragma unroll
+            for (int j = 0; j < kVpt; ++j) {
+                const int vi = j * kThreads + tid;
+                v[j] = vi < nvec ? sp[vi] : make_uint4(pw, pw, pw, pw);
+            }
+        }
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&bars.empty[s]);   // the stage is in registers: release it
+
+        float x[kVpt][N];
+        float vm[kVpt];
+#pragma unroll
+        for (int j = 0; j < kVpt; ++j) {
+#pragma unroll
+            for (int e = 0; e < N; ++e) x[j][e] = Elem<DT>::get(v[j], e);
+            if constexpr (N == 8) {
+                vm[j] = max3(max3(x[j][0], x[j][1], x[j][2]), max3(x[j][3], x[j][4], x[j][5]),
+                             fmaxf(x[j][6], x[j][7]));
+            } else {
+                vm[j] = fmaxf(max3(x[j][0], x[j][1], x[j][2]), x[j][3]);
+            }
+        }
+        const float tm = fmaxf(fmaxf(vm[0], vm[1]), fmaxf(vm[2], vm[3]));
+
+        float thr_now;
+        if (t == 0) {
+            bootstrap_threshold<SY>(sm, tm, K);       // consumers only; no candidate exists yet
+            thr_now = sm.thr_v;
+        } else {
+            thr_now = *reinterpret_cast<volatile float *>(&sm.thr_v);
+        }
+        if (thr_now > thr) {
+            thr = thr_now;
+            if constexpr (SUMS) raise_ref(thr * kLog2e);
+        }
+        if (tm >= thr) {
+            if constexpr (SUMS) raise_ref(tm * kLog2e);
+            const int ebase = s0 + t * TE + tid * N;
+#pragma unroll
+            for (int j = 0; j < kVpt; ++j) {
+                if (vm[j] >= thr) {
+#pragma unroll
+                    for (int e = 0; e < N; ++e) {
+                        const float xv = x[j][e];
+                        const int idx = ebase + j * kThreads * N + e;
+                        if (xv >= thr && xv > -CUDART_INF_F && idx < s1) {
+                            const int pos = atomicAdd(&sm.cnt, 1);
+                            if (pos < kCandCap) sm.cand[pos] = make_key(xv, idx);
+                            else sm.overflow = 1;
+                        }
+                    }
+                }
+            }
+        }
+        if constexpr (SUMS) {
+            const float nc = -c;
+#pragma unroll
+            for (int j = 0; j < kVpt; ++j) {
+#pragma unroll
+                for (int e = 0; e < N; ++e) {
+                    const float a = fmaf(x[j][e], kLog2e, nc);
+                    const float ex = ex2_approx(a);
+                    S += ex;
+                    T = fmaf(ex, a, T);
+                }
+            }
+        }
+    }
+    // this warp's appends are complete: tell the service warp, then meet it
+    __syncwarp();
+    if (lane == 0) {
+        __threadfence_block();
+        atomicAdd(&ctl.done_warps, 1);
+        if (timed_out) ctl.timed_out = 1;
+    }
+    stream_sync_all();
+    const int nsel = ctl.nsel;
+    const unsigned long long mine = tid < nsel ? sm.sel[tid] : 0ull;
+    SY::sync();
+    if (tid < nsel) sm.cand[tid] = mine;
+    if (tid == 0) sm.cnt = nsel;
+    SY::sync();
+    if (sm.overflow) topk_careful<DT, SY>(row, s0, s1, K, sm);
+
+    if constexpr (SUMS) {
+        reduce_sums<DT, SY>(row, s0, s1, sm, c, S, T, c_out, S_out, T_out);
+    } else {
+        c_out = kRefFloor; S_out = 0.0; T_out = 0.0;
+    }
+}
+
+// The ring needs more dynamic shared memory than the default limit: raise the limit of `kernel`
+// once per device (the attribute is per device).  `rec` is the caller's per-kernel record.
+struct RingSmemDone {
+    bool dev[64] = {};
+};
+template <typename KernelT>
+inline cudaError_t allow_ring_smem(KernelT *kernel, RingSmemDone &rec) {
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (dev >= 0 && dev < 64 && rec.dev[dev]) return cudaSuccess;
+    e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kRingBytes);
+    if (e == cudaSuccess && dev >= 0 && dev < 64) rec.dev[dev] = true;
+    return e;
+}
+
+// True if rows of this layout can be streamed with bulk copies.
+inline bool stream_layout_ok(const void *base, size_t elem_bytes, int V, long long stride_b,
+                             long long stride_l) {
+    return (reinterpret_cast<uintptr_t>(base) & 15) == 0 && ((size_t)V * elem_bytes) % 16 == 0 &&
+           ((size_t)stride_b * elem_bytes) % 16 == 0 && ((size_t)stride_l * elem_bytes) % 16 == 0;
+}
+
+}  // namespace dsp

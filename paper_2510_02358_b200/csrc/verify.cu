@@ -7,7 +7,7 @@
 // a sampling job (stochastic: residual at the first rejection, or bonus from row m).
 // Kernel 2 (residual_kernel): for each job, one more pass over ONE target row (and ONE draft
 // row): per-chunk sums of max(0, p - q) in token order; the CTA arriving last inverts the CDF.
-#include "scan_core.cuh"
+#include "stream_core.cuh"
 
 namespace dsp {
 
@@ -128,23 +128,14 @@ __device__ void accept_row(const VerifyArgs &a, int b) {
     }
 }
 
-template <typename DT>
-__global__ void __launch_bounds__(kThreads, 4) target_kernel(const VerifyArgs a) {
-    __shared__ ScanSmem sm;
+// Everything after the scan of one slice of a target row: publish the slice's best key and
+// sums, let the CTA arriving last finish the row (argmax, log-sum-exp), and let the CTA that
+// finishes the last row of a batch row run that row's acceptance scan.
+template <typename DT, typename SY>
+__device__ void target_finish(const VerifyArgs &a, ScanSmem &sm, long long row, int slice, int b,
+                              bool sums, float c, double S, double T, unsigned extra_status) {
     const int tid = threadIdx.x;
-    const long long row = blockIdx.x / a.nslices;
-    const int slice = blockIdx.x - (int)(row * a.nslices);
-    const int b = (int)(row / a.Lt);
-    const DT *rowp = trow_ptr<DT>(a, row);
-    const int s0 = slice * a.slice_elems;
-    const int s1 = min(a.V, s0 + a.slice_elems);
-    const bool sums = !a.all_greedy && a.mode[b] != 0;
-
-    float c;
-    double S, T;
-    if (sums) scan_slice<DT, true>(rowp, s0, s1, 1, sm, c, S, T);
-    else      scan_slice<DT, false>(rowp, s0, s1, 1, sm, c, S, T);
-
+    if (extra_status && tid == 0) atomicOr(&a.b_status[b], extra_status);
     unsigned long long best = sm.cnt > 0 ? sm.cand[0] : 0ull;
     if (a.nslices > 1) {
         SlicePartial *part = a.partials + row * a.nslices;
@@ -155,7 +146,7 @@ __global__ void __launch_bounds__(kThreads, 4) target_kernel(const VerifyArgs a)
             __threadfence();
             sm.flag = (int)atomicAdd(&a.row_ticket[row], 1u);
         }
-        __syncthreads();
+        SY::sync();
         if (sm.flag != a.nslices - 1) return;
         __threadfence();
         if (tid == 0) {
@@ -184,10 +175,59 @@ __global__ void __launch_bounds__(kThreads, 4) target_kernel(const VerifyArgs a)
         __threadfence();
         sm.flag = (int)atomicAdd(&a.b_ticket[b], 1u);
     }
-    __syncthreads();
+    SY::sync();
     if (sm.flag != a.Lt - 1) return;
     __threadfence();
     if (tid < 32) accept_row<DT>(a, b);
+}
+
+
+// Element-wise kernel: any layout.
+template <typename DT>
+__global__ void __launch_bounds__(kThreads, 4) target_kernel(const VerifyArgs a) {
+    __shared__ ScanSmem sm;
+    const long long row = blockIdx.x / a.nslices;
+    const int slice = blockIdx.x - (int)(row * a.nslices);
+    const int b = (int)(row / a.Lt);
+    const DT *rowp = trow_ptr<DT>(a, row);
+    const int s0 = slice * a.slice_elems;
+    const int s1 = min(a.V, s0 + a.slice_elems);
+    const bool sums = !a.all_greedy && a.mode[b] != 0;
+    float c;
+    double S, T;
+    if (sums) scan_slice<DT, true>(rowp, s0, s1, 1, sm, c, S, T);
+    else      scan_slice<DT, false>(rowp, s0, s1, 1, sm, c, S, T);
+    target_finish<DT, SyncAll>(a, sm, row, slice, b, sums, c, S, T, 0u);
+}
+
+// Streaming kernel for 16-byte aligned layouts (see stream_core.cuh).
+template <typename DT>
+__global__ void __launch_bounds__(kStreamThreads, 3) target_stream_kernel(const VerifyArgs a) {
+    extern __shared__ __align__(128) unsigned char ring[];
+    __shared__ ScanSmem sm;
+    __shared__ StreamBars bars;
+    __shared__ StreamCtl ctl;
+    const int tid = threadIdx.x;
+    const long long row = blockIdx.x / a.nslices;
+    const int slice = blockIdx.x - (int)(row * a.nslices);
+    const int b = (int)(row / a.Lt);
+    const DT *rowp = trow_ptr<DT>(a, row);
+    const int s0 = slice * a.slice_elems;
+    const int s1 = min(a.V, s0 + a.slice_elems);
+    const bool sums = !a.all_greedy && a.mode[b] != 0;
+    stream_begin(sm, ctl, bars);
+    if (tid >= kThreads) {                                  // service warp: copies + running best
+        stream_service(reinterpret_cast<const char *>(rowp + s0), (s1 - s0) * (int)sizeof(DT), 1, sm, ctl,
+                       ring, bars);
+        stream_sync_all();
+        return;
+    }
+    float c;
+    double S, T;
+    if (sums) scan_slice_stream<DT, true>(rowp, s0, s1, 1, sm, ctl, ring, bars, c, S, T);
+    else      scan_slice_stream<DT, false>(rowp, s0, s1, 1, sm, ctl, ring, bars, c, S, T);
+    target_finish<DT, SyncConsumers>(a, sm, row, slice, b, sums, c, S, T,
+                                     ctl.timed_out ? DSP_ROW_TIMEOUT : 0u);
 }
 
 // ---- residual / bonus sampling -------------------------------------------------------------
@@ -408,7 +448,13 @@ static int32_t launch_verify(VerifyArgs &a, void *workspace, size_t workspace_by
     DSP_CUDA_TRY(cudaMemsetAsync(ws, 0, w.zero_bytes, st));
     const long long nblocks = nrows * a.nslices;
     if (nblocks > 0x7FFFFFFFLL) return DSP_ERR_UNSUPPORTED;
-    target_kernel<DT><<<(unsigned)nblocks, kThreads, 0, st>>>(a);
+    if (stream_layout_ok(a.target, sizeof(DT), a.V, a.tstride_b, a.tstride_l)) {
+        static RingSmemDone smem_done;                       // one per element type
+        DSP_CUDA_TRY(allow_ring_smem(target_stream_kernel<DT>, smem_done));
+        target_stream_kernel<DT><<<(unsigned)nblocks, kStreamThreads, kRingBytes, st>>>(a);
+    } else {
+        target_kernel<DT><<<(unsigned)nblocks, kThreads, 0, st>>>(a);
+    }
     DSP_CUDA_TRY(cudaGetLastError());
     if (!a.all_greedy) {
         residual_kernel<DT><<<(unsigned)(a.B * a.res_slices), kThreads, 0, st>>>(a);

@@ -146,6 +146,7 @@ def check_step(g: SimpleNamespace, inp: dict, *, K: int, W: int, tau: float = 0.
         a, o = G.ver.ratio[good], Ov.ratio[good]
         err("ratio", a, o)
         assert _close(a, o, 1e-5, 1e-4).all(), f"ratio off by {rep['max_err']['ratio']}"
+    assert not (G.lat.row_status & dsp.ROW_TIMEOUT).any(), "a bounded wait inside a kernel ran out"
     flags = dsp.ROW_NO_BONUS_ROW | dsp.ROW_EOS_ACCEPTED | dsp.ROW_ZERO_RESIDUAL
     for b in range(B):
         if bad_any[b]:
