@@ -184,9 +184,9 @@ __global__ void __launch_bounds__(kThreads, 4) lattice_kernel(const LatticeArgs 
     lattice_finish<DT, SyncAll>(a, sm, row, slice, b, rowp, c, S, T, 0u);
 }
 
-// Streaming kernel for 16-byte aligned layouts: a service warp feeds the slice through a
-// shared-memory ring with bulk asynchronous copies and keeps the running top-K; the consumers
-// scan the ring (see stream_core.cuh).
+// Streaming kernel for 16-byte aligned layouts: a producer warp feeds the slice through a
+// shared-memory ring with bulk asynchronous copies; the consumers scan the ring (see
+// stream_core.cuh).
 template <typename DT>
 __global__ void __launch_bounds__(kStreamThreads, 3) lattice_stream_kernel(const LatticeArgs a) {
     extern __shared__ __align__(128) unsigned char ring[];
@@ -201,10 +201,10 @@ __global__ void __launch_bounds__(kStreamThreads, 3) lattice_stream_kernel(const
     const int s0 = slice * a.slice_elems;
     const int s1 = min(a.V, s0 + a.slice_elems);
     stream_begin(sm, ctl, bars);
-    if (tid >= kThreads) {                                  // service warp: copies + running top-K
-        stream_service(reinterpret_cast<const char *>(rowp + s0), (s1 - s0) * (int)sizeof(DT), a.K, sm,
-                       ctl, ring, bars);
-        stream_sync_all();
+    if (tid >= kThreads) {                                  // producer warp
+        if (tid == kThreads)
+            stream_produce(reinterpret_cast<const char *>(rowp + s0), (s1 - s0) * (int)sizeof(DT), ring, bars,
+                           ctl);
         return;
     }
     float c;

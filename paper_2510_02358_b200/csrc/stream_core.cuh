@@ -1,12 +1,11 @@
 // TMA-fed variant of the one-pass slice scan for rows whose start, strides and length are
-// multiples of 16 bytes.  A service warp streams the slice through a ring of shared-memory
-// stages with bulk asynchronous copies (cp.async.bulk, completion counted on an mbarrier per
-// stage, no multicast); the kThreads consumer threads read each stage with one 128-bit shared
-// load per vector, release it at once and do the arithmetic from registers.  Logits at or
-// above the current threshold are appended to a candidate list; the service warp turns that
-// list into the running top-K and a tighter threshold while the consumers keep streaming, so
-// the scan has no block-wide barrier except the first tile's threshold bootstrap.  Results are
-// the same as scan_slice's (scan_core.cuh): log-sum-exp terms and the exact top-K.
+// multiples of 16 bytes.  One thread of a producer warp streams the slice through a ring of
+// shared-memory stages with bulk asynchronous copies (cp.async.bulk, completion counted on an
+// mbarrier per stage, no multicast); the kThreads consumer threads read each stage with one
+// 128-bit shared load per vector, release it at once and do the arithmetic from registers.
+// Logits at or above the current threshold are appended to a candidate list that the
+// consumers prune to the best K a few times per slice.  Results are the same as scan_slice's
+// (scan_core.cuh): log-sum-exp terms and the exact top-K.
 #pragma once
 
 #include "scan_core.cuh"
@@ -15,10 +14,9 @@ namespace dsp {
 
 constexpr int kTileBytes = kThreads * kVpt * 16;     // one ring stage = one tile of either dtype
 constexpr int kStages = 4;
-constexpr int kStreamThreads = kThreads + 32;        // consumers + the service warp
+constexpr int kStreamThreads = kThreads + 32;        // consumers + the producer warp
 constexpr int kRingBytes = kStages * kTileBytes;
-constexpr int kWaitTries = 1 << 22;                  // bound of every mbarrier wait and spin
-constexpr int kIdleLimit = 1 << 22;                  // idle polls of the service warp before it gives up
+constexpr long long kWaitCycles = 400000000LL;       // every wait gives up after this many SM clocks (~0.2 s)
 
 __device__ __forceinline__ uint32_t smem_addr(const void *p) {
     return (uint32_t)__cvta_generic_to_shared(p);
@@ -36,10 +34,12 @@ __device__ __forceinline__ void mbar_expect_tx(uint64_t *bar, uint32_t bytes) {
 __device__ __forceinline__ void mbar_arrive(uint64_t *bar) {
     asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_addr(bar)) : "memory");
 }
-// Bounded wait for the phase with the given parity; false if it never completed.
-__device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity) {
+// Bounded wait for the phase with the given parity: gives up after kWaitCycles, or at once when
+// another wait of this CTA has already given up (`abort` non-zero).  False if it gave up.
+__device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, volatile int *abort) {
     const uint32_t a = smem_addr(bar);
-    for (int i = 0; i < kWaitTries; ++i) {
+    const long long t0 = clock64();
+    for (;;) {
         uint32_t ok;
         asm volatile(
             "{\n"
@@ -51,8 +51,8 @@ __device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity) {
             : "r"(a), "r"(parity)
             : "memory");
         if (ok) return true;
+        if (*abort || clock64() - t0 > kWaitCycles) return false;
     }
-    return false;
 }
 // Non-blocking test of a phase.
 __device__ __forceinline__ bool mbar_test(uint64_t *bar, uint32_t parity) {
@@ -85,113 +85,38 @@ struct StreamBars {
     uint64_t empty[kStages];
 };
 
-// Shared state between the consumers and the service warp of one slice scan.
+// Per-CTA record of bounded waits that gave up.
 struct StreamCtl {
-    int done_warps;      // consumer warps that have finished their last tile
-    int nsel;            // number of keys the service warp left in ScanSmem::sel
-    int timed_out;       // a bounded wait ran out
+    int timed_out;
 };
 
-// Barrier of all kStreamThreads threads of the CTA (named barrier 2).
-__device__ __forceinline__ void stream_sync_all() {
-    asm volatile("bar.sync 2, %0;" ::"n"(kStreamThreads) : "memory");
-}
-
-// Called by every thread before service/consume start (ends with a CTA-wide barrier).
+// Called by every thread before produce/consume start (ends with a CTA-wide barrier).
 __device__ __forceinline__ void stream_begin(ScanSmem &sm, StreamCtl &ctl, StreamBars &bars) {
-    const int tid = threadIdx.x;
-    if (tid == 0) {
+    if (threadIdx.x == 0) {
         for (int s = 0; s < kStages; ++s) {
             mbar_init(&bars.full[s], 1);
             mbar_init(&bars.empty[s], kWarps);
         }
         mbar_init_fence();
         sm.cnt = 0; sm.thrkey = 0ull; sm.thr_v = -CUDART_INF_F; sm.overflow = 0;
-        ctl.done_warps = 0; ctl.nsel = 0; ctl.timed_out = 0;
+        ctl.timed_out = 0;
     }
-    for (int i = tid; i < kCandCap; i += kStreamThreads) sm.cand[i] = 0ull;   // 0 = not written yet
     __syncthreads();
 }
 
-// The service warp of a slice scan (32 threads, all of them call this).  Two duties:
-//  - lane 0 streams bytes [0, nbytes) at `src` through the ring, one bulk copy per free stage;
-//  - the warp keeps the best 32 keys seen so far, one per lane, sorted descending.  It reads the
-//    candidate keys that the consumers append to sm.cand (an append-only list during the scan),
-//    inserts those that beat its K-th key, and publishes the K-th key's value as the new
-//    threshold sm.thr_v.  The consumers never stop for this: they pick the threshold up at
-//    their next tile.  The K-th best of any subset of the slice is a valid lower bound.
-// On return (all tiles issued, all consumer warps done, every appended key processed) the best
-// min(K, #keys) keys are in sm.sel[0 .. ctl.nsel), sorted.
-__device__ __forceinline__ void stream_service(const char *src, int nbytes, int K, ScanSmem &sm,
-                                               StreamCtl &ctl, unsigned char *ring, StreamBars &bars) {
-    const int lane = threadIdx.x & 31;
+// Producer (one thread): stream bytes [0, nbytes) at `src` through the ring.  If a wait for a
+// free stage gives up, the copy is issued all the same so that every consumer wait still ends.
+__device__ __forceinline__ void stream_produce(const char *src, int nbytes, unsigned char *ring,
+                                               StreamBars &bars, StreamCtl &ctl) {
+    volatile int *abort = &ctl.timed_out;
     const int ntiles = (nbytes + kTileBytes - 1) / kTileBytes;
-    int t_next = 0;                                   // lane 0: next tile to issue
-    unsigned long long mykey = 0ull;                  // 0 = empty slot (below every real key)
-    unsigned long long kth = 0ull;                    // key of rank K-1, 0 while fewer than K are held
-    float thr_pub = -CUDART_INF_F;
-    int processed = 0, idle = 0;
-    volatile int *v_cnt = &sm.cnt;
-    volatile int *v_done = &ctl.done_warps;
-    volatile unsigned long long *v_cand = sm.cand;
-    for (;;) {
-        if (lane == 0) {
-            while (t_next < ntiles) {
-                const int s = t_next % kStages;
-                if (t_next >= kStages && !mbar_test(&bars.empty[s], ((t_next / kStages) - 1) & 1)) break;
-                const uint32_t bytes = (uint32_t)min(kTileBytes, nbytes - t_next * kTileBytes);
-                mbar_expect_tx(&bars.full[s], bytes);
-                bulk_load(ring + (size_t)s * kTileBytes, src + (size_t)t_next * kTileBytes, bytes,
-                          &bars.full[s]);
-                ++t_next;
-            }
-        }
-        const bool all_issued = __shfl_sync(0xFFFFFFFFu, (int)(t_next >= ntiles), 0) != 0;
-        const int done_w = *v_done;                   // read before the count: once every warp is
-        __threadfence_block();                        // done, the count that follows is final
-        const int cnt = min(*v_cnt, kCandCap);
-        if (processed < cnt) {
-            idle = 0;
-            const int i = processed + lane;
-            unsigned long long key = 0ull;
-            if (i < cnt) {                            // a slot is claimed before it is written
-                for (int spin = 0; spin < kWaitTries; ++spin) {
-                    key = v_cand[i];
-                    if (key != 0ull) break;
-                }
-            }
-            unsigned pending = __ballot_sync(0xFFFFFFFFu, key > kth);
-            while (pending) {
-                const int from = __ffs(pending) - 1;
-                pending &= pending - 1;
-                const unsigned long long nk = __shfl_sync(0xFFFFFFFFu, key, from);
-                const int p = __popc(__ballot_sync(0xFFFFFFFFu, mykey > nk));   // keys ahead of nk
-                const unsigned long long up = __shfl_up_sync(0xFFFFFFFFu, mykey, 1);
-                if (lane == p) mykey = nk;
-                else if (lane > p) mykey = up;
-            }
-            processed = min(cnt, processed + 32);
-            kth = __shfl_sync(0xFFFFFFFFu, mykey, K - 1);
-            if (lane == 0 && kth != 0ull) {
-                const float v = key_value(kth);
-                if (v > thr_pub) {
-                    thr_pub = v;
-                    *reinterpret_cast<volatile float *>(&sm.thr_v) = v;
-                }
-            }
-        } else if (all_issued && done_w == kWarps) {
-            break;
-        } else {
-            if (++idle > kIdleLimit) {
-                if (lane == 0) ctl.timed_out = 1;
-                break;
-            }
-            __nanosleep(100);
-        }
+    for (int t = 0; t < ntiles; ++t) {
+        const int s = t % kStages;
+        if (t >= kStages && !mbar_wait(&bars.empty[s], ((t / kStages) - 1) & 1, abort)) ctl.timed_out = 1;
+        const uint32_t bytes = (uint32_t)min(kTileBytes, nbytes - t * kTileBytes);
+        mbar_expect_tx(&bars.full[s], bytes);
+        bulk_load(ring + (size_t)s * kTileBytes, src + (size_t)t * kTileBytes, bytes, &bars.full[s]);
     }
-    const unsigned have = __ballot_sync(0xFFFFFFFFu, mykey != 0ull && lane < K);
-    if (lane < DSP_MAX_K) sm.sel[lane] = mykey;
-    if (lane == 0) ctl.nsel = __popc(have);
 }
 
 // Padding for the vectors past the end of a ragged last tile: -2^124, below every finite
@@ -201,8 +126,7 @@ template <typename DT> struct Pad;
 template <> struct Pad<__nv_bfloat16> { static constexpr uint32_t kWord = 0xFD80FD80u; };
 template <> struct Pad<float> { static constexpr uint32_t kWord = 0xFD800000u; };
 
-// Consumer side of the scan of [s0, s1) of `row` (kThreads threads, barriers via SyncConsumers;
-// the service warp runs stream_service meanwhile and both sides meet in stream_sync_all).
+// Consumer side of the scan of [s0, s1) of `row` (kThreads threads, barriers via SyncConsumers).
 // Same contract as scan_slice.
 template <typename DT, bool SUMS>
 __device__ void scan_slice_stream(const DT *__restrict__ row, int s0, int s1, int K, ScanSmem &sm,
@@ -219,7 +143,8 @@ __device__ void scan_slice_stream(const DT *__restrict__ row, int s0, int s1, in
 
     float c = kRefFloor, S = 0.f, T = 0.f;
     float thr = -CUDART_INF_F;
-    bool timed_out = false;
+    int next_prune = 1;                              // prune after tiles 1, 7, 31, ... and the last
+    volatile int *abort = &ctl.timed_out;
 
     // the reference exponent must bound every logit below the threshold (those skip the test)
     auto raise_ref = [&](float ts) {
@@ -234,7 +159,7 @@ __device__ void scan_slice_stream(const DT *__restrict__ row, int s0, int s1, in
 
     for (int t = 0; t < ntiles; ++t) {
         const int s = t % kStages;
-        if (!mbar_wait(&bars.full[s], (t / kStages) & 1)) timed_out = true;
+        if (!mbar_wait(&bars.full[s], (t / kStages) & 1, abort)) ctl.timed_out = 1;
         const int nvec = min(kTileBytes, nbytes - t * kTileBytes) >> 4;
         const uint4 *sp = reinterpret_cast<const uint4 *>(ring + (size_t)s * kTileBytes);
         uint4 v[kVpt];
@@ -267,16 +192,10 @@ __device__ void scan_slice_stream(const DT *__restrict__ row, int s0, int s1, in
         }
         const float tm = fmaxf(fmaxf(vm[0], vm[1]), fmaxf(vm[2], vm[3]));
 
-        float thr_now;
         if (t == 0) {
-            bootstrap_threshold<SY>(sm, tm, K);       // consumers only; no candidate exists yet
-            thr_now = sm.thr_v;
-        } else {
-            thr_now = *reinterpret_cast<volatile float *>(&sm.thr_v);
-        }
-        if (thr_now > thr) {
-            thr = thr_now;
-            if constexpr (SUMS) raise_ref(thr * kLog2e);
+            bootstrap_threshold<SY>(sm, tm, K);
+            thr = sm.thr_v;
+            if constexpr (SUMS) { if (thr > -CUDART_INF_F) raise_ref(thr * kLog2e); }
         }
         if (tm >= thr) {
             if constexpr (SUMS) raise_ref(tm * kLog2e);
@@ -291,7 +210,6 @@ __device__ void scan_slice_stream(const DT *__restrict__ row, int s0, int s1, in
                         if (xv >= thr && xv > -CUDART_INF_F && idx < s1) {
                             const int pos = atomicAdd(&sm.cnt, 1);
                             if (pos < kCandCap) sm.cand[pos] = make_key(xv, idx);
-                            else sm.overflow = 1;
                         }
                     }
                 }
@@ -310,21 +228,13 @@ __device__ void scan_slice_stream(const DT *__restrict__ row, int s0, int s1, in
                 }
             }
         }
+        if (t == next_prune || t == ntiles - 1) {
+            prune<SY>(sm, K);
+            thr = sm.thr_v;
+            if constexpr (SUMS) { if (thr > -CUDART_INF_F) raise_ref(thr * kLog2e); }
+            next_prune = next_prune * 4 + 3;
+        }
     }
-    // this warp's appends are complete: tell the service warp, then meet it
-    __syncwarp();
-    if (lane == 0) {
-        __threadfence_block();
-        atomicAdd(&ctl.done_warps, 1);
-        if (timed_out) ctl.timed_out = 1;
-    }
-    stream_sync_all();
-    const int nsel = ctl.nsel;
-    const unsigned long long mine = tid < nsel ? sm.sel[tid] : 0ull;
-    SY::sync();
-    if (tid < nsel) sm.cand[tid] = mine;
-    if (tid == 0) sm.cnt = nsel;
-    SY::sync();
     if (sm.overflow) topk_careful<DT, SY>(row, s0, s1, K, sm);
 
     if constexpr (SUMS) {
