@@ -217,7 +217,7 @@ __global__ void __launch_bounds__(kStreamThreads, 3) lattice_stream_kernel(const
 template <typename DT>
 static int32_t launch_lattice(LatticeArgs &a, void *workspace, size_t workspace_bytes, cudaStream_t st) {
     const long long nrows = (long long)a.B * a.L;
-    const SlicePlan plan = plan_slices<DT>(nrows, a.V, 148 * 8);
+    const SlicePlan plan = plan_slices<DT>(nrows, a.V, kTargetCtas);
     a.nslices = plan.nslices;
     a.slice_elems = plan.slice_elems;
     const LatticeWs w = lattice_ws_layout(a.B, a.L, a.nslices, a.K);
@@ -244,7 +244,7 @@ static int32_t launch_lattice(LatticeArgs &a, void *workspace, size_t workspace_
 
 template <typename DT>
 static size_t lattice_ws_bytes(int B, int L, int V, int K) {
-    const SlicePlan plan = plan_slices<DT>((long long)B * L, V, 148 * 8);
+    const SlicePlan plan = plan_slices<DT>((long long)B * L, V, kTargetCtas);
     return lattice_ws_layout(B, L, plan.nslices, K).total;
 }
 

@@ -3,8 +3,8 @@
 // shared-memory stages with bulk asynchronous copies (cp.async.bulk, completion counted on an
 // mbarrier per stage, no multicast); the kThreads consumer threads read each stage with one
 // 128-bit shared load per vector, release it at once and do the arithmetic from registers.
-// Logits at or above the current threshold are appended to a candidate list that the
-// consumers prune to the best K a few times per slice.  Results are the same as scan_slice's
+// Logits at or above the current threshold are appended to a candidate list that warp 0 folds
+// into a register-resident sorted top-K a few times per slice.  Results are the same as scan_slice's
 // (scan_core.cuh): log-sum-exp terms and the exact top-K.
 #pragma once
 
@@ -119,6 +119,43 @@ __device__ __forceinline__ void stream_produce(const char *src, int nbytes, unsi
     }
 }
 
+// Running top-K of a slice kept by warp 0 of the consumers: the best 32 keys seen so far, one
+// per lane in `mykey`, sorted descending (0 = empty slot, below every real key).  Block-wide:
+// folds the candidate keys appended since the last call into the list, empties the candidate
+// list and refreshes the threshold (value of the K-th key).  Work is proportional to the number
+// of new candidates: a batch of 32 is read at once, those that do not beat the current K-th key
+// are dropped by one ballot, the others are inserted one by one (ballot, shuffle-up, select).
+template <typename SY>
+__device__ __forceinline__ void fold_candidates(ScanSmem &sm, int K, unsigned long long &mykey) {
+    SY::sync();
+    if (threadIdx.x < 32) {
+        const int lane = threadIdx.x;
+        const int total = sm.cnt;
+        const int n = min(total, kCandCap);
+        unsigned long long kth = __shfl_sync(0xFFFFFFFFu, mykey, K - 1);
+        for (int base = 0; base < n; base += 32) {
+            const unsigned long long key = base + lane < n ? sm.cand[base + lane] : 0ull;
+            unsigned pending = __ballot_sync(0xFFFFFFFFu, key > kth);
+            while (pending) {
+                const int from = __ffs(pending) - 1;
+                pending &= pending - 1;
+                const unsigned long long nk = __shfl_sync(0xFFFFFFFFu, key, from);
+                const int p = __popc(__ballot_sync(0xFFFFFFFFu, mykey > nk));   // keys ahead of nk
+                const unsigned long long up = __shfl_up_sync(0xFFFFFFFFu, mykey, 1);
+                if (lane == p) mykey = nk;
+                else if (lane > p) mykey = up;
+            }
+            kth = __shfl_sync(0xFFFFFFFFu, mykey, K - 1);
+        }
+        if (lane == 0) {
+            if (total > kCandCap) sm.overflow = 1;
+            sm.cnt = 0;
+            if (kth != 0ull) { sm.thrkey = kth; sm.thr_v = key_value(kth); }
+        }
+    }
+    SY::sync();
+}
+
 // Padding for the vectors past the end of a ragged last tile: -2^124, below every finite
 // logit the interface allows, finite when scaled by log2(e), never a candidate (its index is
 // past the row).
@@ -143,7 +180,7 @@ __device__ void scan_slice_stream(const DT *__restrict__ row, int s0, int s1, in
 
     float c = kRefFloor, S = 0.f, T = 0.f;
     float thr = -CUDART_INF_F;
-    int next_prune = 1;                              // prune after tiles 1, 7, 31, ... and the last
+    unsigned long long mykey = 0ull;                 // warp 0: its lane's key of the running top-K
     volatile int *abort = &ctl.timed_out;
 
     // the reference exponent must bound every logit below the threshold (those skip the test)
@@ -174,9 +211,6 @@ __device__ void scan_slice_stream(const DT *__restrict__ row, int s0, int s1, in
                 v[j] = vi < nvec ? sp[vi] : make_uint4(pw, pw, pw, pw);
             }
         }
-        __syncwarp();
-        if (lane == 0) mbar_arrive(&bars.empty[s]);   // the stage is in registers: release it
-
         float x[kVpt][N];
         float vm[kVpt];
 #pragma unroll
@@ -199,15 +233,20 @@ __device__ void scan_slice_stream(const DT *__restrict__ row, int s0, int s1, in
         }
         if (tm >= thr) {
             if constexpr (SUMS) raise_ref(tm * kLog2e);
-            const int ebase = s0 + t * TE + tid * N;
+            const DT *tile = reinterpret_cast<const DT *>(sp);
 #pragma unroll
             for (int j = 0; j < kVpt; ++j) {
                 if (vm[j] >= thr) {
+                    unsigned hits = 0;
 #pragma unroll
-                    for (int e = 0; e < N; ++e) {
-                        const float xv = x[j][e];
-                        const int idx = ebase + j * kThreads * N + e;
-                        if (xv >= thr && xv > -CUDART_INF_F && idx < s1) {
+                    for (int e = 0; e < N; ++e) hits |= (x[j][e] >= thr ? 1u : 0u) << e;
+                    const int vpos = (j * kThreads + tid) * N;           // element offset inside the tile
+                    while (hits) {
+                        const int e = __ffs(hits) - 1;
+                        hits &= hits - 1;
+                        const int idx = s0 + t * TE + vpos + e;
+                        const float xv = Elem<DT>::load1(tile + vpos + e);   // still in the ring stage
+                        if (xv > -CUDART_INF_F && idx < s1) {
                             const int pos = atomicAdd(&sm.cnt, 1);
                             if (pos < kCandCap) sm.cand[pos] = make_key(xv, idx);
                         }
@@ -215,6 +254,8 @@ __device__ void scan_slice_stream(const DT *__restrict__ row, int s0, int s1, in
                 }
             }
         }
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&bars.empty[s]);   // done with the stage: release it
         if constexpr (SUMS) {
             const float nc = -c;
 #pragma unroll
@@ -228,13 +269,19 @@ __device__ void scan_slice_stream(const DT *__restrict__ row, int s0, int s1, in
                 }
             }
         }
-        if (t == next_prune || t == ntiles - 1) {
-            prune<SY>(sm, K);
+        if (((t + 1) & t) == 0 || t == ntiles - 1) {   // after tiles 0, 1, 3, 7, 15, ... and the last
+            fold_candidates<SY>(sm, K, mykey);
             thr = sm.thr_v;
             if constexpr (SUMS) { if (thr > -CUDART_INF_F) raise_ref(thr * kLog2e); }
-            next_prune = next_prune * 4 + 3;
         }
     }
+    // the slice's best keys, sorted, go to the front of the candidate list
+    if (tid < 32) {
+        const unsigned have = __ballot_sync(0xFFFFFFFFu, mykey != 0ull && tid < K);
+        if (mykey != 0ull && tid < K) sm.cand[tid] = mykey;
+        if (tid == 0) sm.cnt = __popc(have);
+    }
+    SY::sync();
     if (sm.overflow) topk_careful<DT, SY>(row, s0, s1, K, sm);
 
     if constexpr (SUMS) {

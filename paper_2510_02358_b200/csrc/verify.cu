@@ -413,14 +413,14 @@ static int nchunks_of(int V) { return (V + 32 * Elem<DT>::N - 1) / (32 * Elem<DT
 
 template <typename DT>
 static size_t verify_ws_bytes(int B, int Lt, int V) {
-    const SlicePlan plan = plan_slices<DT>((long long)B * Lt, V, 148 * 8);
+    const SlicePlan plan = plan_slices<DT>((long long)B * Lt, V, kTargetCtas);
     return verify_ws_layout(B, Lt, plan.nslices, nchunks_of<DT>(V)).total;
 }
 
 template <typename DT>
 static int32_t launch_verify(VerifyArgs &a, void *workspace, size_t workspace_bytes, cudaStream_t st) {
     const long long nrows = (long long)a.B * a.Lt;
-    const SlicePlan plan = plan_slices<DT>(nrows, a.V, 148 * 8);
+    const SlicePlan plan = plan_slices<DT>(nrows, a.V, kTargetCtas);
     a.nslices = plan.nslices;
     a.slice_elems = plan.slice_elems;
     a.nchunks = nchunks_of<DT>(a.V);

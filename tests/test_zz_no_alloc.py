@@ -49,11 +49,11 @@ def test_static_scratch_build_matches_the_workspace_build_on_two_calls_in_a_row(
 
 def test_static_scratch_rejects_problems_beyond_its_limit():
     # host-side check only: nothing is enqueued, so this runs without a GPU
-    need = dsp.dsp_lattice_workspace_bytes(256, 64, 256000, dsp.DSP_BF16, 16)
+    need = dsp.dsp_lattice_workspace_bytes(2048, 64, 256000, dsp.DSP_BF16, 16)
     assert need > dsp.DSP_STATIC_WS_BYTES
     import ctypes as C
     one = C.c_void_p(256)
-    rc = dsp.lib().dsp_lattice_build_static(one, dsp.DSP_BF16, 256, 64, 256000, C.c_int64(64 * 256000),
+    rc = dsp.lib().dsp_lattice_build_static(one, dsp.DSP_BF16, 2048, 64, 256000, C.c_int64(64 * 256000),
                                             C.c_int64(256000), 16, C.c_float(0), -1, one, one, one, one,
                                             one, one, one, one, one, C.c_void_p(0))
     assert rc == dsp.DSP_ERR_STATIC_SCRATCH
