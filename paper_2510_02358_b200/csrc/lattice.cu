@@ -201,10 +201,9 @@ __global__ void __launch_bounds__(kStreamThreads, 3) lattice_stream_kernel(const
     const int s0 = slice * a.slice_elems;
     const int s1 = min(a.V, s0 + a.slice_elems);
     stream_begin(sm, ctl, bars);
-    if (tid >= kThreads) {                                  // producer warp
-        if (tid == kThreads)
-            stream_produce(reinterpret_cast<const char *>(rowp + s0), (s1 - s0) * (int)sizeof(DT), ring, bars,
-                           ctl);
+    if (tid >= kThreads) {                                  // producer warp: copies + top-K folds
+        stream_service(reinterpret_cast<const char *>(rowp + s0), (s1 - s0) * (int)sizeof(DT), a.K, sm, ctl,
+                       ring, bars);
         return;
     }
     float c;

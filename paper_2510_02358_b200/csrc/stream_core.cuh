@@ -3,8 +3,12 @@
 // shared-memory stages with bulk asynchronous copies (cp.async.bulk, completion counted on an
 // mbarrier per stage, no multicast); the kThreads consumer threads read each stage with one
 // 128-bit shared load per vector, release it at once and do the arithmetic from registers.
-// Logits at or above the current threshold are appended to a candidate list that warp 0 folds
-// into a register-resident sorted top-K a few times per slice.  Results are the same as scan_slice's
+// Logits at or above the current threshold are appended to one of two candidate lists.  At a
+// few fold points per slice the consumers switch lists and go on; the producer warp, between
+// its copies, folds the list they left into a register-resident sorted top-K and publishes a
+// tighter threshold that the consumers pick up at their next tile.  The two sides hand over
+// through two mbarriers with time-bounded waits, so the consumers meet no block-wide barrier
+// after the first tile's threshold bootstrap.  Results are the same as scan_slice's
 // (scan_core.cuh): log-sum-exp terms and the exact top-K.
 #pragma once
 
@@ -81,13 +85,22 @@ __device__ __forceinline__ float max3(float a, float b, float c) {
 }
 
 struct StreamBars {
-    uint64_t full[kStages];
-    uint64_t empty[kStages];
+    uint64_t full[kStages];      // stage filled by its bulk copy
+    uint64_t empty[kStages];     // stage released by all consumer warps
+    uint64_t listed;             // phase i: every consumer warp has passed fold point i
+    uint64_t folded;             // phase i: the producer warp has folded the list of fold point i
 };
 
-// Per-CTA record of bounded waits that gave up.
+constexpr int kListCap = kCandCap / 2;               // entries of each of the two candidate lists
+
+// Fold points of a slice of ntiles tiles: after tiles 0, 3, 15, 63, ... and after the last tile.
+__device__ __forceinline__ int next_fold_tile(int f) { return f * 4 + 3; }
+
+// Shared state of one slice scan besides ScanSmem.
 struct StreamCtl {
-    int timed_out;
+    int cnt[2];          // entries appended to each candidate list (may exceed kListCap: overflow)
+    int nsel;            // keys the producer warp left in ScanSmem::sel after the last fold
+    int timed_out;       // non-zero once a bounded wait gave up
 };
 
 // Called by every thread before produce/consume start (ends with a CTA-wide barrier).
@@ -97,63 +110,91 @@ __device__ __forceinline__ void stream_begin(ScanSmem &sm, StreamCtl &ctl, Strea
             mbar_init(&bars.full[s], 1);
             mbar_init(&bars.empty[s], kWarps);
         }
+        mbar_init(&bars.listed, kWarps);
+        mbar_init(&bars.folded, 1);
         mbar_init_fence();
         sm.cnt = 0; sm.thrkey = 0ull; sm.thr_v = -CUDART_INF_F; sm.overflow = 0;
-        ctl.timed_out = 0;
+        ctl.cnt[0] = 0; ctl.cnt[1] = 0; ctl.nsel = 0; ctl.timed_out = 0;
     }
     __syncthreads();
 }
 
-// Producer (one thread): stream bytes [0, nbytes) at `src` through the ring.  If a wait for a
-// free stage gives up, the copy is issued all the same so that every consumer wait still ends.
-__device__ __forceinline__ void stream_produce(const char *src, int nbytes, unsigned char *ring,
-                                               StreamBars &bars, StreamCtl &ctl) {
-    volatile int *abort = &ctl.timed_out;
-    const int ntiles = (nbytes + kTileBytes - 1) / kTileBytes;
-    for (int t = 0; t < ntiles; ++t) {
-        const int s = t % kStages;
-        if (t >= kStages && !mbar_wait(&bars.empty[s], ((t / kStages) - 1) & 1, abort)) ctl.timed_out = 1;
-        const uint32_t bytes = (uint32_t)min(kTileBytes, nbytes - t * kTileBytes);
-        mbar_expect_tx(&bars.full[s], bytes);
-        bulk_load(ring + (size_t)s * kTileBytes, src + (size_t)t * kTileBytes, bytes, &bars.full[s]);
+// Fold candidate list `which` into the warp's sorted top-32 (one key per lane in `mykey`,
+// descending, 0 = empty slot below every real key): a batch of 32 keys is read at once, those
+// that do not beat the K-th key are dropped by one ballot, the others are inserted one by one
+// (ballot, shuffle-up, select).  Empties the list.  Whole warp.
+__device__ __forceinline__ void fold_list(ScanSmem &sm, StreamCtl &ctl, int which, int K,
+                                          unsigned long long &mykey) {
+    const int lane = threadIdx.x & 31;
+    const unsigned long long *list = sm.cand + which * kListCap;
+    const int total = ctl.cnt[which];
+    const int n = min(total, kListCap);
+    unsigned long long kth = __shfl_sync(0xFFFFFFFFu, mykey, K - 1);
+    for (int base = 0; base < n; base += 32) {
+        const unsigned long long key = base + lane < n ? list[base + lane] : 0ull;
+        unsigned pending = __ballot_sync(0xFFFFFFFFu, key > kth);
+        while (pending) {
+            const int from = __ffs(pending) - 1;
+            pending &= pending - 1;
+            const unsigned long long nk = __shfl_sync(0xFFFFFFFFu, key, from);
+            const int p = __popc(__ballot_sync(0xFFFFFFFFu, mykey > nk));   // keys ahead of nk
+            const unsigned long long up = __shfl_up_sync(0xFFFFFFFFu, mykey, 1);
+            if (lane == p) mykey = nk;
+            else if (lane > p) mykey = up;
+        }
+        kth = __shfl_sync(0xFFFFFFFFu, mykey, K - 1);
+    }
+    if (lane == 0) {
+        if (total > kListCap) sm.overflow = 1;
+        ctl.cnt[which] = 0;
+        if (kth != 0ull) *reinterpret_cast<volatile float *>(&sm.thr_v) = key_value(kth);
     }
 }
 
-// Running top-K of a slice kept by warp 0 of the consumers: the best 32 keys seen so far, one
-// per lane in `mykey`, sorted descending (0 = empty slot, below every real key).  Block-wide:
-// folds the candidate keys appended since the last call into the list, empties the candidate
-// list and refreshes the threshold (value of the K-th key).  Work is proportional to the number
-// of new candidates: a batch of 32 is read at once, those that do not beat the current K-th key
-// are dropped by one ballot, the others are inserted one by one (ballot, shuffle-up, select).
-template <typename SY>
-__device__ __forceinline__ void fold_candidates(ScanSmem &sm, int K, unsigned long long &mykey) {
-    SY::sync();
-    if (threadIdx.x < 32) {
-        const int lane = threadIdx.x;
-        const int total = sm.cnt;
-        const int n = min(total, kCandCap);
-        unsigned long long kth = __shfl_sync(0xFFFFFFFFu, mykey, K - 1);
-        for (int base = 0; base < n; base += 32) {
-            const unsigned long long key = base + lane < n ? sm.cand[base + lane] : 0ull;
-            unsigned pending = __ballot_sync(0xFFFFFFFFu, key > kth);
-            while (pending) {
-                const int from = __ffs(pending) - 1;
-                pending &= pending - 1;
-                const unsigned long long nk = __shfl_sync(0xFFFFFFFFu, key, from);
-                const int p = __popc(__ballot_sync(0xFFFFFFFFu, mykey > nk));   // keys ahead of nk
-                const unsigned long long up = __shfl_up_sync(0xFFFFFFFFu, mykey, 1);
-                if (lane == p) mykey = nk;
-                else if (lane > p) mykey = up;
-            }
-            kth = __shfl_sync(0xFFFFFFFFu, mykey, K - 1);
-        }
+// The producer warp of a slice scan (32 threads, all of them call this; it takes part in no
+// barrier of the CTA after stream_begin and exits when it returns).  Lane 0 streams bytes
+// [0, nbytes) at `src` through the ring in order.  Fold point i (after tile f_i) is served right
+// after tile min(f_i + 2, last) has been issued, so the consumers always have copies in flight
+// while the warp folds: it waits until every consumer warp has passed the point (phase i of
+// bars.listed), folds list i & 1, publishes the threshold and completes phase i of bars.folded.
+// After the last fold the best min(K, #keys) keys are in sm.sel[0 .. ctl.nsel), sorted.
+// If a wait gives up, the work goes on all the same so that every other wait still ends.
+__device__ __forceinline__ void stream_service(const char *src, int nbytes, int K, ScanSmem &sm,
+                                               StreamCtl &ctl, unsigned char *ring, StreamBars &bars) {
+    const int lane = threadIdx.x & 31;
+    volatile int *abort = &ctl.timed_out;
+    const int ntiles = (nbytes + kTileBytes - 1) / kTileBytes;
+    unsigned long long mykey = 0ull;
+    int fold = 0;                                     // index of the next fold point
+    int fold_tile = 0;                                // tile after which that point lies
+    for (int t = 0; t < ntiles; ++t) {
         if (lane == 0) {
-            if (total > kCandCap) sm.overflow = 1;
-            sm.cnt = 0;
-            if (kth != 0ull) { sm.thrkey = kth; sm.thr_v = key_value(kth); }
+            const int s = t % kStages;
+            if (t >= kStages && !mbar_wait(&bars.empty[s], ((t / kStages) - 1) & 1, abort)) ctl.timed_out = 1;
+            const uint32_t bytes = (uint32_t)min(kTileBytes, nbytes - t * kTileBytes);
+            mbar_expect_tx(&bars.full[s], bytes);
+            bulk_load(ring + (size_t)s * kTileBytes, src + (size_t)t * kTileBytes, bytes, &bars.full[s]);
+        }
+        __syncwarp();
+        while (fold_tile <= ntiles - 1 && min(fold_tile + 2, ntiles - 1) == t) {
+            const bool last = fold_tile == ntiles - 1;
+            if (!mbar_wait(&bars.listed, fold & 1, abort)) ctl.timed_out = 1;
+            fold_list(sm, ctl, fold & 1, K, mykey);
+            if (last) {
+                const unsigned have = __ballot_sync(0xFFFFFFFFu, mykey != 0ull && lane < K);
+                if (lane < DSP_MAX_K) sm.sel[lane] = mykey;
+                if (lane == 0) ctl.nsel = __popc(have);
+            }
+            __syncwarp();
+            if (lane == 0) {
+                __threadfence_block();
+                mbar_arrive(&bars.folded);
+            }
+            ++fold;
+            if (last) fold_tile = ntiles;             // no further point
+            else fold_tile = min(next_fold_tile(fold_tile), ntiles - 1);
         }
     }
-    SY::sync();
 }
 
 // Padding for the vectors past the end of a ragged last tile: -2^124, below every finite
@@ -163,8 +204,8 @@ template <typename DT> struct Pad;
 template <> struct Pad<__nv_bfloat16> { static constexpr uint32_t kWord = 0xFD80FD80u; };
 template <> struct Pad<float> { static constexpr uint32_t kWord = 0xFD800000u; };
 
-// Consumer side of the scan of [s0, s1) of `row` (kThreads threads, barriers via SyncConsumers).
-// Same contract as scan_slice.
+// Consumer side of the scan of [s0, s1) of `row` (kThreads threads, barriers via SyncConsumers;
+// the producer warp runs stream_service meanwhile).  Same contract as scan_slice.
 template <typename DT, bool SUMS>
 __device__ void scan_slice_stream(const DT *__restrict__ row, int s0, int s1, int K, ScanSmem &sm,
                                   StreamCtl &ctl, const unsigned char *ring, StreamBars &bars,
@@ -180,7 +221,7 @@ __device__ void scan_slice_stream(const DT *__restrict__ row, int s0, int s1, in
 
     float c = kRefFloor, S = 0.f, T = 0.f;
     float thr = -CUDART_INF_F;
-    unsigned long long mykey = 0ull;                 // warp 0: its lane's key of the running top-K
+    int fold = 0, fold_tile = 0;                     // next fold point and the tile it follows
     volatile int *abort = &ctl.timed_out;
 
     // the reference exponent must bound every logit below the threshold (those skip the test)
@@ -226,10 +267,16 @@ __device__ void scan_slice_stream(const DT *__restrict__ row, int s0, int s1, in
         }
         const float tm = fmaxf(fmaxf(vm[0], vm[1]), fmaxf(vm[2], vm[3]));
 
+        float thr_now;
         if (t == 0) {
-            bootstrap_threshold<SY>(sm, tm, K);
-            thr = sm.thr_v;
-            if constexpr (SUMS) { if (thr > -CUDART_INF_F) raise_ref(thr * kLog2e); }
+            bootstrap_threshold<SY>(sm, tm, K);       // consumers only; no candidate exists yet
+            thr_now = sm.thr_v;
+        } else {
+            thr_now = *reinterpret_cast<volatile float *>(&sm.thr_v);
+        }
+        if (thr_now > thr) {
+            thr = thr_now;
+            if constexpr (SUMS) raise_ref(thr * kLog2e);
         }
         if (tm >= thr) {
             if constexpr (SUMS) raise_ref(tm * kLog2e);
@@ -247,8 +294,8 @@ __device__ void scan_slice_stream(const DT *__restrict__ row, int s0, int s1, in
                         const int idx = s0 + t * TE + vpos + e;
                         const float xv = Elem<DT>::load1(tile + vpos + e);   // still in the ring stage
                         if (xv > -CUDART_INF_F && idx < s1) {
-                            const int pos = atomicAdd(&sm.cnt, 1);
-                            if (pos < kCandCap) sm.cand[pos] = make_key(xv, idx);
+                            const int pos = atomicAdd(&ctl.cnt[fold & 1], 1);
+                            if (pos < kListCap) sm.cand[(fold & 1) * kListCap + pos] = make_key(xv, idx);
                         }
                     }
                 }
@@ -269,18 +316,21 @@ __device__ void scan_slice_stream(const DT *__restrict__ row, int s0, int s1, in
                 }
             }
         }
-        if (((t + 1) & t) == 0 || t == ntiles - 1) {   // after tiles 0, 1, 3, 7, 15, ... and the last
-            fold_candidates<SY>(sm, K, mykey);
-            thr = sm.thr_v;
-            if constexpr (SUMS) { if (thr > -CUDART_INF_F) raise_ref(thr * kLog2e); }
+        if (t == fold_tile) {
+            // fold point: the list this warp appended to is complete; switch to the other list,
+            // which the producer warp emptied when it served the previous point
+            if (fold >= 1 && !mbar_wait(&bars.folded, (fold - 1) & 1, abort)) ctl.timed_out = 1;
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&bars.listed);
+            ++fold;
+            fold_tile = min(next_fold_tile(fold_tile), ntiles - 1);
         }
     }
-    // the slice's best keys, sorted, go to the front of the candidate list
-    if (tid < 32) {
-        const unsigned have = __ballot_sync(0xFFFFFFFFu, mykey != 0ull && tid < K);
-        if (mykey != 0ull && tid < K) sm.cand[tid] = mykey;
-        if (tid == 0) sm.cnt = __popc(have);
-    }
+    // the last fold leaves the slice's best keys, sorted, in sm.sel
+    if (!mbar_wait(&bars.folded, (fold - 1) & 1, abort)) ctl.timed_out = 1;
+    const int nsel = min(ctl.nsel, K);
+    if (tid < nsel) sm.cand[tid] = sm.sel[tid];
+    if (tid == 0) sm.cnt = nsel;
     SY::sync();
     if (sm.overflow) topk_careful<DT, SY>(row, s0, s1, K, sm);
 

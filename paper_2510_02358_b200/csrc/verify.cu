@@ -216,10 +216,9 @@ __global__ void __launch_bounds__(kStreamThreads, 3) target_stream_kernel(const 
     const int s1 = min(a.V, s0 + a.slice_elems);
     const bool sums = !a.all_greedy && a.mode[b] != 0;
     stream_begin(sm, ctl, bars);
-    if (tid >= kThreads) {                                  // producer warp
-        if (tid == kThreads)
-            stream_produce(reinterpret_cast<const char *>(rowp + s0), (s1 - s0) * (int)sizeof(DT), ring, bars,
-                           ctl);
+    if (tid >= kThreads) {                                  // producer warp: copies + top-K folds
+        stream_service(reinterpret_cast<const char *>(rowp + s0), (s1 - s0) * (int)sizeof(DT), 1, sm, ctl,
+                       ring, bars);
         return;
     }
     float c;
