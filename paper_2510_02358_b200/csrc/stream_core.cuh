@@ -93,8 +93,8 @@ struct StreamBars {
 
 constexpr int kListCap = kCandCap / 2;               // entries of each of the two candidate lists
 
-// Fold points of a slice of ntiles tiles: after tiles 0, 3, 15, 63, ... and after the last tile.
-__device__ __forceinline__ int next_fold_tile(int f) { return f * 4 + 3; }
+// Fold points of a slice: after every tile (a fold costs the consumers one mbarrier arrival).
+__device__ __forceinline__ int next_fold_tile(int f) { return f + 1; }
 
 // Shared state of one slice scan besides ScanSmem.
 struct StreamCtl {
@@ -119,10 +119,42 @@ __device__ __forceinline__ void stream_begin(ScanSmem &sm, StreamCtl &ctl, Strea
     __syncthreads();
 }
 
+__device__ __forceinline__ unsigned long long umax64(unsigned long long a, unsigned long long b) { return a > b ? a : b; }
+__device__ __forceinline__ unsigned long long umin64(unsigned long long a, unsigned long long b) { return a < b ? a : b; }
+
+// Sort 32 keys, one per lane, descending over the lanes (bitonic network).
+__device__ __forceinline__ unsigned long long sort32_desc(unsigned long long v, int lane) {
+#pragma unroll
+    for (int k = 2; k <= 32; k <<= 1) {
+#pragma unroll
+        for (int j = k >> 1; j > 0; j >>= 1) {
+            const unsigned long long o = __shfl_xor_sync(0xFFFFFFFFu, v, j);
+            const bool up = (lane & k) == 0;
+            const bool lower = (lane & j) == 0;
+            v = (lower == up) ? umax64(v, o) : umin64(v, o);
+        }
+    }
+    return v;
+}
+
+// Best 32 of two descending 32-key lists (one key per lane each), descending: the lane-wise
+// maximum of one list and the other reversed is bitonic and holds the best 32; five
+// compare-exchange stages sort it.
+__device__ __forceinline__ unsigned long long merge_top32(unsigned long long a, unsigned long long b, int lane) {
+    unsigned long long v = umax64(a, __shfl_sync(0xFFFFFFFFu, b, 31 - lane));
+#pragma unroll
+    for (int j = 16; j > 0; j >>= 1) {
+        const unsigned long long o = __shfl_xor_sync(0xFFFFFFFFu, v, j);
+        v = (lane & j) == 0 ? umax64(v, o) : umin64(v, o);
+    }
+    return v;
+}
+
 // Fold candidate list `which` into the warp's sorted top-32 (one key per lane in `mykey`,
-// descending, 0 = empty slot below every real key): a batch of 32 keys is read at once, those
-// that do not beat the K-th key are dropped by one ballot, the others are inserted one by one
-// (ballot, shuffle-up, select).  Empties the list.  Whole warp.
+// descending, 0 = empty slot below every real key).  A batch of 32 keys is read at once and
+// those that do not beat the K-th key are dropped by one ballot; a few survivors are inserted
+// one by one (ballot, shuffle-up, select), many are sorted and merged in.  Empties the list and
+// publishes the K-th key's value as the new threshold.  Whole warp.
 __device__ __forceinline__ void fold_list(ScanSmem &sm, StreamCtl &ctl, int which, int K,
                                           unsigned long long &mykey) {
     const int lane = threadIdx.x & 31;
@@ -131,16 +163,21 @@ __device__ __forceinline__ void fold_list(ScanSmem &sm, StreamCtl &ctl, int whic
     const int n = min(total, kListCap);
     unsigned long long kth = __shfl_sync(0xFFFFFFFFu, mykey, K - 1);
     for (int base = 0; base < n; base += 32) {
-        const unsigned long long key = base + lane < n ? list[base + lane] : 0ull;
-        unsigned pending = __ballot_sync(0xFFFFFFFFu, key > kth);
-        while (pending) {
-            const int from = __ffs(pending) - 1;
-            pending &= pending - 1;
-            const unsigned long long nk = __shfl_sync(0xFFFFFFFFu, key, from);
-            const int p = __popc(__ballot_sync(0xFFFFFFFFu, mykey > nk));   // keys ahead of nk
-            const unsigned long long up = __shfl_up_sync(0xFFFFFFFFu, mykey, 1);
-            if (lane == p) mykey = nk;
-            else if (lane > p) mykey = up;
+        unsigned long long key = base + lane < n ? list[base + lane] : 0ull;
+        if (!(key > kth)) key = 0ull;
+        unsigned pending = __ballot_sync(0xFFFFFFFFu, key != 0ull);
+        if (__popc(pending) > 3) {
+            mykey = merge_top32(mykey, sort32_desc(key, lane), lane);
+        } else {
+            while (pending) {
+                const int from = __ffs(pending) - 1;
+                pending &= pending - 1;
+                const unsigned long long nk = __shfl_sync(0xFFFFFFFFu, key, from);
+                const int p = __popc(__ballot_sync(0xFFFFFFFFu, mykey > nk));   // keys ahead of nk
+                const unsigned long long up = __shfl_up_sync(0xFFFFFFFFu, mykey, 1);
+                if (lane == p) mykey = nk;
+                else if (lane > p) mykey = up;
+            }
         }
         kth = __shfl_sync(0xFFFFFFFFu, mykey, K - 1);
     }
@@ -149,6 +186,43 @@ __device__ __forceinline__ void fold_list(ScanSmem &sm, StreamCtl &ctl, int whic
         ctl.cnt[which] = 0;
         if (kth != 0ull) *reinterpret_cast<volatile float *>(&sm.thr_v) = key_value(kth);
     }
+}
+
+// First threshold of a slice from the thread maxima of its first tile, for the consumers of a
+// streaming kernel: with r = ceil(K / #warps), the smallest over the warps of each warp's r-th
+// largest thread maximum has K distinct logits at or above it.  One barrier; every thread
+// derives the value itself and thread 0 also stores it in sm.thr_v.  If some warp has fewer
+// than r finite maxima (masked rows) the general rule of bootstrap_threshold applies.
+template <typename SY>
+__device__ __forceinline__ float bootstrap_threshold_fast(ScanSmem &sm, float tm, int K) {
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const float s = bitonic_desc(tm == tm ? tm : -CUDART_INF_F, lane);
+    sm.wsorted[warp][lane] = s;
+    SY::sync();
+    const int r = (K + kWarps - 1) / kWarps;
+    float t = CUDART_INF_F;
+#pragma unroll
+    for (int w = 0; w < kWarps; ++w) t = fminf(t, sm.wsorted[w][r - 1]);
+    if (t > -CUDART_INF_F) {
+        if (tid == 0) sm.thr_v = t;
+        return t;
+    }
+    if (tid == 0) {
+        float g = -CUDART_INF_F;
+        for (int rr = 1; rr <= 32; ++rr) {
+            int nw = 0;
+            float lo = CUDART_INF_F;
+            for (int w = 0; w < kWarps; ++w) {
+                const float x = sm.wsorted[w][rr - 1];
+                if (x > -CUDART_INF_F) { ++nw; lo = fminf(lo, x); }
+            }
+            if (nw == 0) break;
+            if (rr * nw >= K) { g = lo; break; }
+        }
+        sm.thr_v = g;
+    }
+    SY::sync();
+    return sm.thr_v;
 }
 
 // The producer warp of a slice scan (32 threads, all of them call this; it takes part in no
@@ -269,8 +343,7 @@ __device__ void scan_slice_stream(const DT *__restrict__ row, int s0, int s1, in
 
         float thr_now;
         if (t == 0) {
-            bootstrap_threshold<SY>(sm, tm, K);       // consumers only; no candidate exists yet
-            thr_now = sm.thr_v;
+            thr_now = bootstrap_threshold_fast<SY>(sm, tm, K);   // consumers only; no candidate exists yet
         } else {
             thr_now = *reinterpret_cast<volatile float *>(&sm.thr_v);
         }
