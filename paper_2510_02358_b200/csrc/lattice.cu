@@ -184,9 +184,9 @@ __global__ void __launch_bounds__(kThreads, 4) lattice_kernel(const LatticeArgs 
     lattice_finish<DT, SyncAll>(a, sm, row, slice, b, rowp, c, S, T, 0u);
 }
 
-// Streaming kernel for 16-byte aligned layouts: a producer warp feeds the slice through a
-// shared-memory ring with bulk asynchronous copies; the consumers scan the ring (see
-// stream_core.cuh).
+// Streaming kernel for 16-byte aligned layouts: the slice streams through a shared-memory
+// ring of bulk asynchronous copies, the consumers scan the ring and a ninth warp keeps the
+// running top-K (see stream_core.cuh).
 template <typename DT>
 __global__ void __launch_bounds__(kStreamThreads, 3) lattice_stream_kernel(const LatticeArgs a) {
     extern __shared__ __align__(128) unsigned char ring[];
@@ -201,9 +201,8 @@ __global__ void __launch_bounds__(kStreamThreads, 3) lattice_stream_kernel(const
     const int s0 = slice * a.slice_elems;
     const int s1 = min(a.V, s0 + a.slice_elems);
     stream_begin(sm, ctl, bars);
-    if (tid >= kThreads) {                                  // producer warp: copies + top-K folds
-        stream_service(reinterpret_cast<const char *>(rowp + s0), (s1 - s0) * (int)sizeof(DT), a.K, sm, ctl,
-                       ring, bars);
+    if (tid >= kThreads) {                                  // fold warp: running top-K
+        stream_service((s1 - s0) * (int)sizeof(DT), a.K, sm, ctl, bars);
         return;
     }
     float c;

@@ -1,14 +1,13 @@
 // TMA-fed variant of the one-pass slice scan for rows whose start, strides and length are
-// multiples of 16 bytes.  One thread of a producer warp streams the slice through a ring of
-// shared-memory stages with bulk asynchronous copies (cp.async.bulk, completion counted on an
-// mbarrier per stage, no multicast); the kThreads consumer threads read each stage with one
-// 128-bit shared load per vector, release it at once and do the arithmetic from registers.
-// Logits at or above the current threshold are appended to one of two candidate lists.  At a
-// few fold points per slice the consumers switch lists and go on; the producer warp, between
-// its copies, folds the list they left into a register-resident sorted top-K and publishes a
-// tighter threshold that the consumers pick up at their next tile.  The two sides hand over
-// through two mbarriers with time-bounded waits, so the consumers meet no block-wide barrier
-// after the first tile's threshold bootstrap.  Results are the same as scan_slice's
+// multiples of 16 bytes.  The slice streams through a ring of shared-memory stages by bulk
+// asynchronous copies (cp.async.bulk, completion counted on an mbarrier per stage, no
+// multicast) that one consumer thread issues three tiles ahead; the kThreads consumer threads
+// read each stage with one 128-bit shared load per vector and do the arithmetic from registers.
+// Logits at or above the current threshold are appended to the candidate list of their tile
+// (four lists in rotation).  A ninth warp, the fold warp, folds each tile's list into
+// a register-resident sorted top-K and publishes a tighter threshold that the consumers pick
+// up at their next tile.  The two sides hand over through mbarriers with time-bounded waits,
+// so the consumers meet no block-wide barrier after the first tile's threshold bootstrap.  Results are the same as scan_slice's
 // (scan_core.cuh): log-sum-exp terms and the exact top-K.
 #pragma once
 
@@ -18,7 +17,7 @@ namespace dsp {
 
 constexpr int kTileBytes = kThreads * kVpt * 16;     // one ring stage = one tile of either dtype
 constexpr int kStages = 4;
-constexpr int kStreamThreads = kThreads + 32;        // consumers + the producer warp
+constexpr int kStreamThreads = kThreads + 32;        // consumers + the fold warp
 constexpr int kRingBytes = kStages * kTileBytes;
 constexpr long long kWaitCycles = 400000000LL;       // every wait gives up after this many SM clocks (~0.2 s)
 
@@ -87,19 +86,20 @@ __device__ __forceinline__ float max3(float a, float b, float c) {
 struct StreamBars {
     uint64_t full[kStages];      // stage filled by its bulk copy
     uint64_t empty[kStages];     // stage released by all consumer warps
-    uint64_t listed;             // phase i: every consumer warp has passed fold point i
-    uint64_t folded;             // phase i: the producer warp has folded the list of fold point i
+    uint64_t listed[4];          // list l, phase n: every consumer warp is past tile 4n + l
+    uint64_t folded[4];          // list l, phase n: the fold warp has folded tile 4n + l's candidates
 };
 
-constexpr int kListCap = kCandCap / 2;               // entries of each of the two candidate lists
-
-// Fold points of a slice: after every tile (a fold costs the consumers one mbarrier arrival).
-__device__ __forceinline__ int next_fold_tile(int f) { return f + 1; }
+// The candidates of tile t go to list t % kLists; the list is folded after the tile and must be
+// empty again before tile t + kLists, which leaves the fold warp three tiles of slack.
+constexpr int kLists = 4;
+constexpr int kListCap = kCandCap / kLists;
+static_assert(kLists == 4, "StreamBars holds four barriers of each kind");
 
 // Shared state of one slice scan besides ScanSmem.
 struct StreamCtl {
-    int cnt[2];          // entries appended to each candidate list (may exceed kListCap: overflow)
-    int nsel;            // keys the producer warp left in ScanSmem::sel after the last fold
+    int cnt[kLists];     // entries appended to each candidate list (may exceed kListCap: overflow)
+    int nsel;            // keys the fold warp left in ScanSmem::sel after the last fold
     int timed_out;       // non-zero once a bounded wait gave up
 };
 
@@ -110,11 +110,14 @@ __device__ __forceinline__ void stream_begin(ScanSmem &sm, StreamCtl &ctl, Strea
             mbar_init(&bars.full[s], 1);
             mbar_init(&bars.empty[s], kWarps);
         }
-        mbar_init(&bars.listed, kWarps);
-        mbar_init(&bars.folded, 1);
+        for (int l = 0; l < kLists; ++l) {
+            mbar_init(&bars.listed[l], kWarps);
+            mbar_init(&bars.folded[l], 1);
+            ctl.cnt[l] = 0;
+        }
         mbar_init_fence();
         sm.cnt = 0; sm.thrkey = 0ull; sm.thr_v = -CUDART_INF_F; sm.overflow = 0;
-        ctl.cnt[0] = 0; ctl.cnt[1] = 0; ctl.nsel = 0; ctl.timed_out = 0;
+        ctl.nsel = 0; ctl.timed_out = 0;
     }
     __syncthreads();
 }
@@ -225,48 +228,40 @@ __device__ __forceinline__ float bootstrap_threshold_fast(ScanSmem &sm, float tm
     return sm.thr_v;
 }
 
-// The producer warp of a slice scan (32 threads, all of them call this; it takes part in no
-// barrier of the CTA after stream_begin and exits when it returns).  Lane 0 streams bytes
-// [0, nbytes) at `src` through the ring in order.  Fold point i (after tile f_i) is served right
-// after tile min(f_i + 2, last) has been issued, so the consumers always have copies in flight
-// while the warp folds: it waits until every consumer warp has passed the point (phase i of
-// bars.listed), folds list i & 1, publishes the threshold and completes phase i of bars.folded.
-// After the last fold the best min(K, #keys) keys are in sm.sel[0 .. ctl.nsel), sorted.
-// If a wait gives up, the work goes on all the same so that every other wait still ends.
-__device__ __forceinline__ void stream_service(const char *src, int nbytes, int K, ScanSmem &sm,
-                                               StreamCtl &ctl, unsigned char *ring, StreamBars &bars) {
+// Issue the bulk copy of tile t of the slice at `src` into its ring stage (one thread).
+__device__ __forceinline__ void issue_tile(const char *src, int nbytes, int t, unsigned char *ring,
+                                           StreamBars &bars) {
+    const int s = t % kStages;
+    const uint32_t bytes = (uint32_t)min(kTileBytes, nbytes - t * kTileBytes);
+    mbar_expect_tx(&bars.full[s], bytes);
+    bulk_load(ring + (size_t)s * kTileBytes, src + (size_t)t * kTileBytes, bytes, &bars.full[s]);
+}
+
+// The fold warp of a slice scan (32 threads, all of them call this; it takes part in no barrier
+// of the CTA after stream_begin and exits when it returns).  For every tile i in order it waits
+// until every consumer warp is past the tile (bars.listed), folds list i % kLists into its
+// sorted top-32, publishes the threshold and completes the list's bars.folded phase.  After the
+// last fold the best min(K, #keys) keys are in sm.sel[0 .. ctl.nsel), sorted.  If a wait gives
+// up, the work goes on all the same so that every other wait still ends.
+__device__ __forceinline__ void stream_service(int nbytes, int K, ScanSmem &sm, StreamCtl &ctl,
+                                               StreamBars &bars) {
     const int lane = threadIdx.x & 31;
     volatile int *abort = &ctl.timed_out;
     const int ntiles = (nbytes + kTileBytes - 1) / kTileBytes;
     unsigned long long mykey = 0ull;
-    int fold = 0;                                     // index of the next fold point
-    int fold_tile = 0;                                // tile after which that point lies
-    for (int t = 0; t < ntiles; ++t) {
-        if (lane == 0) {
-            const int s = t % kStages;
-            if (t >= kStages && !mbar_wait(&bars.empty[s], ((t / kStages) - 1) & 1, abort)) ctl.timed_out = 1;
-            const uint32_t bytes = (uint32_t)min(kTileBytes, nbytes - t * kTileBytes);
-            mbar_expect_tx(&bars.full[s], bytes);
-            bulk_load(ring + (size_t)s * kTileBytes, src + (size_t)t * kTileBytes, bytes, &bars.full[s]);
+    for (int fold = 0; fold < ntiles; ++fold) {
+        const int l = fold % kLists;
+        if (!mbar_wait(&bars.listed[l], (fold / kLists) & 1, abort)) ctl.timed_out = 1;
+        fold_list(sm, ctl, l, K, mykey);
+        if (fold == ntiles - 1) {
+            const unsigned have = __ballot_sync(0xFFFFFFFFu, mykey != 0ull && lane < K);
+            if (lane < DSP_MAX_K) sm.sel[lane] = mykey;
+            if (lane == 0) ctl.nsel = __popc(have);
         }
         __syncwarp();
-        while (fold_tile <= ntiles - 1 && min(fold_tile + 2, ntiles - 1) == t) {
-            const bool last = fold_tile == ntiles - 1;
-            if (!mbar_wait(&bars.listed, fold & 1, abort)) ctl.timed_out = 1;
-            fold_list(sm, ctl, fold & 1, K, mykey);
-            if (last) {
-                const unsigned have = __ballot_sync(0xFFFFFFFFu, mykey != 0ull && lane < K);
-                if (lane < DSP_MAX_K) sm.sel[lane] = mykey;
-                if (lane == 0) ctl.nsel = __popc(have);
-            }
-            __syncwarp();
-            if (lane == 0) {
-                __threadfence_block();
-                mbar_arrive(&bars.folded);
-            }
-            ++fold;
-            if (last) fold_tile = ntiles;             // no further point
-            else fold_tile = min(next_fold_tile(fold_tile), ntiles - 1);
+        if (lane == 0) {
+            __threadfence_block();
+            mbar_arrive(&bars.folded[l]);
         }
     }
 }
@@ -279,10 +274,10 @@ template <> struct Pad<__nv_bfloat16> { static constexpr uint32_t kWord = 0xFD80
 template <> struct Pad<float> { static constexpr uint32_t kWord = 0xFD800000u; };
 
 // Consumer side of the scan of [s0, s1) of `row` (kThreads threads, barriers via SyncConsumers;
-// the producer warp runs stream_service meanwhile).  Same contract as scan_slice.
+// the fold warp runs stream_service meanwhile).  Same contract as scan_slice.
 template <typename DT, bool SUMS>
 __device__ void scan_slice_stream(const DT *__restrict__ row, int s0, int s1, int K, ScanSmem &sm,
-                                  StreamCtl &ctl, const unsigned char *ring, StreamBars &bars,
+                                  StreamCtl &ctl, unsigned char *ring, StreamBars &bars,
                                   float &c_out, double &S_out, double &T_out) {
     using SY = SyncConsumers;
     constexpr int N = Elem<DT>::N;
@@ -295,7 +290,6 @@ __device__ void scan_slice_stream(const DT *__restrict__ row, int s0, int s1, in
 
     float c = kRefFloor, S = 0.f, T = 0.f;
     float thr = -CUDART_INF_F;
-    int fold = 0, fold_tile = 0;                     // next fold point and the tile it follows
     volatile int *abort = &ctl.timed_out;
 
     // the reference exponent must bound every logit below the threshold (those skip the test)
@@ -309,7 +303,17 @@ __device__ void scan_slice_stream(const DT *__restrict__ row, int s0, int s1, in
         }
     };
 
+    // Thread 0 also issues the copies, kStages - 1 tiles ahead of the tile being scanned.
+    const char *src = reinterpret_cast<const char *>(row + s0);
+    if (tid == 0) {
+        for (int tt = 0; tt < min(kStages, ntiles); ++tt) issue_tile(src, nbytes, tt, ring, bars);
+    }
     for (int t = 0; t < ntiles; ++t) {
+        if (tid == 0 && t >= 1 && t + kStages - 1 < ntiles) {
+            const int tt = t + kStages - 1;           // its stage held tile t - 1
+            if (!mbar_wait(&bars.empty[tt % kStages], ((tt / kStages) - 1) & 1, abort)) ctl.timed_out = 1;
+            issue_tile(src, nbytes, tt, ring, bars);
+        }
         const int s = t % kStages;
         if (!mbar_wait(&bars.full[s], (t / kStages) & 1, abort)) ctl.timed_out = 1;
         const int nvec = min(kTileBytes, nbytes - t * kTileBytes) >> 4;
@@ -351,24 +355,25 @@ __device__ void scan_slice_stream(const DT *__restrict__ row, int s0, int s1, in
             thr = thr_now;
             if constexpr (SUMS) raise_ref(thr * kLog2e);
         }
-        if (tm >= thr) {
-            if constexpr (SUMS) raise_ref(tm * kLog2e);
+        // Vectors holding a logit at or above the threshold are few: the warp takes them one at a
+        // time and its first N lanes test one logit each, read back from the ring stage.
+        if (__ballot_sync(0xFFFFFFFFu, tm >= thr)) {
+            if constexpr (SUMS) { if (tm >= thr) raise_ref(tm * kLog2e); }
             const DT *tile = reinterpret_cast<const DT *>(sp);
+            const int l = t % kLists;
 #pragma unroll
             for (int j = 0; j < kVpt; ++j) {
-                if (vm[j] >= thr) {
-                    unsigned hits = 0;
-#pragma unroll
-                    for (int e = 0; e < N; ++e) hits |= (x[j][e] >= thr ? 1u : 0u) << e;
-                    const int vpos = (j * kThreads + tid) * N;           // element offset inside the tile
-                    while (hits) {
-                        const int e = __ffs(hits) - 1;
-                        hits &= hits - 1;
-                        const int idx = s0 + t * TE + vpos + e;
-                        const float xv = Elem<DT>::load1(tile + vpos + e);   // still in the ring stage
-                        if (xv > -CUDART_INF_F && idx < s1) {
-                            const int pos = atomicAdd(&ctl.cnt[fold & 1], 1);
-                            if (pos < kListCap) sm.cand[(fold & 1) * kListCap + pos] = make_key(xv, idx);
+                unsigned hitters = __ballot_sync(0xFFFFFFFFu, vm[j] >= thr);
+                while (hitters) {
+                    const int from = __ffs(hitters) - 1;
+                    hitters &= hitters - 1;
+                    if (lane < N) {
+                        const int pos_in_tile = (j * kThreads + (tid - lane) + from) * N + lane;
+                        const int idx = s0 + t * TE + pos_in_tile;
+                        const float xv = Elem<DT>::load1(tile + pos_in_tile);
+                        if (xv >= thr && xv > -CUDART_INF_F && idx < s1) {
+                            const int pos = atomicAdd(&ctl.cnt[l], 1);
+                            if (pos < kListCap) sm.cand[l * kListCap + pos] = make_key(xv, idx);
                         }
                     }
                 }
@@ -389,18 +394,16 @@ __device__ void scan_slice_stream(const DT *__restrict__ row, int s0, int s1, in
                 }
             }
         }
-        if (t == fold_tile) {
-            // fold point: the list this warp appended to is complete; switch to the other list,
-            // which the producer warp emptied when it served the previous point
-            if (fold >= 1 && !mbar_wait(&bars.folded, (fold - 1) & 1, abort)) ctl.timed_out = 1;
-            __syncwarp();
-            if (lane == 0) mbar_arrive(&bars.listed);
-            ++fold;
-            fold_tile = min(next_fold_tile(fold_tile), ntiles - 1);
-        }
+        // this warp's candidates of tile t are complete; the list of the next tile must have
+        // been folded (emptied) since it was last used, kLists tiles earlier
+        if (t + 1 < ntiles && t + 1 >= kLists &&
+            !mbar_wait(&bars.folded[(t + 1) % kLists], ((t + 1 - kLists) / kLists) & 1, abort))
+            ctl.timed_out = 1;
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&bars.listed[t % kLists]);
     }
     // the last fold leaves the slice's best keys, sorted, in sm.sel
-    if (!mbar_wait(&bars.folded, (fold - 1) & 1, abort)) ctl.timed_out = 1;
+    if (!mbar_wait(&bars.folded[(ntiles - 1) % kLists], ((ntiles - 1) / kLists) & 1, abort)) ctl.timed_out = 1;
     const int nsel = min(ctl.nsel, K);
     if (tid < nsel) sm.cand[tid] = sm.sel[tid];
     if (tid == 0) sm.cnt = nsel;

@@ -216,9 +216,8 @@ __global__ void __launch_bounds__(kStreamThreads, 3) target_stream_kernel(const 
     const int s1 = min(a.V, s0 + a.slice_elems);
     const bool sums = !a.all_greedy && a.mode[b] != 0;
     stream_begin(sm, ctl, bars);
-    if (tid >= kThreads) {                                  // producer warp: copies + top-K folds
-        stream_service(reinterpret_cast<const char *>(rowp + s0), (s1 - s0) * (int)sizeof(DT), 1, sm, ctl,
-                       ring, bars);
+    if (tid >= kThreads) {                                  // fold warp: running top-K
+        stream_service((s1 - s0) * (int)sizeof(DT), 1, sm, ctl, bars);
         return;
     }
     float c;
