@@ -1,14 +1,21 @@
 // dsp_cps_search: causal-consistency path search (Sec. 3.2 "Scoring and search", Eq. 8).
 //
-// One CTA per batch row walks the lattice left to right.  At each depth the (live beams x
-// candidates) expansions are scored in fp32 in a fixed operation order, ranked under
-// (cum desc, token id asc, parent rank asc) by counting, and the best W survive with
-// back-pointers kept in shared memory; paths are rebuilt by walking the back-pointers.
+// One CTA per batch row walks the lattice left to right.  The step score of a candidate,
+//   step = fl( fl(lambda * (x - x_top1)) + fl((1 - lambda) * l^ng(prev, cur)) ),
+// depends on the previous position's candidate slot and on its own slot but not on the beam, so
+// for a window of depths all (depth, previous slot, slot) steps are gathered and computed in
+// parallel before the depths of the window are walked; the sequential part of a depth is then
+// one shared-memory read and one fp32 add per expansion and the selection of the best W.
+// Expansions become unique 64-bit keys (cum | token-id rank | parent rank | slot) whose integer
+// order is the beam order (cum desc, token id asc, parent rank asc); every warp sorts 32 keys
+// with a bitonic network and the warps' lists are merged pairwise through shared memory.
+// Back-pointers stay in shared memory; paths are rebuilt by walking them.
 #include "dsp_common.cuh"
 
 namespace dsp {
 
-constexpr int kMaxExp = DSP_MAX_W * (DSP_MAX_K + 1);
+constexpr int kMaxKC = DSP_MAX_K + 1;
+constexpr int kStepBudgetBytes = 48 * 1024;        // shared memory for one window of step scores
 
 struct CpsArgs {
     const int32_t *cand_id;
@@ -30,7 +37,23 @@ struct CpsArgs {
     int32_t *beam_ids;
     float *beam_score, *beam_cum;
     uint32_t *row_status;
+    int D;                       // depths per window
 };
+
+// Depths per window and dynamic shared memory of a launch.
+inline int cps_window_depths(int L, int KC) {
+    int d = kStepBudgetBytes / (KC * KC * 4);
+    if (d < 1) d = 1;
+    return d < L ? d : L;
+}
+inline size_t cps_smem_bytes(int L, int W, int KC, int D) {
+    size_t o = align_up((size_t)2 * L * W, 16);                 // back-pointers
+    o += (size_t)D * KC * KC * 4;                               // step scores
+    o += (size_t)D * KC * 4;                                    // candidate ids
+    o += align_up((size_t)D * KC, 4);                           // token-id ranks
+    o += (size_t)D * 4;                                         // candidate counts
+    return o;
+}
 
 __device__ __forceinline__ float proxy_score(const CpsArgs &a, int prev, int cur) {
     if (a.proxy_kind == 1) return __ldg(&a.table[(long long)prev * a.V + cur]);
@@ -43,73 +66,139 @@ __device__ __forceinline__ float proxy_score(const CpsArgs &a, int prev, int cur
     return __ldg(&a.table[h >> (32 - a.table_log2)]);
 }
 
-__global__ void __launch_bounds__(kThreads) cps_kernel(const CpsArgs a) {
-    extern __shared__ unsigned char bp[];              // [L][W] parent rank, then [L][W] slot
-    __shared__ float ecum[kMaxExp];
-    __shared__ int etok[kMaxExp];
-    __shared__ float bcum[2][DSP_MAX_W];
-    __shared__ int btok[2][DSP_MAX_W];
-    __shared__ int cid[DSP_MAX_K + 1];
-    __shared__ float clg[DSP_MAX_K + 1];
+__device__ __forceinline__ unsigned long long kmax(unsigned long long a, unsigned long long b) { return a > b ? a : b; }
+__device__ __forceinline__ unsigned long long kmin(unsigned long long a, unsigned long long b) { return a < b ? a : b; }
 
-    const int tid = threadIdx.x;
+// Sort 32 keys, one per lane, descending over the lanes (bitonic network).
+__device__ __forceinline__ unsigned long long sort_keys_desc(unsigned long long v, int lane) {
+#pragma unroll
+    for (int k = 2; k <= 32; k <<= 1) {
+#pragma unroll
+        for (int j = k >> 1; j > 0; j >>= 1) {
+            const unsigned long long o = __shfl_xor_sync(0xFFFFFFFFu, v, j);
+            const bool up = (lane & k) == 0;
+            const bool lower = (lane & j) == 0;
+            v = (lower == up) ? kmax(v, o) : kmin(v, o);
+        }
+    }
+    return v;
+}
+// Best 32 of this warp's descending list `a` and another descending list given reversed
+// (`b_rev` = the other list's key of lane 31 - lane), descending: the lane-wise maximum is
+// bitonic and holds the best 32; five compare-exchange stages sort it.
+__device__ __forceinline__ unsigned long long merge_keys(unsigned long long a, unsigned long long b_rev, int lane) {
+    unsigned long long v = kmax(a, b_rev);
+#pragma unroll
+    for (int j = 16; j > 0; j >>= 1) {
+        const unsigned long long o = __shfl_xor_sync(0xFFFFFFFFu, v, j);
+        v = (lane & j) == 0 ? kmax(v, o) : kmin(v, o);
+    }
+    return v;
+}
+
+__global__ void __launch_bounds__(kThreads) cps_kernel(const CpsArgs a) {
+    extern __shared__ __align__(16) unsigned char dyn[];
+    __shared__ unsigned long long xch[kWarps][32];     // sorted keys of each warp, for the merges
+    __shared__ float bcum[2][DSP_MAX_W];
+    __shared__ int bslot[2][DSP_MAX_W];                // slot of each beam's last token
+    __shared__ int s_top_tok;                          // token of the rank-0 survivor
+
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int b = blockIdx.x;
-    const int L = a.L, W = a.W, KC = a.KC;
-    unsigned char *bp_parent = bp;
-    unsigned char *bp_slot = bp + (size_t)L * W;
+    const int L = a.L, W = a.W, KC = a.KC, D = a.D;
+    unsigned char *bp_parent = dyn;
+    unsigned char *bp_slot = dyn + (size_t)L * W;
+    float *step = reinterpret_cast<float *>(dyn + align_up((size_t)2 * L * W, 16));
+    int *cid = reinterpret_cast<int *>(step + (size_t)D * KC * KC);
+    unsigned char *trank = reinterpret_cast<unsigned char *>(cid + (size_t)D * KC);
+    int *ccnt = reinterpret_cast<int *>(trank + align_up((size_t)D * KC, 4));
     const float lam = a.lambda;
     const float oml = __fsub_rn(1.0f, lam);
+    const long long row0 = (long long)b * L;
 
     int live = 1, cur = 0, m = L;
     bool stopped = false;
-    if (tid == 0) bcum[0][0] = 0.f;
-    __syncthreads();
+    if (tid == 0) { bcum[0][0] = 0.f; bslot[0][0] = 0; }
 
-    for (int i = 0; i < L; ++i) {
-        const long long r = (long long)b * L + i;
-        int cnt = a.cand_count[r];
-        cnt = max(0, min(cnt, KC));
-        if (tid < cnt) {
-            cid[tid] = a.cand_id[r * KC + tid];
-            clg[tid] = a.cand_logit[r * KC + tid];
-        }
+    for (int i0 = 0; i0 < L && m == L && !stopped; i0 += D) {
+        const int nd = min(D, L - i0);
+        // ---- window set-up: ids and counts, then step scores and token-id ranks, in parallel ----
         __syncthreads();
-        const int n = live * cnt;
-        if (n == 0) { m = i; break; }                   // an empty position ends the lattice
-        const float top1 = clg[0];
-        for (int e = tid; e < n; e += kThreads) {
-            const int w = e / cnt, k = e - w * cnt;
-            const int tok = cid[k];
-            const float g = __fsub_rn(clg[k], top1);
-            const int prev = i == 0 ? a.prev_token[b] : btok[cur][w];
-            const float ng = proxy_score(a, prev, tok);
-            const float step = __fadd_rn(__fmul_rn(lam, g), __fmul_rn(oml, ng));
-            ecum[e] = __fadd_rn(bcum[cur][w], step);
-            etok[e] = tok;
-        }
+        for (int x = tid; x < nd; x += kThreads) ccnt[x] = max(0, min(a.cand_count[row0 + i0 + x], KC));
+        for (int x = tid; x < nd * KC; x += kThreads) cid[x] = a.cand_id[(row0 + i0) * KC + x];
         __syncthreads();
-        const int nxt = cur ^ 1;
-        for (int e = tid; e < n; e += kThreads) {
-            const float s = ecum[e];
-            const int tok = etok[e];
-            int rank = 0;
-            for (int f = 0; f < n; ++f) {
-                const float sf = ecum[f];
-                const int tf = etok[f];
-                rank += (sf > s) || (sf == s && (tf < tok || (tf == tok && f < e)));
-            }
-            if (rank < W) {
-                const int w = e / cnt;
-                bcum[nxt][rank] = s;
-                btok[nxt][rank] = tok;
-                bp_parent[(size_t)i * W + rank] = (unsigned char)w;
-                bp_slot[(size_t)i * W + rank] = (unsigned char)(e - w * cnt);
+        for (int x = tid; x < nd * KC * KC; x += kThreads) {
+            const int d = x / (KC * KC), rem = x - d * KC * KC;
+            const int p = rem / KC, k = rem - p * KC;
+            const int i = i0 + d;
+            const int pc = i == 0 ? 1 : (d > 0 ? ccnt[d - 1] : max(0, min(a.cand_count[row0 + i - 1], KC)));
+            if (k < ccnt[d] && p < pc) {
+                const int prev = i == 0 ? a.prev_token[b]
+                                        : (d > 0 ? cid[(d - 1) * KC + p] : a.cand_id[(row0 + i - 1) * KC + p]);
+                const float *lg = a.cand_logit + (row0 + i) * KC;
+                const float g = __fsub_rn(lg[k], lg[0]);
+                const float ng = proxy_score(a, prev, cid[d * KC + k]);
+                step[x] = __fadd_rn(__fmul_rn(lam, g), __fmul_rn(oml, ng));
             }
         }
+        for (int x = tid; x < nd * KC; x += kThreads) {
+            const int d = x / KC, k = x - d * KC;
+            int r = 0;
+            if (k < ccnt[d]) {
+                const int tok = cid[x];
+                for (int q = 0; q < ccnt[d]; ++q) r += cid[d * KC + q] < tok;
+            }
+            trank[x] = (unsigned char)r;
+        }
         __syncthreads();
-        live = min(W, n);
-        cur = nxt;
-        if (a.eos_id >= 0 && btok[cur][0] == a.eos_id) { m = i + 1; stopped = true; break; }
+
+        // ---- the depths of the window, one after the other ----
+        for (int d = 0; d < nd; ++d) {
+            const int i = i0 + d;
+            const int cnt = ccnt[d];
+            const int n = live * cnt;
+            if (n == 0) { m = i; break; }               // an empty position ends the lattice
+            // every warp: its expansions, 32 at a time, sorted and merged into `best`
+            unsigned long long best = 0ull;
+            for (int base = warp * 32; base < n; base += kThreads) {
+                const int e = base + lane;
+                unsigned long long key = 0ull;
+                if (e < n) {
+                    const int w = e / cnt, k = e - w * cnt;
+                    const float cum = __fadd_rn(bcum[cur][w], step[(d * KC + bslot[cur][w]) * KC + k]);
+                    key = ((unsigned long long)ord_bits(cum) << 32) |
+                          ((unsigned long long)(255 - trank[d * KC + k]) << 24) |
+                          ((unsigned long long)(255 - w) << 16) | ((unsigned long long)(255 - k) << 8) | 1ull;
+                }
+                const unsigned long long sorted = sort_keys_desc(key, lane);
+                best = base < kThreads ? sorted : merge_keys(best, __shfl_sync(0xFFFFFFFFu, sorted, 31 - lane), lane);
+            }
+            // pairwise merges of the warps' lists (only as many levels as n needs)
+#pragma unroll
+            for (int span = 1; span < kWarps; span <<= 1) {
+                if (n > 32 * span) {
+                    xch[warp][lane] = best;
+                    __syncthreads();
+                    if ((warp & (2 * span - 1)) == 0) best = merge_keys(best, xch[warp + span][31 - lane], lane);
+                    __syncthreads();
+                }
+            }
+            // warp 0 holds the best min(32, n) expansions: the first min(W, n) survive
+            const int keep = min(W, n);
+            const int nxt = cur ^ 1;
+            if (warp == 0 && lane < keep) {
+                const int w = 255 - (int)((best >> 16) & 0xFF), k = 255 - (int)((best >> 8) & 0xFF);
+                bcum[nxt][lane] = __fadd_rn(bcum[cur][w], step[(d * KC + bslot[cur][w]) * KC + k]);
+                bslot[nxt][lane] = k;
+                bp_parent[(size_t)i * W + lane] = (unsigned char)w;
+                bp_slot[(size_t)i * W + lane] = (unsigned char)k;
+                if (lane == 0) s_top_tok = cid[d * KC + k];
+            }
+            __syncthreads();
+            live = keep;
+            cur = nxt;
+            if (a.eos_id >= 0 && s_top_tok == a.eos_id) { m = i + 1; stopped = true; break; }
+        }
     }
     __syncthreads();
 
@@ -188,12 +277,19 @@ extern "C" int32_t dsp_cps_search(const int32_t *cand_id, const float *cand_logi
     a.path = path; a.path_slot = path_slot; a.path_len = path_len; a.path_score = path_score;
     a.beam_ids = beam_ids; a.beam_score = beam_score; a.beam_cum = beam_cum;
     a.row_status = row_status;
-    const size_t dyn = (size_t)L * W * 2;
-    static bool attr_set = false;
-    if (!attr_set) {
-        DSP_CUDA_TRY(cudaFuncSetAttribute(cps_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                          DSP_MAX_L * DSP_MAX_W * 2));
-        attr_set = true;
+    a.D = cps_window_depths(L, KC);
+    const size_t dyn = cps_smem_bytes(L, W, KC, a.D);
+    {
+        // raise the kernel's dynamic shared memory limit once per device (the attribute is per device)
+        static bool done[64] = {};
+        int dev = 0;
+        DSP_CUDA_TRY(cudaGetDevice(&dev));
+        if (dev < 0 || dev >= 64 || !done[dev]) {
+            DSP_CUDA_TRY(cudaFuncSetAttribute(
+                cps_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                (int)cps_smem_bytes(DSP_MAX_L, DSP_MAX_W, kMaxKC, cps_window_depths(DSP_MAX_L, kMaxKC))));
+            if (dev >= 0 && dev < 64) done[dev] = true;
+        }
     }
     cps_kernel<<<B, kThreads, dyn, reinterpret_cast<cudaStream_t>(stream)>>>(a);
     DSP_CUDA_TRY(cudaGetLastError());

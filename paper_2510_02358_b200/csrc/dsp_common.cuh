@@ -34,7 +34,7 @@ inline int32_t cuda_fail(cudaError_t e) {
         if (e__ != cudaSuccess) return ::dsp::cuda_fail(e__); \
     } while (0)
 
-inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+__host__ __device__ inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 // ---- order-preserving 64-bit keys: larger key = better under (logit desc, id asc) ----
 __device__ __forceinline__ uint32_t ord_bits(float x) {
