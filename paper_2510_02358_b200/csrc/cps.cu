@@ -9,7 +9,8 @@
 // Expansions become unique 64-bit keys (cum | token-id rank | parent rank | slot) whose integer
 // order is the beam order (cum desc, token id asc, parent rank asc); every warp sorts 32 keys
 // with a bitonic network and the warps' lists are merged pairwise through shared memory.
-// Back-pointers stay in shared memory; paths are rebuilt by walking them.
+// Back-pointers stay in shared memory; each surviving beam's slots are recovered by walking them
+// and the token ids are then fetched by all threads at once.
 #include "dsp_common.cuh"
 
 namespace dsp {
@@ -47,7 +48,7 @@ inline int cps_window_depths(int L, int KC) {
     return d < L ? d : L;
 }
 inline size_t cps_smem_bytes(int L, int W, int KC, int D) {
-    size_t o = align_up((size_t)2 * L * W, 16);                 // back-pointers
+    size_t o = align_up((size_t)3 * L * W, 16);                 // back-pointers and walked slots
     o += (size_t)D * KC * KC * 4;                               // step scores
     o += (size_t)D * KC * 4;                                    // candidate ids
     o += align_up((size_t)D * KC, 4);                           // token-id ranks
@@ -98,7 +99,7 @@ __device__ __forceinline__ unsigned long long merge_keys(unsigned long long a, u
 
 __global__ void __launch_bounds__(kThreads) cps_kernel(const CpsArgs a) {
     extern __shared__ __align__(16) unsigned char dyn[];
-    __shared__ unsigned long long xch[kWarps][32];     // sorted keys of each warp, for the merges
+    __shared__ unsigned long long xch[2][kWarps][32];  // sorted keys of each warp, for the merges (two buffers in turn)
     __shared__ float bcum[2][DSP_MAX_W];
     __shared__ int bslot[2][DSP_MAX_W];                // slot of each beam's last token
     __shared__ int s_top_tok;                          // token of the rank-0 survivor
@@ -108,7 +109,8 @@ __global__ void __launch_bounds__(kThreads) cps_kernel(const CpsArgs a) {
     const int L = a.L, W = a.W, KC = a.KC, D = a.D;
     unsigned char *bp_parent = dyn;
     unsigned char *bp_slot = dyn + (size_t)L * W;
-    float *step = reinterpret_cast<float *>(dyn + align_up((size_t)2 * L * W, 16));
+    unsigned char *walk = dyn + (size_t)2 * L * W;     // slot of beam w at depth i, after the walk
+    float *step = reinterpret_cast<float *>(dyn + align_up((size_t)3 * L * W, 16));
     int *cid = reinterpret_cast<int *>(step + (size_t)D * KC * KC);
     unsigned char *trank = reinterpret_cast<unsigned char *>(cid + (size_t)D * KC);
     int *ccnt = reinterpret_cast<int *>(trank + align_up((size_t)D * KC, 4));
@@ -174,13 +176,14 @@ __global__ void __launch_bounds__(kThreads) cps_kernel(const CpsArgs a) {
                 best = base < kThreads ? sorted : merge_keys(best, __shfl_sync(0xFFFFFFFFu, sorted, 31 - lane), lane);
             }
             // pairwise merges of the warps' lists (only as many levels as n needs)
+            int buf = 0;
 #pragma unroll
             for (int span = 1; span < kWarps; span <<= 1) {
                 if (n > 32 * span) {
-                    xch[warp][lane] = best;
+                    xch[buf][warp][lane] = best;
                     __syncthreads();
-                    if ((warp & (2 * span - 1)) == 0) best = merge_keys(best, xch[warp + span][31 - lane], lane);
-                    __syncthreads();
+                    if ((warp & (2 * span - 1)) == 0) best = merge_keys(best, xch[buf][warp + span][31 - lane], lane);
+                    buf ^= 1;                           // the next level writes the other buffer
                 }
             }
             // warp 0 holds the best min(32, n) expansions: the first min(W, n) survive
@@ -202,40 +205,51 @@ __global__ void __launch_bounds__(kThreads) cps_kernel(const CpsArgs a) {
     }
     __syncthreads();
 
-    // common term of Eq. 8 dropped from the ranking: lambda * sum_i (lse_i - x_top1,i)
+    // ---- outputs ----
+    // common term of Eq. 8 dropped from the ranking: lambda * sum_i (lse_i - x_top1,i), in double
+    __shared__ double s_off[kWarps];
     double off = 0.0;
-    for (int i = 0; i < m; ++i) {
-        const long long r = (long long)b * L + i;
-        off += a.lse64[r] - (double)a.cand_logit[r * KC];
+    for (int i = tid; i < m; i += kThreads) off += a.lse64[row0 + i] - (double)a.cand_logit[(row0 + i) * KC];
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) off += __shfl_xor_sync(0xFFFFFFFFu, off, o);
+    if (lane == 0) s_off[warp] = off;
+    // walk the back-pointers (shared memory only), one thread per surviving beam
+    const int nlive = m > 0 ? live : 0;
+    if (tid < nlive) {
+        int at = tid;
+        for (int i = m - 1; i >= 0; --i) {
+            walk[(size_t)i * W + tid] = bp_slot[(size_t)i * W + at];
+            at = bp_parent[(size_t)i * W + at];
+        }
+    }
+    __syncthreads();
+    off = 0.0;
+#pragma unroll
+    for (int w = 0; w < kWarps; ++w) off += s_off[w];
+    // token ids of every beam: all threads, independent loads
+    for (int x = tid; x < W * L; x += kThreads) {
+        const int w = x / L, i = x - w * L;
+        int id = -1, slot = -1;
+        if (w < nlive && i < m) {
+            slot = walk[(size_t)i * W + w];
+            id = a.cand_id[(row0 + i) * KC + slot];
+        }
+        if (a.beam_ids) a.beam_ids[((long long)b * W + w) * L + i] = id;
+        if (w == 0) {
+            a.path[row0 + i] = id;
+            a.path_slot[row0 + i] = slot;
+        }
     }
     if (tid < W) {
         const int w = tid;
-        const bool alive = w < live && m > 0;
         float score = -CUDART_INF_F, cumv = -CUDART_INF_F;
-        if (alive) {
+        if (w < nlive) {
             cumv = bcum[cur][w];
             score = (float)((double)cumv - (double)lam * off);
-            int at = w;
-            for (int i = m - 1; i >= 0; --i) {
-                const int slot = bp_slot[(size_t)i * W + at];
-                const int id = a.cand_id[((long long)b * L + i) * KC + slot];
-                if (a.beam_ids) a.beam_ids[((long long)b * W + w) * L + i] = id;
-                if (w == 0) {
-                    a.path[(long long)b * L + i] = id;
-                    a.path_slot[(long long)b * L + i] = slot;
-                }
-                at = bp_parent[(size_t)i * W + at];
-            }
         }
-        if (a.beam_ids)
-            for (int i = alive ? m : 0; i < L; ++i) a.beam_ids[((long long)b * W + w) * L + i] = -1;
         if (a.beam_score) a.beam_score[(long long)b * W + w] = score;
         if (a.beam_cum) a.beam_cum[(long long)b * W + w] = cumv;
         if (w == 0) {
-            for (int i = m; i < L; ++i) {
-                a.path[(long long)b * L + i] = -1;
-                a.path_slot[(long long)b * L + i] = -1;
-            }
             a.path_len[b] = m;
             a.path_score[b] = score;
             if (a.row_status && stopped) atomicOr(&a.row_status[b], DSP_ROW_EOS_STOPPED);
