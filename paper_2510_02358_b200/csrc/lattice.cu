@@ -184,32 +184,25 @@ __global__ void __launch_bounds__(kThreads, 4) lattice_kernel(const LatticeArgs 
     lattice_finish<DT, SyncAll>(a, sm, row, slice, b, rowp, c, S, T, 0u);
 }
 
-// Streaming kernel for 16-byte aligned layouts: the slice streams through a shared-memory
-// ring of bulk asynchronous copies, the consumers scan the ring and a ninth warp keeps the
-// running top-K (see stream_core.cuh).
+// Streaming kernel for 16-byte aligned layouts: the slice streams through a shared-memory ring
+// of bulk asynchronous copies and the top-K is selected from a table of per-thread tile maxima
+// once the slice has been read (see stream_core.cuh).
 template <typename DT>
-__global__ void __launch_bounds__(kStreamThreads, 3) lattice_stream_kernel(const LatticeArgs a) {
-    extern __shared__ __align__(128) unsigned char ring[];
+__global__ void __launch_bounds__(kThreads, 3) lattice_stream_kernel(const LatticeArgs a) {
+    extern __shared__ __align__(128) unsigned char dyn[];
     __shared__ ScanSmem sm;
     __shared__ StreamBars bars;
-    __shared__ StreamCtl ctl;
-    const int tid = threadIdx.x;
     const long long row = blockIdx.x / a.nslices;
     const int slice = blockIdx.x - (int)(row * a.nslices);
     const int b = (int)(row / a.L), l = (int)(row - (long long)b * a.L);
     const DT *rowp = reinterpret_cast<const DT *>(a.logits) + b * a.stride_b + l * a.stride_l;
     const int s0 = slice * a.slice_elems;
     const int s1 = min(a.V, s0 + a.slice_elems);
-    stream_begin(sm, ctl, bars);
-    if (tid >= kThreads) {                                  // fold warp: running top-K
-        stream_service((s1 - s0) * (int)sizeof(DT), a.K, sm, ctl, bars);
-        return;
-    }
+    stream_begin(sm, bars);
     float c;
     double S, T;
-    scan_slice_stream<DT, true>(rowp, s0, s1, a.K, sm, ctl, ring, bars, c, S, T);
-    lattice_finish<DT, SyncConsumers>(a, sm, row, slice, b, rowp, c, S, T,
-                                      ctl.timed_out ? DSP_ROW_TIMEOUT : 0u);
+    scan_slice_stream<DT, true>(rowp, s0, s1, a.K, sm, bars, dyn, reinterpret_cast<DT *>(dyn + kRingBytes), c, S, T);
+    lattice_finish<DT, SyncAll>(a, sm, row, slice, b, rowp, c, S, T, bars.timed_out ? DSP_ROW_TIMEOUT : 0u);
 }
 
 template <typename DT>
@@ -229,10 +222,10 @@ static int32_t launch_lattice(LatticeArgs &a, void *workspace, size_t workspace_
     DSP_CUDA_TRY(cudaMemsetAsync(ws, 0, w.zero_bytes, st));
     const long long nblocks = nrows * a.nslices;
     if (nblocks > 0x7FFFFFFFLL) return DSP_ERR_UNSUPPORTED;
-    if (stream_layout_ok(a.logits, sizeof(DT), a.V, a.stride_b, a.stride_l)) {
+    if (stream_layout_ok<DT>(a.logits, a.V, a.stride_b, a.stride_l, a.slice_elems)) {
         static RingSmemDone smem_done;                       // one per element type
         DSP_CUDA_TRY(allow_ring_smem(lattice_stream_kernel<DT>, smem_done));
-        lattice_stream_kernel<DT><<<(unsigned)nblocks, kStreamThreads, kRingBytes, st>>>(a);
+        lattice_stream_kernel<DT><<<(unsigned)nblocks, kThreads, kStreamDynBytes, st>>>(a);
     } else {
         lattice_kernel<DT><<<(unsigned)nblocks, kThreads, 0, st>>>(a);
     }

@@ -360,7 +360,8 @@ inline SlicePlan plan_slices(int64_t nrows, int V, int target_ctas) {
     int want = (int)((target_ctas + nrows - 1) / (nrows > 0 ? nrows : 1));   // slices per row wanted
     if (want < 1) want = 1;
     int tps = (ntiles + want - 1) / want;            // tiles per slice
-    if (tps > 32) tps = 32;                          // bounds the time one CTA holds its SM slot
+    const int cap = 64 / (int)sizeof(DT);            // tiles per slice the streaming kernels' table of tile maxima holds
+    if (tps > cap) tps = cap;
     const int min_tps = (ntiles + kMaxSlices - 1) / kMaxSlices;
     if (tps < min_tps) tps = min_tps;
     if (tps < 1) tps = 1;

@@ -1,14 +1,16 @@
 // TMA-fed variant of the one-pass slice scan for rows whose start, strides and length are
 // multiples of 16 bytes.  The slice streams through a ring of shared-memory stages by bulk
 // asynchronous copies (cp.async.bulk, completion counted on an mbarrier per stage, no
-// multicast) that one consumer thread issues three tiles ahead; the kThreads consumer threads
-// read each stage with one 128-bit shared load per vector and do the arithmetic from registers.
-// Logits at or above the current threshold are appended to the candidate list of their tile
-// (four lists in rotation).  A ninth warp, the fold warp, folds each tile's list into
-// a register-resident sorted top-K and publishes a tighter threshold that the consumers pick
-// up at their next tile.  The two sides hand over through mbarriers with time-bounded waits,
-// so the consumers meet no block-wide barrier after the first tile's threshold bootstrap.  Results are the same as scan_slice's
-// (scan_core.cuh): log-sum-exp terms and the exact top-K.
+// multicast) that one thread issues two tiles ahead; all kThreads threads read each stage with
+// one 128-bit shared load per vector and do the arithmetic from registers.
+//
+// The streaming loop has no block-wide barrier and does nothing for the top-K except to keep,
+// per thread and tile, the largest of the thread's kVpt vectors of that tile in a shared-memory
+// table.  The exact top-K is selected from that table when the slice has been streamed: a
+// threshold with at least K table entries at or above it, the exact K-th largest entry among
+// those, and a second look (from global memory, L2 hits) at the few (tile, thread) shares whose
+// maximum reaches it.  Results are the same as scan_slice's (scan_core.cuh): log-sum-exp terms
+// and the exact top-K.
 #pragma once
 
 #include "scan_core.cuh"
@@ -16,10 +18,15 @@
 namespace dsp {
 
 constexpr int kTileBytes = kThreads * kVpt * 16;     // one ring stage = one tile of either dtype
-constexpr int kStages = 4;
-constexpr int kStreamThreads = kThreads + 32;        // consumers + the fold warp
+constexpr int kStages = 3;
 constexpr int kRingBytes = kStages * kTileBytes;
+constexpr int kMaxTableBytes = 16384;                // table of per-thread tile maxima
 constexpr long long kWaitCycles = 400000000LL;       // every wait gives up after this many SM clocks (~0.2 s)
+
+// Tiles per slice the table has room for: 32 for bf16 rows, 16 for fp32 rows.
+template <typename DT> constexpr int max_stream_tiles() { return kMaxTableBytes / (kThreads * (int)sizeof(DT)); }
+static_assert(max_stream_tiles<float>() == 64 / 4 && max_stream_tiles<__nv_bfloat16>() == 64 / 2,
+              "plan_slices caps the tiles per slice at 64 / sizeof(element)");
 
 __device__ __forceinline__ uint32_t smem_addr(const void *p) {
     return (uint32_t)__cvta_generic_to_shared(p);
@@ -57,20 +64,6 @@ __device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, volati
         if (*abort || clock64() - t0 > kWaitCycles) return false;
     }
 }
-// Non-blocking test of a phase.
-__device__ __forceinline__ bool mbar_test(uint64_t *bar, uint32_t parity) {
-    uint32_t ok;
-    asm volatile(
-        "{\n"
-        ".reg .pred p;\n"
-        "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n"
-        "selp.u32 %0, 1, 0, p;\n"
-        "}"
-        : "=r"(ok)
-        : "r"(smem_addr(bar)), "r"(parity)
-        : "memory");
-    return ok != 0;
-}
 // Bulk copy global -> this CTA's shared memory; both addresses and the size are multiples of 16.
 __device__ __forceinline__ void bulk_load(void *dst, const void *src, uint32_t bytes, uint64_t *bar) {
     asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
@@ -83,119 +76,56 @@ __device__ __forceinline__ float max3(float a, float b, float c) {
     return d;
 }
 
+// Shared state of a streaming kernel besides ScanSmem.
 struct StreamBars {
     uint64_t full[kStages];      // stage filled by its bulk copy
-    uint64_t empty[kStages];     // stage released by all consumer warps
-    uint64_t listed[4];          // list l, phase n: every consumer warp is past tile 4n + l
-    uint64_t folded[4];          // list l, phase n: the fold warp has folded tile 4n + l's candidates
+    uint64_t empty[kStages];     // stage released by all warps
+    int timed_out;               // non-zero once a bounded wait gave up
+    int cnt2;                    // entries of the second list of the selection
 };
+// Dynamic shared memory: the ring first (16-byte aligned), then the table of tile maxima.
+constexpr int kStreamDynBytes = kRingBytes + kMaxTableBytes;
 
-// The candidates of tile t go to list t % kLists; the list is folded after the tile and must be
-// empty again before tile t + kLists, which leaves the fold warp three tiles of slack.
-constexpr int kLists = 4;
-constexpr int kListCap = kCandCap / kLists;
-static_assert(kLists == 4, "StreamBars holds four barriers of each kind");
-
-// Shared state of one slice scan besides ScanSmem.
-struct StreamCtl {
-    int cnt[kLists];     // entries appended to each candidate list (may exceed kListCap: overflow)
-    int nsel;            // keys the fold warp left in ScanSmem::sel after the last fold
-    int timed_out;       // non-zero once a bounded wait gave up
-};
-
-// Called by every thread before produce/consume start (ends with a CTA-wide barrier).
-__device__ __forceinline__ void stream_begin(ScanSmem &sm, StreamCtl &ctl, StreamBars &bars) {
+// Called by every thread before the scan starts (ends with a CTA-wide barrier).
+__device__ __forceinline__ void stream_begin(ScanSmem &sm, StreamBars &bars) {
     if (threadIdx.x == 0) {
         for (int s = 0; s < kStages; ++s) {
             mbar_init(&bars.full[s], 1);
             mbar_init(&bars.empty[s], kWarps);
         }
-        for (int l = 0; l < kLists; ++l) {
-            mbar_init(&bars.listed[l], kWarps);
-            mbar_init(&bars.folded[l], 1);
-            ctl.cnt[l] = 0;
-        }
         mbar_init_fence();
         sm.cnt = 0; sm.thrkey = 0ull; sm.thr_v = -CUDART_INF_F; sm.overflow = 0;
-        ctl.nsel = 0; ctl.timed_out = 0;
+        bars.timed_out = 0; bars.cnt2 = 0;
     }
     __syncthreads();
 }
 
-__device__ __forceinline__ unsigned long long umax64(unsigned long long a, unsigned long long b) { return a > b ? a : b; }
-__device__ __forceinline__ unsigned long long umin64(unsigned long long a, unsigned long long b) { return a < b ? a : b; }
-
-// Sort 32 keys, one per lane, descending over the lanes (bitonic network).
-__device__ __forceinline__ unsigned long long sort32_desc(unsigned long long v, int lane) {
-#pragma unroll
-    for (int k = 2; k <= 32; k <<= 1) {
-#pragma unroll
-        for (int j = k >> 1; j > 0; j >>= 1) {
-            const unsigned long long o = __shfl_xor_sync(0xFFFFFFFFu, v, j);
-            const bool up = (lane & k) == 0;
-            const bool lower = (lane & j) == 0;
-            v = (lower == up) ? umax64(v, o) : umin64(v, o);
-        }
-    }
-    return v;
+// Issue the bulk copy of tile t of the slice at `src` into its ring stage (one thread).
+__device__ __forceinline__ void issue_tile(const char *src, int nbytes, int t, unsigned char *ring,
+                                           StreamBars &bars) {
+    const int s = t % kStages;
+    const uint32_t bytes = (uint32_t)min(kTileBytes, nbytes - t * kTileBytes);
+    mbar_expect_tx(&bars.full[s], bytes);
+    bulk_load(ring + (size_t)s * kTileBytes, src + (size_t)t * kTileBytes, bytes, &bars.full[s]);
 }
 
-// Best 32 of two descending 32-key lists (one key per lane each), descending: the lane-wise
-// maximum of one list and the other reversed is bitonic and holds the best 32; five
-// compare-exchange stages sort it.
-__device__ __forceinline__ unsigned long long merge_top32(unsigned long long a, unsigned long long b, int lane) {
-    unsigned long long v = umax64(a, __shfl_sync(0xFFFFFFFFu, b, 31 - lane));
-#pragma unroll
-    for (int j = 16; j > 0; j >>= 1) {
-        const unsigned long long o = __shfl_xor_sync(0xFFFFFFFFu, v, j);
-        v = (lane & j) == 0 ? umax64(v, o) : umin64(v, o);
-    }
-    return v;
-}
+// Padding for the vectors past the end of a ragged last tile: -2^124, below every finite
+// logit the interface allows, finite when scaled by log2(e), never a candidate (its index is
+// past the row).
+template <typename DT> struct Pad;
+template <> struct Pad<__nv_bfloat16> { static constexpr uint32_t kWord = 0xFD80FD80u; };
+template <> struct Pad<float> { static constexpr uint32_t kWord = 0xFD800000u; };
 
-// Fold candidate list `which` into the warp's sorted top-32 (one key per lane in `mykey`,
-// descending, 0 = empty slot below every real key).  A batch of 32 keys is read at once and
-// those that do not beat the K-th key are dropped by one ballot; a few survivors are inserted
-// one by one (ballot, shuffle-up, select), many are sorted and merged in.  Empties the list and
-// publishes the K-th key's value as the new threshold.  Whole warp.
-__device__ __forceinline__ void fold_list(ScanSmem &sm, StreamCtl &ctl, int which, int K,
-                                          unsigned long long &mykey) {
-    const int lane = threadIdx.x & 31;
-    const unsigned long long *list = sm.cand + which * kListCap;
-    const int total = ctl.cnt[which];
-    const int n = min(total, kListCap);
-    unsigned long long kth = __shfl_sync(0xFFFFFFFFu, mykey, K - 1);
-    for (int base = 0; base < n; base += 32) {
-        unsigned long long key = base + lane < n ? list[base + lane] : 0ull;
-        if (!(key > kth)) key = 0ull;
-        unsigned pending = __ballot_sync(0xFFFFFFFFu, key != 0ull);
-        if (__popc(pending) > 3) {
-            mykey = merge_top32(mykey, sort32_desc(key, lane), lane);
-        } else {
-            while (pending) {
-                const int from = __ffs(pending) - 1;
-                pending &= pending - 1;
-                const unsigned long long nk = __shfl_sync(0xFFFFFFFFu, key, from);
-                const int p = __popc(__ballot_sync(0xFFFFFFFFu, mykey > nk));   // keys ahead of nk
-                const unsigned long long up = __shfl_up_sync(0xFFFFFFFFu, mykey, 1);
-                if (lane == p) mykey = nk;
-                else if (lane > p) mykey = up;
-            }
-        }
-        kth = __shfl_sync(0xFFFFFFFFu, mykey, K - 1);
-    }
-    if (lane == 0) {
-        if (total > kListCap) sm.overflow = 1;
-        ctl.cnt[which] = 0;
-        if (kth != 0ull) *reinterpret_cast<volatile float *>(&sm.thr_v) = key_value(kth);
-    }
+// Entry of the table of per-thread tile maxima, stored in the row's own element type (exact).
+__device__ __forceinline__ void table_store(__nv_bfloat16 *tab, int i, float v) {
+    reinterpret_cast<unsigned short *>(tab)[i] = (unsigned short)(__float_as_uint(v) >> 16);
 }
+__device__ __forceinline__ void table_store(float *tab, int i, float v) { tab[i] = v; }
 
-// First threshold of a slice from the thread maxima of its first tile, for the consumers of a
-// streaming kernel: with r = ceil(K / #warps), the smallest over the warps of each warp's r-th
-// largest thread maximum has K distinct logits at or above it.  One barrier; every thread
-// derives the value itself and thread 0 also stores it in sm.thr_v.  If some warp has fewer
-// than r finite maxima (masked rows) the general rule of bootstrap_threshold applies.
+// First threshold from one value per thread (its largest logit): with r = ceil(K / #warps), the
+// smallest over the warps of each warp's r-th largest value has K distinct logits at or above
+// it.  One barrier; every thread derives the value itself.  If some warp has fewer than r finite
+// values (masked rows) the general rule of bootstrap_threshold applies (two more barriers).
 template <typename SY>
 __device__ __forceinline__ float bootstrap_threshold_fast(ScanSmem &sm, float tm, int K) {
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -206,10 +136,8 @@ __device__ __forceinline__ float bootstrap_threshold_fast(ScanSmem &sm, float tm
     float t = CUDART_INF_F;
 #pragma unroll
     for (int w = 0; w < kWarps; ++w) t = fminf(t, sm.wsorted[w][r - 1]);
-    if (t > -CUDART_INF_F) {
-        if (tid == 0) sm.thr_v = t;
-        return t;
-    }
+    if (t > -CUDART_INF_F) return t;
+    SY::sync();
     if (tid == 0) {
         float g = -CUDART_INF_F;
         for (int rr = 1; rr <= 32; ++rr) {
@@ -228,80 +156,111 @@ __device__ __forceinline__ float bootstrap_threshold_fast(ScanSmem &sm, float tm
     return sm.thr_v;
 }
 
-// Issue the bulk copy of tile t of the slice at `src` into its ring stage (one thread).
-__device__ __forceinline__ void issue_tile(const char *src, int nbytes, int t, unsigned char *ring,
-                                           StreamBars &bars) {
-    const int s = t % kStages;
-    const uint32_t bytes = (uint32_t)min(kTileBytes, nbytes - t * kTileBytes);
-    mbar_expect_tx(&bars.full[s], bytes);
-    bulk_load(ring + (size_t)s * kTileBytes, src + (size_t)t * kTileBytes, bytes, &bars.full[s]);
-}
-
-// The fold warp of a slice scan (32 threads, all of them call this; it takes part in no barrier
-// of the CTA after stream_begin and exits when it returns).  For every tile i in order it waits
-// until every consumer warp is past the tile (bars.listed), folds list i % kLists into its
-// sorted top-32, publishes the threshold and completes the list's bars.folded phase.  After the
-// last fold the best min(K, #keys) keys are in sm.sel[0 .. ctl.nsel), sorted.  If a wait gives
-// up, the work goes on all the same so that every other wait still ends.
-__device__ __forceinline__ void stream_service(int nbytes, int K, ScanSmem &sm, StreamCtl &ctl,
-                                               StreamBars &bars) {
-    const int lane = threadIdx.x & 31;
-    volatile int *abort = &ctl.timed_out;
-    const int ntiles = (nbytes + kTileBytes - 1) / kTileBytes;
-    unsigned long long mykey = 0ull;
-    for (int fold = 0; fold < ntiles; ++fold) {
-        const int l = fold % kLists;
-        if (!mbar_wait(&bars.listed[l], (fold / kLists) & 1, abort)) ctl.timed_out = 1;
-        fold_list(sm, ctl, l, K, mykey);
-        if (fold == ntiles - 1) {
-            const unsigned have = __ballot_sync(0xFFFFFFFFu, mykey != 0ull && lane < K);
-            if (lane < DSP_MAX_K) sm.sel[lane] = mykey;
-            if (lane == 0) ctl.nsel = __popc(have);
-        }
-        __syncwarp();
-        if (lane == 0) {
-            __threadfence_block();
-            mbar_arrive(&bars.folded[l]);
-        }
-    }
-}
-
-// Padding for the vectors past the end of a ragged last tile: -2^124, below every finite
-// logit the interface allows, finite when scaled by log2(e), never a candidate (its index is
-// past the row).
-template <typename DT> struct Pad;
-template <> struct Pad<__nv_bfloat16> { static constexpr uint32_t kWord = 0xFD80FD80u; };
-template <> struct Pad<float> { static constexpr uint32_t kWord = 0xFD800000u; };
-
-// Consumer side of the scan of [s0, s1) of `row` (kThreads threads, barriers via SyncConsumers;
-// the fold warp runs stream_service meanwhile).  Same contract as scan_slice.
-template <typename DT, bool SUMS>
-__device__ void scan_slice_stream(const DT *__restrict__ row, int s0, int s1, int K, ScanSmem &sm,
-                                  StreamCtl &ctl, unsigned char *ring, StreamBars &bars,
-                                  float &c_out, double &S_out, double &T_out) {
-    using SY = SyncConsumers;
+// Exact top-K of the slice from the table of per-thread tile maxima (`tab`, ntiles x kThreads,
+// entry [t][thread]) and the thread's own largest logit `rm`.  On return sm.cand[0 .. sm.cnt)
+// holds the best min(K, #finite) keys, sorted (after a barrier).  Rows with very many equal top
+// values overflow the lists and take topk_careful instead.  Block-wide.
+template <typename DT, typename SY>
+__device__ void select_from_table(const DT *__restrict__ row, int s0, int s1, int K, int ntiles,
+                                  const DT *tab, float rm, ScanSmem &sm, StreamBars &bars) {
     constexpr int N = Elem<DT>::N;
     constexpr int TE = tile_elems<DT>();
+    constexpr int kHalf = kCandCap / 2;              // entries first, element keys in the upper half
+    const int tid = threadIdx.x;
+    // 1. a threshold with at least K table entries at or above it
+    const float t0 = bootstrap_threshold_fast<SY>(sm, rm, K);
+    // 2. the table entries that reach it (each thread looks at its own column)
+    for (int t = 0; t < ntiles; ++t) {
+        const float v = Elem<DT>::load1(tab + t * kThreads + tid);
+        if (v >= t0 && v > -CUDART_INF_F) {
+            const int pos = atomicAdd(&sm.cnt, 1);
+            if (pos < kHalf) sm.cand[pos] = make_key(v, t * kThreads + tid);
+        }
+    }
+    SY::sync();
+    const int n = sm.cnt;
+    if (n > kHalf) {                                 // block-uniform
+        topk_careful<DT, SY>(row, s0, s1, K, sm);
+        return;
+    }
+    // 3. the K-th largest of them (all of them if there are fewer than K), by counting
+    const int kk = min(K, n);
+    for (int i = tid; i < n; i += kThreads) {
+        const unsigned long long key = sm.cand[i];
+        int rank = 0;
+        for (int j = 0; j < n; ++j) rank += sm.cand[j] > key;
+        if (rank == kk - 1) sm.thrkey = key;
+    }
+    SY::sync();
+    // 4. the shares whose maximum reaches that value hold every logit of the slice's top K:
+    //    look at their logits again and list those that reach it
+    if (n > 0) {
+        // with fewer than K entries (the threshold was -inf: every finite entry is listed) every
+        // finite logit of the listed shares is wanted
+        const float tk = n >= K ? key_value(sm.thrkey) : -CUDART_INF_F;
+        for (int i = tid; i < n; i += kThreads) {
+            const unsigned long long key = sm.cand[i];
+            if (key_value(key) >= tk) {
+                const int id = key_id(key);
+                const int e00 = s0 + (id / kThreads) * TE + (id % kThreads) * N;
+#pragma unroll
+                for (int j = 0; j < kVpt; ++j) {
+                    const int e0 = e00 + j * kThreads * N;
+                    if (e0 < s1) {                   // vectors are whole: the row length is a multiple of N
+                        const uint4 v = ldg_stream(row + e0);
+#pragma unroll
+                        for (int e = 0; e < N; ++e) {
+                            const float x = Elem<DT>::get(v, e);
+                            if (x >= tk && x > -CUDART_INF_F) {
+                                const int pos = atomicAdd(&bars.cnt2, 1);
+                                if (pos < kHalf) sm.cand[kHalf + pos] = make_key(x, e0 + e);
+                            }
+                        }
+                    }
+                }
+            }
+        }
+    }
+    SY::sync();
+    const int n2 = bars.cnt2;
+    if (n2 > kHalf) {                                // block-uniform
+        topk_careful<DT, SY>(row, s0, s1, K, sm);
+        return;
+    }
+    // 5. the best K of the listed logits, sorted, to the front
+    unsigned long long mine[kHalf / kThreads];
+#pragma unroll
+    for (int q = 0; q < kHalf / kThreads; ++q) {
+        const int i = q * kThreads + tid;
+        mine[q] = i < n2 ? sm.cand[kHalf + i] : 0ull;
+    }
+    SY::sync();
+#pragma unroll
+    for (int q = 0; q < kHalf / kThreads; ++q) {
+        const int i = q * kThreads + tid;
+        if (i < n2) sm.cand[i] = mine[q];
+    }
+    if (tid == 0) sm.cnt = n2;
+    prune<SY>(sm, K);
+}
+
+// Scan [s0, s1) of `row` (all kThreads threads of the CTA).  Same contract as scan_slice.
+// `ring` and `tab` are the dynamic shared memory (kRingBytes and kMaxTableBytes).
+template <typename DT, bool SUMS>
+__device__ void scan_slice_stream(const DT *__restrict__ row, int s0, int s1, int K, ScanSmem &sm,
+                                  StreamBars &bars, unsigned char *ring, DT *tab,
+                                  float &c_out, double &S_out, double &T_out) {
+    using SY = SyncAll;
+    constexpr int N = Elem<DT>::N;
     constexpr int VT = kTileBytes / 16;
-    static_assert(VT == kThreads * kVpt && TE * (int)sizeof(DT) == kTileBytes, "tile geometry");
+    static_assert(VT == kThreads * kVpt && tile_elems<DT>() * (int)sizeof(DT) == kTileBytes, "tile geometry");
     const int tid = threadIdx.x, lane = tid & 31;
     const int nbytes = (s1 - s0) * (int)sizeof(DT);
     const int ntiles = (nbytes + kTileBytes - 1) / kTileBytes;
+    volatile int *abort = &bars.timed_out;
 
     float c = kRefFloor, S = 0.f, T = 0.f;
-    float thr = -CUDART_INF_F;
-    volatile int *abort = &ctl.timed_out;
-
-    // the reference exponent must bound every logit below the threshold (those skip the test)
-    auto raise_ref = [&](float ts) {
-        if (ts > c) {
-            const float d = c - ts;
-            const float sc = ex2_approx(d);
-            T = (T + S * d) * sc;
-            S = S * sc;
-            c = ts;
-        }
-    };
+    float rm = -CUDART_INF_F;                        // this thread's largest logit so far
 
     // Thread 0 also issues the copies, kStages - 1 tiles ahead of the tile being scanned.
     const char *src = reinterpret_cast<const char *>(row + s0);
@@ -311,11 +270,11 @@ __device__ void scan_slice_stream(const DT *__restrict__ row, int s0, int s1, in
     for (int t = 0; t < ntiles; ++t) {
         if (tid == 0 && t >= 1 && t + kStages - 1 < ntiles) {
             const int tt = t + kStages - 1;           // its stage held tile t - 1
-            if (!mbar_wait(&bars.empty[tt % kStages], ((tt / kStages) - 1) & 1, abort)) ctl.timed_out = 1;
+            if (!mbar_wait(&bars.empty[tt % kStages], ((tt / kStages) - 1) & 1, abort)) bars.timed_out = 1;
             issue_tile(src, nbytes, tt, ring, bars);
         }
         const int s = t % kStages;
-        if (!mbar_wait(&bars.full[s], (t / kStages) & 1, abort)) ctl.timed_out = 1;
+        if (!mbar_wait(&bars.full[s], (t / kStages) & 1, abort)) bars.timed_out = 1;
         const int nvec = min(kTileBytes, nbytes - t * kTileBytes) >> 4;
         const uint4 *sp = reinterpret_cast<const uint4 *>(ring + (size_t)s * kTileBytes);
         uint4 v[kVpt];
@@ -330,6 +289,9 @@ __device__ void scan_slice_stream(const DT *__restrict__ row, int s0, int s1, in
                 v[j] = vi < nvec ? sp[vi] : make_uint4(pw, pw, pw, pw);
             }
         }
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&bars.empty[s]);   // the stage is in registers: release it
+
         float x[kVpt][N];
         float vm[kVpt];
 #pragma unroll
@@ -344,44 +306,18 @@ __device__ void scan_slice_stream(const DT *__restrict__ row, int s0, int s1, in
             }
         }
         const float tm = fmaxf(fmaxf(vm[0], vm[1]), fmaxf(vm[2], vm[3]));
+        table_store(tab, t * kThreads + tid, tm);
+        rm = fmaxf(rm, tm);
 
-        float thr_now;
-        if (t == 0) {
-            thr_now = bootstrap_threshold_fast<SY>(sm, tm, K);   // consumers only; no candidate exists yet
-        } else {
-            thr_now = *reinterpret_cast<volatile float *>(&sm.thr_v);
-        }
-        if (thr_now > thr) {
-            thr = thr_now;
-            if constexpr (SUMS) raise_ref(thr * kLog2e);
-        }
-        // Vectors holding a logit at or above the threshold are few: the warp takes them one at a
-        // time and its first N lanes test one logit each, read back from the ring stage.
-        if (__ballot_sync(0xFFFFFFFFu, tm >= thr)) {
-            if constexpr (SUMS) { if (tm >= thr) raise_ref(tm * kLog2e); }
-            const DT *tile = reinterpret_cast<const DT *>(sp);
-            const int l = t % kLists;
-#pragma unroll
-            for (int j = 0; j < kVpt; ++j) {
-                unsigned hitters = __ballot_sync(0xFFFFFFFFu, vm[j] >= thr);
-                while (hitters) {
-                    const int from = __ffs(hitters) - 1;
-                    hitters &= hitters - 1;
-                    if (lane < N) {
-                        const int pos_in_tile = (j * kThreads + (tid - lane) + from) * N + lane;
-                        const int idx = s0 + t * TE + pos_in_tile;
-                        const float xv = Elem<DT>::load1(tile + pos_in_tile);
-                        if (xv >= thr && xv > -CUDART_INF_F && idx < s1) {
-                            const int pos = atomicAdd(&ctl.cnt[l], 1);
-                            if (pos < kListCap) sm.cand[l * kListCap + pos] = make_key(xv, idx);
-                        }
-                    }
-                }
-            }
-        }
-        __syncwarp();
-        if (lane == 0) mbar_arrive(&bars.empty[s]);   // done with the stage: release it
         if constexpr (SUMS) {
+            const float ts = tm * kLog2e;             // the reference exponent bounds every logit seen
+            if (ts > c) {
+                const float d = c - ts;
+                const float sc = ex2_approx(d);
+                T = (T + S * d) * sc;
+                S = S * sc;
+                c = ts;
+            }
             const float nc = -c;
 #pragma unroll
             for (int j = 0; j < kVpt; ++j) {
@@ -394,21 +330,8 @@ __device__ void scan_slice_stream(const DT *__restrict__ row, int s0, int s1, in
                 }
             }
         }
-        // this warp's candidates of tile t are complete; the list of the next tile must have
-        // been folded (emptied) since it was last used, kLists tiles earlier
-        if (t + 1 < ntiles && t + 1 >= kLists &&
-            !mbar_wait(&bars.folded[(t + 1) % kLists], ((t + 1 - kLists) / kLists) & 1, abort))
-            ctl.timed_out = 1;
-        __syncwarp();
-        if (lane == 0) mbar_arrive(&bars.listed[t % kLists]);
     }
-    // the last fold leaves the slice's best keys, sorted, in sm.sel
-    if (!mbar_wait(&bars.folded[(ntiles - 1) % kLists], ((ntiles - 1) / kLists) & 1, abort)) ctl.timed_out = 1;
-    const int nsel = min(ctl.nsel, K);
-    if (tid < nsel) sm.cand[tid] = sm.sel[tid];
-    if (tid == 0) sm.cnt = nsel;
-    SY::sync();
-    if (sm.overflow) topk_careful<DT, SY>(row, s0, s1, K, sm);
+    select_from_table<DT, SY>(row, s0, s1, K, ntiles, tab, rm, sm, bars);
 
     if constexpr (SUMS) {
         reduce_sums<DT, SY>(row, s0, s1, sm, c, S, T, c_out, S_out, T_out);
@@ -417,8 +340,9 @@ __device__ void scan_slice_stream(const DT *__restrict__ row, int s0, int s1, in
     }
 }
 
-// The ring needs more dynamic shared memory than the default limit: raise the limit of `kernel`
-// once per device (the attribute is per device).  `rec` is the caller's per-kernel record.
+// The streaming kernels need more dynamic shared memory than the default limit: raise the limit
+// of `kernel` once per device (the attribute is per device).  `rec` is the caller's per-kernel
+// record.
 struct RingSmemDone {
     bool dev[64] = {};
 };
@@ -428,16 +352,19 @@ inline cudaError_t allow_ring_smem(KernelT *kernel, RingSmemDone &rec) {
     cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess) return e;
     if (dev >= 0 && dev < 64 && rec.dev[dev]) return cudaSuccess;
-    e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kRingBytes);
+    e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kStreamDynBytes);
     if (e == cudaSuccess && dev >= 0 && dev < 64) rec.dev[dev] = true;
     return e;
 }
 
-// True if rows of this layout can be streamed with bulk copies.
-inline bool stream_layout_ok(const void *base, size_t elem_bytes, int V, long long stride_b,
-                             long long stride_l) {
-    return (reinterpret_cast<uintptr_t>(base) & 15) == 0 && ((size_t)V * elem_bytes) % 16 == 0 &&
-           ((size_t)stride_b * elem_bytes) % 16 == 0 && ((size_t)stride_l * elem_bytes) % 16 == 0;
+// True if rows of this layout can be streamed with bulk copies and a slice of `slice_elems`
+// logits fits the table of tile maxima.
+template <typename DT>
+inline bool stream_layout_ok(const void *base, int V, long long stride_b, long long stride_l, int slice_elems) {
+    const size_t es = sizeof(DT);
+    return (reinterpret_cast<uintptr_t>(base) & 15) == 0 && ((size_t)V * es) % 16 == 0 &&
+           ((size_t)stride_b * es) % 16 == 0 && ((size_t)stride_l * es) % 16 == 0 &&
+           slice_elems <= max_stream_tiles<DT>() * tile_elems<DT>();
 }
 
 }  // namespace dsp

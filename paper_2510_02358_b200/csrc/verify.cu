@@ -202,12 +202,10 @@ __global__ void __launch_bounds__(kThreads, 4) target_kernel(const VerifyArgs a)
 
 // Streaming kernel for 16-byte aligned layouts (see stream_core.cuh).
 template <typename DT>
-__global__ void __launch_bounds__(kStreamThreads, 3) target_stream_kernel(const VerifyArgs a) {
-    extern __shared__ __align__(128) unsigned char ring[];
+__global__ void __launch_bounds__(kThreads, 3) target_stream_kernel(const VerifyArgs a) {
+    extern __shared__ __align__(128) unsigned char dyn[];
     __shared__ ScanSmem sm;
     __shared__ StreamBars bars;
-    __shared__ StreamCtl ctl;
-    const int tid = threadIdx.x;
     const long long row = blockIdx.x / a.nslices;
     const int slice = blockIdx.x - (int)(row * a.nslices);
     const int b = (int)(row / a.Lt);
@@ -215,17 +213,13 @@ __global__ void __launch_bounds__(kStreamThreads, 3) target_stream_kernel(const 
     const int s0 = slice * a.slice_elems;
     const int s1 = min(a.V, s0 + a.slice_elems);
     const bool sums = !a.all_greedy && a.mode[b] != 0;
-    stream_begin(sm, ctl, bars);
-    if (tid >= kThreads) {                                  // fold warp: running top-K
-        stream_service((s1 - s0) * (int)sizeof(DT), 1, sm, ctl, bars);
-        return;
-    }
+    stream_begin(sm, bars);
+    DT *tab = reinterpret_cast<DT *>(dyn + kRingBytes);
     float c;
     double S, T;
-    if (sums) scan_slice_stream<DT, true>(rowp, s0, s1, 1, sm, ctl, ring, bars, c, S, T);
-    else      scan_slice_stream<DT, false>(rowp, s0, s1, 1, sm, ctl, ring, bars, c, S, T);
-    target_finish<DT, SyncConsumers>(a, sm, row, slice, b, sums, c, S, T,
-                                     ctl.timed_out ? DSP_ROW_TIMEOUT : 0u);
+    if (sums) scan_slice_stream<DT, true>(rowp, s0, s1, 1, sm, bars, dyn, tab, c, S, T);
+    else      scan_slice_stream<DT, false>(rowp, s0, s1, 1, sm, bars, dyn, tab, c, S, T);
+    target_finish<DT, SyncAll>(a, sm, row, slice, b, sums, c, S, T, bars.timed_out ? DSP_ROW_TIMEOUT : 0u);
 }
 
 // ---- residual / bonus sampling -------------------------------------------------------------
@@ -446,10 +440,10 @@ static int32_t launch_verify(VerifyArgs &a, void *workspace, size_t workspace_by
     DSP_CUDA_TRY(cudaMemsetAsync(ws, 0, w.zero_bytes, st));
     const long long nblocks = nrows * a.nslices;
     if (nblocks > 0x7FFFFFFFLL) return DSP_ERR_UNSUPPORTED;
-    if (stream_layout_ok(a.target, sizeof(DT), a.V, a.tstride_b, a.tstride_l)) {
+    if (stream_layout_ok<DT>(a.target, a.V, a.tstride_b, a.tstride_l, a.slice_elems)) {
         static RingSmemDone smem_done;                       // one per element type
         DSP_CUDA_TRY(allow_ring_smem(target_stream_kernel<DT>, smem_done));
-        target_stream_kernel<DT><<<(unsigned)nblocks, kStreamThreads, kRingBytes, st>>>(a);
+        target_stream_kernel<DT><<<(unsigned)nblocks, kThreads, kStreamDynBytes, st>>>(a);
     } else {
         target_kernel<DT><<<(unsigned)nblocks, kThreads, 0, st>>>(a);
     }
