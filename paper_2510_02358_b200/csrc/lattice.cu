@@ -201,7 +201,7 @@ __global__ void __launch_bounds__(kThreads, 3) lattice_stream_kernel(const Latti
     stream_begin(sm, bars);
     float c;
     double S, T;
-    scan_slice_stream<DT, true>(rowp, s0, s1, a.K, sm, bars, dyn, reinterpret_cast<DT *>(dyn + kRingBytes), c, S, T);
+    scan_slice_stream<DT>(rowp, s0, s1, a.K, true, sm, bars, dyn, reinterpret_cast<DT *>(dyn + kRingBytes), c, S, T);
     lattice_finish<DT, SyncAll>(a, sm, row, slice, b, rowp, c, S, T, bars.timed_out ? DSP_ROW_TIMEOUT : 0u);
 }
 

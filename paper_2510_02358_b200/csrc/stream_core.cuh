@@ -165,7 +165,7 @@ __device__ void select_from_table(const DT *__restrict__ row, int s0, int s1, in
                                   const DT *tab, float rm, ScanSmem &sm, StreamBars &bars) {
     constexpr int N = Elem<DT>::N;
     constexpr int TE = tile_elems<DT>();
-    constexpr int kHalf = kCandCap / 2;              // entries first, element keys in the upper half
+    constexpr int kHalf = kCandCap / 2;              // element keys first, table entries in the upper half
     const int tid = threadIdx.x;
     // 1. a threshold with at least K table entries at or above it
     const float t0 = bootstrap_threshold_fast<SY>(sm, rm, K);
@@ -174,7 +174,7 @@ __device__ void select_from_table(const DT *__restrict__ row, int s0, int s1, in
         const float v = Elem<DT>::load1(tab + t * kThreads + tid);
         if (v >= t0 && v > -CUDART_INF_F) {
             const int pos = atomicAdd(&sm.cnt, 1);
-            if (pos < kHalf) sm.cand[pos] = make_key(v, t * kThreads + tid);
+            if (pos < kHalf) sm.cand[kHalf + pos] = make_key(v, t * kThreads + tid);
         }
     }
     SY::sync();
@@ -185,10 +185,11 @@ __device__ void select_from_table(const DT *__restrict__ row, int s0, int s1, in
     }
     // 3. the K-th largest of them (all of them if there are fewer than K), by counting
     const int kk = min(K, n);
+    const unsigned long long *entries = sm.cand + kHalf;
     for (int i = tid; i < n; i += kThreads) {
-        const unsigned long long key = sm.cand[i];
+        const unsigned long long key = entries[i];
         int rank = 0;
-        for (int j = 0; j < n; ++j) rank += sm.cand[j] > key;
+        for (int j = 0; j < n; ++j) rank += entries[j] > key;
         if (rank == kk - 1) sm.thrkey = key;
     }
     SY::sync();
@@ -199,7 +200,7 @@ __device__ void select_from_table(const DT *__restrict__ row, int s0, int s1, in
         // finite logit of the listed shares is wanted
         const float tk = n >= K ? key_value(sm.thrkey) : -CUDART_INF_F;
         for (int i = tid; i < n; i += kThreads) {
-            const unsigned long long key = sm.cand[i];
+            const unsigned long long key = entries[i];
             if (key_value(key) >= tk) {
                 const int id = key_id(key);
                 const int e00 = s0 + (id / kThreads) * TE + (id % kThreads) * N;
@@ -213,7 +214,7 @@ __device__ void select_from_table(const DT *__restrict__ row, int s0, int s1, in
                             const float x = Elem<DT>::get(v, e);
                             if (x >= tk && x > -CUDART_INF_F) {
                                 const int pos = atomicAdd(&bars.cnt2, 1);
-                                if (pos < kHalf) sm.cand[kHalf + pos] = make_key(x, e0 + e);
+                                if (pos < kHalf) sm.cand[pos] = make_key(x, e0 + e);
                             }
                         }
                     }
@@ -228,26 +229,16 @@ __device__ void select_from_table(const DT *__restrict__ row, int s0, int s1, in
         return;
     }
     // 5. the best K of the listed logits, sorted, to the front
-    unsigned long long mine[kHalf / kThreads];
-#pragma unroll
-    for (int q = 0; q < kHalf / kThreads; ++q) {
-        const int i = q * kThreads + tid;
-        mine[q] = i < n2 ? sm.cand[kHalf + i] : 0ull;
-    }
-    SY::sync();
-#pragma unroll
-    for (int q = 0; q < kHalf / kThreads; ++q) {
-        const int i = q * kThreads + tid;
-        if (i < n2) sm.cand[i] = mine[q];
-    }
     if (tid == 0) sm.cnt = n2;
     prune<SY>(sm, K);
 }
 
 // Scan [s0, s1) of `row` (all kThreads threads of the CTA).  Same contract as scan_slice.
 // `ring` and `tab` are the dynamic shared memory (kRingBytes and kMaxTableBytes).
-template <typename DT, bool SUMS>
-__device__ void scan_slice_stream(const DT *__restrict__ row, int s0, int s1, int K, ScanSmem &sm,
+// `sums` (block-uniform) says whether the log-sum-exp terms are wanted; one copy of the loop
+// serves both cases so that rows of both kinds share the instruction cache.
+template <typename DT>
+__device__ void scan_slice_stream(const DT *__restrict__ row, int s0, int s1, int K, bool sums, ScanSmem &sm,
                                   StreamBars &bars, unsigned char *ring, DT *tab,
                                   float &c_out, double &S_out, double &T_out) {
     using SY = SyncAll;
@@ -309,7 +300,7 @@ __device__ void scan_slice_stream(const DT *__restrict__ row, int s0, int s1, in
         table_store(tab, t * kThreads + tid, tm);
         rm = fmaxf(rm, tm);
 
-        if constexpr (SUMS) {
+        if (sums) {
             const float ts = tm * kLog2e;             // the reference exponent bounds every logit seen
             if (ts > c) {
                 const float d = c - ts;
@@ -333,7 +324,7 @@ __device__ void scan_slice_stream(const DT *__restrict__ row, int s0, int s1, in
     }
     select_from_table<DT, SY>(row, s0, s1, K, ntiles, tab, rm, sm, bars);
 
-    if constexpr (SUMS) {
+    if (sums) {
         reduce_sums<DT, SY>(row, s0, s1, sm, c, S, T, c_out, S_out, T_out);
     } else {
         c_out = kRefFloor; S_out = 0.0; T_out = 0.0;

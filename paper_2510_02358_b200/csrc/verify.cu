@@ -217,8 +217,7 @@ __global__ void __launch_bounds__(kThreads, 3) target_stream_kernel(const Verify
     DT *tab = reinterpret_cast<DT *>(dyn + kRingBytes);
     float c;
     double S, T;
-    if (sums) scan_slice_stream<DT, true>(rowp, s0, s1, 1, sm, bars, dyn, tab, c, S, T);
-    else      scan_slice_stream<DT, false>(rowp, s0, s1, 1, sm, bars, dyn, tab, c, S, T);
+    scan_slice_stream<DT>(rowp, s0, s1, 1, sums, sm, bars, dyn, tab, c, S, T);
     target_finish<DT, SyncAll>(a, sm, row, slice, b, sums, c, S, T, bars.timed_out ? DSP_ROW_TIMEOUT : 0u);
 }
 
