@@ -76,6 +76,26 @@ __device__ __forceinline__ float max3(float a, float b, float c) {
     return d;
 }
 
+// Two fp32 operations in one instruction on a register pair (Blackwell's packed fp32 pipe).
+__device__ __forceinline__ unsigned long long pack2(float lo, float hi) {
+    unsigned long long r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+    return r;
+}
+__device__ __forceinline__ void unpack2(unsigned long long v, float &lo, float &hi) {
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ unsigned long long fma2(unsigned long long a, unsigned long long b, unsigned long long c) {
+    unsigned long long d;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+    return d;
+}
+__device__ __forceinline__ unsigned long long add2(unsigned long long a, unsigned long long b) {
+    unsigned long long d;
+    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+    return d;
+}
+
 // Shared state of a streaming kernel besides ScanSmem.
 struct StreamBars {
     uint64_t full[kStages];      // stage filled by its bulk copy
@@ -309,17 +329,26 @@ __device__ void scan_slice_stream(const DT *__restrict__ row, int s0, int s1, in
                 S = S * sc;
                 c = ts;
             }
-            const float nc = -c;
+            // two logits per instruction: a = x * log2(e) - c, S += 2^a, T += 2^a * a
+            const unsigned long long nc2 = pack2(-c, -c), l2e2 = pack2(kLog2e, kLog2e);
+            unsigned long long S2 = pack2(S, 0.f), T2 = pack2(T, 0.f);
 #pragma unroll
             for (int j = 0; j < kVpt; ++j) {
 #pragma unroll
-                for (int e = 0; e < N; ++e) {
-                    const float a = fmaf(x[j][e], kLog2e, nc);
-                    const float ex = ex2_approx(a);
-                    S += ex;
-                    T = fmaf(ex, a, T);
+                for (int e = 0; e < N; e += 2) {
+                    const unsigned long long a2 = fma2(pack2(x[j][e], x[j][e + 1]), l2e2, nc2);
+                    float a0, a1;
+                    unpack2(a2, a0, a1);
+                    const unsigned long long e2 = pack2(ex2_approx(a0), ex2_approx(a1));
+                    S2 = add2(S2, e2);
+                    T2 = fma2(e2, a2, T2);
                 }
             }
+            float s0f, s1f, t0f, t1f;
+            unpack2(S2, s0f, s1f);
+            unpack2(T2, t0f, t1f);
+            S = s0f + s1f;
+            T = t0f + t1f;
         }
     }
     select_from_table<DT, SY>(row, s0, s1, K, ntiles, tab, rm, sm, bars);
