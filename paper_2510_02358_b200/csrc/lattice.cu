@@ -1,9 +1,13 @@
 // dsp_lattice_build: draft logits -> token lattice (Sec. 3.2 "Lattice and pruning", Eq. 7, Eq. 9).
 //
-// One kernel.  Each row (b,l) is cut into slices of whole tiles; one CTA streams one slice
-// once from HBM (log-sum-exp terms + exact top-K, see scan_core.cuh).  A row split over
-// several CTAs is finished by whichever CTA arrives last (atomic ticket): no CTA waits.
-// The CTA that finishes the last row of a batch row also writes gen_len and row_status.
+// Rows whose layout is 16-byte aligned take two kernels: lattice_scan_kernel streams every row
+// slice once from HBM (one CTA per slice, no block-wide barrier: log-sum-exp terms per warp and
+// a table of per-thread tile maxima, see stream_core.cuh); lattice_rows_kernel (one CTA per
+// row) adds up the sums, selects the exact top-K from the table and finalises the row.
+// Any other layout takes lattice_kernel: one CTA streams one slice element-wise and does the
+// top-K on the way; a row split over several CTAs is finished by whichever CTA arrives last
+// (atomic ticket): no CTA waits.  In both paths the CTA that finishes the last row of a batch
+// row also writes gen_len and row_status.
 #include "stream_core.cuh"
 
 namespace dsp {
@@ -29,14 +33,20 @@ struct LatticeArgs {
     unsigned *row_ticket;     // [B*L]   zeroed per call
     unsigned *b_ticket;       // [B]     zeroed per call
     unsigned *b_status;       // [B]     zeroed per call
-    SlicePartial *partials;   // [B*L, nslices]
-    unsigned long long *keys; // [B*L, nslices, K]
+    SlicePartial *partials;   // [B*L, nslices]               (element-wise path)
+    unsigned long long *keys; // [B*L, nslices, K]            (element-wise path)
+    WarpPartial *wpart;       // [B*L, nslices, kWarps]       (streaming path)
+    void *table;              // [B*L, ntiles_row, kThreads]  (streaming path), element type of the logits
+    int ntiles_row;           // tiles of a whole row
 };
 
+// Both paths share the zeroed head; the rest is laid out for the element-wise path (partials,
+// keys) and for the streaming path (wpart, table) over the same bytes: a call takes one path.
 struct LatticeWs {
-    size_t off_row_ticket, off_b_ticket, off_b_status, zero_bytes, off_partials, off_keys, total;
+    size_t off_row_ticket, off_b_ticket, off_b_status, zero_bytes, off_partials, off_keys;
+    size_t off_wpart, off_table, total;
 };
-static LatticeWs lattice_ws_layout(int64_t B, int64_t L, int nslices, int K) {
+static LatticeWs lattice_ws_layout(int64_t B, int64_t L, int nslices, int K, int ntiles_row, size_t es) {
     LatticeWs w;
     size_t o = 0;
     w.off_row_ticket = o; o += align_up((size_t)(B * L) * 4, 256);
@@ -45,9 +55,16 @@ static LatticeWs lattice_ws_layout(int64_t B, int64_t L, int nslices, int K) {
     w.zero_bytes = o;
     w.off_partials = o;   o += align_up((size_t)(B * L) * nslices * sizeof(SlicePartial), 256);
     w.off_keys = o;       o += align_up((size_t)(B * L) * nslices * K * 8, 256);
-    w.total = o;
+    size_t o2 = w.zero_bytes;
+    w.off_wpart = o2;     o2 += align_up((size_t)(B * L) * nslices * kWarps * sizeof(WarpPartial), 256);
+    w.off_table = o2;     o2 += align_up((size_t)(B * L) * ntiles_row * kThreads * es, 256);
+    w.total = o > o2 ? o : o2;
     return w;
 }
+
+template <typename DT, typename SY>
+__device__ void lattice_finalise(const LatticeArgs &a, ScanSmem &sm, long long row, int b, const DT *rowp,
+                                 float c, double S, double T);
 
 // Everything after the scan of one slice: publish the slice's partial result, let the CTA that
 // arrives last merge the row, finalise the row (Eq. 7 count, EOS slot, outputs) and, for the
@@ -94,7 +111,16 @@ __device__ void lattice_finish(const LatticeArgs &a, ScanSmem &sm, long long row
         S = sm.fin[0]; T = sm.fin[1]; c = sm.redc[0];
     }
 
-    // ---- finalise the row: sm.cand[0..cnt) sorted best keys, (c,S,T) whole-row sums ----
+    lattice_finalise<DT, SY>(a, sm, row, b, rowp, c, S, T);
+}
+
+// Finalise a row from its sorted best keys sm.cand[0 .. sm.cnt) and its whole-row sums (c, S, T):
+// log-sum-exp, entropy, Eq. 7 count, EOS slot, candidate outputs; the CTA that finishes the last
+// row of a batch row also writes gen_len (Eq. 9) and row_status.
+template <typename DT, typename SY>
+__device__ void lattice_finalise(const LatticeArgs &a, ScanSmem &sm, long long row, int b, const DT *rowp,
+                                 float c, double S, double T) {
+    const int tid = threadIdx.x;
     const int nk = sm.cnt;
     double lse, mean_x;
     const bool ok = row_log_stats(c, S, T, lse, mean_x) && nk > 0;
@@ -184,13 +210,10 @@ __global__ void __launch_bounds__(kThreads, 4) lattice_kernel(const LatticeArgs 
     lattice_finish<DT, SyncAll>(a, sm, row, slice, b, rowp, c, S, T, 0u);
 }
 
-// Streaming kernel for 16-byte aligned layouts: the slice streams through a shared-memory ring
-// of bulk asynchronous copies and the top-K is selected from a table of per-thread tile maxima
-// once the slice has been read (see stream_core.cuh).
+// Streaming path, pass 1: one CTA per row slice (see stream_core.cuh).
 template <typename DT>
-__global__ void __launch_bounds__(kThreads, 3) lattice_stream_kernel(const LatticeArgs a) {
-    extern __shared__ __align__(128) unsigned char dyn[];
-    __shared__ ScanSmem sm;
+__global__ void __launch_bounds__(kThreads, 4) lattice_scan_kernel(const LatticeArgs a) {
+    extern __shared__ __align__(128) unsigned char ring[];
     __shared__ StreamBars bars;
     const long long row = blockIdx.x / a.nslices;
     const int slice = blockIdx.x - (int)(row * a.nslices);
@@ -198,11 +221,29 @@ __global__ void __launch_bounds__(kThreads, 3) lattice_stream_kernel(const Latti
     const DT *rowp = reinterpret_cast<const DT *>(a.logits) + b * a.stride_b + l * a.stride_l;
     const int s0 = slice * a.slice_elems;
     const int s1 = min(a.V, s0 + a.slice_elems);
-    stream_begin(sm, bars);
+    stream_begin(bars);
+    DT *tab = reinterpret_cast<DT *>(a.table) +
+              (row * a.ntiles_row + (long long)(s0 / tile_elems<DT>())) * kThreads;
+    stream_slice<DT>(rowp, s0, s1, true, bars, ring, tab, a.wpart + (row * a.nslices + slice) * kWarps);
+    if (threadIdx.x == 0 && bars.timed_out) atomicOr(&a.b_status[b], DSP_ROW_TIMEOUT);
+}
+
+// Streaming path, pass 2: one CTA per row.
+template <typename DT>
+__global__ void __launch_bounds__(kThreads) lattice_rows_kernel(const LatticeArgs a) {
+    __shared__ ScanSmem sm;
+    const int tid = threadIdx.x;
+    const long long row = blockIdx.x;
+    const int b = (int)(row / a.L), l = (int)(row - (long long)b * a.L);
+    const DT *rowp = reinterpret_cast<const DT *>(a.logits) + b * a.stride_b + l * a.stride_l;
+    if (tid == 0) { sm.cnt = 0; sm.flag = 0; sm.thrkey = 0ull; sm.thr_v = -CUDART_INF_F; sm.overflow = 0; }
     float c;
     double S, T;
-    scan_slice_stream<DT>(rowp, s0, s1, a.K, true, sm, bars, dyn, reinterpret_cast<DT *>(dyn + kRingBytes), c, S, T);
-    lattice_finish<DT, SyncAll>(a, sm, row, slice, b, rowp, c, S, T, bars.timed_out ? DSP_ROW_TIMEOUT : 0u);
+    merge_warp_partials<SyncAll>(a.wpart + row * a.nslices * kWarps, a.nslices * kWarps, sm, c, S, T);
+    if (T != T && S == S && S < CUDART_INF) redo_sums<DT, SyncAll>(rowp, 0, a.V, sm, c, S, T);
+    select_from_table<DT, SyncAll>(rowp, 0, a.V, a.K, a.ntiles_row,
+                                   reinterpret_cast<const DT *>(a.table) + row * a.ntiles_row * kThreads, sm);
+    lattice_finalise<DT, SyncAll>(a, sm, row, b, rowp, c, S, T);
 }
 
 template <typename DT>
@@ -211,7 +252,8 @@ static int32_t launch_lattice(LatticeArgs &a, void *workspace, size_t workspace_
     const SlicePlan plan = plan_slices<DT>(nrows, a.V, kTargetCtas);
     a.nslices = plan.nslices;
     a.slice_elems = plan.slice_elems;
-    const LatticeWs w = lattice_ws_layout(a.B, a.L, a.nslices, a.K);
+    a.ntiles_row = (a.V + tile_elems<DT>() - 1) / tile_elems<DT>();
+    const LatticeWs w = lattice_ws_layout(a.B, a.L, a.nslices, a.K, a.ntiles_row, sizeof(DT));
     if (workspace_bytes < w.total) return DSP_ERR_WORKSPACE;
     char *ws = reinterpret_cast<char *>(workspace);
     a.row_ticket = reinterpret_cast<unsigned *>(ws + w.off_row_ticket);
@@ -219,13 +261,18 @@ static int32_t launch_lattice(LatticeArgs &a, void *workspace, size_t workspace_
     a.b_status = reinterpret_cast<unsigned *>(ws + w.off_b_status);
     a.partials = reinterpret_cast<SlicePartial *>(ws + w.off_partials);
     a.keys = reinterpret_cast<unsigned long long *>(ws + w.off_keys);
+    a.wpart = reinterpret_cast<WarpPartial *>(ws + w.off_wpart);
+    a.table = ws + w.off_table;
     DSP_CUDA_TRY(cudaMemsetAsync(ws, 0, w.zero_bytes, st));
     const long long nblocks = nrows * a.nslices;
     if (nblocks > 0x7FFFFFFFLL) return DSP_ERR_UNSUPPORTED;
-    if (stream_layout_ok<DT>(a.logits, a.V, a.stride_b, a.stride_l, a.slice_elems)) {
+    if (a.nslices * kWarps <= kThreads && nrows <= 0x7FFFFFFFLL &&
+        stream_layout_ok<DT>(a.logits, a.V, a.stride_b, a.stride_l)) {
         static RingSmemDone smem_done;                       // one per element type
-        DSP_CUDA_TRY(allow_ring_smem(lattice_stream_kernel<DT>, smem_done));
-        lattice_stream_kernel<DT><<<(unsigned)nblocks, kThreads, kStreamDynBytes, st>>>(a);
+        DSP_CUDA_TRY(allow_ring_smem(lattice_scan_kernel<DT>, smem_done));
+        lattice_scan_kernel<DT><<<(unsigned)nblocks, kThreads, kRingBytes, st>>>(a);
+        DSP_CUDA_TRY(cudaGetLastError());
+        lattice_rows_kernel<DT><<<(unsigned)nrows, kThreads, 0, st>>>(a);
     } else {
         lattice_kernel<DT><<<(unsigned)nblocks, kThreads, 0, st>>>(a);
     }
@@ -236,7 +283,8 @@ static int32_t launch_lattice(LatticeArgs &a, void *workspace, size_t workspace_
 template <typename DT>
 static size_t lattice_ws_bytes(int B, int L, int V, int K) {
     const SlicePlan plan = plan_slices<DT>((long long)B * L, V, kTargetCtas);
-    return lattice_ws_layout(B, L, plan.nslices, K).total;
+    const int ntiles_row = (V + tile_elems<DT>() - 1) / tile_elems<DT>();
+    return lattice_ws_layout(B, L, plan.nslices, K, ntiles_row, sizeof(DT)).total;
 }
 
 }  // namespace dsp

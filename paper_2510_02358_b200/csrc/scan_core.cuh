@@ -156,6 +156,42 @@ __device__ void topk_careful(const DT *__restrict__ row, int s0, int s1, int K, 
     prune<SY>(sm, K);
 }
 
+// Sums of [s0, s1) of `row` against the known reference exponent cb with the exponent clamped:
+// used when masked (-inf) logits poisoned T only (0 * -inf) in the streaming pass.  Block-wide.
+template <typename DT, typename SY>
+__device__ void redo_sums(const DT *__restrict__ row, int s0, int s1, ScanSmem &sm, float cb,
+                          double &Sd, double &Td) {
+    constexpr int N = Elem<DT>::N;
+    constexpr int TE = tile_elems<DT>();
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const bool aligned = (reinterpret_cast<uintptr_t>(row) & 15) == 0;
+    const int ntiles = (s1 - s0 + TE - 1) / TE;
+    const float nc = -cb;
+    float S2 = 0.f, T2 = 0.f;
+    for (int t = 0; t < ntiles; ++t) {
+        const int base = s0 + t * TE;
+#pragma unroll
+        for (int j = 0; j < kVpt; ++j) {
+            const uint4 vv = load_vec<DT>(row, base + (j * kThreads + tid) * N, s1, aligned);
+#pragma unroll
+            for (int e = 0; e < N; ++e) {
+                const float x = Elem<DT>::get(vv, e);
+                const float a2 = fmaxf(fmaf(x, kLog2e, nc), -1000.f);
+                const float ex = ex2_approx(a2);
+                S2 += ex;
+                T2 = fmaf(ex, a2, T2);
+            }
+        }
+    }
+    double S2d = warp_sum((double)S2), T2d = warp_sum((double)T2);
+    if (lane == 0) { sm.redS[warp] = S2d; sm.redT[warp] = T2d; }
+    SY::sync();
+    Sd = 0.0; Td = 0.0;
+#pragma unroll
+    for (int w = 0; w < kWarps; ++w) { Sd += sm.redS[w]; Td += sm.redT[w]; }
+    SY::sync();
+}
+
 // Block reduction of the per-thread sums (c, S, T) of a slice to one reference exponent, in
 // double.  If masked (-inf) logits poisoned T only (0 * -inf), the slice's sums are redone from
 // global memory against the now known reference with the exponent clamped.
@@ -184,34 +220,7 @@ __device__ void reduce_sums(const DT *__restrict__ row, int s0, int s1, ScanSmem
     for (int w = 0; w < kWarps; ++w) { Sd += sm.redS[w]; Td += sm.redT[w]; }
     SY::sync();
 
-    if (Td != Td && Sd == Sd && Sd < CUDART_INF) {
-        // 0 * -inf from masked (-inf) logits poisoned T only: redo the sums of this
-        // slice against the now known reference with the exponent clamped.
-        const float nc = -cb;
-        float S2 = 0.f, T2 = 0.f;
-        for (int t = 0; t < ntiles; ++t) {
-            const int base = s0 + t * TE;
-#pragma unroll
-            for (int j = 0; j < kVpt; ++j) {
-                const uint4 vv = load_vec<DT>(row, base + (j * kThreads + tid) * N, s1, aligned);
-#pragma unroll
-                for (int e = 0; e < N; ++e) {
-                    const float x = Elem<DT>::get(vv, e);
-                    const float a2 = fmaxf(fmaf(x, kLog2e, nc), -1000.f);
-                    const float ex = ex2_approx(a2);
-                    S2 += ex;
-                    T2 = fmaf(ex, a2, T2);
-                }
-            }
-        }
-        double S2d = warp_sum((double)S2), T2d = warp_sum((double)T2);
-        if (lane == 0) { sm.redS[warp] = S2d; sm.redT[warp] = T2d; }
-        SY::sync();
-        Sd = 0.0; Td = 0.0;
-#pragma unroll
-        for (int w = 0; w < kWarps; ++w) { Sd += sm.redS[w]; Td += sm.redT[w]; }
-        SY::sync();
-    }
+    if (Td != Td && Sd == Sd && Sd < CUDART_INF) redo_sums<DT, SY>(row, s0, s1, sm, cb, Sd, Td);
     c_out = cb; S_out = Sd; T_out = Td;
 }
 
@@ -360,8 +369,7 @@ inline SlicePlan plan_slices(int64_t nrows, int V, int target_ctas) {
     int want = (int)((target_ctas + nrows - 1) / (nrows > 0 ? nrows : 1));   // slices per row wanted
     if (want < 1) want = 1;
     int tps = (ntiles + want - 1) / want;            // tiles per slice
-    const int cap = 64 / (int)sizeof(DT);            // tiles per slice the streaming kernels' table of tile maxima holds
-    if (tps > cap) tps = cap;
+    if (tps > 32) tps = 32;                          // bounds the time one CTA holds its SM slot
     const int min_tps = (ntiles + kMaxSlices - 1) / kMaxSlices;
     if (tps < min_tps) tps = min_tps;
     if (tps < 1) tps = 1;

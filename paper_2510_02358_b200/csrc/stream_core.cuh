@@ -1,16 +1,19 @@
-// TMA-fed variant of the one-pass slice scan for rows whose start, strides and length are
-// multiples of 16 bytes.  The slice streams through a ring of shared-memory stages by bulk
-// asynchronous copies (cp.async.bulk, completion counted on an mbarrier per stage, no
-// multicast) that one thread issues two tiles ahead; all kThreads threads read each stage with
-// one 128-bit shared load per vector and do the arithmetic from registers.
+// Streaming pass for rows whose start, strides and length are multiples of 16 bytes, and the
+// selection of the exact top-K from what it leaves behind.
 //
-// The streaming loop has no block-wide barrier and does nothing for the top-K except to keep,
-// per thread and tile, the largest of the thread's kVpt vectors of that tile in a shared-memory
-// table.  The exact top-K is selected from that table when the slice has been streamed: a
-// threshold with at least K table entries at or above it, the exact K-th largest entry among
-// those, and a second look (from global memory, L2 hits) at the few (tile, thread) shares whose
-// maximum reaches it.  Results are the same as scan_slice's (scan_core.cuh): log-sum-exp terms
-// and the exact top-K.
+// Pass 1 (stream_slice, one CTA per row slice): the slice streams through a ring of
+// shared-memory stages by bulk asynchronous copies (cp.async.bulk, completion counted on an
+// mbarrier per stage, no multicast) that one thread issues ahead; all kThreads threads read each
+// stage with one 128-bit shared load per vector and do the arithmetic from registers.  The loop
+// has no block-wide barrier.  It leaves in global memory, per row: a table with, for every tile
+// and thread, the largest logit of the thread's kVpt vectors of that tile, and per slice and
+// warp the log-sum-exp terms.
+//
+// Pass 2 (one CTA per row, run by the kernels in lattice.cu / verify.cu): merge_warp_partials
+// adds up the sums, select_from_table picks the exact top-K: a threshold with at least K
+// logits at or above it, the exact K-th largest table entry among those that reach it, and a
+// second look (L2 hits) at the few (tile, thread) shares whose maximum reaches that value.
+// Results are the same as scan_slice's (scan_core.cuh).
 #pragma once
 
 #include "scan_core.cuh"
@@ -19,14 +22,8 @@ namespace dsp {
 
 constexpr int kTileBytes = kThreads * kVpt * 16;     // one ring stage = one tile of either dtype
 constexpr int kStages = 3;
-constexpr int kRingBytes = kStages * kTileBytes;
-constexpr int kMaxTableBytes = 16384;                // table of per-thread tile maxima
+constexpr int kRingBytes = kStages * kTileBytes;     // dynamic shared memory of a streaming kernel
 constexpr long long kWaitCycles = 400000000LL;       // every wait gives up after this many SM clocks (~0.2 s)
-
-// Tiles per slice the table has room for: 32 for bf16 rows, 16 for fp32 rows.
-template <typename DT> constexpr int max_stream_tiles() { return kMaxTableBytes / (kThreads * (int)sizeof(DT)); }
-static_assert(max_stream_tiles<float>() == 64 / 4 && max_stream_tiles<__nv_bfloat16>() == 64 / 2,
-              "plan_slices caps the tiles per slice at 64 / sizeof(element)");
 
 __device__ __forceinline__ uint32_t smem_addr(const void *p) {
     return (uint32_t)__cvta_generic_to_shared(p);
@@ -96,26 +93,22 @@ __device__ __forceinline__ unsigned long long add2(unsigned long long a, unsigne
     return d;
 }
 
-// Shared state of a streaming kernel besides ScanSmem.
+// Static shared state of a streaming kernel.
 struct StreamBars {
     uint64_t full[kStages];      // stage filled by its bulk copy
     uint64_t empty[kStages];     // stage released by all warps
     int timed_out;               // non-zero once a bounded wait gave up
-    int cnt2;                    // entries of the second list of the selection
 };
-// Dynamic shared memory: the ring first (16-byte aligned), then the table of tile maxima.
-constexpr int kStreamDynBytes = kRingBytes + kMaxTableBytes;
 
 // Called by every thread before the scan starts (ends with a CTA-wide barrier).
-__device__ __forceinline__ void stream_begin(ScanSmem &sm, StreamBars &bars) {
+__device__ __forceinline__ void stream_begin(StreamBars &bars) {
     if (threadIdx.x == 0) {
         for (int s = 0; s < kStages; ++s) {
             mbar_init(&bars.full[s], 1);
             mbar_init(&bars.empty[s], kWarps);
         }
         mbar_init_fence();
-        sm.cnt = 0; sm.thrkey = 0ull; sm.thr_v = -CUDART_INF_F; sm.overflow = 0;
-        bars.timed_out = 0; bars.cnt2 = 0;
+        bars.timed_out = 0;
     }
     __syncthreads();
 }
@@ -176,18 +169,21 @@ __device__ __forceinline__ float bootstrap_threshold_fast(ScanSmem &sm, float tm
     return sm.thr_v;
 }
 
-// Exact top-K of the slice from the table of per-thread tile maxima (`tab`, ntiles x kThreads,
-// entry [t][thread]) and the thread's own largest logit `rm`.  On return sm.cand[0 .. sm.cnt)
-// holds the best min(K, #finite) keys, sorted (after a barrier).  Rows with very many equal top
-// values overflow the lists and take topk_careful instead.  Block-wide.
+// Exact top-K of [s0, s1) of `row` from its table of per-thread tile maxima (`tab`, ntiles x
+// kThreads, entry [t][thread], in global memory).  On return sm.cand[0 .. sm.cnt) holds the best
+// min(K, #finite) keys, sorted (after a barrier).  Rows with very many equal top values overflow
+// the lists and take topk_careful instead.  Block-wide; sm.cnt and sm.flag must be 0 on entry
+// (before a barrier).
 template <typename DT, typename SY>
 __device__ void select_from_table(const DT *__restrict__ row, int s0, int s1, int K, int ntiles,
-                                  const DT *tab, float rm, ScanSmem &sm, StreamBars &bars) {
+                                  const DT *tab, ScanSmem &sm) {
     constexpr int N = Elem<DT>::N;
     constexpr int TE = tile_elems<DT>();
     constexpr int kHalf = kCandCap / 2;              // element keys first, table entries in the upper half
     const int tid = threadIdx.x;
-    // 1. a threshold with at least K table entries at or above it
+    // 1. a threshold with at least K table entries at or above it, from each thread's largest
+    float rm = -CUDART_INF_F;
+    for (int t = 0; t < ntiles; ++t) rm = fmaxf(rm, Elem<DT>::load1(tab + t * kThreads + tid));
     const float t0 = bootstrap_threshold_fast<SY>(sm, rm, K);
     // 2. the table entries that reach it (each thread looks at its own column)
     for (int t = 0; t < ntiles; ++t) {
@@ -233,7 +229,7 @@ __device__ void select_from_table(const DT *__restrict__ row, int s0, int s1, in
                         for (int e = 0; e < N; ++e) {
                             const float x = Elem<DT>::get(v, e);
                             if (x >= tk && x > -CUDART_INF_F) {
-                                const int pos = atomicAdd(&bars.cnt2, 1);
+                                const int pos = atomicAdd(&sm.flag, 1);
                                 if (pos < kHalf) sm.cand[pos] = make_key(x, e0 + e);
                             }
                         }
@@ -243,7 +239,7 @@ __device__ void select_from_table(const DT *__restrict__ row, int s0, int s1, in
         }
     }
     SY::sync();
-    const int n2 = bars.cnt2;
+    const int n2 = sm.flag;
     if (n2 > kHalf) {                                // block-uniform
         topk_careful<DT, SY>(row, s0, s1, K, sm);
         return;
@@ -253,25 +249,29 @@ __device__ void select_from_table(const DT *__restrict__ row, int s0, int s1, in
     prune<SY>(sm, K);
 }
 
-// Scan [s0, s1) of `row` (all kThreads threads of the CTA).  Same contract as scan_slice.
-// `ring` and `tab` are the dynamic shared memory (kRingBytes and kMaxTableBytes).
-// `sums` (block-uniform) says whether the log-sum-exp terms are wanted; one copy of the loop
-// serves both cases so that rows of both kinds share the instruction cache.
+// Log-sum-exp terms of one warp of one slice, as pass 1 leaves them.
+struct WarpPartial {
+    double S, T;
+    float c;
+    int pad;
+};
+
+// Pass 1 over [s0, s1) of `row` (all kThreads threads of the CTA).  Writes the slice's part of
+// the row's table of per-thread tile maxima (`tab` points at the slice's first tile: entry
+// [t][thread]) and, with `sums` (block-uniform), this warp's sums relative to its own reference
+// exponent into wpart[warp] (c = kRefFloor, S = 0 if the warp saw no finite logit).
 template <typename DT>
-__device__ void scan_slice_stream(const DT *__restrict__ row, int s0, int s1, int K, bool sums, ScanSmem &sm,
-                                  StreamBars &bars, unsigned char *ring, DT *tab,
-                                  float &c_out, double &S_out, double &T_out) {
-    using SY = SyncAll;
+__device__ void stream_slice(const DT *__restrict__ row, int s0, int s1, bool sums, StreamBars &bars,
+                             unsigned char *ring, DT *__restrict__ tab, WarpPartial *wpart) {
     constexpr int N = Elem<DT>::N;
     constexpr int VT = kTileBytes / 16;
     static_assert(VT == kThreads * kVpt && tile_elems<DT>() * (int)sizeof(DT) == kTileBytes, "tile geometry");
-    const int tid = threadIdx.x, lane = tid & 31;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int nbytes = (s1 - s0) * (int)sizeof(DT);
     const int ntiles = (nbytes + kTileBytes - 1) / kTileBytes;
     volatile int *abort = &bars.timed_out;
 
     float c = kRefFloor, S = 0.f, T = 0.f;
-    float rm = -CUDART_INF_F;                        // this thread's largest logit so far
 
     // Thread 0 also issues the copies, kStages - 1 tiles ahead of the tile being scanned.
     const char *src = reinterpret_cast<const char *>(row + s0);
@@ -318,7 +318,6 @@ __device__ void scan_slice_stream(const DT *__restrict__ row, int s0, int s1, in
         }
         const float tm = fmaxf(fmaxf(vm[0], vm[1]), fmaxf(vm[2], vm[3]));
         table_store(tab, t * kThreads + tid, tm);
-        rm = fmaxf(rm, tm);
 
         if (sums) {
             const float ts = tm * kLog2e;             // the reference exponent bounds every logit seen
@@ -351,13 +350,55 @@ __device__ void scan_slice_stream(const DT *__restrict__ row, int s0, int s1, in
             T = t0f + t1f;
         }
     }
-    select_from_table<DT, SY>(row, s0, s1, K, ntiles, tab, rm, sm, bars);
-
     if (sums) {
-        reduce_sums<DT, SY>(row, s0, s1, sm, c, S, T, c_out, S_out, T_out);
-    } else {
-        c_out = kRefFloor; S_out = 0.0; T_out = 0.0;
+        // this warp's sums against one reference exponent, in double (shuffles only)
+        const float cw = warp_max(c);
+        const float d = c - cw;
+        const float a = ex2_approx(d);
+        const double Sd = warp_sum((double)(S * a));
+        const double Td = warp_sum((double)((T + S * d) * a));
+        if (lane == 0) {
+            WarpPartial p;
+            p.S = Sd; p.T = Td; p.c = cw; p.pad = 0;
+            wpart[warp] = p;
+        }
     }
+}
+
+// Pass 2: the n = nslices * kWarps warp partials of a row into one (c, S, T), in double and in
+// a fixed order.  Partials without finite logits are skipped.  Block-wide (n <= kThreads).
+template <typename SY>
+__device__ void merge_warp_partials(const WarpPartial *p, int n, ScanSmem &sm, float &c_out, double &S_out,
+                                    double &T_out) {
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    float c = kRefFloor;
+    double S = 0.0, T = 0.0;
+    if (tid < n) {
+        S = __ldcg(&p[tid].S); T = __ldcg(&p[tid].T); c = __ldcg(&p[tid].c);
+    }
+    const bool live = S > 0.0 || !(S == S);          // NaN sums must stay visible
+    float cm = warp_max(live ? c : kRefFloor);
+    if (lane == 0) sm.redc[warp] = cm;
+    SY::sync();
+    cm = sm.redc[0];
+#pragma unroll
+    for (int w = 1; w < kWarps; ++w) cm = fmaxf(cm, sm.redc[w]);
+    double Sm = 0.0, Tm = 0.0;
+    if (S != 0.0) {
+        const double d = (double)c - (double)cm;
+        const double a = exp2(d);
+        Sm = a * S;
+        Tm = a * (T + S * d);
+    }
+    Sm = warp_sum(Sm);
+    Tm = warp_sum(Tm);
+    if (lane == 0) { sm.redS[warp] = Sm; sm.redT[warp] = Tm; }
+    SY::sync();
+    Sm = 0.0; Tm = 0.0;
+#pragma unroll
+    for (int w = 0; w < kWarps; ++w) { Sm += sm.redS[w]; Tm += sm.redT[w]; }
+    SY::sync();
+    c_out = cm; S_out = Sm; T_out = Tm;
 }
 
 // The streaming kernels need more dynamic shared memory than the default limit: raise the limit
@@ -372,19 +413,17 @@ inline cudaError_t allow_ring_smem(KernelT *kernel, RingSmemDone &rec) {
     cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess) return e;
     if (dev >= 0 && dev < 64 && rec.dev[dev]) return cudaSuccess;
-    e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kStreamDynBytes);
+    e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kRingBytes);
     if (e == cudaSuccess && dev >= 0 && dev < 64) rec.dev[dev] = true;
     return e;
 }
 
-// True if rows of this layout can be streamed with bulk copies and a slice of `slice_elems`
-// logits fits the table of tile maxima.
+// True if rows of this layout can be streamed with bulk copies.
 template <typename DT>
-inline bool stream_layout_ok(const void *base, int V, long long stride_b, long long stride_l, int slice_elems) {
+inline bool stream_layout_ok(const void *base, int V, long long stride_b, long long stride_l) {
     const size_t es = sizeof(DT);
     return (reinterpret_cast<uintptr_t>(base) & 15) == 0 && ((size_t)V * es) % 16 == 0 &&
-           ((size_t)stride_b * es) % 16 == 0 && ((size_t)stride_l * es) % 16 == 0 &&
-           slice_elems <= max_stream_tiles<DT>() * tile_elems<DT>();
+           ((size_t)stride_b * es) % 16 == 0 && ((size_t)stride_l * es) % 16 == 0;
 }
 
 }  // namespace dsp

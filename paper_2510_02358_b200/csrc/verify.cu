@@ -1,8 +1,11 @@
 // dsp_verify: verification of the chosen path against the target logits
 // (Sec. 2: Eq. 1 acceptance, residual resampling, Eq. 2 accepted length; greedy = temperature 0).
 //
-// Kernel 1 (target_kernel): every target row is streamed once (argmax; log-sum-exp terms only
-// for stochastic batch rows).  The CTA that finishes the last row of a batch row runs that
+// Every target row is streamed once (argmax; log-sum-exp terms only for stochastic batch rows):
+// 16-byte aligned layouts by target_scan_kernel (one CTA per row slice, no block-wide barrier,
+// see stream_core.cuh) followed by target_rows_kernel (one CTA per row: argmax from the table
+// of tile maxima, sums added up), any other layout by target_kernel (element-wise, slices
+// merged by the CTA arriving last).  The CTA that finishes the last row of a batch row runs that
 // row's left-to-right acceptance scan and either writes the next token (greedy) or records
 // a sampling job (stochastic: residual at the first rejection, or bonus from row m).
 // Kernel 2 (residual_kernel): for each job, one more pass over ONE target row (and ONE draft
@@ -46,6 +49,9 @@ struct VerifyArgs {
     unsigned long long *keys;  // [B*Lt, nslices]
     int32_t *argmax;           // [B*Lt]
     double *tlse64;            // [B*Lt]
+    WarpPartial *wpart;        // [B*Lt, nslices, kWarps]        (streaming path)
+    void *table;               // [B*Lt, ntiles_row, kThreads]   (streaming path), element type of the logits
+    int ntiles_row;            // tiles of a whole row
     SampleJob *jobs;           // [B]
     double *chunk_sums;        // [B, nchunks]
     int nchunks, res_slices, chunks_per_slice;
@@ -128,6 +134,10 @@ __device__ void accept_row(const VerifyArgs &a, int b) {
     }
 }
 
+template <typename DT, typename SY>
+__device__ void target_finish_row(const VerifyArgs &a, ScanSmem &sm, long long row, int b, bool sums,
+                                  unsigned long long best, float c, double S, double T);
+
 // Everything after the scan of one slice of a target row: publish the slice's best key and
 // sums, let the CTA arriving last finish the row (argmax, log-sum-exp), and let the CTA that
 // finishes the last row of a batch row run that row's acceptance scan.
@@ -158,6 +168,16 @@ __device__ void target_finish(const VerifyArgs &a, ScanSmem &sm, long long row, 
             if (sums) merge_partials(part, a.nslices, c, S, T);
         }
     }
+    target_finish_row<DT, SY>(a, sm, row, b, sums, best, c, S, T);
+}
+
+// A target row is complete (thread 0 holds its best key and, with `sums`, its whole-row sums):
+// write argmax and log-sum-exp; the CTA that finishes the last row of a batch row then runs that
+// row's acceptance scan.
+template <typename DT, typename SY>
+__device__ void target_finish_row(const VerifyArgs &a, ScanSmem &sm, long long row, int b, bool sums,
+                                  unsigned long long best, float c, double S, double T) {
+    const int tid = threadIdx.x;
     if (tid == 0) {
         const int am = best ? key_id(best) : 0;
         a.argmax[row] = am;
@@ -200,11 +220,10 @@ __global__ void __launch_bounds__(kThreads, 4) target_kernel(const VerifyArgs a)
     target_finish<DT, SyncAll>(a, sm, row, slice, b, sums, c, S, T, 0u);
 }
 
-// Streaming kernel for 16-byte aligned layouts (see stream_core.cuh).
+// Streaming path, pass 1: one CTA per row slice (see stream_core.cuh).
 template <typename DT>
-__global__ void __launch_bounds__(kThreads, 3) target_stream_kernel(const VerifyArgs a) {
-    extern __shared__ __align__(128) unsigned char dyn[];
-    __shared__ ScanSmem sm;
+__global__ void __launch_bounds__(kThreads, 4) target_scan_kernel(const VerifyArgs a) {
+    extern __shared__ __align__(128) unsigned char ring[];
     __shared__ StreamBars bars;
     const long long row = blockIdx.x / a.nslices;
     const int slice = blockIdx.x - (int)(row * a.nslices);
@@ -213,12 +232,35 @@ __global__ void __launch_bounds__(kThreads, 3) target_stream_kernel(const Verify
     const int s0 = slice * a.slice_elems;
     const int s1 = min(a.V, s0 + a.slice_elems);
     const bool sums = !a.all_greedy && a.mode[b] != 0;
-    stream_begin(sm, bars);
-    DT *tab = reinterpret_cast<DT *>(dyn + kRingBytes);
-    float c;
-    double S, T;
-    scan_slice_stream<DT>(rowp, s0, s1, 1, sums, sm, bars, dyn, tab, c, S, T);
-    target_finish<DT, SyncAll>(a, sm, row, slice, b, sums, c, S, T, bars.timed_out ? DSP_ROW_TIMEOUT : 0u);
+    stream_begin(bars);
+    DT *tab = reinterpret_cast<DT *>(a.table) +
+              (row * a.ntiles_row + (long long)(s0 / tile_elems<DT>())) * kThreads;
+    stream_slice<DT>(rowp, s0, s1, sums, bars, ring, tab, a.wpart + (row * a.nslices + slice) * kWarps);
+    if (threadIdx.x == 0 && bars.timed_out) atomicOr(&a.b_status[b], DSP_ROW_TIMEOUT);
+}
+
+// Streaming path, pass 2: one CTA per row.
+template <typename DT>
+__global__ void __launch_bounds__(kThreads) target_rows_kernel(const VerifyArgs a) {
+    __shared__ ScanSmem sm;
+    const int tid = threadIdx.x;
+    const long long row = blockIdx.x;
+    const int b = (int)(row / a.Lt);
+    const DT *rowp = trow_ptr<DT>(a, row);
+    const bool sums = !a.all_greedy && a.mode[b] != 0;
+    if (tid == 0) { sm.cnt = 0; sm.flag = 0; sm.thrkey = 0ull; sm.thr_v = -CUDART_INF_F; sm.overflow = 0; }
+    float c = kRefFloor;
+    double S = 0.0, T = 0.0;
+    if (sums) {
+        merge_warp_partials<SyncAll>(a.wpart + row * a.nslices * kWarps, a.nslices * kWarps, sm, c, S, T);
+        if (T != T && S == S && S < CUDART_INF) redo_sums<DT, SyncAll>(rowp, 0, a.V, sm, c, S, T);
+    } else {
+        __syncthreads();
+    }
+    select_from_table<DT, SyncAll>(rowp, 0, a.V, 1, a.ntiles_row,
+                                   reinterpret_cast<const DT *>(a.table) + row * a.ntiles_row * kThreads, sm);
+    const unsigned long long best = sm.cnt > 0 ? sm.cand[0] : 0ull;
+    target_finish_row<DT, SyncAll>(a, sm, row, b, sums, best, c, S, T);
 }
 
 // ---- residual / bonus sampling -------------------------------------------------------------
@@ -379,9 +421,9 @@ __global__ void __launch_bounds__(kThreads, 4) residual_kernel(const VerifyArgs 
 
 struct VerifyWs {
     size_t off_row_ticket, off_b_ticket, off_res_ticket, off_b_status, zero_bytes;
-    size_t off_partials, off_keys, off_argmax, off_tlse, off_jobs, off_chunks, total;
+    size_t off_partials, off_keys, off_argmax, off_tlse, off_jobs, off_chunks, off_wpart, off_table, total;
 };
-static VerifyWs verify_ws_layout(int64_t B, int64_t Lt, int nslices, int nchunks) {
+static VerifyWs verify_ws_layout(int64_t B, int64_t Lt, int nslices, int nchunks, int ntiles_row, size_t es) {
     VerifyWs w;
     size_t o = 0;
     w.off_row_ticket = o; o += align_up((size_t)(B * Lt) * 4, 256);
@@ -395,6 +437,8 @@ static VerifyWs verify_ws_layout(int64_t B, int64_t Lt, int nslices, int nchunks
     w.off_tlse = o;       o += align_up((size_t)(B * Lt) * 8, 256);
     w.off_jobs = o;       o += align_up((size_t)B * sizeof(SampleJob), 256);
     w.off_chunks = o;     o += align_up((size_t)B * nchunks * 8, 256);
+    w.off_wpart = o;      o += align_up((size_t)(B * Lt) * nslices * kWarps * sizeof(WarpPartial), 256);
+    w.off_table = o;      o += align_up((size_t)(B * Lt) * ntiles_row * kThreads * es, 256);
     w.total = o;
     return w;
 }
@@ -405,7 +449,8 @@ static int nchunks_of(int V) { return (V + 32 * Elem<DT>::N - 1) / (32 * Elem<DT
 template <typename DT>
 static size_t verify_ws_bytes(int B, int Lt, int V) {
     const SlicePlan plan = plan_slices<DT>((long long)B * Lt, V, kTargetCtas);
-    return verify_ws_layout(B, Lt, plan.nslices, nchunks_of<DT>(V)).total;
+    const int ntiles_row = (V + tile_elems<DT>() - 1) / tile_elems<DT>();
+    return verify_ws_layout(B, Lt, plan.nslices, nchunks_of<DT>(V), ntiles_row, sizeof(DT)).total;
 }
 
 template <typename DT>
@@ -415,7 +460,8 @@ static int32_t launch_verify(VerifyArgs &a, void *workspace, size_t workspace_by
     a.nslices = plan.nslices;
     a.slice_elems = plan.slice_elems;
     a.nchunks = nchunks_of<DT>(a.V);
-    const VerifyWs w = verify_ws_layout(a.B, a.Lt, a.nslices, a.nchunks);
+    a.ntiles_row = (a.V + tile_elems<DT>() - 1) / tile_elems<DT>();
+    const VerifyWs w = verify_ws_layout(a.B, a.Lt, a.nslices, a.nchunks, a.ntiles_row, sizeof(DT));
     if (workspace_bytes < w.total) return DSP_ERR_WORKSPACE;
     char *ws = reinterpret_cast<char *>(workspace);
     a.row_ticket = reinterpret_cast<unsigned *>(ws + w.off_row_ticket);
@@ -427,6 +473,8 @@ static int32_t launch_verify(VerifyArgs &a, void *workspace, size_t workspace_by
     a.argmax = reinterpret_cast<int32_t *>(ws + w.off_argmax);
     a.tlse64 = reinterpret_cast<double *>(ws + w.off_tlse);
     a.jobs = reinterpret_cast<SampleJob *>(ws + w.off_jobs);
+    a.wpart = reinterpret_cast<WarpPartial *>(ws + w.off_wpart);
+    a.table = ws + w.off_table;
     a.chunk_sums = reinterpret_cast<double *>(ws + w.off_chunks);
     // residual pass: about 4 CTAs per SM over all jobs, at least one chunk per warp
     int rsl = (148 * 4 + a.B - 1) / a.B;
@@ -439,10 +487,13 @@ static int32_t launch_verify(VerifyArgs &a, void *workspace, size_t workspace_by
     DSP_CUDA_TRY(cudaMemsetAsync(ws, 0, w.zero_bytes, st));
     const long long nblocks = nrows * a.nslices;
     if (nblocks > 0x7FFFFFFFLL) return DSP_ERR_UNSUPPORTED;
-    if (stream_layout_ok<DT>(a.target, a.V, a.tstride_b, a.tstride_l, a.slice_elems)) {
+    if (a.nslices * kWarps <= kThreads && nrows <= 0x7FFFFFFFLL &&
+        stream_layout_ok<DT>(a.target, a.V, a.tstride_b, a.tstride_l)) {
         static RingSmemDone smem_done;                       // one per element type
-        DSP_CUDA_TRY(allow_ring_smem(target_stream_kernel<DT>, smem_done));
-        target_stream_kernel<DT><<<(unsigned)nblocks, kThreads, kStreamDynBytes, st>>>(a);
+        DSP_CUDA_TRY(allow_ring_smem(target_scan_kernel<DT>, smem_done));
+        target_scan_kernel<DT><<<(unsigned)nblocks, kThreads, kRingBytes, st>>>(a);
+        DSP_CUDA_TRY(cudaGetLastError());
+        target_rows_kernel<DT><<<(unsigned)nrows, kThreads, 0, st>>>(a);
     } else {
         target_kernel<DT><<<(unsigned)nblocks, kThreads, 0, st>>>(a);
     }
