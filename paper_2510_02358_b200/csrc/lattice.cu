@@ -2,13 +2,14 @@
 //
 // Rows whose layout is 16-byte aligned take two kernels: lattice_scan_kernel streams every row
 // slice once from HBM (one CTA per slice, no block-wide barrier: log-sum-exp terms per warp and
-// a table of per-thread tile maxima, see stream_core.cuh); lattice_rows_kernel (one CTA per
-// row) adds up the sums, selects the exact top-K from the table and finalises the row.
+// a table of per-thread tile maxima, see stream_core.cuh); lattice_rows_kernel (one warp per
+// row, see row_warp.cuh) adds up the sums, selects the exact top-K from the table and finalises
+// the row.
 // Any other layout takes lattice_kernel: one CTA streams one slice element-wise and does the
 // top-K on the way; a row split over several CTAs is finished by whichever CTA arrives last
 // (atomic ticket): no CTA waits.  In both paths the CTA that finishes the last row of a batch
 // row also writes gen_len and row_status.
-#include "stream_core.cuh"
+#include "row_warp.cuh"
 
 namespace dsp {
 
@@ -228,22 +229,96 @@ __global__ void __launch_bounds__(kThreads, 4) lattice_scan_kernel(const Lattice
     if (threadIdx.x == 0 && bars.timed_out) atomicOr(&a.b_status[b], DSP_ROW_TIMEOUT);
 }
 
-// Streaming path, pass 2: one CTA per row.
+// Streaming path, pass 2: one warp per row (see row_warp.cuh): add up the row's sums, select
+// its exact top-K from the table, finalise it (log-sum-exp, entropy, Eq. 7 count, EOS slot,
+// candidate outputs); the warp that finishes the last row of a batch row also writes gen_len
+// (Eq. 9) and row_status.
 template <typename DT>
 __global__ void __launch_bounds__(kThreads) lattice_rows_kernel(const LatticeArgs a) {
-    __shared__ ScanSmem sm;
-    const int tid = threadIdx.x;
-    const long long row = blockIdx.x;
+    __shared__ WarpScratch scratch[kRowWarps];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const long long row = (long long)blockIdx.x * kRowWarps + warp;
+    if (row >= (long long)a.B * a.L) return;
     const int b = (int)(row / a.L), l = (int)(row - (long long)b * a.L);
     const DT *rowp = reinterpret_cast<const DT *>(a.logits) + b * a.stride_b + l * a.stride_l;
-    if (tid == 0) { sm.cnt = 0; sm.flag = 0; sm.thrkey = 0ull; sm.thr_v = -CUDART_INF_F; sm.overflow = 0; }
+
     float c;
     double S, T;
-    merge_warp_partials<SyncAll>(a.wpart + row * a.nslices * kWarps, a.nslices * kWarps, sm, c, S, T);
-    if (T != T && S == S && S < CUDART_INF) redo_sums<DT, SyncAll>(rowp, 0, a.V, sm, c, S, T);
-    select_from_table<DT, SyncAll>(rowp, 0, a.V, a.K, a.ntiles_row,
-                                   reinterpret_cast<const DT *>(a.table) + row * a.ntiles_row * kThreads, sm);
-    lattice_finalise<DT, SyncAll>(a, sm, row, b, rowp, c, S, T);
+    warp_merge_partials(a.wpart + row * a.nslices * kWarps, a.nslices * kWarps, lane, c, S, T);
+    if (T != T && S == S && S < CUDART_INF) warp_redo_sums<DT>(rowp, a.V, lane, c, S, T);
+    const unsigned long long key = warp_select_topk<DT>(
+        rowp, a.V, a.K, reinterpret_cast<const DT *>(a.table) + row * a.ntiles_row * kThreads, a.ntiles_row,
+        scratch[warp], lane);
+    const int nk = __popc(__ballot_sync(0xFFFFFFFFu, key != 0ull && lane < a.K));
+
+    double lse, mean_x;
+    const bool ok = row_log_stats(c, S, T, lse, mean_x) && nk > 0;
+    int count = nk;
+    if (a.tau > 0.f && a.tau <= 1.f && ok) {           // Eq. 7 on full-vocabulary probabilities
+        const double p = lane < nk ? exp((double)key_value(key) - lse) : 0.0;
+        const double tau = (double)a.tau;
+        double cum = 0.0;
+        bool found = false;
+        for (int k = 0; k < nk; ++k) {                 // in rank order, every lane alike
+            cum += __shfl_sync(0xFFFFFFFFu, p, k);
+            if (!found && cum >= tau) { count = k + 1; found = true; }
+        }
+    }
+    int eos_slot = -1;
+    float eos_x = 0.f;
+    if (a.eos_id >= 0 && a.eos_id < a.V) {              // always keep EOS
+        const bool has = __ballot_sync(0xFFFFFFFFu, lane < count && key_id(key) == a.eos_id) != 0u;
+        if (!has) {
+            eos_x = Elem<DT>::load1(rowp + a.eos_id);
+            if (eos_x > -CUDART_INF_F && eos_x < CUDART_INF_F) eos_slot = count;
+        }
+    }
+    if (lane == 0) {
+        a.cand_count[row] = count + (eos_slot >= 0 ? 1 : 0);
+        if (a.lse) a.lse[row] = (float)lse;
+        a.lse64[row] = lse;
+        if (a.entropy) a.entropy[row] = (float)(lse - mean_x);
+        if (!ok) atomicOr(&a.b_status[b], DSP_ROW_NONFINITE_INPUT);
+    }
+    for (int slot = lane; slot < a.KC; slot += 32) {      // slot 32 can only be the EOS slot
+        const unsigned long long ks = key;                  // slot == lane whenever slot < count <= 32
+        int id = -1;
+        float x = -CUDART_INF_F, lp = -CUDART_INF_F;
+        if (slot < count) {
+            id = key_id(ks);
+            x = key_value(ks);
+            lp = (float)((double)x - lse);
+        } else if (slot == eos_slot) {
+            id = a.eos_id;
+            x = eos_x;
+            lp = (float)((double)x - lse);
+        }
+        const long long o = row * a.KC + slot;
+        a.cand_id[o] = id;
+        a.cand_logit[o] = x;
+        a.cand_logp[o] = lp;
+    }
+    // ---- last row of this batch row: generation length (Eq. 9) and status ----
+    __threadfence();
+    __syncwarp();
+    unsigned ticket = 0;
+    if (lane == 0) ticket = atomicAdd(&a.b_ticket[b], 1u);
+    ticket = __shfl_sync(0xFFFFFFFFu, ticket, 0);
+    if (ticket != (unsigned)a.L - 1) return;
+    __threadfence();
+    int g = a.L;
+    if (a.eos_id >= 0) {
+        for (int i0 = 0; i0 < a.L && g == a.L; i0 += 32) {
+            const int i = i0 + lane;
+            const bool eos = i < a.L && __ldcg(&a.cand_id[((long long)b * a.L + i) * a.KC]) == a.eos_id;
+            const unsigned m = __ballot_sync(0xFFFFFFFFu, eos);
+            if (m) g = i0 + __ffs(m) - 1;
+        }
+    }
+    if (lane == 0) {
+        a.gen_len[b] = g;
+        a.row_status[b] = atomicOr(&a.b_status[b], 0u);
+    }
 }
 
 template <typename DT>
@@ -272,7 +347,7 @@ static int32_t launch_lattice(LatticeArgs &a, void *workspace, size_t workspace_
         DSP_CUDA_TRY(allow_ring_smem(lattice_scan_kernel<DT>, smem_done));
         lattice_scan_kernel<DT><<<(unsigned)nblocks, kThreads, kRingBytes, st>>>(a);
         DSP_CUDA_TRY(cudaGetLastError());
-        lattice_rows_kernel<DT><<<(unsigned)nrows, kThreads, 0, st>>>(a);
+        lattice_rows_kernel<DT><<<(unsigned)((nrows + kRowWarps - 1) / kRowWarps), kThreads, 0, st>>>(a);
     } else {
         lattice_kernel<DT><<<(unsigned)nblocks, kThreads, 0, st>>>(a);
     }

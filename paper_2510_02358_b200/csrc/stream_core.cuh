@@ -9,11 +9,9 @@
 // and thread, the largest logit of the thread's kVpt vectors of that tile, and per slice and
 // warp the log-sum-exp terms.
 //
-// Pass 2 (one CTA per row, run by the kernels in lattice.cu / verify.cu): merge_warp_partials
-// adds up the sums, select_from_table picks the exact top-K: a threshold with at least K
-// logits at or above it, the exact K-th largest table entry among those that reach it, and a
-// second look (L2 hits) at the few (tile, thread) shares whose maximum reaches that value.
-// Results are the same as scan_slice's (scan_core.cuh).
+// Pass 2 (one warp per row, row_warp.cuh, run by the kernels in lattice.cu / verify.cu) adds up
+// the sums and picks the exact top-K from the table.  Results are the same as scan_slice's
+// (scan_core.cuh).
 #pragma once
 
 #include "scan_core.cuh"
@@ -135,120 +133,6 @@ __device__ __forceinline__ void table_store(__nv_bfloat16 *tab, int i, float v) 
 }
 __device__ __forceinline__ void table_store(float *tab, int i, float v) { tab[i] = v; }
 
-// First threshold from one value per thread (its largest logit): with r = ceil(K / #warps), the
-// smallest over the warps of each warp's r-th largest value has K distinct logits at or above
-// it.  One barrier; every thread derives the value itself.  If some warp has fewer than r finite
-// values (masked rows) the general rule of bootstrap_threshold applies (two more barriers).
-template <typename SY>
-__device__ __forceinline__ float bootstrap_threshold_fast(ScanSmem &sm, float tm, int K) {
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const float s = bitonic_desc(tm == tm ? tm : -CUDART_INF_F, lane);
-    sm.wsorted[warp][lane] = s;
-    SY::sync();
-    const int r = (K + kWarps - 1) / kWarps;
-    float t = CUDART_INF_F;
-#pragma unroll
-    for (int w = 0; w < kWarps; ++w) t = fminf(t, sm.wsorted[w][r - 1]);
-    if (t > -CUDART_INF_F) return t;
-    SY::sync();
-    if (tid == 0) {
-        float g = -CUDART_INF_F;
-        for (int rr = 1; rr <= 32; ++rr) {
-            int nw = 0;
-            float lo = CUDART_INF_F;
-            for (int w = 0; w < kWarps; ++w) {
-                const float x = sm.wsorted[w][rr - 1];
-                if (x > -CUDART_INF_F) { ++nw; lo = fminf(lo, x); }
-            }
-            if (nw == 0) break;
-            if (rr * nw >= K) { g = lo; break; }
-        }
-        sm.thr_v = g;
-    }
-    SY::sync();
-    return sm.thr_v;
-}
-
-// Exact top-K of [s0, s1) of `row` from its table of per-thread tile maxima (`tab`, ntiles x
-// kThreads, entry [t][thread], in global memory).  On return sm.cand[0 .. sm.cnt) holds the best
-// min(K, #finite) keys, sorted (after a barrier).  Rows with very many equal top values overflow
-// the lists and take topk_careful instead.  Block-wide; sm.cnt and sm.flag must be 0 on entry
-// (before a barrier).
-template <typename DT, typename SY>
-__device__ void select_from_table(const DT *__restrict__ row, int s0, int s1, int K, int ntiles,
-                                  const DT *tab, ScanSmem &sm) {
-    constexpr int N = Elem<DT>::N;
-    constexpr int TE = tile_elems<DT>();
-    constexpr int kHalf = kCandCap / 2;              // element keys first, table entries in the upper half
-    const int tid = threadIdx.x;
-    // 1. a threshold with at least K table entries at or above it, from each thread's largest
-    float rm = -CUDART_INF_F;
-    for (int t = 0; t < ntiles; ++t) rm = fmaxf(rm, Elem<DT>::load1(tab + t * kThreads + tid));
-    const float t0 = bootstrap_threshold_fast<SY>(sm, rm, K);
-    // 2. the table entries that reach it (each thread looks at its own column)
-    for (int t = 0; t < ntiles; ++t) {
-        const float v = Elem<DT>::load1(tab + t * kThreads + tid);
-        if (v >= t0 && v > -CUDART_INF_F) {
-            const int pos = atomicAdd(&sm.cnt, 1);
-            if (pos < kHalf) sm.cand[kHalf + pos] = make_key(v, t * kThreads + tid);
-        }
-    }
-    SY::sync();
-    const int n = sm.cnt;
-    if (n > kHalf) {                                 // block-uniform
-        topk_careful<DT, SY>(row, s0, s1, K, sm);
-        return;
-    }
-    // 3. the K-th largest of them (all of them if there are fewer than K), by counting
-    const int kk = min(K, n);
-    const unsigned long long *entries = sm.cand + kHalf;
-    for (int i = tid; i < n; i += kThreads) {
-        const unsigned long long key = entries[i];
-        int rank = 0;
-        for (int j = 0; j < n; ++j) rank += entries[j] > key;
-        if (rank == kk - 1) sm.thrkey = key;
-    }
-    SY::sync();
-    // 4. the shares whose maximum reaches that value hold every logit of the slice's top K:
-    //    look at their logits again and list those that reach it
-    if (n > 0) {
-        // with fewer than K entries (the threshold was -inf: every finite entry is listed) every
-        // finite logit of the listed shares is wanted
-        const float tk = n >= K ? key_value(sm.thrkey) : -CUDART_INF_F;
-        for (int i = tid; i < n; i += kThreads) {
-            const unsigned long long key = entries[i];
-            if (key_value(key) >= tk) {
-                const int id = key_id(key);
-                const int e00 = s0 + (id / kThreads) * TE + (id % kThreads) * N;
-#pragma unroll
-                for (int j = 0; j < kVpt; ++j) {
-                    const int e0 = e00 + j * kThreads * N;
-                    if (e0 < s1) {                   // vectors are whole: the row length is a multiple of N
-                        const uint4 v = ldg_stream(row + e0);
-#pragma unroll
-                        for (int e = 0; e < N; ++e) {
-                            const float x = Elem<DT>::get(v, e);
-                            if (x >= tk && x > -CUDART_INF_F) {
-                                const int pos = atomicAdd(&sm.flag, 1);
-                                if (pos < kHalf) sm.cand[pos] = make_key(x, e0 + e);
-                            }
-                        }
-                    }
-                }
-            }
-        }
-    }
-    SY::sync();
-    const int n2 = sm.flag;
-    if (n2 > kHalf) {                                // block-uniform
-        topk_careful<DT, SY>(row, s0, s1, K, sm);
-        return;
-    }
-    // 5. the best K of the listed logits, sorted, to the front
-    if (tid == 0) sm.cnt = n2;
-    prune<SY>(sm, K);
-}
-
 // Log-sum-exp terms of one warp of one slice, as pass 1 leaves them.
 struct WarpPartial {
     double S, T;
@@ -363,42 +247,6 @@ __device__ void stream_slice(const DT *__restrict__ row, int s0, int s1, bool su
             wpart[warp] = p;
         }
     }
-}
-
-// Pass 2: the n = nslices * kWarps warp partials of a row into one (c, S, T), in double and in
-// a fixed order.  Partials without finite logits are skipped.  Block-wide (n <= kThreads).
-template <typename SY>
-__device__ void merge_warp_partials(const WarpPartial *p, int n, ScanSmem &sm, float &c_out, double &S_out,
-                                    double &T_out) {
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    float c = kRefFloor;
-    double S = 0.0, T = 0.0;
-    if (tid < n) {
-        S = __ldcg(&p[tid].S); T = __ldcg(&p[tid].T); c = __ldcg(&p[tid].c);
-    }
-    const bool live = S > 0.0 || !(S == S);          // NaN sums must stay visible
-    float cm = warp_max(live ? c : kRefFloor);
-    if (lane == 0) sm.redc[warp] = cm;
-    SY::sync();
-    cm = sm.redc[0];
-#pragma unroll
-    for (int w = 1; w < kWarps; ++w) cm = fmaxf(cm, sm.redc[w]);
-    double Sm = 0.0, Tm = 0.0;
-    if (S != 0.0) {
-        const double d = (double)c - (double)cm;
-        const double a = exp2(d);
-        Sm = a * S;
-        Tm = a * (T + S * d);
-    }
-    Sm = warp_sum(Sm);
-    Tm = warp_sum(Tm);
-    if (lane == 0) { sm.redS[warp] = Sm; sm.redT[warp] = Tm; }
-    SY::sync();
-    Sm = 0.0; Tm = 0.0;
-#pragma unroll
-    for (int w = 0; w < kWarps; ++w) { Sm += sm.redS[w]; Tm += sm.redT[w]; }
-    SY::sync();
-    c_out = cm; S_out = Sm; T_out = Tm;
 }
 
 // The streaming kernels need more dynamic shared memory than the default limit: raise the limit

@@ -3,14 +3,14 @@
 //
 // Every target row is streamed once (argmax; log-sum-exp terms only for stochastic batch rows):
 // 16-byte aligned layouts by target_scan_kernel (one CTA per row slice, no block-wide barrier,
-// see stream_core.cuh) followed by target_rows_kernel (one CTA per row: argmax from the table
+// see stream_core.cuh) followed by target_rows_kernel (one warp per row: argmax from the table
 // of tile maxima, sums added up), any other layout by target_kernel (element-wise, slices
 // merged by the CTA arriving last).  The CTA that finishes the last row of a batch row runs that
 // row's left-to-right acceptance scan and either writes the next token (greedy) or records
 // a sampling job (stochastic: residual at the first rejection, or bonus from row m).
 // Kernel 2 (residual_kernel): for each job, one more pass over ONE target row (and ONE draft
 // row): per-chunk sums of max(0, p - q) in token order; the CTA arriving last inverts the CDF.
-#include "stream_core.cuh"
+#include "row_warp.cuh"
 
 namespace dsp {
 
@@ -239,28 +239,50 @@ __global__ void __launch_bounds__(kThreads, 4) target_scan_kernel(const VerifyAr
     if (threadIdx.x == 0 && bars.timed_out) atomicOr(&a.b_status[b], DSP_ROW_TIMEOUT);
 }
 
-// Streaming path, pass 2: one CTA per row.
+// Streaming path, pass 2: one warp per row (see row_warp.cuh): argmax from the table of tile
+// maxima, log-sum-exp from the warp sums; the warp that finishes the last row of a batch row
+// runs that row's acceptance scan.
 template <typename DT>
 __global__ void __launch_bounds__(kThreads) target_rows_kernel(const VerifyArgs a) {
-    __shared__ ScanSmem sm;
-    const int tid = threadIdx.x;
-    const long long row = blockIdx.x;
+    __shared__ WarpScratch scratch[kRowWarps];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const long long row = (long long)blockIdx.x * kRowWarps + warp;
+    if (row >= (long long)a.B * a.Lt) return;
     const int b = (int)(row / a.Lt);
     const DT *rowp = trow_ptr<DT>(a, row);
     const bool sums = !a.all_greedy && a.mode[b] != 0;
-    if (tid == 0) { sm.cnt = 0; sm.flag = 0; sm.thrkey = 0ull; sm.thr_v = -CUDART_INF_F; sm.overflow = 0; }
     float c = kRefFloor;
     double S = 0.0, T = 0.0;
     if (sums) {
-        merge_warp_partials<SyncAll>(a.wpart + row * a.nslices * kWarps, a.nslices * kWarps, sm, c, S, T);
-        if (T != T && S == S && S < CUDART_INF) redo_sums<DT, SyncAll>(rowp, 0, a.V, sm, c, S, T);
-    } else {
-        __syncthreads();
+        warp_merge_partials(a.wpart + row * a.nslices * kWarps, a.nslices * kWarps, lane, c, S, T);
+        if (T != T && S == S && S < CUDART_INF) warp_redo_sums<DT>(rowp, a.V, lane, c, S, T);
     }
-    select_from_table<DT, SyncAll>(rowp, 0, a.V, 1, a.ntiles_row,
-                                   reinterpret_cast<const DT *>(a.table) + row * a.ntiles_row * kThreads, sm);
-    const unsigned long long best = sm.cnt > 0 ? sm.cand[0] : 0ull;
-    target_finish_row<DT, SyncAll>(a, sm, row, b, sums, best, c, S, T);
+    const unsigned long long key = warp_select_topk<DT>(
+        rowp, a.V, 1, reinterpret_cast<const DT *>(a.table) + row * a.ntiles_row * kThreads, a.ntiles_row,
+        scratch[warp], lane);
+    const unsigned long long best = __shfl_sync(0xFFFFFFFFu, key, 0);
+    unsigned ticket = 0;
+    if (lane == 0) {
+        const int am = best ? key_id(best) : 0;
+        a.argmax[row] = am;
+        if (a.tgt_argmax) a.tgt_argmax[row] = am;
+        bool ok = best != 0ull;
+        if (sums) {
+            double lse, mean_x;
+            ok = row_log_stats(c, S, T, lse, mean_x) && ok;
+            a.tlse64[row] = lse;
+            if (a.tgt_lse) a.tgt_lse[row] = (float)lse;
+        } else if (a.tgt_lse && !a.all_greedy) {
+            a.tgt_lse[row] = CUDART_NAN_F;             // greedy row of a mixed batch: not computed
+        }
+        if (!ok) atomicOr(&a.b_status[b], DSP_ROW_NONFINITE_INPUT);
+        __threadfence();
+        ticket = atomicAdd(&a.b_ticket[b], 1u);
+    }
+    ticket = __shfl_sync(0xFFFFFFFFu, ticket, 0);
+    if (ticket != (unsigned)a.Lt - 1) return;
+    __threadfence();
+    accept_row<DT>(a, b);
 }
 
 // ---- residual / bonus sampling -------------------------------------------------------------
@@ -493,7 +515,7 @@ static int32_t launch_verify(VerifyArgs &a, void *workspace, size_t workspace_by
         DSP_CUDA_TRY(allow_ring_smem(target_scan_kernel<DT>, smem_done));
         target_scan_kernel<DT><<<(unsigned)nblocks, kThreads, kRingBytes, st>>>(a);
         DSP_CUDA_TRY(cudaGetLastError());
-        target_rows_kernel<DT><<<(unsigned)nrows, kThreads, 0, st>>>(a);
+        target_rows_kernel<DT><<<(unsigned)((nrows + kRowWarps - 1) / kRowWarps), kThreads, 0, st>>>(a);
     } else {
         target_kernel<DT><<<(unsigned)nblocks, kThreads, 0, st>>>(a);
     }
