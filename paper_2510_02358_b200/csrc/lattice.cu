@@ -37,7 +37,7 @@ struct LatticeArgs {
     SlicePartial *partials;   // [B*L, nslices]               (element-wise path)
     unsigned long long *keys; // [B*L, nslices, K]            (element-wise path)
     WarpPartial *wpart;       // [B*L, nslices, kWarps]       (streaming path)
-    void *table;              // [B*L, ntiles_row, kThreads]  (streaming path), element type of the logits
+    void *table;              // [B*L, ntiles_row + nslices, kThreads]  (streaming path), element type of the logits
     int ntiles_row;           // tiles of a whole row
 };
 
@@ -58,7 +58,7 @@ static LatticeWs lattice_ws_layout(int64_t B, int64_t L, int nslices, int K, int
     w.off_keys = o;       o += align_up((size_t)(B * L) * nslices * K * 8, 256);
     size_t o2 = w.zero_bytes;
     w.off_wpart = o2;     o2 += align_up((size_t)(B * L) * nslices * kWarps * sizeof(WarpPartial), 256);
-    w.off_table = o2;     o2 += align_up((size_t)(B * L) * ntiles_row * kThreads * es, 256);
+    w.off_table = o2;     o2 += align_up((size_t)(B * L) * (ntiles_row + nslices) * kThreads * es, 256);
     w.total = o > o2 ? o : o2;
     return w;
 }
@@ -223,9 +223,10 @@ __global__ void __launch_bounds__(kThreads, 4) lattice_scan_kernel(const Lattice
     const int s0 = slice * a.slice_elems;
     const int s1 = min(a.V, s0 + a.slice_elems);
     stream_begin(bars);
-    DT *tab = reinterpret_cast<DT *>(a.table) +
-              (row * a.ntiles_row + (long long)(s0 / tile_elems<DT>())) * kThreads;
-    stream_slice<DT>(rowp, s0, s1, true, bars, ring, tab, a.wpart + (row * a.nslices + slice) * kWarps);
+    DT *trow = reinterpret_cast<DT *>(a.table) + row * (a.ntiles_row + a.nslices) * kThreads;   // the row's table
+    DT *tab = trow + (long long)(s0 / tile_elems<DT>()) * kThreads;
+    DT *smax = trow + (long long)(a.ntiles_row + slice) * kThreads;
+    stream_slice<DT>(rowp, s0, s1, true, bars, ring, tab, smax, a.wpart + (row * a.nslices + slice) * kWarps);
     if (threadIdx.x == 0 && bars.timed_out) atomicOr(&a.b_status[b], DSP_ROW_TIMEOUT);
 }
 
@@ -247,8 +248,8 @@ __global__ void __launch_bounds__(kThreads) lattice_rows_kernel(const LatticeArg
     warp_merge_partials(a.wpart + row * a.nslices * kWarps, a.nslices * kWarps, lane, c, S, T);
     if (T != T && S == S && S < CUDART_INF) warp_redo_sums<DT>(rowp, a.V, lane, c, S, T);
     const unsigned long long key = warp_select_topk<DT>(
-        rowp, a.V, a.K, reinterpret_cast<const DT *>(a.table) + row * a.ntiles_row * kThreads, a.ntiles_row,
-        scratch[warp], lane);
+        rowp, a.V, a.K, reinterpret_cast<const DT *>(a.table) + row * (a.ntiles_row + a.nslices) * kThreads, a.ntiles_row,
+        a.nslices, scratch[warp], lane);
     const int nk = __popc(__ballot_sync(0xFFFFFFFFu, key != 0ull && lane < a.K));
 
     double lse, mean_x;

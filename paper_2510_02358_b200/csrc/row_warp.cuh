@@ -129,40 +129,56 @@ __device__ unsigned long long warp_topk_careful(const DT *__restrict__ row, int 
 // Exact top-K of a row from its table of per-thread tile maxima (`tab`, ntiles x kThreads, entry
 // [t][thread], in global memory) by one warp.  Returns the best 32 keys, one per lane,
 // descending (0 = none): the first min(K, #finite) are the row's top K.
-//  1. every lane takes 8 table columns; the K-th largest of the lanes' maxima has at least K
-//     logits at or above it (-inf if fewer than K lanes saw a finite logit);
+//  1. every lane takes 8 table columns; the K-th largest of the lanes' maxima (from the slices'
+//     per-thread maxima that pass 1 left after the table's ntiles rows) has at least K logits at
+//     or above it (-inf if fewer than K lanes saw a finite logit);
 //  2. the (tile, thread) shares whose maximum reaches it are listed, then looked at again, one
 //     share per lane (from global memory: L2 hits), and their logits that reach it are listed;
 //  3. the list holds the whole top K: it is sorted 32 keys at a time and merged.
 // A list that overflows (very many equal top values) sends the row to warp_topk_careful.
 template <typename DT>
 __device__ unsigned long long warp_select_topk(const DT *__restrict__ row, int V, int K, const DT *tab, int ntiles,
-                                               WarpScratch &ws, int lane) {
+                                               int nslices, WarpScratch &ws, int lane) {
     constexpr int N = Elem<DT>::N;
     constexpr int TE = tile_elems<DT>();
     constexpr int VPL = 8 / N;                   // 16-byte vectors holding a lane's 8 table columns
     if (lane == 0) { ws.nkeys = 0; ws.nshares = 0; }
-    float rm = -CUDART_INF_F;
-    for (int t = 0; t < ntiles; ++t) {
+    float rm = -CUDART_INF_F;                    // over the slices' per-thread maxima (the table's last rows)
+    for (int sl = 0; sl < nslices; ++sl) {
 #pragma unroll
         for (int q = 0; q < VPL; ++q) {
-            const uint4 v = __ldcg(reinterpret_cast<const uint4 *>(tab + t * kThreads + lane * 8 + q * N));
+            const uint4 v = __ldcg(reinterpret_cast<const uint4 *>(tab + (ntiles + sl) * kThreads + lane * 8 + q * N));
 #pragma unroll
             for (int e = 0; e < N; ++e) rm = fmaxf(rm, Elem<DT>::get(v, e));
         }
     }
     const float t0 = __shfl_sync(0xFFFFFFFFu, bitonic_desc(rm, lane), K - 1);
     __syncwarp();
-    for (int t = 0; t < ntiles; ++t) {
+    constexpr int kBatch = 8;                    // tiles whose table vectors are in flight together
+    for (int tb = 0; tb < ntiles; tb += kBatch) {
+        uint4 v[kBatch][VPL];
 #pragma unroll
-        for (int q = 0; q < VPL; ++q) {
-            const uint4 v = __ldcg(reinterpret_cast<const uint4 *>(tab + t * kThreads + lane * 8 + q * N));
+        for (int u = 0; u < kBatch; ++u) {
 #pragma unroll
-            for (int e = 0; e < N; ++e) {
-                const float m = Elem<DT>::get(v, e);
-                if (m >= t0 && m > -CUDART_INF_F) {
-                    const int pos = atomicAdd(&ws.nshares, 1);
-                    if (pos < kWarpShareCap) ws.shares[pos] = (uint32_t)(t * kThreads + lane * 8 + q * N + e);
+            for (int q = 0; q < VPL; ++q) {
+                if (tb + u < ntiles)
+                    v[u][q] = __ldcg(reinterpret_cast<const uint4 *>(tab + (tb + u) * kThreads + lane * 8 + q * N));
+            }
+        }
+#pragma unroll
+        for (int u = 0; u < kBatch; ++u) {
+            if (tb + u < ntiles) {
+#pragma unroll
+                for (int q = 0; q < VPL; ++q) {
+#pragma unroll
+                    for (int e = 0; e < N; ++e) {
+                        const float m = Elem<DT>::get(v[u][q], e);
+                        if (m >= t0 && m > -CUDART_INF_F) {
+                            const int pos = atomicAdd(&ws.nshares, 1);
+                            if (pos < kWarpShareCap)
+                                ws.shares[pos] = (uint32_t)((tb + u) * kThreads + lane * 8 + q * N + e);
+                        }
+                    }
                 }
             }
         }

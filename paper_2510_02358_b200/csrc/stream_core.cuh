@@ -142,11 +142,12 @@ struct WarpPartial {
 
 // Pass 1 over [s0, s1) of `row` (all kThreads threads of the CTA).  Writes the slice's part of
 // the row's table of per-thread tile maxima (`tab` points at the slice's first tile: entry
-// [t][thread]) and, with `sums` (block-uniform), this warp's sums relative to its own reference
-// exponent into wpart[warp] (c = kRefFloor, S = 0 if the warp saw no finite logit).
+// [t][thread]), every thread's largest logit of the whole slice (smax[thread]) and, with `sums`
+// (block-uniform), this warp's sums relative to its own reference exponent into wpart[warp]
+// (c = kRefFloor, S = 0 if the warp saw no finite logit).
 template <typename DT>
 __device__ void stream_slice(const DT *__restrict__ row, int s0, int s1, bool sums, StreamBars &bars,
-                             unsigned char *ring, DT *__restrict__ tab, WarpPartial *wpart) {
+                             unsigned char *ring, DT *__restrict__ tab, DT *__restrict__ smax, WarpPartial *wpart) {
     constexpr int N = Elem<DT>::N;
     constexpr int VT = kTileBytes / 16;
     static_assert(VT == kThreads * kVpt && tile_elems<DT>() * (int)sizeof(DT) == kTileBytes, "tile geometry");
@@ -156,6 +157,7 @@ __device__ void stream_slice(const DT *__restrict__ row, int s0, int s1, bool su
     volatile int *abort = &bars.timed_out;
 
     float c = kRefFloor, S = 0.f, T = 0.f;
+    float rm = -CUDART_INF_F;                        // this thread's largest logit so far
 
     // Thread 0 also issues the copies, kStages - 1 tiles ahead of the tile being scanned.
     const char *src = reinterpret_cast<const char *>(row + s0);
@@ -202,6 +204,7 @@ __device__ void stream_slice(const DT *__restrict__ row, int s0, int s1, bool su
         }
         const float tm = fmaxf(fmaxf(vm[0], vm[1]), fmaxf(vm[2], vm[3]));
         table_store(tab, t * kThreads + tid, tm);
+        rm = fmaxf(rm, tm);
 
         if (sums) {
             const float ts = tm * kLog2e;             // the reference exponent bounds every logit seen
@@ -234,6 +237,7 @@ __device__ void stream_slice(const DT *__restrict__ row, int s0, int s1, bool su
             T = t0f + t1f;
         }
     }
+    table_store(smax, tid, rm);
     if (sums) {
         // this warp's sums against one reference exponent, in double (shuffles only)
         const float cw = warp_max(c);

@@ -50,7 +50,7 @@ struct VerifyArgs {
     int32_t *argmax;           // [B*Lt]
     double *tlse64;            // [B*Lt]
     WarpPartial *wpart;        // [B*Lt, nslices, kWarps]        (streaming path)
-    void *table;               // [B*Lt, ntiles_row, kThreads]   (streaming path), element type of the logits
+    void *table;               // [B*Lt, ntiles_row + nslices, kThreads]  (streaming path), element type of the logits
     int ntiles_row;            // tiles of a whole row
     SampleJob *jobs;           // [B]
     double *chunk_sums;        // [B, nchunks]
@@ -233,9 +233,10 @@ __global__ void __launch_bounds__(kThreads, 4) target_scan_kernel(const VerifyAr
     const int s1 = min(a.V, s0 + a.slice_elems);
     const bool sums = !a.all_greedy && a.mode[b] != 0;
     stream_begin(bars);
-    DT *tab = reinterpret_cast<DT *>(a.table) +
-              (row * a.ntiles_row + (long long)(s0 / tile_elems<DT>())) * kThreads;
-    stream_slice<DT>(rowp, s0, s1, sums, bars, ring, tab, a.wpart + (row * a.nslices + slice) * kWarps);
+    DT *trow = reinterpret_cast<DT *>(a.table) + row * (a.ntiles_row + a.nslices) * kThreads;   // the row's table
+    DT *tab = trow + (long long)(s0 / tile_elems<DT>()) * kThreads;
+    DT *smax = trow + (long long)(a.ntiles_row + slice) * kThreads;
+    stream_slice<DT>(rowp, s0, s1, sums, bars, ring, tab, smax, a.wpart + (row * a.nslices + slice) * kWarps);
     if (threadIdx.x == 0 && bars.timed_out) atomicOr(&a.b_status[b], DSP_ROW_TIMEOUT);
 }
 
@@ -258,8 +259,8 @@ __global__ void __launch_bounds__(kThreads) target_rows_kernel(const VerifyArgs 
         if (T != T && S == S && S < CUDART_INF) warp_redo_sums<DT>(rowp, a.V, lane, c, S, T);
     }
     const unsigned long long key = warp_select_topk<DT>(
-        rowp, a.V, 1, reinterpret_cast<const DT *>(a.table) + row * a.ntiles_row * kThreads, a.ntiles_row,
-        scratch[warp], lane);
+        rowp, a.V, 1, reinterpret_cast<const DT *>(a.table) + row * (a.ntiles_row + a.nslices) * kThreads, a.ntiles_row,
+        a.nslices, scratch[warp], lane);
     const unsigned long long best = __shfl_sync(0xFFFFFFFFu, key, 0);
     unsigned ticket = 0;
     if (lane == 0) {
@@ -460,7 +461,7 @@ static VerifyWs verify_ws_layout(int64_t B, int64_t Lt, int nslices, int nchunks
     w.off_jobs = o;       o += align_up((size_t)B * sizeof(SampleJob), 256);
     w.off_chunks = o;     o += align_up((size_t)B * nchunks * 8, 256);
     w.off_wpart = o;      o += align_up((size_t)(B * Lt) * nslices * kWarps * sizeof(WarpPartial), 256);
-    w.off_table = o;      o += align_up((size_t)(B * Lt) * ntiles_row * kThreads * es, 256);
+    w.off_table = o;      o += align_up((size_t)(B * Lt) * (ntiles_row + nslices) * kThreads * es, 256);
     w.total = o;
     return w;
 }
