@@ -68,9 +68,23 @@ enum dsp_dtype { DSP_F32 = 0, DSP_BF16 = 1 };
 #define DSP_MAX_W 32      /* largest beam width */
 #define DSP_MAX_L 1024    /* largest draft length */
 
+/* Kernels whose launch dsp_profile_events can bracket with events. */
+enum dsp_profile_point {
+    DSP_PROFILE_LATTICE_SCAN = 0,   /* the pass over the draft logits inside dsp_lattice_build */
+    DSP_PROFILE_TARGET_SCAN = 1     /* the pass over the target logits inside dsp_verify */
+};
+
 const char *dsp_strerror(int32_t status);   /* host; static string */
 int32_t dsp_last_cuda_error(void);          /* host; the cudaError_t behind the last DSP_ERR_CUDA */
 int32_t dsp_version(void);                  /* host; ABI version, currently 1 */
+
+/* Measurement aid (host; not thread-safe; no counterpart in the paper).  While `start` and
+ * `stop` (caller-owned cudaEvent_t handles created with timing enabled) are set for a point,
+ * every later call that launches that kernel records `start` right before and `stop` right
+ * after the launch on the call's stream, so that cudaEventElapsedTime gives the kernel's own
+ * duration without the call's other work.  Two NULLs switch the point off again.
+ * Errors: INVALID_ARG (unknown point, or only one of the two events given). */
+int32_t dsp_profile_events(int32_t point, void *start, void *stop);
 
 /* -------------------------------------------------------------------------
  * Lattice build  (Sec. 3.2 "Lattice and pruning", Eq. 7; Alg. 1 stage 1;

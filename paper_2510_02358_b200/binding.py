@@ -26,7 +26,7 @@ ROW_NONFINITE_INPUT, ROW_ZERO_RESIDUAL, ROW_NO_BONUS_ROW, ROW_EOS_ACCEPTED, ROW_
 ROW_TIMEOUT = 32
 DSP_MAX_K, DSP_MAX_W, DSP_MAX_L = 32, 32, 1024
 
-EXPORTS = ["dsp_strerror", "dsp_last_cuda_error", "dsp_version", "dsp_lattice_workspace_bytes",
+EXPORTS = ["dsp_strerror", "dsp_last_cuda_error", "dsp_version", "dsp_profile_events", "dsp_lattice_workspace_bytes",
            "dsp_lattice_build", "dsp_lattice_build_static", "dsp_cps_search", "dsp_verify_workspace_bytes", "dsp_verify",
            "dsp_adl_init", "dsp_adl_update"]
 
@@ -99,6 +99,16 @@ def _logits3(t: torch.Tensor, name: str):
 
 def dsp_version() -> int:
     return lib().dsp_version()
+
+
+PROFILE_LATTICE_SCAN, PROFILE_TARGET_SCAN = 0, 1
+
+
+def dsp_profile_events(point: int, start: Optional[torch.cuda.Event], stop: Optional[torch.cuda.Event]) -> None:
+    """Bracket the launches of one streaming kernel with two timing events (None, None = off).
+    The events must have been recorded once before, so that torch has created them."""
+    h = lambda e: C.c_void_p(0 if e is None else e.cuda_event)
+    _check("dsp_profile_events", lib().dsp_profile_events(point, h(start), h(stop)))
 
 
 def dsp_lattice_workspace_bytes(B: int, L: int, V: int, dtype: int, K_max: int) -> int:

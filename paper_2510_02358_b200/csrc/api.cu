@@ -6,6 +6,15 @@
 
 namespace dsp {
 int32_t g_last_cuda_error = 0;
+ProfileEvents g_profile[2] = {{nullptr, nullptr}, {nullptr, nullptr}};
+}
+
+extern "C" int32_t dsp_profile_events(int32_t point, void *start, void *stop) {
+    if (point != DSP_PROFILE_LATTICE_SCAN && point != DSP_PROFILE_TARGET_SCAN) return DSP_ERR_INVALID_ARG;
+    if ((start == nullptr) != (stop == nullptr)) return DSP_ERR_INVALID_ARG;
+    dsp::g_profile[point].start = reinterpret_cast<cudaEvent_t>(start);
+    dsp::g_profile[point].stop = reinterpret_cast<cudaEvent_t>(stop);
+    return DSP_OK;
 }
 
 extern "C" const char *dsp_strerror(int32_t status) {

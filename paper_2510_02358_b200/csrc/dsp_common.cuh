@@ -24,6 +24,11 @@ constexpr float kRefFloor = -3.0e38f;          // finite stand-in for "no refere
 
 // Host-side record of the last CUDA error seen by an entry point.
 extern int32_t g_last_cuda_error;
+// Events that bracket a kernel launch while set (see dsp_profile_events).
+struct ProfileEvents {
+    cudaEvent_t start, stop;
+};
+extern ProfileEvents g_profile[2];
 inline int32_t cuda_fail(cudaError_t e) {
     g_last_cuda_error = (int32_t)e;
     return DSP_ERR_CUDA;

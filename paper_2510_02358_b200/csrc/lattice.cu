@@ -346,8 +346,11 @@ static int32_t launch_lattice(LatticeArgs &a, void *workspace, size_t workspace_
         stream_layout_ok<DT>(a.logits, a.V, a.stride_b, a.stride_l)) {
         static RingSmemDone smem_done;                       // one per element type
         DSP_CUDA_TRY(allow_ring_smem(lattice_scan_kernel<DT>, smem_done));
+        const ProfileEvents pe = g_profile[DSP_PROFILE_LATTICE_SCAN];
+        if (pe.start) DSP_CUDA_TRY(cudaEventRecord(pe.start, st));
         lattice_scan_kernel<DT><<<(unsigned)nblocks, kThreads, kRingBytes, st>>>(a);
         DSP_CUDA_TRY(cudaGetLastError());
+        if (pe.stop) DSP_CUDA_TRY(cudaEventRecord(pe.stop, st));
         lattice_rows_kernel<DT><<<(unsigned)((nrows + kRowWarps - 1) / kRowWarps), kThreads, 0, st>>>(a);
     } else {
         lattice_kernel<DT><<<(unsigned)nblocks, kThreads, 0, st>>>(a);

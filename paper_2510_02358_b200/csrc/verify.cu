@@ -514,8 +514,11 @@ static int32_t launch_verify(VerifyArgs &a, void *workspace, size_t workspace_by
         stream_layout_ok<DT>(a.target, a.V, a.tstride_b, a.tstride_l)) {
         static RingSmemDone smem_done;                       // one per element type
         DSP_CUDA_TRY(allow_ring_smem(target_scan_kernel<DT>, smem_done));
+        const ProfileEvents pe = g_profile[DSP_PROFILE_TARGET_SCAN];
+        if (pe.start) DSP_CUDA_TRY(cudaEventRecord(pe.start, st));
         target_scan_kernel<DT><<<(unsigned)nblocks, kThreads, kRingBytes, st>>>(a);
         DSP_CUDA_TRY(cudaGetLastError());
+        if (pe.stop) DSP_CUDA_TRY(cudaEventRecord(pe.stop, st));
         target_rows_kernel<DT><<<(unsigned)((nrows + kRowWarps - 1) / kRowWarps), kThreads, 0, st>>>(a);
     } else {
         target_kernel<DT><<<(unsigned)nblocks, kThreads, 0, st>>>(a);
