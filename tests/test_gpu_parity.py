@@ -78,6 +78,9 @@ def test_workloads_full_size_sampled_rows(cid, rows):
     (2, 4, 8200, 1, 1, torch.bfloat16),      # K = 1, W = 1, just over one tile
     (2, 3, 4099, 32, 32, torch.float32),     # largest K and W
     (5, 7, 1000, 15, 3, torch.bfloat16),     # the paper's defaults M_max = 15, beam 3
+    (2, 3, 8192, 32, 32, torch.bfloat16),    # largest K and W on a 16-byte aligned layout (streaming kernels)
+    (1, 2, 1048576, 16, 8, torch.bfloat16),  # a million-token vocabulary: rows cut into long slices
+    (3, 2, 12288, 8, 4, torch.float32),      # fp32 rows of exactly three tiles
 ])
 def test_edge_shapes(B, L, V, K, W, dtype):
     inp = _to(wl.tiny_random(B, L, V, dtype=dtype, seed=B * 100 + L))
@@ -179,3 +182,24 @@ def test_adl_closed_loop_matches_oracle():
         assert nxt == ref.update(g.ver.accepted_len, g.lat.gen_len)
         assert abs(st.ema_gen - ref.ema_gen) < 1e-12 and abs(st.ema_acc - ref.ema_acc) < 1e-12
     assert len(seen) >= 2
+
+
+def test_profile_events_bracket_the_scan_kernels():
+    w = wl.CONFIGS[3].scaled(B=2, L=4, V=152064)
+    inp = wl.make_inputs(w, device=DEV)
+    pairs = []
+    for point in (dsp.PROFILE_LATTICE_SCAN, dsp.PROFILE_TARGET_SCAN):
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(); b.record()
+        dsp.dsp_profile_events(point, a, b)
+        pairs.append((a, b))
+    try:
+        g = gpu_step(inp, **_params(w))
+    finally:
+        for point in (dsp.PROFILE_LATTICE_SCAN, dsp.PROFILE_TARGET_SCAN):
+            dsp.dsp_profile_events(point, None, None)
+    check_step(g, inp, **_params(w))
+    for a, b in pairs:
+        assert 0.0 < a.elapsed_time(b) < 50.0          # milliseconds
+    with pytest.raises(dsp.DspError):
+        dsp.dsp_profile_events(7, None, None)
