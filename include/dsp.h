@@ -268,6 +268,41 @@ int32_t dsp_verify(const void *target_logits, int32_t dtype,
                    void *workspace, size_t workspace_bytes, dsp_stream_t stream);
 
 /* -------------------------------------------------------------------------
+ * One whole step in one call  (Alg. 1 stages 1-3 on logits)
+ *
+ * dsp_lattice_build, dsp_cps_search and dsp_verify with the arguments and
+ * results of the three calls (KC = K_max + (eos_id >= 0 ? 1 : 0); row_status is
+ * overwritten by the lattice part and OR-ed into by the others; every output of
+ * the three calls is written, nullable ones as there).  The one call lets the
+ * statistics of the target rows, which need only the target logits, run on a
+ * second stream beside the lattice's finish and the path search; the
+ * decisions wait for both.  All work is ordered after what was enqueued on
+ * `stream` before the call, and work enqueued on `stream` after it is ordered
+ * after all of it.
+ * The second stream and two events are created at the first call on each
+ * device and kept until the process exits (host-side handles; no device
+ * memory is allocated).
+ * lattice_workspace / verify_workspace: as for dsp_lattice_build / dsp_verify.
+ * Errors: those of the three calls.
+ */
+int32_t dsp_draft_verify_step(
+    const void *draft_logits, const void *target_logits, int32_t dtype,
+    int32_t B, int32_t L, int32_t Lt, int32_t V,
+    int64_t dstride_b, int64_t dstride_l, int64_t tstride_b, int64_t tstride_l,
+    int32_t K_max, float tau, int32_t eos_id,
+    const int32_t *prev_token, int32_t proxy_kind, const float *proxy_table, int32_t table_log2,
+    uint32_t hash_seed, int32_t W, float lambda,
+    int32_t all_greedy, const uint8_t *mode, const float *u,
+    int32_t *cand_id, float *cand_logit, float *cand_logp, int32_t *cand_count,
+    float *lse, double *lse64, float *entropy, int32_t *gen_len,
+    int32_t *path, int32_t *path_slot, int32_t *path_len, float *path_score,
+    int32_t *beam_ids, float *beam_score, float *beam_cum,
+    int32_t *accepted_len, int32_t *next_token, float *ratio, int32_t *tgt_argmax, float *tgt_lse,
+    uint32_t *row_status,
+    void *lattice_workspace, size_t lattice_workspace_bytes,
+    void *verify_workspace, size_t verify_workspace_bytes, dsp_stream_t stream);
+
+/* -------------------------------------------------------------------------
  * Adaptive draft length  (Sec. 3.3, Eq. 9-11; Alg. 1 init and stage 4) -- host.
  *
  * State is plain data owned by the caller (copy it to checkpoint it).

@@ -27,7 +27,7 @@ ROW_TIMEOUT = 32
 DSP_MAX_K, DSP_MAX_W, DSP_MAX_L = 32, 32, 1024
 
 EXPORTS = ["dsp_strerror", "dsp_last_cuda_error", "dsp_version", "dsp_profile_events", "dsp_lattice_workspace_bytes",
-           "dsp_lattice_build", "dsp_lattice_build_static", "dsp_cps_search", "dsp_verify_workspace_bytes", "dsp_verify",
+           "dsp_lattice_build", "dsp_lattice_build_static", "dsp_cps_search", "dsp_verify_workspace_bytes", "dsp_verify", "dsp_draft_verify_step",
            "dsp_adl_init", "dsp_adl_update"]
 
 
@@ -236,6 +236,42 @@ def dsp_verify(target: torch.Tensor, draft: Optional[torch.Tensor], cps: SimpleN
         _ptr(out.tgt_lse), _ptr(row_status), _ptr(workspace), C.c_size_t(workspace.numel()),
         _stream(stream)))
     return out
+
+
+def dsp_draft_verify_step(draft: torch.Tensor, target: torch.Tensor, prev_token: torch.Tensor,
+                          table: torch.Tensor, *, K_max: int, W: int, lam: float, tau: float = 0.0,
+                          eos_id: int = -1, proxy_kind: int = 0, table_log2: int = 0, hash_seed: int = 0,
+                          mode: Optional[torch.Tensor] = None, u: Optional[torch.Tensor] = None,
+                          all_greedy: bool = False, lat: Optional[SimpleNamespace] = None,
+                          cps: Optional[SimpleNamespace] = None, ver: Optional[SimpleNamespace] = None,
+                          lattice_workspace: Optional[torch.Tensor] = None,
+                          verify_workspace: Optional[torch.Tensor] = None, stream=None):
+    """The three device calls of a step in one (same results); returns (lat, cps, ver)."""
+    B, L, V, dsb, dsl = _logits3(draft, "draft")
+    Bt, Lt, Vt, tsb, tsl = _logits3(target, "target")
+    if (Bt, Vt) != (B, V) or target.dtype != draft.dtype:
+        raise ValueError("target must be [B, Lt, V] with the draft's dtype")
+    dt = _dtype(draft)
+    dev = draft.device
+    lat = lattice_outputs(B, L, K_max, eos_id, dev) if lat is None else lat
+    cps = cps_outputs(B, L, W, dev, True) if cps is None else cps
+    ver = verify_outputs(B, L, Lt, dev) if ver is None else ver
+    if lattice_workspace is None:
+        lattice_workspace = alloc_workspace(dsp_lattice_workspace_bytes(B, L, V, dt, K_max), dev)
+    if verify_workspace is None:
+        verify_workspace = alloc_workspace(dsp_verify_workspace_bytes(B, L, Lt, V, dt), dev)
+    _check("dsp_draft_verify_step", lib().dsp_draft_verify_step(
+        _ptr(draft), _ptr(target), dt, B, L, Lt, V, C.c_int64(dsb), C.c_int64(dsl), C.c_int64(tsb),
+        C.c_int64(tsl), K_max, C.c_float(tau), eos_id, _ptr(prev_token), proxy_kind, _ptr(table), table_log2,
+        C.c_uint32(hash_seed & 0xFFFFFFFF), W, C.c_float(lam), 1 if all_greedy else 0, _ptr(mode), _ptr(u),
+        _ptr(lat.cand_id), _ptr(lat.cand_logit), _ptr(lat.cand_logp), _ptr(lat.cand_count), _ptr(lat.lse),
+        _ptr(lat.lse64), _ptr(lat.entropy), _ptr(lat.gen_len),
+        _ptr(cps.path), _ptr(cps.path_slot), _ptr(cps.path_len), _ptr(cps.path_score), _ptr(cps.beam_ids),
+        _ptr(cps.beam_score), _ptr(cps.beam_cum),
+        _ptr(ver.accepted_len), _ptr(ver.next_token), _ptr(ver.ratio), _ptr(ver.tgt_argmax), _ptr(ver.tgt_lse),
+        _ptr(lat.row_status), _ptr(lattice_workspace), C.c_size_t(lattice_workspace.numel()),
+        _ptr(verify_workspace), C.c_size_t(verify_workspace.numel()), _stream(stream)))
+    return lat, cps, ver
 
 
 def dsp_adl_init(k_min=20, k_max=30, delta=10.0, rho=0.5, granularity=1):

@@ -1,0 +1,31 @@
+// Entry points shared between the translation units of the library (not part of the C ABI).
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace dsp {
+
+// The two parts of dsp_verify: the target statistics need only the target logits (and mode);
+// the decisions also need the chosen path.
+constexpr int kVerifyStats = 1;
+constexpr int kVerifyDecide = 2;
+
+// dsp_verify with a choice of parts (same arguments, checks and errors).
+int32_t verify_impl(const void *target_logits, int32_t dtype, int32_t B, int32_t L, int32_t Lt, int32_t V,
+                    int64_t tstride_b, int64_t tstride_l, const void *draft_logits, int64_t dstride_b,
+                    int64_t dstride_l, const int32_t *path, const int32_t *path_slot, const int32_t *path_len,
+                    const float *cand_logit, const double *draft_lse64, int32_t KC, int32_t all_greedy,
+                    const uint8_t *mode, const float *u, int32_t eos_id, int32_t *accepted_len,
+                    int32_t *next_token, float *ratio, int32_t *tgt_argmax, float *tgt_lse,
+                    uint32_t *row_status, void *workspace, size_t workspace_bytes, cudaStream_t st, int phases);
+
+// dsp_lattice_build that also records `after_scan` (if not null) on the stream once the pass over
+// the draft logits has been enqueued: what follows it in the call no longer reads them.
+int32_t lattice_build_impl(const void *draft_logits, int32_t dtype, int32_t B, int32_t L, int32_t V,
+                           int64_t stride_b, int64_t stride_l, int32_t K_max, float tau, int32_t eos_id,
+                           int32_t *cand_id, float *cand_logit, float *cand_logp, int32_t *cand_count,
+                           float *lse, double *lse64, float *entropy, int32_t *gen_len, uint32_t *row_status,
+                           void *workspace, size_t workspace_bytes, cudaStream_t st, cudaEvent_t after_scan);
+
+}  // namespace dsp

@@ -9,6 +9,7 @@
 // top-K on the way; a row split over several CTAs is finished by whichever CTA arrives last
 // (atomic ticket): no CTA waits.  In both paths the CTA that finishes the last row of a batch
 // row also writes gen_len and row_status.
+#include "dsp_internal.h"
 #include "row_warp.cuh"
 
 namespace dsp {
@@ -323,7 +324,8 @@ __global__ void __launch_bounds__(kThreads) lattice_rows_kernel(const LatticeArg
 }
 
 template <typename DT>
-static int32_t launch_lattice(LatticeArgs &a, void *workspace, size_t workspace_bytes, cudaStream_t st) {
+static int32_t launch_lattice(LatticeArgs &a, void *workspace, size_t workspace_bytes, cudaStream_t st,
+                              cudaEvent_t after_scan) {
     const long long nrows = (long long)a.B * a.L;
     const SlicePlan plan = plan_slices<DT>(nrows, a.V, kTargetCtas);
     a.nslices = plan.nslices;
@@ -351,10 +353,12 @@ static int32_t launch_lattice(LatticeArgs &a, void *workspace, size_t workspace_
         lattice_scan_kernel<DT><<<(unsigned)nblocks, kThreads, kRingBytes, st>>>(a);
         DSP_CUDA_TRY(cudaGetLastError());
         if (pe.stop) DSP_CUDA_TRY(cudaEventRecord(pe.stop, st));
+        if (after_scan) { DSP_CUDA_TRY(cudaEventRecord(after_scan, st)); after_scan = nullptr; }
         lattice_rows_kernel<DT><<<(unsigned)((nrows + kRowWarps - 1) / kRowWarps), kThreads, 0, st>>>(a);
     } else {
         lattice_kernel<DT><<<(unsigned)nblocks, kThreads, 0, st>>>(a);
     }
+    if (after_scan) DSP_CUDA_TRY(cudaEventRecord(after_scan, st));
     DSP_CUDA_TRY(cudaGetLastError());
     return DSP_OK;
 }
@@ -389,14 +393,14 @@ extern "C" int32_t dsp_lattice_workspace_bytes(int32_t B, int32_t L, int32_t V, 
     return DSP_OK;
 }
 
-extern "C" int32_t dsp_lattice_build(const void *draft_logits, int32_t dtype,
-                                     int32_t B, int32_t L, int32_t V,
-                                     int64_t stride_b, int64_t stride_l,
-                                     int32_t K_max, float tau, int32_t eos_id,
-                                     int32_t *cand_id, float *cand_logit, float *cand_logp,
-                                     int32_t *cand_count, float *lse, double *lse64, float *entropy,
-                                     int32_t *gen_len, uint32_t *row_status,
-                                     void *workspace, size_t workspace_bytes, dsp_stream_t stream) {
+int32_t dsp::lattice_build_impl(const void *draft_logits, int32_t dtype,
+                                int32_t B, int32_t L, int32_t V,
+                                int64_t stride_b, int64_t stride_l,
+                                int32_t K_max, float tau, int32_t eos_id,
+                                int32_t *cand_id, float *cand_logit, float *cand_logp,
+                                int32_t *cand_count, float *lse, double *lse64, float *entropy,
+                                int32_t *gen_len, uint32_t *row_status,
+                                void *workspace, size_t workspace_bytes, cudaStream_t st, cudaEvent_t after_scan) {
     const int32_t rc = check_lattice_shape(B, L, V, dtype, K_max);
     if (rc != DSP_OK) return rc;
     if (B == 0) return DSP_OK;
@@ -422,9 +426,21 @@ extern "C" int32_t dsp_lattice_build(const void *draft_logits, int32_t dtype,
     a.cand_id = cand_id; a.cand_logit = cand_logit; a.cand_logp = cand_logp;
     a.cand_count = cand_count; a.lse = lse; a.lse64 = lse64; a.entropy = entropy;
     a.gen_len = gen_len; a.row_status = row_status;
-    cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
-    return dtype == DSP_BF16 ? launch_lattice<__nv_bfloat16>(a, workspace, workspace_bytes, st)
-                             : launch_lattice<float>(a, workspace, workspace_bytes, st);
+    return dtype == DSP_BF16 ? launch_lattice<__nv_bfloat16>(a, workspace, workspace_bytes, st, after_scan)
+                             : launch_lattice<float>(a, workspace, workspace_bytes, st, after_scan);
+}
+
+extern "C" int32_t dsp_lattice_build(const void *draft_logits, int32_t dtype,
+                                     int32_t B, int32_t L, int32_t V,
+                                     int64_t stride_b, int64_t stride_l,
+                                     int32_t K_max, float tau, int32_t eos_id,
+                                     int32_t *cand_id, float *cand_logit, float *cand_logp,
+                                     int32_t *cand_count, float *lse, double *lse64, float *entropy,
+                                     int32_t *gen_len, uint32_t *row_status,
+                                     void *workspace, size_t workspace_bytes, dsp_stream_t stream) {
+    return lattice_build_impl(draft_logits, dtype, B, L, V, stride_b, stride_l, K_max, tau, eos_id, cand_id,
+                              cand_logit, cand_logp, cand_count, lse, lse64, entropy, gen_len, row_status,
+                              workspace, workspace_bytes, reinterpret_cast<cudaStream_t>(stream), nullptr);
 }
 
 // ---- dsp_lattice_build_static: the same build for callers that cannot allocate ----------------

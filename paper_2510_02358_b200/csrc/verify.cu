@@ -5,11 +5,14 @@
 // 16-byte aligned layouts by target_scan_kernel (one CTA per row slice, no block-wide barrier,
 // see stream_core.cuh) followed by target_rows_kernel (one warp per row: argmax from the table
 // of tile maxima, sums added up), any other layout by target_kernel (element-wise, slices
-// merged by the CTA arriving last).  The CTA that finishes the last row of a batch row runs that
-// row's left-to-right acceptance scan and either writes the next token (greedy) or records
-// a sampling job (stochastic: residual at the first rejection, or bonus from row m).
+// merged by the CTA arriving last).  accept_kernel then runs every batch row's left-to-right
+// acceptance scan (one warp each) and either writes the next token (greedy) or records a
+// sampling job (stochastic: residual at the first rejection, or bonus from row m).
+// The first part needs only the target logits: dsp_draft_verify_step (step.cu) runs it beside
+// the lattice finish and the path search.
 // Kernel 2 (residual_kernel): for each job, one more pass over ONE target row (and ONE draft
 // row): per-chunk sums of max(0, p - q) in token order; the CTA arriving last inverts the CDF.
+#include "dsp_internal.h"
 #include "row_warp.cuh"
 
 namespace dsp {
@@ -172,8 +175,7 @@ __device__ void target_finish(const VerifyArgs &a, ScanSmem &sm, long long row, 
 }
 
 // A target row is complete (thread 0 holds its best key and, with `sums`, its whole-row sums):
-// write argmax and log-sum-exp; the CTA that finishes the last row of a batch row then runs that
-// row's acceptance scan.
+// write argmax and log-sum-exp.
 template <typename DT, typename SY>
 __device__ void target_finish_row(const VerifyArgs &a, ScanSmem &sm, long long row, int b, bool sums,
                                   unsigned long long best, float c, double S, double T) {
@@ -192,13 +194,7 @@ __device__ void target_finish_row(const VerifyArgs &a, ScanSmem &sm, long long r
             a.tgt_lse[row] = CUDART_NAN_F;             // greedy row of a mixed batch: not computed
         }
         if (!ok) atomicOr(&a.b_status[b], DSP_ROW_NONFINITE_INPUT);
-        __threadfence();
-        sm.flag = (int)atomicAdd(&a.b_ticket[b], 1u);
     }
-    SY::sync();
-    if (sm.flag != a.Lt - 1) return;
-    __threadfence();
-    if (tid < 32) accept_row<DT>(a, b);
 }
 
 
@@ -241,8 +237,7 @@ __global__ void __launch_bounds__(kThreads, 4) target_scan_kernel(const VerifyAr
 }
 
 // Streaming path, pass 2: one warp per row (see row_warp.cuh): argmax from the table of tile
-// maxima, log-sum-exp from the warp sums; the warp that finishes the last row of a batch row
-// runs that row's acceptance scan.
+// maxima, log-sum-exp from the warp sums.
 template <typename DT>
 __global__ void __launch_bounds__(kThreads) target_rows_kernel(const VerifyArgs a) {
     __shared__ WarpScratch scratch[kRowWarps];
@@ -262,7 +257,6 @@ __global__ void __launch_bounds__(kThreads) target_rows_kernel(const VerifyArgs 
         rowp, a.V, 1, reinterpret_cast<const DT *>(a.table) + row * (a.ntiles_row + a.nslices) * kThreads, a.ntiles_row,
         a.nslices, scratch[warp], lane);
     const unsigned long long best = __shfl_sync(0xFFFFFFFFu, key, 0);
-    unsigned ticket = 0;
     if (lane == 0) {
         const int am = best ? key_id(best) : 0;
         a.argmax[row] = am;
@@ -277,13 +271,15 @@ __global__ void __launch_bounds__(kThreads) target_rows_kernel(const VerifyArgs 
             a.tgt_lse[row] = CUDART_NAN_F;             // greedy row of a mixed batch: not computed
         }
         if (!ok) atomicOr(&a.b_status[b], DSP_ROW_NONFINITE_INPUT);
-        __threadfence();
-        ticket = atomicAdd(&a.b_ticket[b], 1u);
     }
-    ticket = __shfl_sync(0xFFFFFFFFu, ticket, 0);
-    if (ticket != (unsigned)a.Lt - 1) return;
-    __threadfence();
-    accept_row<DT>(a, b);
+}
+
+// The left-to-right acceptance of every batch row (Eq. 1, Eq. 2), one warp per batch row, once
+// the target statistics of all rows are there.
+template <typename DT>
+__global__ void __launch_bounds__(kThreads) accept_kernel(const VerifyArgs a) {
+    const int b = blockIdx.x * kWarps + (threadIdx.x >> 5);
+    if (b < a.B) accept_row<DT>(a, b);
 }
 
 // ---- residual / bonus sampling -------------------------------------------------------------
@@ -477,7 +473,8 @@ static size_t verify_ws_bytes(int B, int Lt, int V) {
 }
 
 template <typename DT>
-static int32_t launch_verify(VerifyArgs &a, void *workspace, size_t workspace_bytes, cudaStream_t st) {
+static int32_t launch_verify(VerifyArgs &a, void *workspace, size_t workspace_bytes, cudaStream_t st,
+                             int phases) {
     const long long nrows = (long long)a.B * a.Lt;
     const SlicePlan plan = plan_slices<DT>(nrows, a.V, kTargetCtas);
     a.nslices = plan.nslices;
@@ -507,9 +504,10 @@ static int32_t launch_verify(VerifyArgs &a, void *workspace, size_t workspace_by
     a.chunks_per_slice = (a.nchunks + rsl - 1) / rsl;
     a.res_slices = (a.nchunks + a.chunks_per_slice - 1) / a.chunks_per_slice;
 
-    DSP_CUDA_TRY(cudaMemsetAsync(ws, 0, w.zero_bytes, st));
     const long long nblocks = nrows * a.nslices;
     if (nblocks > 0x7FFFFFFFLL) return DSP_ERR_UNSUPPORTED;
+    if (phases & kVerifyStats) {
+    DSP_CUDA_TRY(cudaMemsetAsync(ws, 0, w.zero_bytes, st));
     if (a.nslices * kWarps <= kThreads && nrows <= 0x7FFFFFFFLL &&
         stream_layout_ok<DT>(a.target, a.V, a.tstride_b, a.tstride_l)) {
         static RingSmemDone smem_done;                       // one per element type
@@ -524,9 +522,14 @@ static int32_t launch_verify(VerifyArgs &a, void *workspace, size_t workspace_by
         target_kernel<DT><<<(unsigned)nblocks, kThreads, 0, st>>>(a);
     }
     DSP_CUDA_TRY(cudaGetLastError());
-    if (!a.all_greedy) {
-        residual_kernel<DT><<<(unsigned)(a.B * a.res_slices), kThreads, 0, st>>>(a);
+    }
+    if (phases & kVerifyDecide) {
+        accept_kernel<DT><<<(unsigned)((a.B + kWarps - 1) / kWarps), kThreads, 0, st>>>(a);
         DSP_CUDA_TRY(cudaGetLastError());
+        if (!a.all_greedy) {
+            residual_kernel<DT><<<(unsigned)(a.B * a.res_slices), kThreads, 0, st>>>(a);
+            DSP_CUDA_TRY(cudaGetLastError());
+        }
     }
     return DSP_OK;
 }
@@ -553,16 +556,16 @@ extern "C" int32_t dsp_verify_workspace_bytes(int32_t B, int32_t L, int32_t Lt, 
     return DSP_OK;
 }
 
-extern "C" int32_t dsp_verify(const void *target_logits, int32_t dtype,
-                              int32_t B, int32_t L, int32_t Lt, int32_t V,
-                              int64_t tstride_b, int64_t tstride_l,
-                              const void *draft_logits, int64_t dstride_b, int64_t dstride_l,
-                              const int32_t *path, const int32_t *path_slot, const int32_t *path_len,
-                              const float *cand_logit, const double *draft_lse64, int32_t KC,
-                              int32_t all_greedy, const uint8_t *mode, const float *u, int32_t eos_id,
-                              int32_t *accepted_len, int32_t *next_token, float *ratio,
-                              int32_t *tgt_argmax, float *tgt_lse, uint32_t *row_status,
-                              void *workspace, size_t workspace_bytes, dsp_stream_t stream) {
+int32_t dsp::verify_impl(const void *target_logits, int32_t dtype,
+                         int32_t B, int32_t L, int32_t Lt, int32_t V,
+                         int64_t tstride_b, int64_t tstride_l,
+                         const void *draft_logits, int64_t dstride_b, int64_t dstride_l,
+                         const int32_t *path, const int32_t *path_slot, const int32_t *path_len,
+                         const float *cand_logit, const double *draft_lse64, int32_t KC,
+                         int32_t all_greedy, const uint8_t *mode, const float *u, int32_t eos_id,
+                         int32_t *accepted_len, int32_t *next_token, float *ratio,
+                         int32_t *tgt_argmax, float *tgt_lse, uint32_t *row_status,
+                         void *workspace, size_t workspace_bytes, cudaStream_t st, int phases) {
     const int32_t rc = check_verify_shape(B, L, Lt, V, dtype);
     if (rc != DSP_OK) return rc;
     if (B == 0) return DSP_OK;
@@ -593,7 +596,22 @@ extern "C" int32_t dsp_verify(const void *target_logits, int32_t dtype,
     a.all_greedy = all_greedy ? 1 : 0; a.mode = mode; a.u = u; a.eos_id = eos_id;
     a.accepted_len = accepted_len; a.next_token = next_token; a.ratio = ratio;
     a.tgt_argmax = tgt_argmax; a.tgt_lse = tgt_lse; a.row_status = row_status;
-    cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
-    return dtype == DSP_BF16 ? launch_verify<__nv_bfloat16>(a, workspace, workspace_bytes, st)
-                             : launch_verify<float>(a, workspace, workspace_bytes, st);
+    return dtype == DSP_BF16 ? launch_verify<__nv_bfloat16>(a, workspace, workspace_bytes, st, phases)
+                             : launch_verify<float>(a, workspace, workspace_bytes, st, phases);
+}
+
+extern "C" int32_t dsp_verify(const void *target_logits, int32_t dtype,
+                              int32_t B, int32_t L, int32_t Lt, int32_t V,
+                              int64_t tstride_b, int64_t tstride_l,
+                              const void *draft_logits, int64_t dstride_b, int64_t dstride_l,
+                              const int32_t *path, const int32_t *path_slot, const int32_t *path_len,
+                              const float *cand_logit, const double *draft_lse64, int32_t KC,
+                              int32_t all_greedy, const uint8_t *mode, const float *u, int32_t eos_id,
+                              int32_t *accepted_len, int32_t *next_token, float *ratio,
+                              int32_t *tgt_argmax, float *tgt_lse, uint32_t *row_status,
+                              void *workspace, size_t workspace_bytes, dsp_stream_t stream) {
+    return verify_impl(target_logits, dtype, B, L, Lt, V, tstride_b, tstride_l, draft_logits, dstride_b,
+                       dstride_l, path, path_slot, path_len, cand_logit, draft_lse64, KC, all_greedy, mode, u,
+                       eos_id, accepted_len, next_token, ratio, tgt_argmax, tgt_lse, row_status, workspace,
+                       workspace_bytes, reinterpret_cast<cudaStream_t>(stream), kVerifyStats | kVerifyDecide);
 }

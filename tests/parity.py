@@ -30,11 +30,21 @@ NEAR = 1e-6
 
 
 def gpu_step(inp: dict, *, K: int, W: int, tau: float = 0.0, lam: float = 0.5, eos_id: int = -1,
-             all_greedy: bool = False, proxy_kind: int = 0, target=None, draft=None) -> SimpleNamespace:
-    """One step on the GPU; ``inp`` holds CUDA tensors. Returns CPU copies of every output."""
+             all_greedy: bool = False, proxy_kind: int = 0, target=None, draft=None,
+             fused: bool = False) -> SimpleNamespace:
+    """One step on the GPU; ``inp`` holds CUDA tensors. Returns CPU copies of every output.
+    ``fused`` takes the single-call entry point instead of the three calls."""
     draft = inp["draft"] if draft is None else draft
     target = inp["target"] if target is None else target
     V = draft.shape[2]
+    cpu = lambda ns: SimpleNamespace(**{k: (v.cpu() if v is not None else None) for k, v in vars(ns).items()})
+    if fused:
+        lat, cps, ver = dsp.dsp_draft_verify_step(
+            draft, target, inp["prev_token"], inp["table"], K_max=K, W=W, lam=lam, tau=tau, eos_id=eos_id,
+            proxy_kind=proxy_kind, table_log2=inp.get("table_log2", 0), hash_seed=inp.get("hash_seed", 0),
+            mode=None if all_greedy else inp["mode"], u=None if all_greedy else inp["u"], all_greedy=all_greedy)
+        torch.cuda.synchronize()
+        return SimpleNamespace(lat=cpu(lat), cps=cpu(cps), ver=cpu(ver))
     lat = dsp.dsp_lattice_build(draft, K, tau, eos_id)
     cps = dsp.dsp_cps_search(lat, inp["prev_token"], inp["table"], W=W, lam=lam, eos_id=eos_id,
                              proxy_kind=proxy_kind, table_log2=inp.get("table_log2", 0),
@@ -46,7 +56,6 @@ def gpu_step(inp: dict, *, K: int, W: int, tau: float = 0.0, lam: float = 0.5, e
         ver = dsp.dsp_verify(target, draft, cps, lat, mode=inp["mode"], u=inp["u"], eos_id=eos_id,
                              row_status=lat.row_status)
     torch.cuda.synchronize()
-    cpu = lambda ns: SimpleNamespace(**{k: (v.cpu() if v is not None else None) for k, v in vars(ns).items()})
     return SimpleNamespace(lat=cpu(lat), cps=cpu(cps), ver=cpu(ver))
 
 

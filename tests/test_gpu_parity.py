@@ -203,3 +203,28 @@ def test_profile_events_bracket_the_scan_kernels():
         assert 0.0 < a.elapsed_time(b) < 50.0          # milliseconds
     with pytest.raises(dsp.DspError):
         dsp.dsp_profile_events(7, None, None)
+
+
+@pytest.mark.parametrize("cid", [1, 2, 3, 4, 5])
+def test_single_call_step_equals_the_three_calls(cid):
+    w = wl.CONFIGS[cid].scaled(**SMALL[cid])
+    if cid == 4:
+        w = w.scaled(V=50048)                              # an aligned layout: the streaming kernels
+    inp = wl.make_inputs(w, step=2, device=DEV)
+    for rep in range(2):                                  # twice: the second stream is reused
+        a = gpu_step(inp, **_params(w))
+        b = gpu_step(inp, fused=True, **_params(w))
+        for s in ("lat", "cps", "ver"):
+            for k, v in vars(getattr(a, s)).items():
+                if v is None:
+                    continue
+                o = getattr(getattr(b, s), k)
+                if all_greedy_unused(w, s, k):
+                    continue
+                assert torch.equal(v.view(torch.uint8), o.view(torch.uint8)), (s, k)
+    check_step(b, inp, **_params(w))
+
+
+def all_greedy_unused(w, s, k):
+    """Outputs that a greedy-only verification does not write."""
+    return w.verify == "greedy" and s == "ver" and k in ("ratio", "tgt_lse")
