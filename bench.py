@@ -117,10 +117,21 @@ class GpuStep:
         self.ws_l = dsp.alloc_workspace(dsp.dsp_lattice_workspace_bytes(w.B, w.L, w.V, dt, w.K), device)
         self.ws_v = dsp.alloc_workspace(dsp.dsp_verify_workspace_bytes(w.B, w.L, w.Lt, w.V, dt), device)
         self.all_greedy = w.verify == "greedy"
-        # lattice scan + rows, cps, target scan + rows (+ residual); memsets are not counted
-        self.kernels_per_step = 5 if self.all_greedy else 6
+        # lattice scan + rows, cps, target scan + rows, accept (+ residual); memsets are not counted
+        self.kernels_per_step = 6 if self.all_greedy else 7
+
+    def step(self, inp):
+        """One step through the single-call entry point (what `value` and `e2e` time)."""
+        dsp, w = self.dsp, self.w
+        dsp.dsp_draft_verify_step(
+            inp["draft"], inp["target"], inp["prev_token"], inp["table"], K_max=w.K, W=w.W, lam=w.lam,
+            tau=w.tau, eos_id=w.eos_id, table_log2=inp["table_log2"], hash_seed=inp["hash_seed"],
+            mode=None if self.all_greedy else inp["mode"], u=None if self.all_greedy else inp["u"],
+            all_greedy=self.all_greedy, lat=self.lat, cps=self.cps, ver=self.ver,
+            lattice_workspace=self.ws_l, verify_workspace=self.ws_v)
 
     def run(self, inp, ev=None):
+        """The same step as three calls, with an event after each (the per-stage times)."""
         dsp, w = self.dsp, self.w
         if ev:
             ev[0].record()
@@ -172,17 +183,16 @@ def time_workload(w, device, steps, warmup, dist=None, stages=True, seed_base=0)
     """Device-timed throughput of one workload; returns a dict of measurements."""
     sets = input_sets(w, device, seed_base)
     st = GpuStep(w, device)
+    dsp = st.dsp
     for i in range(warmup):
-        st.run(sets[i % len(sets)])
+        st.step(sets[i % len(sets)])
     torch.cuda.synchronize()
-    evs = [[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in range(steps)] if stages else None
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     if dist is not None:
         dist.barrier()
     torch.cuda.synchronize()
     # the dominant kernel's own duration: every 8th timed step its launch is bracketed by a pair
     # of events inside the library (same stream, same timed region)
-    dsp = st.dsp
     scan_evs = []
     e0.record()
     for i in range(steps):
@@ -191,7 +201,7 @@ def time_workload(w, device, steps, warmup, dist=None, stages=True, seed_base=0)
             pair[0].record(); pair[1].record()          # torch creates an event at its first record
             dsp.dsp_profile_events(dsp.PROFILE_LATTICE_SCAN, *pair)
             scan_evs.append(pair)
-        st.run(sets[i % len(sets)], evs[i] if stages else None)
+        st.step(sets[i % len(sets)])
         if stages and i % 8 == 0:
             dsp.dsp_profile_events(dsp.PROFILE_LATTICE_SCAN, None, None)
     e1.record()
@@ -204,10 +214,16 @@ def time_workload(w, device, steps, warmup, dist=None, stages=True, seed_base=0)
         ts = [a.elapsed_time(b) for a, b in scan_evs]
         out.update(ms_lattice_scan=sum(ts) / len(ts), ms_lattice_scan_min=min(ts), scan_samples=len(ts))
     if stages:
+        # per-stage times: the same step as three calls with an event after each (outside the timed region)
+        n = min(steps, 200)
+        evs = [[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in range(n)]
+        for i in range(n):
+            st.run(sets[i % len(sets)], evs[i])
+        torch.cuda.synchronize()
         tl = [e[0].elapsed_time(e[1]) for e in evs]
         tc = [e[1].elapsed_time(e[2]) for e in evs]
         tv = [e[2].elapsed_time(e[3]) for e in evs]
-        out.update(ms_lattice=sum(tl) / steps, ms_cps=sum(tc) / steps, ms_verify=sum(tv) / steps,
+        out.update(ms_lattice=sum(tl) / n, ms_cps=sum(tc) / n, ms_verify=sum(tv) / n,
                    ms_lattice_min=min(tl), ms_verify_min=min(tv))
     out["mean_accepted_len"] = st.ver.accepted_len.float().mean().item()
     out["mean_path_len"] = st.cps.path_len.float().mean().item()
@@ -229,7 +245,7 @@ def time_e2e(w, st, sets, device, steps):
         for k in host:
             dev[k].copy_(host[k], non_blocking=True)
         staged.update(dev)
-        st.run(staged)
+        st.step(staged)
         res_host[0].copy_(st.ver.accepted_len, non_blocking=True)
         res_host[1].copy_(st.ver.next_token, non_blocking=True)
         res_host[2].copy_(st.lat.gen_len, non_blocking=True)
@@ -394,7 +410,9 @@ def main():
                    "l2": "inputs larger than L2" if m["sets"] == 1 else "rotating %d input sets" % m["sets"]},
         "logits_gbs": {"lattice_build": gbs_lat, "verify": gbs_ver, "lattice_plus_verify": gbs_both,
                        "frac_of_8000": gbs_both / 8000.0, "frac_of_%s_copy_peak" % peak_kind: gbs_both / peak},
-        "stage_ms": {"lattice_build": m["ms_lattice"], "cps_search": m["ms_cps"], "verify": m["ms_verify"]},
+        "stage_ms": {"lattice_build": m["ms_lattice"], "cps_search": m["ms_cps"], "verify": m["ms_verify"],
+                     "note": "the three calls one after the other; `value` times dsp_draft_verify_step, "
+                             "which overlaps the target statistics with the path search"},
         "mean_accepted_len": m["mean_accepted_len"], "mean_path_len": m["mean_path_len"],
         "roofline": {"bound": "hbm", "kernel": "lattice_scan_kernel", "achieved": gbs_scan, "peak": peak,
                      "peak_kind": "%s copy bandwidth" % peak_kind, "unit": "GB/s", "frac": gbs_scan / peak,
