@@ -12,8 +12,9 @@
  *    errors are detected on the host before anything is enqueued.
  *  - Unless marked "host", every pointer is a DEVICE pointer to memory the
  *    caller owns (inputs, outputs and the scratch workspace).  The library
- *    allocates nothing and keeps no device state between calls (the one
- *    exception, dsp_lattice_build_static, holds its scratch in a static array).
+ *    allocates nothing and keeps no device state between calls (two
+ *    exceptions: dsp_lattice_build_static holds its scratch in a static array,
+ *    and dsp_draft_verify_step keeps one stream and two events per device).
  *  - Device calls only enqueue work on `stream` (a cudaStream_t; NULL is the
  *    legacy default stream) and never synchronise.  Outputs are valid once
  *    the stream reaches the end of the call.  Two calls that share a

@@ -22,13 +22,9 @@ struct ScanSmem {
     int flag;
 };
 
-// Block-wide barrier policies: every thread of the CTA, or only the kThreads consumer threads
-// of a kernel that also runs a service warp (named barrier 1).
+// Block-wide barrier policy of the helpers below: every thread of the CTA.
 struct SyncAll {
     static __device__ __forceinline__ void sync() { __syncthreads(); }
-};
-struct SyncConsumers {
-    static __device__ __forceinline__ void sync() { asm volatile("bar.sync 1, %0;" ::"n"(kThreads) : "memory"); }
 };
 
 template <typename DT>
