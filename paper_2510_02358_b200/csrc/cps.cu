@@ -7,8 +7,10 @@
 // parallel before the depths of the window are walked; the sequential part of a depth is then
 // one shared-memory read and one fp32 add per expansion and the selection of the best W.
 // Expansions become unique 64-bit keys (cum | token-id rank | parent rank | slot) whose integer
-// order is the beam order (cum desc, token id asc, parent rank asc); every warp sorts 32 keys
-// with a bitonic network and the warps' lists are merged pairwise through shared memory.
+// order is the beam order (cum desc, token id asc, parent rank asc).  The best W are found by
+// pruning and ranking, not sorting: an expansion below the worst of the beams' own best
+// expansions cannot be among the best W and is dropped; the few that remain count the keys
+// above them (all pairs); the keys are unique, so the ranks below W name one key each.
 // Back-pointers stay in shared memory; each surviving beam's slots are recovered by walking them
 // and the token ids are then fetched by all threads at once.
 #include "dsp_common.cuh"
@@ -50,9 +52,11 @@ inline int cps_window_depths(int L, int KC) {
 inline size_t cps_smem_bytes(int L, int W, int KC, int D) {
     size_t o = align_up((size_t)3 * L * W, 16);                 // back-pointers and walked slots
     o += (size_t)D * KC * KC * 4;                               // step scores
-    o += (size_t)D * KC * 4;                                    // candidate ids
+    o += (size_t)(D + 1) * KC * 4;                              // candidate ids (and the depth before the window)
+    o += (size_t)D * KC * 4;                                    // candidate logits
+    o += (size_t)(D + 1) * 4 + (size_t)D * 4;                   // candidate counts, their division constants
+    o += (size_t)D * KC * 4;                                    // best step score after each previous slot
     o += align_up((size_t)D * KC, 4);                           // token-id ranks
-    o += (size_t)D * 4;                                         // candidate counts
     return o;
 }
 
@@ -67,41 +71,21 @@ __device__ __forceinline__ float proxy_score(const CpsArgs &a, int prev, int cur
     return __ldg(&a.table[h >> (32 - a.table_log2)]);
 }
 
-__device__ __forceinline__ unsigned long long kmax(unsigned long long a, unsigned long long b) { return a > b ? a : b; }
-__device__ __forceinline__ unsigned long long kmin(unsigned long long a, unsigned long long b) { return a < b ? a : b; }
+constexpr int kMaxExpansions = DSP_MAX_W * kMaxKC;        // expansions of one depth
+constexpr int kGatherBatch = 8;                             // proxy gathers a thread has in flight
 
-// Sort 32 keys, one per lane, descending over the lanes (bitonic network).
-__device__ __forceinline__ unsigned long long sort_keys_desc(unsigned long long v, int lane) {
-#pragma unroll
-    for (int k = 2; k <= 32; k <<= 1) {
-#pragma unroll
-        for (int j = k >> 1; j > 0; j >>= 1) {
-            const unsigned long long o = __shfl_xor_sync(0xFFFFFFFFu, v, j);
-            const bool up = (lane & k) == 0;
-            const bool lower = (lane & j) == 0;
-            v = (lower == up) ? kmax(v, o) : kmin(v, o);
-        }
-    }
-    return v;
-}
-// Best 32 of this warp's descending list `a` and another descending list given reversed
-// (`b_rev` = the other list's key of lane 31 - lane), descending: the lane-wise maximum is
-// bitonic and holds the best 32; five compare-exchange stages sort it.
-__device__ __forceinline__ unsigned long long merge_keys(unsigned long long a, unsigned long long b_rev, int lane) {
-    unsigned long long v = kmax(a, b_rev);
-#pragma unroll
-    for (int j = 16; j > 0; j >>= 1) {
-        const unsigned long long o = __shfl_xor_sync(0xFFFFFFFFu, v, j);
-        v = (lane & j) == 0 ? kmax(v, o) : kmin(v, o);
-    }
-    return v;
-}
+// floor(x / d) as a multiplication: m = floor(2^32 / d) + 1 is exact while x * d < 2^32
+// (here x < 2^16 and d <= 33^2).
+__device__ __forceinline__ unsigned long long div_magic(int d) { return (1ull << 32) / (unsigned)d + 1ull; }
+__device__ __forceinline__ int div_by(int x, unsigned long long m) { return (int)(((unsigned long long)(unsigned)x * m) >> 32); }
 
 __global__ void __launch_bounds__(kThreads) cps_kernel(const CpsArgs a) {
     extern __shared__ __align__(16) unsigned char dyn[];
-    __shared__ unsigned long long xch[2][kWarps][32];  // sorted keys of each warp, for the merges (two buffers in turn)
+    __shared__ __align__(16) unsigned long long surv[kMaxExpansions + 2];   // keys that can still be among the best W
     __shared__ float bcum[2][DSP_MAX_W];
     __shared__ int bslot[2][DSP_MAX_W];                // slot of each beam's last token
+    __shared__ __align__(16) uint32_t bbest[2][DSP_MAX_W];   // ord_bits of each beam's best expansion (free slots: all ones)
+    __shared__ int s_nsurv[2];                         // survivors of this depth / of the next (in turn)
     __shared__ int s_top_tok;                          // token of the rank-0 survivor
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -111,91 +95,154 @@ __global__ void __launch_bounds__(kThreads) cps_kernel(const CpsArgs a) {
     unsigned char *bp_slot = dyn + (size_t)L * W;
     unsigned char *walk = dyn + (size_t)2 * L * W;     // slot of beam w at depth i, after the walk
     float *step = reinterpret_cast<float *>(dyn + align_up((size_t)3 * L * W, 16));
-    int *cid = reinterpret_cast<int *>(step + (size_t)D * KC * KC);
-    unsigned char *trank = reinterpret_cast<unsigned char *>(cid + (size_t)D * KC);
-    int *ccnt = reinterpret_cast<int *>(trank + align_up((size_t)D * KC, 4));
+    int *cid = reinterpret_cast<int *>(step + (size_t)D * KC * KC);   // row 0: the depth before the window
+    float *clg = reinterpret_cast<float *>(cid + (size_t)(D + 1) * KC);
+    int *ccnt = reinterpret_cast<int *>(clg + (size_t)D * KC);        // entry 0: the depth before the window
+    unsigned *cinv = reinterpret_cast<unsigned *>(ccnt + D + 1);
+    float *smax = reinterpret_cast<float *>(cinv + D);                // [d][previous slot]: best step score
+    unsigned char *trank = reinterpret_cast<unsigned char *>(smax + (size_t)D * KC);
     const float lam = a.lambda;
     const float oml = __fsub_rn(1.0f, lam);
     const long long row0 = (long long)b * L;
+    const int KK = KC * KC;
+    const unsigned long long mKK = div_magic(KK), mKC = div_magic(KC);
 
-    int live = 1, cur = 0, m = L;
+    int live = 1, cur = 0, m = L, turn = 0;
     bool stopped = false;
-    if (tid == 0) { bcum[0][0] = 0.f; bslot[0][0] = 0; }
+    if (tid < 2 * DSP_MAX_W) {                          // both beam buffers: in-bounds values everywhere
+        (&bcum[0][0])[tid] = 0.f;
+        (&bslot[0][0])[tid] = 0;
+        (&bbest[0][0])[tid] = 0xFFFFFFFFu;
+    }
+    if (tid < 2) s_nsurv[tid] = 0;
 
     for (int i0 = 0; i0 < L && m == L && !stopped; i0 += D) {
         const int nd = min(D, L - i0);
-        // ---- window set-up: ids and counts, then step scores and token-id ranks, in parallel ----
+        // ---- window set-up: ids, logits and counts; step scores and token-id ranks; best steps ----
         __syncthreads();
-        for (int x = tid; x < nd; x += kThreads) ccnt[x] = max(0, min(a.cand_count[row0 + i0 + x], KC));
-        for (int x = tid; x < nd * KC; x += kThreads) cid[x] = a.cand_id[(row0 + i0) * KC + x];
+        for (int x = tid; x < nd; x += kThreads) {
+            const int c = max(0, min(a.cand_count[row0 + i0 + x], KC));
+            ccnt[1 + x] = c;
+            cinv[x] = c > 0 ? 65536u / (unsigned)c + 1u : 0u;       // floor(e / c) = (e * cinv) >> 16 for e < 2048
+        }
+        if (tid == 0) ccnt[0] = i0 == 0 ? 1 : max(0, min(a.cand_count[row0 + i0 - 1], KC));
+        for (int x = tid; x < nd * KC; x += kThreads) {
+            cid[KC + x] = a.cand_id[(row0 + i0) * KC + x];
+            clg[x] = a.cand_logit[(row0 + i0) * KC + x];
+        }
+        for (int x = tid; x < KC; x += kThreads) cid[x] = i0 == 0 ? a.prev_token[b] : a.cand_id[(row0 + i0 - 1) * KC + x];
         __syncthreads();
-        for (int x = tid; x < nd * KC * KC; x += kThreads) {
-            const int d = x / (KC * KC), rem = x - d * KC * KC;
-            const int p = rem / KC, k = rem - p * KC;
-            const int i = i0 + d;
-            const int pc = i == 0 ? 1 : (d > 0 ? ccnt[d - 1] : max(0, min(a.cand_count[row0 + i - 1], KC)));
-            if (k < ccnt[d] && p < pc) {
-                const int prev = i == 0 ? a.prev_token[b]
-                                        : (d > 0 ? cid[(d - 1) * KC + p] : a.cand_id[(row0 + i - 1) * KC + p]);
-                const float *lg = a.cand_logit + (row0 + i) * KC;
-                const float g = __fsub_rn(lg[k], lg[0]);
-                const float ng = proxy_score(a, prev, cid[d * KC + k]);
-                step[x] = __fadd_rn(__fmul_rn(lam, g), __fmul_rn(oml, ng));
+        const int total = nd * KK;
+        for (int x0 = tid; x0 < total; x0 += kThreads * kGatherBatch) {
+            float ng[kGatherBatch];
+            int at[kGatherBatch];                           // d * KC + k of a live entry, else -1
+#pragma unroll
+            for (int u = 0; u < kGatherBatch; ++u) {        // no branches: the gathers of a batch overlap
+                const int x = min(x0 + u * kThreads, total - 1);
+                const int d = div_by(x, mKK), rem = x - d * KK;
+                const int p = div_by(rem, mKC), k = rem - p * KC;
+                const bool ok = x0 + u * kThreads < total && k < ccnt[1 + d] && p < ccnt[d];
+                at[u] = ok ? d * KC + k : -1;
+                ng[u] = proxy_score(a, ok ? cid[d * KC + p] : 0, ok ? cid[(d + 1) * KC + k] : 0);
+            }
+#pragma unroll
+            for (int u = 0; u < kGatherBatch; ++u) {
+                if (at[u] >= 0) {
+                    const int d = div_by(at[u], mKC);
+                    const float g = __fsub_rn(clg[at[u]], clg[d * KC]);
+                    step[x0 + u * kThreads] = __fadd_rn(__fmul_rn(lam, g), __fmul_rn(oml, ng[u]));
+                }
             }
         }
         for (int x = tid; x < nd * KC; x += kThreads) {
-            const int d = x / KC, k = x - d * KC;
+            const int d = div_by(x, mKC), k = x - d * KC;
             int r = 0;
-            if (k < ccnt[d]) {
-                const int tok = cid[x];
-                for (int q = 0; q < ccnt[d]; ++q) r += cid[d * KC + q] < tok;
+            if (k < ccnt[1 + d]) {
+                const int tok = cid[KC + x];
+                for (int q = 0; q < ccnt[1 + d]; ++q) r += cid[(d + 1) * KC + q] < tok;
             }
             trank[x] = (unsigned char)r;
         }
         __syncthreads();
+        for (int x = tid; x < nd * KC; x += kThreads) {     // best step score after previous slot p
+            const int d = div_by(x, mKC), p = x - d * KC;
+            float best = -CUDART_INF_F;
+            if (p < ccnt[d])
+                for (int k = 0; k < ccnt[1 + d]; ++k) best = fmaxf(best, step[x * KC + k]);
+            smax[x] = best;
+        }
+        if (tid < live) {                                   // the beams' best expansions at the window's first depth
+            float best = -CUDART_INF_F;
+            const int p = bslot[cur][tid];
+            for (int k = 0; k < ccnt[1]; ++k) best = fmaxf(best, step[p * KC + k]);
+            bbest[cur][tid] = ord_bits(__fadd_rn(bcum[cur][tid], best));
+        }
+        __syncthreads();
 
         // ---- the depths of the window, one after the other ----
-        for (int d = 0; d < nd; ++d) {
+        for (int d = 0; d < nd; ++d, turn ^= 1) {
             const int i = i0 + d;
-            const int cnt = ccnt[d];
+            const int cnt = ccnt[1 + d];
             const int n = live * cnt;
             if (n == 0) { m = i; break; }               // an empty position ends the lattice
-            // every warp: its expansions, 32 at a time, sorted and merged into `best`
-            unsigned long long best = 0ull;
-            for (int base = warp * 32; base < n; base += kThreads) {
-                const int e = base + lane;
-                unsigned long long key = 0ull;
-                if (e < n) {
-                    const int w = e / cnt, k = e - w * cnt;
-                    const float cum = __fadd_rn(bcum[cur][w], step[(d * KC + bslot[cur][w]) * KC + k]);
-                    key = ((unsigned long long)ord_bits(cum) << 32) |
-                          ((unsigned long long)(255 - trank[d * KC + k]) << 24) |
-                          ((unsigned long long)(255 - w) << 16) | ((unsigned long long)(255 - k) << 8) | 1ull;
-                }
-                const unsigned long long sorted = sort_keys_desc(key, lane);
-                best = base < kThreads ? sorted : merge_keys(best, __shfl_sync(0xFFFFFFFFu, sorted, 31 - lane), lane);
-            }
-            // pairwise merges of the warps' lists (only as many levels as n needs)
-            int buf = 0;
-#pragma unroll
-            for (int span = 1; span < kWarps; span <<= 1) {
-                if (n > 32 * span) {
-                    xch[buf][warp][lane] = best;
-                    __syncthreads();
-                    if ((warp & (2 * span - 1)) == 0) best = merge_keys(best, xch[buf][warp + span][31 - lane], lane);
-                    buf ^= 1;                           // the next level writes the other buffer
-                }
-            }
-            // warp 0 holds the best min(32, n) expansions: the first min(W, n) survive
             const int keep = min(W, n);
             const int nxt = cur ^ 1;
-            if (warp == 0 && lane < keep) {
-                const int w = 255 - (int)((best >> 16) & 0xFF), k = 255 - (int)((best >> 8) & 0xFF);
-                bcum[nxt][lane] = __fadd_rn(bcum[cur][w], step[(d * KC + bslot[cur][w]) * KC + k]);
-                bslot[nxt][lane] = k;
-                bp_parent[(size_t)i * W + lane] = (unsigned char)w;
-                bp_slot[(size_t)i * W + lane] = (unsigned char)k;
-                if (lane == 0) s_top_tok = cid[d * KC + k];
+            // Every beam's best expansion is one of the n; with `keep` beams or more, the keep-th
+            // best expansion is at least the smallest of those, so anything below it is out.
+            uint32_t floor_ord = 0u;
+            if (live >= keep) {
+                floor_ord = 0xFFFFFFFFu;
+                const uint4 *bb = reinterpret_cast<const uint4 *>(bbest[cur]);
+#pragma unroll
+                for (int j = 0; j < DSP_MAX_W / 4; ++j) {
+                    const uint4 v = bb[j];
+                    floor_ord = min(min(floor_ord, min(v.x, v.y)), min(v.z, v.w));
+                }
+            }
+            const unsigned inv = cinv[d];
+            for (int e0 = warp * 32; e0 < n; e0 += kThreads) {
+                const int e = e0 + lane;
+                unsigned long long key = 0ull;
+                bool in = false;
+                if (e < n) {
+                    const int w = (int)(((unsigned)e * inv) >> 16), k = e - w * cnt;
+                    const float cum = __fadd_rn(bcum[cur][w], step[(d * KC + bslot[cur][w]) * KC + k]);
+                    const uint32_t ob = ord_bits(cum);
+                    in = ob >= floor_ord;
+                    key = ((unsigned long long)ob << 32) | ((unsigned long long)(255 - trank[d * KC + k]) << 24) |
+                          ((unsigned long long)(255 - w) << 16) | ((unsigned long long)(255 - k) << 8) | 1ull;
+                }
+                const unsigned ballot = __ballot_sync(0xFFFFFFFFu, in);
+                int base = 0;
+                if (lane == 0 && ballot) base = atomicAdd(&s_nsurv[turn], __popc(ballot));
+                base = __shfl_sync(0xFFFFFFFFu, base, 0);
+                if (in) surv[base + __popc(ballot & ((1u << lane) - 1u))] = key;
+            }
+            __syncthreads();
+            // The survivors are ranked by counting (all pairs; the keys are unique): the ranks
+            // below `keep` name the next beams, in order.
+            const int S = s_nsurv[turn];
+            if (tid == 0) s_nsurv[turn ^ 1] = 0;
+            const ulonglong2 *sp = reinterpret_cast<const ulonglong2 *>(surv);
+            for (int t = tid; t < S; t += kThreads) {
+                const unsigned long long q = surv[t];
+                int rank = 0;
+#pragma unroll 4
+                for (int j = 0; j < (S >> 1); ++j) {
+                    const ulonglong2 v = sp[j];
+                    rank += (v.x > q ? 1 : 0) + (v.y > q ? 1 : 0);
+                }
+                if (S & 1) rank += surv[S - 1] > q ? 1 : 0;
+                if (rank < keep) {
+                    const int w = 255 - (int)((q >> 16) & 0xFF), k = 255 - (int)((q >> 8) & 0xFF);
+                    const float cum = __fadd_rn(bcum[cur][w], step[(d * KC + bslot[cur][w]) * KC + k]);
+                    bcum[nxt][rank] = cum;
+                    bslot[nxt][rank] = k;
+                    if (d + 1 < nd) bbest[nxt][rank] = ord_bits(__fadd_rn(cum, smax[(d + 1) * KC + k]));
+                    bp_parent[(size_t)i * W + rank] = (unsigned char)w;
+                    bp_slot[(size_t)i * W + rank] = (unsigned char)k;
+                    if (rank == 0) s_top_tok = cid[(d + 1) * KC + k];
+                }
             }
             __syncthreads();
             live = keep;

@@ -194,11 +194,7 @@ __device__ void redo_sums(const DT *__restrict__ row, int s0, int s1, ScanSmem &
 template <typename DT, typename SY>
 __device__ void reduce_sums(const DT *__restrict__ row, int s0, int s1, ScanSmem &sm, float c, float S,
                             float T, float &c_out, double &S_out, double &T_out) {
-    constexpr int N = Elem<DT>::N;
-    constexpr int TE = tile_elems<DT>();
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const bool aligned = (reinterpret_cast<uintptr_t>(row) & 15) == 0;
-    const int ntiles = (s1 - s0 + TE - 1) / TE;
     float cb = warp_max(c);
     if (lane == 0) sm.redc[warp] = cb;
     SY::sync();
