@@ -81,10 +81,12 @@ __device__ __forceinline__ int div_by(int x, unsigned long long m) { return (int
 
 __global__ void __launch_bounds__(kThreads) cps_kernel(const CpsArgs a) {
     extern __shared__ __align__(16) unsigned char dyn[];
-    __shared__ __align__(16) unsigned long long surv[kMaxExpansions + 2];   // keys that can still be among the best W
+    // keys that can still be among the best W: two buffers in turn, the one not in use is zeroed
+    // meanwhile, so that the slots after the last key read as "below every key"
+    __shared__ __align__(16) unsigned long long surv[2][kMaxExpansions + 8];
     __shared__ float bcum[2][DSP_MAX_W];
     __shared__ int bslot[2][DSP_MAX_W];                // slot of each beam's last token
-    __shared__ __align__(16) uint32_t bbest[2][DSP_MAX_W];   // ord_bits of each beam's best expansion (free slots: all ones)
+    __shared__ uint32_t s_floor[2];                    // smallest ord_bits among the beams' own best expansions
     __shared__ int s_nsurv[2];                         // survivors of this depth / of the next (in turn)
     __shared__ int s_top_tok;                          // token of the rank-0 survivor
 
@@ -112,9 +114,9 @@ __global__ void __launch_bounds__(kThreads) cps_kernel(const CpsArgs a) {
     if (tid < 2 * DSP_MAX_W) {                          // both beam buffers: in-bounds values everywhere
         (&bcum[0][0])[tid] = 0.f;
         (&bslot[0][0])[tid] = 0;
-        (&bbest[0][0])[tid] = 0xFFFFFFFFu;
     }
     if (tid < 2) s_nsurv[tid] = 0;
+    for (int x = tid; x < 2 * (kMaxExpansions + 8); x += kThreads) (&surv[0][0])[x] = 0ull;
 
     for (int i0 = 0; i0 < L && m == L && !stopped; i0 += D) {
         const int nd = min(D, L - i0);
@@ -125,7 +127,10 @@ __global__ void __launch_bounds__(kThreads) cps_kernel(const CpsArgs a) {
             ccnt[1 + x] = c;
             cinv[x] = c > 0 ? 65536u / (unsigned)c + 1u : 0u;       // floor(e / c) = (e * cinv) >> 16 for e < 2048
         }
-        if (tid == 0) ccnt[0] = i0 == 0 ? 1 : max(0, min(a.cand_count[row0 + i0 - 1], KC));
+        if (tid == 0) {
+            ccnt[0] = i0 == 0 ? 1 : max(0, min(a.cand_count[row0 + i0 - 1], KC));
+            s_floor[cur] = 0xFFFFFFFFu;
+        }
         for (int x = tid; x < nd * KC; x += kThreads) {
             cid[KC + x] = a.cand_id[(row0 + i0) * KC + x];
             clg[x] = a.cand_logit[(row0 + i0) * KC + x];
@@ -175,7 +180,7 @@ __global__ void __launch_bounds__(kThreads) cps_kernel(const CpsArgs a) {
             float best = -CUDART_INF_F;
             const int p = bslot[cur][tid];
             for (int k = 0; k < ccnt[1]; ++k) best = fmaxf(best, step[p * KC + k]);
-            bbest[cur][tid] = ord_bits(__fadd_rn(bcum[cur][tid], best));
+            atomicMin(&s_floor[cur], ord_bits(__fadd_rn(bcum[cur][tid], best)));
         }
         __syncthreads();
 
@@ -189,16 +194,8 @@ __global__ void __launch_bounds__(kThreads) cps_kernel(const CpsArgs a) {
             const int nxt = cur ^ 1;
             // Every beam's best expansion is one of the n; with `keep` beams or more, the keep-th
             // best expansion is at least the smallest of those, so anything below it is out.
-            uint32_t floor_ord = 0u;
-            if (live >= keep) {
-                floor_ord = 0xFFFFFFFFu;
-                const uint4 *bb = reinterpret_cast<const uint4 *>(bbest[cur]);
-#pragma unroll
-                for (int j = 0; j < DSP_MAX_W / 4; ++j) {
-                    const uint4 v = bb[j];
-                    floor_ord = min(min(floor_ord, min(v.x, v.y)), min(v.z, v.w));
-                }
-            }
+            const uint32_t floor_ord = live >= keep ? s_floor[cur] : 0u;
+            if (tid == 0) s_floor[nxt] = 0xFFFFFFFFu;
             const unsigned inv = cinv[d];
             for (int e0 = warp * 32; e0 < n; e0 += kThreads) {
                 const int e = e0 + lane;
@@ -216,29 +213,30 @@ __global__ void __launch_bounds__(kThreads) cps_kernel(const CpsArgs a) {
                 int base = 0;
                 if (lane == 0 && ballot) base = atomicAdd(&s_nsurv[turn], __popc(ballot));
                 base = __shfl_sync(0xFFFFFFFFu, base, 0);
-                if (in) surv[base + __popc(ballot & ((1u << lane) - 1u))] = key;
+                if (in) surv[turn][base + __popc(ballot & ((1u << lane) - 1u))] = key;
             }
             __syncthreads();
             // The survivors are ranked by counting (all pairs; the keys are unique): the ranks
             // below `keep` name the next beams, in order.
             const int S = s_nsurv[turn];
             if (tid == 0) s_nsurv[turn ^ 1] = 0;
-            const ulonglong2 *sp = reinterpret_cast<const ulonglong2 *>(surv);
+            for (int x = tid; x < W * KC + 8; x += kThreads) surv[turn ^ 1][x] = 0ull;
+            const ulonglong2 *sp = reinterpret_cast<const ulonglong2 *>(surv[turn]);
             for (int t = tid; t < S; t += kThreads) {
-                const unsigned long long q = surv[t];
+                const unsigned long long q = surv[turn][t];
                 int rank = 0;
-#pragma unroll 4
-                for (int j = 0; j < (S >> 1); ++j) {
-                    const ulonglong2 v = sp[j];
-                    rank += (v.x > q ? 1 : 0) + (v.y > q ? 1 : 0);
+                for (int j = 0; j < S; j += 8) {            // eight keys a round; the slots after the last key are zero
+                    const ulonglong2 v0 = sp[(j >> 1) + 0], v1 = sp[(j >> 1) + 1], v2 = sp[(j >> 1) + 2],
+                                     v3 = sp[(j >> 1) + 3];
+                    rank += ((v0.x > q ? 1 : 0) + (v0.y > q ? 1 : 0)) + ((v1.x > q ? 1 : 0) + (v1.y > q ? 1 : 0)) +
+                            ((v2.x > q ? 1 : 0) + (v2.y > q ? 1 : 0)) + ((v3.x > q ? 1 : 0) + (v3.y > q ? 1 : 0));
                 }
-                if (S & 1) rank += surv[S - 1] > q ? 1 : 0;
                 if (rank < keep) {
                     const int w = 255 - (int)((q >> 16) & 0xFF), k = 255 - (int)((q >> 8) & 0xFF);
-                    const float cum = __fadd_rn(bcum[cur][w], step[(d * KC + bslot[cur][w]) * KC + k]);
+                    const float cum = ord_value((uint32_t)(q >> 32));    // as added up for the key (-0 reads as +0)
                     bcum[nxt][rank] = cum;
                     bslot[nxt][rank] = k;
-                    if (d + 1 < nd) bbest[nxt][rank] = ord_bits(__fadd_rn(cum, smax[(d + 1) * KC + k]));
+                    if (d + 1 < nd) atomicMin(&s_floor[nxt], ord_bits(__fadd_rn(cum, smax[(d + 1) * KC + k])));
                     bp_parent[(size_t)i * W + rank] = (unsigned char)w;
                     bp_slot[(size_t)i * W + rank] = (unsigned char)k;
                     if (rank == 0) s_top_tok = cid[(d + 1) * KC + k];
