@@ -198,7 +198,8 @@ int32_t dsp_lattice_build_static(const void *draft_logits, int32_t dtype,
  *          dsp_lattice_build (KC = their last dimension); prev_token int32 [B].
  * Outputs: path       int32 [B,L]   rank-0 path, -1 beyond path_len
  *          path_slot  int32 [B,L]   candidate slot of each path token, -1 beyond
- *          path_len   int32 [B]     m
+ *          path_len   int32 [B]     m (0 if the first position has no candidate: the one
+ *                                   surviving beam is then the empty path, score 0)
  *          path_score float [B]     Eq. 8 of the rank-0 path
  *          beam_ids   int32 [B,W,L] (nullable) all survivors by rank, -1 padded
  *          beam_score float [B,W]   (nullable) Eq. 8 per survivor, -inf if none

@@ -259,7 +259,7 @@ __global__ void __launch_bounds__(kThreads) cps_kernel(const CpsArgs a) {
     for (int o = 16; o > 0; o >>= 1) off += __shfl_xor_sync(0xFFFFFFFFu, off, o);
     if (lane == 0) s_off[warp] = off;
     // walk the back-pointers (shared memory only), one thread per surviving beam
-    const int nlive = m > 0 ? live : 0;
+    const int nlive = live;                            // m == 0: the one empty path, score 0
     if (tid < nlive) {
         int at = tid;
         for (int i = m - 1; i >= 0; --i) {

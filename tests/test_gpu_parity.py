@@ -1,9 +1,11 @@
 """GPU parity: the CUDA path, called through the C ABI, against the CPU oracle on the same bytes."""
 import math
+from types import SimpleNamespace
 
 import pytest
 import torch
 
+import oracle
 from paper_2510_02358_b200 import binding as dsp
 from paper_2510_02358_b200 import workloads as wl
 from parity import check_step, gpu_step
@@ -182,6 +184,63 @@ def test_adl_closed_loop_matches_oracle():
         assert nxt == ref.update(g.ver.accepted_len, g.lat.gen_len)
         assert abs(st.ema_gen - ref.ema_gen) < 1e-12 and abs(st.ema_acc - ref.ema_acc) < 1e-12
     assert len(seen) >= 2
+
+
+# ---- the path search alone, on lattices made by hand (sizes and ties the scans rarely give) ----
+def _hand_lattice(B, L, KC, V, seed, *, flat=False, counts=None):
+    g = torch.Generator().manual_seed(seed)
+    cand_id = torch.stack([torch.stack([torch.randperm(V, generator=g)[:KC] for _ in range(L)]) for _ in range(B)])
+    if flat:
+        logit = torch.zeros(B, L, KC)
+    else:
+        logit = torch.sort(torch.randn(B, L, KC, generator=g) * 2.0, dim=2, descending=True).values
+        logit = torch.round(logit * 4) / 4                 # quarter steps: many equal sums
+    cnt = torch.randint(1, KC + 1, (B, L), generator=g) if counts is None else counts
+    lse64 = torch.logsumexp(logit.double(), dim=2) + 0.5
+    return SimpleNamespace(cand_id=cand_id.int(), cand_logit=logit.float(), lse64=lse64, cand_count=cnt.int())
+
+
+@pytest.mark.parametrize("B,L,K,W,eos,lam,flat,case", [
+    (3, 128, 32, 32, True, 0.5, False, "max"),     # largest L, K, W with the EOS slot: 1056 expansions, several windows
+    (4, 40, 16, 16, True, 0.0, True, "flat"),      # equal logits and a constant proxy: every expansion ties
+    (4, 24, 8, 8, False, 1.0, False, "holes"),     # positions without candidates end the lattice
+    (6, 32, 16, 16, True, 0.5, False, "eos"),      # the best beam meets EOS and stops
+    (5, 33, 5, 7, False, 0.3, False, "odd"),       # W > K, odd sizes
+])
+def test_path_search_on_hand_made_lattices(B, L, K, W, eos, lam, flat, case):
+    V = 5000
+    KC = K + (1 if eos else 0)
+    eos_id = 17 if eos else -1
+    lat = _hand_lattice(B, L, KC, V, seed=L * 7 + K, flat=flat)
+    if case == "holes":
+        lat.cand_count[0, 5] = 0
+        lat.cand_count[1, 0] = 0
+        lat.cand_count[2, L - 1] = 0
+    if case == "eos":
+        lat.cand_id[0, 3, 0] = eos_id
+        lat.cand_id[1, 0, 0] = eos_id
+        lat.cand_count[1, 0] = 1                           # the only candidate: the search must stop at once
+        lat.cand_id[2, L - 1, 0] = eos_id
+        lat.cand_count[2, L - 1] = 1
+        lat.cand_id[3, 9, 1] = eos_id                      # not the best candidate: may or may not stop
+    g = torch.Generator().manual_seed(99)
+    table = torch.zeros(1 << 12) if flat else torch.round(torch.randn(1 << 12, generator=g) * 8) / 8 - 3.0
+    prev = torch.randint(0, V, (B,), generator=g).int()
+    kw = dict(W=W, lam=lam, eos_id=eos_id, table_log2=12, hash_seed=5, V=V)
+    o = oracle.cps_search(lat.cand_id, lat.cand_logit, lat.lse64, lat.cand_count, prev, table, **kw)
+    dlat = SimpleNamespace(**{k: v.to(DEV) for k, v in vars(lat).items()})
+    status = torch.zeros(B, dtype=torch.int32, device=DEV)
+    for _ in range(2):                                     # twice: the kernel's state starts clean each time
+        c = dsp.dsp_cps_search(dlat, prev.to(DEV), table.to(DEV), row_status=status, **kw)
+        torch.cuda.synchronize()
+        for name in ("path", "path_slot", "path_len", "beam_ids", "beam_cum"):
+            assert torch.equal(getattr(c, name).cpu(), getattr(o, name)), f"{case}: {name} differs"
+        assert torch.allclose(c.beam_score.cpu(), o.beam_score, atol=1e-3, rtol=1e-5, equal_nan=True)
+    assert torch.equal((status.cpu() & dsp.ROW_EOS_STOPPED) != 0, (o.row_status & oracle.EOS_STOPPED) != 0)
+    if case == "holes":
+        assert o.path_len[:3].tolist() == [5, 0, L - 1]
+    if case == "eos":
+        assert o.path_len[1] == 1 and o.path_len[2] == L and (o.row_status[1:3] & oracle.EOS_STOPPED).all()
 
 
 def test_profile_events_bracket_the_scan_kernels():
