@@ -12,9 +12,10 @@
  *    errors are detected on the host before anything is enqueued.
  *  - Unless marked "host", every pointer is a DEVICE pointer to memory the
  *    caller owns (inputs, outputs and the scratch workspace).  The library
- *    allocates nothing and keeps no device state between calls (two
- *    exceptions: dsp_lattice_build_static holds its scratch in a static array,
- *    and dsp_draft_verify_step keeps one stream and two events per device).
+ *    allocates nothing and keeps no device state between calls (exceptions:
+ *    dsp_lattice_build_static holds its scratch in a static array,
+ *    dsp_draft_verify_step keeps one stream and two events per device, and a
+ *    dsp_step_graph is a CUDA graph object).
  *  - Device calls only enqueue work on `stream` (a cudaStream_t; NULL is the
  *    legacy default stream) and never synchronise.  Outputs are valid once
  *    the stream reaches the end of the call.  Two calls that share a
@@ -303,6 +304,50 @@ int32_t dsp_draft_verify_step(
     uint32_t *row_status,
     void *lattice_workspace, size_t lattice_workspace_bytes,
     void *verify_workspace, size_t verify_workspace_bytes, dsp_stream_t stream);
+
+/* -------------------------------------------------------------------------
+ * A step recorded as a CUDA graph  (Alg. 1 stages 1-3 replayed; the draft
+ * length changes between steps by Eq. 11, over few values: one graph each).
+ *
+ * dsp_step_graph_create records one dsp_draft_verify_step call (same
+ * arguments, no stream) as a CUDA graph and returns a handle (host object,
+ * owned by the caller until dsp_step_graph_destroy).  Nothing runs at creation.
+ * dsp_step_graph_launch replays it on `stream`: same kernels, same results as
+ * the direct call, with the host's launch work of two memsets and up to seven
+ * kernels on two streams replaced by one graph launch.  The graph holds the
+ * addresses, sizes and scalar arguments given at creation: keep every buffer
+ * alive and in place while the handle lives, refresh inputs in place, and
+ * order launches that share buffers or workspaces (same stream).  One graph
+ * per draft length L (and per set of buffers); graphs of different L may
+ * share input buffers (strides) and workspaces sized for the largest L.
+ * Creation allocates (CUDA's graph objects), must not overlap another thread's
+ * dsp_draft_verify_step on the same device, and is refused (UNSUPPORTED)
+ * while events are set through dsp_profile_events.
+ * Errors : create: those of dsp_draft_verify_step, INVALID_ARG (out is null),
+ *          CUDA; launch: INVALID_ARG (null handle), CUDA; destroy: CUDA (a null
+ *          handle is fine).
+ */
+typedef struct dsp_step_graph dsp_step_graph;
+
+int32_t dsp_step_graph_create(
+    dsp_step_graph **out /* host, out */,
+    const void *draft_logits, const void *target_logits, int32_t dtype,
+    int32_t B, int32_t L, int32_t Lt, int32_t V,
+    int64_t dstride_b, int64_t dstride_l, int64_t tstride_b, int64_t tstride_l,
+    int32_t K_max, float tau, int32_t eos_id,
+    const int32_t *prev_token, int32_t proxy_kind, const float *proxy_table, int32_t table_log2,
+    uint32_t hash_seed, int32_t W, float lambda,
+    int32_t all_greedy, const uint8_t *mode, const float *u,
+    int32_t *cand_id, float *cand_logit, float *cand_logp, int32_t *cand_count,
+    float *lse, double *lse64, float *entropy, int32_t *gen_len,
+    int32_t *path, int32_t *path_slot, int32_t *path_len, float *path_score,
+    int32_t *beam_ids, float *beam_score, float *beam_cum,
+    int32_t *accepted_len, int32_t *next_token, float *ratio, int32_t *tgt_argmax, float *tgt_lse,
+    uint32_t *row_status,
+    void *lattice_workspace, size_t lattice_workspace_bytes,
+    void *verify_workspace, size_t verify_workspace_bytes);
+int32_t dsp_step_graph_launch(dsp_step_graph *graph, dsp_stream_t stream);
+int32_t dsp_step_graph_destroy(dsp_step_graph *graph);
 
 /* -------------------------------------------------------------------------
  * Adaptive draft length  (Sec. 3.3, Eq. 9-11; Alg. 1 init and stage 4) -- host.

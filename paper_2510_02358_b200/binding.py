@@ -28,6 +28,7 @@ DSP_MAX_K, DSP_MAX_W, DSP_MAX_L = 32, 32, 1024
 
 EXPORTS = ["dsp_strerror", "dsp_last_cuda_error", "dsp_version", "dsp_profile_events", "dsp_lattice_workspace_bytes",
            "dsp_lattice_build", "dsp_lattice_build_static", "dsp_cps_search", "dsp_verify_workspace_bytes", "dsp_verify", "dsp_draft_verify_step",
+           "dsp_step_graph_create", "dsp_step_graph_launch", "dsp_step_graph_destroy",
            "dsp_adl_init", "dsp_adl_update"]
 
 
@@ -238,15 +239,9 @@ def dsp_verify(target: torch.Tensor, draft: Optional[torch.Tensor], cps: SimpleN
     return out
 
 
-def dsp_draft_verify_step(draft: torch.Tensor, target: torch.Tensor, prev_token: torch.Tensor,
-                          table: torch.Tensor, *, K_max: int, W: int, lam: float, tau: float = 0.0,
-                          eos_id: int = -1, proxy_kind: int = 0, table_log2: int = 0, hash_seed: int = 0,
-                          mode: Optional[torch.Tensor] = None, u: Optional[torch.Tensor] = None,
-                          all_greedy: bool = False, lat: Optional[SimpleNamespace] = None,
-                          cps: Optional[SimpleNamespace] = None, ver: Optional[SimpleNamespace] = None,
-                          lattice_workspace: Optional[torch.Tensor] = None,
-                          verify_workspace: Optional[torch.Tensor] = None, stream=None):
-    """The three device calls of a step in one (same results); returns (lat, cps, ver)."""
+def _step_call(draft, target, prev_token, table, K_max, W, lam, tau, eos_id, proxy_kind, table_log2, hash_seed,
+               mode, u, all_greedy, lat, cps, ver, lattice_workspace, verify_workspace):
+    """Buffers (made where not given) and the argument list shared by the step and its graph."""
     B, L, V, dsb, dsl = _logits3(draft, "draft")
     Bt, Lt, Vt, tsb, tsl = _logits3(target, "target")
     if (Bt, Vt) != (B, V) or target.dtype != draft.dtype:
@@ -260,7 +255,7 @@ def dsp_draft_verify_step(draft: torch.Tensor, target: torch.Tensor, prev_token:
         lattice_workspace = alloc_workspace(dsp_lattice_workspace_bytes(B, L, V, dt, K_max), dev)
     if verify_workspace is None:
         verify_workspace = alloc_workspace(dsp_verify_workspace_bytes(B, L, Lt, V, dt), dev)
-    _check("dsp_draft_verify_step", lib().dsp_draft_verify_step(
+    args = (
         _ptr(draft), _ptr(target), dt, B, L, Lt, V, C.c_int64(dsb), C.c_int64(dsl), C.c_int64(tsb),
         C.c_int64(tsl), K_max, C.c_float(tau), eos_id, _ptr(prev_token), proxy_kind, _ptr(table), table_log2,
         C.c_uint32(hash_seed & 0xFFFFFFFF), W, C.c_float(lam), 1 if all_greedy else 0, _ptr(mode), _ptr(u),
@@ -270,8 +265,64 @@ def dsp_draft_verify_step(draft: torch.Tensor, target: torch.Tensor, prev_token:
         _ptr(cps.beam_score), _ptr(cps.beam_cum),
         _ptr(ver.accepted_len), _ptr(ver.next_token), _ptr(ver.ratio), _ptr(ver.tgt_argmax), _ptr(ver.tgt_lse),
         _ptr(lat.row_status), _ptr(lattice_workspace), C.c_size_t(lattice_workspace.numel()),
-        _ptr(verify_workspace), C.c_size_t(verify_workspace.numel()), _stream(stream)))
+        _ptr(verify_workspace), C.c_size_t(verify_workspace.numel()))
+    keep = (draft, target, prev_token, table, mode, u, lattice_workspace, verify_workspace)
+    return args, lat, cps, ver, keep
+
+
+def dsp_draft_verify_step(draft: torch.Tensor, target: torch.Tensor, prev_token: torch.Tensor,
+                          table: torch.Tensor, *, K_max: int, W: int, lam: float, tau: float = 0.0,
+                          eos_id: int = -1, proxy_kind: int = 0, table_log2: int = 0, hash_seed: int = 0,
+                          mode: Optional[torch.Tensor] = None, u: Optional[torch.Tensor] = None,
+                          all_greedy: bool = False, lat: Optional[SimpleNamespace] = None,
+                          cps: Optional[SimpleNamespace] = None, ver: Optional[SimpleNamespace] = None,
+                          lattice_workspace: Optional[torch.Tensor] = None,
+                          verify_workspace: Optional[torch.Tensor] = None, stream=None):
+    """The three device calls of a step in one (same results); returns (lat, cps, ver)."""
+    args, lat, cps, ver, _ = _step_call(draft, target, prev_token, table, K_max, W, lam, tau, eos_id, proxy_kind,
+                                        table_log2, hash_seed, mode, u, all_greedy, lat, cps, ver,
+                                        lattice_workspace, verify_workspace)
+    _check("dsp_draft_verify_step", lib().dsp_draft_verify_step(*args, _stream(stream)))
     return lat, cps, ver
+
+
+class StepGraph:
+    """Handle of dsp_step_graph_create: ``launch()`` replays the recorded step; ``lat``, ``cps``,
+    ``ver`` are its output buffers.  Holds references to every buffer the graph points at."""
+
+    def __init__(self, handle, lat, cps, ver, keep):
+        self._h, self.lat, self.cps, self.ver, self._keep = handle, lat, cps, ver, keep
+
+    def launch(self, stream=None):
+        _check("dsp_step_graph_launch", lib().dsp_step_graph_launch(self._h, _stream(stream)))
+
+    def destroy(self):
+        if self._h is not None:
+            h, self._h = self._h, None
+            _check("dsp_step_graph_destroy", lib().dsp_step_graph_destroy(h))
+
+    def __del__(self):
+        try:
+            self.destroy()
+        except Exception:
+            pass
+
+
+def dsp_step_graph_create(draft: torch.Tensor, target: torch.Tensor, prev_token: torch.Tensor,
+                          table: torch.Tensor, *, K_max: int, W: int, lam: float, tau: float = 0.0,
+                          eos_id: int = -1, proxy_kind: int = 0, table_log2: int = 0, hash_seed: int = 0,
+                          mode: Optional[torch.Tensor] = None, u: Optional[torch.Tensor] = None,
+                          all_greedy: bool = False, lat: Optional[SimpleNamespace] = None,
+                          cps: Optional[SimpleNamespace] = None, ver: Optional[SimpleNamespace] = None,
+                          lattice_workspace: Optional[torch.Tensor] = None,
+                          verify_workspace: Optional[torch.Tensor] = None) -> StepGraph:
+    """Record dsp_draft_verify_step on these buffers as a CUDA graph (nothing runs yet)."""
+    args, lat, cps, ver, keep = _step_call(draft, target, prev_token, table, K_max, W, lam, tau, eos_id,
+                                           proxy_kind, table_log2, hash_seed, mode, u, all_greedy, lat, cps, ver,
+                                           lattice_workspace, verify_workspace)
+    h = C.c_void_p(0)
+    _check("dsp_step_graph_create", lib().dsp_step_graph_create(C.byref(h), *args))
+    return StepGraph(h, lat, cps, ver, keep)
 
 
 def dsp_adl_init(k_min=20, k_max=30, delta=10.0, rho=0.5, granularity=1):

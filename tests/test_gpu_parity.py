@@ -243,6 +243,73 @@ def test_path_search_on_hand_made_lattices(B, L, K, W, eos, lam, flat, case):
         assert o.path_len[1] == 1 and o.path_len[2] == L and (o.row_status[1:3] & oracle.EOS_STOPPED).all()
 
 
+# ---- the step recorded as a CUDA graph ----
+def _same_outputs(a, b, w=None):
+    for s in ("lat", "cps", "ver"):
+        for k, v in vars(getattr(a, s)).items():
+            if v is None or (w is not None and all_greedy_unused(w, s, k)):
+                continue
+            assert torch.equal(v.cpu().view(torch.uint8), getattr(getattr(b, s), k).cpu().view(torch.uint8)), (s, k)
+
+
+def _graph_kwargs(inp, p):
+    kw = dict(K_max=p["K"], W=p["W"], lam=p["lam"], tau=p["tau"], eos_id=p["eos_id"],
+              table_log2=inp["table_log2"], hash_seed=inp["hash_seed"], all_greedy=p["all_greedy"])
+    if not p["all_greedy"]:
+        kw.update(mode=inp["mode"], u=inp["u"])
+    return kw
+
+
+@pytest.mark.parametrize("cid", [1, 2, 3, 4])
+def test_step_graph_replays_the_step(cid):
+    w = wl.CONFIGS[cid].scaled(**SMALL[cid])
+    if cid == 4:
+        w = w.scaled(V=50048)
+    p = _params(w)
+    inp = wl.make_inputs(w, step=3, device=DEV)
+    other = wl.make_inputs(w, step=4, device=DEV)
+    graph = dsp.dsp_step_graph_create(inp["draft"], inp["target"], inp["prev_token"], inp["table"],
+                                      **_graph_kwargs(inp, p))
+    for rep in range(3):
+        if rep == 1:                                       # new logits in place: the graph reads the same addresses
+            for k in ("draft", "target", "prev_token", "u"):
+                inp[k].copy_(other[k])
+        graph.launch()
+        torch.cuda.synchronize()
+        ns = SimpleNamespace(lat=graph.lat, cps=graph.cps, ver=graph.ver)
+        _same_outputs(gpu_step(inp, fused=True, **p), ns, w)
+    cpu = lambda x: SimpleNamespace(**{k: (v.cpu() if v is not None else None) for k, v in vars(x).items()})
+    check_step(SimpleNamespace(lat=cpu(graph.lat), cps=cpu(graph.cps), ver=cpu(graph.ver)), inp, **p)
+    graph.destroy()
+    graph.destroy()                                        # a second destroy is harmless
+
+
+def test_step_graphs_per_draft_length_share_buffers():
+    """One graph per draft length (the controller's buckets) over the same logits buffers and workspaces."""
+    B, Lmax, V, K, W = 3, 16, 16384, 8, 4
+    inp = _to(wl.tiny_random(B, Lmax, V, dtype=torch.bfloat16, seed=21))
+    p = dict(K=K, W=W, tau=0.0, lam=0.5, eos_id=-1, all_greedy=False)
+    dt = dsp.DSP_BF16
+    ws_l = dsp.alloc_workspace(dsp.dsp_lattice_workspace_bytes(B, Lmax, V, dt, K), DEV)
+    ws_v = dsp.alloc_workspace(dsp.dsp_verify_workspace_bytes(B, Lmax, Lmax, V, dt), DEV)
+    graphs = {}
+    for L in (4, 8, 16):
+        view = dict(inp, draft=inp["draft"][:, :L], target=inp["target"][:, :L], u=inp["u"][:, :L + 1].contiguous())
+        graphs[L] = (view, dsp.dsp_step_graph_create(view["draft"], view["target"], view["prev_token"], view["table"],
+                                                     lattice_workspace=ws_l, verify_workspace=ws_v,
+                                                     **_graph_kwargs(view, p)))
+    for L in (8, 16, 4, 16):
+        view, graph = graphs[L]
+        graph.launch()
+        torch.cuda.synchronize()
+        _same_outputs(gpu_step(view, fused=True, **p), SimpleNamespace(lat=graph.lat, cps=graph.cps, ver=graph.ver))
+    with pytest.raises(dsp.DspError):                      # argument errors surface at creation, nothing is left captured
+        dsp.dsp_step_graph_create(inp["draft"], inp["target"], inp["prev_token"], inp["table"], K_max=K, W=999,
+                                  lam=0.5, table_log2=10, mode=inp["mode"], u=inp["u"])
+    g = gpu_step(inp, fused=True, **p)                     # the library still works after the refused capture
+    check_step(g, inp, **p)
+
+
 def test_profile_events_bracket_the_scan_kernels():
     w = wl.CONFIGS[3].scaled(B=2, L=4, V=152064)
     inp = wl.make_inputs(w, device=DEV)
