@@ -130,6 +130,16 @@ class GpuStep:
             all_greedy=self.all_greedy, lat=self.lat, cps=self.cps, ver=self.ver,
             lattice_workspace=self.ws_l, verify_workspace=self.ws_v)
 
+    def graph(self, inp):
+        """The single-call step on ``inp`` recorded as a CUDA graph (same outputs and workspaces)."""
+        dsp, w = self.dsp, self.w
+        return dsp.dsp_step_graph_create(
+            inp["draft"], inp["target"], inp["prev_token"], inp["table"], K_max=w.K, W=w.W, lam=w.lam,
+            tau=w.tau, eos_id=w.eos_id, table_log2=inp["table_log2"], hash_seed=inp["hash_seed"],
+            mode=None if self.all_greedy else inp["mode"], u=None if self.all_greedy else inp["u"],
+            all_greedy=self.all_greedy, lat=self.lat, cps=self.cps, ver=self.ver,
+            lattice_workspace=self.ws_l, verify_workspace=self.ws_v)
+
     def run(self, inp, ev=None):
         """The same step as three calls, with an event after each (the per-stage times)."""
         dsp, w = self.dsp, self.w
@@ -227,6 +237,22 @@ def time_workload(w, device, steps, warmup, dist=None, stages=True, seed_base=0)
                    ms_lattice_min=min(tl), ms_verify_min=min(tv))
     out["mean_accepted_len"] = st.ver.accepted_len.float().mean().item()
     out["mean_path_len"] = st.cps.path_len.float().mean().item()
+    if stages:
+        # the same step replayed from CUDA graphs (one per input set: a graph holds its addresses)
+        graphs = [st.graph(inp) for inp in sets]
+        for i in range(min(warmup, 2 * len(graphs))):
+            graphs[i % len(graphs)].launch()
+        torch.cuda.synchronize()
+        n = min(steps, 500)
+        g0, g1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        g0.record()
+        for i in range(n):
+            graphs[i % len(graphs)].launch()
+        g1.record()
+        torch.cuda.synchronize()
+        out["ms_graph_step"] = g0.elapsed_time(g1) / n
+        for g in graphs:
+            g.destroy()
     return out, st, sets
 
 
@@ -413,6 +439,9 @@ def main():
         "stage_ms": {"lattice_build": m["ms_lattice"], "cps_search": m["ms_cps"], "verify": m["ms_verify"],
                      "note": "the three calls one after the other; `value` times dsp_draft_verify_step, "
                              "which overlaps the target statistics with the path search"},
+        "graph_replay": {"ms_per_step": m.get("ms_graph_step"),
+                         "steps_per_s": 1e3 / m["ms_graph_step"] * world if m.get("ms_graph_step") else None,
+                         "note": "the same step replayed through dsp_step_graph_launch (not the timed `value`)"},
         "mean_accepted_len": m["mean_accepted_len"], "mean_path_len": m["mean_path_len"],
         "roofline": {"bound": "hbm", "kernel": "lattice_scan_kernel", "achieved": gbs_scan, "peak": peak,
                      "peak_kind": "%s copy bandwidth" % peak_kind, "unit": "GB/s", "frac": gbs_scan / peak,
@@ -439,6 +468,7 @@ def main():
                 tb = wv.logits_bytes
                 extras[wv.name] = {
                     "steps_per_s": 1e3 / mm["ms_per_step"], "ms_per_step": mm["ms_per_step"],
+                    "graph_ms_per_step": mm.get("ms_graph_step"),
                     "stage_ms": {"lattice_build": mm["ms_lattice"], "cps_search": mm["ms_cps"],
                                  "verify": mm["ms_verify"]},
                     "logits_gbs": 2 * tb / ((mm["ms_lattice"] + mm["ms_verify"]) * 1e-3) / 1e9,
