@@ -147,6 +147,23 @@ def proxy_score(table, prev: int, cur: int, *, proxy_kind=0, table_log2=0, hash_
                                        C.c_uint32(hash_seed & 0xFFFFFFFF), C.c_int64(V), prev, cur))
 
 
+def unmask_step(logits: torch.Tensor, tokens, masked, n_update: int):
+    """One refinement step (Eq. 5, top-K by confidence); returns new tokens / masked and the per-position
+    argmax, confidence (log-probability of the argmax, fp32), n_left and row_status."""
+    logits = logits.contiguous()
+    B, L, V = logits.shape
+    o = SimpleNamespace(
+        tokens=_np(tokens, np.int32).copy(), masked=_np(masked, np.uint8).copy(),
+        argmax=np.empty((B, L), np.int32), confidence=np.empty((B, L), np.float32),
+        n_left=np.empty((B,), np.int32), row_status=np.zeros((B,), np.uint32))
+    rc = lib().orc_unmask_step(_logits_ptr(logits), _dtype_code(logits), B, L, C.c_int64(V), int(n_update),
+                               _p(o.tokens), _p(o.masked), _p(o.argmax), _p(o.confidence), _p(o.n_left),
+                               _p(o.row_status))
+    if rc != 0:
+        raise ValueError("orc_unmask_step: bad arguments")
+    return SimpleNamespace(**{k: torch.from_numpy(v) for k, v in vars(o).items()})
+
+
 def verify(target: torch.Tensor, draft, path, path_len, mode=None, u=None, eos_id: int = -1):
     target = target.contiguous()
     B, Lt, V = target.shape

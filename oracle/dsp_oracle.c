@@ -529,6 +529,65 @@ int orc_verify(const void *target, const void *draft, int dtype, int B, int L, i
 }
 
 /*
+ * One refinement step of the diffusion drafter, on its logits (Sec. 3.1,
+ * Eq. 5, with the update set "top-K by confidence").
+ * For every position i of batch row b that is still masked:
+ *   a_i    = argmax_v x_{i,v}            (lowest id on ties)
+ *   conf_i = log q(a_i) = x_max - lse     (rounded to fp32: the precision in
+ *            which positions are compared)
+ * U = the min(n_update, |M|) masked positions with the largest conf (equal
+ * conf: the lower position first).  For i in U: tokens[i] = a_i and
+ * masked[i] = 0; every other entry of tokens / masked stays as it is.
+ * argmax / confidence report a_i / conf_i of the positions that were masked
+ * on entry and -1 / -inf elsewhere; n_left[b] = |M| on return.
+ * A masked row with NaN / +inf or without a finite logit flags the batch row
+ * (ORC_NONFINITE_INPUT) and takes conf = -inf.
+ */
+int orc_unmask_step(const void *logits, int dtype, int B, int L, int64_t V, int n_update,
+                    int32_t *tokens, uint8_t *masked, int32_t *argmax, float *confidence,
+                    int32_t *n_left, uint32_t *row_status)
+{
+    if (B < 0 || L < 1 || V < 1 || n_update < 1) return -1;
+    #pragma omp parallel for schedule(dynamic)
+    for (int b = 0; b < B; ++b) {
+        uint32_t status = 0;
+        int nmask = 0;
+        for (int i = 0; i < L; ++i) {
+            const int64_t r = (int64_t)b * L + i;
+            argmax[r] = -1;
+            confidence[r] = -INFINITY;
+            if (!masked[r]) continue;
+            ++nmask;
+            const char *row = (const char *)logits + (size_t)r * (size_t)V * (dtype == 0 ? 4 : 2);
+            double lse;
+            int64_t am;
+            if (row_stats(row, dtype, V, &lse, NULL, &am)) {
+                status |= ORC_NONFINITE_INPUT;
+                argmax[r] = (int32_t)am;
+                continue;
+            }
+            argmax[r] = (int32_t)am;
+            confidence[r] = (float)(logit_at(row, dtype, am) - lse);
+        }
+        const int take = n_update < nmask ? n_update : nmask;
+        for (int t = 0; t < take; ++t) {
+            int best = -1;
+            for (int i = 0; i < L; ++i) {                 /* strict >: the lower position wins ties */
+                const int64_t r = (int64_t)b * L + i;
+                if (!masked[r]) continue;
+                if (best < 0 || confidence[r] > confidence[(int64_t)b * L + best]) best = i;
+            }
+            const int64_t r = (int64_t)b * L + best;
+            tokens[r] = argmax[r];
+            masked[r] = 0;
+        }
+        n_left[b] = nmask - take;
+        if (row_status) row_status[b] = status;
+    }
+    return 0;
+}
+
+/*
  * Adaptive draft length (Sec. 3.3, Eq. 9-11; Alg. 1 init and stage 4).
  * state = { ema_gen, ema_acc, k }.  Init: both averages 0, k = k_max.
  * Update with the batch means of gen_len and accepted_len (batch 1 is the
