@@ -306,6 +306,44 @@ int32_t dsp_draft_verify_step(
     void *verify_workspace, size_t verify_workspace_bytes, dsp_stream_t stream);
 
 /* -------------------------------------------------------------------------
+ * Refinement step of the diffusion drafter  (Sec. 3.1, Eq. 5: iterative
+ * refinement with the update set "top-K by confidence"; the paper's default
+ * S = 1 needs a single call with n_update >= L, S > 1 is its ablation).
+ *
+ * logits [B,L,V] are the drafter's per-position conditionals for the block at
+ * this refinement step.  For every position i of batch row b with
+ * masked[b,i] != 0:
+ *   a_i    = argmax_v x[b,i,v]            (lowest id on ties)
+ *   conf_i = log q(a_i) = x_max - lse     (fp32; positions are compared in fp32)
+ * The min(n_update, #masked) masked positions of largest conf (equal conf: the
+ * lower position first) are revealed: tokens[b,i] = a_i, masked[b,i] = 0.
+ * Rows of positions that are already revealed are not read.
+ *
+ * Inputs : logits (dtype, strides in elements, as for dsp_lattice_build);
+ *          n_update >= 1.
+ * In/out : tokens int32 [B,L], masked uint8 [B,L] (entries of revealed
+ *          positions are left as they are).
+ * Outputs: argmax int32 [B,L], confidence float [B,L]: a_i and conf_i of the
+ *          positions masked on entry, -1 and -inf elsewhere;
+ *          n_left int32 [B] = positions still masked on return;
+ *          row_status uint32 [B] (written): DSP_ROW_NONFINITE_INPUT if a masked
+ *          row holds NaN / +inf or no finite logit (that position takes
+ *          conf = -inf; the batch row's outputs are then unspecified but in
+ *          bounds), DSP_ROW_TIMEOUT.
+ * workspace: dsp_unmask_workspace_bytes(B, L, V, dtype), 256-byte aligned.
+ * Errors : INVALID_ARG (null pointer, sizes, strides, n_update < 1,
+ *          alignment), UNSUPPORTED (dtype, L > DSP_MAX_L, V > 2^30), WORKSPACE,
+ *          CUDA.
+ */
+int32_t dsp_unmask_workspace_bytes(int32_t B, int32_t L, int32_t V, int32_t dtype,
+                                   size_t *bytes /* host, out */);
+int32_t dsp_unmask_step(const void *logits, int32_t dtype, int32_t B, int32_t L, int32_t V,
+                        int64_t stride_b, int64_t stride_l, int32_t n_update,
+                        int32_t *tokens, uint8_t *masked, int32_t *argmax, float *confidence,
+                        int32_t *n_left, uint32_t *row_status,
+                        void *workspace, size_t workspace_bytes, dsp_stream_t stream);
+
+/* -------------------------------------------------------------------------
  * A step recorded as a CUDA graph  (Alg. 1 stages 1-3 replayed; the draft
  * length changes between steps by Eq. 11, over few values: one graph each).
  *

@@ -29,6 +29,7 @@ DSP_MAX_K, DSP_MAX_W, DSP_MAX_L = 32, 32, 1024
 EXPORTS = ["dsp_strerror", "dsp_last_cuda_error", "dsp_version", "dsp_profile_events", "dsp_lattice_workspace_bytes",
            "dsp_lattice_build", "dsp_lattice_build_static", "dsp_cps_search", "dsp_verify_workspace_bytes", "dsp_verify", "dsp_draft_verify_step",
            "dsp_step_graph_create", "dsp_step_graph_launch", "dsp_step_graph_destroy",
+           "dsp_unmask_workspace_bytes", "dsp_unmask_step",
            "dsp_adl_init", "dsp_adl_update"]
 
 
@@ -323,6 +324,36 @@ def dsp_step_graph_create(draft: torch.Tensor, target: torch.Tensor, prev_token:
     h = C.c_void_p(0)
     _check("dsp_step_graph_create", lib().dsp_step_graph_create(C.byref(h), *args))
     return StepGraph(h, lat, cps, ver, keep)
+
+
+def dsp_unmask_workspace_bytes(B: int, L: int, V: int, dtype: int) -> int:
+    n = C.c_size_t(0)
+    _check("dsp_unmask_workspace_bytes", lib().dsp_unmask_workspace_bytes(B, L, V, dtype, C.byref(n)))
+    return n.value
+
+
+def dsp_unmask_step(logits: torch.Tensor, tokens: torch.Tensor, masked: torch.Tensor, n_update: int, *,
+                    out: Optional[SimpleNamespace] = None, workspace: Optional[torch.Tensor] = None,
+                    stream=None) -> SimpleNamespace:
+    """One refinement step of the drafter: ``tokens`` (int32 [B,L]) and ``masked`` (uint8 [B,L]) are
+    updated in place; returns argmax, confidence, n_left, row_status."""
+    B, L, V, sb, sl = _logits3(logits, "logits")
+    dev = logits.device
+    for t, dt in ((tokens, torch.int32), (masked, torch.uint8)):
+        if t.dtype != dt or tuple(t.shape) != (B, L) or not t.is_contiguous() or t.device != dev:
+            raise ValueError("tokens / masked must be contiguous [B, L] int32 / uint8 tensors on the logits' device")
+    if out is None:
+        e = lambda shape, dt: torch.empty(shape, dtype=dt, device=dev)
+        out = SimpleNamespace(argmax=e((B, L), torch.int32), confidence=e((B, L), torch.float32),
+                              n_left=e((B,), torch.int32), row_status=e((B,), torch.int32))
+    dt = _dtype(logits)
+    if workspace is None:
+        workspace = alloc_workspace(dsp_unmask_workspace_bytes(B, L, V, dt), dev)
+    _check("dsp_unmask_step", lib().dsp_unmask_step(
+        _ptr(logits), dt, B, L, V, C.c_int64(sb), C.c_int64(sl), int(n_update), _ptr(tokens), _ptr(masked),
+        _ptr(out.argmax), _ptr(out.confidence), _ptr(out.n_left), _ptr(out.row_status), _ptr(workspace),
+        C.c_size_t(workspace.numel()), _stream(stream)))
+    return out
 
 
 def dsp_adl_init(k_min=20, k_max=30, delta=10.0, rho=0.5, granularity=1):

@@ -1,0 +1,270 @@
+// dsp_unmask_step: one refinement step of the diffusion drafter on its logits (Sec. 3.1, Eq. 5,
+// with the update set "top-K by confidence").
+//
+// For every position that is still masked the step needs the row's argmax and its probability:
+// the same whole-vocabulary statistics as the lattice and the verification, with K = 1.  Rows
+// whose first element is 16-byte aligned take the same two passes: unmask_scan_kernel streams the
+// masked rows (stream_core.cuh; CTAs of revealed rows leave at once, so a later refinement step
+// reads only what is still masked), unmask_rows_kernel (one warp per row, row_warp.cuh) adds up
+// the sums and takes the argmax from the table of tile maxima.  Any other layout is read
+// element-wise by the row's warp (slower, same results).  The warp that finishes the last row of
+// a batch row ranks the masked positions by confidence (counting; equal confidence: the lower
+// position first), reveals the best n_update and writes what is left.
+#include "dsp_internal.h"
+#include "row_warp.cuh"
+
+namespace dsp {
+
+struct UnmaskArgs {
+    const void *logits;
+    int B, L, V;
+    long long stride_b, stride_l;
+    int n_update;
+    int32_t *tokens;
+    uint8_t *masked;
+    int32_t *argmax;
+    float *confidence;
+    int32_t *n_left;
+    uint32_t *row_status;
+    int streaming;            // 1: the rows were streamed by unmask_scan_kernel
+    int nslices, slice_elems, ntiles_row;
+    // workspace
+    unsigned *b_ticket;       // [B]  zeroed per call
+    unsigned *b_status;       // [B]  zeroed per call
+    WarpPartial *wpart;       // [B*L, nslices, kWarps]
+    void *table;              // [B*L, ntiles_row + nslices, kThreads], element type of the logits
+};
+
+struct UnmaskWs {
+    size_t off_b_ticket, off_b_status, zero_bytes, off_wpart, off_table, total;
+};
+static UnmaskWs unmask_ws_layout(int64_t B, int64_t L, int nslices, int ntiles_row, size_t es) {
+    UnmaskWs w;
+    size_t o = 0;
+    w.off_b_ticket = o; o += align_up((size_t)B * 4, 256);
+    w.off_b_status = o; o += align_up((size_t)B * 4, 256);
+    w.zero_bytes = o;
+    w.off_wpart = o;    o += align_up((size_t)(B * L) * nslices * kWarps * sizeof(WarpPartial), 256);
+    w.off_table = o;    o += align_up((size_t)(B * L) * (ntiles_row + nslices) * kThreads * es, 256);
+    w.total = o;
+    return w;
+}
+
+// Pass 1 over the rows that are still masked: one CTA per row slice.
+template <typename DT>
+__global__ void __launch_bounds__(kThreads, 4) unmask_scan_kernel(const UnmaskArgs a) {
+    extern __shared__ __align__(128) unsigned char ring[];
+    __shared__ StreamBars bars;
+    const long long row = blockIdx.x / a.nslices;
+    if (!a.masked[row]) return;                          // revealed earlier: nothing to compute (whole CTA)
+    const int slice = blockIdx.x - (int)(row * a.nslices);
+    const int b = (int)(row / a.L), l = (int)(row - (long long)b * a.L);
+    const DT *rowp = reinterpret_cast<const DT *>(a.logits) + b * a.stride_b + l * a.stride_l;
+    const int s0 = slice * a.slice_elems;
+    const int s1 = min(a.V, s0 + a.slice_elems);
+    stream_begin(bars);
+    DT *trow = reinterpret_cast<DT *>(a.table) + row * (a.ntiles_row + a.nslices) * kThreads;
+    DT *tab = trow + (long long)(s0 / tile_elems<DT>()) * kThreads;
+    DT *smax = trow + (long long)(a.ntiles_row + slice) * kThreads;
+    stream_slice<DT>(rowp, s0, s1, true, bars, ring, tab, smax, a.wpart + (row * a.nslices + slice) * kWarps);
+    if (threadIdx.x == 0 && bars.timed_out) atomicOr(&a.b_status[b], DSP_ROW_TIMEOUT);
+}
+
+// Argmax (lowest id on ties), its logit and the row's log-sum-exp by one warp, element by
+// element: for rows that cannot be streamed.  Returns false for NaN / +inf or no finite logit.
+template <typename DT>
+__device__ bool warp_row_stats_elementwise(const DT *__restrict__ row, int V, int lane, int &am, float &xmax,
+                                           double &lse) {
+    float m = -CUDART_INF_F;
+    int id = 0x7FFFFFFF;
+    bool bad = false;
+    for (int v = lane; v < V; v += 32) {
+        const float x = Elem<DT>::load1(row + v);
+        bad |= x != x || x == CUDART_INF_F;
+        if (x > m) { m = x; id = v; }                    // ascending ids: the first of equals stays
+    }
+    bad = __any_sync(0xFFFFFFFFu, bad);
+    const float mm = warp_max(m);
+    int cand = m == mm ? id : 0x7FFFFFFF;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) cand = min(cand, __shfl_xor_sync(0xFFFFFFFFu, cand, o));
+    am = cand == 0x7FFFFFFF ? 0 : cand;
+    xmax = mm;
+    if (bad || !(mm > -CUDART_INF_F)) { lse = CUDART_NAN; return false; }
+    double S = 0.0;
+    for (int v0 = lane; v0 < V; v0 += 32 * 64) {         // fp32 partial sums of 64 terms, added up in double
+        float s = 0.f;
+        for (int q = 0; q < 64; ++q) {
+            const int v = v0 + q * 32;
+            if (v < V) s += ex2_approx((Elem<DT>::load1(row + v) - mm) * kLog2e);
+        }
+        S += (double)s;
+    }
+    S = warp_sum(S);
+    lse = (double)mm + kLn2 * log2(S);
+    return true;
+}
+
+// Pass 2 and the update: one warp per row; the warp arriving last for a batch row reveals the
+// best n_update masked positions.
+template <typename DT>
+__global__ void __launch_bounds__(kThreads) unmask_rows_kernel(const UnmaskArgs a) {
+    __shared__ WarpScratch scratch[kRowWarps];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const long long row = (long long)blockIdx.x * kRowWarps + warp;
+    if (row >= (long long)a.B * a.L) return;
+    const int b = (int)(row / a.L), l = (int)(row - (long long)b * a.L);
+    const DT *rowp = reinterpret_cast<const DT *>(a.logits) + b * a.stride_b + l * a.stride_l;
+
+    int am = -1;
+    float conf = -CUDART_INF_F;
+    if (a.masked[row]) {                                 // read before anyone's update: updates follow the last ticket
+        bool ok;
+        float xmax = 0.f;
+        double lse = 0.0;
+        if (a.streaming) {
+            float c;
+            double S, T;
+            warp_merge_partials(a.wpart + row * a.nslices * kWarps, a.nslices * kWarps, lane, c, S, T);
+            if (T != T && S == S && S < CUDART_INF) warp_redo_sums<DT>(rowp, a.V, lane, c, S, T);
+            const unsigned long long key = warp_select_topk<DT>(
+                rowp, a.V, 1, reinterpret_cast<const DT *>(a.table) + row * (a.ntiles_row + a.nslices) * kThreads,
+                a.ntiles_row, a.nslices, scratch[warp], lane);
+            const unsigned long long best = __shfl_sync(0xFFFFFFFFu, key, 0);
+            double mean_x;
+            ok = row_log_stats(c, S, T, lse, mean_x) && best != 0ull;
+            am = best ? key_id(best) : 0;
+            xmax = best ? key_value(best) : 0.f;
+        } else {
+            ok = warp_row_stats_elementwise<DT>(rowp, a.V, lane, am, xmax, lse);
+        }
+        if (ok) conf = (float)((double)xmax - lse);
+        else if (lane == 0) atomicOr(&a.b_status[b], DSP_ROW_NONFINITE_INPUT);
+    }
+    if (lane == 0) {
+        a.argmax[row] = am;
+        a.confidence[row] = conf;
+    }
+    // ---- last row of this batch row: rank the masked positions and reveal the best ----
+    __threadfence();
+    __syncwarp();
+    unsigned ticket = 0;
+    if (lane == 0) ticket = atomicAdd(&a.b_ticket[b], 1u);
+    ticket = __shfl_sync(0xFFFFFFFFu, ticket, 0);
+    if (ticket != (unsigned)a.L - 1) return;
+    __threadfence();
+    static_assert(DSP_MAX_L <= 32 * 32, "one reveal bit per position and lane");
+    const long long r0 = (long long)b * a.L;
+    int nmask = 0;
+    for (int i0 = 0; i0 < a.L; i0 += 32) {
+        const int i = i0 + lane;
+        nmask += __popc(__ballot_sync(0xFFFFFFFFu, i < a.L && a.masked[r0 + i] != 0));
+    }
+    const int take = min(a.n_update, nmask);
+    unsigned reveal = 0u;                                // bit q: this lane's q-th position is revealed
+    for (int i = lane, q = 0; i < a.L; i += 32, ++q) {
+        if (!a.masked[r0 + i]) continue;
+        const float ci = __ldcg(&a.confidence[r0 + i]);
+        int before = 0;                                  // masked positions that come first
+        for (int j = 0; j < a.L; ++j) {
+            const float cj = __ldcg(&a.confidence[r0 + j]);
+            before += (a.masked[r0 + j] && (cj > ci || (cj == ci && j < i))) ? 1 : 0;
+        }
+        if (before < take) reveal |= 1u << q;
+    }
+    __syncwarp();                                        // every lane has read the mask: now it may change
+    for (int i = lane, q = 0; i < a.L; i += 32, ++q) {
+        if (reveal & (1u << q)) {
+            a.tokens[r0 + i] = __ldcg(&a.argmax[r0 + i]);
+            a.masked[r0 + i] = 0;
+        }
+    }
+    if (lane == 0) {
+        a.n_left[b] = nmask - take;
+        a.row_status[b] = atomicOr(&a.b_status[b], 0u);
+    }
+}
+
+template <typename DT>
+static int32_t launch_unmask(UnmaskArgs &a, void *workspace, size_t workspace_bytes, cudaStream_t st) {
+    const long long nrows = (long long)a.B * a.L;
+    const SlicePlan plan = plan_slices<DT>(nrows, a.V, kTargetCtas);
+    a.nslices = plan.nslices;
+    a.slice_elems = plan.slice_elems;
+    a.ntiles_row = (a.V + tile_elems<DT>() - 1) / tile_elems<DT>();
+    const UnmaskWs w = unmask_ws_layout(a.B, a.L, a.nslices, a.ntiles_row, sizeof(DT));
+    if (workspace_bytes < w.total) return DSP_ERR_WORKSPACE;
+    unsigned char *ws = static_cast<unsigned char *>(workspace);
+    a.b_ticket = reinterpret_cast<unsigned *>(ws + w.off_b_ticket);
+    a.b_status = reinterpret_cast<unsigned *>(ws + w.off_b_status);
+    a.wpart = reinterpret_cast<WarpPartial *>(ws + w.off_wpart);
+    a.table = ws + w.off_table;
+    DSP_CUDA_TRY(cudaMemsetAsync(ws, 0, w.zero_bytes, st));
+    const long long nblocks = nrows * a.nslices;
+    if (nblocks > 0x7FFFFFFFLL) return DSP_ERR_UNSUPPORTED;
+    a.streaming = a.nslices * kWarps <= kThreads && stream_layout_ok<DT>(a.logits, a.V, a.stride_b, a.stride_l);
+    if (a.streaming) {
+        static RingSmemDone smem_done;                   // one per element type
+        DSP_CUDA_TRY(allow_ring_smem(unmask_scan_kernel<DT>, smem_done));
+        unmask_scan_kernel<DT><<<(unsigned)nblocks, kThreads, kRingBytes, st>>>(a);
+        DSP_CUDA_TRY(cudaGetLastError());
+    }
+    unmask_rows_kernel<DT><<<(unsigned)((nrows + kRowWarps - 1) / kRowWarps), kThreads, 0, st>>>(a);
+    DSP_CUDA_TRY(cudaGetLastError());
+    return DSP_OK;
+}
+
+template <typename DT>
+static size_t unmask_ws_bytes(int B, int L, int V) {
+    const SlicePlan plan = plan_slices<DT>((long long)B * L, V, kTargetCtas);
+    const int ntiles_row = (V + tile_elems<DT>() - 1) / tile_elems<DT>();
+    return unmask_ws_layout(B, L, plan.nslices, ntiles_row, sizeof(DT)).total;
+}
+
+}  // namespace dsp
+
+using namespace dsp;
+
+static int32_t check_unmask_shape(int32_t B, int32_t L, int32_t V, int32_t dtype) {
+    if (B < 0 || L < 1 || V < 1) return DSP_ERR_INVALID_ARG;
+    if (dtype != DSP_F32 && dtype != DSP_BF16) return DSP_ERR_UNSUPPORTED;
+    if (L > DSP_MAX_L || V > (1 << 30)) return DSP_ERR_UNSUPPORTED;
+    return DSP_OK;
+}
+
+extern "C" int32_t dsp_unmask_workspace_bytes(int32_t B, int32_t L, int32_t V, int32_t dtype, size_t *bytes) {
+    if (!bytes) return DSP_ERR_INVALID_ARG;
+    const int32_t rc = check_unmask_shape(B, L, V, dtype);
+    if (rc != DSP_OK) return rc;
+    const int Bq = B > 0 ? B : 1;
+    *bytes = dtype == DSP_BF16 ? unmask_ws_bytes<__nv_bfloat16>(Bq, L, V) : unmask_ws_bytes<float>(Bq, L, V);
+    return DSP_OK;
+}
+
+extern "C" int32_t dsp_unmask_step(const void *logits, int32_t dtype, int32_t B, int32_t L, int32_t V,
+                                   int64_t stride_b, int64_t stride_l, int32_t n_update,
+                                   int32_t *tokens, uint8_t *masked, int32_t *argmax, float *confidence,
+                                   int32_t *n_left, uint32_t *row_status,
+                                   void *workspace, size_t workspace_bytes, dsp_stream_t stream) {
+    const int32_t rc = check_unmask_shape(B, L, V, dtype);
+    if (rc != DSP_OK) return rc;
+    if (n_update < 1) return DSP_ERR_INVALID_ARG;
+    if (B == 0) return DSP_OK;
+    if (!logits || !tokens || !masked || !argmax || !confidence || !n_left || !row_status || !workspace)
+        return DSP_ERR_INVALID_ARG;
+    if (stride_l < V || stride_b < 0 || (B > 1 && stride_b < (int64_t)(L - 1) * stride_l + V))
+        return DSP_ERR_INVALID_ARG;
+    if ((reinterpret_cast<uintptr_t>(workspace) & 255) != 0) return DSP_ERR_INVALID_ARG;
+    const size_t es = dtype == DSP_BF16 ? 2 : 4;
+    if ((reinterpret_cast<uintptr_t>(logits) & (es - 1)) != 0) return DSP_ERR_INVALID_ARG;
+    UnmaskArgs a;
+    a.logits = logits;
+    a.B = B; a.L = L; a.V = V;
+    a.stride_b = stride_b; a.stride_l = stride_l;
+    a.n_update = n_update;
+    a.tokens = tokens; a.masked = masked; a.argmax = argmax; a.confidence = confidence;
+    a.n_left = n_left; a.row_status = row_status;
+    cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+    return dtype == DSP_BF16 ? launch_unmask<__nv_bfloat16>(a, workspace, workspace_bytes, st)
+                             : launch_unmask<float>(a, workspace, workspace_bytes, st);
+}

@@ -201,7 +201,7 @@ def _hand_lattice(B, L, KC, V, seed, *, flat=False, counts=None):
 
 
 @pytest.mark.parametrize("B,L,K,W,eos,lam,flat,case", [
-    (3, 128, 32, 32, True, 0.5, False, "max"),     # largest L, K, W with the EOS slot: 1056 expansions, several windows
+    (3, 128, 32, 32, True, 0.5, False, "max"),     # largest K and W with the EOS slot: 1056 expansions, several windows
     (4, 40, 16, 16, True, 0.0, True, "flat"),      # equal logits and a constant proxy: every expansion ties
     (4, 24, 8, 8, False, 1.0, False, "holes"),     # positions without candidates end the lattice
     (6, 32, 16, 16, True, 0.5, False, "eos"),      # the best beam meets EOS and stops
@@ -308,6 +308,78 @@ def test_step_graphs_per_draft_length_share_buffers():
                                   lam=0.5, table_log2=10, mode=inp["mode"], u=inp["u"])
     g = gpu_step(inp, fused=True, **p)                     # the library still works after the refused capture
     check_step(g, inp, **p)
+
+
+# ---- the drafter's refinement step (Eq. 5) ----
+def _check_unmask(x, tokens, masked, n, ws=None):
+    """One step on both sides from the same state; returns the new state (the GPU's)."""
+    t_gpu, m_gpu = tokens.to(DEV), masked.to(DEV)
+    g = dsp.dsp_unmask_step(x, t_gpu, m_gpu, n, workspace=ws)
+    torch.cuda.synchronize()
+    o = oracle.unmask_step(x.cpu(), tokens, masked, n)
+    good = (o.row_status & oracle.NONFINITE_INPUT) == 0
+    assert torch.equal((g.row_status.cpu() & dsp.ROW_NONFINITE_INPUT) != 0, ~good)
+    was = masked.bool()
+    assert torch.equal(g.argmax.cpu()[good], o.argmax[good])
+    conf = g.confidence.cpu()
+    assert torch.equal(torch.isinf(conf), torch.isinf(o.confidence))
+    fin = torch.isfinite(o.confidence) & good.view(-1, 1)
+    assert (conf[fin] - o.confidence[fin]).abs().max().item() <= 1e-3 if fin.any() else True
+    assert (g.argmax.cpu()[~was] == -1).all()
+    assert torch.equal(g.n_left.cpu()[good], o.n_left[good])
+    for b in torch.nonzero(good).flatten().tolist():
+        if torch.equal(m_gpu[b].cpu(), o.masked[b]):
+            assert torch.equal(t_gpu[b].cpu(), o.tokens[b])
+            continue
+        # a different choice is only right where the two confidences are a rounding apart
+        diff = torch.nonzero(m_gpu[b].cpu() != o.masked[b]).flatten().tolist()
+        cs = o.confidence[b, diff]
+        assert len(diff) == 2 and (cs.max() - cs.min()).item() <= 2e-5, (b, diff, cs)
+    return t_gpu.cpu(), m_gpu.cpu()
+
+
+@pytest.mark.parametrize("B,L,V,dtype,S", [
+    (3, 6, 152064, torch.bfloat16, 3),       # the drafter's vocabulary: several tiles, ragged tail, slices
+    (2, 5, 12288, torch.float32, 2),         # fp32 rows of exactly three tiles
+    (4, 7, 50021, torch.bfloat16, 4),        # odd V: rows are not 16-byte aligned -> element-wise path
+    (2, 40, 37, torch.float32, 1),           # S = 1: everything at once
+    (1, 1, 1, torch.float32, 1),             # one position, one token
+])
+def test_unmask_step_matches_oracle_over_a_whole_refinement(B, L, V, dtype, S):
+    g = torch.Generator().manual_seed(B * 1000 + L)
+    x = (3.0 * torch.randn((B, L, V), generator=g)).to(dtype).to(DEV)
+    tokens = torch.full((B, L), -7, dtype=torch.int32)
+    masked = torch.ones((B, L), dtype=torch.uint8)
+    if B > 1:
+        masked[1, ::2] = 0                                # a batch row that starts half revealed
+    n = -(-L // S)
+    ws = dsp.alloc_workspace(dsp.dsp_unmask_workspace_bytes(B, L, V, dsp.DSP_BF16 if dtype == torch.bfloat16 else dsp.DSP_F32), DEV)
+    for s in range(S):
+        tokens, masked = _check_unmask(x, tokens, masked, n, ws)
+    assert masked.sum() == 0
+    am = x.float().argmax(dim=-1).cpu().int()
+    keep = tokens != -7
+    assert torch.equal(tokens[keep], am[keep])
+
+
+def test_unmask_step_ties_masked_logits_and_flags():
+    B, L, V = 4, 5, 16384
+    g = torch.Generator().manual_seed(8)
+    x = (2.0 * torch.randn((B, L, V), generator=g)).to(torch.bfloat16)
+    x[0] = 0.5                                            # every position ties: lower positions first, argmax 0
+    x[1, :, 100:] = float("-inf")                         # masked vocabulary
+    x[2, 3, 77] = float("nan")                            # flagged only while position 3 is masked
+    x[3, 1, :] = float("-inf")                            # no finite logit
+    x = x.to(DEV)
+    tokens = torch.zeros((B, L), dtype=torch.int32)
+    masked = torch.ones((B, L), dtype=torch.uint8)
+    masked[2, 3] = 0
+    t1, m1 = _check_unmask(x, tokens, masked, 2)
+    assert m1[0].tolist() == [0, 0, 1, 1, 1] and t1[0].tolist() == [0, 0, 0, 0, 0]
+    masked[2, 3] = 1
+    _check_unmask(x, tokens, masked, 2)
+    with pytest.raises(dsp.DspError):
+        dsp.dsp_unmask_step(x, tokens.to(DEV), masked.to(DEV), 0)
 
 
 def test_profile_events_bracket_the_scan_kernels():
