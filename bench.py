@@ -256,6 +256,42 @@ def time_workload(w, device, steps, warmup, dist=None, stages=True, seed_base=0)
     return out, st, sets
 
 
+def time_unmask(w, device, reps=40):
+    """The drafter's refinement step (dsp_unmask_step) on logits of the headline workload's shape:
+    S = 1 (every position masked, one call) and S = 4 (four calls, a quarter of the block each;
+    rows revealed earlier are not read)."""
+    from paper_2510_02358_b200 import binding as dsp
+    sets = input_sets(w, device, 7)
+    dt = dsp.DSP_BF16 if w.dtype == torch.bfloat16 else dsp.DSP_F32
+    ws = dsp.alloc_workspace(dsp.dsp_unmask_workspace_bytes(w.B, w.L, w.V, dt), device)
+    out = None
+    res = {}
+    row_bytes = w.V * (2 if w.dtype == torch.bfloat16 else 4)
+    for S in (1, 4):
+        n = -(-w.L // S)
+        tokens = torch.zeros((w.B, w.L), dtype=torch.int32, device=device)
+        masked = torch.empty((w.B, w.L), dtype=torch.uint8, device=device)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        total, rows_read = 0.0, 0
+        for r in range(reps + 3):
+            x = sets[r % len(sets)]["draft"]
+            masked.fill_(1)
+            e0.record()
+            for s in range(S):
+                out = dsp.dsp_unmask_step(x, tokens, masked, n, out=out, workspace=ws)
+            e1.record()
+            torch.cuda.synchronize()
+            if r >= 3:
+                total += e0.elapsed_time(e1)
+        rows_read = sum(max(w.L - s * n, 0) for s in range(S)) * w.B
+        ms = total / reps
+        res["S%d" % S] = {"ms": ms, "calls": S, "rows_read": rows_read,
+                          "logits_gbs": rows_read * row_bytes / (ms * 1e-3) / 1e9}
+        assert int(masked.sum().item()) == 0
+    res["workload"] = "logits of %s" % w.name
+    return res
+
+
 def time_e2e(w, st, sets, device, steps):
     """Same step through the public calls with HOST buffers: pinned logits are copied to the
     device inside the timed region and the step's results are read back every step."""
@@ -477,6 +513,7 @@ def main():
                 del s2, i2
                 torch.cuda.empty_cache()
         line["workloads"] = extras
+        line["unmask_step"] = time_unmask(w, device)
     print(json.dumps(line))
     if dist is not None:
         dist.destroy_process_group()
