@@ -312,6 +312,7 @@ __global__ void __launch_bounds__(kThreads, 4) residual_kernel(const VerifyArgs 
     constexpr int N = Elem<DT>::N;
     constexpr int CE = 32 * N;                  // elements per chunk: one warp-wide vector load
     __shared__ double s_scan[kThreads];
+    __shared__ double s_wtot[kWarps];
     __shared__ double s_total;
     __shared__ int s_found;
     __shared__ int s_flag;
@@ -330,16 +331,30 @@ __global__ void __launch_bounds__(kThreads, 4) residual_kernel(const VerifyArgs 
     const int V = a.V;
 
     const int c0 = rs * a.chunks_per_slice, c1 = min(a.nchunks, c0 + a.chunks_per_slice);
-    for (int ch = c0 + warp; ch < c1; ch += kWarps) {
-        const int e0 = ch * CE + lane * N;
-        const uint4 vt = load_vec<DT>(tp, e0, V, aligned);
-        const uint4 vd = has_q ? load_vec<DT>(dp, e0, V, aligned) : vt;
-        float s = 0.f;
+    constexpr int kChunkBatch = 4;              // chunks whose loads a warp has in flight together
+    for (int ch0 = c0 + warp; ch0 < c1; ch0 += kWarps * kChunkBatch) {
+        uint4 vt[kChunkBatch], vd[kChunkBatch];
 #pragma unroll
-        for (int e = 0; e < N; ++e)
-            s = __fadd_rn(s, residual(Elem<DT>::get(vt, e), Elem<DT>::get(vd, e), pt, pd, has_q));
-        const double cs = warp_sum((double)s);
-        if (lane == 0) sums[ch] = cs;
+        for (int u = 0; u < kChunkBatch; ++u) {
+            const int ch = ch0 + u * kWarps;
+            if (ch < c1) {
+                const int e0 = ch * CE + lane * N;
+                vt[u] = load_vec<DT>(tp, e0, V, aligned);
+                vd[u] = has_q ? load_vec<DT>(dp, e0, V, aligned) : vt[u];
+            }
+        }
+#pragma unroll
+        for (int u = 0; u < kChunkBatch; ++u) {
+            const int ch = ch0 + u * kWarps;
+            if (ch < c1) {
+                float s = 0.f;
+#pragma unroll
+                for (int e = 0; e < N; ++e)
+                    s = __fadd_rn(s, residual(Elem<DT>::get(vt[u], e), Elem<DT>::get(vd[u], e), pt, pd, has_q));
+                const double cs = warp_sum((double)s);
+                if (lane == 0) sums[ch] = cs;
+            }
+        }
     }
     __threadfence();
     __syncthreads();
@@ -353,15 +368,21 @@ __global__ void __launch_bounds__(kThreads, 4) residual_kernel(const VerifyArgs 
     const int k0 = min(a.nchunks, tid * per), k1 = min(a.nchunks, k0 + per);
     double mine = 0.0;
     for (int k = k0; k < k1; ++k) mine += __ldcg(&sums[k]);
-    s_scan[tid] = mine;
     if (tid == 0) s_found = 0x7FFFFFFF;
-    __syncthreads();
-    // exclusive prefix of the 256 thread sums (serial in thread 0: 256 adds, fixed order)
-    if (tid == 0) {
-        double run = 0.0;
-        for (int t = 0; t < kThreads; ++t) { const double x = s_scan[t]; s_scan[t] = run; run += x; }
-        s_total = run;
+    // exclusive prefix of the 256 thread sums, in a fixed order: inside each warp, then over the warps
+    double tincl = mine;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const double up = __shfl_up_sync(0xFFFFFFFFu, tincl, o);
+        if (lane >= o) tincl += up;
     }
+    const double upto = __shfl_up_sync(0xFFFFFFFFu, tincl, 1);
+    if (lane == 31) s_wtot[warp] = tincl;
+    __syncthreads();
+    double wbase = 0.0;
+    for (int w = 0; w < warp; ++w) wbase += s_wtot[w];
+    s_scan[tid] = lane == 0 ? wbase : wbase + upto;
+    if (tid == kThreads - 1) s_total = wbase + tincl;
     __syncthreads();
     const double R = s_total;
     if (!(R > 0.0)) {
