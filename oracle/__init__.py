@@ -53,6 +53,7 @@ def lib():
             _lib = C.CDLL(build())
             _lib.orc_residual_probe.restype = C.c_int64
             _lib.orc_proxy_score.restype = C.c_float
+            _lib.orc_trigram_score.restype = C.c_float
     return _lib
 
 
@@ -162,6 +163,12 @@ def unmask_step(logits: torch.Tensor, tokens, masked, n_update: int):
     if rc != 0:
         raise ValueError("orc_unmask_step: bad arguments")
     return SimpleNamespace(**{k: torch.from_numpy(v) for k, v in vars(o).items()})
+
+
+def trigram_score(table, prev2: int, prev: int, cur: int, *, table_log2=0, hash_seed=0) -> float:
+    table = _np(table, np.float32)
+    return float(lib().orc_trigram_score(_p(table), table_log2, C.c_uint32(hash_seed & 0xFFFFFFFF),
+                                         prev2, prev, cur))
 
 
 def verify(target: torch.Tensor, draft, path, path_len, mode=None, u=None, eos_id: int = -1):

@@ -231,6 +231,63 @@ float orc_proxy_score(int kind, const float *table, int table_log2, uint32_t see
     return proxy_score(kind, table, table_log2, seed, V, prev, cur);
 }
 
+/*
+ * Hashed trigram proxy (the paper's causal proxy is a 3-gram model, Sec. 4):
+ * l^ng(cur | prev2, prev) = table[mix3(prev2, prev, cur) >> (32 - table_log2)],
+ *   g = prev2 * 0xC2B2AE35;  g ^= g >> 16;
+ *   h = (prev ^ g) * 0x9E3779B1;  h ^= cur + seed;  h *= 0x9E3779B1;
+ *   h ^= h >> 15;  h *= 0x9E3779B1;  h ^= h >> 13          (all in uint32).
+ */
+static float trigram_score(const float *table, int table_log2, uint32_t seed,
+                           int32_t prev2, int32_t prev, int32_t cur)
+{
+    uint32_t g = (uint32_t)prev2 * 0xC2B2AE35u;
+    g ^= g >> 16;
+    uint32_t h = ((uint32_t)prev ^ g) * 0x9E3779B1u;
+    h ^= (uint32_t)cur + seed;
+    h *= 0x9E3779B1u;
+    h ^= h >> 15;
+    h *= 0x9E3779B1u;
+    h ^= h >> 13;
+    uint32_t idx = table_log2 >= 32 ? h : (table_log2 <= 0 ? 0u : h >> (32 - table_log2));
+    return table[idx];
+}
+
+float orc_trigram_score(const float *table, int table_log2, uint32_t seed,
+                        int32_t prev2, int32_t prev, int32_t cur)
+{
+    return trigram_score(table, table_log2, seed, prev2, prev, cur);
+}
+
+/*
+ * l^ng of candidate slot k at position i of batch row b, for a path whose
+ * earlier tokens / slots are ids[0..i) / slots[0..i)  (Eq. 8's causal term):
+ *   kind 0, 1: bigram on (previous token, token): hashed table or dense [V,V];
+ *              position 0 conditions on prev_token[b];
+ *   kind 2   : a tensor [B,L,KC,KC] of scores the caller computed (a small
+ *              causal model): entry [b][i][p][k], p = the previous position's
+ *              slot (row p = 0 at position 0);
+ *   kind 3   : hashed trigram on (token before, previous token, token);
+ *              prev_token is [B,2] (oldest first) and supplies what the path
+ *              does not have yet.
+ */
+static float proxy_at(int kind, const float *table, int table_log2, uint32_t seed, int64_t V,
+                      const int32_t *prev_token, int b, int L, int KC, int i, int k, int32_t tok,
+                      const int32_t *ids, const int32_t *slots)
+{
+    if (kind == 2) {
+        const int p = i == 0 ? 0 : slots[i - 1];
+        return table[(((int64_t)b * L + i) * KC + p) * KC + k];
+    }
+    if (kind == 3) {
+        const int32_t prev = i == 0 ? prev_token[2 * b + 1] : ids[i - 1];
+        const int32_t prev2 = i == 0 ? prev_token[2 * b] : (i == 1 ? prev_token[2 * b + 1] : ids[i - 2]);
+        return trigram_score(table, table_log2, seed, prev2, prev, tok);
+    }
+    const int32_t prev = i == 0 ? prev_token[b] : ids[i - 1];
+    return proxy_score(kind, table, table_log2, seed, V, prev, tok);
+}
+
 typedef struct {
     float cum;
     int32_t tok;
@@ -257,6 +314,7 @@ static int exp_before(const expansion *a, const expansion *b)
  * evaluated in fp32 in this exact order:
  *   g = fp32(x - x_top1);  step = fp32( fp32(lambda*g) + fp32((1-lambda)*n) );
  *   cum = fp32(parent_cum + step),   1-lambda = fp32(1 - lambda).
+ * l^ng comes from one of four proxies (see proxy_at above).
  * Survivors: the best min(W, #expansions) under (cum desc, token id asc,
  * parent rank asc).  The search stops after the depth at which the rank-0
  * survivor's new token is EOS (early stop at the first EOS placed).
@@ -298,11 +356,11 @@ int orc_cps_search(const int32_t *cand_id, const float *cand_logit, const double
             const float top1 = cand_logit[r * KC];
             int n = 0;
             for (int w = 0; w < live; ++w) {
-                int32_t prev = i == 0 ? prev_token[b] : ids[w * L + i - 1];
                 for (int k = 0; k < cnt; ++k) {
                     int32_t tok = cand_id[r * KC + k];
                     volatile float g = cand_logit[r * KC + k] - top1;
-                    float ng = proxy_score(proxy_kind, table, table_log2, hash_seed, V, prev, tok);
+                    float ng = proxy_at(proxy_kind, table, table_log2, hash_seed, V, prev_token, b, L, KC,
+                                        i, k, tok, ids + w * L, slots + w * L);
                     volatile float a = lambda * g;
                     volatile float c = oml * ng;
                     volatile float step = a + c;
@@ -351,10 +409,10 @@ int orc_cps_search(const int32_t *cand_id, const float *cand_logit, const double
                 s = 0.0;
                 for (int i = 0; i < m; ++i) {
                     const int64_t r = (int64_t)b * L + i;
-                    int32_t prev = i == 0 ? prev_token[b] : ids[w * L + i - 1];
                     double ldlm = (double)cand_logit[r * KC + slots[w * L + i]] - lse64[r];
-                    double lng = (double)proxy_score(proxy_kind, table, table_log2, hash_seed, V,
-                                                     prev, ids[w * L + i]);
+                    double lng = (double)proxy_at(proxy_kind, table, table_log2, hash_seed, V, prev_token,
+                                                  b, L, KC, i, slots[w * L + i], ids[w * L + i],
+                                                  ids + w * L, slots + w * L);
                     s += (double)lambda * ldlm + (double)oml * lng;
                 }
             }

@@ -220,3 +220,87 @@ def test_hashed_proxy_index_follows_the_stated_mix():
         assert int(s) == idx(prev, cur, 7, log2)
         hits.add(int(s))
     assert len(hits) > 250                                 # spreads over the table
+
+
+# ---- the richer causal proxies: a tensor of scores per (position, previous slot, slot), a hashed trigram ----
+def _mix3(prev2, prev, cur, seed, log2):
+    """The header text of the hashed trigram table, restated with Python integers."""
+    M = 0xFFFFFFFF
+    g = (prev2 * 0xC2B2AE35) & M
+    g ^= g >> 16
+    h = ((prev ^ g) * 0x9E3779B1) & M
+    h ^= (cur + seed) & M
+    h = (h * 0x9E3779B1) & M
+    h ^= h >> 15
+    h = (h * 0x9E3779B1) & M
+    h ^= h >> 13
+    return h >> (32 - log2)
+
+
+def test_trigram_index_follows_the_stated_mix_and_uses_all_three_tokens():
+    log2 = 14
+    table = torch.arange(1 << log2, dtype=torch.float32)
+    g = torch.Generator().manual_seed(1)
+    for p2, p1, c in torch.randint(0, 152064, (300, 3), generator=g).tolist():
+        assert int(oracle.trigram_score(table, p2, p1, c, table_log2=log2, hash_seed=3)) == _mix3(p2, p1, c, 3, log2)
+    base = oracle.trigram_score(table, 5, 6, 7, table_log2=log2, hash_seed=3)
+    others = [oracle.trigram_score(table, 9, 6, 7, table_log2=log2, hash_seed=3),
+              oracle.trigram_score(table, 5, 9, 7, table_log2=log2, hash_seed=3),
+              oracle.trigram_score(table, 5, 6, 9, table_log2=log2, hash_seed=3),
+              oracle.trigram_score(table, 6, 5, 7, table_log2=log2, hash_seed=3)]
+    assert all(o != base for o in others)
+
+
+@pytest.mark.parametrize("kind", [2, 3])
+@pytest.mark.parametrize("L,K,seed", [(3, 4, 0), (4, 3, 1), (5, 2, 2), (2, 5, 3)])
+def test_wide_beam_equals_brute_force_with_tensor_and_trigram_proxies(kind, L, K, seed):
+    V, lam, log2, hseed = 12, 0.4, 9, 11
+    _, lat, _, _ = _lattice(L, V, K, seed)
+    g = torch.Generator().manual_seed(100 + seed)
+    KC = lat.cand_id.shape[2]
+    if kind == 2:
+        table = -6.0 * torch.rand((1, L, KC, KC), generator=g)
+        prev = torch.tensor([4], dtype=torch.int32)
+        ng = lambda i, ids, slots: float(table[0, i, 0 if i == 0 else slots[i - 1], slots[i]])
+    else:
+        table = -6.0 * torch.rand((1 << log2,), generator=g)
+        prev = torch.tensor([[4, 9]], dtype=torch.int32)
+        hist = lambda i, ids: ([4, 9] + list(ids))[i:i + 2]              # the two tokens before position i
+        ng = lambda i, ids, slots: float(table[_mix3(hist(i, ids)[0], hist(i, ids)[1], ids[i], hseed, log2)])
+    W = K ** (L - 1)
+    out = oracle.cps_search(lat.cand_id, lat.cand_logit, lat.lse64, lat.cand_count, prev, table, W=W, lam=lam,
+                            proxy_kind=kind, table_log2=log2, hash_seed=hseed, V=V)
+    counts = lat.cand_count[0].tolist()
+    scored = []
+    for slots in itertools.product(*[range(c) for c in counts]):
+        ids = [int(lat.cand_id[0, i, k]) for i, k in enumerate(slots)]
+        s = sum(lam * (float(lat.cand_logit[0, i, k]) - float(lat.lse64[0, i])) + (1.0 - lam) * ng(i, ids, slots)
+                for i, k in enumerate(slots))
+        scored.append((s, ids))
+    scored.sort(key=lambda t: -t[0])
+    assert abs(out.path_score.item() - scored[0][0]) < 1e-4
+    if scored[0][0] - scored[1][0] > 1e-4:
+        assert out.path[0].tolist() == scored[0][1]
+    nb = min(W, len(scored))
+    assert np.allclose(out.beam_score[0, :nb].double().numpy(), np.array([s for s, _ in scored[:nb]]), atol=1e-4)
+
+
+def test_tensor_proxy_built_from_the_dense_table_gives_the_dense_search():
+    L, V, K, W, lam = 6, 30, 4, 3, 0.5
+    _, lat, table, prev = _lattice(L, V, K, 9, B=2)
+    dense = oracle.cps_search(lat.cand_id, lat.cand_logit, lat.lse64, lat.cand_count, prev, table, W=W, lam=lam,
+                              proxy_kind=1, V=V)
+    B, _, KC = lat.cand_id.shape
+    tens = torch.zeros((B, L, KC, KC))
+    for b in range(B):
+        for i in range(L):
+            for p in range(KC):
+                pt = int(prev[b]) if i == 0 else int(lat.cand_id[b, i - 1, p])
+                for k in range(KC):
+                    ct = int(lat.cand_id[b, i, k])
+                    if pt >= 0 and ct >= 0:
+                        tens[b, i, p, k] = table[pt, ct]
+    out = oracle.cps_search(lat.cand_id, lat.cand_logit, lat.lse64, lat.cand_count, prev, tens, W=W, lam=lam,
+                            proxy_kind=2, V=V)
+    for k in ("path", "path_slot", "path_len", "beam_ids", "beam_cum", "path_score", "beam_score"):
+        assert torch.equal(getattr(out, k), getattr(dense, k)), k
