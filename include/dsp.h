@@ -186,17 +186,29 @@ int32_t dsp_lattice_build_static(const void *draft_logits, int32_t dtype,
  * ascending).  The search stops after the first depth at which the rank-0
  * survivor's new token is eos_id (row flag DSP_ROW_EOS_STOPPED).
  *
- * Causal proxy l^ng (the paper's n-gram model, here a caller-supplied bigram
- * table of fp32 scores):
+ * Causal proxy l^ng (the paper's n-gram model or small causal model, here
+ * caller-supplied fp32 scores):
  *   proxy_kind 0: hashed table of 2^table_log2 entries, 1 <= table_log2 <= 31.
  *     With all arithmetic on uint32 modulo 2^32:
  *       h = prev * 0x9E3779B1;  h ^= cur + hash_seed;  h *= 0x9E3779B1;
  *       h ^= h >> 15;  h *= 0x9E3779B1;  h ^= h >> 13;
  *       l^ng = proxy_table[h >> (32 - table_log2)]
  *   proxy_kind 1: dense table [V,V]: l^ng = proxy_table[prev * V + cur].
+ *   proxy_kind 2: a tensor [B,L,KC,KC] of scores the caller computed for the
+ *     lattice (a small causal model): l^ng of candidate slot k at position i
+ *     after candidate slot p at position i-1 is proxy_table[b][i][p][k]; at
+ *     position 0 row p = 0 is read.  prev_token, V, table_log2, hash_seed unused.
+ *   proxy_kind 3: hashed trigram table of 2^table_log2 entries (the paper's
+ *     proxy is a 3-gram model): l^ng(cur | prev2, prev) with
+ *       g = prev2 * 0xC2B2AE35;  g ^= g >> 16;
+ *       h = (prev ^ g) * 0x9E3779B1;  h ^= cur + hash_seed;  h *= 0x9E3779B1;
+ *       h ^= h >> 15;  h *= 0x9E3779B1;  h ^= h >> 13;
+ *       l^ng = proxy_table[h >> (32 - table_log2)]
+ *     and prev_token int32 [B,2]: the prefix's last two tokens, oldest first.
  *
  * Inputs : cand_id, cand_logit, cand_count, lse64 as written by
- *          dsp_lattice_build (KC = their last dimension); prev_token int32 [B].
+ *          dsp_lattice_build (KC = their last dimension); prev_token int32 [B]
+ *          ([B,2] for proxy_kind 3).
  * Outputs: path       int32 [B,L]   rank-0 path, -1 beyond path_len
  *          path_slot  int32 [B,L]   candidate slot of each path token, -1 beyond
  *          path_len   int32 [B]     m (0 if the first position has no candidate: the one

@@ -18,7 +18,7 @@
 namespace dsp {
 
 constexpr int kMaxKC = DSP_MAX_K + 1;
-constexpr int kStepBudgetBytes = 48 * 1024;        // shared memory for one window of step scores
+constexpr int kStepBudgetBytes = 48 * 1024;        // shared memory for one window of depths
 
 struct CpsArgs {
     const int32_t *cand_id;
@@ -41,17 +41,18 @@ struct CpsArgs {
     float *beam_score, *beam_cum;
     uint32_t *row_status;
     int D;                       // depths per window
+    int SW;                      // step-table entries per depth: KC * KC, or KC for the trigram proxy
 };
 
-// Depths per window and dynamic shared memory of a launch.
-inline int cps_window_depths(int L, int KC) {
-    int d = kStepBudgetBytes / (KC * KC * 4);
+// Depths per window and dynamic shared memory of a launch (SW = step-table entries per depth).
+inline int cps_window_depths(int L, int KC, int SW) {
+    int d = kStepBudgetBytes / (SW * 4 + KC * 13 + 8);          // everything a depth keeps in shared memory
     if (d < 1) d = 1;
     return d < L ? d : L;
 }
-inline size_t cps_smem_bytes(int L, int W, int KC, int D) {
+inline size_t cps_smem_bytes(int L, int W, int KC, int D, int SW) {
     size_t o = align_up((size_t)3 * L * W, 16);                 // back-pointers and walked slots
-    o += (size_t)D * KC * KC * 4;                               // step scores
+    o += (size_t)D * SW * 4;                                    // step scores
     o += (size_t)(D + 1) * KC * 4;                              // candidate ids (and the depth before the window)
     o += (size_t)D * KC * 4;                                    // candidate logits
     o += (size_t)(D + 1) * 4 + (size_t)D * 4;                   // candidate counts, their division constants
@@ -60,9 +61,22 @@ inline size_t cps_smem_bytes(int L, int W, int KC, int D) {
     return o;
 }
 
+// Bigram proxies: the dense [V,V] table or the hashed table (the mix is part of the ABI).
 __device__ __forceinline__ float proxy_score(const CpsArgs &a, int prev, int cur) {
     if (a.proxy_kind == 1) return __ldg(&a.table[(long long)prev * a.V + cur]);
     uint32_t h = (uint32_t)prev * 0x9E3779B1u;
+    h ^= (uint32_t)cur + a.hash_seed;
+    h *= 0x9E3779B1u;
+    h ^= h >> 15;
+    h *= 0x9E3779B1u;
+    h ^= h >> 13;
+    return __ldg(&a.table[h >> (32 - a.table_log2)]);
+}
+// Hashed trigram proxy (the mix is part of the ABI).
+__device__ __forceinline__ float trigram_score(const CpsArgs &a, int prev2, int prev, int cur) {
+    uint32_t g = (uint32_t)prev2 * 0xC2B2AE35u;
+    g ^= g >> 16;
+    uint32_t h = ((uint32_t)prev ^ g) * 0x9E3779B1u;
     h ^= (uint32_t)cur + a.hash_seed;
     h *= 0x9E3779B1u;
     h ^= h >> 15;
@@ -79,6 +93,11 @@ constexpr int kGatherBatch = 8;                             // proxy gathers a t
 __device__ __forceinline__ unsigned long long div_magic(int d) { return (1ull << 32) / (unsigned)d + 1ull; }
 __device__ __forceinline__ int div_by(int x, unsigned long long m) { return (int)(((unsigned long long)(unsigned)x * m) >> 32); }
 
+// TRI: the hashed trigram proxy.  Its score depends on the beam's last two tokens, so it cannot be
+// tabulated per window: every expansion gathers its own score in the depth loop (one more memory
+// round trip per depth), the beams' best expansions are found with shared-memory atomics, and one
+// more block barrier separates them from the pruning.
+template <bool TRI>
 __global__ void __launch_bounds__(kThreads) cps_kernel(const CpsArgs a) {
     extern __shared__ __align__(16) unsigned char dyn[];
     // keys that can still be among the best W: two buffers in turn, the one not in use is zeroed
@@ -89,6 +108,10 @@ __global__ void __launch_bounds__(kThreads) cps_kernel(const CpsArgs a) {
     __shared__ uint32_t s_floor[2];                    // smallest ord_bits among the beams' own best expansions
     __shared__ int s_nsurv[2];                         // survivors of this depth / of the next (in turn)
     __shared__ int s_top_tok;                          // token of the rank-0 survivor
+    // trigram proxy only: every expansion's key, each beam's last two tokens, each beam's best expansion
+    __shared__ unsigned long long tkeys[TRI ? kMaxExpansions : 1];
+    __shared__ int btok[2][TRI ? DSP_MAX_W : 1], btok2[2][TRI ? DSP_MAX_W : 1];
+    __shared__ __align__(16) uint32_t tbest[2][TRI ? DSP_MAX_W : 4];
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int b = blockIdx.x;
@@ -97,7 +120,7 @@ __global__ void __launch_bounds__(kThreads) cps_kernel(const CpsArgs a) {
     unsigned char *bp_slot = dyn + (size_t)L * W;
     unsigned char *walk = dyn + (size_t)2 * L * W;     // slot of beam w at depth i, after the walk
     float *step = reinterpret_cast<float *>(dyn + align_up((size_t)3 * L * W, 16));
-    int *cid = reinterpret_cast<int *>(step + (size_t)D * KC * KC);   // row 0: the depth before the window
+    int *cid = reinterpret_cast<int *>(step + (size_t)D * a.SW);   // row 0: the depth before the window
     float *clg = reinterpret_cast<float *>(cid + (size_t)(D + 1) * KC);
     int *ccnt = reinterpret_cast<int *>(clg + (size_t)D * KC);        // entry 0: the depth before the window
     unsigned *cinv = reinterpret_cast<unsigned *>(ccnt + D + 1);
@@ -116,6 +139,14 @@ __global__ void __launch_bounds__(kThreads) cps_kernel(const CpsArgs a) {
         (&bslot[0][0])[tid] = 0;
     }
     if (tid < 2) s_nsurv[tid] = 0;
+    if constexpr (TRI) {
+        if (tid < 2 * DSP_MAX_W) {
+            (&btok[0][0])[tid] = 0;
+            (&btok2[0][0])[tid] = 0;
+            (&tbest[0][0])[tid] = tid == 0 ? 0u : 0xFFFFFFFFu;      // one live beam at the start
+        }
+        if (tid == 0) { btok2[0][0] = a.prev_token[2 * b]; btok[0][0] = a.prev_token[2 * b + 1]; }
+    }
     for (int x = tid; x < 2 * (kMaxExpansions + 8); x += kThreads) (&surv[0][0])[x] = 0ull;
 
     for (int i0 = 0; i0 < L && m == L && !stopped; i0 += D) {
@@ -135,27 +166,33 @@ __global__ void __launch_bounds__(kThreads) cps_kernel(const CpsArgs a) {
             cid[KC + x] = a.cand_id[(row0 + i0) * KC + x];
             clg[x] = a.cand_logit[(row0 + i0) * KC + x];
         }
-        for (int x = tid; x < KC; x += kThreads) cid[x] = i0 == 0 ? a.prev_token[b] : a.cand_id[(row0 + i0 - 1) * KC + x];
+        for (int x = tid; x < KC; x += kThreads)
+            cid[x] = i0 == 0 ? a.prev_token[TRI ? 2 * b + 1 : b] : a.cand_id[(row0 + i0 - 1) * KC + x];
         __syncthreads();
-        const int total = nd * KK;
-        for (int x0 = tid; x0 < total; x0 += kThreads * kGatherBatch) {
-            float ng[kGatherBatch];
-            int at[kGatherBatch];                           // d * KC + k of a live entry, else -1
+        if constexpr (!TRI) {
+            const int total = nd * KK;
+            for (int x0 = tid; x0 < total; x0 += kThreads * kGatherBatch) {
+                float ng[kGatherBatch];
+                int at[kGatherBatch];                           // d * KC + k of a live entry, else -1
 #pragma unroll
-            for (int u = 0; u < kGatherBatch; ++u) {        // no branches: the gathers of a batch overlap
-                const int x = min(x0 + u * kThreads, total - 1);
-                const int d = div_by(x, mKK), rem = x - d * KK;
-                const int p = div_by(rem, mKC), k = rem - p * KC;
-                const bool ok = x0 + u * kThreads < total && k < ccnt[1 + d] && p < ccnt[d];
-                at[u] = ok ? d * KC + k : -1;
-                ng[u] = proxy_score(a, ok ? cid[d * KC + p] : 0, ok ? cid[(d + 1) * KC + k] : 0);
-            }
+                for (int u = 0; u < kGatherBatch; ++u) {        // no branches: the gathers of a batch overlap
+                    const int x = min(x0 + u * kThreads, total - 1);
+                    const int d = div_by(x, mKK), rem = x - d * KK;
+                    const int p = div_by(rem, mKC), k = rem - p * KC;
+                    const bool ok = x0 + u * kThreads < total && k < ccnt[1 + d] && p < ccnt[d];
+                    at[u] = ok ? d * KC + k : -1;
+                    if (a.proxy_kind == 2)                      // the caller's tensor [B,L,KC,KC]: same index order as x
+                        ng[u] = __ldg(&a.table[(row0 + i0) * KK + (ok ? x : 0)]);
+                    else
+                        ng[u] = proxy_score(a, ok ? cid[d * KC + p] : 0, ok ? cid[(d + 1) * KC + k] : 0);
+                }
 #pragma unroll
-            for (int u = 0; u < kGatherBatch; ++u) {
-                if (at[u] >= 0) {
-                    const int d = div_by(at[u], mKC);
-                    const float g = __fsub_rn(clg[at[u]], clg[d * KC]);
-                    step[x0 + u * kThreads] = __fadd_rn(__fmul_rn(lam, g), __fmul_rn(oml, ng[u]));
+                for (int u = 0; u < kGatherBatch; ++u) {
+                    if (at[u] >= 0) {
+                        const int d = div_by(at[u], mKC);
+                        const float g = __fsub_rn(clg[at[u]], clg[d * KC]);
+                        step[x0 + u * kThreads] = __fadd_rn(__fmul_rn(lam, g), __fmul_rn(oml, ng[u]));
+                    }
                 }
             }
         }
@@ -169,18 +206,20 @@ __global__ void __launch_bounds__(kThreads) cps_kernel(const CpsArgs a) {
             trank[x] = (unsigned char)r;
         }
         __syncthreads();
-        for (int x = tid; x < nd * KC; x += kThreads) {     // best step score after previous slot p
-            const int d = div_by(x, mKC), p = x - d * KC;
-            float best = -CUDART_INF_F;
-            if (p < ccnt[d])
-                for (int k = 0; k < ccnt[1 + d]; ++k) best = fmaxf(best, step[x * KC + k]);
-            smax[x] = best;
-        }
-        if (tid < live) {                                   // the beams' best expansions at the window's first depth
-            float best = -CUDART_INF_F;
-            const int p = bslot[cur][tid];
-            for (int k = 0; k < ccnt[1]; ++k) best = fmaxf(best, step[p * KC + k]);
-            atomicMin(&s_floor[cur], ord_bits(__fadd_rn(bcum[cur][tid], best)));
+        if constexpr (!TRI) {
+            for (int x = tid; x < nd * KC; x += kThreads) {     // best step score after previous slot p
+                const int d = div_by(x, mKC), p = x - d * KC;
+                float best = -CUDART_INF_F;
+                if (p < ccnt[d])
+                    for (int k = 0; k < ccnt[1 + d]; ++k) best = fmaxf(best, step[x * KC + k]);
+                smax[x] = best;
+            }
+            if (tid < live) {                                   // the beams' best expansions at the window's first depth
+                float best = -CUDART_INF_F;
+                const int p = bslot[cur][tid];
+                for (int k = 0; k < ccnt[1]; ++k) best = fmaxf(best, step[p * KC + k]);
+                atomicMin(&s_floor[cur], ord_bits(__fadd_rn(bcum[cur][tid], best)));
+            }
         }
         __syncthreads();
 
@@ -194,20 +233,53 @@ __global__ void __launch_bounds__(kThreads) cps_kernel(const CpsArgs a) {
             const int nxt = cur ^ 1;
             // Every beam's best expansion is one of the n; with `keep` beams or more, the keep-th
             // best expansion is at least the smallest of those, so anything below it is out.
-            const uint32_t floor_ord = live >= keep ? s_floor[cur] : 0u;
-            if (tid == 0) s_floor[nxt] = 0xFFFFFFFFu;
+            uint32_t floor_ord = 0u;
             const unsigned inv = cinv[d];
+            if constexpr (TRI) {
+                // every expansion gathers its causal score; each beam's best expansion by atomicMax
+                for (int e = tid; e < n; e += kThreads) {
+                    const int w = (int)(((unsigned)e * inv) >> 16), k = e - w * cnt;
+                    const float ng = trigram_score(a, btok2[cur][w], btok[cur][w], cid[(d + 1) * KC + k]);
+                    const float g = __fsub_rn(clg[d * KC + k], clg[d * KC]);       // the drafter's part: x - x_top1
+                    const float cum = __fadd_rn(bcum[cur][w], __fadd_rn(__fmul_rn(lam, g), __fmul_rn(oml, ng)));
+                    const uint32_t ob = ord_bits(cum);
+                    atomicMax(&tbest[cur][w], ob);
+                    tkeys[e] = ((unsigned long long)ob << 32) | ((unsigned long long)(255 - trank[d * KC + k]) << 24) |
+                               ((unsigned long long)(255 - w) << 16) | ((unsigned long long)(255 - k) << 8) | 1ull;
+                }
+                if (tid < DSP_MAX_W) tbest[nxt][tid] = tid < keep ? 0u : 0xFFFFFFFFu;   // for the next depth
+                __syncthreads();
+                if (live >= keep) {
+                    floor_ord = 0xFFFFFFFFu;
+                    const uint4 *tb = reinterpret_cast<const uint4 *>(tbest[cur]);
+#pragma unroll
+                    for (int j = 0; j < DSP_MAX_W / 4; ++j) {
+                        const uint4 v = tb[j];
+                        floor_ord = min(min(floor_ord, min(v.x, v.y)), min(v.z, v.w));
+                    }
+                }
+            } else {
+                // Every beam's best expansion is one of the n; with `keep` beams or more, the keep-th
+                // best expansion is at least the smallest of those, so anything below it is out.
+                floor_ord = live >= keep ? s_floor[cur] : 0u;
+                if (tid == 0) s_floor[nxt] = 0xFFFFFFFFu;
+            }
             for (int e0 = warp * 32; e0 < n; e0 += kThreads) {
                 const int e = e0 + lane;
                 unsigned long long key = 0ull;
                 bool in = false;
                 if (e < n) {
-                    const int w = (int)(((unsigned)e * inv) >> 16), k = e - w * cnt;
-                    const float cum = __fadd_rn(bcum[cur][w], step[(d * KC + bslot[cur][w]) * KC + k]);
-                    const uint32_t ob = ord_bits(cum);
-                    in = ob >= floor_ord;
-                    key = ((unsigned long long)ob << 32) | ((unsigned long long)(255 - trank[d * KC + k]) << 24) |
-                          ((unsigned long long)(255 - w) << 16) | ((unsigned long long)(255 - k) << 8) | 1ull;
+                    if constexpr (TRI) {
+                        key = tkeys[e];
+                        in = (uint32_t)(key >> 32) >= floor_ord;
+                    } else {
+                        const int w = (int)(((unsigned)e * inv) >> 16), k = e - w * cnt;
+                        const float cum = __fadd_rn(bcum[cur][w], step[(d * KC + bslot[cur][w]) * KC + k]);
+                        const uint32_t ob = ord_bits(cum);
+                        in = ob >= floor_ord;
+                        key = ((unsigned long long)ob << 32) | ((unsigned long long)(255 - trank[d * KC + k]) << 24) |
+                              ((unsigned long long)(255 - w) << 16) | ((unsigned long long)(255 - k) << 8) | 1ull;
+                    }
                 }
                 const unsigned ballot = __ballot_sync(0xFFFFFFFFu, in);
                 int base = 0;
@@ -236,7 +308,12 @@ __global__ void __launch_bounds__(kThreads) cps_kernel(const CpsArgs a) {
                     const float cum = ord_value((uint32_t)(q >> 32));    // as added up for the key (-0 reads as +0)
                     bcum[nxt][rank] = cum;
                     bslot[nxt][rank] = k;
-                    if (d + 1 < nd) atomicMin(&s_floor[nxt], ord_bits(__fadd_rn(cum, smax[(d + 1) * KC + k])));
+                    if constexpr (TRI) {
+                        btok2[nxt][rank] = btok[cur][w];
+                        btok[nxt][rank] = cid[(d + 1) * KC + k];
+                    } else {
+                        if (d + 1 < nd) atomicMin(&s_floor[nxt], ord_bits(__fadd_rn(cum, smax[(d + 1) * KC + k])));
+                    }
                     bp_parent[(size_t)i * W + rank] = (unsigned char)w;
                     bp_slot[(size_t)i * W + rank] = (unsigned char)k;
                     if (rank == 0) s_top_tok = cid[(d + 1) * KC + k];
@@ -319,8 +396,8 @@ extern "C" int32_t dsp_cps_search(const int32_t *cand_id, const float *cand_logi
                                   uint32_t *row_status, dsp_stream_t stream) {
     if (B < 0 || L < 1 || KC < 1 || V < 1) return DSP_ERR_INVALID_ARG;
     if (W < 1 || W > DSP_MAX_W || KC > DSP_MAX_K + 1 || L > DSP_MAX_L) return DSP_ERR_UNSUPPORTED;
-    if (proxy_kind != 0 && proxy_kind != 1) return DSP_ERR_UNSUPPORTED;
-    if (proxy_kind == 0 && (table_log2 < 1 || table_log2 > 31)) return DSP_ERR_INVALID_ARG;
+    if (proxy_kind < 0 || proxy_kind > 3) return DSP_ERR_UNSUPPORTED;
+    if ((proxy_kind == 0 || proxy_kind == 3) && (table_log2 < 1 || table_log2 > 31)) return DSP_ERR_INVALID_ARG;
     if (!(lambda >= 0.f && lambda <= 1.f)) return DSP_ERR_INVALID_ARG;
     if (B == 0) return DSP_OK;
     if (!cand_id || !cand_logit || !lse64 || !cand_count || !prev_token || !proxy_table || !path ||
@@ -336,21 +413,28 @@ extern "C" int32_t dsp_cps_search(const int32_t *cand_id, const float *cand_logi
     a.path = path; a.path_slot = path_slot; a.path_len = path_len; a.path_score = path_score;
     a.beam_ids = beam_ids; a.beam_score = beam_score; a.beam_cum = beam_cum;
     a.row_status = row_status;
-    a.D = cps_window_depths(L, KC);
-    const size_t dyn = cps_smem_bytes(L, W, KC, a.D);
+    const bool tri = proxy_kind == 3;
+    a.SW = tri ? KC : KC * KC;
+    a.D = cps_window_depths(L, KC, a.SW);
+    const size_t dyn = cps_smem_bytes(L, W, KC, a.D, a.SW);
     {
-        // raise the kernel's dynamic shared memory limit once per device (the attribute is per device)
+        // raise the kernels' dynamic shared memory limit once per device (the attribute is per device)
         static bool done[64] = {};
         int dev = 0;
         DSP_CUDA_TRY(cudaGetDevice(&dev));
         if (dev < 0 || dev >= 64 || !done[dev]) {
+            const int sw2 = kMaxKC * kMaxKC;
             DSP_CUDA_TRY(cudaFuncSetAttribute(
-                cps_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                (int)cps_smem_bytes(DSP_MAX_L, DSP_MAX_W, kMaxKC, cps_window_depths(DSP_MAX_L, kMaxKC))));
+                cps_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                (int)cps_smem_bytes(DSP_MAX_L, DSP_MAX_W, kMaxKC, cps_window_depths(DSP_MAX_L, kMaxKC, sw2), sw2)));
+            DSP_CUDA_TRY(cudaFuncSetAttribute(
+                cps_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                (int)cps_smem_bytes(DSP_MAX_L, DSP_MAX_W, kMaxKC, cps_window_depths(DSP_MAX_L, kMaxKC, kMaxKC), kMaxKC)));
             if (dev >= 0 && dev < 64) done[dev] = true;
         }
     }
-    cps_kernel<<<B, kThreads, dyn, reinterpret_cast<cudaStream_t>(stream)>>>(a);
+    if (tri) cps_kernel<true><<<B, kThreads, dyn, reinterpret_cast<cudaStream_t>(stream)>>>(a);
+    else cps_kernel<false><<<B, kThreads, dyn, reinterpret_cast<cudaStream_t>(stream)>>>(a);
     DSP_CUDA_TRY(cudaGetLastError());
     return DSP_OK;
 }

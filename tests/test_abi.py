@@ -71,7 +71,7 @@ def test_device_entry_points_reject_bad_arguments_on_the_host():
         return lib.dsp_cps_search(one, one, one, one, 1, 8, 5, one, kind, one, log2, C.c_uint32(0), 100,
                                   W, C.c_float(lam), -1, one, one, one, one, z, z, z, z, z)
     assert cps(W=33) == dsp.DSP_ERR_UNSUPPORTED and cps(log2=0) == dsp.DSP_ERR_INVALID_ARG
-    assert cps(lam=1.5) == dsp.DSP_ERR_INVALID_ARG and cps(kind=2) == dsp.DSP_ERR_UNSUPPORTED
+    assert cps(lam=1.5) == dsp.DSP_ERR_INVALID_ARG and cps(kind=4) == dsp.DSP_ERR_UNSUPPORTED
     # verify: stochastic rows need the draft side
     assert lib.dsp_verify(one, 0, 1, 8, 8, 100, C.c_int64(800), C.c_int64(100), z, C.c_int64(0), C.c_int64(0),
                           one, one, one, z, z, 5, 0, z, z, -1, one, one, z, z, z, one, one,

@@ -200,6 +200,7 @@ def _hand_lattice(B, L, KC, V, seed, *, flat=False, counts=None):
     return SimpleNamespace(cand_id=cand_id.int(), cand_logit=logit.float(), lse64=lse64, cand_count=cnt.int())
 
 
+@pytest.mark.parametrize("kind", [0, 2, 3])             # hashed bigram, tensor of scores, hashed trigram
 @pytest.mark.parametrize("B,L,K,W,eos,lam,flat,case", [
     (3, 128, 32, 32, True, 0.5, False, "max"),     # largest K and W with the EOS slot: 1056 expansions, several windows
     (4, 40, 16, 16, True, 0.0, True, "flat"),      # equal logits and a constant proxy: every expansion ties
@@ -207,7 +208,7 @@ def _hand_lattice(B, L, KC, V, seed, *, flat=False, counts=None):
     (6, 32, 16, 16, True, 0.5, False, "eos"),      # the best beam meets EOS and stops
     (5, 33, 5, 7, False, 0.3, False, "odd"),       # W > K, odd sizes
 ])
-def test_path_search_on_hand_made_lattices(B, L, K, W, eos, lam, flat, case):
+def test_path_search_on_hand_made_lattices(B, L, K, W, eos, lam, flat, case, kind):
     V = 5000
     KC = K + (1 if eos else 0)
     eos_id = 17 if eos else -1
@@ -224,9 +225,10 @@ def test_path_search_on_hand_made_lattices(B, L, K, W, eos, lam, flat, case):
         lat.cand_count[2, L - 1] = 1
         lat.cand_id[3, 9, 1] = eos_id                      # not the best candidate: may or may not stop
     g = torch.Generator().manual_seed(99)
-    table = torch.zeros(1 << 12) if flat else torch.round(torch.randn(1 << 12, generator=g) * 8) / 8 - 3.0
-    prev = torch.randint(0, V, (B,), generator=g).int()
-    kw = dict(W=W, lam=lam, eos_id=eos_id, table_log2=12, hash_seed=5, V=V)
+    tshape = (B, L, KC, KC) if kind == 2 else (1 << 12,)
+    table = torch.zeros(tshape) if flat else torch.round(torch.randn(tshape, generator=g) * 8) / 8 - 3.0
+    prev = torch.randint(0, V, (B, 2) if kind == 3 else (B,), generator=g).int()
+    kw = dict(W=W, lam=lam, eos_id=eos_id, table_log2=12, hash_seed=5, V=V, proxy_kind=kind)
     o = oracle.cps_search(lat.cand_id, lat.cand_logit, lat.lse64, lat.cand_count, prev, table, **kw)
     dlat = SimpleNamespace(**{k: v.to(DEV) for k, v in vars(lat).items()})
     status = torch.zeros(B, dtype=torch.int32, device=DEV)
@@ -308,6 +310,21 @@ def test_step_graphs_per_draft_length_share_buffers():
                                   lam=0.5, table_log2=10, mode=inp["mode"], u=inp["u"])
     g = gpu_step(inp, fused=True, **p)                     # the library still works after the refused capture
     check_step(g, inp, **p)
+
+
+@pytest.mark.parametrize("kind", [2, 3])
+def test_whole_step_with_tensor_and_trigram_proxies(kind):
+    w = wl.CONFIGS[3].scaled(**SMALL[3])
+    inp = wl.make_inputs(w, step=5, device=DEV)
+    p = _params(w)
+    g = torch.Generator().manual_seed(kind)
+    if kind == 2:
+        KC = w.K + (1 if w.eos_id >= 0 else 0)
+        inp["table"] = (-6.0 * torch.rand((w.B, w.L, KC, KC), generator=g)).to(DEV)
+    else:
+        inp["prev_token"] = torch.randint(0, w.V, (w.B, 2), generator=g, dtype=torch.int32).to(DEV)
+    for fused in (False, True):
+        check_step(gpu_step(inp, proxy_kind=kind, fused=fused, **p), inp, proxy_kind=kind, **p)
 
 
 # ---- the drafter's refinement step (Eq. 5) ----
