@@ -256,6 +256,31 @@ def time_workload(w, device, steps, warmup, dist=None, stages=True, seed_base=0)
     return out, st, sets
 
 
+def time_proxies(w, st, sets, device, reps=50):
+    """dsp_cps_search on the headline workload's lattice with each causal proxy (device time per call)."""
+    dsp = st.dsp
+    inp = sets[0]
+    st.run(inp)
+    KC = st.lat.cand_id.shape[2]
+    g = torch.Generator(device=device).manual_seed(3)
+    tensor = -6.0 * torch.rand((w.B, w.L, KC, KC), generator=g, device=device)
+    prev2 = torch.stack([inp["prev_token"], inp["prev_token"]], dim=1).contiguous()
+    cases = {"hashed_bigram": (0, inp["table"], inp["prev_token"]), "tensor": (2, tensor, inp["prev_token"]),
+             "hashed_trigram": (3, inp["table"], prev2)}
+    out = {}
+    for name, (kind, table, prev) in cases.items():
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        for r in range(reps + 3):
+            if r == 3:
+                e0.record()
+            dsp.dsp_cps_search(st.lat, prev, table, W=w.W, lam=w.lam, eos_id=w.eos_id, proxy_kind=kind,
+                               table_log2=inp["table_log2"], hash_seed=inp["hash_seed"], V=w.V, out=st.cps)
+        e1.record()
+        torch.cuda.synchronize()
+        out[name] = e0.elapsed_time(e1) / reps
+    return out
+
+
 def time_unmask(w, device, reps=40):
     """The drafter's refinement step (dsp_unmask_step) on logits of the headline workload's shape:
     S = 1 (every position masked, one call) and S = 4 (four calls, a quarter of the block each;
@@ -490,6 +515,7 @@ def main():
     }
     if not args.no_extras and world == 1:
         line["cpu_baseline"] = cpu_baseline(w, sets[0])
+        line["cps_proxies_ms"] = time_proxies(w, st, sets, device)
         extras = {}
         del st, sets
         torch.cuda.empty_cache()
