@@ -318,6 +318,56 @@ int32_t dsp_draft_verify_step(
     void *verify_workspace, size_t verify_workspace_bytes, dsp_stream_t stream);
 
 /* -------------------------------------------------------------------------
+ * Lattice of a vocabulary-sharded drafter head  (Sec. 3.2 "Lattice and
+ * pruning", Eq. 7, Eq. 9, computed from slices of the vocabulary; the paper
+ * runs one GPU, a tensor-parallel output layer leaves every GPU one slice).
+ *
+ * dsp_lattice_shard reduces one slice [B,L,Vs] of the logits, holding the
+ * tokens vocab_offset .. vocab_offset+Vs-1, to one record per row:
+ *   sums[b,l] : S = sum 2^(x*log2e - c), T = sum 2^(x*log2e - c)*(x*log2e - c)
+ *               over the slice, against the slice's reference exponent c (S = 0
+ *               if the slice has no finite logit), and the logit of eos_id if
+ *               the slice holds that token (NaN otherwise);
+ *   keys[b,l,:]: the slice's best min(K_max, Vs) tokens as sortable 64-bit keys
+ *               (logit, global token id), best first, 0 = none.
+ * The records of all G slices, gathered slice-major into [G,B,L] / [G,B,L,K_max]
+ * / [G,B] buffers in local memory (one all-gather of (24 + 8*K_max) bytes per
+ * row and slice), go to dsp_lattice_merge, which writes the same outputs as
+ * dsp_lattice_build on the whole rows [B,L,V]: identical candidates and counts
+ * (integer compares on the keys), sums added in double.  K_max, eos_id must
+ * agree between the calls; the slices must tile 0..V-1.
+ * Records are plain data but their content is only meaningful to the merge.
+ *
+ * workspace: dsp_shard_workspace_bytes(B, L, Vs, dtype, K_max) for a slice,
+ *            dsp_merge_workspace_bytes(B) for the merge; 256-byte aligned.
+ * shard_status uint32 [B] (written): DSP_ROW_TIMEOUT; the merge ORs the slices'
+ * flags into row_status and adds DSP_ROW_NONFINITE_INPUT as dsp_lattice_build.
+ * Errors : as dsp_lattice_build; INVALID_ARG also for vocab_offset < 0, G < 1;
+ *          UNSUPPORTED for G > 1024.
+ */
+typedef struct dsp_shard_sums {
+    double S, T;
+    float c;
+    float eos_logit;
+} dsp_shard_sums;
+
+int32_t dsp_shard_workspace_bytes(int32_t B, int32_t L, int32_t Vs, int32_t dtype, int32_t K_max,
+                                  size_t *bytes /* host, out */);
+int32_t dsp_lattice_shard(const void *logits, int32_t dtype, int32_t B, int32_t L, int32_t Vs,
+                          int64_t stride_b, int64_t stride_l, int32_t vocab_offset,
+                          int32_t K_max, int32_t eos_id,
+                          dsp_shard_sums *sums, uint64_t *keys, uint32_t *shard_status,
+                          void *workspace, size_t workspace_bytes, dsp_stream_t stream);
+int32_t dsp_merge_workspace_bytes(int32_t B, size_t *bytes /* host, out */);
+int32_t dsp_lattice_merge(int32_t G, const dsp_shard_sums *sums, const uint64_t *keys,
+                          const uint32_t *shard_status,
+                          int32_t B, int32_t L, int32_t V, int32_t K_max, float tau, int32_t eos_id,
+                          int32_t *cand_id, float *cand_logit, float *cand_logp,
+                          int32_t *cand_count, float *lse, double *lse64, float *entropy,
+                          int32_t *gen_len, uint32_t *row_status,
+                          void *workspace, size_t workspace_bytes, dsp_stream_t stream);
+
+/* -------------------------------------------------------------------------
  * Refinement step of the diffusion drafter  (Sec. 3.1, Eq. 5: iterative
  * refinement with the update set "top-K by confidence"; the paper's default
  * S = 1 needs a single call with n_update >= L, S > 1 is its ablation).

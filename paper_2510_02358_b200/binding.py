@@ -30,6 +30,7 @@ EXPORTS = ["dsp_strerror", "dsp_last_cuda_error", "dsp_version", "dsp_profile_ev
            "dsp_lattice_build", "dsp_lattice_build_static", "dsp_cps_search", "dsp_verify_workspace_bytes", "dsp_verify", "dsp_draft_verify_step",
            "dsp_step_graph_create", "dsp_step_graph_launch", "dsp_step_graph_destroy",
            "dsp_unmask_workspace_bytes", "dsp_unmask_step",
+           "dsp_shard_workspace_bytes", "dsp_lattice_shard", "dsp_merge_workspace_bytes", "dsp_lattice_merge",
            "dsp_adl_init", "dsp_adl_update"]
 
 
@@ -324,6 +325,75 @@ def dsp_step_graph_create(draft: torch.Tensor, target: torch.Tensor, prev_token:
     h = C.c_void_p(0)
     _check("dsp_step_graph_create", lib().dsp_step_graph_create(C.byref(h), *args))
     return StepGraph(h, lat, cps, ver, keep)
+
+
+SHARD_SUMS_BYTES = 24      # sizeof(dsp_shard_sums)
+
+
+def dsp_shard_workspace_bytes(B: int, L: int, Vs: int, dtype: int, K_max: int) -> int:
+    n = C.c_size_t(0)
+    _check("dsp_shard_workspace_bytes", lib().dsp_shard_workspace_bytes(B, L, Vs, dtype, K_max, C.byref(n)))
+    return n.value
+
+
+def dsp_lattice_shard(logits: torch.Tensor, vocab_offset: int, K_max: int, eos_id: int = -1, *,
+                      out: Optional[SimpleNamespace] = None, workspace: Optional[torch.Tensor] = None,
+                      stream=None) -> SimpleNamespace:
+    """Records of one vocabulary slice [B,L,Vs]: sums (uint8 [B,L,24], raw dsp_shard_sums), keys
+    (int64 [B,L,K_max], raw 64-bit keys), status (int32 [B])."""
+    B, L, Vs, sb, sl = _logits3(logits, "logits")
+    dev = logits.device
+    if out is None:
+        out = SimpleNamespace(sums=torch.empty((B, L, SHARD_SUMS_BYTES), dtype=torch.uint8, device=dev),
+                              keys=torch.empty((B, L, K_max), dtype=torch.int64, device=dev),
+                              status=torch.empty((B,), dtype=torch.int32, device=dev))
+    dt = _dtype(logits)
+    if workspace is None:
+        workspace = alloc_workspace(dsp_shard_workspace_bytes(B, L, Vs, dt, K_max), dev)
+    _check("dsp_lattice_shard", lib().dsp_lattice_shard(
+        _ptr(logits), dt, B, L, Vs, C.c_int64(sb), C.c_int64(sl), int(vocab_offset), K_max, eos_id,
+        _ptr(out.sums), _ptr(out.keys), _ptr(out.status), _ptr(workspace), C.c_size_t(workspace.numel()),
+        _stream(stream)))
+    return out
+
+
+def dsp_lattice_merge(sums: torch.Tensor, keys: torch.Tensor, status: torch.Tensor, V: int, K_max: int,
+                      tau: float = 0.0, eos_id: int = -1, *, out: Optional[SimpleNamespace] = None,
+                      workspace: Optional[torch.Tensor] = None, stream=None) -> SimpleNamespace:
+    """Finish the lattice from the gathered records of all G slices: sums [G,B,L,24] uint8, keys
+    [G,B,L,K_max] int64, status [G,B] int32 (slice-major, contiguous).  Same outputs as dsp_lattice_build."""
+    G, B, L = sums.shape[0], sums.shape[1], sums.shape[2]
+    dev = sums.device
+    if (tuple(sums.shape) != (G, B, L, SHARD_SUMS_BYTES) or tuple(keys.shape) != (G, B, L, K_max)
+            or tuple(status.shape) != (G, B) or not (sums.is_contiguous() and keys.is_contiguous()
+                                                    and status.is_contiguous())):
+        raise ValueError("records must be contiguous [G,B,L,24] / [G,B,L,K_max] / [G,B] tensors")
+    if out is None:
+        out = lattice_outputs(B, L, K_max, eos_id, dev)
+    n = C.c_size_t(0)
+    _check("dsp_merge_workspace_bytes", lib().dsp_merge_workspace_bytes(B, C.byref(n)))
+    if workspace is None:
+        workspace = alloc_workspace(n.value, dev)
+    _check("dsp_lattice_merge", lib().dsp_lattice_merge(
+        G, _ptr(sums), _ptr(keys), _ptr(status), B, L, int(V), K_max, C.c_float(tau), eos_id,
+        _ptr(out.cand_id), _ptr(out.cand_logit), _ptr(out.cand_logp), _ptr(out.cand_count), _ptr(out.lse),
+        _ptr(out.lse64), _ptr(out.entropy), _ptr(out.gen_len), _ptr(out.row_status), _ptr(workspace),
+        C.c_size_t(workspace.numel()), _stream(stream)))
+    return out
+
+
+def gather_shard_records(rec: SimpleNamespace, group=None) -> SimpleNamespace:
+    """All-gather one rank's slice records into the slice-major buffers dsp_lattice_merge reads
+    (rank r holds slice r).  Plain torch.distributed collectives on the records' device."""
+    import torch.distributed as dist
+    G = dist.get_world_size(group)
+    out = SimpleNamespace()
+    for name in ("sums", "keys", "status"):
+        t = getattr(rec, name).contiguous()
+        parts = [torch.empty_like(t) for _ in range(G)]
+        dist.all_gather(parts, t, group=group)
+        setattr(out, name, torch.stack(parts, dim=0).contiguous())
+    return out
 
 
 def dsp_unmask_workspace_bytes(B: int, L: int, V: int, dtype: int) -> int:

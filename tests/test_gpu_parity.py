@@ -327,6 +327,63 @@ def test_whole_step_with_tensor_and_trigram_proxies(kind):
         check_step(gpu_step(inp, proxy_kind=kind, fused=fused, **p), inp, proxy_kind=kind, **p)
 
 
+# ---- the lattice from vocabulary slices (tensor-parallel drafter head) ----
+def _sharded_lattice(x, cuts, K, tau, eos_id):
+    """Slice records one after the other on this GPU, stacked slice-major (the all-gather's layout), merged."""
+    recs = []
+    for lo, hi in zip(cuts[:-1], cuts[1:]):
+        recs.append(dsp.dsp_lattice_shard(x[:, :, lo:hi], lo, K, eos_id))
+    stack = lambda name: torch.stack([getattr(r, name) for r in recs], dim=0).contiguous()
+    return dsp.dsp_lattice_merge(stack("sums"), stack("keys"), stack("status"), x.shape[2], K, tau, eos_id)
+
+
+@pytest.mark.parametrize("B,L,V,dtype,K,cuts", [
+    (3, 5, 152064, torch.bfloat16, 16, [0, 38016, 76032, 114048, 152064]),      # four equal, aligned slices
+    (2, 4, 152064, torch.bfloat16, 32, [0, 19008 * 3, 19008 * 4, 152064]),      # unequal slices
+    (2, 3, 50021, torch.bfloat16, 8, [0, 16384, 16391, 50021]),                 # unaligned slices: element-wise path
+    (2, 6, 12288, torch.float32, 4, [0, 12288]),                                # one slice
+    (1, 2, 4096, torch.float32, 32, [0, 8, 16, 24, 4096]),                      # slices shorter than K_max
+])
+def test_lattice_from_vocabulary_slices_equals_the_whole_row_build(B, L, V, dtype, K, cuts):
+    g = torch.Generator().manual_seed(V + K)
+    x = (2.5 * torch.randn((B, L, V), generator=g)).to(dtype)
+    x[0, 0, 100:200] = float("-inf")                       # masked tokens
+    if B > 1:
+        x[1, 1, :cuts[1]] = float("-inf")                  # a slice without a finite logit
+    eos = V - 3
+    x[0, L - 1, eos] = 30.0                                # EOS on top at the last position: gen_len = L - 1
+    x = x.to(DEV)
+    for tau, eos_id in ((0.0, -1), (0.8, eos)):
+        whole = dsp.dsp_lattice_build(x, K, tau, eos_id)
+        parts = _sharded_lattice(x, cuts, K, tau, eos_id)
+        torch.cuda.synchronize()
+        for name in ("cand_id", "cand_logit", "cand_count", "gen_len", "row_status"):
+            assert torch.equal(getattr(parts, name), getattr(whole, name)), name
+        assert torch.allclose(parts.lse64, whole.lse64, atol=1e-6, rtol=0, equal_nan=True)
+        assert torch.allclose(parts.entropy, whole.entropy, atol=1e-5, rtol=0, equal_nan=True)
+        assert torch.allclose(parts.cand_logp, whole.cand_logp, atol=1e-5, rtol=0, equal_nan=True)
+        o = oracle.lattice_build(x.cpu(), K, tau=tau, eos_id=eos_id)
+        good = (o.row_status & oracle.NONFINITE_INPUT) == 0     # a row without a finite logit flags its batch row
+        assert torch.equal(parts.row_status.cpu() != 0, ~good)
+        assert torch.equal(parts.cand_id.cpu()[good], o.cand_id[good])
+        assert torch.equal(parts.cand_count.cpu()[good], o.cand_count[good])
+        assert torch.equal(parts.gen_len.cpu()[good], o.gen_len[good])
+        assert torch.allclose(parts.lse64.cpu()[good], o.lse64[good], atol=1e-5, rtol=0)
+        assert torch.allclose(parts.entropy.cpu()[good], o.entropy[good], atol=1e-3, rtol=0)
+        fin = torch.isfinite(o.cand_logp) & good.view(-1, 1, 1)
+        assert (parts.cand_logp.cpu()[fin] - o.cand_logp[fin]).abs().max() <= 1e-3
+
+
+def test_lattice_from_slices_flags_nonfinite_rows():
+    B, L, V, K = 2, 3, 16384, 4
+    x = torch.randn((B, L, V)).to(torch.bfloat16)
+    x[1, 2, 9000] = float("nan")
+    x = x.to(DEV)
+    out = _sharded_lattice(x, [0, 8192, 16384], K, 0.0, -1)
+    torch.cuda.synchronize()
+    assert out.row_status.cpu().tolist() == [0, dsp.ROW_NONFINITE_INPUT]
+
+
 # ---- the drafter's refinement step (Eq. 5) ----
 def _check_unmask(x, tokens, masked, n, ws=None):
     """One step on both sides from the same state; returns the new state (the GPU's)."""

@@ -59,3 +59,38 @@ def test_two_ranks_gloo():
     assert r0["value"] == r1["value"] == 2 * 20 / 0.015       # both ranks' steps over the slowest time
     assert r0["k"] == r1["k"] and r0["k"][0] == r0["k"][1]    # every rank derives the same next length
     assert r0["draft_sum"] != r1["draft_sum"]                 # different rows per rank
+
+
+def _gather_worker(rank, world, port, out):
+    sys.path.insert(0, ROOT)
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port), RANK=str(rank), WORLD_SIZE=str(world))
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    from types import SimpleNamespace
+    from paper_2510_02358_b200 import binding as dsp
+    B, L, K = 2, 3, 4
+    # stand-ins for one rank's slice records (their content is the kernels' business, the layout is the host's)
+    rec = SimpleNamespace(sums=torch.full((B, L, dsp.SHARD_SUMS_BYTES), rank + 1, dtype=torch.uint8),
+                          keys=torch.arange(B * L * K, dtype=torch.int64).view(B, L, K) + 1000 * rank,
+                          status=torch.full((B,), 32 * rank, dtype=torch.int32))
+    g = dsp.gather_shard_records(rec)
+    out[rank] = dict(sums=g.sums.clone(), keys=g.keys.clone(), status=g.status.clone())
+    dist.barrier()
+    dist.destroy_process_group()
+
+
+def test_slice_records_are_gathered_slice_major_on_every_rank():
+    """The vocabulary-sharded lattice: rank r holds slice r; every rank ends with the [G, ...] buffers
+    that dsp_lattice_merge reads, slice r at index r."""
+    world = 2
+    port = 31500 + os.getpid() % 2000
+    mgr = mp.Manager()
+    out = mgr.dict()
+    mp.spawn(_gather_worker, args=(world, port, out), nprocs=world, join=True)
+    for r in range(world):
+        o = out[r]
+        assert tuple(o["sums"].shape) == (world, 2, 3, 24) and tuple(o["keys"].shape) == (world, 2, 3, 4)
+        assert tuple(o["status"].shape) == (world, 2)
+        for s in range(world):
+            assert (o["sums"][s] == s + 1).all() and o["keys"][s, 0, 0, 0] == 1000 * s
+            assert (o["status"][s] == 32 * s).all()
+    assert torch.equal(out[0]["keys"], out[1]["keys"])
