@@ -423,13 +423,12 @@ extern "C" int32_t dsp_cps_search(const int32_t *cand_id, const float *cand_logi
         int dev = 0;
         DSP_CUDA_TRY(cudaGetDevice(&dev));
         if (dev < 0 || dev >= 64 || !done[dev]) {
-            const int sw2 = kMaxKC * kMaxKC;
-            DSP_CUDA_TRY(cudaFuncSetAttribute(
-                cps_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                (int)cps_smem_bytes(DSP_MAX_L, DSP_MAX_W, kMaxKC, cps_window_depths(DSP_MAX_L, kMaxKC, sw2), sw2)));
-            DSP_CUDA_TRY(cudaFuncSetAttribute(
-                cps_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                (int)cps_smem_bytes(DSP_MAX_L, DSP_MAX_W, kMaxKC, cps_window_depths(DSP_MAX_L, kMaxKC, kMaxKC), kMaxKC)));
+            // largest request of any shape: the back-pointers of the longest, widest search and a full
+            // window (a window's arrays fill the budget up to one depth's worth of rounding)
+            const int most = (int)(align_up((size_t)3 * DSP_MAX_L * DSP_MAX_W, 16) + kStepBudgetBytes +
+                                   (size_t)kMaxKC * 8 + 64);
+            DSP_CUDA_TRY(cudaFuncSetAttribute(cps_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, most));
+            DSP_CUDA_TRY(cudaFuncSetAttribute(cps_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, most));
             if (dev >= 0 && dev < 64) done[dev] = true;
         }
     }

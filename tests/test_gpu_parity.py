@@ -207,6 +207,7 @@ def _hand_lattice(B, L, KC, V, seed, *, flat=False, counts=None):
     (4, 24, 8, 8, False, 1.0, False, "holes"),     # positions without candidates end the lattice
     (6, 32, 16, 16, True, 0.5, False, "eos"),      # the best beam meets EOS and stops
     (5, 33, 5, 7, False, 0.3, False, "odd"),       # W > K, odd sizes
+    (2, 1024, 3, 32, True, 0.5, False, "long"),    # the longest draft the library takes
 ])
 def test_path_search_on_hand_made_lattices(B, L, K, W, eos, lam, flat, case, kind):
     V = 5000
@@ -454,6 +455,21 @@ def test_unmask_step_ties_masked_logits_and_flags():
     _check_unmask(x, tokens, masked, 2)
     with pytest.raises(dsp.DspError):
         dsp.dsp_unmask_step(x, tokens.to(DEV), masked.to(DEV), 0)
+
+
+def test_longest_draft_through_the_whole_step_and_the_refinement():
+    """L = DSP_MAX_L with a small vocabulary: every kernel's per-batch-row bookkeeping at its largest."""
+    B, L, V = 2, dsp.DSP_MAX_L, 2048
+    inp = _to(wl.tiny_random(B, L, V, dtype=torch.bfloat16, seed=31))
+    p = dict(K=4, W=4, tau=0.0, lam=0.5, eos_id=-1)
+    check_step(gpu_step(inp, fused=True, **p), inp, **p)
+    tokens = torch.zeros((B, L), dtype=torch.int32)
+    masked = torch.ones((B, L), dtype=torch.uint8)
+    for _ in range(2):
+        tokens, masked = _check_unmask(inp["draft"], tokens, masked, L // 2)
+    assert masked.sum() == 0
+    with pytest.raises(dsp.DspError):
+        dsp.dsp_lattice_build(torch.zeros((1, L + 1, 64), device=DEV), 4)
 
 
 def test_profile_events_bracket_the_scan_kernels():
