@@ -472,6 +472,18 @@ def test_longest_draft_through_the_whole_step_and_the_refinement():
         dsp.dsp_lattice_build(torch.zeros((1, L + 1, 64), device=DEV), 4)
 
 
+def test_many_batch_rows():
+    """Thousands of short rows: grids, tickets and per-batch-row state far beyond the benchmark's batch sizes."""
+    B, L, V = 6000, 2, 256
+    inp = _to(wl.tiny_random(B, L, V, dtype=torch.float32, seed=41))
+    p = dict(K=4, W=2, tau=0.7, lam=0.5, eos_id=5)
+    rep = check_step(gpu_step(inp, fused=True, **p), inp, **p)
+    assert rep["near_accept"] + rep["near_token"] + rep["near_tau"] <= 6
+    tokens = torch.zeros((B, L), dtype=torch.int32)
+    masked = torch.ones((B, L), dtype=torch.uint8)
+    _check_unmask(inp["draft"], tokens, masked, 1)
+
+
 def test_profile_events_bracket_the_scan_kernels():
     w = wl.CONFIGS[3].scaled(B=2, L=4, V=152064)
     inp = wl.make_inputs(w, device=DEV)
