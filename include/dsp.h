@@ -368,6 +368,59 @@ int32_t dsp_lattice_merge(int32_t G, const dsp_shard_sums *sums, const uint64_t 
                           void *workspace, size_t workspace_bytes, dsp_stream_t stream);
 
 /* -------------------------------------------------------------------------
+ * Verification with a vocabulary-sharded target head  (Sec. 2 Eq. 1, Eq. 2,
+ * residual resampling; greedy decoding of Sec. 4 -- dsp_verify computed from
+ * slices of the target's vocabulary, as a tensor-parallel verifier leaves them).
+ *
+ * 1. dsp_target_shard: every GPU reduces its slice [B,Lt,Vs] of the target
+ *    logits to one record per row (as dsp_lattice_shard with one key: the
+ *    slice's argmax; the record's probe logit is the target logit of the row's
+ *    path token if the slice holds that token).  All-gather the records.
+ * 2. dsp_verify_merge (every GPU, same result): argmax and log-sum-exp of every
+ *    target row from the records, then the acceptance scan exactly as
+ *    dsp_verify.  Greedy rows are finished (next_token).  For a stochastic row
+ *    that needs a draw, job_trow[b] names the target row (b*Lt + i) to sample
+ *    from and job_drow[b] the draft row (b*L + i) of the residual, or -1 for a
+ *    bonus draw from p; job_trow[b] = -1: nothing to draw; next_token[b] = -1
+ *    until step 3.  tgt_lse64 [B,Lt] (double) is an output the draw needs.
+ * 3. The caller gathers, into local memory, the named rows' slices from all
+ *    GPUs into whole rows target_rows [B,V] and draft_rows [B,V] (row b = batch
+ *    row b's row; rows of batch rows without a job are not read; strides in
+ *    elements), and dsp_residual_sample draws next_token[b] as dsp_verify does
+ *    (inverse CDF of [p - q]_+ or of p with u[b,L]; DSP_ROW_ZERO_RESIDUAL).
+ * The draft side (cand_logit, draft_lse64) comes from the lattice, sharded or
+ * not.  Other arguments, outputs, flags and errors as dsp_verify.
+ * workspace: dsp_shard_workspace_bytes(B, Lt, Vs, dtype, 1),
+ *            dsp_verify_merge_workspace_bytes(B, Lt),
+ *            dsp_residual_sample_workspace_bytes(B, V, dtype); 256-byte aligned.
+ */
+int32_t dsp_target_shard(const void *logits, int32_t dtype, int32_t B, int32_t L, int32_t Lt, int32_t Vs,
+                         int64_t stride_b, int64_t stride_l, int32_t vocab_offset,
+                         const int32_t *path, const int32_t *path_len,
+                         dsp_shard_sums *sums, uint64_t *keys /* [B,Lt,1] */, uint32_t *shard_status,
+                         void *workspace, size_t workspace_bytes, dsp_stream_t stream);
+int32_t dsp_verify_merge_workspace_bytes(int32_t B, int32_t Lt, size_t *bytes /* host, out */);
+int32_t dsp_verify_merge(int32_t G, const dsp_shard_sums *sums /* [G,B,Lt] */, const uint64_t *keys /* [G,B,Lt] */,
+                         const uint32_t *shard_status /* [G,B] */,
+                         int32_t B, int32_t L, int32_t Lt,
+                         const int32_t *path, const int32_t *path_slot, const int32_t *path_len,
+                         const float *cand_logit, const double *draft_lse64, int32_t KC,
+                         int32_t all_greedy, const uint8_t *mode, const float *u, int32_t eos_id,
+                         int32_t *accepted_len, int32_t *next_token, float *ratio /* nullable */,
+                         int32_t *tgt_argmax, float *tgt_lse /* nullable */, double *tgt_lse64,
+                         int32_t *job_trow, int32_t *job_drow, uint32_t *row_status,
+                         void *workspace, size_t workspace_bytes, dsp_stream_t stream);
+int32_t dsp_residual_sample_workspace_bytes(int32_t B, int32_t V, int32_t dtype, size_t *bytes /* host, out */);
+int32_t dsp_residual_sample(const void *target_rows, const void *draft_rows, int32_t dtype,
+                            int32_t B, int32_t L, int32_t Lt, int32_t V,
+                            int64_t tstride, int64_t dstride,
+                            const int32_t *job_trow, const int32_t *job_drow,
+                            const double *tgt_lse64, const double *draft_lse64,
+                            const int32_t *tgt_argmax, const float *u,
+                            int32_t *next_token, uint32_t *row_status,
+                            void *workspace, size_t workspace_bytes, dsp_stream_t stream);
+
+/* -------------------------------------------------------------------------
  * Refinement step of the diffusion drafter  (Sec. 3.1, Eq. 5: iterative
  * refinement with the update set "top-K by confidence"; the paper's default
  * S = 1 needs a single call with n_update >= L, S > 1 is its ablation).

@@ -31,6 +31,8 @@ EXPORTS = ["dsp_strerror", "dsp_last_cuda_error", "dsp_version", "dsp_profile_ev
            "dsp_step_graph_create", "dsp_step_graph_launch", "dsp_step_graph_destroy",
            "dsp_unmask_workspace_bytes", "dsp_unmask_step",
            "dsp_shard_workspace_bytes", "dsp_lattice_shard", "dsp_merge_workspace_bytes", "dsp_lattice_merge",
+           "dsp_target_shard", "dsp_verify_merge_workspace_bytes", "dsp_verify_merge",
+           "dsp_residual_sample_workspace_bytes", "dsp_residual_sample",
            "dsp_adl_init", "dsp_adl_update"]
 
 
@@ -380,6 +382,77 @@ def dsp_lattice_merge(sums: torch.Tensor, keys: torch.Tensor, status: torch.Tens
         _ptr(out.lse64), _ptr(out.entropy), _ptr(out.gen_len), _ptr(out.row_status), _ptr(workspace),
         C.c_size_t(workspace.numel()), _stream(stream)))
     return out
+
+
+def dsp_target_shard(logits: torch.Tensor, vocab_offset: int, cps: SimpleNamespace, *,
+                     out: Optional[SimpleNamespace] = None, workspace: Optional[torch.Tensor] = None,
+                     stream=None) -> SimpleNamespace:
+    """Records of one vocabulary slice [B,Lt,Vs] of the target logits for the path in ``cps``."""
+    B, Lt, Vs, sb, sl = _logits3(logits, "logits")
+    L = cps.path.shape[1]
+    dev = logits.device
+    if out is None:
+        out = SimpleNamespace(sums=torch.empty((B, Lt, SHARD_SUMS_BYTES), dtype=torch.uint8, device=dev),
+                              keys=torch.empty((B, Lt, 1), dtype=torch.int64, device=dev),
+                              status=torch.empty((B,), dtype=torch.int32, device=dev))
+    dt = _dtype(logits)
+    if workspace is None:
+        workspace = alloc_workspace(dsp_shard_workspace_bytes(B, Lt, Vs, dt, 1), dev)
+    _check("dsp_target_shard", lib().dsp_target_shard(
+        _ptr(logits), dt, B, L, Lt, Vs, C.c_int64(sb), C.c_int64(sl), int(vocab_offset), _ptr(cps.path),
+        _ptr(cps.path_len), _ptr(out.sums), _ptr(out.keys), _ptr(out.status), _ptr(workspace),
+        C.c_size_t(workspace.numel()), _stream(stream)))
+    return out
+
+
+def dsp_verify_merge(sums: torch.Tensor, keys: torch.Tensor, status: torch.Tensor, cps: SimpleNamespace,
+                     lat: Optional[SimpleNamespace], *, mode: Optional[torch.Tensor] = None,
+                     u: Optional[torch.Tensor] = None, eos_id: int = -1, all_greedy: bool = False,
+                     row_status: Optional[torch.Tensor] = None, workspace: Optional[torch.Tensor] = None,
+                     stream=None) -> SimpleNamespace:
+    """Verification from the gathered target records ([G,B,Lt,24] / [G,B,Lt,1] / [G,B]); returns
+    dsp_verify's outputs plus tgt_lse64, job_trow, job_drow (see include/dsp.h)."""
+    G, B, Lt = sums.shape[0], sums.shape[1], sums.shape[2]
+    L = cps.path.shape[1]
+    dev = sums.device
+    out = verify_outputs(B, L, Lt, dev)
+    e = lambda shape, dt: torch.empty(shape, dtype=dt, device=dev)
+    out.tgt_lse64, out.job_trow, out.job_drow = e((B, Lt), torch.float64), e((B,), torch.int32), e((B,), torch.int32)
+    out.row_status = torch.zeros((B,), dtype=torch.int32, device=dev) if row_status is None else row_status
+    n = C.c_size_t(0)
+    _check("dsp_verify_merge_workspace_bytes", lib().dsp_verify_merge_workspace_bytes(B, Lt, C.byref(n)))
+    if workspace is None:
+        workspace = alloc_workspace(n.value, dev)
+    KC = 1 if lat is None else lat.cand_logit.shape[2]
+    _check("dsp_verify_merge", lib().dsp_verify_merge(
+        G, _ptr(sums.contiguous()), _ptr(keys.contiguous()), _ptr(status.contiguous()), B, L, Lt,
+        _ptr(cps.path), _ptr(cps.path_slot), _ptr(cps.path_len),
+        _ptr(None if lat is None else lat.cand_logit), _ptr(None if lat is None else lat.lse64), KC,
+        1 if all_greedy else 0, _ptr(mode), _ptr(u), eos_id, _ptr(out.accepted_len), _ptr(out.next_token),
+        _ptr(out.ratio), _ptr(out.tgt_argmax), _ptr(out.tgt_lse), _ptr(out.tgt_lse64), _ptr(out.job_trow),
+        _ptr(out.job_drow), _ptr(out.row_status), _ptr(workspace), C.c_size_t(workspace.numel()), _stream(stream)))
+    return out
+
+
+def dsp_residual_sample(target_rows: torch.Tensor, draft_rows: torch.Tensor, ver: SimpleNamespace,
+                        lat: SimpleNamespace, u: torch.Tensor, L: int, *,
+                        workspace: Optional[torch.Tensor] = None, stream=None) -> None:
+    """Draw the pending tokens of ``ver`` (from dsp_verify_merge) from the gathered whole rows
+    [B,V]; ``ver.next_token`` and ``ver.row_status`` are updated in place."""
+    B, V = target_rows.shape
+    Lt = ver.tgt_argmax.shape[1]
+    if target_rows.stride(1) != 1 or draft_rows.stride(1) != 1 or tuple(draft_rows.shape) != (B, V):
+        raise ValueError("target_rows / draft_rows must be [B, V] with a contiguous vocabulary dimension")
+    dt = _dtype(target_rows)
+    n = C.c_size_t(0)
+    _check("dsp_residual_sample_workspace_bytes", lib().dsp_residual_sample_workspace_bytes(B, V, dt, C.byref(n)))
+    if workspace is None:
+        workspace = alloc_workspace(n.value, target_rows.device)
+    _check("dsp_residual_sample", lib().dsp_residual_sample(
+        _ptr(target_rows), _ptr(draft_rows), dt, B, L, Lt, V, C.c_int64(target_rows.stride(0)),
+        C.c_int64(draft_rows.stride(0)), _ptr(ver.job_trow), _ptr(ver.job_drow), _ptr(ver.tgt_lse64),
+        _ptr(lat.lse64), _ptr(ver.tgt_argmax), _ptr(u), _ptr(ver.next_token), _ptr(ver.row_status),
+        _ptr(workspace), C.c_size_t(workspace.numel()), _stream(stream)))
 
 
 def gather_shard_records(rec: SimpleNamespace, group=None) -> SimpleNamespace:

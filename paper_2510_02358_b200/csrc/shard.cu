@@ -20,6 +20,8 @@ struct ShardArgs {
     int B, L, V;              // V: the slice's length
     long long stride_b, stride_l;
     int vocab_offset, K, K_max, eos_id;
+    const int32_t *path, *path_len;   // target side: the row's probe token is its path token (else eos_id)
+    int Lp;                           // row length of `path`
     dsp_shard_sums *sums;     // [B,L]
     unsigned long long *keys; // [B,L,K_max]
     uint32_t *shard_status;   // [B]
@@ -137,8 +139,10 @@ __global__ void __launch_bounds__(kThreads) shard_rows_kernel(const ShardArgs a)
     if (lane == 0) {
         dsp_shard_sums r;
         r.S = S; r.T = T; r.c = c;
-        const int e = a.eos_id - a.vocab_offset;
-        r.eos_logit = (a.eos_id >= 0 && e >= 0 && e < a.V) ? Elem<DT>::load1(rowp + e) : CUDART_NAN_F;
+        int probe = a.eos_id;                  // the one token whose logit the record carries
+        if (a.path) probe = (l < a.Lp && l < __ldg(&a.path_len[b])) ? __ldg(&a.path[(long long)b * a.Lp + l]) : -1;
+        const int e = probe - a.vocab_offset;
+        r.eos_logit = (probe >= 0 && e >= 0 && e < a.V) ? Elem<DT>::load1(rowp + e) : CUDART_NAN_F;
         a.sums[row] = r;
     }
     // the warp finishing a batch row's last row publishes its status (time-outs of pass 1)
@@ -262,11 +266,11 @@ extern "C" int32_t dsp_shard_workspace_bytes(int32_t B, int32_t L, int32_t V, in
     return DSP_OK;
 }
 
-extern "C" int32_t dsp_lattice_shard(const void *logits, int32_t dtype, int32_t B, int32_t L, int32_t V,
-                                     int64_t stride_b, int64_t stride_l, int32_t vocab_offset,
-                                     int32_t K_max, int32_t eos_id,
-                                     dsp_shard_sums *sums, uint64_t *keys, uint32_t *shard_status,
-                                     void *workspace, size_t workspace_bytes, dsp_stream_t stream) {
+static int32_t shard_impl(const void *logits, int32_t dtype, int32_t B, int32_t L, int32_t V,
+                          int64_t stride_b, int64_t stride_l, int32_t vocab_offset,
+                          int32_t K_max, int32_t eos_id, const int32_t *path, const int32_t *path_len, int32_t Lp,
+                          dsp_shard_sums *sums, uint64_t *keys, uint32_t *shard_status,
+                          void *workspace, size_t workspace_bytes, dsp_stream_t stream) {
     const int32_t rc = check_shard_shape(B, L, V, dtype, K_max);
     if (rc != DSP_OK) return rc;
     if (vocab_offset < 0 || (int64_t)vocab_offset + V > (int64_t)1 << 30) return DSP_ERR_INVALID_ARG;
@@ -285,12 +289,35 @@ extern "C" int32_t dsp_lattice_shard(const void *logits, int32_t dtype, int32_t 
     a.K_max = K_max;
     a.K = K_max < V ? K_max : V;
     a.eos_id = eos_id;
+    a.path = path; a.path_len = path_len; a.Lp = Lp;
     a.sums = sums;
     a.keys = reinterpret_cast<unsigned long long *>(keys);
     a.shard_status = shard_status;
     cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
     return dtype == DSP_BF16 ? launch_shard<__nv_bfloat16>(a, workspace, workspace_bytes, st)
                              : launch_shard<float>(a, workspace, workspace_bytes, st);
+}
+
+extern "C" int32_t dsp_lattice_shard(const void *logits, int32_t dtype, int32_t B, int32_t L, int32_t V,
+                                     int64_t stride_b, int64_t stride_l, int32_t vocab_offset,
+                                     int32_t K_max, int32_t eos_id,
+                                     dsp_shard_sums *sums, uint64_t *keys, uint32_t *shard_status,
+                                     void *workspace, size_t workspace_bytes, dsp_stream_t stream) {
+    return shard_impl(logits, dtype, B, L, V, stride_b, stride_l, vocab_offset, K_max, eos_id, nullptr, nullptr, 0,
+                      sums, keys, shard_status, workspace, workspace_bytes, stream);
+}
+
+// The target side: one key (the slice's argmax) and, as the record's probe logit, the logit of
+// the row's path token if the slice holds it.
+extern "C" int32_t dsp_target_shard(const void *logits, int32_t dtype, int32_t B, int32_t L, int32_t Lt, int32_t V,
+                                    int64_t stride_b, int64_t stride_l, int32_t vocab_offset,
+                                    const int32_t *path, const int32_t *path_len,
+                                    dsp_shard_sums *sums, uint64_t *keys, uint32_t *shard_status,
+                                    void *workspace, size_t workspace_bytes, dsp_stream_t stream) {
+    if (L < 1 || Lt < L || Lt > L + 1) return DSP_ERR_INVALID_ARG;
+    if (B > 0 && (!path || !path_len)) return DSP_ERR_INVALID_ARG;
+    return shard_impl(logits, dtype, B, Lt, V, stride_b, stride_l, vocab_offset, 1, -1, path, path_len, L,
+                      sums, keys, shard_status, workspace, workspace_bytes, stream);
 }
 
 extern "C" int32_t dsp_merge_workspace_bytes(int32_t B, size_t *bytes) {

@@ -58,6 +58,10 @@ struct VerifyArgs {
     SampleJob *jobs;           // [B]
     double *chunk_sums;        // [B, nchunks]
     int nchunks, res_slices, chunks_per_slice;
+    // sharded target head (dsp_verify_merge): the path tokens' target logits come from the slices' records,
+    // and the rows to sample from are reported to the caller
+    const float *xt_probe;     // [B*Lt] or null
+    int32_t *job_trow, *job_drow;   // [B] or null
 };
 
 template <typename DT>
@@ -90,7 +94,8 @@ __device__ void accept_row(const VerifyArgs &a, int b) {
                 rej = y != __ldcg(&a.argmax[(long long)b * Lt + i]);
             } else {
                 const int slot = __ldcg(&a.path_slot[(long long)b * L + i]);
-                const double xt = (double)Elem<DT>::load1(trow_ptr<DT>(a, (long long)b * Lt + i) + y);
+                const double xt = a.xt_probe ? (double)__ldcg(&a.xt_probe[(long long)b * Lt + i])
+                                             : (double)Elem<DT>::load1(trow_ptr<DT>(a, (long long)b * Lt + i) + y);
                 const double xd = (double)__ldcg(&a.cand_logit[((long long)b * L + i) * a.KC + slot]);
                 const double lp = xt - __ldcg(&a.tlse64[(long long)b * Lt + i]);
                 const double lq = xd - __ldcg(&a.draft_lse64[(long long)b * L + i]);
@@ -133,6 +138,7 @@ __device__ void accept_row(const VerifyArgs &a, int b) {
         a.accepted_len[b] = acc;
         a.next_token[b] = nt;
         if (!a.all_greedy) a.jobs[b] = job;
+        if (a.job_trow) { a.job_trow[b] = job.trow; a.job_drow[b] = job.drow; }
         if (status) atomicOr(&a.row_status[b], status);
     }
 }
@@ -555,6 +561,160 @@ static int32_t launch_verify(VerifyArgs &a, void *workspace, size_t workspace_by
     return DSP_OK;
 }
 
+// ---- sharded target head: statistics from the slices' records, sampling from gathered rows ----
+
+struct TargetMergeArgs {
+    int G, B, Lt;
+    const dsp_shard_sums *sums;        // [G,B,Lt]
+    const unsigned long long *keys;    // [G,B,Lt] (one key per slice and row)
+    const uint32_t *shard_status;      // [G,B]
+    int32_t *argmax;                   // [B*Lt]
+    double *tlse64;                    // [B*Lt]
+    float *xt;                         // [B*Lt] target logit of the row's path token (NaN: none)
+    int32_t *tgt_argmax;
+    float *tgt_lse;
+    unsigned *b_status;
+};
+
+// One warp per target row: argmax = the best of the slices' keys, log-sum-exp from the slices'
+// sums against a common reference exponent, the path token's logit from the slice that holds it.
+__global__ void __launch_bounds__(kThreads) target_merge_kernel(const TargetMergeArgs m) {
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const long long nrows = (long long)m.B * m.Lt;
+    const long long row = (long long)blockIdx.x * kWarps + warp;
+    if (row >= nrows) return;
+    const int b = (int)(row / m.Lt);
+    float cm = kRefFloor, xt = CUDART_NAN_F;
+    unsigned long long best = 0ull;
+    for (int g = lane; g < m.G; g += 32) {
+        const dsp_shard_sums r = m.sums[g * nrows + row];
+        if (r.S > 0.0 || !(r.S == r.S)) cm = fmaxf(cm, r.c);
+        if (r.eos_logit == r.eos_logit) xt = r.eos_logit;
+        const unsigned long long k = m.keys[g * nrows + row];
+        best = k > best ? k : best;
+    }
+    cm = warp_max(cm);
+    best = warp_max(best);
+    double S = 0.0, T = 0.0;
+    for (int g = lane; g < m.G; g += 32) {
+        const dsp_shard_sums r = m.sums[g * nrows + row];
+        if (r.S != 0.0) {
+            const double d = (double)r.c - (double)cm;
+            const double w = exp2(d);
+            S += w * r.S;
+            T += w * (r.T + r.S * d);
+        }
+    }
+    S = warp_sum(S);
+    T = warp_sum(T);
+    const unsigned has = __ballot_sync(0xFFFFFFFFu, xt == xt);
+    xt = has ? __shfl_sync(0xFFFFFFFFu, xt, __ffs(has) - 1) : CUDART_NAN_F;
+    if (lane == 0) {
+        double lse, mean_x;
+        const bool ok = row_log_stats(cm, S, T, lse, mean_x) && best != 0ull;
+        const int am = best ? key_id(best) : 0;
+        m.argmax[row] = am;
+        m.tlse64[row] = lse;
+        m.xt[row] = xt;
+        if (m.tgt_argmax) m.tgt_argmax[row] = am;
+        if (m.tgt_lse) m.tgt_lse[row] = (float)lse;
+        unsigned st = ok ? 0u : DSP_ROW_NONFINITE_INPUT;
+        if (row == (long long)b * m.Lt)
+            for (int g = 0; g < m.G; ++g) st |= m.shard_status[(long long)g * m.B + b];
+        if (st) atomicOr(&m.b_status[b], st);
+    }
+}
+
+struct SampleArgs {
+    int B, L, Lt;
+    const int32_t *job_trow, *job_drow;    // [B]
+    const double *tgt_lse64, *draft_lse64; // [B*Lt], [B*L]
+    const int32_t *tgt_argmax;             // [B*Lt]
+    const float *u;                        // [B,L+1]
+    SampleJob *jobs;                       // [B]
+    double *tlse_g, *dlse_g;               // [B]
+};
+// Jobs over the gathered rows: row b of the gathered arrays is batch row b's row to sample from.
+__global__ void sample_prepare_kernel(const SampleArgs s) {
+    const int b = blockIdx.x * blockDim.x + threadIdx.x;
+    if (b >= s.B) return;
+    SampleJob job;
+    job.trow = -1; job.drow = -1; job.u = 0.f; job.fallback = -1;
+    const int tr = s.job_trow[b], dr = s.job_drow[b];
+    double tl = 0.0, dl = 0.0;
+    if (tr >= 0) {
+        job.trow = b;
+        job.drow = dr >= 0 ? b : -1;
+        job.u = s.u[(long long)b * (s.L + 1) + s.L];
+        job.fallback = s.tgt_argmax[tr];
+        tl = s.tgt_lse64[tr];
+        if (dr >= 0) dl = s.draft_lse64[dr];
+    }
+    s.jobs[b] = job;
+    s.tlse_g[b] = tl;
+    s.dlse_g[b] = dl;
+}
+
+struct MergeWs {
+    size_t off_b_status, zero_bytes, off_argmax, off_tlse, off_xt, off_jobs, total;
+};
+static MergeWs verify_merge_ws_layout(int64_t B, int64_t Lt) {
+    MergeWs w;
+    size_t o = 0;
+    w.off_b_status = o; o += align_up((size_t)B * 4, 256);
+    w.zero_bytes = o;
+    w.off_argmax = o;   o += align_up((size_t)(B * Lt) * 4, 256);
+    w.off_tlse = o;     o += align_up((size_t)(B * Lt) * 8, 256);
+    w.off_xt = o;       o += align_up((size_t)(B * Lt) * 4, 256);
+    w.off_jobs = o;     o += align_up((size_t)B * sizeof(SampleJob), 256);
+    w.total = o;
+    return w;
+}
+
+struct SampleWs {
+    size_t off_res_ticket, zero_bytes, off_jobs, off_tlse, off_dlse, off_chunks, total;
+};
+static SampleWs sample_ws_layout(int64_t B, int nchunks) {
+    SampleWs w;
+    size_t o = 0;
+    w.off_res_ticket = o; o += align_up((size_t)B * 4, 256);
+    w.zero_bytes = o;
+    w.off_jobs = o;       o += align_up((size_t)B * sizeof(SampleJob), 256);
+    w.off_tlse = o;       o += align_up((size_t)B * 8, 256);
+    w.off_dlse = o;       o += align_up((size_t)B * 8, 256);
+    w.off_chunks = o;     o += align_up((size_t)B * nchunks * 8, 256);
+    w.total = o;
+    return w;
+}
+
+template <typename DT>
+static int32_t launch_sample(VerifyArgs &a, SampleArgs &s, void *workspace, size_t workspace_bytes, cudaStream_t st) {
+    a.nchunks = nchunks_of<DT>(a.V);
+    const SampleWs w = sample_ws_layout(a.B, a.nchunks);
+    if (workspace_bytes < w.total) return DSP_ERR_WORKSPACE;
+    char *ws = reinterpret_cast<char *>(workspace);
+    a.res_ticket = reinterpret_cast<unsigned *>(ws + w.off_res_ticket);
+    a.jobs = reinterpret_cast<SampleJob *>(ws + w.off_jobs);
+    a.tlse64 = reinterpret_cast<double *>(ws + w.off_tlse);
+    s.tlse_g = a.tlse64;
+    s.dlse_g = reinterpret_cast<double *>(ws + w.off_dlse);
+    a.draft_lse64 = s.dlse_g;
+    s.jobs = a.jobs;
+    a.chunk_sums = reinterpret_cast<double *>(ws + w.off_chunks);
+    int rsl = (148 * 4 + a.B - 1) / a.B;
+    const int max_rsl = (a.nchunks + kWarps - 1) / kWarps;
+    if (rsl > max_rsl) rsl = max_rsl;
+    if (rsl < 1) rsl = 1;
+    a.chunks_per_slice = (a.nchunks + rsl - 1) / rsl;
+    a.res_slices = (a.nchunks + a.chunks_per_slice - 1) / a.chunks_per_slice;
+    DSP_CUDA_TRY(cudaMemsetAsync(ws, 0, w.zero_bytes, st));
+    sample_prepare_kernel<<<(unsigned)((a.B + 127) / 128), 128, 0, st>>>(s);
+    DSP_CUDA_TRY(cudaGetLastError());
+    residual_kernel<DT><<<(unsigned)(a.B * a.res_slices), kThreads, 0, st>>>(a);
+    DSP_CUDA_TRY(cudaGetLastError());
+    return DSP_OK;
+}
+
 }  // namespace dsp
 
 using namespace dsp;
@@ -617,6 +777,7 @@ int32_t dsp::verify_impl(const void *target_logits, int32_t dtype,
     a.all_greedy = all_greedy ? 1 : 0; a.mode = mode; a.u = u; a.eos_id = eos_id;
     a.accepted_len = accepted_len; a.next_token = next_token; a.ratio = ratio;
     a.tgt_argmax = tgt_argmax; a.tgt_lse = tgt_lse; a.row_status = row_status;
+    a.xt_probe = nullptr; a.job_trow = nullptr; a.job_drow = nullptr;
     return dtype == DSP_BF16 ? launch_verify<__nv_bfloat16>(a, workspace, workspace_bytes, st, phases)
                              : launch_verify<float>(a, workspace, workspace_bytes, st, phases);
 }
@@ -635,4 +796,112 @@ extern "C" int32_t dsp_verify(const void *target_logits, int32_t dtype,
                        dstride_l, path, path_slot, path_len, cand_logit, draft_lse64, KC, all_greedy, mode, u,
                        eos_id, accepted_len, next_token, ratio, tgt_argmax, tgt_lse, row_status, workspace,
                        workspace_bytes, reinterpret_cast<cudaStream_t>(stream), kVerifyStats | kVerifyDecide);
+}
+
+// ---- dsp_verify_merge / dsp_residual_sample: verification with a vocabulary-sharded target head ----
+
+extern "C" int32_t dsp_verify_merge_workspace_bytes(int32_t B, int32_t Lt, size_t *bytes) {
+    if (!bytes || B < 0 || Lt < 1) return DSP_ERR_INVALID_ARG;
+    *bytes = verify_merge_ws_layout(B > 0 ? B : 1, Lt).total;
+    return DSP_OK;
+}
+
+extern "C" int32_t dsp_verify_merge(int32_t G, const dsp_shard_sums *sums, const uint64_t *keys,
+                                    const uint32_t *shard_status,
+                                    int32_t B, int32_t L, int32_t Lt,
+                                    const int32_t *path, const int32_t *path_slot, const int32_t *path_len,
+                                    const float *cand_logit, const double *draft_lse64, int32_t KC,
+                                    int32_t all_greedy, const uint8_t *mode, const float *u, int32_t eos_id,
+                                    int32_t *accepted_len, int32_t *next_token, float *ratio,
+                                    int32_t *tgt_argmax, float *tgt_lse, double *tgt_lse64,
+                                    int32_t *job_trow, int32_t *job_drow, uint32_t *row_status,
+                                    void *workspace, size_t workspace_bytes, dsp_stream_t stream) {
+    if (G < 1 || B < 0 || L < 1 || Lt < L || Lt > L + 1) return DSP_ERR_INVALID_ARG;
+    if (L > DSP_MAX_L || G > 1024) return DSP_ERR_UNSUPPORTED;
+    if (B == 0) return DSP_OK;
+    if (!sums || !keys || !shard_status || !path || !path_len || !accepted_len || !next_token || !tgt_argmax ||
+        !tgt_lse64 || !job_trow || !job_drow || !row_status || !workspace)
+        return DSP_ERR_INVALID_ARG;
+    if (!all_greedy) {
+        if (!path_slot || !cand_logit || !draft_lse64 || !mode || !u) return DSP_ERR_INVALID_ARG;
+        if (KC < 1 || KC > DSP_MAX_K + 1) return DSP_ERR_UNSUPPORTED;
+    }
+    if ((reinterpret_cast<uintptr_t>(workspace) & 255) != 0) return DSP_ERR_INVALID_ARG;
+    const MergeWs w = verify_merge_ws_layout(B, Lt);
+    if (workspace_bytes < w.total) return DSP_ERR_WORKSPACE;
+    cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+    char *ws = reinterpret_cast<char *>(workspace);
+    DSP_CUDA_TRY(cudaMemsetAsync(ws, 0, w.zero_bytes, st));
+    TargetMergeArgs m;
+    m.G = G; m.B = B; m.Lt = Lt;
+    m.sums = sums;
+    m.keys = reinterpret_cast<const unsigned long long *>(keys);
+    m.shard_status = shard_status;
+    m.argmax = reinterpret_cast<int32_t *>(ws + w.off_argmax);
+    m.tlse64 = tgt_lse64;
+    m.xt = reinterpret_cast<float *>(ws + w.off_xt);
+    m.tgt_argmax = tgt_argmax;
+    m.tgt_lse = tgt_lse;
+    m.b_status = reinterpret_cast<unsigned *>(ws + w.off_b_status);
+    const long long nrows = (long long)B * Lt;
+    target_merge_kernel<<<(unsigned)((nrows + kWarps - 1) / kWarps), kThreads, 0, st>>>(m);
+    DSP_CUDA_TRY(cudaGetLastError());
+    VerifyArgs a = VerifyArgs();
+    a.B = B; a.L = L; a.Lt = Lt; a.V = 1;
+    a.path = path; a.path_slot = path_slot; a.path_len = path_len;
+    a.cand_logit = cand_logit; a.draft_lse64 = draft_lse64; a.KC = KC;
+    a.all_greedy = all_greedy ? 1 : 0; a.mode = mode; a.u = u; a.eos_id = eos_id;
+    a.accepted_len = accepted_len; a.next_token = next_token; a.ratio = ratio;
+    a.row_status = row_status;
+    a.argmax = m.argmax; a.tlse64 = tgt_lse64; a.xt_probe = m.xt;
+    a.b_status = m.b_status;
+    a.jobs = reinterpret_cast<SampleJob *>(ws + w.off_jobs);
+    a.job_trow = job_trow; a.job_drow = job_drow;
+    accept_kernel<float><<<(unsigned)((B + kWarps - 1) / kWarps), kThreads, 0, st>>>(a);
+    DSP_CUDA_TRY(cudaGetLastError());
+    return DSP_OK;
+}
+
+extern "C" int32_t dsp_residual_sample_workspace_bytes(int32_t B, int32_t V, int32_t dtype, size_t *bytes) {
+    if (!bytes || B < 0 || V < 1) return DSP_ERR_INVALID_ARG;
+    if (dtype != DSP_F32 && dtype != DSP_BF16) return DSP_ERR_UNSUPPORTED;
+    const int Bq = B > 0 ? B : 1;
+    *bytes = sample_ws_layout(Bq, dtype == DSP_BF16 ? nchunks_of<__nv_bfloat16>(V) : nchunks_of<float>(V)).total;
+    return DSP_OK;
+}
+
+extern "C" int32_t dsp_residual_sample(const void *target_rows, const void *draft_rows, int32_t dtype,
+                                       int32_t B, int32_t L, int32_t Lt, int32_t V,
+                                       int64_t tstride, int64_t dstride,
+                                       const int32_t *job_trow, const int32_t *job_drow,
+                                       const double *tgt_lse64, const double *draft_lse64,
+                                       const int32_t *tgt_argmax, const float *u,
+                                       int32_t *next_token, uint32_t *row_status,
+                                       void *workspace, size_t workspace_bytes, dsp_stream_t stream) {
+    if (B < 0 || L < 1 || Lt < L || Lt > L + 1 || V < 1) return DSP_ERR_INVALID_ARG;
+    if (dtype != DSP_F32 && dtype != DSP_BF16) return DSP_ERR_UNSUPPORTED;
+    if (V > (1 << 30)) return DSP_ERR_UNSUPPORTED;
+    if (B == 0) return DSP_OK;
+    if (!target_rows || !draft_rows || !job_trow || !job_drow || !tgt_lse64 || !draft_lse64 || !tgt_argmax || !u ||
+        !next_token || !row_status || !workspace)
+        return DSP_ERR_INVALID_ARG;
+    if (tstride < V || dstride < V) return DSP_ERR_INVALID_ARG;
+    if ((reinterpret_cast<uintptr_t>(workspace) & 255) != 0) return DSP_ERR_INVALID_ARG;
+    const size_t es = dtype == DSP_BF16 ? 2 : 4;
+    if (((reinterpret_cast<uintptr_t>(target_rows) | reinterpret_cast<uintptr_t>(draft_rows)) & (es - 1)) != 0)
+        return DSP_ERR_INVALID_ARG;
+    VerifyArgs a = VerifyArgs();
+    a.target = target_rows; a.draft = draft_rows;
+    a.B = B; a.L = 1; a.Lt = 1; a.V = V;               // the gathered arrays hold one row per batch row
+    a.tstride_b = tstride; a.tstride_l = tstride;
+    a.dstride_b = dstride; a.dstride_l = dstride;
+    a.next_token = next_token; a.row_status = row_status;
+    SampleArgs s;
+    s.B = B; s.L = L; s.Lt = Lt;
+    s.job_trow = job_trow; s.job_drow = job_drow;
+    s.tgt_lse64 = tgt_lse64; s.draft_lse64 = draft_lse64;
+    s.tgt_argmax = tgt_argmax; s.u = u;
+    cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+    return dtype == DSP_BF16 ? launch_sample<__nv_bfloat16>(a, s, workspace, workspace_bytes, st)
+                             : launch_sample<float>(a, s, workspace, workspace_bytes, st);
 }

@@ -385,6 +385,76 @@ def test_lattice_from_slices_flags_nonfinite_rows():
     assert out.row_status.cpu().tolist() == [0, dsp.ROW_NONFINITE_INPUT]
 
 
+def _sharded_verify(inp, lat, cps, cuts, eos_id, all_greedy):
+    """dsp_verify from vocabulary slices of the target: records per slice, merge, gathered rows, draw."""
+    target, draft = inp["target"], inp["draft"]
+    B, Lt, V = target.shape
+    L = draft.shape[1]
+    recs = [dsp.dsp_target_shard(target[:, :, lo:hi], lo, cps) for lo, hi in zip(cuts[:-1], cuts[1:])]
+    stack = lambda name: torch.stack([getattr(r, name) for r in recs], dim=0).contiguous()
+    ver = dsp.dsp_verify_merge(stack("sums"), stack("keys"), stack("status"), cps, None if all_greedy else lat,
+                               mode=None if all_greedy else inp["mode"], u=None if all_greedy else inp["u"],
+                               eos_id=eos_id, all_greedy=all_greedy)
+    if not all_greedy:
+        # what the all-gather of the named rows' slices leaves on every GPU: the whole rows, one per batch row
+        trow = ver.job_trow.long().clamp(min=0)
+        drow = ver.job_drow.long().clamp(min=0)
+        target_rows = torch.cat([target[:, :, lo:hi].reshape(B * Lt, hi - lo)[trow] for lo, hi in zip(cuts[:-1], cuts[1:])], dim=1)
+        draft_rows = torch.cat([draft[:, :, lo:hi].reshape(B * L, hi - lo)[drow] for lo, hi in zip(cuts[:-1], cuts[1:])], dim=1)
+        dsp.dsp_residual_sample(target_rows.contiguous(), draft_rows.contiguous(), ver, lat, inp["u"], L)
+    torch.cuda.synchronize()
+    return ver
+
+
+@pytest.mark.parametrize("cid,cuts", [(3, [0, 38016, 76032, 114048, 152064]), (4, [0, 16384, 50048]),
+                                      (1, [0, 8000, 16000, 24000, 32000]), (5, [0, 128000, 256000])])
+def test_verification_from_vocabulary_slices_of_the_target(cid, cuts):
+    w = wl.CONFIGS[cid].scaled(**SMALL[cid])
+    if cid == 4:
+        w = w.scaled(V=50048)
+    p = _params(w)
+    inp = wl.make_inputs(w, step=6, device=DEV)
+    whole = gpu_step(inp, **p)                             # the three unsharded calls, CPU copies
+    lat = dsp.dsp_lattice_build(inp["draft"], w.K, w.tau, w.eos_id)
+    cps = dsp.dsp_cps_search(lat, inp["prev_token"], inp["table"], W=w.W, lam=w.lam, eos_id=w.eos_id,
+                             table_log2=inp["table_log2"], hash_seed=inp["hash_seed"], V=w.V)
+    ver = _sharded_verify(inp, lat, cps, cuts, w.eos_id, p["all_greedy"])
+    assert torch.equal(ver.accepted_len.cpu(), whole.ver.accepted_len)
+    assert torch.equal(ver.tgt_argmax.cpu(), whole.ver.tgt_argmax)
+    assert torch.equal(ver.next_token.cpu(), whole.ver.next_token)
+    if not p["all_greedy"]:
+        stoch = inp["mode"].cpu() != 0
+        assert torch.allclose(ver.tgt_lse.cpu()[stoch], whole.ver.tgt_lse[stoch], atol=1e-5, rtol=0)
+        assert torch.allclose(ver.ratio.cpu(), whole.ver.ratio, atol=1e-5, rtol=1e-4)
+    # and against the oracle: the sharded verification in place of the unsharded one
+    cpu = lambda x: SimpleNamespace(**{k: (v.cpu() if isinstance(v, torch.Tensor) else v) for k, v in vars(x).items()})
+    g = SimpleNamespace(lat=whole.lat, cps=whole.cps, ver=cpu(ver))
+    g.lat.row_status = whole.lat.row_status | ver.row_status.cpu()
+    if not p["all_greedy"]:
+        greedy = inp["mode"].cpu() == 0
+        g.ver.tgt_lse[greedy] = float("nan")               # dsp_verify leaves these unset
+    check_step(g, inp, **p)
+
+
+def test_sharded_verification_with_a_bonus_row():
+    """Lt = L + 1 and a target that accepts everything: the draw comes from the extra row (no draft row)."""
+    B, L, V = 4, 5, 4096
+    inp = _to(wl.tiny_random(B, L, V, dtype=torch.bfloat16, seed=3))
+    extra = (inp["target"][:, :1].float() * 0.5).to(torch.bfloat16)
+    inp["target"] = torch.cat([inp["target"], extra], dim=1).contiguous()
+    inp["target"][:, :L] = inp["draft"]
+    p = dict(K=4, W=4, lam=1.0)
+    whole = gpu_step(inp, **p)
+    lat = dsp.dsp_lattice_build(inp["draft"], 4)
+    cps = dsp.dsp_cps_search(lat, inp["prev_token"], inp["table"], W=4, lam=1.0, table_log2=inp["table_log2"],
+                             hash_seed=inp["hash_seed"], V=V)
+    ver = _sharded_verify(inp, lat, cps, [0, 1024, 1032, 4096], -1, False)
+    stoch = inp["mode"].cpu() != 0
+    assert (ver.job_drow.cpu()[stoch] == -1).all() and (ver.job_trow.cpu()[~stoch] == -1).all()
+    assert torch.equal(ver.accepted_len.cpu(), whole.ver.accepted_len)
+    assert torch.equal(ver.next_token.cpu(), whole.ver.next_token) and (ver.next_token >= 0).all()
+
+
 # ---- the drafter's refinement step (Eq. 5) ----
 def _check_unmask(x, tokens, masked, n, ws=None):
     """One step on both sides from the same state; returns the new state (the GPU's)."""
