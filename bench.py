@@ -281,6 +281,38 @@ def time_proxies(w, st, sets, device, reps=50):
     return out
 
 
+def time_sharded(w, device, G=4, reps=40):
+    """One rank's share of the lattice of a drafter head sharded G ways over the vocabulary, on the
+    headline workload's logits: dsp_lattice_shard on a V/G slice and dsp_lattice_merge of G records
+    (the all-gather between them is not timed: one GPU here)."""
+    from paper_2510_02358_b200 import binding as dsp
+    x = input_sets(w, device, 9)[0]["draft"]
+    Vs = w.V // G // 8 * 8
+    dt = dsp.DSP_BF16 if w.dtype == torch.bfloat16 else dsp.DSP_F32
+    ws = dsp.alloc_workspace(dsp.dsp_shard_workspace_bytes(w.B, w.L, Vs, dt, w.K), device)
+    sl = x[:, :, :Vs]
+    rec = dsp.dsp_lattice_shard(sl, 0, w.K, w.eos_id, workspace=ws)
+    stack = lambda t: torch.stack([t] * G, dim=0).contiguous()
+    sums, keys, status = stack(rec.sums), stack(rec.keys), stack(rec.status)
+    out = dsp.lattice_outputs(w.B, w.L, w.K, w.eos_id, device)
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(3)]
+    ts, tm = 0.0, 0.0
+    for r in range(reps + 3):
+        ev[0].record()
+        dsp.dsp_lattice_shard(sl, 0, w.K, w.eos_id, out=rec, workspace=ws)
+        ev[1].record()
+        dsp.dsp_lattice_merge(sums, keys, status, w.V, w.K, w.tau, w.eos_id, out=out)
+        ev[2].record()
+        torch.cuda.synchronize()
+        if r >= 3:
+            ts += ev[0].elapsed_time(ev[1])
+            tm += ev[1].elapsed_time(ev[2])
+    nbytes = w.B * w.L * Vs * (2 if w.dtype == torch.bfloat16 else 4)
+    return {"G": G, "slice_V": Vs, "shard_ms": ts / reps, "merge_ms": tm / reps,
+            "slice_logits_gbs": nbytes / (ts / reps * 1e-3) / 1e9,
+            "record_bytes_per_row_and_slice": 24 + 8 * w.K, "workload": "draft logits of %s" % w.name}
+
+
 def time_unmask(w, device, reps=40):
     """The drafter's refinement step (dsp_unmask_step) on logits of the headline workload's shape:
     S = 1 (every position masked, one call) and S = 4 (four calls, a quarter of the block each;
@@ -540,6 +572,7 @@ def main():
                 torch.cuda.empty_cache()
         line["workloads"] = extras
         line["unmask_step"] = time_unmask(w, device)
+        line["vocab_sharded_lattice"] = time_sharded(w, device)
     print(json.dumps(line))
     if dist is not None:
         dist.destroy_process_group()
