@@ -148,6 +148,38 @@ def proxy_score(table, prev: int, cur: int, *, proxy_kind=0, table_log2=0, hash_
                                        C.c_uint32(hash_seed & 0xFFFFFFFF), C.c_int64(V), prev, cur))
 
 
+def beam_tree(beam_ids, path_len):
+    """Token tree of the beams [B,W,L]: node_token / node_parent / node_depth [B,W*L], beam_node [B,W,L], n_nodes [B]."""
+    beam_ids = _np(beam_ids, np.int32)
+    path_len = _np(path_len, np.int32)
+    B, W, L = beam_ids.shape
+    N = W * L
+    o = SimpleNamespace(node_token=np.empty((B, N), np.int32), node_parent=np.empty((B, N), np.int32),
+                        node_depth=np.empty((B, N), np.int32), beam_node=np.empty((B, W, L), np.int32),
+                        n_nodes=np.empty((B,), np.int32))
+    rc = lib().orc_beam_tree(_p(beam_ids), _p(path_len), B, W, L, _p(o.node_token), _p(o.node_parent),
+                             _p(o.node_depth), _p(o.beam_node), _p(o.n_nodes))
+    if rc != 0:
+        raise ValueError("orc_beam_tree: bad arguments")
+    return SimpleNamespace(**{k: torch.from_numpy(v) for k, v in vars(o).items()})
+
+
+def verify_tree(target: torch.Tensor, tree: SimpleNamespace, L: int):
+    """Greedy verification of the tree; target is [B, 1 + N, V] (row 0: after the prefix, row 1+n: after node n)."""
+    target = target.contiguous()
+    B, N1, V = target.shape
+    N = N1 - 1
+    o = SimpleNamespace(accepted_len=np.empty((B,), np.int32), accepted_node=np.empty((B, L), np.int32),
+                        next_token=np.empty((B,), np.int32), row_status=np.zeros((B,), np.uint32))
+    rc = lib().orc_verify_tree(_logits_ptr(target), _dtype_code(target), B, N, C.c_int64(V),
+                               _p(_np(tree.node_token, np.int32)), _p(_np(tree.node_parent, np.int32)),
+                               _p(_np(tree.n_nodes, np.int32)), L, _p(o.accepted_len), _p(o.accepted_node),
+                               _p(o.next_token), _p(o.row_status))
+    if rc != 0:
+        raise ValueError("orc_verify_tree: bad arguments")
+    return SimpleNamespace(**{k: torch.from_numpy(v) for k, v in vars(o).items()})
+
+
 def unmask_step(logits: torch.Tensor, tokens, masked, n_update: int):
     """One refinement step (Eq. 5, top-K by confidence); returns new tokens / masked and the per-position
     argmax, confidence (log-probability of the argmax, fp32), n_left and row_status."""

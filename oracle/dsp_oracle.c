@@ -646,6 +646,93 @@ int orc_unmask_step(const void *logits, int dtype, int B, int L, int64_t V, int 
 }
 
 /*
+ * Token tree of the surviving beams, for verifying several paths in one target
+ * pass (Sec. 2 names tree-based parallel verification as verifier-side
+ * engineering; the paper verifies the rank-0 path only).
+ * Beams that share a prefix share its nodes.  Nodes are numbered in the order
+ * (beam rank ascending, depth ascending) of their first use, so the rank-0 path
+ * is nodes 0 .. m-1.  node_parent is the node before it on its path (-1 at depth
+ * 0).  beam_node[b,w,i] = node of beam w at depth i (-1 where the beam has no
+ * token).  Unused node slots hold token -1, parent -1, depth -1.
+ */
+int orc_beam_tree(const int32_t *beam_ids, const int32_t *path_len, int B, int W, int L,
+                  int32_t *node_token, int32_t *node_parent, int32_t *node_depth,
+                  int32_t *beam_node, int32_t *n_nodes)
+{
+    if (B < 0 || W < 1 || L < 1) return -1;
+    const int N = W * L;
+    for (int b = 0; b < B; ++b) {
+        int32_t *tok = node_token + (int64_t)b * N, *par = node_parent + (int64_t)b * N;
+        int32_t *dep = node_depth + (int64_t)b * N, *bn = beam_node + (int64_t)b * N;
+        for (int n = 0; n < N; ++n) { tok[n] = -1; par[n] = -1; dep[n] = -1; bn[n] = -1; }
+        const int m = path_len[b] < 0 ? 0 : (path_len[b] > L ? L : path_len[b]);
+        int count = 0;
+        for (int w = 0; w < W; ++w) {
+            const int32_t *ids = beam_ids + ((int64_t)b * W + w) * L;
+            int parent = -1;
+            for (int i = 0; i < m; ++i) {
+                if (ids[i] < 0) break;                  /* this beam does not exist */
+                int found = -1;
+                for (int n = 0; n < count; ++n)         /* a child of `parent` with this token? */
+                    if (dep[n] == i && par[n] == parent && tok[n] == ids[i]) { found = n; break; }
+                if (found < 0) {
+                    found = count++;
+                    tok[found] = ids[i]; par[found] = parent; dep[found] = i;
+                }
+                bn[w * L + i] = found;
+                parent = found;
+            }
+        }
+        n_nodes[b] = count;
+    }
+    return 0;
+}
+
+/*
+ * Greedy verification of a token tree (the greedy rule of Sec. 4 applied along
+ * the tree): target row 0 is the distribution after the prefix, row 1+n the
+ * distribution after node n.  Starting at the root, the argmax (lowest id on
+ * ties) of the current row selects the child that carries that token; the walk
+ * ends where no child does.  accepted_len = nodes walked, accepted_node[b,i] =
+ * the i-th of them (-1 beyond), next_token = the argmax of the row the walk
+ * ended at (correction, or bonus after a leaf).
+ * target is [B, 1 + N, V] with N = W*L node slots; only rows of existing nodes
+ * are read.  A row with NaN / +inf or no finite logit that the walk reads flags
+ * the batch row.
+ */
+int orc_verify_tree(const void *target, int dtype, int B, int N, int64_t V,
+                    const int32_t *node_token, const int32_t *node_parent, const int32_t *n_nodes,
+                    int L, int32_t *accepted_len, int32_t *accepted_node, int32_t *next_token,
+                    uint32_t *row_status)
+{
+    if (B < 0 || N < 1 || V < 1 || L < 1) return -1;
+    const size_t es = dtype == 0 ? 4 : 2;
+    #pragma omp parallel for schedule(dynamic)
+    for (int b = 0; b < B; ++b) {
+        const int32_t *tok = node_token + (int64_t)b * N, *par = node_parent + (int64_t)b * N;
+        uint32_t status = 0;
+        int ctx = -1, acc = 0;                          /* node the walk stands on; -1 = root */
+        for (int i = 0; i < L; ++i) accepted_node[(int64_t)b * L + i] = -1;
+        int64_t am = 0;
+        for (;;) {
+            const char *row = (const char *)target + ((size_t)b * (size_t)(1 + N) + (size_t)(1 + ctx)) * (size_t)V * es;
+            if (row_stats(row, dtype, V, NULL, NULL, &am)) status |= ORC_NONFINITE_INPUT;
+            int child = -1;
+            for (int n = 0; n < n_nodes[b]; ++n)
+                if (par[n] == ctx && tok[n] == (int32_t)am) { child = n; break; }
+            if (child < 0 || acc >= L) break;
+            accepted_node[(int64_t)b * L + acc] = child;
+            ++acc;
+            ctx = child;
+        }
+        accepted_len[b] = acc;
+        next_token[b] = (int32_t)am;
+        if (row_status) row_status[b] = status;
+    }
+    return 0;
+}
+
+/*
  * Adaptive draft length (Sec. 3.3, Eq. 9-11; Alg. 1 init and stage 4).
  * state = { ema_gen, ema_acc, k }.  Init: both averages 0, k = k_max.
  * Update with the batch means of gen_len and accepted_len (batch 1 is the
