@@ -421,6 +421,46 @@ int32_t dsp_residual_sample(const void *target_rows, const void *draft_rows, int
                             void *workspace, size_t workspace_bytes, dsp_stream_t stream);
 
 /* -------------------------------------------------------------------------
+ * Several paths in one target pass  (Sec. 2 names tree-based parallel
+ * verification as verifier-side engineering; the paper verifies the rank-0
+ * path only -- this is the greedy rule of Sec. 4 applied along a token tree of
+ * the beams dsp_cps_search leaves in beam_ids).
+ *
+ * dsp_beam_tree: beams that share a prefix share its nodes.  N = W*L node slots
+ * per batch row; nodes are numbered in the order (beam rank, depth) of their
+ * first use, so the rank-0 path is nodes 0 .. m-1 (m = path_len[b]).
+ *   node_token / node_parent / node_depth int32 [B,N]: token, the node before
+ *     it on its path (-1 at depth 0), depth; -1 in unused slots;
+ *   beam_node int32 [B,W,L]: node of beam w at depth i, -1 where there is none;
+ *   n_nodes int32 [B].
+ * The caller runs the target model on the tree (tree attention) and supplies
+ * target_logits [B, 1+N, V]: row 0 = the distribution after the prefix, row
+ * 1+n = the distribution after node n (rows of unused slots are not read).
+ * dsp_verify_tree walks from the root: the argmax (lowest id on ties) of the
+ * current row picks the child that carries that token; the walk ends where no
+ * child does.  accepted_len [B] = nodes walked, accepted_node int32 [B,L] = the
+ * nodes in order (-1 beyond), next_token [B] = the argmax of the row where the
+ * walk ended (correction, or bonus after a leaf), tgt_argmax int32 [B,1+N]
+ * (-1 for unused rows), row_status (written): DSP_ROW_NONFINITE_INPUT if an
+ * existing row holds NaN / +inf or no finite logit, DSP_ROW_TIMEOUT.
+ * Stochastic tree verification is not provided.
+ * workspace: dsp_verify_tree_workspace_bytes(B, N, V, dtype), 256-byte aligned.
+ * Errors : INVALID_ARG, UNSUPPORTED (W > DSP_MAX_W, L > DSP_MAX_L,
+ *          N + 1 > DSP_MAX_L, dtype), WORKSPACE, CUDA.
+ */
+int32_t dsp_beam_tree(const int32_t *beam_ids, const int32_t *path_len, int32_t B, int32_t W, int32_t L,
+                      int32_t *node_token, int32_t *node_parent, int32_t *node_depth,
+                      int32_t *beam_node, int32_t *n_nodes, dsp_stream_t stream);
+int32_t dsp_verify_tree_workspace_bytes(int32_t B, int32_t N, int32_t V, int32_t dtype,
+                                        size_t *bytes /* host, out */);
+int32_t dsp_verify_tree(const void *target_logits, int32_t dtype, int32_t B, int32_t N, int32_t V,
+                        int64_t stride_b, int64_t stride_l,
+                        const int32_t *node_token, const int32_t *node_parent, const int32_t *n_nodes,
+                        int32_t L, int32_t *accepted_len, int32_t *accepted_node, int32_t *next_token,
+                        int32_t *tgt_argmax, uint32_t *row_status,
+                        void *workspace, size_t workspace_bytes, dsp_stream_t stream);
+
+/* -------------------------------------------------------------------------
  * Refinement step of the diffusion drafter  (Sec. 3.1, Eq. 5: iterative
  * refinement with the update set "top-K by confidence"; the paper's default
  * S = 1 needs a single call with n_update >= L, S > 1 is its ablation).

@@ -697,8 +697,8 @@ int orc_beam_tree(const int32_t *beam_ids, const int32_t *path_len, int B, int W
  * the i-th of them (-1 beyond), next_token = the argmax of the row the walk
  * ended at (correction, or bonus after a leaf).
  * target is [B, 1 + N, V] with N = W*L node slots; only rows of existing nodes
- * are read.  A row with NaN / +inf or no finite logit that the walk reads flags
- * the batch row.
+ * are read.  An existing row with NaN / +inf or no finite logit flags the batch
+ * row.
  */
 int orc_verify_tree(const void *target, int dtype, int B, int N, int64_t V,
                     const int32_t *node_token, const int32_t *node_parent, const int32_t *n_nodes,
@@ -714,9 +714,13 @@ int orc_verify_tree(const void *target, int dtype, int B, int N, int64_t V,
         int ctx = -1, acc = 0;                          /* node the walk stands on; -1 = root */
         for (int i = 0; i < L; ++i) accepted_node[(int64_t)b * L + i] = -1;
         int64_t am = 0;
+        for (int r = 0; r <= n_nodes[b]; ++r) {         /* every existing row is checked, as in orc_verify */
+            const char *row = (const char *)target + ((size_t)b * (size_t)(1 + N) + (size_t)r) * (size_t)V * es;
+            if (row_stats(row, dtype, V, NULL, NULL, &am)) status |= ORC_NONFINITE_INPUT;
+        }
         for (;;) {
             const char *row = (const char *)target + ((size_t)b * (size_t)(1 + N) + (size_t)(1 + ctx)) * (size_t)V * es;
-            if (row_stats(row, dtype, V, NULL, NULL, &am)) status |= ORC_NONFINITE_INPUT;
+            row_stats(row, dtype, V, NULL, NULL, &am);
             int child = -1;
             for (int n = 0; n < n_nodes[b]; ++n)
                 if (par[n] == ctx && tok[n] == (int32_t)am) { child = n; break; }

@@ -33,6 +33,7 @@ EXPORTS = ["dsp_strerror", "dsp_last_cuda_error", "dsp_version", "dsp_profile_ev
            "dsp_shard_workspace_bytes", "dsp_lattice_shard", "dsp_merge_workspace_bytes", "dsp_lattice_merge",
            "dsp_target_shard", "dsp_verify_merge_workspace_bytes", "dsp_verify_merge",
            "dsp_residual_sample_workspace_bytes", "dsp_residual_sample",
+           "dsp_beam_tree", "dsp_verify_tree_workspace_bytes", "dsp_verify_tree",
            "dsp_adl_init", "dsp_adl_update"]
 
 
@@ -453,6 +454,43 @@ def dsp_residual_sample(target_rows: torch.Tensor, draft_rows: torch.Tensor, ver
         C.c_int64(draft_rows.stride(0)), _ptr(ver.job_trow), _ptr(ver.job_drow), _ptr(ver.tgt_lse64),
         _ptr(lat.lse64), _ptr(ver.tgt_argmax), _ptr(u), _ptr(ver.next_token), _ptr(ver.row_status),
         _ptr(workspace), C.c_size_t(workspace.numel()), _stream(stream)))
+
+
+def dsp_beam_tree(cps: SimpleNamespace, stream=None) -> SimpleNamespace:
+    """Token tree of the beams in ``cps`` (beam_ids [B,W,L], path_len [B])."""
+    B, W, L = cps.beam_ids.shape
+    dev = cps.beam_ids.device
+    e = lambda shape: torch.empty(shape, dtype=torch.int32, device=dev)
+    out = SimpleNamespace(node_token=e((B, W * L)), node_parent=e((B, W * L)), node_depth=e((B, W * L)),
+                          beam_node=e((B, W, L)), n_nodes=e((B,)))
+    _check("dsp_beam_tree", lib().dsp_beam_tree(
+        _ptr(cps.beam_ids), _ptr(cps.path_len), B, W, L, _ptr(out.node_token), _ptr(out.node_parent),
+        _ptr(out.node_depth), _ptr(out.beam_node), _ptr(out.n_nodes), _stream(stream)))
+    return out
+
+
+def dsp_verify_tree(target: torch.Tensor, tree: SimpleNamespace, L: int, *,
+                    workspace: Optional[torch.Tensor] = None, stream=None) -> SimpleNamespace:
+    """Greedy verification of the token tree; ``target`` is [B, 1 + N, V]."""
+    B, N1, V, sb, sl = _logits3(target, "target")
+    N = N1 - 1
+    if tuple(tree.node_token.shape) != (B, N):
+        raise ValueError("target must have one row per node slot plus one")
+    dev = target.device
+    dt = _dtype(target)
+    e = lambda shape: torch.empty(shape, dtype=torch.int32, device=dev)
+    out = SimpleNamespace(accepted_len=e((B,)), accepted_node=e((B, L)), next_token=e((B,)),
+                          tgt_argmax=e((B, N1)), row_status=e((B,)))
+    n = C.c_size_t(0)
+    _check("dsp_verify_tree_workspace_bytes", lib().dsp_verify_tree_workspace_bytes(B, N, V, dt, C.byref(n)))
+    if workspace is None:
+        workspace = alloc_workspace(n.value, dev)
+    _check("dsp_verify_tree", lib().dsp_verify_tree(
+        _ptr(target), dt, B, N, V, C.c_int64(sb), C.c_int64(sl), _ptr(tree.node_token), _ptr(tree.node_parent),
+        _ptr(tree.n_nodes), L, _ptr(out.accepted_len), _ptr(out.accepted_node), _ptr(out.next_token),
+        _ptr(out.tgt_argmax), _ptr(out.row_status), _ptr(workspace), C.c_size_t(workspace.numel()),
+        _stream(stream)))
+    return out
 
 
 def gather_shard_records(rec: SimpleNamespace, group=None) -> SimpleNamespace:

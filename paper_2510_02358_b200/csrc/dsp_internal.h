@@ -28,4 +28,12 @@ int32_t lattice_build_impl(const void *draft_logits, int32_t dtype, int32_t B, i
                            float *lse, double *lse64, float *entropy, int32_t *gen_len, uint32_t *row_status,
                            void *workspace, size_t workspace_bytes, cudaStream_t st, cudaEvent_t after_scan);
 
+// dsp_unmask_step that also takes n_update = 0 (row statistics of the masked rows only, nothing
+// revealed): the per-row argmax of a chosen set of rows, used by the tree verification.
+int32_t unmask_impl(const void *logits, int32_t dtype, int32_t B, int32_t L, int32_t V,
+                    int64_t stride_b, int64_t stride_l, int32_t n_update,
+                    int32_t *tokens, uint8_t *masked, int32_t *argmax, float *confidence,
+                    int32_t *n_left, uint32_t *row_status,
+                    void *workspace, size_t workspace_bytes, cudaStream_t st);
+
 }  // namespace dsp

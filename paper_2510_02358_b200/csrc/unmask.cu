@@ -241,14 +241,14 @@ extern "C" int32_t dsp_unmask_workspace_bytes(int32_t B, int32_t L, int32_t V, i
     return DSP_OK;
 }
 
-extern "C" int32_t dsp_unmask_step(const void *logits, int32_t dtype, int32_t B, int32_t L, int32_t V,
-                                   int64_t stride_b, int64_t stride_l, int32_t n_update,
-                                   int32_t *tokens, uint8_t *masked, int32_t *argmax, float *confidence,
-                                   int32_t *n_left, uint32_t *row_status,
-                                   void *workspace, size_t workspace_bytes, dsp_stream_t stream) {
+int32_t dsp::unmask_impl(const void *logits, int32_t dtype, int32_t B, int32_t L, int32_t V,
+                         int64_t stride_b, int64_t stride_l, int32_t n_update,
+                         int32_t *tokens, uint8_t *masked, int32_t *argmax, float *confidence,
+                         int32_t *n_left, uint32_t *row_status,
+                         void *workspace, size_t workspace_bytes, cudaStream_t st) {
     const int32_t rc = check_unmask_shape(B, L, V, dtype);
     if (rc != DSP_OK) return rc;
-    if (n_update < 1) return DSP_ERR_INVALID_ARG;
+    if (n_update < 0) return DSP_ERR_INVALID_ARG;
     if (B == 0) return DSP_OK;
     if (!logits || !tokens || !masked || !argmax || !confidence || !n_left || !row_status || !workspace)
         return DSP_ERR_INVALID_ARG;
@@ -264,7 +264,16 @@ extern "C" int32_t dsp_unmask_step(const void *logits, int32_t dtype, int32_t B,
     a.n_update = n_update;
     a.tokens = tokens; a.masked = masked; a.argmax = argmax; a.confidence = confidence;
     a.n_left = n_left; a.row_status = row_status;
-    cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
     return dtype == DSP_BF16 ? launch_unmask<__nv_bfloat16>(a, workspace, workspace_bytes, st)
                              : launch_unmask<float>(a, workspace, workspace_bytes, st);
+}
+
+extern "C" int32_t dsp_unmask_step(const void *logits, int32_t dtype, int32_t B, int32_t L, int32_t V,
+                                   int64_t stride_b, int64_t stride_l, int32_t n_update,
+                                   int32_t *tokens, uint8_t *masked, int32_t *argmax, float *confidence,
+                                   int32_t *n_left, uint32_t *row_status,
+                                   void *workspace, size_t workspace_bytes, dsp_stream_t stream) {
+    if (n_update < 1) return DSP_ERR_INVALID_ARG;
+    return unmask_impl(logits, dtype, B, L, V, stride_b, stride_l, n_update, tokens, masked, argmax, confidence,
+                       n_left, row_status, workspace, workspace_bytes, reinterpret_cast<cudaStream_t>(stream));
 }

@@ -455,6 +455,48 @@ def test_sharded_verification_with_a_bonus_row():
     assert torch.equal(ver.next_token.cpu(), whole.ver.next_token) and (ver.next_token >= 0).all()
 
 
+# ---- several paths in one target pass: the beams as a token tree, verified greedily ----
+@pytest.mark.parametrize("B,L,V,K,W,dtype", [
+    (3, 6, 32000, 4, 8, torch.float32),
+    (2, 8, 152064, 8, 16, torch.bfloat16),
+    (4, 5, 50021, 3, 4, torch.bfloat16),     # rows that are not 16-byte aligned
+    (2, 12, 4096, 2, 1, torch.float32),      # one beam: a chain
+])
+def test_beam_tree_and_its_greedy_verification(B, L, V, K, W, dtype):
+    inp = _to(wl.tiny_random(B, L, V, dtype=dtype, seed=L + W))
+    lat = dsp.dsp_lattice_build(inp["draft"], K)
+    cps = dsp.dsp_cps_search(lat, inp["prev_token"], inp["table"], W=W, lam=0.5, table_log2=inp["table_log2"],
+                             hash_seed=inp["hash_seed"], V=V)
+    tree = dsp.dsp_beam_tree(cps)
+    torch.cuda.synchronize()
+    ot = oracle.beam_tree(cps.beam_ids.cpu(), cps.path_len.cpu())
+    for name in ("node_token", "node_parent", "node_depth", "beam_node", "n_nodes"):
+        assert torch.equal(getattr(tree, name).cpu(), getattr(ot, name)), name
+    assert int(ot.n_nodes.max()) > L or W == 1              # the beams do branch
+    # target rows: noise plus a push towards one child's token at every existing context, so walks go deep
+    N = W * L
+    g = torch.Generator().manual_seed(5)
+    target = torch.randn((B, 1 + N, V), generator=g)
+    for b in range(B):
+        for n in range(int(ot.n_nodes[b])):
+            if (n * 7 + b) % 3:                              # two contexts in three favour a child
+                target[b, 1 + int(ot.node_parent[b, n]), int(ot.node_token[b, n])] += 9.0
+        target[b, 1 + int(ot.n_nodes[b]):] = float("nan")    # rows of unused slots must not matter
+    target = target.to(dtype)
+    out = dsp.dsp_verify_tree(target.to(DEV), tree, L)
+    torch.cuda.synchronize()
+    o = oracle.verify_tree(target, ot, L)
+    assert (o.row_status == 0).all() and (out.row_status.cpu() == 0).all()
+    for name in ("accepted_len", "accepted_node", "next_token"):
+        assert torch.equal(getattr(out, name).cpu(), getattr(o, name)), name
+    assert int(o.accepted_len.max()) >= 2
+    target[0, 1, 5] = float("nan")                           # an existing row goes bad: the batch row is flagged
+    out = dsp.dsp_verify_tree(target.to(DEV), tree, L)
+    o = oracle.verify_tree(target, ot, L)
+    torch.cuda.synchronize()
+    assert (out.row_status.cpu() != 0).tolist() == (o.row_status != 0).tolist() == [True] + [False] * (B - 1)
+
+
 # ---- the drafter's refinement step (Eq. 5) ----
 def _check_unmask(x, tokens, masked, n, ws=None):
     """One step on both sides from the same state; returns the new state (the GPU's)."""
