@@ -14,6 +14,12 @@ workload on its own rows (weak scaling, no collective on the data path); the
 time is the maximum over ranks and the value the steps all ranks completed per
 second.
 
+Beside the contract's keys the line carries: per-stage times and logits GB/s
+(as fractions of the nominal 8 TB/s, of the measured copy bandwidth and of
+``read_probe``, a read-only pass over the same logits timed in the same run),
+the other four workloads, and ``parity``: the timed binary's outputs on a timed
+input set compared with the oracle on sampled batch rows, near-ties counted.
+
 --impl reference times the CPU oracle (plain C, as it stands) on a bounded
 sample of the same workload on this machine's host cores.
 """
@@ -436,6 +442,55 @@ def cpu_baseline(w, inp, budget_s=12.0):
                        % (rows, w.B, n, total))
 
 
+def parity_recheck(w, st, inp, max_rows):
+    """The timed binary against the oracle inside the benchmark run: one more step on a timed
+    input set, then up to ``max_rows`` evenly spaced batch rows compared field by field by the
+    same comparison the tests use (integers exact, log-probabilities within 1e-3, near-ties of
+    the floating-point decisions counted).  Part of the CPU-baseline leg: it runs the oracle."""
+    from types import SimpleNamespace
+    tdir = os.path.join(os.path.dirname(os.path.abspath(__file__)), "tests")
+    if tdir not in sys.path:
+        sys.path.insert(0, tdir)
+    from parity import check_step
+    st.step(inp)
+    torch.cuda.synchronize()
+    n = min(w.B, max_rows)
+    rows = sorted({round(i * (w.B - 1) / max(1, n - 1)) for i in range(n)})
+    idx = torch.as_tensor(rows, dtype=torch.long, device=inp["draft"].device)
+    take = lambda v: v[idx].cpu() if isinstance(v, torch.Tensor) and v.dim() >= 1 and v.shape[0] == w.B else v
+    small = {k: (v if k == "table" else take(v)) for k, v in inp.items()}
+    g = SimpleNamespace(**{name: SimpleNamespace(**{k: take(v) for k, v in vars(getattr(st, name)).items()})
+                           for name in ("lat", "cps", "ver")})
+    out = {"rows_checked": len(rows), "of_rows": w.B}
+    try:
+        rep = check_step(g, small, K=w.K, W=w.W, tau=w.tau, lam=w.lam, eos_id=w.eos_id,
+                         all_greedy=w.verify == "greedy")
+        out.update(status="ok", near_tau=rep["near_tau"], near_accept=rep["near_accept"],
+                   near_token=rep["near_token"], max_abs_err=rep["max_err"])
+    except AssertionError as e:
+        out.update(status="FAILED", detail=str(e)[:300])
+    return out
+
+
+def time_read_probe(sets, device, reps=40):
+    """Read bandwidth of this GPU on the timed logits themselves: dsp_read_probe (a kernel that only
+    reads, coalesced 128-bit loads) over the draft tensors of the input sets in turn."""
+    from paper_2510_02358_b200 import binding as dsp
+    sink = torch.zeros(1, dtype=torch.int32, device=device)
+    bufs = [s["draft"] for s in sets] + ([s["target"] for s in sets] if len(sets) == 1 else [])
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    for r in range(reps + 3):
+        if r == 3:
+            e0.record()
+        dsp.dsp_read_probe(bufs[r % len(bufs)], sink)
+    e1.record()
+    torch.cuda.synchronize()
+    nbytes = bufs[0].numel() * bufs[0].element_size()
+    us = e0.elapsed_time(e1) / reps * 1e3
+    return {"gbs": nbytes / us / 1e3, "us_per_launch": us, "bytes_per_launch": nbytes,
+            "note": "dsp_read_probe over the draft logits of the timed input sets, back to back launches"}
+
+
 def run_reference(args, rank, world):
     if rank != 0:
         return
@@ -513,6 +568,7 @@ def main():
         return
 
     peak, peak_kind = measured_peak()
+    probe = time_read_probe(sets, device)
     tensor_bytes = w.logits_bytes
     gbs_lat = tensor_bytes / (m["ms_lattice"] * 1e-3) / 1e9
     gbs_ver = tensor_bytes / (m["ms_verify"] * 1e-3) / 1e9
@@ -528,7 +584,8 @@ def main():
                    "tau": w.tau, "verify": w.verify, "parallelism": "batch rows sharded, no collective",
                    "l2": "inputs larger than L2" if m["sets"] == 1 else "rotating %d input sets" % m["sets"]},
         "logits_gbs": {"lattice_build": gbs_lat, "verify": gbs_ver, "lattice_plus_verify": gbs_both,
-                       "frac_of_8000": gbs_both / 8000.0, "frac_of_%s_copy_peak" % peak_kind: gbs_both / peak},
+                       "frac_of_8000": gbs_both / 8000.0, "frac_of_%s_copy_peak" % peak_kind: gbs_both / peak,
+                       "frac_of_read_probe": gbs_both / probe["gbs"]},
         "stage_ms": {"lattice_build": m["ms_lattice"], "cps_search": m["ms_cps"], "verify": m["ms_verify"],
                      "note": "the three calls one after the other; `value` times dsp_draft_verify_step, "
                              "which overlaps the target statistics with the path search"},
@@ -540,13 +597,17 @@ def main():
                      "peak_kind": "%s copy bandwidth" % peak_kind, "unit": "GB/s", "frac": gbs_scan / peak,
                      "traffic": NCU_TRAFFIC_BYTES.get(w.cid),
                      "algorithmic_bytes_per_launch": tensor_bytes,
-                     "launch_us": m["ms_lattice_scan"] * 1e3, "launches_timed": m["scan_samples"]},
+                     "launch_us": m["ms_lattice_scan"] * 1e3, "launches_timed": m["scan_samples"],
+                     "frac_of_read_probe": gbs_scan / probe["gbs"]},
+        "read_probe": probe,
+        "row_steps_per_s": whole_job_steps_per_s(world, args.steps, ms) * w.B,
         "e2e": e2e,
         "gpu_launches": m["kernels_per_step"] * args.steps,
         "clocks": clocks,
     }
     if not args.no_extras and world == 1:
         line["cpu_baseline"] = cpu_baseline(w, sets[0])
+        line["parity"] = parity_recheck(w, st, sets[0], 16)
         line["cps_proxies_ms"] = time_proxies(w, st, sets, device)
         extras = {}
         del st, sets
@@ -567,7 +628,8 @@ def main():
                                  "verify": mm["ms_verify"]},
                     "logits_gbs": 2 * tb / ((mm["ms_lattice"] + mm["ms_verify"]) * 1e-3) / 1e9,
                     "frac_of_8000": 2 * tb / ((mm["ms_lattice"] + mm["ms_verify"]) * 1e-3) / 1e9 / 8000.0,
-                    "input_sets": mm["sets"], "mean_accepted_len": mm["mean_accepted_len"]}
+                    "input_sets": mm["sets"], "mean_accepted_len": mm["mean_accepted_len"],
+                    "parity": parity_recheck(wv, s2, i2[0], 4 if cid == 5 else 16)}
                 del s2, i2
                 torch.cuda.empty_cache()
         line["workloads"] = extras

@@ -88,6 +88,16 @@ int32_t dsp_version(void);                  /* host; ABI version, currently 1 */
  * Errors: INVALID_ARG (unknown point, or only one of the two events given). */
 int32_t dsp_profile_events(int32_t point, void *start, void *stop);
 
+/* Measurement aid (no counterpart in the paper): a kernel that only reads `bytes` bytes (rounded
+ * down to a multiple of 16) of device memory at `buffer` (device, 16-byte aligned) once, with
+ * coalesced 128-bit loads, and keeps nothing.  Timed by the caller with events on `stream`, it
+ * gives the read bandwidth this GPU reaches on a buffer of that size: the ceiling for the passes
+ * over the logits, which read and hardly write.  `sink` (device, one uint32, caller-owned) is
+ * written only if the folded data equals one fixed value; its content means nothing.
+ * Enqueues on `stream` and returns.  Errors: INVALID_ARG (null or misaligned pointer,
+ * bytes < 16), UNSUPPORTED (more than 2^31 - 1 pieces of 16 KB), CUDA. */
+int32_t dsp_read_probe(const void *buffer, size_t bytes, uint32_t *sink, dsp_stream_t stream);
+
 /* -------------------------------------------------------------------------
  * Lattice build  (Sec. 3.2 "Lattice and pruning", Eq. 7; Alg. 1 stage 1;
  *                 the generation-length signal of Eq. 9)

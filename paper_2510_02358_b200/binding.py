@@ -26,7 +26,7 @@ ROW_NONFINITE_INPUT, ROW_ZERO_RESIDUAL, ROW_NO_BONUS_ROW, ROW_EOS_ACCEPTED, ROW_
 ROW_TIMEOUT = 32
 DSP_MAX_K, DSP_MAX_W, DSP_MAX_L = 32, 32, 1024
 
-EXPORTS = ["dsp_strerror", "dsp_last_cuda_error", "dsp_version", "dsp_profile_events", "dsp_lattice_workspace_bytes",
+EXPORTS = ["dsp_strerror", "dsp_last_cuda_error", "dsp_version", "dsp_profile_events", "dsp_read_probe", "dsp_lattice_workspace_bytes",
            "dsp_lattice_build", "dsp_lattice_build_static", "dsp_cps_search", "dsp_verify_workspace_bytes", "dsp_verify", "dsp_draft_verify_step",
            "dsp_step_graph_create", "dsp_step_graph_launch", "dsp_step_graph_destroy",
            "dsp_unmask_workspace_bytes", "dsp_unmask_step",
@@ -115,6 +115,15 @@ def dsp_profile_events(point: int, start: Optional[torch.cuda.Event], stop: Opti
     The events must have been recorded once before, so that torch has created them."""
     h = lambda e: C.c_void_p(0 if e is None else e.cuda_event)
     _check("dsp_profile_events", lib().dsp_profile_events(point, h(start), h(stop)))
+
+
+def dsp_read_probe(buffer: torch.Tensor, sink: torch.Tensor) -> None:
+    """Enqueue one read-only pass over ``buffer`` (contiguous CUDA tensor) on the current stream;
+    ``sink`` is a CUDA tensor with at least 4 bytes that the kernel may write."""
+    if not (buffer.is_cuda and buffer.is_contiguous() and sink.is_cuda and sink.numel() * sink.element_size() >= 4):
+        raise ValueError("buffer must be a contiguous CUDA tensor and sink a CUDA tensor of at least 4 bytes")
+    _check("dsp_read_probe", lib().dsp_read_probe(_ptr(buffer), C.c_size_t(buffer.numel() * buffer.element_size()),
+                                                   _ptr(sink), _stream(None)))
 
 
 def dsp_lattice_workspace_bytes(B: int, L: int, V: int, dtype: int, K_max: int) -> int:

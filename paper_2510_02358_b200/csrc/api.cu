@@ -17,6 +17,41 @@ extern "C" int32_t dsp_profile_events(int32_t point, void *start, void *stop) {
     return DSP_OK;
 }
 
+// Read-only streaming probe: every thread of a CTA takes four 128-bit vectors of one 16 KB piece
+// (coalesced, read-only path, lines not kept in L1) and folds them into one word that is stored
+// only if it equals a value the data never produces, so the loads cannot be dropped.
+namespace dsp {
+constexpr int kProbeVpt = 4;
+__global__ void __launch_bounds__(kThreads) read_probe_kernel(const uint4 *p, unsigned long long nvec,
+                                                              uint32_t *sink) {
+    const unsigned long long base = (unsigned long long)blockIdx.x * (kThreads * kProbeVpt) + threadIdx.x;
+    uint4 v[kProbeVpt];
+#pragma unroll
+    for (int j = 0; j < kProbeVpt; ++j) {
+        const unsigned long long i = base + (unsigned long long)j * kThreads;
+        v[j] = i < nvec ? ldg_stream(p + i) : make_uint4(0u, 0u, 0u, 0u);
+    }
+    uint32_t acc = 0u;
+#pragma unroll
+    for (int j = 0; j < kProbeVpt; ++j) acc += (v[j].x ^ v[j].y) + (v[j].z ^ v[j].w);
+    if (acc == 0x9E3779B1u && sink) *sink = acc;
+}
+}  // namespace dsp
+
+extern "C" int32_t dsp_read_probe(const void *buffer, size_t bytes, uint32_t *sink, dsp_stream_t stream) {
+    using namespace dsp;
+    if (!buffer || !sink || bytes < 16) return DSP_ERR_INVALID_ARG;
+    if ((reinterpret_cast<uintptr_t>(buffer) & 15) != 0) return DSP_ERR_INVALID_ARG;
+    const unsigned long long nvec = bytes / 16;
+    const unsigned long long per_cta = (unsigned long long)kThreads * kProbeVpt;
+    const unsigned long long nblocks = (nvec + per_cta - 1) / per_cta;
+    if (nblocks > 0x7FFFFFFFull) return DSP_ERR_UNSUPPORTED;
+    read_probe_kernel<<<(unsigned)nblocks, kThreads, 0, reinterpret_cast<cudaStream_t>(stream)>>>(
+        reinterpret_cast<const uint4 *>(buffer), nvec, sink);
+    DSP_CUDA_TRY(cudaGetLastError());
+    return DSP_OK;
+}
+
 extern "C" const char *dsp_strerror(int32_t status) {
     switch (status) {
         case DSP_OK: return "ok";
