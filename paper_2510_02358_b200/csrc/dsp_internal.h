@@ -21,12 +21,25 @@ int32_t verify_impl(const void *target_logits, int32_t dtype, int32_t B, int32_t
                     uint32_t *row_status, void *workspace, size_t workspace_bytes, cudaStream_t st, int phases);
 
 // dsp_lattice_build that also records `after_scan` (if not null) on the stream once the pass over
-// the draft logits has been enqueued: what follows it in the call no longer reads them.
+// the draft logits has been enqueued: what follows it in the call no longer reads them.  With
+// `rows_stream` (needs `after_scan`) everything after that pass is enqueued on `rows_stream`
+// instead, which waits for `after_scan`: when the call returns, `rows_stream` carries the rest
+// of the build and `st` is free for work that does not need the lattice.
 int32_t lattice_build_impl(const void *draft_logits, int32_t dtype, int32_t B, int32_t L, int32_t V,
                            int64_t stride_b, int64_t stride_l, int32_t K_max, float tau, int32_t eos_id,
                            int32_t *cand_id, float *cand_logit, float *cand_logp, int32_t *cand_count,
                            float *lse, double *lse64, float *entropy, int32_t *gen_len, uint32_t *row_status,
-                           void *workspace, size_t workspace_bytes, cudaStream_t st, cudaEvent_t after_scan);
+                           void *workspace, size_t workspace_bytes, cudaStream_t st, cudaEvent_t after_scan,
+                           cudaStream_t rows_stream);
+
+// dsp_cps_search with a choice of SM sharing: with `whole_sm` every CTA of the search asks for
+// enough shared memory to keep the CTAs of a streaming kernel off its SM.
+int32_t cps_search_impl(const int32_t *cand_id, const float *cand_logit, const double *lse64,
+                        const int32_t *cand_count, int32_t B, int32_t L, int32_t KC, const int32_t *prev_token,
+                        int32_t proxy_kind, const float *proxy_table, int32_t table_log2, uint32_t hash_seed,
+                        int32_t V, int32_t W, float lambda, int32_t eos_id, int32_t *path, int32_t *path_slot,
+                        int32_t *path_len, float *path_score, int32_t *beam_ids, float *beam_score,
+                        float *beam_cum, uint32_t *row_status, cudaStream_t stream, bool whole_sm);
 
 // dsp_unmask_step that also takes n_update = 0 (row statistics of the masked rows only, nothing
 // revealed): the per-row argmax of a chosen set of rows, used by the tree verification.

@@ -229,7 +229,7 @@ __global__ void __launch_bounds__(kThreads) lattice_rows_kernel(const LatticeArg
 
 template <typename DT>
 static int32_t launch_lattice(LatticeArgs &a, void *workspace, size_t workspace_bytes, cudaStream_t st,
-                              cudaEvent_t after_scan) {
+                              cudaEvent_t after_scan, cudaStream_t rows_stream) {
     const long long nrows = (long long)a.B * a.L;
     const SlicePlan plan = plan_slices<DT>(nrows, a.V, kTargetCtas);
     a.nslices = plan.nslices;
@@ -257,12 +257,23 @@ static int32_t launch_lattice(LatticeArgs &a, void *workspace, size_t workspace_
         lattice_scan_kernel<DT><<<(unsigned)nblocks, kThreads, kRingBytes, st>>>(a);
         DSP_CUDA_TRY(cudaGetLastError());
         if (pe.stop) DSP_CUDA_TRY(cudaEventRecord(pe.stop, st));
-        if (after_scan) { DSP_CUDA_TRY(cudaEventRecord(after_scan, st)); after_scan = nullptr; }
-        lattice_rows_kernel<DT><<<(unsigned)((nrows + kRowWarps - 1) / kRowWarps), kThreads, 0, st>>>(a);
+        cudaStream_t rs = st;
+        if (after_scan) {
+            DSP_CUDA_TRY(cudaEventRecord(after_scan, st));
+            if (rows_stream) {                            // pass 2 follows the scan on the other stream
+                DSP_CUDA_TRY(cudaStreamWaitEvent(rows_stream, after_scan, 0));
+                rs = rows_stream;
+            }
+            after_scan = nullptr;
+        }
+        lattice_rows_kernel<DT><<<(unsigned)((nrows + kRowWarps - 1) / kRowWarps), kThreads, 0, rs>>>(a);
     } else {
         lattice_kernel<DT><<<(unsigned)nblocks, kThreads, 0, st>>>(a);
     }
-    if (after_scan) DSP_CUDA_TRY(cudaEventRecord(after_scan, st));
+    if (after_scan) {
+        DSP_CUDA_TRY(cudaEventRecord(after_scan, st));
+        if (rows_stream) DSP_CUDA_TRY(cudaStreamWaitEvent(rows_stream, after_scan, 0));
+    }
     DSP_CUDA_TRY(cudaGetLastError());
     return DSP_OK;
 }
@@ -304,7 +315,8 @@ int32_t dsp::lattice_build_impl(const void *draft_logits, int32_t dtype,
                                 int32_t *cand_id, float *cand_logit, float *cand_logp,
                                 int32_t *cand_count, float *lse, double *lse64, float *entropy,
                                 int32_t *gen_len, uint32_t *row_status,
-                                void *workspace, size_t workspace_bytes, cudaStream_t st, cudaEvent_t after_scan) {
+                                void *workspace, size_t workspace_bytes, cudaStream_t st, cudaEvent_t after_scan,
+                                cudaStream_t rows_stream) {
     const int32_t rc = check_lattice_shape(B, L, V, dtype, K_max);
     if (rc != DSP_OK) return rc;
     if (B == 0) return DSP_OK;
@@ -330,8 +342,8 @@ int32_t dsp::lattice_build_impl(const void *draft_logits, int32_t dtype,
     a.cand_id = cand_id; a.cand_logit = cand_logit; a.cand_logp = cand_logp;
     a.cand_count = cand_count; a.lse = lse; a.lse64 = lse64; a.entropy = entropy;
     a.gen_len = gen_len; a.row_status = row_status;
-    return dtype == DSP_BF16 ? launch_lattice<__nv_bfloat16>(a, workspace, workspace_bytes, st, after_scan)
-                             : launch_lattice<float>(a, workspace, workspace_bytes, st, after_scan);
+    return dtype == DSP_BF16 ? launch_lattice<__nv_bfloat16>(a, workspace, workspace_bytes, st, after_scan, rows_stream)
+                             : launch_lattice<float>(a, workspace, workspace_bytes, st, after_scan, rows_stream);
 }
 
 extern "C" int32_t dsp_lattice_build(const void *draft_logits, int32_t dtype,
@@ -344,7 +356,7 @@ extern "C" int32_t dsp_lattice_build(const void *draft_logits, int32_t dtype,
                                      void *workspace, size_t workspace_bytes, dsp_stream_t stream) {
     return lattice_build_impl(draft_logits, dtype, B, L, V, stride_b, stride_l, K_max, tau, eos_id, cand_id,
                               cand_logit, cand_logp, cand_count, lse, lse64, entropy, gen_len, row_status,
-                              workspace, workspace_bytes, reinterpret_cast<cudaStream_t>(stream), nullptr);
+                              workspace, workspace_bytes, reinterpret_cast<cudaStream_t>(stream), nullptr, nullptr);
 }
 
 // ---- dsp_lattice_build_static: the same build for callers that cannot allocate ----------------

@@ -2,11 +2,15 @@
 //
 // Same kernels and results as dsp_lattice_build, dsp_cps_search and dsp_verify called one after
 // the other.  What the single call adds is overlap: the statistics of the target rows (argmax,
-// log-sum-exp) need only the target logits, so they run on a second stream beside the lattice's
-// finish and the path search, which are short, latency-bound kernels that leave HBM idle.  The
-// target pass starts when the pass over the draft logits has been enqueued and completed (the
-// two would only share the memory bandwidth); the decisions (acceptance scan, residual draw)
-// wait for both sides.
+// log-sum-exp) need only the target logits, so the pass over the target logits runs beside the
+// lattice's finish and the path search, which are short, latency-bound kernels that leave HBM
+// idle; the decisions (acceptance scan, residual draw) wait for both sides.  The two sides run on
+// the caller's stream and on a stream of the library.  When the passes are long (their grid is
+// several times what the SMs hold at once) the library's stream, which has the highest priority
+// the device offers, takes the lattice's finish and the search: their few CTAs get the next free
+// places on the SMs instead of queueing behind the target pass's grid, and the search keeps its
+// SMs to itself (see cps_search_impl), because sharing one with streaming CTAs makes it 2.5 times
+// slower.
 #include <mutex>
 
 #include "dsp_common.cuh"
@@ -15,6 +19,12 @@
 namespace {
 
 constexpr int kMaxDevices = 64;
+// Target logits from which the pass over them counts as long: its grid is then several times
+// what the SMs hold at once, and a kernel launched behind it waits for most of the pass.
+constexpr long long kLongPassBytes = 400ll << 20;
+// Beside a long pass the search keeps its SMs to itself while it (one CTA per batch row) takes at
+// most half of a B200's 148 SMs; with more rows it shares them.
+constexpr int kWholeSmMaxCtas = 74;
 struct SideStream {
     cudaStream_t stream = nullptr;
     cudaEvent_t fork = nullptr, join = nullptr;
@@ -30,7 +40,9 @@ int32_t side_stream(SideStream **out) {
     std::lock_guard<std::mutex> lock(g_side_mutex);
     SideStream &s = g_side[dev];
     if (!s.stream) {
-        DSP_CUDA_TRY(cudaStreamCreateWithFlags(&s.stream, cudaStreamNonBlocking));
+        int least = 0, greatest = 0;                     // numerically lower = higher priority
+        DSP_CUDA_TRY(cudaDeviceGetStreamPriorityRange(&least, &greatest));
+        DSP_CUDA_TRY(cudaStreamCreateWithPriority(&s.stream, cudaStreamNonBlocking, greatest));
         DSP_CUDA_TRY(cudaEventCreateWithFlags(&s.fork, cudaEventDisableTiming));
         DSP_CUDA_TRY(cudaEventCreateWithFlags(&s.join, cudaEventDisableTiming));
     }
@@ -64,26 +76,44 @@ extern "C" int32_t dsp_draft_verify_step(
     int32_t rc = side_stream(&side);
     if (rc != DSP_OK) return rc;
 
-    // stage 1 on the caller's stream; `fork` marks the end of the pass over the draft logits
-    rc = lattice_build_impl(draft_logits, dtype, B, L, V, dstride_b, dstride_l, K_max, tau, eos_id, cand_id,
-                            cand_logit, cand_logp, cand_count, lse, lse64, entropy, gen_len, row_status,
-                            lattice_workspace, lattice_workspace_bytes, st, side->fork);
-    if (rc != DSP_OK) return rc;
-    // target statistics on the second stream from that point on
-    DSP_CUDA_TRY(cudaStreamWaitEvent(side->stream, side->fork, 0));
-    rc = verify_impl(target_logits, dtype, B, L, Lt, V, tstride_b, tstride_l, draft_logits, dstride_b, dstride_l,
-                     path, path_slot, path_len, cand_logit, lse64, KC, all_greedy, mode, u, eos_id, accepted_len,
-                     next_token, ratio, tgt_argmax, tgt_lse, row_status, verify_workspace, verify_workspace_bytes,
-                     side->stream, kVerifyStats);
-    const cudaError_t e_rec = cudaEventRecord(side->join, side->stream);
-    // stage 2 on the caller's stream, beside the target statistics
+    const long long target_bytes = (long long)B * Lt * V * (dtype == DSP_BF16 ? 2 : 4);
+    const bool long_pass = target_bytes >= kLongPassBytes;
+    const bool whole_sm = long_pass && B <= kWholeSmMaxCtas;
+    auto stats = [&](cudaStream_t s) {
+        return verify_impl(target_logits, dtype, B, L, Lt, V, tstride_b, tstride_l, draft_logits, dstride_b,
+                           dstride_l, path, path_slot, path_len, cand_logit, lse64, KC, all_greedy, mode, u, eos_id,
+                           accepted_len, next_token, ratio, tgt_argmax, tgt_lse, row_status, verify_workspace,
+                           verify_workspace_bytes, s, kVerifyStats);
+    };
+    auto search = [&](cudaStream_t s) {
+        return cps_search_impl(cand_id, cand_logit, lse64, cand_count, B, L, KC, prev_token, proxy_kind,
+                               proxy_table, table_log2, hash_seed, V, W, lambda, eos_id, path, path_slot, path_len,
+                               path_score, beam_ids, beam_score, beam_cum, row_status, s, whole_sm);
+    };
     int32_t rc2 = DSP_OK;
-    if (rc == DSP_OK && e_rec == cudaSuccess)
-        rc2 = dsp_cps_search(cand_id, cand_logit, lse64, cand_count, B, L, KC, prev_token, proxy_kind,
-                             proxy_table, table_log2, hash_seed, V, W, lambda, eos_id, path, path_slot, path_len,
-                             path_score, beam_ids, beam_score, beam_cum, row_status, stream);
+    if (long_pass) {
+        // The pass over the target logits follows the pass over the draft logits on the caller's
+        // stream; the lattice's finish and the search go to the second stream, whose priority lets
+        // their CTAs in ahead of the target pass's grid.
+        rc = lattice_build_impl(draft_logits, dtype, B, L, V, dstride_b, dstride_l, K_max, tau, eos_id, cand_id,
+                                cand_logit, cand_logp, cand_count, lse, lse64, entropy, gen_len, row_status,
+                                lattice_workspace, lattice_workspace_bytes, st, side->fork, side->stream);
+        if (rc != DSP_OK) return rc;
+        rc = stats(st);
+        if (rc == DSP_OK) rc2 = search(side->stream);
+    } else {
+        // Short passes leave SMs free anyway: the build and the search stay on the caller's stream
+        // (no event between them) and the target statistics take the second stream.
+        rc = lattice_build_impl(draft_logits, dtype, B, L, V, dstride_b, dstride_l, K_max, tau, eos_id, cand_id,
+                                cand_logit, cand_logp, cand_count, lse, lse64, entropy, gen_len, row_status,
+                                lattice_workspace, lattice_workspace_bytes, st, side->fork, nullptr);
+        if (rc != DSP_OK) return rc;
+        DSP_CUDA_TRY(cudaStreamWaitEvent(side->stream, side->fork, 0));
+        rc = stats(side->stream);
+        if (rc == DSP_OK) rc2 = search(st);
+    }
     // whatever happened, the caller's stream joins the second stream again
-    cudaError_t e = e_rec;
+    cudaError_t e = cudaEventRecord(side->join, side->stream);
     if (e == cudaSuccess) e = cudaStreamWaitEvent(st, side->join, 0);
     if (rc != DSP_OK) return rc;
     if (e != cudaSuccess) return cuda_fail(e);
