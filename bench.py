@@ -195,9 +195,12 @@ def input_sets(w, device, seed_base=0):
     return [wl.make_inputs(w, step=seed_base + i, device=device) for i in range(n)]
 
 
-def time_workload(w, device, steps, warmup, dist=None, stages=True, seed_base=0):
-    """Device-timed throughput of one workload; returns a dict of measurements."""
+def time_workload(w, device, steps, warmup, dist=None, stages=True, seed_base=0, one_set=False):
+    """Device-timed throughput of one workload; returns a dict of measurements.  ``one_set``: the
+    same input set every step (inputs smaller than L2 then stay in it)."""
     sets = input_sets(w, device, seed_base)
+    if one_set:
+        sets = sets[:1]
     st = GpuStep(w, device)
     dsp = st.dsp
     for i in range(warmup):
@@ -491,6 +494,51 @@ def time_read_probe(sets, device, reps=40):
             "note": "dsp_read_probe over the draft logits of the timed input sets, back to back launches"}
 
 
+def time_adl_loop(device, n_steps=256):
+    """Workload 2 as the closed loop the controller runs in (Sec. 3.3): every step's draft length
+    is the one dsp_adl_update asked for after the step before, from that step's accepted and
+    generated lengths copied to the host (the step's one device-to-host crossing, with a stream
+    synchronisation).  Fresh logits every step (seed = step), drawn beforehand at the longest
+    length with EOS as the drafter's top-1 from a seeded random-walk position on; a step of length
+    L reads their first L rows.  Wall-clock over the loop, the synchronisations included."""
+    from paper_2510_02358_b200 import binding as dsp
+    base = wl.CONFIGS[2]
+    walk = wl.eos_walk(n_steps)
+    lengths = (8, 16, 24, 32)
+    sets = [wl.make_inputs(base.scaled(L=32, eos_from=c if c < 32 else -1), step=t, device=device)
+            for t, c in enumerate(walk)]
+    steps = {L: GpuStep(base.scaled(L=L), device) for L in lengths}
+    host = torch.empty((2,), dtype=torch.int32).pin_memory()
+    view = lambda inp, L: dict(inp, draft=inp["draft"][:, :L], target=inp["target"][:, :L], u=inp["u"])
+
+    def loop(n):
+        st, prm = dsp.dsp_adl_init(**wl.ADL_C2)
+        hist, acc, gen = {L: 0 for L in lengths}, 0, 0
+        for t in range(n):
+            L = st.k
+            g = steps[L]
+            g.step(view(sets[t], L))
+            host[0:1].copy_(g.ver.accepted_len, non_blocking=True)
+            host[1:2].copy_(g.lat.gen_len, non_blocking=True)
+            torch.cuda.current_stream().synchronize()
+            dsp.dsp_adl_update(st, prm, host[0:1], host[1:2])
+            hist[L] += 1
+            acc += int(host[0])
+            gen += int(host[1])
+        return hist, acc, gen
+
+    loop(16)                                          # warm-up
+    torch.cuda.synchronize()
+    t0 = time.perf_counter()
+    hist, acc, gen = loop(n_steps)
+    dt = time.perf_counter() - t0
+    return {"steps": n_steps, "steps_per_s": n_steps / dt, "us_per_step": dt / n_steps * 1e6,
+            "draft_length_histogram": hist, "mean_draft_length": sum(L * c for L, c in hist.items()) / n_steps,
+            "mean_accepted_len": acc / n_steps, "mean_gen_len": gen / n_steps,
+            "controller": wl.ADL_C2,
+            "note": "dsp_draft_verify_step + copy of 2 int32 to the host + synchronise + dsp_adl_update per step"}
+
+
 def run_reference(args, rank, world):
     if rank != 0:
         return
@@ -630,9 +678,14 @@ def main():
                     "frac_of_8000": 2 * tb / ((mm["ms_lattice"] + mm["ms_verify"]) * 1e-3) / 1e9 / 8000.0,
                     "input_sets": mm["sets"], "mean_accepted_len": mm["mean_accepted_len"],
                     "parity": parity_recheck(wv, s2, i2[0], 4 if cid == 5 else 16)}
+                if 2 * tb < L2_BYTES:                   # also with the one input set left in L2
+                    mw, s3, i3 = time_workload(wv, device, n, 5, stages=False, one_set=True)
+                    extras[wv.name]["ms_per_step_inputs_in_l2"] = mw["ms_per_step"]
+                    del s3, i3
                 del s2, i2
                 torch.cuda.empty_cache()
         line["workloads"] = extras
+        line["adl_closed_loop_c2"] = time_adl_loop(device)
         line["unmask_step"] = time_unmask(w, device)
         line["vocab_sharded_lattice"] = time_sharded(w, device)
     print(json.dumps(line))
