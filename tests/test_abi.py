@@ -66,6 +66,11 @@ def test_device_entry_points_reject_bad_arguments_on_the_host():
     # batch of zero rows is a no-op
     assert lib.dsp_lattice_build(z, 0, 0, 8, 100, C.c_int64(800), C.c_int64(100), 4, C.c_float(0), -1,
                                  z, z, z, z, z, z, z, z, z, z, C.c_size_t(0), z) == dsp.DSP_OK
+    # read probe: null and misaligned pointers, too few bytes
+    assert lib.dsp_read_probe(z, C.c_size_t(1024), one, z) == dsp.DSP_ERR_INVALID_ARG
+    assert lib.dsp_read_probe(one, C.c_size_t(1024), z, z) == dsp.DSP_ERR_INVALID_ARG
+    assert lib.dsp_read_probe(C.c_void_p(264), C.c_size_t(1024), one, z) == dsp.DSP_ERR_INVALID_ARG
+    assert lib.dsp_read_probe(one, C.c_size_t(8), one, z) == dsp.DSP_ERR_INVALID_ARG
     # path search: beam too wide, bad table size, bad lambda
     def cps(W=4, log2=10, lam=0.5, kind=0):
         return lib.dsp_cps_search(one, one, one, one, 1, 8, 5, one, kind, one, log2, C.c_uint32(0), 100,

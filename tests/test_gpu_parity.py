@@ -637,6 +637,40 @@ def test_single_call_step_equals_the_three_calls(cid):
     check_step(b, inp, **_params(w))
 
 
+@pytest.mark.parametrize("B,L", [(64, 32), (96, 24)])
+def test_single_call_step_on_long_passes_equals_the_three_calls(B, L):
+    """Logits tensors of 400 MB and more take the other stream arrangement of the single call (the
+    lattice's finish and the search on the library's high-priority stream); up to 74 batch rows
+    the search also keeps its SMs to itself, with more it shares them.  Same bytes either way."""
+    w = wl.CONFIGS[4].scaled(B=B, L=L)
+    assert w.logits_bytes >= 400 << 20
+    inp = wl.make_inputs(w, step=5, device=DEV)
+    a = gpu_step(inp, **_params(w))
+    for rep in range(2):
+        b = gpu_step(inp, fused=True, **_params(w))
+        for s in ("lat", "cps", "ver"):
+            for k, v in vars(getattr(a, s)).items():
+                if v is not None:
+                    assert torch.equal(v.view(torch.uint8), getattr(getattr(b, s), k).view(torch.uint8)), (s, k)
+    check_step(b, inp, rows=[0, 1, B // 2, B - 1], **_params(w))
+    del inp
+    torch.cuda.empty_cache()
+
+
+def test_read_probe_runs_and_rejects_bad_arguments():
+    x = torch.zeros(1 << 22, dtype=torch.bfloat16, device=DEV)
+    sink = torch.zeros(1, dtype=torch.int32, device=DEV)
+    for _ in range(3):
+        dsp.dsp_read_probe(x, sink)
+    dsp.dsp_read_probe(x[: 8 * 1000 + 8], sink)           # a ragged last piece
+    torch.cuda.synchronize()
+    assert int(sink[0]) == 0                              # zeros never fold to the stored value
+    with pytest.raises(dsp.DspError):
+        dsp.dsp_read_probe(x[1:9], sink)                  # not 16-byte aligned
+    with pytest.raises(dsp.DspError):
+        dsp.dsp_read_probe(x[:4], sink)                   # fewer than 16 bytes
+
+
 def all_greedy_unused(w, s, k):
     """Outputs that a greedy-only verification does not write."""
     return w.verify == "greedy" and s == "ver" and k in ("ratio", "tgt_lse")
