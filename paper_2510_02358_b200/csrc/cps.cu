@@ -115,6 +115,7 @@ __global__ void __launch_bounds__(kThreads) cps_kernel(const CpsArgs a) {
     __shared__ int btok[2][TRI ? DSP_MAX_W : 1], btok2[2][TRI ? DSP_MAX_W : 1];
     __shared__ __align__(16) uint32_t tbest[2][TRI ? DSP_MAX_W : 4];
 
+    grid_dependency_wait();                            // the lattice is complete from here on
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int b = blockIdx.x;
     const int L = a.L, W = a.W, KC = a.KC, D = a.D;
@@ -439,9 +440,7 @@ int32_t dsp::cps_search_impl(const int32_t *cand_id, const float *cand_logit,
             if (dev >= 0 && dev < 64) done[dev] = true;
         }
     }
-    if (tri) cps_kernel<true><<<B, kThreads, dyn, stream>>>(a);
-    else cps_kernel<false><<<B, kThreads, dyn, stream>>>(a);
-    DSP_CUDA_TRY(cudaGetLastError());
+    DSP_CUDA_TRY(launch_dependent(tri ? cps_kernel<true> : cps_kernel<false>, (unsigned)B, kThreads, dyn, stream, a));
     return DSP_OK;
 }
 

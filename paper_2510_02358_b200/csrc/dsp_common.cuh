@@ -41,6 +41,29 @@ inline int32_t cuda_fail(cudaError_t e) {
 
 __host__ __device__ inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
+// ---- programmatic dependent launch: a kernel that only consumes what the kernel before it in
+// the stream produced is launched with launch_dependent; the device may then place its CTAs as
+// soon as every CTA of that kernel has called grid_launch_dependents (or left), and they sit in
+// grid_dependency_wait until that kernel has completed and its writes are visible.  The wait is
+// the first thing such a kernel does; launched without the attribute, both calls do nothing.
+__device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void grid_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+template <typename Arg>
+inline cudaError_t launch_dependent(void (*kernel)(Arg), unsigned grid, unsigned block, size_t smem,
+                                    cudaStream_t st, const Arg &a) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(grid);
+    cfg.blockDim = dim3(block);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, a);
+}
+
 // ---- order-preserving 64-bit keys: larger key = better under (logit desc, id asc) ----
 __device__ __forceinline__ uint32_t ord_bits(float x) {
     uint32_t b = __float_as_uint(x + 0.0f);                 // -0.0 -> +0.0

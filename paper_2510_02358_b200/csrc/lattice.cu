@@ -197,6 +197,7 @@ __global__ void __launch_bounds__(kThreads, 4) lattice_scan_kernel(const Lattice
     const int s0 = slice * a.slice_elems;
     const int s1 = min(a.V, s0 + a.slice_elems);
     stream_begin(bars);
+    grid_launch_dependents();
     DT *trow = reinterpret_cast<DT *>(a.table) + row * (a.ntiles_row + a.nslices) * kThreads;   // the row's table
     DT *tab = trow + (long long)(s0 / tile_elems<DT>()) * kThreads;
     DT *smax = trow + (long long)(a.ntiles_row + slice) * kThreads;
@@ -211,6 +212,8 @@ __global__ void __launch_bounds__(kThreads, 4) lattice_scan_kernel(const Lattice
 template <typename DT>
 __global__ void __launch_bounds__(kThreads) lattice_rows_kernel(const LatticeArgs a) {
     __shared__ WarpScratch scratch[kRowWarps];
+    grid_dependency_wait();                            // pass 1 is complete from here on
+    grid_launch_dependents();
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const long long row = (long long)blockIdx.x * kRowWarps + warp;
     if (row >= (long long)a.B * a.L) return;
@@ -266,7 +269,7 @@ static int32_t launch_lattice(LatticeArgs &a, void *workspace, size_t workspace_
             }
             after_scan = nullptr;
         }
-        lattice_rows_kernel<DT><<<(unsigned)((nrows + kRowWarps - 1) / kRowWarps), kThreads, 0, rs>>>(a);
+        DSP_CUDA_TRY(launch_dependent(lattice_rows_kernel<DT>, (unsigned)((nrows + kRowWarps - 1) / kRowWarps), kThreads, 0, rs, a));
     } else {
         lattice_kernel<DT><<<(unsigned)nblocks, kThreads, 0, st>>>(a);
     }

@@ -235,6 +235,7 @@ __global__ void __launch_bounds__(kThreads, 4) target_scan_kernel(const VerifyAr
     const int s1 = min(a.V, s0 + a.slice_elems);
     const bool sums = !a.all_greedy && a.mode[b] != 0;
     stream_begin(bars);
+    grid_launch_dependents();
     DT *trow = reinterpret_cast<DT *>(a.table) + row * (a.ntiles_row + a.nslices) * kThreads;   // the row's table
     DT *tab = trow + (long long)(s0 / tile_elems<DT>()) * kThreads;
     DT *smax = trow + (long long)(a.ntiles_row + slice) * kThreads;
@@ -247,6 +248,8 @@ __global__ void __launch_bounds__(kThreads, 4) target_scan_kernel(const VerifyAr
 template <typename DT>
 __global__ void __launch_bounds__(kThreads) target_rows_kernel(const VerifyArgs a) {
     __shared__ WarpScratch scratch[kRowWarps];
+    grid_dependency_wait();                            // pass 1 is complete from here on
+    grid_launch_dependents();
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const long long row = (long long)blockIdx.x * kRowWarps + warp;
     if (row >= (long long)a.B * a.Lt) return;
@@ -284,6 +287,8 @@ __global__ void __launch_bounds__(kThreads) target_rows_kernel(const VerifyArgs 
 // the target statistics of all rows are there.
 template <typename DT>
 __global__ void __launch_bounds__(kThreads) accept_kernel(const VerifyArgs a) {
+    grid_dependency_wait();                            // target statistics and path are complete from here on
+    grid_launch_dependents();
     const int b = blockIdx.x * kWarps + (threadIdx.x >> 5);
     if (b < a.B) accept_row<DT>(a, b);
 }
@@ -322,6 +327,7 @@ __global__ void __launch_bounds__(kThreads, 4) residual_kernel(const VerifyArgs 
     __shared__ double s_total;
     __shared__ int s_found;
     __shared__ int s_flag;
+    grid_dependency_wait();                            // the sampling jobs are complete from here on
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int b = blockIdx.x / a.res_slices;
     const int rs = blockIdx.x - b * a.res_slices;
@@ -544,19 +550,16 @@ static int32_t launch_verify(VerifyArgs &a, void *workspace, size_t workspace_by
         target_scan_kernel<DT><<<(unsigned)nblocks, kThreads, kRingBytes, st>>>(a);
         DSP_CUDA_TRY(cudaGetLastError());
         if (pe.stop) DSP_CUDA_TRY(cudaEventRecord(pe.stop, st));
-        target_rows_kernel<DT><<<(unsigned)((nrows + kRowWarps - 1) / kRowWarps), kThreads, 0, st>>>(a);
+        DSP_CUDA_TRY(launch_dependent(target_rows_kernel<DT>, (unsigned)((nrows + kRowWarps - 1) / kRowWarps), kThreads, 0, st, a));
     } else {
         target_kernel<DT><<<(unsigned)nblocks, kThreads, 0, st>>>(a);
     }
     DSP_CUDA_TRY(cudaGetLastError());
     }
     if (phases & kVerifyDecide) {
-        accept_kernel<DT><<<(unsigned)((a.B + kWarps - 1) / kWarps), kThreads, 0, st>>>(a);
-        DSP_CUDA_TRY(cudaGetLastError());
-        if (!a.all_greedy) {
-            residual_kernel<DT><<<(unsigned)(a.B * a.res_slices), kThreads, 0, st>>>(a);
-            DSP_CUDA_TRY(cudaGetLastError());
-        }
+        DSP_CUDA_TRY(launch_dependent(accept_kernel<DT>, (unsigned)((a.B + kWarps - 1) / kWarps), kThreads, 0, st, a));
+        if (!a.all_greedy)
+            DSP_CUDA_TRY(launch_dependent(residual_kernel<DT>, (unsigned)(a.B * a.res_slices), kThreads, 0, st, a));
     }
     return DSP_OK;
 }
