@@ -440,7 +440,8 @@ int32_t dsp::cps_search_impl(const int32_t *cand_id, const float *cand_logit,
             if (dev >= 0 && dev < 64) done[dev] = true;
         }
     }
-    DSP_CUDA_TRY(launch_dependent(tri ? cps_kernel<true> : cps_kernel<false>, (unsigned)B, kThreads, dyn, stream, a));
+    DSP_CUDA_TRY(launch_dependent(tri ? cps_kernel<true> : cps_kernel<false>, (unsigned)B, kThreads, dyn, stream, a,
+                                  short_kernel_follows_early(stream, (long long)B * L)));
     return DSP_OK;
 }
 

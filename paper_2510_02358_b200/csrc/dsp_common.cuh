@@ -48,9 +48,14 @@ __host__ __device__ inline size_t align_up(size_t x, size_t a) { return (x + a -
 // the first thing such a kernel does; launched without the attribute, both calls do nothing.
 __device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 __device__ __forceinline__ void grid_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+// `programmatic` false: an ordinary launch (full dependency on the kernel before).
 template <typename Arg>
 inline cudaError_t launch_dependent(void (*kernel)(Arg), unsigned grid, unsigned block, size_t smem,
-                                    cudaStream_t st, const Arg &a) {
+                                    cudaStream_t st, const Arg &a, bool programmatic) {
+    if (!programmatic) {
+        kernel<<<grid, block, smem, st>>>(a);
+        return cudaGetLastError();
+    }
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(grid);
     cfg.blockDim = dim3(block);
@@ -62,6 +67,31 @@ inline cudaError_t launch_dependent(void (*kernel)(Arg), unsigned grid, unsigned
     cfg.attrs = attr;
     cfg.numAttrs = 1;
     return cudaLaunchKernelEx(&cfg, kernel, a);
+}
+
+// Where the early placement pays (measured on a B200).  Between the short kernels of a call it
+// saves 1 to 2 us per launch.  Behind a pass over the logits whose grid is several times what the
+// SMs hold, CTAs of the next kernel that sit waiting beside the pass's last wave cost more than
+// the launch they save (+4 % on 16384 rows), so a rows kernel follows such a pass the ordinary
+// way.  In a captured graph the programmatic edges pay only on large problems (small ones replay
+// 2 us slower with them).
+constexpr long long kDependentScanCtas = 2 * 148 * 4;     // largest pass a rows kernel follows early
+constexpr long long kDependentGraphRows = 1024;           // fewest logits rows for programmatic edges in a graph
+inline bool stream_is_capturing(cudaStream_t st) {
+    cudaStreamCaptureStatus cs = cudaStreamCaptureStatusNone;
+    if (cudaStreamIsCapturing(st, &cs) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return true;                                       // unknown: take the ordinary launch
+    }
+    return cs != cudaStreamCaptureStatusNone;
+}
+// A rows kernel (pass 2) behind its pass over the logits (`scan_ctas` CTAs).
+inline bool rows_follow_early(cudaStream_t st, long long scan_ctas) {
+    return scan_ctas <= kDependentScanCtas && !stream_is_capturing(st);
+}
+// A short kernel behind another short kernel, in a call over `nrows` rows of logits.
+inline bool short_kernel_follows_early(cudaStream_t st, long long nrows) {
+    return nrows >= kDependentGraphRows || !stream_is_capturing(st);
 }
 
 // ---- order-preserving 64-bit keys: larger key = better under (logit desc, id asc) ----

@@ -269,7 +269,8 @@ static int32_t launch_lattice(LatticeArgs &a, void *workspace, size_t workspace_
             }
             after_scan = nullptr;
         }
-        DSP_CUDA_TRY(launch_dependent(lattice_rows_kernel<DT>, (unsigned)((nrows + kRowWarps - 1) / kRowWarps), kThreads, 0, rs, a));
+        DSP_CUDA_TRY(launch_dependent(lattice_rows_kernel<DT>, (unsigned)((nrows + kRowWarps - 1) / kRowWarps), kThreads, 0, rs, a,
+                                      rows_follow_early(rs, nblocks)));
     } else {
         lattice_kernel<DT><<<(unsigned)nblocks, kThreads, 0, st>>>(a);
     }

@@ -59,6 +59,7 @@ __global__ void __launch_bounds__(kThreads, 4) shard_scan_kernel(const ShardArgs
     const int s0 = slice * a.slice_elems;
     const int s1 = min(a.V, s0 + a.slice_elems);
     stream_begin(bars);
+    grid_launch_dependents();
     DT *trow = reinterpret_cast<DT *>(a.table) + row * (a.ntiles_row + a.nslices) * kThreads;
     DT *tab = trow + (long long)(s0 / tile_elems<DT>()) * kThreads;
     DT *smax = trow + (long long)(a.ntiles_row + slice) * kThreads;
@@ -113,6 +114,7 @@ __device__ unsigned long long warp_row_elementwise(const DT *__restrict__ row, i
 template <typename DT>
 __global__ void __launch_bounds__(kThreads) shard_rows_kernel(const ShardArgs a) {
     __shared__ WarpScratch scratch[kRowWarps];
+    grid_dependency_wait();                            // pass 1 is complete from here on
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const long long row = (long long)blockIdx.x * kRowWarps + warp;
     if (row >= (long long)a.B * a.L) return;
@@ -233,8 +235,8 @@ static int32_t launch_shard(ShardArgs &a, void *workspace, size_t workspace_byte
         shard_scan_kernel<DT><<<(unsigned)nblocks, kThreads, kRingBytes, st>>>(a);
         DSP_CUDA_TRY(cudaGetLastError());
     }
-    shard_rows_kernel<DT><<<(unsigned)((nrows + kRowWarps - 1) / kRowWarps), kThreads, 0, st>>>(a);
-    DSP_CUDA_TRY(cudaGetLastError());
+    DSP_CUDA_TRY(launch_dependent(shard_rows_kernel<DT>, (unsigned)((nrows + kRowWarps - 1) / kRowWarps), kThreads, 0, st, a,
+                                  a.streaming && rows_follow_early(st, nblocks)));
     return DSP_OK;
 }
 

@@ -63,6 +63,7 @@ __global__ void __launch_bounds__(kThreads, 4) unmask_scan_kernel(const UnmaskAr
     const int s0 = slice * a.slice_elems;
     const int s1 = min(a.V, s0 + a.slice_elems);
     stream_begin(bars);
+    grid_launch_dependents();
     DT *trow = reinterpret_cast<DT *>(a.table) + row * (a.ntiles_row + a.nslices) * kThreads;
     DT *tab = trow + (long long)(s0 / tile_elems<DT>()) * kThreads;
     DT *smax = trow + (long long)(a.ntiles_row + slice) * kThreads;
@@ -110,6 +111,7 @@ __device__ bool warp_row_stats_elementwise(const DT *__restrict__ row, int V, in
 template <typename DT>
 __global__ void __launch_bounds__(kThreads) unmask_rows_kernel(const UnmaskArgs a) {
     __shared__ WarpScratch scratch[kRowWarps];
+    grid_dependency_wait();                            // pass 1 is complete from here on
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const long long row = (long long)blockIdx.x * kRowWarps + warp;
     if (row >= (long long)a.B * a.L) return;
@@ -209,8 +211,8 @@ static int32_t launch_unmask(UnmaskArgs &a, void *workspace, size_t workspace_by
         unmask_scan_kernel<DT><<<(unsigned)nblocks, kThreads, kRingBytes, st>>>(a);
         DSP_CUDA_TRY(cudaGetLastError());
     }
-    unmask_rows_kernel<DT><<<(unsigned)((nrows + kRowWarps - 1) / kRowWarps), kThreads, 0, st>>>(a);
-    DSP_CUDA_TRY(cudaGetLastError());
+    DSP_CUDA_TRY(launch_dependent(unmask_rows_kernel<DT>, (unsigned)((nrows + kRowWarps - 1) / kRowWarps), kThreads, 0, st, a,
+                                  a.streaming && rows_follow_early(st, nblocks)));
     return DSP_OK;
 }
 

@@ -550,16 +550,18 @@ static int32_t launch_verify(VerifyArgs &a, void *workspace, size_t workspace_by
         target_scan_kernel<DT><<<(unsigned)nblocks, kThreads, kRingBytes, st>>>(a);
         DSP_CUDA_TRY(cudaGetLastError());
         if (pe.stop) DSP_CUDA_TRY(cudaEventRecord(pe.stop, st));
-        DSP_CUDA_TRY(launch_dependent(target_rows_kernel<DT>, (unsigned)((nrows + kRowWarps - 1) / kRowWarps), kThreads, 0, st, a));
+        DSP_CUDA_TRY(launch_dependent(target_rows_kernel<DT>, (unsigned)((nrows + kRowWarps - 1) / kRowWarps), kThreads, 0, st, a,
+                                      short_kernel_follows_early(st, nrows)));
     } else {
         target_kernel<DT><<<(unsigned)nblocks, kThreads, 0, st>>>(a);
     }
     DSP_CUDA_TRY(cudaGetLastError());
     }
     if (phases & kVerifyDecide) {
-        DSP_CUDA_TRY(launch_dependent(accept_kernel<DT>, (unsigned)((a.B + kWarps - 1) / kWarps), kThreads, 0, st, a));
+        const bool early = short_kernel_follows_early(st, nrows);
+        DSP_CUDA_TRY(launch_dependent(accept_kernel<DT>, (unsigned)((a.B + kWarps - 1) / kWarps), kThreads, 0, st, a, early));
         if (!a.all_greedy)
-            DSP_CUDA_TRY(launch_dependent(residual_kernel<DT>, (unsigned)(a.B * a.res_slices), kThreads, 0, st, a));
+            DSP_CUDA_TRY(launch_dependent(residual_kernel<DT>, (unsigned)(a.B * a.res_slices), kThreads, 0, st, a, early));
     }
     return DSP_OK;
 }
