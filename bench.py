@@ -123,8 +123,9 @@ class GpuStep:
         self.ws_l = dsp.alloc_workspace(dsp.dsp_lattice_workspace_bytes(w.B, w.L, w.V, dt, w.K), device)
         self.ws_v = dsp.alloc_workspace(dsp.dsp_verify_workspace_bytes(w.B, w.L, w.Lt, w.V, dt), device)
         self.all_greedy = w.verify == "greedy"
-        # lattice scan + rows, cps, target scan + rows, accept (+ residual); memsets are not counted
-        self.kernels_per_step = 6 if self.all_greedy else 7
+        # lattice scan + rows, cps, target scan + rows, accept (greedy) or residual with the acceptance
+        # scan inside (stochastic rows); memsets are not counted
+        self.kernels_per_step = 6
 
     def step(self, inp):
         """One step through the single-call entry point (what `value` and `e2e` time)."""

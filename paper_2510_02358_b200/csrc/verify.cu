@@ -5,13 +5,14 @@
 // 16-byte aligned layouts by target_scan_kernel (one CTA per row slice, no block-wide barrier,
 // see stream_core.cuh) followed by target_rows_kernel (one warp per row: argmax from the table
 // of tile maxima, sums added up), any other layout by target_kernel (element-wise, slices
-// merged by the CTA arriving last).  accept_kernel then runs every batch row's left-to-right
-// acceptance scan (one warp each) and either writes the next token (greedy) or records a
-// sampling job (stochastic: residual at the first rejection, or bonus from row m).
-// The first part needs only the target logits: dsp_draft_verify_step (step.cu) runs it beside
-// the lattice finish and the path search.
-// Kernel 2 (residual_kernel): for each job, one more pass over ONE target row (and ONE draft
-// row): per-chunk sums of max(0, p - q) in token order; the CTA arriving last inverts the CDF.
+// merged by the CTA arriving last).  Every batch row's left-to-right acceptance scan (one warp)
+// then either gives the next token (greedy) or a sampling job (stochastic: residual at the first
+// rejection, or bonus from row m).  The first part needs only the target logits:
+// dsp_draft_verify_step (step.cu) runs it beside the lattice finish and the path search.
+// residual_kernel: for each job, one more pass over ONE target row (and ONE draft row):
+// per-chunk sums of max(0, p - q) in token order; the CTA arriving last inverts the CDF.
+// When every row is greedy the scans run in accept_kernel and that is all; otherwise they run
+// inside residual_kernel (each CTA scans its own batch row first): one launch less in the chain.
 #include "dsp_internal.h"
 #include "row_warp.cuh"
 
@@ -75,9 +76,11 @@ __device__ __forceinline__ const DT *drow_ptr(const VerifyArgs &a, long long dro
     return reinterpret_cast<const DT *>(a.draft) + b * a.dstride_b + i * a.dstride_l;
 }
 
-// Left-to-right acceptance of batch row b by one warp (Eq. 1, Eq. 2).
+// Left-to-right acceptance of batch row b by one warp (Eq. 1, Eq. 2).  Returns (in lane 0) the
+// sampling job of the row (trow < 0: none); with `write` it also writes the row's outputs
+// (without: the same decisions, no side effects: for CTAs that only need the job).
 template <typename DT>
-__device__ void accept_row(const VerifyArgs &a, int b) {
+__device__ SampleJob accept_row(const VerifyArgs &a, int b, bool write) {
     const int lane = threadIdx.x & 31;
     const int L = a.L, Lt = a.Lt;
     const int m = max(0, min(__ldcg(&a.path_len[b]), L));
@@ -104,7 +107,7 @@ __device__ void accept_row(const VerifyArgs &a, int b) {
                 rt_out = (float)rt;
             }
         }
-        if (a.ratio && i < L) a.ratio[(long long)b * L + i] = rt_out;
+        if (write && a.ratio && i < L) a.ratio[(long long)b * L + i] = rt_out;
         const unsigned bal = __ballot_sync(0xFFFFFFFFu, rej);
         if (bal && acc == m) acc = i0 + __ffs(bal) - 1;
     }
@@ -115,11 +118,11 @@ __device__ void accept_row(const VerifyArgs &a, int b) {
             if (__ballot_sync(0xFFFFFFFFu, e)) eos_seen_before_acc = true;
         }
     }
+    SampleJob job;
+    job.trow = -1; job.drow = -1; job.u = 0.f; job.fallback = -1;
     if (lane == 0) {
-        unsigned status = atomicOr(&a.b_status[b], 0u);
+        unsigned status = write ? atomicOr(&a.b_status[b], 0u) : 0u;
         if (eos_seen_before_acc) status |= DSP_ROW_EOS_ACCEPTED;
-        SampleJob job;
-        job.trow = -1; job.drow = -1; job.u = 0.f; job.fallback = -1;
         int nt = -1;
         const int at = acc < m ? acc : m;              // row the next token comes from
         if (acc < m || m < Lt) {
@@ -135,12 +138,15 @@ __device__ void accept_row(const VerifyArgs &a, int b) {
         } else {
             status |= DSP_ROW_NO_BONUS_ROW;
         }
-        a.accepted_len[b] = acc;
-        a.next_token[b] = nt;
-        if (!a.all_greedy) a.jobs[b] = job;
-        if (a.job_trow) { a.job_trow[b] = job.trow; a.job_drow[b] = job.drow; }
-        if (status) atomicOr(&a.row_status[b], status);
+        if (write) {
+            a.accepted_len[b] = acc;
+            a.next_token[b] = nt;
+            if (!a.all_greedy) a.jobs[b] = job;
+            if (a.job_trow) { a.job_trow[b] = job.trow; a.job_drow[b] = job.drow; }
+            if (status) atomicOr(&a.row_status[b], status);
+        }
     }
+    return job;
 }
 
 template <typename DT, typename SY>
@@ -290,7 +296,7 @@ __global__ void __launch_bounds__(kThreads) accept_kernel(const VerifyArgs a) {
     grid_dependency_wait();                            // target statistics and path are complete from here on
     grid_launch_dependents();
     const int b = blockIdx.x * kWarps + (threadIdx.x >> 5);
-    if (b < a.B) accept_row<DT>(a, b);
+    if (b < a.B) accept_row<DT>(a, b, true);
 }
 
 // ---- residual / bonus sampling -------------------------------------------------------------
@@ -318,7 +324,11 @@ __device__ __forceinline__ float residual(float xt, float xd, const RowProb &pt,
     return r > 0.f ? r : 0.f;                  // NaN -> 0
 }
 
-template <typename DT>
+// ACCEPT: the kernel follows the target statistics directly and every CTA first runs its batch
+// row's acceptance scan itself (one warp; the row's first CTA writes the scan's outputs), which
+// takes the acceptance kernel and its launch out of the chain; otherwise the jobs are read from
+// a.jobs, written by an earlier kernel.
+template <typename DT, bool ACCEPT>
 __global__ void __launch_bounds__(kThreads, 4) residual_kernel(const VerifyArgs a) {
     constexpr int N = Elem<DT>::N;
     constexpr int CE = 32 * N;                  // elements per chunk: one warp-wide vector load
@@ -327,11 +337,19 @@ __global__ void __launch_bounds__(kThreads, 4) residual_kernel(const VerifyArgs 
     __shared__ double s_total;
     __shared__ int s_found;
     __shared__ int s_flag;
-    grid_dependency_wait();                            // the sampling jobs are complete from here on
+    __shared__ SampleJob s_job;
+    grid_dependency_wait();                            // what the kernels before wrote is complete from here on
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int b = blockIdx.x / a.res_slices;
     const int rs = blockIdx.x - b * a.res_slices;
-    const SampleJob job = a.jobs[b];
+    if constexpr (ACCEPT) {
+        if (warp == 0) {
+            const SampleJob j = accept_row<DT>(a, b, rs == 0);
+            if (lane == 0) s_job = j;
+        }
+        __syncthreads();
+    }
+    const SampleJob job = ACCEPT ? s_job : a.jobs[b];
     if (job.trow < 0) return;
     const bool has_q = job.drow >= 0;
     const DT *tp = trow_ptr<DT>(a, job.trow);
@@ -559,9 +577,10 @@ static int32_t launch_verify(VerifyArgs &a, void *workspace, size_t workspace_by
     }
     if (phases & kVerifyDecide) {
         const bool early = short_kernel_follows_early(st, nrows);
-        DSP_CUDA_TRY(launch_dependent(accept_kernel<DT>, (unsigned)((a.B + kWarps - 1) / kWarps), kThreads, 0, st, a, early));
-        if (!a.all_greedy)
-            DSP_CUDA_TRY(launch_dependent(residual_kernel<DT>, (unsigned)(a.B * a.res_slices), kThreads, 0, st, a, early));
+        if (a.all_greedy)
+            DSP_CUDA_TRY(launch_dependent(accept_kernel<DT>, (unsigned)((a.B + kWarps - 1) / kWarps), kThreads, 0, st, a, early));
+        else           // the acceptance scan runs inside the residual kernel
+            DSP_CUDA_TRY(launch_dependent(residual_kernel<DT, true>, (unsigned)(a.B * a.res_slices), kThreads, 0, st, a, early));
     }
     return DSP_OK;
 }
@@ -715,7 +734,7 @@ static int32_t launch_sample(VerifyArgs &a, SampleArgs &s, void *workspace, size
     DSP_CUDA_TRY(cudaMemsetAsync(ws, 0, w.zero_bytes, st));
     sample_prepare_kernel<<<(unsigned)((a.B + 127) / 128), 128, 0, st>>>(s);
     DSP_CUDA_TRY(cudaGetLastError());
-    residual_kernel<DT><<<(unsigned)(a.B * a.res_slices), kThreads, 0, st>>>(a);
+    residual_kernel<DT, false><<<(unsigned)(a.B * a.res_slices), kThreads, 0, st>>>(a);
     DSP_CUDA_TRY(cudaGetLastError());
     return DSP_OK;
 }
