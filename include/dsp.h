@@ -160,8 +160,8 @@ int32_t dsp_lattice_build(const void *draft_logits, int32_t dtype,
  *  - This function calls no allocating routine (no cudaMalloc / cudaFree).
  *  - Limit: dsp_lattice_workspace_bytes(B, L, V, dtype, K_max) must not exceed
  *    DSP_STATIC_WS_BYTES, else DSP_ERR_STATIC_SCRATCH is returned and nothing
- *    is enqueued.  (The scratch is about 3.3 % of the draft logits' bytes:
- *    B*L*V up to about 60 million bf16 logits fits; ask the query call.)
+ *    is enqueued.  (The scratch is about 2.4 % of the draft logits' bytes:
+ *    B*L*V up to about 80 million bf16 logits fits; ask the query call.)
  *  - The first call on each device looks up the array's device address (a
  *    host-side, once-per-device step with that device current).  Make that
  *    first call outside any stream capture.

@@ -175,7 +175,7 @@ template <> struct Elem<float> {
                      fmaxf(__uint_as_float(v.z), __uint_as_float(v.w)));
     }
 };
-constexpr int kVpt = 4;                         // vectors per thread per tile
+constexpr int kVpt = 6;                         // vectors per thread per tile
 
 template <typename DT> __host__ __device__ constexpr int tile_elems() { return kThreads * kVpt * Elem<DT>::N; }
 

@@ -187,15 +187,15 @@ __global__ void __launch_bounds__(kThreads, 4) lattice_kernel(const LatticeArgs 
 
 // Streaming path, pass 1: one CTA per row slice (see stream_core.cuh).
 template <typename DT>
-__global__ void __launch_bounds__(kThreads, 4) lattice_scan_kernel(const LatticeArgs a) {
+__global__ void __launch_bounds__(kThreads, 3) lattice_scan_kernel(const LatticeArgs a) {
     extern __shared__ __align__(128) unsigned char ring[];
     __shared__ StreamBars bars;
     const long long row = blockIdx.x / a.nslices;
     const int slice = blockIdx.x - (int)(row * a.nslices);
     const int b = (int)(row / a.L), l = (int)(row - (long long)b * a.L);
     const DT *rowp = reinterpret_cast<const DT *>(a.logits) + b * a.stride_b + l * a.stride_l;
-    const int s0 = slice * a.slice_elems;
-    const int s1 = min(a.V, s0 + a.slice_elems);
+    int s0, s1;
+    slice_range<DT>(slice, a.nslices, a.ntiles_row, a.V, s0, s1);
     stream_begin(bars);
     grid_launch_dependents();
     DT *trow = reinterpret_cast<DT *>(a.table) + row * (a.ntiles_row + a.nslices) * kThreads;   // the row's table

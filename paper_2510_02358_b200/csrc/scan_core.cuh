@@ -245,7 +245,7 @@ __device__ void scan_slice(const DT *__restrict__ row, int s0, int s1, int K, Sc
         float vm[kVpt];
 #pragma unroll
         for (int j = 0; j < kVpt; ++j) vm[j] = Elem<DT>::vmax(v[j]);
-        const float tm = fmaxf(fmaxf(vm[0], vm[1]), fmaxf(vm[2], vm[3]));
+        const float tm = fmaxf(fmaxf(fmaxf(vm[0], vm[1]), fmaxf(vm[2], vm[3])), fmaxf(vm[4], vm[5]));
 
         if constexpr (SUMS) {
             const float cn = fmaxf(c, tm * kLog2e);

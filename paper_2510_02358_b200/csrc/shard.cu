@@ -49,15 +49,15 @@ static ShardWs shard_ws_layout(int64_t B, int64_t L, int nslices, int ntiles_row
 
 // Pass 1 over the slice's rows: one CTA per row slice (stream_core.cuh).
 template <typename DT>
-__global__ void __launch_bounds__(kThreads, 4) shard_scan_kernel(const ShardArgs a) {
+__global__ void __launch_bounds__(kThreads, 3) shard_scan_kernel(const ShardArgs a) {
     extern __shared__ __align__(128) unsigned char ring[];
     __shared__ StreamBars bars;
     const long long row = blockIdx.x / a.nslices;
     const int slice = blockIdx.x - (int)(row * a.nslices);
     const int b = (int)(row / a.L), l = (int)(row - (long long)b * a.L);
     const DT *rowp = reinterpret_cast<const DT *>(a.logits) + b * a.stride_b + l * a.stride_l;
-    const int s0 = slice * a.slice_elems;
-    const int s1 = min(a.V, s0 + a.slice_elems);
+    int s0, s1;
+    slice_range<DT>(slice, a.nslices, a.ntiles_row, a.V, s0, s1);
     stream_begin(bars);
     grid_launch_dependents();
     DT *trow = reinterpret_cast<DT *>(a.table) + row * (a.ntiles_row + a.nslices) * kThreads;

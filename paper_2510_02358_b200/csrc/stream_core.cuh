@@ -116,6 +116,15 @@ __device__ __forceinline__ void stream_begin(StreamBars &bars) {
     __syncthreads();
 }
 
+// The tiles of a row dealt to its slices as evenly as whole tiles allow: slice s of n covers the
+// tiles [s * T / n, (s + 1) * T / n) of the row's T tiles (n <= T, so no slice is empty).
+template <typename DT>
+__device__ __forceinline__ void slice_range(int slice, int nslices, int ntiles_row, int V, int &s0, int &s1) {
+    constexpr int TE = tile_elems<DT>();
+    s0 = (int)((long long)slice * ntiles_row / nslices) * TE;
+    s1 = min(V, (int)((long long)(slice + 1) * ntiles_row / nslices) * TE);
+}
+
 // Issue the bulk copy of tile t of the slice at `src` into its ring stage (one thread).
 __device__ __forceinline__ void issue_tile(const char *src, int nbytes, int t, unsigned char *ring,
                                            StreamBars &bars) {
@@ -207,7 +216,7 @@ __device__ void stream_slice(const DT *__restrict__ row, int s0, int s1, bool su
                 vm[j] = fmaxf(max3(x[j][0], x[j][1], x[j][2]), x[j][3]);
             }
         }
-        const float tm = fmaxf(fmaxf(vm[0], vm[1]), fmaxf(vm[2], vm[3]));
+        const float tm = fmaxf(fmaxf(fmaxf(vm[0], vm[1]), fmaxf(vm[2], vm[3])), fmaxf(vm[4], vm[5]));
         table_store(tab, t * kThreads + tid, tm);
         rm = fmaxf(rm, tm);
 

@@ -52,7 +52,7 @@ static UnmaskWs unmask_ws_layout(int64_t B, int64_t L, int nslices, int ntiles_r
 
 // Pass 1 over the rows that are still masked: one CTA per row slice.
 template <typename DT>
-__global__ void __launch_bounds__(kThreads, 4) unmask_scan_kernel(const UnmaskArgs a) {
+__global__ void __launch_bounds__(kThreads, 3) unmask_scan_kernel(const UnmaskArgs a) {
     extern __shared__ __align__(128) unsigned char ring[];
     __shared__ StreamBars bars;
     const long long row = blockIdx.x / a.nslices;
@@ -60,8 +60,8 @@ __global__ void __launch_bounds__(kThreads, 4) unmask_scan_kernel(const UnmaskAr
     const int slice = blockIdx.x - (int)(row * a.nslices);
     const int b = (int)(row / a.L), l = (int)(row - (long long)b * a.L);
     const DT *rowp = reinterpret_cast<const DT *>(a.logits) + b * a.stride_b + l * a.stride_l;
-    const int s0 = slice * a.slice_elems;
-    const int s1 = min(a.V, s0 + a.slice_elems);
+    int s0, s1;
+    slice_range<DT>(slice, a.nslices, a.ntiles_row, a.V, s0, s1);
     stream_begin(bars);
     grid_launch_dependents();
     DT *trow = reinterpret_cast<DT *>(a.table) + row * (a.ntiles_row + a.nslices) * kThreads;

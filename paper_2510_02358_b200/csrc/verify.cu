@@ -230,15 +230,15 @@ __global__ void __launch_bounds__(kThreads, 4) target_kernel(const VerifyArgs a)
 
 // Streaming path, pass 1: one CTA per row slice (see stream_core.cuh).
 template <typename DT>
-__global__ void __launch_bounds__(kThreads, 4) target_scan_kernel(const VerifyArgs a) {
+__global__ void __launch_bounds__(kThreads, 3) target_scan_kernel(const VerifyArgs a) {
     extern __shared__ __align__(128) unsigned char ring[];
     __shared__ StreamBars bars;
     const long long row = blockIdx.x / a.nslices;
     const int slice = blockIdx.x - (int)(row * a.nslices);
     const int b = (int)(row / a.Lt);
     const DT *rowp = trow_ptr<DT>(a, row);
-    const int s0 = slice * a.slice_elems;
-    const int s1 = min(a.V, s0 + a.slice_elems);
+    int s0, s1;
+    slice_range<DT>(slice, a.nslices, a.ntiles_row, a.V, s0, s1);
     const bool sums = !a.all_greedy && a.mode[b] != 0;
     stream_begin(bars);
     grid_launch_dependents();
