@@ -41,21 +41,25 @@ __device__ __forceinline__ void mbar_arrive(uint64_t *bar) {
 }
 // Bounded wait for the phase with the given parity: gives up after kWaitCycles, or at once when
 // another wait of this CTA has already given up (`abort` non-zero).  False if it gave up.
+__device__ __forceinline__ bool mbar_try(uint32_t bar_addr, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n"
+        ".reg .pred p;\n"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n"
+        "selp.u32 %0, 1, 0, p;\n"
+        "}"
+        : "=r"(ok)
+        : "r"(bar_addr), "r"(parity)
+        : "memory");
+    return ok != 0u;
+}
 __device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, volatile int *abort) {
     const uint32_t a = smem_addr(bar);
+    if (mbar_try(a, parity)) return true;              // the usual case: no clock is read
     const long long t0 = clock64();
     for (;;) {
-        uint32_t ok;
-        asm volatile(
-            "{\n"
-            ".reg .pred p;\n"
-            "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n"
-            "selp.u32 %0, 1, 0, p;\n"
-            "}"
-            : "=r"(ok)
-            : "r"(a), "r"(parity)
-            : "memory");
-        if (ok) return true;
+        if (mbar_try(a, parity)) return true;
         if (*abort || clock64() - t0 > kWaitCycles) return false;
     }
 }
@@ -88,6 +92,11 @@ __device__ __forceinline__ void unpack2(unsigned long long v, float &lo, float &
 __device__ __forceinline__ unsigned long long fma2(unsigned long long a, unsigned long long b, unsigned long long c) {
     unsigned long long d;
     asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+    return d;
+}
+__device__ __forceinline__ unsigned long long mul2(unsigned long long a, unsigned long long b) {
+    unsigned long long d;
+    asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
     return d;
 }
 __device__ __forceinline__ unsigned long long add2(unsigned long long a, unsigned long long b) {
@@ -125,10 +134,9 @@ __device__ __forceinline__ void slice_range(int slice, int nslices, int ntiles_r
     s1 = min(V, (int)((long long)(slice + 1) * ntiles_row / nslices) * TE);
 }
 
-// Issue the bulk copy of tile t of the slice at `src` into its ring stage (one thread).
-__device__ __forceinline__ void issue_tile(const char *src, int nbytes, int t, unsigned char *ring,
+// Issue the bulk copy of tile t of the slice at `src` into its ring stage s = t % kStages (one thread).
+__device__ __forceinline__ void issue_tile(const char *src, int nbytes, int t, int s, unsigned char *ring,
                                            StreamBars &bars) {
-    const int s = t % kStages;
     const uint32_t bytes = (uint32_t)min(kTileBytes, nbytes - t * kTileBytes);
     mbar_expect_tx(&bars.full[s], bytes);
     bulk_load(ring + (size_t)s * kTileBytes, src + (size_t)t * kTileBytes, bytes, &bars.full[s]);
@@ -176,16 +184,21 @@ __device__ void stream_slice(const DT *__restrict__ row, int s0, int s1, bool su
     // Thread 0 also issues the copies, kStages - 1 tiles ahead of the tile being scanned.
     const char *src = reinterpret_cast<const char *>(row + s0);
     if (tid == 0) {
-        for (int tt = 0; tt < min(kStages, ntiles); ++tt) issue_tile(src, nbytes, tt, ring, bars);
+        for (int tt = 0; tt < min(kStages, ntiles); ++tt) issue_tile(src, nbytes, tt, tt, ring, bars);
     }
-    for (int t = 0; t < ntiles; ++t) {
+    int s = 0;                                       // stage of tile t: t % kStages
+    uint32_t ph = 0u;                                // phase parity of tile t in its stage: (t / kStages) & 1
+    DT *tp = tab + tid;                              // this thread's table entry of tile t
+    // the sums of this thread's even and odd logits (register pairs), against the reference exponent c
+    unsigned long long S2 = pack2(0.f, 0.f), T2 = pack2(0.f, 0.f);
+    for (int t = 0; t < ntiles; ++t, tp += kThreads) {
         if (tid == 0 && t >= 1 && t + kStages - 1 < ntiles) {
-            const int tt = t + kStages - 1;           // its stage held tile t - 1
-            if (!mbar_wait(&bars.empty[tt % kStages], ((tt / kStages) - 1) & 1, abort)) bars.timed_out = 1;
-            issue_tile(src, nbytes, tt, ring, bars);
+            // tile t + kStages - 1 goes to the stage that held tile t - 1, once every warp has released it
+            const int es = s == 0 ? kStages - 1 : s - 1;
+            if (!mbar_wait(&bars.empty[es], s == 0 ? ph ^ 1u : ph, abort)) bars.timed_out = 1;
+            issue_tile(src, nbytes, t + kStages - 1, es, ring, bars);
         }
-        const int s = t % kStages;
-        if (!mbar_wait(&bars.full[s], (t / kStages) & 1, abort)) bars.timed_out = 1;
+        if (!mbar_wait(&bars.full[s], ph, abort)) bars.timed_out = 1;
         const int nvec = min(kTileBytes, nbytes - t * kTileBytes) >> 4;
         const uint4 *sp = reinterpret_cast<const uint4 *>(ring + (size_t)s * kTileBytes);
         uint4 v[kVpt];
@@ -217,21 +230,21 @@ __device__ void stream_slice(const DT *__restrict__ row, int s0, int s1, bool su
             }
         }
         const float tm = fmaxf(fmaxf(fmaxf(vm[0], vm[1]), fmaxf(vm[2], vm[3])), fmaxf(vm[4], vm[5]));
-        table_store(tab, t * kThreads + tid, tm);
+        table_store(tp, 0, tm);
         rm = fmaxf(rm, tm);
 
         if (sums) {
             const float ts = tm * kLog2e;             // the reference exponent bounds every logit seen
-            if (ts > c) {
+            if (ts > c) {                              // both halves move to the new reference exponent
                 const float d = c - ts;
                 const float sc = ex2_approx(d);
-                T = (T + S * d) * sc;
-                S = S * sc;
+                const unsigned long long sc2 = pack2(sc, sc);
+                T2 = mul2(fma2(S2, pack2(d, d), T2), sc2);
+                S2 = mul2(S2, sc2);
                 c = ts;
             }
             // two logits per instruction: a = x * log2(e) - c, S += 2^a, T += 2^a * a
             const unsigned long long nc2 = pack2(-c, -c), l2e2 = pack2(kLog2e, kLog2e);
-            unsigned long long S2 = pack2(S, 0.f), T2 = pack2(T, 0.f);
 #pragma unroll
             for (int j = 0; j < kVpt; ++j) {
 #pragma unroll
@@ -244,12 +257,15 @@ __device__ void stream_slice(const DT *__restrict__ row, int s0, int s1, bool su
                     T2 = fma2(e2, a2, T2);
                 }
             }
-            float s0f, s1f, t0f, t1f;
-            unpack2(S2, s0f, s1f);
-            unpack2(T2, t0f, t1f);
-            S = s0f + s1f;
-            T = t0f + t1f;
         }
+        if (++s == kStages) { s = 0; ph ^= 1u; }
+    }
+    {
+        float s0f, s1f, t0f, t1f;
+        unpack2(S2, s0f, s1f);
+        unpack2(T2, t0f, t1f);
+        S = s0f + s1f;
+        T = t0f + t1f;
     }
     table_store(smax, tid, rm);
     if (sums) {
