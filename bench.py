@@ -45,7 +45,7 @@ L2_BYTES = 126 * 1024 * 1024
 HEADLINE = 4
 # DRAM bytes (read + write) per launch of lattice_scan_kernel from one ncu capture of this workload
 # (see profiles/); absent = not captured since the kernel last changed.
-NCU_TRAFFIC_BYTES = {4: 622878208 + 7515392}
+NCU_TRAFFIC_BYTES = {4: 622871296 + 7646464}
 
 
 def measured_peak():
