@@ -13,7 +13,7 @@ namespace dsp {
 constexpr int kThreads = 256;                 // threads per CTA of every streaming kernel
 constexpr int kWarps = kThreads / 32;
 constexpr int kCandCap = 1024;                // candidate buffer entries per CTA (>= 32 slices * DSP_MAX_K)
-constexpr int kTargetCtas = 148 * 6;            // rows are cut into slices until about this many CTAs exist
+constexpr int kTargetCtas = 148;                // rows are cut into slices until about this many CTAs exist (one per SM)
 constexpr int kMaxSlices = 32;                // slices per row a single finaliser merges
 constexpr float kLog2e = 1.44269502162933349609375f;      // fp32 nearest to log2(e)
 constexpr double kLn2 = 0.693147180559945309417232;
