@@ -111,3 +111,30 @@ def test_tree_walk_equals_the_best_single_path_verification(W, L, V):
             assert int(tree.node_depth[b, n]) == i
             assert int(tree.node_parent[b, n]) == (nodes[i - 1] if i else -1)
             assert int(tree.node_token[b, n]) == int(x[b, 1 + (nodes[i - 1] if i else -1)].argmax())
+
+
+def test_nonfinite_rows_flag_existing_nodes_only():
+    """Written by hand: two beams (5,6) and (5,7) give nodes 0:5, 1:6 (child of 0), 2:7 (child of 0);
+    rows 0..3 exist, rows 4.. are unused slots."""
+    beams = torch.tensor([[[5, 6], [5, 7]]], dtype=torch.int32)
+    tree = oracle.beam_tree(beams, torch.tensor([2], dtype=torch.int32))
+    assert tree.n_nodes.tolist() == [3]
+    V, N = 8, 4
+    x = torch.zeros((1, 1 + N, V))
+    x[0, 0, 5] = 1.0          # after the prefix: token 5 -> node 0
+    x[0, 1, 6] = 1.0          # after node 0: token 6 -> node 1
+    x[0, 2, 3] = 1.0          # after node 1 (a leaf): bonus token 3
+    x[0, 3, 2] = 1.0          # after node 2: never walked
+    x[0, 4, :] = float("nan")  # unused slot
+    o = oracle.verify_tree(x, tree, 2)
+    assert o.accepted_len.tolist() == [2] and o.accepted_node[0].tolist() == [0, 1] and o.next_token.tolist() == [3]
+    assert o.row_status.tolist() == [0]                       # the NaN slot has no node: not read, not flagged
+    for val in (float("nan"), float("inf")):
+        y = x.clone()
+        y[0, 3, 0] = val                                      # the row of node 2 exists but the walk never reads it
+        o = oracle.verify_tree(y, tree, 2)
+        assert o.row_status.tolist() == [oracle.NONFINITE_INPUT]
+        assert o.accepted_len.tolist() == [2] and o.next_token.tolist() == [3]      # the walk itself is unchanged
+    y = x.clone()
+    y[0, 3, 0] = -float("inf")                                # masking is legal
+    assert oracle.verify_tree(y, tree, 2).row_status.tolist() == [0]

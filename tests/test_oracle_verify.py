@@ -178,3 +178,69 @@ def test_rejection_discards_the_rest():
             t = o.next_token[b].item()
             pr = torch.softmax(tgt[b, want].double(), 0) - torch.softmax(drf[b, want].double(), 0)
             assert pr[t] > 0
+
+
+def _flag_case(poison_target=None, poison_draft=None, mode=1, path_tok=(0, 1), u=None):
+    """Two batch rows, two positions, V = 4; batch row 1 stays clean as the control."""
+    tgt = torch.tensor([[[2.0, 1.0, 0.0, -1.0], [0.0, 3.0, 1.0, 0.5]]]).repeat(2, 1, 1)
+    drf = torch.tensor([[[1.5, 1.0, 0.5, -1.0], [0.5, 2.0, 1.0, 0.0]]]).repeat(2, 1, 1)
+    if poison_target is not None:
+        i, v, val = poison_target
+        tgt[0, i, v] = val
+    if poison_draft is not None:
+        i, v, val = poison_draft
+        drf[0, i, v] = val
+    path = torch.tensor([list(path_tok)] * 2, dtype=torch.int32)
+    if u is None:
+        u = torch.tensor([[0.0, 0.0, 0.5]] * 2)
+    return oracle.verify(tgt, drf, path, torch.tensor([2, 2], dtype=torch.int32),
+                         torch.full((2,), mode, dtype=torch.uint8), u)
+
+
+@pytest.mark.parametrize("val", [float("nan"), float("inf")])
+def test_nonfinite_target_logit_flags_only_its_batch_row(val):
+    # written by hand: NaN or +inf anywhere in a target row flags the batch row, in either mode,
+    # also in a row the scan never reaches (position 1 after a rejection at position 0)
+    for mode in (0, 1):
+        for pos in (0, 1):
+            o = _flag_case(poison_target=(pos, 3, val), mode=mode)
+            assert o.row_status[0].item() & oracle.NONFINITE_INPUT
+            assert o.row_status[1].item() & oracle.NONFINITE_INPUT == 0
+    o = _flag_case(poison_target=(1, 3, val), mode=0, path_tok=(3, 1))   # greedy: rejected at 0, row 1 unread
+    assert o.accepted_len.tolist() == [0, 0] and o.row_status[0].item() & oracle.NONFINITE_INPUT
+    assert o.next_token.tolist() == [0, 0] and o.row_status[1].item() == 0
+
+
+@pytest.mark.parametrize("val", [float("nan"), float("inf")])
+def test_nonfinite_draft_logit_flags_a_stochastic_row_and_is_not_read_by_a_greedy_one(val):
+    o = _flag_case(poison_draft=(0, 2, val), mode=1)
+    assert o.row_status[0].item() & oracle.NONFINITE_INPUT and o.row_status[1].item() & oracle.NONFINITE_INPUT == 0
+    o = _flag_case(poison_draft=(0, 2, val), mode=0)                      # greedy never looks at the draft logits
+    assert o.row_status[0].item() & oracle.NONFINITE_INPUT == 0
+    assert o.accepted_len.tolist() == [2, 2]                              # path (0, 1) is the target argmax twice
+
+
+def test_minus_inf_is_masking_not_an_error():
+    o = _flag_case(poison_target=(0, 3, -float("inf")), poison_draft=(1, 3, -float("inf")), mode=1)
+    assert o.row_status[0].item() & oracle.NONFINITE_INPUT == 0
+
+
+def test_zero_residual_needs_a_poisoned_row():
+    """In double [p - q]_+ has positive mass whenever a token was rejected (p(y) < q(y) and both sum
+    to one), and a bonus draw is from p itself: the flag is reachable only when the sums are not
+    numbers.  Then the token is the target argmax of that row (written by hand) and both flags are up."""
+    u = torch.tensor([[0.999999, 0.0, 0.5]] * 2)                          # reject position 0 on both rows
+    o = _flag_case(poison_target=(0, 3, float("nan")), mode=1, path_tok=(1, 1), u=u)
+    assert o.accepted_len.tolist() == [0, 0]
+    assert o.row_status[0].item() & oracle.ZERO_RESIDUAL and o.row_status[0].item() & oracle.NONFINITE_INPUT
+    assert o.next_token[0].item() == 0                                    # argmax of (2, 1, 0, NaN): NaN never wins
+    assert o.row_status[1].item() == 0 and o.next_token[1].item() == 0   # clean row: residual is all on token 0
+    # clean rows over many seeds never raise it
+    g = torch.Generator().manual_seed(3)
+    B, L, V = 64, 4, 5
+    drf = torch.randn((B, L, V), generator=g) * 3
+    tgt = drf + torch.randn((B, L, V), generator=g)
+    path = torch.randint(0, V, (B, L), generator=g, dtype=torch.int32)
+    o = oracle.verify(tgt, drf, path, torch.full((B,), L, dtype=torch.int32), torch.ones(B, dtype=torch.uint8),
+                      torch.rand((B, L + 1), generator=g))
+    assert (o.row_status & oracle.ZERO_RESIDUAL == 0).all()
