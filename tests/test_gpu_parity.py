@@ -186,6 +186,31 @@ def test_adl_closed_loop_matches_oracle():
     assert len(seen) >= 2
 
 
+@pytest.mark.parametrize("B", [1, 4])
+def test_paper_default_settings(B):
+    """The settings of the paper's experiments (Sec. 4, implementation details): draft block 30, at most 15
+    candidates per position, beam 3, tau = 0.8, lambda = 0.5, EOS kept, and the controller with
+    k in [20, 30], delta = 10, rho = 0.5; greedy verification for batch 1 (the paper's runs), odd rows
+    stochastic in the batch of 4."""
+    w = wl.CONFIGS[2].scaled(B=B, L=30, K=15, W=3, tau=0.8, lam=0.5, eos_from=23,
+                             verify="greedy" if B == 1 else "mixed")
+    adl = dict(k_min=20, k_max=30, delta=10.0, rho=0.5, granularity=1)
+    st, prm = dsp.dsp_adl_init(**adl)
+    ref = oracle.Adl(**adl)
+    assert st.k == ref.k == 30                               # Algorithm 1: the first block has k_max tokens
+    p = _params(w)
+    for step, fused in ((0, False), (1, True)):
+        inp = wl.make_inputs(w, step=step, device=DEV)
+        g = gpu_step(inp, fused=fused, **p)
+        rep = check_step(g, inp, **p)
+        assert rep["near_accept"] + rep["near_token"] + rep["near_tau"] <= 1
+        assert (g.lat.gen_len == 23).all()                   # EOS is the drafter's top-1 from position 23 on
+        assert (g.lat.cand_count <= 16).all() and (g.lat.cand_count >= 1).all()
+        nxt = dsp.dsp_adl_update(st, prm, g.ver.accepted_len, g.lat.gen_len)
+        assert nxt == ref.update(g.ver.accepted_len, g.lat.gen_len) and 20 <= nxt <= 30
+        assert abs(st.ema_gen - ref.ema_gen) < 1e-12 and abs(st.ema_acc - ref.ema_acc) < 1e-12
+
+
 # ---- the path search alone, on lattices made by hand (sizes and ties the scans rarely give) ----
 def _hand_lattice(B, L, KC, V, seed, *, flat=False, counts=None):
     g = torch.Generator().manual_seed(seed)
