@@ -20,17 +20,12 @@ int32_t verify_impl(const void *target_logits, int32_t dtype, int32_t B, int32_t
                     int32_t *next_token, float *ratio, int32_t *tgt_argmax, float *tgt_lse,
                     uint32_t *row_status, void *workspace, size_t workspace_bytes, cudaStream_t st, int phases);
 
-// dsp_lattice_build that also records `after_scan` (if not null) on the stream once the pass over
-// the draft logits has been enqueued: what follows it in the call no longer reads them.  With
-// `rows_stream` (needs `after_scan`) everything after that pass is enqueued on `rows_stream`
-// instead, which waits for `after_scan`: when the call returns, `rows_stream` carries the rest
-// of the build and `st` is free for work that does not need the lattice.
+// dsp_lattice_build on a CUDA stream (same arguments, checks and errors).
 int32_t lattice_build_impl(const void *draft_logits, int32_t dtype, int32_t B, int32_t L, int32_t V,
                            int64_t stride_b, int64_t stride_l, int32_t K_max, float tau, int32_t eos_id,
                            int32_t *cand_id, float *cand_logit, float *cand_logp, int32_t *cand_count,
                            float *lse, double *lse64, float *entropy, int32_t *gen_len, uint32_t *row_status,
-                           void *workspace, size_t workspace_bytes, cudaStream_t st, cudaEvent_t after_scan,
-                           cudaStream_t rows_stream);
+                           void *workspace, size_t workspace_bytes, cudaStream_t st);
 
 // dsp_cps_search with a choice of SM sharing: with `whole_sm` every CTA of the search asks for
 // enough shared memory to keep the CTAs of a streaming kernel off its SM.

@@ -1,10 +1,10 @@
 // dsp_lattice_build: draft logits -> token lattice (Sec. 3.2 "Lattice and pruning", Eq. 7, Eq. 9).
 //
-// Rows whose layout is 16-byte aligned take two kernels: lattice_scan_kernel streams every row
-// slice once from HBM (one CTA per slice, no block-wide barrier: log-sum-exp terms per warp and
-// a table of per-thread tile maxima, see stream_core.cuh); lattice_rows_kernel (one warp per
-// row, see row_warp.cuh) adds up the sums, selects the exact top-K from the table and finalises
-// the row.
+// Rows whose layout is 16-byte aligned take one kernel: lattice_scan_kernel streams every row
+// slice once from HBM (one CTA per slice, no block-wide barrier in the loop, see stream_core.cuh)
+// and the CTA that is through with a row last adds up the sums, selects the exact top-K
+// (row_engine.cuh) and finalises the row; gen_len and row_status, which belong to a batch row,
+// are prepared before the kernel and updated by every row (atomicMin / atomicOr).
 // Any other layout takes lattice_kernel: one CTA streams one slice element-wise and does the
 // top-K on the way; a row split over several CTAs is finished by whichever CTA arrives last
 // (atomic ticket): no CTA waits.  In both paths the CTA that finishes the last row of a batch
@@ -16,12 +16,14 @@ namespace dsp {
 
 
 // Both paths share the zeroed head; the rest is laid out for the element-wise path (partials,
-// keys) and for the streaming path (wpart, table) over the same bytes: a call takes one path.
+// keys) and for the streaming path (column records and warp sums of rows cut into several
+// slices) over the same bytes: a call takes one path.
 struct LatticeWs {
     size_t off_row_ticket, off_b_ticket, off_b_status, zero_bytes, off_partials, off_keys;
-    size_t off_wpart, off_table, total;
+    RowScratchLayout rs;
+    size_t total;
 };
-static LatticeWs lattice_ws_layout(int64_t B, int64_t L, int nslices, int K, int ntiles_row, size_t es) {
+static LatticeWs lattice_ws_layout(int64_t B, int64_t L, int nslices, int K) {
     LatticeWs w;
     size_t o = 0;
     w.off_row_ticket = o; o += align_up((size_t)(B * L) * 4, 256);
@@ -30,10 +32,8 @@ static LatticeWs lattice_ws_layout(int64_t B, int64_t L, int nslices, int K, int
     w.zero_bytes = o;
     w.off_partials = o;   o += align_up((size_t)(B * L) * nslices * sizeof(SlicePartial), 256);
     w.off_keys = o;       o += align_up((size_t)(B * L) * nslices * K * 8, 256);
-    size_t o2 = w.zero_bytes;
-    w.off_wpart = o2;     o2 += align_up((size_t)(B * L) * nslices * kWarps * sizeof(WarpPartial), 256);
-    w.off_table = o2;     o2 += align_up((size_t)(B * L) * (ntiles_row + nslices) * kThreads * es, 256);
-    w.total = o > o2 ? o : o2;
+    w.rs = row_scratch_layout(w.zero_bytes, B * L, nslices);
+    w.total = o > w.rs.end ? o : w.rs.end;
     return w;
 }
 
@@ -185,7 +185,9 @@ __global__ void __launch_bounds__(kThreads, 4) lattice_kernel(const LatticeArgs 
     lattice_finish<DT, SyncAll>(a, sm, row, slice, b, rowp, c, S, T, 0u);
 }
 
-// Streaming path, pass 1: one CTA per row slice (see stream_core.cuh).
+// Streaming path: one CTA per row slice; the CTA that is through with a row last finalises it
+// (log-sum-exp, entropy, Eq. 7 count, EOS slot, candidate outputs, its part of gen_len (Eq. 9)
+// and row_status).
 template <typename DT>
 __global__ void __launch_bounds__(kThreads, 3) lattice_scan_kernel(const LatticeArgs a) {
     extern __shared__ __align__(128) unsigned char ring[];
@@ -194,51 +196,24 @@ __global__ void __launch_bounds__(kThreads, 3) lattice_scan_kernel(const Lattice
     const int slice = blockIdx.x - (int)(row * a.nslices);
     const int b = (int)(row / a.L), l = (int)(row - (long long)b * a.L);
     const DT *rowp = reinterpret_cast<const DT *>(a.logits) + b * a.stride_b + l * a.stride_l;
-    int s0, s1;
-    slice_range<DT>(slice, a.nslices, a.ntiles_row, a.V, s0, s1);
-    stream_begin(bars);
+    stream_begin(bars, a.nstages);
     grid_launch_dependents();
-    DT *trow = reinterpret_cast<DT *>(a.table) + row * (a.ntiles_row + a.nslices) * kThreads;   // the row's table
-    DT *tab = trow + (long long)(s0 / tile_elems<DT>()) * kThreads;
-    DT *smax = trow + (long long)(a.ntiles_row + slice) * kThreads;
-    stream_slice<DT>(rowp, s0, s1, true, bars, ring, tab, smax, a.wpart + (row * a.nslices + slice) * kWarps);
-    if (threadIdx.x == 0 && bars.timed_out) atomicOr(&a.b_status[b], DSP_ROW_TIMEOUT);
-}
-
-// Streaming path, pass 2: one warp per row (see row_warp.cuh): add up the row's sums, select
-// its exact top-K from the table, finalise it (log-sum-exp, entropy, Eq. 7 count, EOS slot,
-// candidate outputs); the warp that finishes the last row of a batch row also writes gen_len
-// (Eq. 9) and row_status.
-template <typename DT>
-__global__ void __launch_bounds__(kThreads) lattice_rows_kernel(const LatticeArgs a) {
-    __shared__ WarpScratch scratch[kRowWarps];
-    grid_dependency_wait();                            // pass 1 is complete from here on
-    grid_launch_dependents();
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const long long row = (long long)blockIdx.x * kRowWarps + warp;
-    if (row >= (long long)a.B * a.L) return;
-    const int b = (int)(row / a.L), l = (int)(row - (long long)b * a.L);
-    const DT *rowp = reinterpret_cast<const DT *>(a.logits) + b * a.stride_b + l * a.stride_l;
-
-    float c;
-    double S, T;
-    warp_merge_partials(a.wpart + row * a.nslices * kWarps, a.nslices * kWarps, lane, c, S, T);
-    if (T != T && S == S && S < CUDART_INF) warp_redo_sums<DT>(rowp, a.V, lane, c, S, T);
-    const unsigned long long key = warp_select_topk<DT>(
-        rowp, a.V, a.K, reinterpret_cast<const DT *>(a.table) + row * (a.ntiles_row + a.nslices) * kThreads, a.ntiles_row,
-        a.nslices, scratch[warp], lane);
-    warp_finalise_row(a, row, b, key, c, S, T, lane, [&]() { return Elem<DT>::load1(rowp + a.eos_id); });
+    RowResult r;
+    if (!row_engine<DT>(rowp, a.V, a.K, true, row, slice, a.nslices, a.ntiles_row, a.nstages, a.rs, &a.row_status[b],
+                        bars, ring, r))
+        return;
+    warp_finalise_row(a, row, b, l, r.key, r.stats_ok && !r.nonfinite, r.lse, r.mean_x, 0u, threadIdx.x & 31,
+                      [&]() { return Elem<DT>::load1(rowp + a.eos_id); });
 }
 
 template <typename DT>
-static int32_t launch_lattice(LatticeArgs &a, void *workspace, size_t workspace_bytes, cudaStream_t st,
-                              cudaEvent_t after_scan, cudaStream_t rows_stream) {
+static int32_t launch_lattice(LatticeArgs &a, void *workspace, size_t workspace_bytes, cudaStream_t st) {
     const long long nrows = (long long)a.B * a.L;
-    const SlicePlan plan = plan_slices<DT>(nrows, a.V, kTargetCtas);
+    const SlicePlan plan = plan_slices<DT>(nrows, a.V, device_sm_count());
     a.nslices = plan.nslices;
     a.slice_elems = plan.slice_elems;
     a.ntiles_row = (a.V + tile_elems<DT>() - 1) / tile_elems<DT>();
-    const LatticeWs w = lattice_ws_layout(a.B, a.L, a.nslices, a.K, a.ntiles_row, sizeof(DT));
+    const LatticeWs w = lattice_ws_layout(a.B, a.L, a.nslices, a.K);
     if (workspace_bytes < w.total) return DSP_ERR_WORKSPACE;
     char *ws = reinterpret_cast<char *>(workspace);
     a.row_ticket = reinterpret_cast<unsigned *>(ws + w.off_row_ticket);
@@ -246,37 +221,29 @@ static int32_t launch_lattice(LatticeArgs &a, void *workspace, size_t workspace_
     a.b_status = reinterpret_cast<unsigned *>(ws + w.off_b_status);
     a.partials = reinterpret_cast<SlicePartial *>(ws + w.off_partials);
     a.keys = reinterpret_cast<unsigned long long *>(ws + w.off_keys);
-    a.wpart = reinterpret_cast<WarpPartial *>(ws + w.off_wpart);
-    a.table = ws + w.off_table;
-    DSP_CUDA_TRY(cudaMemsetAsync(ws, 0, w.zero_bytes, st));
+    a.rs.row_ticket = a.row_ticket;
+    a.rs.cols = reinterpret_cast<uint2 *>(ws + w.rs.off_cols);
+    a.rs.wpart = reinterpret_cast<WarpPartial *>(ws + w.rs.off_wpart);
+    // tickets and status words of the workspace start at zero, row_status at 0, gen_len at L
+    PrepareArgs prep;
+    prep.zero_a = reinterpret_cast<uint32_t *>(ws); prep.n_a = (long long)(w.zero_bytes / 4);
+    prep.zero_b = a.row_status; prep.n_b = a.B;
+    prep.fill = a.gen_len; prep.n_fill = a.B; prep.fill_value = a.L;
+    DSP_CUDA_TRY(launch_prepare(prep, st));
     const long long nblocks = nrows * a.nslices;
     if (nblocks > 0x7FFFFFFFLL) return DSP_ERR_UNSUPPORTED;
-    if (a.nslices * kWarps <= kThreads && nrows <= 0x7FFFFFFFLL &&
-        stream_layout_ok<DT>(a.logits, a.V, a.stride_b, a.stride_l)) {
+    if (a.nslices <= kMaxSlices && nrows <= 0x7FFFFFFFLL && stream_layout_ok<DT>(a.logits, a.V, a.stride_b, a.stride_l)) {
         static RingSmemDone smem_done;                       // one per element type
         DSP_CUDA_TRY(allow_ring_smem(lattice_scan_kernel<DT>, smem_done));
+        a.nstages = ring_stages(nblocks);
         const ProfileEvents pe = g_profile[DSP_PROFILE_LATTICE_SCAN];
         if (pe.start) DSP_CUDA_TRY(cudaEventRecord(pe.start, st));
-        lattice_scan_kernel<DT><<<(unsigned)nblocks, kThreads, kRingBytes, st>>>(a);
-        DSP_CUDA_TRY(cudaGetLastError());
+        // the streaming kernel may start beside the preparation: it waits for it after its rows are streamed
+        DSP_CUDA_TRY(launch_dependent(lattice_scan_kernel<DT>, (unsigned)nblocks, kThreads, (size_t)a.nstages * kTileBytes, st, a,
+                                      !pe.start && short_kernel_follows_early(st, nrows)));
         if (pe.stop) DSP_CUDA_TRY(cudaEventRecord(pe.stop, st));
-        cudaStream_t rs = st;
-        if (after_scan) {
-            DSP_CUDA_TRY(cudaEventRecord(after_scan, st));
-            if (rows_stream) {                            // pass 2 follows the scan on the other stream
-                DSP_CUDA_TRY(cudaStreamWaitEvent(rows_stream, after_scan, 0));
-                rs = rows_stream;
-            }
-            after_scan = nullptr;
-        }
-        DSP_CUDA_TRY(launch_dependent(lattice_rows_kernel<DT>, (unsigned)((nrows + kRowWarps - 1) / kRowWarps), kThreads, 0, rs, a,
-                                      rows_follow_early(rs, nblocks)));
     } else {
         lattice_kernel<DT><<<(unsigned)nblocks, kThreads, 0, st>>>(a);
-    }
-    if (after_scan) {
-        DSP_CUDA_TRY(cudaEventRecord(after_scan, st));
-        if (rows_stream) DSP_CUDA_TRY(cudaStreamWaitEvent(rows_stream, after_scan, 0));
     }
     DSP_CUDA_TRY(cudaGetLastError());
     return DSP_OK;
@@ -284,9 +251,8 @@ static int32_t launch_lattice(LatticeArgs &a, void *workspace, size_t workspace_
 
 template <typename DT>
 static size_t lattice_ws_bytes(int B, int L, int V, int K) {
-    const SlicePlan plan = plan_slices<DT>((long long)B * L, V, kTargetCtas);
-    const int ntiles_row = (V + tile_elems<DT>() - 1) / tile_elems<DT>();
-    return lattice_ws_layout(B, L, plan.nslices, K, ntiles_row, sizeof(DT)).total;
+    const SlicePlan plan = plan_slices<DT>((long long)B * L, V, device_sm_count());
+    return lattice_ws_layout(B, L, plan.nslices, K).total;
 }
 
 }  // namespace dsp
@@ -319,8 +285,7 @@ int32_t dsp::lattice_build_impl(const void *draft_logits, int32_t dtype,
                                 int32_t *cand_id, float *cand_logit, float *cand_logp,
                                 int32_t *cand_count, float *lse, double *lse64, float *entropy,
                                 int32_t *gen_len, uint32_t *row_status,
-                                void *workspace, size_t workspace_bytes, cudaStream_t st, cudaEvent_t after_scan,
-                                cudaStream_t rows_stream) {
+                                void *workspace, size_t workspace_bytes, cudaStream_t st) {
     const int32_t rc = check_lattice_shape(B, L, V, dtype, K_max);
     if (rc != DSP_OK) return rc;
     if (B == 0) return DSP_OK;
@@ -346,8 +311,8 @@ int32_t dsp::lattice_build_impl(const void *draft_logits, int32_t dtype,
     a.cand_id = cand_id; a.cand_logit = cand_logit; a.cand_logp = cand_logp;
     a.cand_count = cand_count; a.lse = lse; a.lse64 = lse64; a.entropy = entropy;
     a.gen_len = gen_len; a.row_status = row_status;
-    return dtype == DSP_BF16 ? launch_lattice<__nv_bfloat16>(a, workspace, workspace_bytes, st, after_scan, rows_stream)
-                             : launch_lattice<float>(a, workspace, workspace_bytes, st, after_scan, rows_stream);
+    return dtype == DSP_BF16 ? launch_lattice<__nv_bfloat16>(a, workspace, workspace_bytes, st)
+                             : launch_lattice<float>(a, workspace, workspace_bytes, st);
 }
 
 extern "C" int32_t dsp_lattice_build(const void *draft_logits, int32_t dtype,
@@ -360,7 +325,7 @@ extern "C" int32_t dsp_lattice_build(const void *draft_logits, int32_t dtype,
                                      void *workspace, size_t workspace_bytes, dsp_stream_t stream) {
     return lattice_build_impl(draft_logits, dtype, B, L, V, stride_b, stride_l, K_max, tau, eos_id, cand_id,
                               cand_logit, cand_logp, cand_count, lse, lse64, entropy, gen_len, row_status,
-                              workspace, workspace_bytes, reinterpret_cast<cudaStream_t>(stream), nullptr, nullptr);
+                              workspace, workspace_bytes, reinterpret_cast<cudaStream_t>(stream));
 }
 
 // ---- dsp_lattice_build_static: the same build for callers that cannot allocate ----------------

@@ -1,8 +1,8 @@
 // What the finish of a lattice row needs, shared by the kernels that finish rows: the lattice
-// build's own pass 2 (lattice.cu) and the merge of vocabulary shards (shard.cu).
+// build's streaming kernel (lattice.cu) and the merge of vocabulary shards (shard.cu).
 #pragma once
 
-#include "row_warp.cuh"
+#include "row_engine.cuh"
 
 namespace dsp {
 
@@ -29,33 +29,34 @@ struct LatticeArgs {
     unsigned *b_status;       // [B]     zeroed per call
     SlicePartial *partials;   // [B*L, nslices]               (element-wise path)
     unsigned long long *keys; // [B*L, nslices, K]            (element-wise path)
-    WarpPartial *wpart;       // [B*L, nslices, kWarps]       (streaming path)
-    void *table;              // [B*L, ntiles_row + nslices, kThreads]  (streaming path), element type of the logits
+    RowScratch rs;            // records of rows cut into several slices (streaming path)
     int ntiles_row;           // tiles of a whole row
+    int nstages;              // ring depth of the streaming kernel
 };
 
 // Finish one row by one warp from its best keys (`key`: one per lane, descending, 0 = none; the
-// first min(K, #finite) count) and its whole-row sums (c, S, T): log-sum-exp, entropy, Eq. 7
-// count, EOS slot (`eos_logit()` fetches the row's EOS logit when it is needed), candidate
-// outputs; the warp that finishes the last row of a batch row also writes gen_len (Eq. 9) and
-// row_status.
+// first min(K, #finite) count) and its log-sum-exp and mean logit (`stats_ok` false: the sums do
+// not describe a finite row): entropy, Eq. 7 count, EOS slot (`eos_logit()` fetches the row's EOS
+// logit when it is needed), candidate outputs.  The batch row's outputs take part of every row:
+// status flags (`flags` and DSP_ROW_NONFINITE_INPUT) are OR-ed into row_status[b] and a row whose
+// best token is EOS lowers gen_len[b] to its position (Eq. 9); both were prepared before the
+// kernel (row_status 0, gen_len L), so no row waits for another.
 template <typename EosLogit>
-__device__ __forceinline__ void warp_finalise_row(const LatticeArgs &a, long long row, int b, unsigned long long key,
-                                                  float c, double S, double T, int lane, EosLogit eos_logit) {
+__device__ __forceinline__ void warp_finalise_row(const LatticeArgs &a, long long row, int b, int l,
+                                                  unsigned long long key, bool stats_ok, double lse, double mean_x,
+                                                  unsigned flags, int lane, EosLogit eos_logit) {
     const int nk = __popc(__ballot_sync(0xFFFFFFFFu, key != 0ull && lane < a.K));
-
-    double lse, mean_x;
-    const bool ok = row_log_stats(c, S, T, lse, mean_x) && nk > 0;
+    const bool ok = stats_ok && nk > 0;
     int count = nk;
     if (a.tau > 0.f && a.tau <= 1.f && ok) {           // Eq. 7 on full-vocabulary probabilities
-        const double p = lane < nk ? exp((double)key_value(key) - lse) : 0.0;
-        const double tau = (double)a.tau;
-        double cum = 0.0;
-        bool found = false;
-        for (int k = 0; k < nk; ++k) {                 // in rank order, every lane alike
-            cum += __shfl_sync(0xFFFFFFFFu, p, k);
-            if (!found && cum >= tau) { count = k + 1; found = true; }
+        double cum = lane < nk ? exp((double)key_value(key) - lse) : 0.0;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {             // cumulative mass in rank order
+            const double up = __shfl_up_sync(0xFFFFFFFFu, cum, o);
+            if (lane >= o) cum += up;
         }
+        const unsigned reached = __ballot_sync(0xFFFFFFFFu, lane < nk && cum >= (double)a.tau);
+        if (reached) count = __ffs(reached);
     }
     int eos_slot = -1;
     float eos_x = 0.f;
@@ -71,7 +72,9 @@ __device__ __forceinline__ void warp_finalise_row(const LatticeArgs &a, long lon
         if (a.lse) a.lse[row] = (float)lse;
         a.lse64[row] = lse;
         if (a.entropy) a.entropy[row] = (float)(lse - mean_x);
-        if (!ok) atomicOr(&a.b_status[b], DSP_ROW_NONFINITE_INPUT);
+        const unsigned fl = flags | (ok ? 0u : (unsigned)DSP_ROW_NONFINITE_INPUT);
+        if (fl) atomicOr(&a.row_status[b], fl);
+        if (a.eos_id >= 0 && nk > 0 && key_id(key) == a.eos_id) atomicMin(&a.gen_len[b], l);   // Eq. 9
     }
     for (int slot = lane; slot < a.KC; slot += 32) {      // slot 32 can only be the EOS slot
         const unsigned long long ks = key;                  // slot == lane whenever slot < count <= 32
@@ -90,27 +93,6 @@ __device__ __forceinline__ void warp_finalise_row(const LatticeArgs &a, long lon
         a.cand_id[o] = id;
         a.cand_logit[o] = x;
         a.cand_logp[o] = lp;
-    }
-    // ---- last row of this batch row: generation length (Eq. 9) and status ----
-    __threadfence();
-    __syncwarp();
-    unsigned ticket = 0;
-    if (lane == 0) ticket = atomicAdd(&a.b_ticket[b], 1u);
-    ticket = __shfl_sync(0xFFFFFFFFu, ticket, 0);
-    if (ticket != (unsigned)a.L - 1) return;
-    __threadfence();
-    int g = a.L;
-    if (a.eos_id >= 0) {
-        for (int i0 = 0; i0 < a.L && g == a.L; i0 += 32) {
-            const int i = i0 + lane;
-            const bool eos = i < a.L && __ldcg(&a.cand_id[((long long)b * a.L + i) * a.KC]) == a.eos_id;
-            const unsigned m = __ballot_sync(0xFFFFFFFFu, eos);
-            if (m) g = i0 + __ffs(m) - 1;
-        }
-    }
-    if (lane == 0) {
-        a.gen_len[b] = g;
-        a.row_status[b] = atomicOr(&a.b_status[b], 0u);
     }
 }
 

@@ -25,29 +25,48 @@ struct ShardArgs {
     dsp_shard_sums *sums;     // [B,L]
     unsigned long long *keys; // [B,L,K_max]
     uint32_t *shard_status;   // [B]
-    int streaming, nslices, slice_elems, ntiles_row;
-    unsigned *b_status;       // [B]  zeroed per call
-    unsigned *b_ticket;       // [B]  zeroed per call
-    WarpPartial *wpart;
-    void *table;
+    int nslices, slice_elems, ntiles_row, nstages;
+    RowScratch rs;            // records of rows cut into several slices (streaming path)
 };
 
 struct ShardWs {
-    size_t off_b_status, off_b_ticket, zero_bytes, off_wpart, off_table, total;
+    size_t off_row_ticket, zero_bytes;
+    RowScratchLayout rs;
+    size_t total;
 };
-static ShardWs shard_ws_layout(int64_t B, int64_t L, int nslices, int ntiles_row, size_t es) {
+static ShardWs shard_ws_layout(int64_t B, int64_t L, int nslices) {
     ShardWs w;
     size_t o = 0;
-    w.off_b_status = o; o += align_up((size_t)B * 4, 256);
-    w.off_b_ticket = o; o += align_up((size_t)B * 4, 256);
+    w.off_row_ticket = o; o += align_up((size_t)(B * L) * 4, 256);
     w.zero_bytes = o;
-    w.off_wpart = o;    o += align_up((size_t)(B * L) * nslices * kWarps * sizeof(WarpPartial), 256);
-    w.off_table = o;    o += align_up((size_t)(B * L) * (ntiles_row + nslices) * kThreads * es, 256);
-    w.total = o;
+    w.rs = row_scratch_layout(o, B * L, nslices);
+    w.total = w.rs.end;
     return w;
 }
 
-// Pass 1 over the slice's rows: one CTA per row slice (stream_core.cuh).
+// The record of one row of the slice, written by one warp from the row's best keys and sums.
+// (shard_status is prepared as 0 before the kernel; a wait that ran out is OR-ed into it.)
+template <typename DT>
+__device__ __forceinline__ void shard_write_row(const ShardArgs &a, long long row, int b, int l, const DT *rowp,
+                                                unsigned long long key, float c, double S, double T, int lane) {
+    // keys carry global token ids
+    if (lane < a.K_max) {
+        unsigned long long out = 0ull;
+        if (lane < a.K && key != 0ull) out = make_key(key_value(key), key_id(key) + a.vocab_offset);
+        a.keys[row * a.K_max + lane] = out;
+    }
+    if (lane == 0) {
+        dsp_shard_sums r;
+        r.S = S; r.T = T; r.c = c;
+        int probe = a.eos_id;                  // the one token whose logit the record carries
+        if (a.path) probe = (l < a.Lp && l < __ldg(&a.path_len[b])) ? __ldg(&a.path[(long long)b * a.Lp + l]) : -1;
+        const int e = probe - a.vocab_offset;
+        r.eos_logit = (probe >= 0 && e >= 0 && e < a.V) ? Elem<DT>::load1(rowp + e) : CUDART_NAN_F;
+        a.sums[row] = r;
+    }
+}
+
+// Streaming path: one CTA per row slice; the CTA that is through with a row last writes its record.
 template <typename DT>
 __global__ void __launch_bounds__(kThreads, 3) shard_scan_kernel(const ShardArgs a) {
     extern __shared__ __align__(128) unsigned char ring[];
@@ -56,15 +75,12 @@ __global__ void __launch_bounds__(kThreads, 3) shard_scan_kernel(const ShardArgs
     const int slice = blockIdx.x - (int)(row * a.nslices);
     const int b = (int)(row / a.L), l = (int)(row - (long long)b * a.L);
     const DT *rowp = reinterpret_cast<const DT *>(a.logits) + b * a.stride_b + l * a.stride_l;
-    int s0, s1;
-    slice_range<DT>(slice, a.nslices, a.ntiles_row, a.V, s0, s1);
-    stream_begin(bars);
-    grid_launch_dependents();
-    DT *trow = reinterpret_cast<DT *>(a.table) + row * (a.ntiles_row + a.nslices) * kThreads;
-    DT *tab = trow + (long long)(s0 / tile_elems<DT>()) * kThreads;
-    DT *smax = trow + (long long)(a.ntiles_row + slice) * kThreads;
-    stream_slice<DT>(rowp, s0, s1, true, bars, ring, tab, smax, a.wpart + (row * a.nslices + slice) * kWarps);
-    if (threadIdx.x == 0 && bars.timed_out) atomicOr(&a.b_status[b], DSP_ROW_TIMEOUT);
+    stream_begin(bars, a.nstages);
+    RowResult r;
+    if (!row_engine<DT>(rowp, a.V, a.K, true, row, slice, a.nslices, a.ntiles_row, a.nstages, a.rs, &a.shard_status[b],
+                        bars, ring, r))
+        return;
+    shard_write_row<DT>(a, row, b, l, rowp, r.key, r.c, r.S, r.T, threadIdx.x & 31);
 }
 
 // Sums and exact top-K of a row that cannot be streamed, element by element, by one warp.
@@ -110,50 +126,18 @@ __device__ unsigned long long warp_row_elementwise(const DT *__restrict__ row, i
     return best;
 }
 
-// Pass 2: one warp per row writes the slice's record.
+// Layouts that cannot be streamed: one warp per row, element by element.
 template <typename DT>
 __global__ void __launch_bounds__(kThreads) shard_rows_kernel(const ShardArgs a) {
-    __shared__ WarpScratch scratch[kRowWarps];
-    grid_dependency_wait();                            // pass 1 is complete from here on
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const long long row = (long long)blockIdx.x * kRowWarps + warp;
+    const long long row = (long long)blockIdx.x * kWarps + warp;
     if (row >= (long long)a.B * a.L) return;
     const int b = (int)(row / a.L), l = (int)(row - (long long)b * a.L);
     const DT *rowp = reinterpret_cast<const DT *>(a.logits) + b * a.stride_b + l * a.stride_l;
     float c;
     double S, T;
-    unsigned long long key;
-    if (a.streaming) {
-        warp_merge_partials(a.wpart + row * a.nslices * kWarps, a.nslices * kWarps, lane, c, S, T);
-        if (T != T && S == S && S < CUDART_INF) warp_redo_sums<DT>(rowp, a.V, lane, c, S, T);
-        key = warp_select_topk<DT>(rowp, a.V, a.K,
-                                   reinterpret_cast<const DT *>(a.table) + row * (a.ntiles_row + a.nslices) * kThreads,
-                                   a.ntiles_row, a.nslices, scratch[warp], lane);
-    } else {
-        key = warp_row_elementwise<DT>(rowp, a.V, a.K, lane, c, S, T);
-    }
-    // keys carry global token ids
-    if (lane < a.K_max) {
-        unsigned long long out = 0ull;
-        if (lane < a.K && key != 0ull) out = make_key(key_value(key), key_id(key) + a.vocab_offset);
-        a.keys[row * a.K_max + lane] = out;
-    }
-    if (lane == 0) {
-        dsp_shard_sums r;
-        r.S = S; r.T = T; r.c = c;
-        int probe = a.eos_id;                  // the one token whose logit the record carries
-        if (a.path) probe = (l < a.Lp && l < __ldg(&a.path_len[b])) ? __ldg(&a.path[(long long)b * a.Lp + l]) : -1;
-        const int e = probe - a.vocab_offset;
-        r.eos_logit = (probe >= 0 && e >= 0 && e < a.V) ? Elem<DT>::load1(rowp + e) : CUDART_NAN_F;
-        a.sums[row] = r;
-    }
-    // the warp finishing a batch row's last row publishes its status (time-outs of pass 1)
-    __threadfence();
-    __syncwarp();
-    unsigned ticket = 0;
-    if (lane == 0) ticket = atomicAdd(&a.b_ticket[b], 1u);
-    ticket = __shfl_sync(0xFFFFFFFFu, ticket, 0);
-    if (ticket == (unsigned)a.L - 1 && lane == 0) a.shard_status[b] = atomicOr(&a.b_status[b], 0u);
+    const unsigned long long key = warp_row_elementwise<DT>(rowp, a.V, a.K, lane, c, S, T);
+    shard_write_row<DT>(a, row, b, l, rowp, key, c, S, T, lane);
 }
 
 struct MergeArgs {
@@ -169,7 +153,7 @@ __global__ void __launch_bounds__(kThreads) shard_merge_kernel(const MergeArgs m
     const LatticeArgs &a = m.lat;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const long long nrows = (long long)a.B * a.L;
-    const long long row = (long long)blockIdx.x * kRowWarps + warp;
+    const long long row = (long long)blockIdx.x * kWarps + warp;
     if (row >= nrows) return;
     const int b = (int)(row / a.L);
     // sums against the largest reference exponent, in slice order per lane, then a shuffle tree
@@ -202,49 +186,51 @@ __global__ void __launch_bounds__(kThreads) shard_merge_kernel(const MergeArgs m
         const unsigned long long k = lane < a.K_max ? m.keys[(g * nrows + row) * a.K_max + lane] : 0ull;
         best = g == 0 ? k : merge_top32(best, k, lane);
     }
-    if (lane == 0) {
-        unsigned st = 0;
-        for (int g = 0; g < m.G; ++g) st |= m.shard_status[(long long)g * a.B + b];
-        if (st) atomicOr(&a.b_status[b], st);
-    }
-    __syncwarp();
-    warp_finalise_row(a, row, b, best, cm, S, T, lane, [&]() { return eos_x; });
+    unsigned st = 0;                                   // the slices' flags of this batch row (time-outs)
+    for (int g = lane; g < m.G; g += 32) st |= m.shard_status[(long long)g * a.B + b];
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) st |= __shfl_xor_sync(0xFFFFFFFFu, st, o);
+    double lse, mean_x;
+    const bool ok = row_log_stats(cm, S, T, lse, mean_x);
+    warp_finalise_row(a, row, b, (int)(row - (long long)b * a.L), best, ok, lse, mean_x, st, lane, [&]() { return eos_x; });
 }
 
 template <typename DT>
 static int32_t launch_shard(ShardArgs &a, void *workspace, size_t workspace_bytes, cudaStream_t st) {
     const long long nrows = (long long)a.B * a.L;
-    const SlicePlan plan = plan_slices<DT>(nrows, a.V, kTargetCtas);
+    const SlicePlan plan = plan_slices<DT>(nrows, a.V, device_sm_count());
     a.nslices = plan.nslices;
     a.slice_elems = plan.slice_elems;
     a.ntiles_row = (a.V + tile_elems<DT>() - 1) / tile_elems<DT>();
-    const ShardWs w = shard_ws_layout(a.B, a.L, a.nslices, a.ntiles_row, sizeof(DT));
+    const ShardWs w = shard_ws_layout(a.B, a.L, a.nslices);
     if (workspace_bytes < w.total) return DSP_ERR_WORKSPACE;
     unsigned char *ws = static_cast<unsigned char *>(workspace);
-    a.b_status = reinterpret_cast<unsigned *>(ws + w.off_b_status);
-    a.b_ticket = reinterpret_cast<unsigned *>(ws + w.off_b_ticket);
-    a.wpart = reinterpret_cast<WarpPartial *>(ws + w.off_wpart);
-    a.table = ws + w.off_table;
-    DSP_CUDA_TRY(cudaMemsetAsync(ws, 0, w.zero_bytes, st));
+    a.rs.row_ticket = reinterpret_cast<unsigned *>(ws + w.off_row_ticket);
+    a.rs.cols = reinterpret_cast<uint2 *>(ws + w.rs.off_cols);
+    a.rs.wpart = reinterpret_cast<WarpPartial *>(ws + w.rs.off_wpart);
+    PrepareArgs prep = PrepareArgs();                    // row tickets and shard_status start at zero
+    prep.zero_a = reinterpret_cast<uint32_t *>(ws); prep.n_a = (long long)(w.zero_bytes / 4);
+    prep.zero_b = a.shard_status; prep.n_b = a.B;
+    DSP_CUDA_TRY(launch_prepare(prep, st));
     const long long nblocks = nrows * a.nslices;
     if (nblocks > 0x7FFFFFFFLL) return DSP_ERR_UNSUPPORTED;
-    a.streaming = a.nslices * kWarps <= kThreads && stream_layout_ok<DT>(a.logits, a.V, a.stride_b, a.stride_l);
-    if (a.streaming) {
+    if (a.nslices <= kMaxSlices && stream_layout_ok<DT>(a.logits, a.V, a.stride_b, a.stride_l)) {
         static RingSmemDone smem_done;                   // one per element type
         DSP_CUDA_TRY(allow_ring_smem(shard_scan_kernel<DT>, smem_done));
-        shard_scan_kernel<DT><<<(unsigned)nblocks, kThreads, kRingBytes, st>>>(a);
-        DSP_CUDA_TRY(cudaGetLastError());
+        a.nstages = ring_stages(nblocks);
+        DSP_CUDA_TRY(launch_dependent(shard_scan_kernel<DT>, (unsigned)nblocks, kThreads, (size_t)a.nstages * kTileBytes, st, a,
+                                      short_kernel_follows_early(st, nrows)));
+    } else {
+        shard_rows_kernel<DT><<<(unsigned)((nrows + kWarps - 1) / kWarps), kThreads, 0, st>>>(a);
     }
-    DSP_CUDA_TRY(launch_dependent(shard_rows_kernel<DT>, (unsigned)((nrows + kRowWarps - 1) / kRowWarps), kThreads, 0, st, a,
-                                  a.streaming && rows_follow_early(st, nblocks)));
+    DSP_CUDA_TRY(cudaGetLastError());
     return DSP_OK;
 }
 
 template <typename DT>
 static size_t shard_ws_bytes(int B, int L, int V) {
-    const SlicePlan plan = plan_slices<DT>((long long)B * L, V, kTargetCtas);
-    const int ntiles_row = (V + tile_elems<DT>() - 1) / tile_elems<DT>();
-    return shard_ws_layout(B, L, plan.nslices, ntiles_row, sizeof(DT)).total;
+    const SlicePlan plan = plan_slices<DT>((long long)B * L, V, device_sm_count());
+    return shard_ws_layout(B, L, plan.nslices).total;
 }
 
 }  // namespace dsp
@@ -362,13 +348,13 @@ extern "C" int32_t dsp_lattice_merge(int32_t G, const dsp_shard_sums *sums, cons
     a.cand_id = cand_id; a.cand_logit = cand_logit; a.cand_logp = cand_logp;
     a.cand_count = cand_count; a.lse = lse; a.lse64 = lse64; a.entropy = entropy;
     a.gen_len = gen_len; a.row_status = row_status;
-    unsigned char *ws = static_cast<unsigned char *>(workspace);
-    a.b_ticket = reinterpret_cast<unsigned *>(ws);
-    a.b_status = reinterpret_cast<unsigned *>(ws + need / 2);
     cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
-    DSP_CUDA_TRY(cudaMemsetAsync(ws, 0, need, st));
+    PrepareArgs prep = PrepareArgs();                    // every row adds its part to row_status and gen_len
+    prep.zero_a = row_status; prep.n_a = B;
+    prep.fill = gen_len; prep.n_fill = B; prep.fill_value = L;
+    DSP_CUDA_TRY(launch_prepare(prep, st));
     const long long nrows = (long long)B * L;
-    shard_merge_kernel<<<(unsigned)((nrows + kRowWarps - 1) / kRowWarps), kThreads, 0, st>>>(m);
+    shard_merge_kernel<<<(unsigned)((nrows + kWarps - 1) / kWarps), kThreads, 0, st>>>(m);
     DSP_CUDA_TRY(cudaGetLastError());
     return DSP_OK;
 }

@@ -3,14 +3,13 @@
 // Same kernels and results as dsp_lattice_build, dsp_cps_search and dsp_verify called one after
 // the other.  What the single call adds is overlap: the statistics of the target rows (argmax,
 // log-sum-exp) need only the target logits, so the pass over the target logits runs beside the
-// lattice's finish and the path search, which are short, latency-bound kernels that leave HBM
-// idle; the decisions (acceptance scan, residual draw) wait for both sides.  The two sides run on
-// the caller's stream and on a stream of the library.  When the passes are long (their grid is
-// several times what the SMs hold at once) the library's stream, which has the highest priority
-// the device offers, takes the lattice's finish and the search: their few CTAs get the next free
-// places on the SMs instead of queueing behind the target pass's grid, and the search keeps its
-// SMs to itself (see cps_search_impl), because sharing one with streaming CTAs makes it 2.5 times
-// slower.
+// pass over the draft logits and the path search; the decisions (acceptance scan, residual draw)
+// wait for both sides.  The two sides run on the caller's stream and on a stream of the library.
+// When the passes are long (their grid is several times what the SMs hold at once) the library's
+// stream, which has the highest priority the device offers, takes the build and the search: the
+// two passes then run back to back without a gap or a drained last wave between them, and the
+// search's few CTAs get the next free places on the SMs instead of queueing behind the target
+// pass's grid.
 #include <mutex>
 
 #include "dsp_common.cuh"
@@ -91,27 +90,21 @@ extern "C" int32_t dsp_draft_verify_step(
                                path_score, beam_ids, beam_score, beam_cum, row_status, s, whole_sm);
     };
     int32_t rc2 = DSP_OK;
-    if (long_pass) {
-        // The pass over the target logits follows the pass over the draft logits on the caller's
-        // stream; the lattice's finish and the search go to the second stream, whose priority lets
-        // their CTAs in ahead of the target pass's grid.
-        rc = lattice_build_impl(draft_logits, dtype, B, L, V, dstride_b, dstride_l, K_max, tau, eos_id, cand_id,
-                                cand_logit, cand_logp, cand_count, lse, lse64, entropy, gen_len, row_status,
-                                lattice_workspace, lattice_workspace_bytes, st, side->fork, side->stream);
-        if (rc != DSP_OK) return rc;
-        rc = stats(st);
-        if (rc == DSP_OK) rc2 = search(side->stream);
-    } else {
-        // Short passes leave SMs free anyway: the build and the search stay on the caller's stream
-        // (no event between them) and the target statistics take the second stream.
-        rc = lattice_build_impl(draft_logits, dtype, B, L, V, dstride_b, dstride_l, K_max, tau, eos_id, cand_id,
-                                cand_logit, cand_logp, cand_count, lse, lse64, entropy, gen_len, row_status,
-                                lattice_workspace, lattice_workspace_bytes, st, side->fork, nullptr);
-        if (rc != DSP_OK) return rc;
-        DSP_CUDA_TRY(cudaStreamWaitEvent(side->stream, side->fork, 0));
-        rc = stats(side->stream);
-        if (rc == DSP_OK) rc2 = search(st);
-    }
+    // The two sides start together: the second stream takes up where the caller's stream stands.
+    DSP_CUDA_TRY(cudaEventRecord(side->fork, st));
+    DSP_CUDA_TRY(cudaStreamWaitEvent(side->stream, side->fork, 0));
+    // Long passes: the build and the search go to the second stream, whose priority hands its CTAs
+    // out first: the draft logits stream first, the target pass's CTAs fill the places the draft
+    // pass's last wave leaves free, and the search gets in ahead of the target pass's grid.
+    // Short passes leave SMs free anyway: the build and the search stay on the caller's stream
+    // (no event on their way) and the target statistics take the second stream.
+    cudaStream_t draft_side = long_pass ? side->stream : st;
+    cudaStream_t target_side = long_pass ? st : side->stream;
+    rc = lattice_build_impl(draft_logits, dtype, B, L, V, dstride_b, dstride_l, K_max, tau, eos_id, cand_id,
+                            cand_logit, cand_logp, cand_count, lse, lse64, entropy, gen_len, row_status,
+                            lattice_workspace, lattice_workspace_bytes, draft_side);
+    if (rc == DSP_OK) rc = stats(target_side);
+    if (rc == DSP_OK) rc2 = search(draft_side);
     // whatever happened, the caller's stream joins the second stream again
     cudaError_t e = cudaEventRecord(side->join, side->stream);
     if (e == cudaSuccess) e = cudaStreamWaitEvent(st, side->join, 0);

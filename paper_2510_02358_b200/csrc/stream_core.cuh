@@ -1,17 +1,15 @@
-// Streaming pass for rows whose start, strides and length are multiples of 16 bytes, and the
-// selection of the exact top-K from what it leaves behind.
+// Streaming pass over row slices whose start, strides and length are multiples of 16 bytes.
 //
-// Pass 1 (stream_slice, one CTA per row slice): the slice streams through a ring of
-// shared-memory stages by bulk asynchronous copies (cp.async.bulk, completion counted on an
-// mbarrier per stage, no multicast) that one thread issues ahead; all kThreads threads read each
-// stage with one 128-bit shared load per vector and do the arithmetic from registers.  The loop
-// has no block-wide barrier.  It leaves in global memory, per row: a table with, for every tile
-// and thread, the largest logit of the thread's kVpt vectors of that tile, and per slice and
-// warp the log-sum-exp terms.
-//
-// Pass 2 (one warp per row, row_warp.cuh, run by the kernels in lattice.cu / verify.cu) adds up
-// the sums and picks the exact top-K from the table.  Results are the same as scan_slice's
-// (scan_core.cuh).
+// stream_slice (one CTA per row slice): the slice streams through a ring of shared-memory stages
+// by bulk asynchronous copies (cp.async.bulk, completion counted on an mbarrier per stage, no
+// multicast) that one thread issues ahead; all kThreads threads read each stage with one 128-bit
+// shared load per vector and do the arithmetic from registers.  The loop has no block-wide
+// barrier and stores nothing to global memory.  Every thread owns one "column" of the slice (its
+// kVpt vectors of every tile) and keeps of it: the largest logit, the tile that holds it, the
+// largest logit of all its other tiles, and (with SUMS) the log-sum-exp terms against its own
+// reference exponent.  The exact top-K of the row is selected from these records afterwards
+// (row_engine.cuh): only columns whose largest logit reaches a threshold can hold a top-K logit,
+// and of such a column only the one recorded tile, unless its second value reaches it too.
 #pragma once
 
 #include "scan_core.cuh"
@@ -19,8 +17,8 @@
 namespace dsp {
 
 constexpr int kTileBytes = kThreads * kVpt * 16;     // one ring stage = one tile of either dtype
-constexpr int kStages = 3;
-constexpr int kRingBytes = kStages * kTileBytes;     // dynamic shared memory of a streaming kernel
+constexpr int kMinStages = 3;                        // ring depth when the grid fills every SM several times over
+constexpr int kMaxStages = 9;                        // ring depth of a CTA that has its SM to itself
 constexpr long long kWaitCycles = 400000000LL;       // every wait gives up after this many SM clocks (~0.2 s)
 
 __device__ __forceinline__ uint32_t smem_addr(const void *p) {
@@ -74,11 +72,6 @@ __device__ __forceinline__ void bulk_load(void *dst, const void *src, uint32_t b
         ::"r"(smem_addr(dst)), "l"(src), "r"(bytes), "r"(smem_addr(bar)), "l"(policy)
         : "memory");
 }
-__device__ __forceinline__ float max3(float a, float b, float c) {
-    float d;
-    asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
-    return d;
-}
 
 // Two fp32 operations in one instruction on a register pair (Blackwell's packed fp32 pipe).
 __device__ __forceinline__ unsigned long long pack2(float lo, float hi) {
@@ -106,16 +99,22 @@ __device__ __forceinline__ unsigned long long add2(unsigned long long a, unsigne
 }
 
 // Static shared state of a streaming kernel.
+struct WarpPartial {             // log-sum-exp terms of one warp of one slice
+    double S, T;
+    float c;
+    int pad;
+};
 struct StreamBars {
-    uint64_t full[kStages];      // stage filled by its bulk copy
-    uint64_t empty[kStages];     // stage released by all warps
+    uint64_t full[kMaxStages];   // stage filled by its bulk copy
+    uint64_t empty[kMaxStages];  // stage released by all warps
+    WarpPartial wp[kWarps];      // the slice's sums, one entry per warp, written when the warp is through
     int timed_out;               // non-zero once a bounded wait gave up
 };
 
 // Called by every thread before the scan starts (ends with a CTA-wide barrier).
-__device__ __forceinline__ void stream_begin(StreamBars &bars) {
+__device__ __forceinline__ void stream_begin(StreamBars &bars, int nstages) {
     if (threadIdx.x == 0) {
-        for (int s = 0; s < kStages; ++s) {
+        for (int s = 0; s < nstages; ++s) {
             mbar_init(&bars.full[s], 1);
             mbar_init(&bars.empty[s], kWarps);
         }
@@ -127,14 +126,17 @@ __device__ __forceinline__ void stream_begin(StreamBars &bars) {
 
 // The tiles of a row dealt to its slices as evenly as whole tiles allow: slice s of n covers the
 // tiles [s * T / n, (s + 1) * T / n) of the row's T tiles (n <= T, so no slice is empty).
+__host__ __device__ __forceinline__ int slice_first_tile(int slice, int nslices, int ntiles_row) {
+    return (int)((long long)slice * ntiles_row / nslices);
+}
 template <typename DT>
 __device__ __forceinline__ void slice_range(int slice, int nslices, int ntiles_row, int V, int &s0, int &s1) {
     constexpr int TE = tile_elems<DT>();
-    s0 = (int)((long long)slice * ntiles_row / nslices) * TE;
-    s1 = min(V, (int)((long long)(slice + 1) * ntiles_row / nslices) * TE);
+    s0 = slice_first_tile(slice, nslices, ntiles_row) * TE;
+    s1 = min(V, slice_first_tile(slice + 1, nslices, ntiles_row) * TE);
 }
 
-// Issue the bulk copy of tile t of the slice at `src` into its ring stage s = t % kStages (one thread).
+// Issue the bulk copy of tile t of the slice at `src` into ring stage s (one thread).
 __device__ __forceinline__ void issue_tile(const char *src, int nbytes, int t, int s, unsigned char *ring,
                                            StreamBars &bars) {
     const uint32_t bytes = (uint32_t)min(kTileBytes, nbytes - t * kTileBytes);
@@ -142,145 +144,189 @@ __device__ __forceinline__ void issue_tile(const char *src, int nbytes, int t, i
     bulk_load(ring + (size_t)s * kTileBytes, src + (size_t)t * kTileBytes, bytes, &bars.full[s]);
 }
 
-// Padding for the vectors past the end of a ragged last tile: -2^124, below every finite
-// logit the interface allows, finite when scaled by log2(e), never a candidate (its index is
-// past the row).
-template <typename DT> struct Pad;
-template <> struct Pad<__nv_bfloat16> { static constexpr uint32_t kWord = 0xFD80FD80u; };
-template <> struct Pad<float> { static constexpr uint32_t kWord = 0xFD800000u; };
-
-// Entry of the table of per-thread tile maxima, stored in the row's own element type (exact).
-__device__ __forceinline__ void table_store(__nv_bfloat16 *tab, int i, float v) {
-    reinterpret_cast<unsigned short *>(tab)[i] = (unsigned short)(__float_as_uint(v) >> 16);
+// Largest of three, NaN if any is NaN (so that one NaN logit shows in a tile's maximum).
+__device__ __forceinline__ float max3_nan(float a, float b, float c) {
+    float d;
+    asm("max.NaN.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+    return d;
 }
-__device__ __forceinline__ void table_store(float *tab, int i, float v) { tab[i] = v; }
+__device__ __forceinline__ float max2_nan(float a, float b) {
+    float d;
+    asm("max.NaN.f32 %0, %1, %2;" : "=f"(d) : "f"(a), "f"(b));
+    return d;
+}
 
-// Log-sum-exp terms of one warp of one slice, as pass 1 leaves them.
-struct WarpPartial {
-    double S, T;
-    float c;
-    int pad;
+// What a thread keeps of its column of a slice.
+struct ColTop {
+    float rm1;      // largest logit of the column (-inf: none finite)
+    float rm2;      // largest logit of the column's other tiles (tiles other than t1)
+    int t1;         // tile of the slice (0-based) that holds rm1
+    float seen;     // NaN-keeping maximum of everything the thread saw: NaN or +inf flags the row
+};
+struct ColSums {    // S = sum 2^(x*kLog2e - c), T = sum 2^(x*kLog2e - c) * (x*kLog2e - c)
+    float c, S, T;
 };
 
-// Pass 1 over [s0, s1) of `row` (all kThreads threads of the CTA).  Writes the slice's part of
-// the row's table of per-thread tile maxima (`tab` points at the slice's first tile: entry
-// [t][thread]), every thread's largest logit of the whole slice (smax[thread]) and, with `sums`
-// (block-uniform), this warp's sums relative to its own reference exponent into wpart[warp]
-// (c = kRefFloor, S = 0 if the warp saw no finite logit).
-template <typename DT>
-__device__ void stream_slice(const DT *__restrict__ row, int s0, int s1, bool sums, StreamBars &bars,
-                             unsigned char *ring, DT *__restrict__ tab, DT *__restrict__ smax, WarpPartial *wpart) {
+// One tile from shared memory into the thread's running values.  nvec: 16-byte vectors of the
+// tile that exist (RAGGED: fewer than a whole tile; the missing ones take no part in anything).
+template <typename DT, bool SUMS, bool RAGGED>
+__device__ __forceinline__ void scan_tile(const uint4 *__restrict__ sp, int nvec, int t, int tid, ColTop &top,
+                                          float &c, unsigned long long &S2, unsigned long long &T2) {
     constexpr int N = Elem<DT>::N;
+    uint4 v[kVpt];
+    if constexpr (!RAGGED) {
+#pragma unroll
+        for (int j = 0; j < kVpt; ++j) v[j] = sp[j * kThreads + tid];
+    } else {
+        const uint32_t nw = Elem<DT>::kNegInfWord;
+#pragma unroll
+        for (int j = 0; j < kVpt; ++j) {
+            const int vi = j * kThreads + tid;
+            v[j] = vi < nvec ? sp[vi] : make_uint4(nw, nw, nw, nw);
+        }
+    }
+    float x[kVpt][N];
+    float vm[kVpt];
+#pragma unroll
+    for (int j = 0; j < kVpt; ++j) {
+#pragma unroll
+        for (int e = 0; e < N; ++e) x[j][e] = Elem<DT>::get(v[j], e);
+        if constexpr (N == 8) {
+            vm[j] = max3_nan(max3_nan(x[j][0], x[j][1], x[j][2]), max3_nan(x[j][3], x[j][4], x[j][5]),
+                             max2_nan(x[j][6], x[j][7]));
+        } else {
+            vm[j] = max2_nan(max3_nan(x[j][0], x[j][1], x[j][2]), x[j][3]);
+        }
+    }
+    const float tm = max2_nan(max3_nan(vm[0], vm[1], vm[2]), max3_nan(vm[3], vm[4], vm[5]));
+    // the column's best tile and the best of the others (a NaN maximum changes neither)
+    const bool gt = tm > top.rm1;
+    top.rm2 = gt ? top.rm1 : fmaxf(top.rm2, tm);
+    top.t1 = gt ? t : top.t1;
+    top.rm1 = gt ? tm : top.rm1;
+    top.seen = max2_nan(top.seen, tm);
+
+    if constexpr (SUMS) {
+        const float ts = tm * kLog2e;                 // the reference exponent bounds every logit seen
+        if (ts > c) {                                  // both halves move to the new reference exponent
+            const float d = c - ts;
+            const float sc = ex2_approx(d);
+            const unsigned long long sc2 = pack2(sc, sc);
+            T2 = mul2(fma2(S2, pack2(d, d), T2), sc2);
+            S2 = mul2(S2, sc2);
+            c = ts;
+        }
+        // two logits per instruction: a = x * log2(e) - c, S += 2^a, T += 2^a * a
+        const unsigned long long nc2 = pack2(-c, -c), l2e2 = pack2(kLog2e, kLog2e);
+#pragma unroll
+        for (int j = 0; j < kVpt; ++j) {
+            if (RAGGED && j * kThreads + tid >= nvec) continue;
+#pragma unroll
+            for (int e = 0; e < N; e += 2) {
+                const unsigned long long a2 = fma2(pack2(x[j][e], x[j][e + 1]), l2e2, nc2);
+                float a0, a1;
+                unpack2(a2, a0, a1);
+                const unsigned long long e2 = pack2(ex2_approx(a0), ex2_approx(a1));
+                S2 = add2(S2, e2);
+                T2 = fma2(e2, a2, T2);
+            }
+        }
+    }
+}
+
+// The sums of this thread's column of [s0, s1) once more, straight from global memory, against
+// the known reference exponent c with the exponent clamped: used when masked (-inf) logits
+// poisoned T only (0 * -inf) in the streaming loop.
+template <typename DT>
+__device__ void redo_column_sums(const DT *__restrict__ row, int s0, int s1, int tid, ColSums &cs) {
+    constexpr int N = Elem<DT>::N;
+    constexpr int TE = tile_elems<DT>();
+    const float nc = -cs.c;
+    float S = 0.f, T = 0.f;
+    for (int base = s0; base < s1; base += TE) {
+#pragma unroll
+        for (int j = 0; j < kVpt; ++j) {
+            const int e0 = base + (j * kThreads + tid) * N;
+            if (e0 < s1) {                                         // vectors are whole: the slice ends on a multiple of N
+                const uint4 vv = ldg_stream(row + e0);
+#pragma unroll
+                for (int e = 0; e < N; ++e) {
+                    const float a = fmaxf(fmaf(Elem<DT>::get(vv, e), kLog2e, nc), -1000.f);
+                    const float ex = ex2_approx(a);
+                    S += ex;
+                    T = fmaf(ex, a, T);
+                }
+            }
+        }
+    }
+    cs.S = S;
+    cs.T = T;
+}
+
+// Streams [s0, s1) of `row` through the ring (all kThreads threads of the CTA; `nstages` stages of
+// kTileBytes in `ring`).  On return `top` holds the thread's column record and, with SUMS, `cs`
+// its sums (c = kRefFloor, S = 0 if the thread saw no finite logit).
+template <typename DT, bool SUMS>
+__device__ void stream_slice(const DT *__restrict__ row, int s0, int s1, int nstages, StreamBars &bars,
+                             unsigned char *ring, ColTop &top, ColSums &cs) {
     constexpr int VT = kTileBytes / 16;
     static_assert(VT == kThreads * kVpt && tile_elems<DT>() * (int)sizeof(DT) == kTileBytes, "tile geometry");
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int tid = threadIdx.x, lane = tid & 31;
     const int nbytes = (s1 - s0) * (int)sizeof(DT);
     const int ntiles = (nbytes + kTileBytes - 1) / kTileBytes;
     volatile int *abort = &bars.timed_out;
 
-    float c = kRefFloor, S = 0.f, T = 0.f;
-    float rm = -CUDART_INF_F;                        // this thread's largest logit so far
-
-    // Thread 0 also issues the copies, kStages - 1 tiles ahead of the tile being scanned.
-    const char *src = reinterpret_cast<const char *>(row + s0);
-    if (tid == 0) {
-        for (int tt = 0; tt < min(kStages, ntiles); ++tt) issue_tile(src, nbytes, tt, tt, ring, bars);
-    }
-    int s = 0;                                       // stage of tile t: t % kStages
-    uint32_t ph = 0u;                                // phase parity of tile t in its stage: (t / kStages) & 1
-    DT *tp = tab + tid;                              // this thread's table entry of tile t
+    top.rm1 = -CUDART_INF_F; top.rm2 = -CUDART_INF_F; top.t1 = 0; top.seen = -CUDART_INF_F;
+    float c = kRefFloor;
     // the sums of this thread's even and odd logits (register pairs), against the reference exponent c
     unsigned long long S2 = pack2(0.f, 0.f), T2 = pack2(0.f, 0.f);
-    for (int t = 0; t < ntiles; ++t, tp += kThreads) {
-        if (tid == 0 && t >= 1 && t + kStages - 1 < ntiles) {
-            // tile t + kStages - 1 goes to the stage that held tile t - 1, once every warp has released it
-            const int es = s == 0 ? kStages - 1 : s - 1;
+
+    // Thread 0 also issues the copies, nstages - 1 tiles ahead of the tile being scanned.
+    const char *src = reinterpret_cast<const char *>(row + s0);
+    if (tid == 0) {
+        for (int tt = 0; tt < min(nstages, ntiles); ++tt) issue_tile(src, nbytes, tt, tt, ring, bars);
+    }
+    int s = 0;                                       // stage of tile t: t % nstages
+    uint32_t ph = 0u;                                // phase parity of tile t in its stage: (t / nstages) & 1
+    for (int t = 0; t < ntiles; ++t) {
+        if (tid == 0 && t >= 1 && t + nstages - 1 < ntiles) {
+            // tile t + nstages - 1 goes to the stage that held tile t - 1, once every warp has released it
+            const int es = s == 0 ? nstages - 1 : s - 1;
             if (!mbar_wait(&bars.empty[es], s == 0 ? ph ^ 1u : ph, abort)) bars.timed_out = 1;
-            issue_tile(src, nbytes, t + kStages - 1, es, ring, bars);
+            issue_tile(src, nbytes, t + nstages - 1, es, ring, bars);
         }
         if (!mbar_wait(&bars.full[s], ph, abort)) bars.timed_out = 1;
         const int nvec = min(kTileBytes, nbytes - t * kTileBytes) >> 4;
         const uint4 *sp = reinterpret_cast<const uint4 *>(ring + (size_t)s * kTileBytes);
-        uint4 v[kVpt];
-        if (nvec == VT) {
-#pragma unroll
-            for (int j = 0; j < kVpt; ++j) v[j] = sp[j * kThreads + tid];
-        } else {
-            const uint32_t pw = Pad<DT>::kWord;
-#pragma unroll
-            for (int j = 0; j < kVpt; ++j) {
-                const int vi = j * kThreads + tid;
-                v[j] = vi < nvec ? sp[vi] : make_uint4(pw, pw, pw, pw);
-            }
-        }
+        if (nvec == VT) scan_tile<DT, SUMS, false>(sp, nvec, t, tid, top, c, S2, T2);
+        else            scan_tile<DT, SUMS, true>(sp, nvec, t, tid, top, c, S2, T2);
         __syncwarp();
-        if (lane == 0) mbar_arrive(&bars.empty[s]);   // the stage is in registers: release it
+        if (lane == 0) mbar_arrive(&bars.empty[s]);   // the stage has been read: release it
+        if (++s == nstages) { s = 0; ph ^= 1u; }
+    }
+    float s0f, s1f, t0f, t1f;
+    unpack2(S2, s0f, s1f);
+    unpack2(T2, t0f, t1f);
+    cs.c = c;
+    cs.S = s0f + s1f;
+    cs.T = t0f + t1f;
+}
 
-        float x[kVpt][N];
-        float vm[kVpt];
-#pragma unroll
-        for (int j = 0; j < kVpt; ++j) {
-#pragma unroll
-            for (int e = 0; e < N; ++e) x[j][e] = Elem<DT>::get(v[j], e);
-            if constexpr (N == 8) {
-                vm[j] = max3(max3(x[j][0], x[j][1], x[j][2]), max3(x[j][3], x[j][4], x[j][5]),
-                             fmaxf(x[j][6], x[j][7]));
-            } else {
-                vm[j] = fmaxf(max3(x[j][0], x[j][1], x[j][2]), x[j][3]);
-            }
-        }
-        const float tm = fmaxf(fmaxf(fmaxf(vm[0], vm[1]), fmaxf(vm[2], vm[3])), fmaxf(vm[4], vm[5]));
-        table_store(tp, 0, tm);
-        rm = fmaxf(rm, tm);
-
-        if (sums) {
-            const float ts = tm * kLog2e;             // the reference exponent bounds every logit seen
-            if (ts > c) {                              // both halves move to the new reference exponent
-                const float d = c - ts;
-                const float sc = ex2_approx(d);
-                const unsigned long long sc2 = pack2(sc, sc);
-                T2 = mul2(fma2(S2, pack2(d, d), T2), sc2);
-                S2 = mul2(S2, sc2);
-                c = ts;
-            }
-            // two logits per instruction: a = x * log2(e) - c, S += 2^a, T += 2^a * a
-            const unsigned long long nc2 = pack2(-c, -c), l2e2 = pack2(kLog2e, kLog2e);
-#pragma unroll
-            for (int j = 0; j < kVpt; ++j) {
-#pragma unroll
-                for (int e = 0; e < N; e += 2) {
-                    const unsigned long long a2 = fma2(pack2(x[j][e], x[j][e + 1]), l2e2, nc2);
-                    float a0, a1;
-                    unpack2(a2, a0, a1);
-                    const unsigned long long e2 = pack2(ex2_approx(a0), ex2_approx(a1));
-                    S2 = add2(S2, e2);
-                    T2 = fma2(e2, a2, T2);
-                }
-            }
-        }
-        if (++s == kStages) { s = 0; ph ^= 1u; }
-    }
-    {
-        float s0f, s1f, t0f, t1f;
-        unpack2(S2, s0f, s1f);
-        unpack2(T2, t0f, t1f);
-        S = s0f + s1f;
-        T = t0f + t1f;
-    }
-    table_store(smax, tid, rm);
-    if (sums) {
-        // this warp's sums against one reference exponent, in double (shuffles only)
-        const float cw = warp_max(c);
-        const float d = c - cw;
-        const float a = ex2_approx(d);
-        const double Sd = warp_sum((double)(S * a));
-        const double Td = warp_sum((double)((T + S * d) * a));
-        if (lane == 0) {
-            WarpPartial p;
-            p.S = Sd; p.T = Td; p.c = cw; p.pad = 0;
-            wpart[warp] = p;
-        }
-    }
+// The sums of the threads of a warp against one reference exponent, in double (shuffles only);
+// lane 0 gets the result.
+__device__ __forceinline__ WarpPartial warp_partial(const ColSums &cs) {
+    const float cw = warp_max(cs.c);
+    const float d = cs.c - cw;
+    const float a = ex2_approx(d);
+    // a thread so far below the warp's reference that its weight is zero adds nothing (its S * d
+    // may overflow), unless its own sum is NaN or infinite (NaN / +inf logits), which must stay
+    // visible; so must a NaN weight (+inf logits of another thread)
+    const bool nothing = a == 0.f && cs.S < CUDART_INF_F;
+    WarpPartial p;
+    p.c = cw; p.pad = 0;
+    p.S = warp_sum(nothing ? 0.0 : (double)(cs.S * a));
+    p.T = warp_sum(nothing ? 0.0 : (double)((cs.T + cs.S * d) * a));
+    return p;
 }
 
 // The streaming kernels need more dynamic shared memory than the default limit: raise the limit
@@ -295,9 +341,33 @@ inline cudaError_t allow_ring_smem(KernelT *kernel, RingSmemDone &rec) {
     cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess) return e;
     if (dev >= 0 && dev < 64 && rec.dev[dev]) return cudaSuccess;
-    e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kRingBytes);
+    e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxStages * kTileBytes);
     if (e == cudaSuccess && dev >= 0 && dev < 64) rec.dev[dev] = true;
     return e;
+}
+
+// Number of SMs of the current device (asked once per device).
+inline int device_sm_count() {
+    static int sms[64] = {};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return 148;
+    if (!sms[dev]) {
+        int n = 0;
+        if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n < 1) n = 148;
+        sms[dev] = n;
+    }
+    return sms[dev];
+}
+
+// Ring depth of a streaming launch of `nblocks` CTAs.  A CTA that shares its SM with two others
+// needs no more than three stages (the SM then has six tiles in flight); with fewer CTAs than SM
+// slots each CTA takes a deeper ring, because one CTA's copies in flight are what bounds its
+// speed: at most two CTAs per SM -> four stages, one CTA per SM -> the whole shared memory.
+inline int ring_stages(long long nblocks) {
+    const int sms = device_sm_count();
+    if (nblocks <= sms) return kMaxStages;
+    if (nblocks <= 2ll * sms) return 4;
+    return kMinStages;
 }
 
 // True if rows of this layout can be streamed with bulk copies.

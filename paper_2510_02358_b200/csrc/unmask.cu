@@ -3,15 +3,14 @@
 //
 // For every position that is still masked the step needs the row's argmax and its probability:
 // the same whole-vocabulary statistics as the lattice and the verification, with K = 1.  Rows
-// whose first element is 16-byte aligned take the same two passes: unmask_scan_kernel streams the
-// masked rows (stream_core.cuh; CTAs of revealed rows leave at once, so a later refinement step
-// reads only what is still masked), unmask_rows_kernel (one warp per row, row_warp.cuh) adds up
-// the sums and takes the argmax from the table of tile maxima.  Any other layout is read
-// element-wise by the row's warp (slower, same results).  The warp that finishes the last row of
-// a batch row ranks the masked positions by confidence (counting; equal confidence: the lower
-// position first), reveals the best n_update and writes what is left.
+// whose layout is 16-byte aligned are streamed by unmask_scan_kernel (stream_core.cuh; CTAs of
+// revealed rows leave at once, so a later refinement step reads only what is still masked) and
+// finished by the CTA that is through with the row last (row_engine.cuh).  Any other layout is
+// read element-wise by one warp per row (slower, same results).  The warp that finishes the last
+// row of a batch row ranks the masked positions by confidence (counting; equal confidence: the
+// lower position first), reveals the best n_update and writes what is left.
 #include "dsp_internal.h"
-#include "row_warp.cuh"
+#include "row_engine.cuh"
 
 namespace dsp {
 
@@ -26,49 +25,28 @@ struct UnmaskArgs {
     float *confidence;
     int32_t *n_left;
     uint32_t *row_status;
-    int streaming;            // 1: the rows were streamed by unmask_scan_kernel
-    int nslices, slice_elems, ntiles_row;
+    int nslices, slice_elems, ntiles_row, nstages;
     // workspace
     unsigned *b_ticket;       // [B]  zeroed per call
     unsigned *b_status;       // [B]  zeroed per call
-    WarpPartial *wpart;       // [B*L, nslices, kWarps]
-    void *table;              // [B*L, ntiles_row + nslices, kThreads], element type of the logits
+    RowScratch rs;            // records of rows cut into several slices (streaming path)
 };
 
 struct UnmaskWs {
-    size_t off_b_ticket, off_b_status, zero_bytes, off_wpart, off_table, total;
+    size_t off_b_ticket, off_b_status, off_row_ticket, zero_bytes;
+    RowScratchLayout rs;
+    size_t total;
 };
-static UnmaskWs unmask_ws_layout(int64_t B, int64_t L, int nslices, int ntiles_row, size_t es) {
+static UnmaskWs unmask_ws_layout(int64_t B, int64_t L, int nslices) {
     UnmaskWs w;
     size_t o = 0;
-    w.off_b_ticket = o; o += align_up((size_t)B * 4, 256);
-    w.off_b_status = o; o += align_up((size_t)B * 4, 256);
+    w.off_b_ticket = o;   o += align_up((size_t)B * 4, 256);
+    w.off_b_status = o;   o += align_up((size_t)B * 4, 256);
+    w.off_row_ticket = o; o += align_up((size_t)(B * L) * 4, 256);
     w.zero_bytes = o;
-    w.off_wpart = o;    o += align_up((size_t)(B * L) * nslices * kWarps * sizeof(WarpPartial), 256);
-    w.off_table = o;    o += align_up((size_t)(B * L) * (ntiles_row + nslices) * kThreads * es, 256);
-    w.total = o;
+    w.rs = row_scratch_layout(o, B * L, nslices);
+    w.total = w.rs.end;
     return w;
-}
-
-// Pass 1 over the rows that are still masked: one CTA per row slice.
-template <typename DT>
-__global__ void __launch_bounds__(kThreads, 3) unmask_scan_kernel(const UnmaskArgs a) {
-    extern __shared__ __align__(128) unsigned char ring[];
-    __shared__ StreamBars bars;
-    const long long row = blockIdx.x / a.nslices;
-    if (!a.masked[row]) return;                          // revealed earlier: nothing to compute (whole CTA)
-    const int slice = blockIdx.x - (int)(row * a.nslices);
-    const int b = (int)(row / a.L), l = (int)(row - (long long)b * a.L);
-    const DT *rowp = reinterpret_cast<const DT *>(a.logits) + b * a.stride_b + l * a.stride_l;
-    int s0, s1;
-    slice_range<DT>(slice, a.nslices, a.ntiles_row, a.V, s0, s1);
-    stream_begin(bars);
-    grid_launch_dependents();
-    DT *trow = reinterpret_cast<DT *>(a.table) + row * (a.ntiles_row + a.nslices) * kThreads;
-    DT *tab = trow + (long long)(s0 / tile_elems<DT>()) * kThreads;
-    DT *smax = trow + (long long)(a.ntiles_row + slice) * kThreads;
-    stream_slice<DT>(rowp, s0, s1, true, bars, ring, tab, smax, a.wpart + (row * a.nslices + slice) * kWarps);
-    if (threadIdx.x == 0 && bars.timed_out) atomicOr(&a.b_status[b], DSP_ROW_TIMEOUT);
 }
 
 // Argmax (lowest id on ties), its logit and the row's log-sum-exp by one warp, element by
@@ -106,43 +84,9 @@ __device__ bool warp_row_stats_elementwise(const DT *__restrict__ row, int V, in
     return true;
 }
 
-// Pass 2 and the update: one warp per row; the warp arriving last for a batch row reveals the
-// best n_update masked positions.
-template <typename DT>
-__global__ void __launch_bounds__(kThreads) unmask_rows_kernel(const UnmaskArgs a) {
-    __shared__ WarpScratch scratch[kRowWarps];
-    grid_dependency_wait();                            // pass 1 is complete from here on
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const long long row = (long long)blockIdx.x * kRowWarps + warp;
-    if (row >= (long long)a.B * a.L) return;
-    const int b = (int)(row / a.L), l = (int)(row - (long long)b * a.L);
-    const DT *rowp = reinterpret_cast<const DT *>(a.logits) + b * a.stride_b + l * a.stride_l;
-
-    int am = -1;
-    float conf = -CUDART_INF_F;
-    if (a.masked[row]) {                                 // read before anyone's update: updates follow the last ticket
-        bool ok;
-        float xmax = 0.f;
-        double lse = 0.0;
-        if (a.streaming) {
-            float c;
-            double S, T;
-            warp_merge_partials(a.wpart + row * a.nslices * kWarps, a.nslices * kWarps, lane, c, S, T);
-            if (T != T && S == S && S < CUDART_INF) warp_redo_sums<DT>(rowp, a.V, lane, c, S, T);
-            const unsigned long long key = warp_select_topk<DT>(
-                rowp, a.V, 1, reinterpret_cast<const DT *>(a.table) + row * (a.ntiles_row + a.nslices) * kThreads,
-                a.ntiles_row, a.nslices, scratch[warp], lane);
-            const unsigned long long best = __shfl_sync(0xFFFFFFFFu, key, 0);
-            double mean_x;
-            ok = row_log_stats(c, S, T, lse, mean_x) && best != 0ull;
-            am = best ? key_id(best) : 0;
-            xmax = best ? key_value(best) : 0.f;
-        } else {
-            ok = warp_row_stats_elementwise<DT>(rowp, a.V, lane, am, xmax, lse);
-        }
-        if (ok) conf = (float)((double)xmax - lse);
-        else if (lane == 0) atomicOr(&a.b_status[b], DSP_ROW_NONFINITE_INPUT);
-    }
+// One row is done (am / conf: its argmax and confidence, -1 / -inf for a row that was not masked);
+// the warp arriving last for a batch row reveals the best n_update masked positions.  One warp.
+__device__ void unmask_row_done(const UnmaskArgs &a, long long row, int b, int am, float conf, int lane) {
     if (lane == 0) {
         a.argmax[row] = am;
         a.confidence[row] = conf;
@@ -187,40 +131,95 @@ __global__ void __launch_bounds__(kThreads) unmask_rows_kernel(const UnmaskArgs 
     }
 }
 
+// Streaming path: one CTA per row slice of the rows that are still masked; the CTA that is
+// through with a row last takes its argmax and confidence.  A row revealed earlier is reported
+// by its first CTA alone, without reading it.  (The mask changes only after every row of the
+// batch row has been reported, so every CTA of a row sees the same mask.)
+template <typename DT>
+__global__ void __launch_bounds__(kThreads, 3) unmask_scan_kernel(const UnmaskArgs a) {
+    extern __shared__ __align__(128) unsigned char ring[];
+    __shared__ StreamBars bars;
+    const long long row = blockIdx.x / a.nslices;
+    const int slice = blockIdx.x - (int)(row * a.nslices);
+    const int b = (int)(row / a.L), l = (int)(row - (long long)b * a.L);
+    const int lane = threadIdx.x & 31;
+    if (!a.masked[row]) {                                // whole CTA alike
+        grid_dependency_wait();                          // the tickets are prepared by the kernel before
+        if (slice == 0 && threadIdx.x < 32) unmask_row_done(a, row, b, -1, -CUDART_INF_F, lane);
+        return;
+    }
+    const DT *rowp = reinterpret_cast<const DT *>(a.logits) + b * a.stride_b + l * a.stride_l;
+    stream_begin(bars, a.nstages);
+    RowResult r;
+    if (!row_engine<DT>(rowp, a.V, 1, true, row, slice, a.nslices, a.ntiles_row, a.nstages, a.rs, &a.b_status[b], bars,
+                        ring, r))
+        return;
+    const unsigned long long best = __shfl_sync(0xFFFFFFFFu, r.key, 0);
+    double lse, mean_x;
+    const bool ok = row_log_stats(r.c, r.S, r.T, lse, mean_x) && best != 0ull;
+    const int am = best ? key_id(best) : 0;
+    float conf = -CUDART_INF_F;
+    if (ok) conf = (float)((double)key_value(best) - lse);
+    else if (lane == 0) atomicOr(&a.b_status[b], DSP_ROW_NONFINITE_INPUT);
+    unmask_row_done(a, row, b, am, conf, lane);
+}
+
+// Layouts that cannot be streamed: one warp per row, element by element.
+template <typename DT>
+__global__ void __launch_bounds__(kThreads) unmask_rows_kernel(const UnmaskArgs a) {
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const long long row = (long long)blockIdx.x * kWarps + warp;
+    if (row >= (long long)a.B * a.L) return;
+    const int b = (int)(row / a.L), l = (int)(row - (long long)b * a.L);
+    const DT *rowp = reinterpret_cast<const DT *>(a.logits) + b * a.stride_b + l * a.stride_l;
+    int am = -1;
+    float conf = -CUDART_INF_F;
+    if (a.masked[row]) {                                 // read before anyone's update: updates follow the last ticket
+        float xmax = 0.f;
+        double lse = 0.0;
+        if (warp_row_stats_elementwise<DT>(rowp, a.V, lane, am, xmax, lse)) conf = (float)((double)xmax - lse);
+        else if (lane == 0) atomicOr(&a.b_status[b], DSP_ROW_NONFINITE_INPUT);
+    }
+    unmask_row_done(a, row, b, am, conf, lane);
+}
+
 template <typename DT>
 static int32_t launch_unmask(UnmaskArgs &a, void *workspace, size_t workspace_bytes, cudaStream_t st) {
     const long long nrows = (long long)a.B * a.L;
-    const SlicePlan plan = plan_slices<DT>(nrows, a.V, kTargetCtas);
+    const SlicePlan plan = plan_slices<DT>(nrows, a.V, device_sm_count());
     a.nslices = plan.nslices;
     a.slice_elems = plan.slice_elems;
     a.ntiles_row = (a.V + tile_elems<DT>() - 1) / tile_elems<DT>();
-    const UnmaskWs w = unmask_ws_layout(a.B, a.L, a.nslices, a.ntiles_row, sizeof(DT));
+    const UnmaskWs w = unmask_ws_layout(a.B, a.L, a.nslices);
     if (workspace_bytes < w.total) return DSP_ERR_WORKSPACE;
     unsigned char *ws = static_cast<unsigned char *>(workspace);
     a.b_ticket = reinterpret_cast<unsigned *>(ws + w.off_b_ticket);
     a.b_status = reinterpret_cast<unsigned *>(ws + w.off_b_status);
-    a.wpart = reinterpret_cast<WarpPartial *>(ws + w.off_wpart);
-    a.table = ws + w.off_table;
-    DSP_CUDA_TRY(cudaMemsetAsync(ws, 0, w.zero_bytes, st));
+    a.rs.row_ticket = reinterpret_cast<unsigned *>(ws + w.off_row_ticket);
+    a.rs.cols = reinterpret_cast<uint2 *>(ws + w.rs.off_cols);
+    a.rs.wpart = reinterpret_cast<WarpPartial *>(ws + w.rs.off_wpart);
+    PrepareArgs prep = PrepareArgs();                    // tickets and status words start at zero
+    prep.zero_a = reinterpret_cast<uint32_t *>(ws); prep.n_a = (long long)(w.zero_bytes / 4);
+    DSP_CUDA_TRY(launch_prepare(prep, st));
     const long long nblocks = nrows * a.nslices;
     if (nblocks > 0x7FFFFFFFLL) return DSP_ERR_UNSUPPORTED;
-    a.streaming = a.nslices * kWarps <= kThreads && stream_layout_ok<DT>(a.logits, a.V, a.stride_b, a.stride_l);
-    if (a.streaming) {
+    if (a.nslices <= kMaxSlices && stream_layout_ok<DT>(a.logits, a.V, a.stride_b, a.stride_l)) {
         static RingSmemDone smem_done;                   // one per element type
         DSP_CUDA_TRY(allow_ring_smem(unmask_scan_kernel<DT>, smem_done));
-        unmask_scan_kernel<DT><<<(unsigned)nblocks, kThreads, kRingBytes, st>>>(a);
-        DSP_CUDA_TRY(cudaGetLastError());
+        a.nstages = ring_stages(nblocks);
+        DSP_CUDA_TRY(launch_dependent(unmask_scan_kernel<DT>, (unsigned)nblocks, kThreads, (size_t)a.nstages * kTileBytes, st, a,
+                                      short_kernel_follows_early(st, nrows)));
+    } else {
+        unmask_rows_kernel<DT><<<(unsigned)((nrows + kWarps - 1) / kWarps), kThreads, 0, st>>>(a);
     }
-    DSP_CUDA_TRY(launch_dependent(unmask_rows_kernel<DT>, (unsigned)((nrows + kRowWarps - 1) / kRowWarps), kThreads, 0, st, a,
-                                  a.streaming && rows_follow_early(st, nblocks)));
+    DSP_CUDA_TRY(cudaGetLastError());
     return DSP_OK;
 }
 
 template <typename DT>
 static size_t unmask_ws_bytes(int B, int L, int V) {
-    const SlicePlan plan = plan_slices<DT>((long long)B * L, V, kTargetCtas);
-    const int ntiles_row = (V + tile_elems<DT>() - 1) / tile_elems<DT>();
-    return unmask_ws_layout(B, L, plan.nslices, ntiles_row, sizeof(DT)).total;
+    const SlicePlan plan = plan_slices<DT>((long long)B * L, V, device_sm_count());
+    return unmask_ws_layout(B, L, plan.nslices).total;
 }
 
 }  // namespace dsp

@@ -2,9 +2,9 @@
 // (Sec. 2: Eq. 1 acceptance, residual resampling, Eq. 2 accepted length; greedy = temperature 0).
 //
 // Every target row is streamed once (argmax; log-sum-exp terms only for stochastic batch rows):
-// 16-byte aligned layouts by target_scan_kernel (one CTA per row slice, no block-wide barrier,
-// see stream_core.cuh) followed by target_rows_kernel (one warp per row: argmax from the table
-// of tile maxima, sums added up), any other layout by target_kernel (element-wise, slices
+// 16-byte aligned layouts by target_scan_kernel (one CTA per row slice, no block-wide barrier in
+// the loop, see stream_core.cuh; the CTA that is through with a row last takes the argmax and
+// adds up the sums, see row_engine.cuh), any other layout by target_kernel (element-wise, slices
 // merged by the CTA arriving last).  Every batch row's left-to-right acceptance scan (one warp)
 // then either gives the next token (greedy) or a sampling job (stochastic: residual at the first
 // rejection, or bonus from row m).  The first part needs only the target logits:
@@ -14,7 +14,7 @@
 // When every row is greedy the scans run in accept_kernel and that is all; otherwise they run
 // inside residual_kernel (each CTA scans its own batch row first): one launch less in the chain.
 #include "dsp_internal.h"
-#include "row_warp.cuh"
+#include "row_engine.cuh"
 
 namespace dsp {
 
@@ -53,9 +53,9 @@ struct VerifyArgs {
     unsigned long long *keys;  // [B*Lt, nslices]
     int32_t *argmax;           // [B*Lt]
     double *tlse64;            // [B*Lt]
-    WarpPartial *wpart;        // [B*Lt, nslices, kWarps]        (streaming path)
-    void *table;               // [B*Lt, ntiles_row + nslices, kThreads]  (streaming path), element type of the logits
+    RowScratch rs;             // records of rows cut into several slices (streaming path)
     int ntiles_row;            // tiles of a whole row
+    int nstages;               // ring depth of the streaming kernel
     SampleJob *jobs;           // [B]
     double *chunk_sums;        // [B, nchunks]
     int nchunks, res_slices, chunks_per_slice;
@@ -228,7 +228,8 @@ __global__ void __launch_bounds__(kThreads, 4) target_kernel(const VerifyArgs a)
     target_finish<DT, SyncAll>(a, sm, row, slice, b, sums, c, S, T, 0u);
 }
 
-// Streaming path, pass 1: one CTA per row slice (see stream_core.cuh).
+// Streaming path: one CTA per row slice; the CTA that is through with a row last writes its
+// argmax (lowest id on ties) and, for a stochastic batch row, its log-sum-exp.
 template <typename DT>
 __global__ void __launch_bounds__(kThreads, 3) target_scan_kernel(const VerifyArgs a) {
     extern __shared__ __align__(128) unsigned char ring[];
@@ -237,51 +238,23 @@ __global__ void __launch_bounds__(kThreads, 3) target_scan_kernel(const VerifyAr
     const int slice = blockIdx.x - (int)(row * a.nslices);
     const int b = (int)(row / a.Lt);
     const DT *rowp = trow_ptr<DT>(a, row);
-    int s0, s1;
-    slice_range<DT>(slice, a.nslices, a.ntiles_row, a.V, s0, s1);
     const bool sums = !a.all_greedy && a.mode[b] != 0;
-    stream_begin(bars);
+    stream_begin(bars, a.nstages);
     grid_launch_dependents();
-    DT *trow = reinterpret_cast<DT *>(a.table) + row * (a.ntiles_row + a.nslices) * kThreads;   // the row's table
-    DT *tab = trow + (long long)(s0 / tile_elems<DT>()) * kThreads;
-    DT *smax = trow + (long long)(a.ntiles_row + slice) * kThreads;
-    stream_slice<DT>(rowp, s0, s1, sums, bars, ring, tab, smax, a.wpart + (row * a.nslices + slice) * kWarps);
-    if (threadIdx.x == 0 && bars.timed_out) atomicOr(&a.b_status[b], DSP_ROW_TIMEOUT);
-}
-
-// Streaming path, pass 2: one warp per row (see row_warp.cuh): argmax from the table of tile
-// maxima, log-sum-exp from the warp sums.
-template <typename DT>
-__global__ void __launch_bounds__(kThreads) target_rows_kernel(const VerifyArgs a) {
-    __shared__ WarpScratch scratch[kRowWarps];
-    grid_dependency_wait();                            // pass 1 is complete from here on
-    grid_launch_dependents();
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const long long row = (long long)blockIdx.x * kRowWarps + warp;
-    if (row >= (long long)a.B * a.Lt) return;
-    const int b = (int)(row / a.Lt);
-    const DT *rowp = trow_ptr<DT>(a, row);
-    const bool sums = !a.all_greedy && a.mode[b] != 0;
-    float c = kRefFloor;
-    double S = 0.0, T = 0.0;
-    if (sums) {
-        warp_merge_partials(a.wpart + row * a.nslices * kWarps, a.nslices * kWarps, lane, c, S, T);
-        if (T != T && S == S && S < CUDART_INF) warp_redo_sums<DT>(rowp, a.V, lane, c, S, T);
-    }
-    const unsigned long long key = warp_select_topk<DT>(
-        rowp, a.V, 1, reinterpret_cast<const DT *>(a.table) + row * (a.ntiles_row + a.nslices) * kThreads, a.ntiles_row,
-        a.nslices, scratch[warp], lane);
-    const unsigned long long best = __shfl_sync(0xFFFFFFFFu, key, 0);
-    if (lane == 0) {
+    RowResult r;
+    if (!row_engine<DT>(rowp, a.V, 1, sums, row, slice, a.nslices, a.ntiles_row, a.nstages, a.rs, &a.b_status[b], bars,
+                        ring, r))
+        return;
+    if ((threadIdx.x & 31) == 0) {
+        const unsigned long long best = r.key;           // lane 0: the row's best key
         const int am = best ? key_id(best) : 0;
         a.argmax[row] = am;
         if (a.tgt_argmax) a.tgt_argmax[row] = am;
-        bool ok = best != 0ull;
+        bool ok = best != 0ull && !r.nonfinite;
         if (sums) {
-            double lse, mean_x;
-            ok = row_log_stats(c, S, T, lse, mean_x) && ok;
-            a.tlse64[row] = lse;
-            if (a.tgt_lse) a.tgt_lse[row] = (float)lse;
+            ok = r.stats_ok && ok;
+            a.tlse64[row] = r.lse;
+            if (a.tgt_lse) a.tgt_lse[row] = (float)r.lse;
         } else if (a.tgt_lse && !a.all_greedy) {
             a.tgt_lse[row] = CUDART_NAN_F;             // greedy row of a mixed batch: not computed
         }
@@ -491,9 +464,11 @@ __global__ void __launch_bounds__(kThreads, 4) residual_kernel(const VerifyArgs 
 
 struct VerifyWs {
     size_t off_row_ticket, off_b_ticket, off_res_ticket, off_b_status, zero_bytes;
-    size_t off_partials, off_keys, off_argmax, off_tlse, off_jobs, off_chunks, off_wpart, off_table, total;
+    size_t off_partials, off_keys, off_argmax, off_tlse, off_jobs, off_chunks;
+    RowScratchLayout rs;
+    size_t total;
 };
-static VerifyWs verify_ws_layout(int64_t B, int64_t Lt, int nslices, int nchunks, int ntiles_row, size_t es) {
+static VerifyWs verify_ws_layout(int64_t B, int64_t Lt, int nslices, int nchunks) {
     VerifyWs w;
     size_t o = 0;
     w.off_row_ticket = o; o += align_up((size_t)(B * Lt) * 4, 256);
@@ -507,9 +482,8 @@ static VerifyWs verify_ws_layout(int64_t B, int64_t Lt, int nslices, int nchunks
     w.off_tlse = o;       o += align_up((size_t)(B * Lt) * 8, 256);
     w.off_jobs = o;       o += align_up((size_t)B * sizeof(SampleJob), 256);
     w.off_chunks = o;     o += align_up((size_t)B * nchunks * 8, 256);
-    w.off_wpart = o;      o += align_up((size_t)(B * Lt) * nslices * kWarps * sizeof(WarpPartial), 256);
-    w.off_table = o;      o += align_up((size_t)(B * Lt) * (ntiles_row + nslices) * kThreads * es, 256);
-    w.total = o;
+    w.rs = row_scratch_layout(o, B * Lt, nslices);
+    w.total = w.rs.end;
     return w;
 }
 
@@ -518,21 +492,20 @@ static int nchunks_of(int V) { return (V + 32 * Elem<DT>::N - 1) / (32 * Elem<DT
 
 template <typename DT>
 static size_t verify_ws_bytes(int B, int Lt, int V) {
-    const SlicePlan plan = plan_slices<DT>((long long)B * Lt, V, kTargetCtas);
-    const int ntiles_row = (V + tile_elems<DT>() - 1) / tile_elems<DT>();
-    return verify_ws_layout(B, Lt, plan.nslices, nchunks_of<DT>(V), ntiles_row, sizeof(DT)).total;
+    const SlicePlan plan = plan_slices<DT>((long long)B * Lt, V, device_sm_count());
+    return verify_ws_layout(B, Lt, plan.nslices, nchunks_of<DT>(V)).total;
 }
 
 template <typename DT>
 static int32_t launch_verify(VerifyArgs &a, void *workspace, size_t workspace_bytes, cudaStream_t st,
                              int phases) {
     const long long nrows = (long long)a.B * a.Lt;
-    const SlicePlan plan = plan_slices<DT>(nrows, a.V, kTargetCtas);
+    const SlicePlan plan = plan_slices<DT>(nrows, a.V, device_sm_count());
     a.nslices = plan.nslices;
     a.slice_elems = plan.slice_elems;
     a.nchunks = nchunks_of<DT>(a.V);
     a.ntiles_row = (a.V + tile_elems<DT>() - 1) / tile_elems<DT>();
-    const VerifyWs w = verify_ws_layout(a.B, a.Lt, a.nslices, a.nchunks, a.ntiles_row, sizeof(DT));
+    const VerifyWs w = verify_ws_layout(a.B, a.Lt, a.nslices, a.nchunks);
     if (workspace_bytes < w.total) return DSP_ERR_WORKSPACE;
     char *ws = reinterpret_cast<char *>(workspace);
     a.row_ticket = reinterpret_cast<unsigned *>(ws + w.off_row_ticket);
@@ -544,11 +517,12 @@ static int32_t launch_verify(VerifyArgs &a, void *workspace, size_t workspace_by
     a.argmax = reinterpret_cast<int32_t *>(ws + w.off_argmax);
     a.tlse64 = reinterpret_cast<double *>(ws + w.off_tlse);
     a.jobs = reinterpret_cast<SampleJob *>(ws + w.off_jobs);
-    a.wpart = reinterpret_cast<WarpPartial *>(ws + w.off_wpart);
-    a.table = ws + w.off_table;
+    a.rs.row_ticket = a.row_ticket;
+    a.rs.cols = reinterpret_cast<uint2 *>(ws + w.rs.off_cols);
+    a.rs.wpart = reinterpret_cast<WarpPartial *>(ws + w.rs.off_wpart);
     a.chunk_sums = reinterpret_cast<double *>(ws + w.off_chunks);
     // residual pass: about 4 CTAs per SM over all jobs, at least one chunk per warp
-    int rsl = (148 * 4 + a.B - 1) / a.B;
+    int rsl = (device_sm_count() * 4 + a.B - 1) / a.B;
     const int max_rsl = (a.nchunks + kWarps - 1) / kWarps;
     if (rsl > max_rsl) rsl = max_rsl;
     if (rsl < 1) rsl = 1;
@@ -558,18 +532,20 @@ static int32_t launch_verify(VerifyArgs &a, void *workspace, size_t workspace_by
     const long long nblocks = nrows * a.nslices;
     if (nblocks > 0x7FFFFFFFLL) return DSP_ERR_UNSUPPORTED;
     if (phases & kVerifyStats) {
-    DSP_CUDA_TRY(cudaMemsetAsync(ws, 0, w.zero_bytes, st));
-    if (a.nslices * kWarps <= kThreads && nrows <= 0x7FFFFFFFLL &&
-        stream_layout_ok<DT>(a.target, a.V, a.tstride_b, a.tstride_l)) {
+    // tickets and status words of the workspace start at zero
+    PrepareArgs prep = PrepareArgs();
+    prep.zero_a = reinterpret_cast<uint32_t *>(ws); prep.n_a = (long long)(w.zero_bytes / 4);
+    DSP_CUDA_TRY(launch_prepare(prep, st));
+    if (a.nslices <= kMaxSlices && nrows <= 0x7FFFFFFFLL && stream_layout_ok<DT>(a.target, a.V, a.tstride_b, a.tstride_l)) {
         static RingSmemDone smem_done;                       // one per element type
         DSP_CUDA_TRY(allow_ring_smem(target_scan_kernel<DT>, smem_done));
+        a.nstages = ring_stages(nblocks);
         const ProfileEvents pe = g_profile[DSP_PROFILE_TARGET_SCAN];
         if (pe.start) DSP_CUDA_TRY(cudaEventRecord(pe.start, st));
-        target_scan_kernel<DT><<<(unsigned)nblocks, kThreads, kRingBytes, st>>>(a);
-        DSP_CUDA_TRY(cudaGetLastError());
+        // the streaming kernel may start beside the preparation: it waits for it after its rows are streamed
+        DSP_CUDA_TRY(launch_dependent(target_scan_kernel<DT>, (unsigned)nblocks, kThreads, (size_t)a.nstages * kTileBytes, st, a,
+                                      !pe.start && short_kernel_follows_early(st, nrows)));
         if (pe.stop) DSP_CUDA_TRY(cudaEventRecord(pe.stop, st));
-        DSP_CUDA_TRY(launch_dependent(target_rows_kernel<DT>, (unsigned)((nrows + kRowWarps - 1) / kRowWarps), kThreads, 0, st, a,
-                                      short_kernel_follows_early(st, nrows)));
     } else {
         target_kernel<DT><<<(unsigned)nblocks, kThreads, 0, st>>>(a);
     }
@@ -725,7 +701,7 @@ static int32_t launch_sample(VerifyArgs &a, SampleArgs &s, void *workspace, size
     a.draft_lse64 = s.dlse_g;
     s.jobs = a.jobs;
     a.chunk_sums = reinterpret_cast<double *>(ws + w.off_chunks);
-    int rsl = (148 * 4 + a.B - 1) / a.B;
+    int rsl = (device_sm_count() * 4 + a.B - 1) / a.B;
     const int max_rsl = (a.nchunks + kWarps - 1) / kWarps;
     if (rsl > max_rsl) rsl = max_rsl;
     if (rsl < 1) rsl = 1;
