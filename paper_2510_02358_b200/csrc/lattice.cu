@@ -209,7 +209,7 @@ __global__ void __launch_bounds__(kThreads, 3) lattice_scan_kernel(const Lattice
 template <typename DT>
 static int32_t launch_lattice(LatticeArgs &a, void *workspace, size_t workspace_bytes, cudaStream_t st) {
     const long long nrows = (long long)a.B * a.L;
-    const SlicePlan plan = plan_slices<DT>(nrows, a.V, device_sm_count());
+    const SlicePlan plan = plan_slices<DT>(nrows, a.V, slice_target_ctas());
     a.nslices = plan.nslices;
     a.slice_elems = plan.slice_elems;
     a.ntiles_row = (a.V + tile_elems<DT>() - 1) / tile_elems<DT>();
@@ -251,7 +251,7 @@ static int32_t launch_lattice(LatticeArgs &a, void *workspace, size_t workspace_
 
 template <typename DT>
 static size_t lattice_ws_bytes(int B, int L, int V, int K) {
-    const SlicePlan plan = plan_slices<DT>((long long)B * L, V, device_sm_count());
+    const SlicePlan plan = plan_slices<DT>((long long)B * L, V, slice_target_ctas());
     return lattice_ws_layout(B, L, plan.nslices, K).total;
 }
 

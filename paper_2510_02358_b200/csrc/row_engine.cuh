@@ -80,6 +80,12 @@ struct RowResult {
     bool nonfinite;           // a NaN or +inf logit was seen
 };
 
+// Barrier 1 of the CTA for its first `nthreads` threads (whole warps): the selecting warps of a
+// row finish meet here while the last warp works on its own.
+__device__ __forceinline__ void select_barrier(int nthreads) {
+    asm volatile("bar.sync 1, %0;" ::"r"(nthreads) : "memory");
+}
+
 // Inclusive prefix sum over the lanes of a warp.
 __device__ __forceinline__ int warp_scan_incl(int v, int lane) {
 #pragma unroll
@@ -124,13 +130,11 @@ __device__ bool row_finish(const DT *__restrict__ rowp, int V, int K, bool sums,
     if (tid == 0) { fs.nkeys = 0; fs.nshares = 0; }
     if (tid < 32) fs.order[tid] = 0ull;
     const bool any_bad = __syncthreads_or(bad) != 0;
-    if (warp == 0) {
-        const float v = fs.wtop[lane];
-        const float t = K == 1 ? warp_max(v) : warp_kth_largest(v, K, lane);
-        if (lane == 0) fs.t0 = t;
-    }
-    // the last warp adds up the row's sums while the others select (it joins them at the barriers)
-    if (warp == kWarps - 1 && sums) {
+    // With sums the last warp leaves the others here: it adds up the row's sums and what follows
+    // from them (double precision, a long dependent chain) while they select, and meets them again
+    // at the last barrier; the others take over its columns.
+    const int nsel = sums ? kThreads - 32 : kThreads;  // selecting threads: they meet at barrier 1
+    if (sums && warp == kWarps - 1) {
         float c;
         double S, T;
         if (wp_own) {
@@ -148,96 +152,104 @@ __device__ bool row_finish(const DT *__restrict__ rowp, int V, int K, bool sums,
         if (lane == 0) {
             fs.c = c; fs.S = S; fs.T = T; fs.lse = lse; fs.mean_x = mean_x; fs.stats_ok = ok ? 1 : 0;
         }
-    }
-    __syncthreads();
-    const float t0 = fs.t0;
-
-    // ---- 2. shares ----
-    for (int s = 0; s < nslices; ++s) {
-        const uint2 r = stash[s * kThreads + tid];
-        const float rm1 = col_rm1(r);
-        const bool in = rm1 >= t0 && rm1 > -CUDART_INF_F;
-        const bool whole = in && col_rm2(r) >= t0;     // more than one tile of this column may hold a top-K logit
-        const int tb = slice_first_tile(s, nslices, ntiles_row);
-        const unsigned m = __ballot_sync(0xFFFFFFFFu, in && !whole);
-        if (m) {                                       // one tile each: one counter update per warp
-            int base = 0;
-            if (lane == 0) base = atomicAdd(&fs.nshares, __popc(m));
-            base = __shfl_sync(0xFFFFFFFFu, base, 0);
-            const int pos = base + __popc(m & ((1u << lane) - 1u));
-            if (in && !whole && pos < kShareCap) fs.shares[pos] = ((uint32_t)(tb + col_t1(r)) << 8) | (uint32_t)tid;
+    } else {
+        if (warp == 0) {
+            const float v = fs.wtop[lane];
+            const float t = K == 1 ? warp_max(v) : warp_kth_largest(v, K, lane);
+            if (lane == 0) fs.t0 = t;
         }
-        if (whole) {
-            const int te = slice_first_tile(s + 1, nslices, ntiles_row);
-            const int pos = atomicAdd(&fs.nshares, te - tb);
-            for (int t = tb; t < te; ++t)
-                if (pos + (t - tb) < kShareCap) fs.shares[pos + (t - tb)] = ((uint32_t)t << 8) | (uint32_t)tid;
-        }
-    }
-    __syncthreads();
-    const int nshares = fs.nshares;
-    bool careful = nshares > kShareCap;
+        select_barrier(nsel);
+        const float t0 = fs.t0;
 
-    // ---- 3. keys ----
-    if (!careful) {
-        const int items = nshares * kVpt;
-        for (int it0 = warp * 32; it0 < items; it0 += kThreads) {
-            const int it = it0 + lane;
-            int e0 = 0;
-            uint4 v = make_uint4(0u, 0u, 0u, 0u);
-            unsigned hits = 0u;                        // bit e: element e of this lane's vector reaches the threshold
-            if (it < items) {
-                const int sh = it / kVpt, j = it - sh * kVpt;
-                const uint32_t id = fs.shares[sh];
-                e0 = (int)(id >> 8) * TE + (j * kThreads + (int)(id & 255u)) * N;
-                if (e0 < V) {                          // vectors are whole: the row length is a multiple of N
-                    v = ldg_stream(rowp + e0);
+        // ---- 2. shares ----
+        for (int col0 = warp * 32; col0 < kThreads; col0 += nsel) {
+            const int col = col0 + lane;
+            for (int s = 0; s < nslices; ++s) {
+                const uint2 r = stash[s * kThreads + col];
+                const float rm1 = col_rm1(r);
+                const bool in = rm1 >= t0 && rm1 > -CUDART_INF_F;
+                const bool whole = in && col_rm2(r) >= t0;     // more than one tile of this column may hold a top-K logit
+                const int tb = slice_first_tile(s, nslices, ntiles_row);
+                const unsigned m = __ballot_sync(0xFFFFFFFFu, in && !whole);
+                if (m) {                                       // one tile each: one counter update per warp
+                    int base = 0;
+                    if (lane == 0) base = atomicAdd(&fs.nshares, __popc(m));
+                    base = __shfl_sync(0xFFFFFFFFu, base, 0);
+                    const int pos = base + __popc(m & ((1u << lane) - 1u));
+                    if (in && !whole && pos < kShareCap) fs.shares[pos] = ((uint32_t)(tb + col_t1(r)) << 8) | (uint32_t)col;
+                }
+                if (whole) {
+                    const int te = slice_first_tile(s + 1, nslices, ntiles_row);
+                    const int pos = atomicAdd(&fs.nshares, te - tb);
+                    for (int t = tb; t < te; ++t)
+                        if (pos + (t - tb) < kShareCap) fs.shares[pos + (t - tb)] = ((uint32_t)t << 8) | (uint32_t)col;
+                }
+            }
+        }
+        select_barrier(nsel);
+        const int nshares = fs.nshares;
+
+        // ---- 3. keys ----
+        if (nshares <= kShareCap) {
+            const int items = nshares * kVpt;
+            for (int it0 = warp * 32; it0 < items; it0 += nsel) {
+                const int it = it0 + lane;
+                int e0 = 0;
+                uint4 v = make_uint4(0u, 0u, 0u, 0u);
+                unsigned hits = 0u;                    // bit e: element e of this lane's vector reaches the threshold
+                if (it < items) {
+                    const int sh = it / kVpt, j = it - sh * kVpt;
+                    const uint32_t id = fs.shares[sh];
+                    e0 = (int)(id >> 8) * TE + (j * kThreads + (int)(id & 255u)) * N;
+                    if (e0 < V) {                      // vectors are whole: the row length is a multiple of N
+                        v = ldg_stream(rowp + e0);
+#pragma unroll
+                        for (int e = 0; e < N; ++e) {
+                            const float x = Elem<DT>::get(v, e);
+                            if (x >= t0 && x > -CUDART_INF_F) hits |= 1u << e;
+                        }
+                    }
+                }
+                const int h = __popc(hits);
+                const int incl = warp_scan_incl(h, lane);
+                const int total = __shfl_sync(0xFFFFFFFFu, incl, 31);
+                if (total) {                           // one counter update per warp
+                    int base = 0;
+                    if (lane == 31) base = atomicAdd(&fs.nkeys, total);
+                    base = __shfl_sync(0xFFFFFFFFu, base, 31);
+                    int pos = base + incl - h;
 #pragma unroll
                     for (int e = 0; e < N; ++e) {
-                        const float x = Elem<DT>::get(v, e);
-                        if (x >= t0 && x > -CUDART_INF_F) hits |= 1u << e;
+                        if (hits & (1u << e)) {
+                            if (pos < kKeyCap) fs.keys[pos] = make_key(Elem<DT>::get(v, e), e0 + e);
+                            ++pos;
+                        }
                     }
                 }
             }
-            const int h = __popc(hits);
-            const int incl = warp_scan_incl(h, lane);
-            const int total = __shfl_sync(0xFFFFFFFFu, incl, 31);
-            if (total) {                               // one counter update per warp
-                int base = 0;
-                if (lane == 31) base = atomicAdd(&fs.nkeys, total);
-                base = __shfl_sync(0xFFFFFFFFu, base, 31);
-                int pos = base + incl - h;
-#pragma unroll
-                for (int e = 0; e < N; ++e) {
-                    if (hits & (1u << e)) {
-                        if (pos < kKeyCap) fs.keys[pos] = make_key(Elem<DT>::get(v, e), e0 + e);
-                        ++pos;
+            select_barrier(nsel);
+            const int nkeys = fs.nkeys;
+            // ---- 4. places ----
+            if (nkeys <= kKeyCap) {
+                if (tid == 0 && (nkeys & 1)) fs.keys[nkeys] = 0ull;    // pad to a whole pair (room: kKeyCap + 2)
+                select_barrier(nsel);
+                const ulonglong2 *kp = reinterpret_cast<const ulonglong2 *>(fs.keys);
+                for (int i = tid; i < nkeys; i += nsel) {
+                    const unsigned long long q = fs.keys[i];
+                    int place = 0;
+                    for (int j = 0; j < ((nkeys + 1) >> 1); ++j) {
+                        const ulonglong2 o = kp[j];
+                        place += (o.x > q ? 1 : 0) + (o.y > q ? 1 : 0);
                     }
+                    if (place < 32) fs.order[place] = q;
                 }
-            }
-        }
-        __syncthreads();
-        const int nkeys = fs.nkeys;
-        careful = nkeys > kKeyCap;
-        // ---- 4. places ----
-        if (!careful) {
-            if (tid == 0 && (nkeys & 1)) fs.keys[nkeys] = 0ull;        // pad to a whole pair (room: kKeyCap + 2)
-            __syncthreads();
-            const ulonglong2 *kp = reinterpret_cast<const ulonglong2 *>(fs.keys);
-            for (int i = tid; i < nkeys; i += kThreads) {
-                const unsigned long long q = fs.keys[i];
-                int place = 0;
-                for (int j = 0; j < ((nkeys + 1) >> 1); ++j) {
-                    const ulonglong2 o = kp[j];
-                    place += (o.x > q ? 1 : 0) + (o.y > q ? 1 : 0);
-                }
-                if (place < 32) fs.order[place] = q;
             }
         }
     }
     __syncthreads();
     if (warp != 0) return false;
 
+    const bool careful = fs.nshares > kShareCap || fs.nkeys > kKeyCap;    // a list overflowed: the slow, bounded way
     res.key = careful ? warp_topk_careful<DT>(rowp, V, K, lane) : fs.order[lane];
     res.nonfinite = any_bad;
     res.c = kRefFloor; res.S = 0.0; res.T = 0.0;

@@ -80,7 +80,8 @@ __global__ void __launch_bounds__(kThreads, 3) shard_scan_kernel(const ShardArgs
     if (!row_engine<DT>(rowp, a.V, a.K, true, row, slice, a.nslices, a.ntiles_row, a.nstages, a.rs, &a.shard_status[b],
                         bars, ring, r))
         return;
-    shard_write_row<DT>(a, row, b, l, rowp, r.key, r.c, r.S, r.T, threadIdx.x & 31);
+    // a NaN or +inf logit must show in the record's sums, whichever unit took its exponential
+    shard_write_row<DT>(a, row, b, l, rowp, r.key, r.c, r.nonfinite ? CUDART_NAN : r.S, r.T, threadIdx.x & 31);
 }
 
 // Sums and exact top-K of a row that cannot be streamed, element by element, by one warp.
@@ -198,7 +199,7 @@ __global__ void __launch_bounds__(kThreads) shard_merge_kernel(const MergeArgs m
 template <typename DT>
 static int32_t launch_shard(ShardArgs &a, void *workspace, size_t workspace_bytes, cudaStream_t st) {
     const long long nrows = (long long)a.B * a.L;
-    const SlicePlan plan = plan_slices<DT>(nrows, a.V, device_sm_count());
+    const SlicePlan plan = plan_slices<DT>(nrows, a.V, slice_target_ctas());
     a.nslices = plan.nslices;
     a.slice_elems = plan.slice_elems;
     a.ntiles_row = (a.V + tile_elems<DT>() - 1) / tile_elems<DT>();
@@ -229,7 +230,7 @@ static int32_t launch_shard(ShardArgs &a, void *workspace, size_t workspace_byte
 
 template <typename DT>
 static size_t shard_ws_bytes(int B, int L, int V) {
-    const SlicePlan plan = plan_slices<DT>((long long)B * L, V, device_sm_count());
+    const SlicePlan plan = plan_slices<DT>((long long)B * L, V, slice_target_ctas());
     return shard_ws_layout(B, L, plan.nslices).total;
 }
 

@@ -198,7 +198,13 @@ __device__ __forceinline__ void scan_tile(const uint4 *__restrict__ sp, int nvec
             vm[j] = max2_nan(max3_nan(x[j][0], x[j][1], x[j][2]), x[j][3]);
         }
     }
-    const float tm = max2_nan(max3_nan(vm[0], vm[1], vm[2]), max3_nan(vm[3], vm[4], vm[5]));
+    float tm = vm[0];
+    if constexpr (kVpt == 6) {
+        tm = max2_nan(max3_nan(vm[0], vm[1], vm[2]), max3_nan(vm[3], vm[4], vm[5]));
+    } else {
+#pragma unroll
+        for (int j = 1; j < kVpt; ++j) tm = max2_nan(tm, vm[j]);
+    }
     // the column's best tile and the best of the others (a NaN maximum changes neither)
     const bool gt = tm > top.rm1;
     top.rm2 = gt ? top.rm1 : fmaxf(top.rm2, tm);
@@ -358,6 +364,10 @@ inline int device_sm_count() {
     }
     return sms[dev];
 }
+
+// Rows are cut into slices until about this many CTAs exist.
+constexpr int kSliceCtasPerSm = 1;
+inline int slice_target_ctas() { return device_sm_count() * kSliceCtasPerSm; }
 
 // Ring depth of a streaming launch of `nblocks` CTAs.  A CTA that shares its SM with two others
 // needs no more than three stages (the SM then has six tiles in flight); with fewer CTAs than SM

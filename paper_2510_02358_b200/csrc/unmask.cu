@@ -155,8 +155,8 @@ __global__ void __launch_bounds__(kThreads, 3) unmask_scan_kernel(const UnmaskAr
                         ring, r))
         return;
     const unsigned long long best = __shfl_sync(0xFFFFFFFFu, r.key, 0);
-    double lse, mean_x;
-    const bool ok = row_log_stats(r.c, r.S, r.T, lse, mean_x) && best != 0ull;
+    const double lse = r.lse;
+    const bool ok = r.stats_ok && !r.nonfinite && best != 0ull;
     const int am = best ? key_id(best) : 0;
     float conf = -CUDART_INF_F;
     if (ok) conf = (float)((double)key_value(best) - lse);
@@ -186,7 +186,7 @@ __global__ void __launch_bounds__(kThreads) unmask_rows_kernel(const UnmaskArgs 
 template <typename DT>
 static int32_t launch_unmask(UnmaskArgs &a, void *workspace, size_t workspace_bytes, cudaStream_t st) {
     const long long nrows = (long long)a.B * a.L;
-    const SlicePlan plan = plan_slices<DT>(nrows, a.V, device_sm_count());
+    const SlicePlan plan = plan_slices<DT>(nrows, a.V, slice_target_ctas());
     a.nslices = plan.nslices;
     a.slice_elems = plan.slice_elems;
     a.ntiles_row = (a.V + tile_elems<DT>() - 1) / tile_elems<DT>();
@@ -218,7 +218,7 @@ static int32_t launch_unmask(UnmaskArgs &a, void *workspace, size_t workspace_by
 
 template <typename DT>
 static size_t unmask_ws_bytes(int B, int L, int V) {
-    const SlicePlan plan = plan_slices<DT>((long long)B * L, V, device_sm_count());
+    const SlicePlan plan = plan_slices<DT>((long long)B * L, V, slice_target_ctas());
     return unmask_ws_layout(B, L, plan.nslices).total;
 }
 

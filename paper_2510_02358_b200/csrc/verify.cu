@@ -492,7 +492,7 @@ static int nchunks_of(int V) { return (V + 32 * Elem<DT>::N - 1) / (32 * Elem<DT
 
 template <typename DT>
 static size_t verify_ws_bytes(int B, int Lt, int V) {
-    const SlicePlan plan = plan_slices<DT>((long long)B * Lt, V, device_sm_count());
+    const SlicePlan plan = plan_slices<DT>((long long)B * Lt, V, slice_target_ctas());
     return verify_ws_layout(B, Lt, plan.nslices, nchunks_of<DT>(V)).total;
 }
 
@@ -500,7 +500,7 @@ template <typename DT>
 static int32_t launch_verify(VerifyArgs &a, void *workspace, size_t workspace_bytes, cudaStream_t st,
                              int phases) {
     const long long nrows = (long long)a.B * a.Lt;
-    const SlicePlan plan = plan_slices<DT>(nrows, a.V, device_sm_count());
+    const SlicePlan plan = plan_slices<DT>(nrows, a.V, slice_target_ctas());
     a.nslices = plan.nslices;
     a.slice_elems = plan.slice_elems;
     a.nchunks = nchunks_of<DT>(a.V);
