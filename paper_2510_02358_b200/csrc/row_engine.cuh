@@ -4,15 +4,15 @@
 // global memory: sums added up, exact top-K selected.  No CTA waits for another (atomic ticket).
 //
 // Selection of the exact top-K under (logit desc, id asc), by all threads of the finishing CTA:
-//  1. every thread takes one column (all slices) and its largest logit; each warp hands in its four
-//     largest columns, and the K-th largest of those 32 values has at least K logits at or above
-//     it (-inf if fewer exist): the threshold;
+//  1. every thread takes one column (all slices) and its largest logit; the columns form 32 groups
+//     of 8, and the K-th largest of the groups' maxima has at least K logits at or above it (-inf
+//     if fewer exist): the threshold;
 //  2. only a column whose largest logit reaches the threshold can hold a top-K logit, and only in
 //     the tile recorded for it, unless the largest logit of its other tiles reaches the threshold
 //     too (then every tile of that column and slice is looked at): these (tile, column) shares are
 //     listed;
-//  3. the shares' vectors are read again from global memory, one vector per thread, and the
-//     logits that reach the threshold are listed as 64-bit keys;
+//  3. the shares' vectors are read again from global memory, one vector per thread so that all of
+//     them are in flight together, and the logits that reach the threshold are listed as keys;
 //  4. the list holds the whole top K: every key counts the keys above it (they are unique), which
 //     is its place.
 // A list that overflows (very many equal top values) sends the row to warp_topk_careful.
@@ -52,7 +52,7 @@ struct FinishSmem {
     __align__(16) unsigned long long keys[kKeyCap + 2];
     unsigned long long order[32];             // the best 32 keys in order
     uint32_t shares[kShareCap];
-    float wtop[kWarps * 4];                   // every warp's four largest columns
+    __align__(16) uint32_t gmax[4 * kWarps];   // largest logit of every group of 8 columns (order-preserving bits)
     double S, T, lse, mean_x;                 // the row's sums and what follows from them (written by the last warp)
     float c;
     int stats_ok;
@@ -110,22 +110,20 @@ __device__ bool row_finish(const DT *__restrict__ rowp, int V, int K, bool sums,
     FinishSmem &fs = *reinterpret_cast<FinishSmem *>(smem);
     const uint2 *stash = reinterpret_cast<const uint2 *>(smem + kFinishBytes);
 
-    // ---- 1. threshold ----
-    float cmax = -CUDART_INF_F;
+    // ---- 1. threshold: the K-th largest of the maxima of 32 groups of 8 neighbouring columns ----
+    uint32_t cmax_ord = ord_bits(-CUDART_INF_F);
     bool bad = false;
     for (int s = 0; s < nslices; ++s) {
         const uint2 r = stash[s * kThreads + tid];
-        cmax = fmaxf(cmax, col_rm1(r));
+        cmax_ord = max(cmax_ord, ord_bits(col_rm1(r)));
         bad |= col_bad(r);
     }
     {
-        int before = 0;                                // columns of this warp that come first
-#pragma unroll
-        for (int j = 0; j < 32; ++j) {
-            const float o = __shfl_sync(0xFFFFFFFFu, cmax, j);
-            before += (o > cmax || (o == cmax && j < lane)) ? 1 : 0;
-        }
-        if (before < 4) fs.wtop[warp * 4 + before] = cmax;
+        // each group holds a logit at or above its maximum: K distinct logits reach the K-th largest
+        // maximum.  The low five bits of a maximum give way to the group's number (keys are then
+        // unique, and lowering a value by less than 32 ulp keeps the threshold valid).
+        const uint32_t g = __reduce_max_sync(0xFFu << (lane & 24), cmax_ord);
+        if ((lane & 7) == 0) fs.gmax[tid >> 3] = (g & ~31u) | (uint32_t)(31 - (tid >> 3));
     }
     if (tid == 0) { fs.nkeys = 0; fs.nshares = 0; }
     if (tid < 32) fs.order[tid] = 0ull;
@@ -153,14 +151,24 @@ __device__ bool row_finish(const DT *__restrict__ rowp, int V, int K, bool sums,
             fs.c = c; fs.S = S; fs.T = T; fs.lse = lse; fs.mean_x = mean_x; fs.stats_ok = ok ? 1 : 0;
         }
     } else {
-        if (warp == 0) {
-            const float v = fs.wtop[lane];
-            const float t = K == 1 ? warp_max(v) : warp_kth_largest(v, K, lane);
-            if (lane == 0) fs.t0 = t;
+        float t0;
+        {
+            // every warp ranks the 32 group maxima itself (lane i: value i, by counting the larger ones)
+            const uint4 *gp = reinterpret_cast<const uint4 *>(fs.gmax);
+            const uint32_t mine = fs.gmax[lane];
+            int b0 = 0, b1 = 0, b2 = 0, b3 = 0;
+#pragma unroll
+            for (int q = 0; q < 8; ++q) {
+                const uint4 v = gp[q];
+                b0 += v.x > mine ? 1 : 0;
+                b1 += v.y > mine ? 1 : 0;
+                b2 += v.z > mine ? 1 : 0;
+                b3 += v.w > mine ? 1 : 0;
+            }
+            const unsigned who = __ballot_sync(0xFFFFFFFFu, (b0 + b1) + (b2 + b3) == K - 1);
+            const uint32_t kb = __shfl_sync(0xFFFFFFFFu, mine, __ffs(who) - 1) & ~31u;
+            t0 = kb <= ord_bits(-CUDART_INF_F) ? -CUDART_INF_F : ord_value(kb);    // fewer than K finite maxima: everything finite
         }
-        select_barrier(nsel);
-        const float t0 = fs.t0;
-
         // ---- 2. shares ----
         for (int col0 = warp * 32; col0 < kThreads; col0 += nsel) {
             const int col = col0 + lane;

@@ -89,17 +89,4 @@ __device__ unsigned long long warp_topk_careful(const DT *__restrict__ row, int 
     return best;
 }
 
-// The K-th largest (K = 1 .. 32) of the lanes' values: every lane counts the lanes that come
-// before it (larger value, or equal value and lower lane); the lane with K - 1 before it has it.
-__device__ __forceinline__ float warp_kth_largest(float v, int K, int lane) {
-    int before = 0;
-#pragma unroll
-    for (int j = 0; j < 32; ++j) {
-        const float o = __shfl_sync(0xFFFFFFFFu, v, j);
-        before += (o > v || (o == v && j < lane)) ? 1 : 0;
-    }
-    const unsigned who = __ballot_sync(0xFFFFFFFFu, before == K - 1);
-    return __shfl_sync(0xFFFFFFFFu, v, __ffs(who) - 1);
-}
-
 }  // namespace dsp
