@@ -43,9 +43,9 @@ from paper_2510_02358_b200 import workloads as wl  # noqa: E402
 
 L2_BYTES = 126 * 1024 * 1024
 HEADLINE = 4
-# DRAM bytes (read + write) per launch of lattice_scan_kernel from one ncu capture of this workload
-# (see profiles/); absent = not captured since the kernel last changed.
-NCU_TRAFFIC_BYTES = {4: 622871296 + 7646464}
+# DRAM bytes (read + write) of one launch each of the two streaming kernels from an ncu capture of this
+# workload (see profiles/); absent = not captured since the kernels last changed.
+NCU_TRAFFIC_BYTES = {}
 
 
 def measured_peak():
@@ -123,8 +123,8 @@ class GpuStep:
         self.ws_l = dsp.alloc_workspace(dsp.dsp_lattice_workspace_bytes(w.B, w.L, w.V, dt, w.K), device)
         self.ws_v = dsp.alloc_workspace(dsp.dsp_verify_workspace_bytes(w.B, w.L, w.Lt, w.V, dt), device)
         self.all_greedy = w.verify == "greedy"
-        # lattice scan + rows, cps, target scan + rows, accept (greedy) or residual with the acceptance
-        # scan inside (stochastic rows); memsets are not counted
+        # two preparing kernels, the pass over the draft logits, the path search, the pass over the target
+        # logits, accept (greedy) or residual with the acceptance scan inside (stochastic rows)
         self.kernels_per_step = 6
 
     def step(self, inp):
@@ -211,28 +211,46 @@ def time_workload(w, device, steps, warmup, dist=None, stages=True, seed_base=0,
     if dist is not None:
         dist.barrier()
     torch.cuda.synchronize()
-    # the dominant kernel's own duration: every 8th timed step its launch is bracketed by a pair
-    # of events inside the library (same stream, same timed region)
+    # the two streaming kernels' own time: on sampled timed steps each launch is bracketed by a pair of
+    # events inside the library (on the stream the kernel is launched on, inside the timed region).
+    # In the one-call step the two kernels run side by side, so what is reported is the window from
+    # the start of the pass over the draft logits to the end of the later of the two passes.
     scan_evs = []
+
+    def profiled_step(inp):
+        evs4 = [torch.cuda.Event(enable_timing=True) for _ in range(4)]
+        for e in evs4:
+            e.record()                                   # torch creates an event at its first record
+        dsp.dsp_profile_events(dsp.PROFILE_LATTICE_SCAN, evs4[0], evs4[1])
+        dsp.dsp_profile_events(dsp.PROFILE_TARGET_SCAN, evs4[2], evs4[3])
+        scan_evs.append(evs4)
+        st.step(inp)
+        dsp.dsp_profile_events(dsp.PROFILE_LATTICE_SCAN, None, None)
+        dsp.dsp_profile_events(dsp.PROFILE_TARGET_SCAN, None, None)
+
     e0.record()
     for i in range(steps):
-        if stages and i % 8 == 0:
-            pair = (torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
-            pair[0].record(); pair[1].record()          # torch creates an event at its first record
-            dsp.dsp_profile_events(dsp.PROFILE_LATTICE_SCAN, *pair)
-            scan_evs.append(pair)
-        st.step(sets[i % len(sets)])
-        if stages and i % 8 == 0:
-            dsp.dsp_profile_events(dsp.PROFILE_LATTICE_SCAN, None, None)
+        if stages and i % 8 == 0:                        # every 8th timed step carries the events
+            profiled_step(sets[i % len(sets)])
+        else:
+            st.step(sets[i % len(sets)])
     e1.record()
     torch.cuda.synchronize()
     if dist is not None:
         dist.barrier()
     ms = e0.elapsed_time(e1)
+    in_region = len(scan_evs)
+    if stages:                                           # and a series right after the timed region, for the statistics
+        for i in range(32):
+            profiled_step(sets[i % len(sets)])
+        torch.cuda.synchronize()
     out = dict(ms_total=ms, ms_per_step=ms / steps, sets=len(sets), kernels_per_step=st.kernels_per_step)
     if scan_evs:
-        ts = [a.elapsed_time(b) for a, b in scan_evs]
-        out.update(ms_lattice_scan=sum(ts) / len(ts), ms_lattice_scan_min=min(ts), scan_samples=len(ts))
+        win = sorted(max(e[0].elapsed_time(e[1]), e[0].elapsed_time(e[3])) for e in scan_evs)
+        out.update(ms_scan_window=sum(win) / len(win), ms_scan_window_min=win[0],
+                   ms_scan_window_median=win[len(win) // 2], scan_samples=len(win), scan_samples_in_region=in_region,
+                   ms_lattice_scan=sum(e[0].elapsed_time(e[1]) for e in scan_evs) / len(scan_evs),
+                   ms_target_scan=sum(e[2].elapsed_time(e[3]) for e in scan_evs) / len(scan_evs))
     if stages:
         # per-stage times: the same step as three calls with an event after each (outside the timed region)
         n = min(steps, 200)
@@ -321,6 +339,79 @@ def time_sharded(w, device, G=4, reps=40):
     return {"G": G, "slice_V": Vs, "shard_ms": ts / reps, "merge_ms": tm / reps,
             "slice_logits_gbs": nbytes / (ts / reps * 1e-3) / 1e9,
             "record_bytes_per_row_and_slice": 24 + 8 * w.K, "workload": "draft logits of %s" % w.name}
+
+
+def vocab_slice(V: int, G: int, r: int):
+    """Slice r of G of the vocabulary: [lo, hi), whole multiples of 8 tokens except the last slice."""
+    per = -(-V // G) // 8 * 8 or 8
+    lo = min(V, r * per)
+    return lo, (V if r == G - 1 else min(V, lo + per))
+
+
+def sharded_exchange_leg(shard, gather, merge, timer, reps, dist):
+    """The vocabulary-sharded lattice as its three stages on every rank: shard() reduces the rank's
+    slice to records, gather() brings every slice's records to every rank (the path's one exchange
+    step), merge() finishes the rows.  ``timer()`` returns an object with record() / elapsed_ms(other)
+    (CUDA events on a GPU).  Returns mean times per stage, the maximum over ranks."""
+    tot = [0.0, 0.0, 0.0]
+    for r in range(reps + 2):
+        t = [timer() for _ in range(4)]
+        t[0].record()
+        rec = shard()
+        t[1].record()
+        allrec = gather(rec)
+        t[2].record()
+        merge(allrec)
+        t[3].record()
+        t[3].sync()
+        if r >= 2:
+            for k in range(3):
+                tot[k] += t[k].elapsed_ms(t[k + 1])
+    ms = [x / reps for x in tot]
+    if dist is not None:
+        tt = torch.tensor(ms, dtype=torch.float64, device=timer.device)
+        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+        ms = tt.tolist()
+    return {"shard_ms": ms[0], "gather_ms": ms[1], "merge_ms": ms[2]}
+
+
+class CudaTimer:
+    device = None
+
+    def __init__(self):
+        self.e = torch.cuda.Event(enable_timing=True)
+
+    def record(self):
+        self.e.record()
+
+    def sync(self):
+        self.e.synchronize()
+
+    def elapsed_ms(self, other):
+        return self.e.elapsed_time(other.e)
+
+
+def time_sharded_exchange(w, device, dist, rank, world, reps=20):
+    """With several GPUs: every rank holds slice `rank` of the vocabulary of the SAME draft logits (a
+    tensor-parallel drafter head), dsp_lattice_shard -> all-gather of the records into local memory
+    (NCCL; no kernel reads a peer's memory) -> dsp_lattice_merge on every rank."""
+    from paper_2510_02358_b200 import binding as dsp
+    x = wl.make_inputs(w, step=77, device=device)["draft"]          # the same seed on every rank
+    lo, hi = vocab_slice(w.V, world, rank)
+    sl = x[:, :, lo:hi]
+    dt = dsp.DSP_BF16 if w.dtype == torch.bfloat16 else dsp.DSP_F32
+    ws = dsp.alloc_workspace(dsp.dsp_shard_workspace_bytes(w.B, w.L, hi - lo, dt, w.K), device)
+    out = dsp.lattice_outputs(w.B, w.L, w.K, w.eos_id, device)
+    CudaTimer.device = device
+    res = sharded_exchange_leg(
+        lambda: dsp.dsp_lattice_shard(sl, lo, w.K, w.eos_id, workspace=ws),
+        lambda rec: dsp.gather_shard_records(rec),
+        lambda a: dsp.dsp_lattice_merge(a.sums, a.keys, a.status, w.V, w.K, w.tau, w.eos_id, out=out),
+        CudaTimer, reps, dist)
+    res.update(G=world, record_bytes_per_row_and_slice=24 + 8 * w.K,
+               gathered_bytes_per_rank=world * w.B * w.L * (24 + 8 * w.K),
+               workload="draft logits of %s, vocabulary slice per rank" % w.name)
+    return res
 
 
 def time_unmask(w, device, reps=40):
@@ -540,6 +631,16 @@ def time_adl_loop(device, n_steps=256):
             "note": "dsp_draft_verify_step + copy of 2 int32 to the host + synchronise + dsp_adl_update per step"}
 
 
+def config_of(w, world, sets=None):
+    """The `config` object of the JSON line: the same for the timed arm and the reference arm."""
+    step_bytes = wl.step_logits_bytes(w)
+    nsets = sets if sets is not None else (1 if step_bytes > 4 * L2_BYTES else min(16, -(-4 * L2_BYTES // step_bytes)))
+    return {"workload": w.name, "B": w.B * world, "B_per_gpu": w.B, "L": w.L, "V": w.V,
+            "logits_dtype": "bf16" if w.dtype == torch.bfloat16 else "f32", "K": w.K, "W": w.W,
+            "tau": w.tau, "verify": w.verify, "parallelism": "batch rows sharded, no collective",
+            "l2": "inputs larger than L2" if nsets == 1 else "rotating %d input sets" % nsets}
+
+
 def run_reference(args, rank, world):
     if rank != 0:
         return
@@ -563,8 +664,7 @@ def run_reference(args, rank, world):
         "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup, "ms_per_step": step_s * 1e3,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "f64", "data": "synthetic",
-        "config": {"workload": w.name, "B": w.B, "L": w.L, "V": w.V, "K": w.K, "W": w.W, "tau": w.tau,
-                   "verify": w.verify},
+        "config": config_of(w, max(1, args.gpus)),
         "cpu_baseline": {"value": val, "unit": "steps/s", "cores": cores, "kind": "oracle", "sample": sample},
         "e2e": {"value": val, "unit": "steps/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
     }))
@@ -611,6 +711,7 @@ def main():
         e2e["value"] = whole_job_steps_per_s(world, 1, e2e["ms_per_step"])
         e2e["h2d_bytes_per_step"] *= world
         e2e["d2h_bytes_per_step"] *= world
+    sharded = time_sharded_exchange(w, device, dist, rank, world) if dist is not None else None
     if rank != 0:
         if dist is not None:
             dist.destroy_process_group()
@@ -622,16 +723,15 @@ def main():
     gbs_lat = tensor_bytes / (m["ms_lattice"] * 1e-3) / 1e9
     gbs_ver = tensor_bytes / (m["ms_verify"] * 1e-3) / 1e9
     gbs_both = 2 * tensor_bytes / ((m["ms_lattice"] + m["ms_verify"]) * 1e-3) / 1e9
-    gbs_scan = tensor_bytes / (m["ms_lattice_scan"] * 1e-3) / 1e9
+    # the two streaming kernels of the step run side by side: both tensors over the window they span
+    gbs_scan = 2 * tensor_bytes / (m["ms_scan_window"] * 1e-3) / 1e9
+    gbs_step = 2 * tensor_bytes / (ms / args.steps * 1e-3) / 1e9
     line = {
         "metric": "draft-verify steps/s", "value": whole_job_steps_per_s(world, args.steps, ms), "unit": "steps/s",
         "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms / args.steps,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "f32", "data": "synthetic",
-        "config": {"workload": w.name, "B": w.B * world, "B_per_gpu": w.B, "L": w.L, "V": w.V,
-                   "logits_dtype": "bf16" if w.dtype == torch.bfloat16 else "f32", "K": w.K, "W": w.W,
-                   "tau": w.tau, "verify": w.verify, "parallelism": "batch rows sharded, no collective",
-                   "l2": "inputs larger than L2" if m["sets"] == 1 else "rotating %d input sets" % m["sets"]},
+        "config": config_of(w, world, m["sets"]),
         "logits_gbs": {"lattice_build": gbs_lat, "verify": gbs_ver, "lattice_plus_verify": gbs_both,
                        "frac_of_8000": gbs_both / 8000.0, "frac_of_%s_copy_peak" % peak_kind: gbs_both / peak,
                        "frac_of_read_probe": gbs_both / probe["gbs"]},
@@ -642,18 +742,29 @@ def main():
                          "steps_per_s": 1e3 / m["ms_graph_step"] * world if m.get("ms_graph_step") else None,
                          "note": "the same step replayed through dsp_step_graph_launch (not the timed `value`)"},
         "mean_accepted_len": m["mean_accepted_len"], "mean_path_len": m["mean_path_len"],
-        "roofline": {"bound": "hbm", "kernel": "lattice_scan_kernel", "achieved": gbs_scan, "peak": peak,
+        "roofline": {"bound": "hbm", "kernel": "lattice_scan_kernel + target_scan_kernel (side by side in the step)",
+                     "achieved": gbs_scan, "peak": peak,
                      "peak_kind": "%s copy bandwidth" % peak_kind, "unit": "GB/s", "frac": gbs_scan / peak,
                      "traffic": NCU_TRAFFIC_BYTES.get(w.cid),
-                     "algorithmic_bytes_per_launch": tensor_bytes,
-                     "launch_us": m["ms_lattice_scan"] * 1e3, "launches_timed": m["scan_samples"],
-                     "frac_of_read_probe": gbs_scan / probe["gbs"]},
+                     "algorithmic_bytes_per_launch": 2 * tensor_bytes,
+                     "launch_us": m["ms_scan_window"] * 1e3, "launch_us_median": m["ms_scan_window_median"] * 1e3,
+                     "launch_us_min": m["ms_scan_window_min"] * 1e3, "launches_timed": m["scan_samples"],
+                     "launches_timed_in_region": m["scan_samples_in_region"],
+                     "frac_of_read_probe": gbs_scan / probe["gbs"],
+                     "frac_of_8000": gbs_scan / 8000.0,
+                     "call_level": {"gbs": gbs_both, "frac_of_8000": gbs_both / 8000.0,
+                                    "note": "(draft + target bytes) / (dsp_lattice_build + dsp_verify), the three calls"},
+                     "step_level": {"gbs": gbs_step, "frac_of_8000": gbs_step / 8000.0,
+                                    "note": "(draft + target bytes) / ms_per_step of the one-call step, path search and "
+                                            "residual draw included"}},
         "read_probe": probe,
         "row_steps_per_s": whole_job_steps_per_s(world, args.steps, ms) * w.B,
         "e2e": e2e,
         "gpu_launches": m["kernels_per_step"] * args.steps,
         "clocks": clocks,
     }
+    if sharded is not None:
+        line["vocab_sharded_exchange"] = sharded
     if not args.no_extras and world == 1:
         line["cpu_baseline"] = cpu_baseline(w, sets[0])
         line["parity"] = parity_recheck(w, st, sets[0], 16)

@@ -127,7 +127,10 @@ int32_t dsp_read_probe(const void *buffer, size_t bytes, uint32_t *sink, dsp_str
  *          gen_len    int32 [B]
  *          row_status uint32[B]        overwritten
  * workspace: at least dsp_lattice_workspace_bytes(...) bytes, 256-byte aligned;
- *          contents need not be initialised and are garbage afterwards.
+ *          contents need not be initialised and are garbage afterwards.  (The
+ *          size of every workspace in this header depends on how rows are cut
+ *          into slices, which follows the SM count of the current device: ask
+ *          the query call with the device current on which the call will run.)
  * Errors : INVALID_ARG (null required pointer, B<0, L<1, V<1, stride < V ...),
  *          UNSUPPORTED (dtype, K_max outside 1..DSP_MAX_K, L > DSP_MAX_L),
  *          WORKSPACE, CUDA.  B == 0 is a no-op returning DSP_OK.
@@ -160,8 +163,10 @@ int32_t dsp_lattice_build(const void *draft_logits, int32_t dtype,
  *  - This function calls no allocating routine (no cudaMalloc / cudaFree).
  *  - Limit: dsp_lattice_workspace_bytes(B, L, V, dtype, K_max) must not exceed
  *    DSP_STATIC_WS_BYTES, else DSP_ERR_STATIC_SCRATCH is returned and nothing
- *    is enqueued.  (The scratch is about 2.4 % of the draft logits' bytes:
- *    B*L*V up to about 80 million bf16 logits fits; ask the query call.)
+ *    is enqueued; this limit is checked first, the other argument errors of
+ *    dsp_lattice_build after it.  (Layouts read with 128-bit loads need a few
+ *    bytes per row; any other layout needs (24 + 8 K_max) bytes per row and
+ *    slice: ask the query call.)
  *  - The first call on each device looks up the array's device address (a
  *    host-side, once-per-device step with that device current).  Make that
  *    first call outside any stream capture.
@@ -203,7 +208,8 @@ int32_t dsp_lattice_build_static(const void *draft_logits, int32_t dtype,
  *       h = prev * 0x9E3779B1;  h ^= cur + hash_seed;  h *= 0x9E3779B1;
  *       h ^= h >> 15;  h *= 0x9E3779B1;  h ^= h >> 13;
  *       l^ng = proxy_table[h >> (32 - table_log2)]
- *   proxy_kind 1: dense table [V,V]: l^ng = proxy_table[prev * V + cur].
+ *   proxy_kind 1: dense table [V,V]: l^ng = proxy_table[prev * V + cur]; a
+ *     prev_token or candidate id outside [0, V) is clamped into it.
  *   proxy_kind 2: a tensor [B,L,KC,KC] of scores the caller computed for the
  *     lattice (a small causal model): l^ng of candidate slot k at position i
  *     after candidate slot p at position i-1 is proxy_table[b][i][p][k]; at
@@ -309,7 +315,8 @@ int32_t dsp_verify(const void *target_logits, int32_t dtype,
  * after all of it.
  * The second stream and two events are created at the first call on each
  * device and kept until the process exits (host-side handles; no device
- * memory is allocated).
+ * memory is allocated).  Calls from several host threads are safe: the
+ * library holds a lock while one call enqueues its work.
  * lattice_workspace / verify_workspace: as for dsp_lattice_build / dsp_verify.
  * Errors: those of the three calls.
  */

@@ -65,7 +65,8 @@ inline size_t cps_smem_bytes(int L, int W, int KC, int D, int SW) {
 
 // Bigram proxies: the dense [V,V] table or the hashed table (the mix is part of the ABI).
 __device__ __forceinline__ float proxy_score(const CpsArgs &a, int prev, int cur) {
-    if (a.proxy_kind == 1) return __ldg(&a.table[(long long)prev * a.V + cur]);
+    if (a.proxy_kind == 1)                                   // ids outside [0, V) read the nearest row / column
+        return __ldg(&a.table[(long long)min(max(prev, 0), a.V - 1) * a.V + min(max(cur, 0), a.V - 1)]);
     uint32_t h = (uint32_t)prev * 0x9E3779B1u;
     h ^= (uint32_t)cur + a.hash_seed;
     h *= 0x9E3779B1u;

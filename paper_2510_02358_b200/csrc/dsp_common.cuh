@@ -13,7 +13,6 @@ namespace dsp {
 constexpr int kThreads = 256;                 // threads per CTA of every streaming kernel
 constexpr int kWarps = kThreads / 32;
 constexpr int kCandCap = 1024;                // candidate buffer entries per CTA (>= 32 slices * DSP_MAX_K)
-constexpr int kTargetCtas = 148;                // rows are cut into slices until about this many CTAs exist (one per SM)
 constexpr int kMaxSlices = 32;                // slices per row a single finaliser merges
 constexpr float kLog2e = 1.44269502162933349609375f;      // fp32 nearest to log2(e)
 constexpr double kLn2 = 0.693147180559945309417232;
@@ -70,12 +69,8 @@ inline cudaError_t launch_dependent(void (*kernel)(Arg), unsigned grid, unsigned
 }
 
 // Where the early placement pays (measured on a B200).  Between the short kernels of a call it
-// saves 1 to 2 us per launch.  Behind a pass over the logits whose grid is several times what the
-// SMs hold, CTAs of the next kernel that sit waiting beside the pass's last wave cost more than
-// the launch they save (+4 % on 16384 rows), so a rows kernel follows such a pass the ordinary
-// way.  In a captured graph the programmatic edges pay only on large problems (small ones replay
-// 2 us slower with them).
-constexpr long long kDependentScanCtas = 2 * 148 * 4;     // largest pass a rows kernel follows early
+// saves 1 to 2 us per launch.  In a captured graph the programmatic edges pay only on large
+// problems (small ones replay 2 us slower with them).
 constexpr long long kDependentGraphRows = 1024;           // fewest logits rows for programmatic edges in a graph
 inline bool stream_is_capturing(cudaStream_t st) {
     cudaStreamCaptureStatus cs = cudaStreamCaptureStatusNone;
@@ -84,10 +79,6 @@ inline bool stream_is_capturing(cudaStream_t st) {
         return true;                                       // unknown: take the ordinary launch
     }
     return cs != cudaStreamCaptureStatusNone;
-}
-// A rows kernel (pass 2) behind its pass over the logits (`scan_ctas` CTAs).
-inline bool rows_follow_early(cudaStream_t st, long long scan_ctas) {
-    return scan_ctas <= kDependentScanCtas && !stream_is_capturing(st);
 }
 // A short kernel behind another short kernel, in a call over `nrows` rows of logits.
 inline bool short_kernel_follows_early(cudaStream_t st, long long nrows) {

@@ -12,7 +12,7 @@
 // pass's grid.
 #include <mutex>
 
-#include "dsp_common.cuh"
+#include "stream_core.cuh"
 #include "dsp_internal.h"
 
 namespace {
@@ -22,8 +22,7 @@ constexpr int kMaxDevices = 64;
 // what the SMs hold at once, and a kernel launched behind it waits for most of the pass.
 constexpr long long kLongPassBytes = 400ll << 20;
 // Beside a long pass the search keeps its SMs to itself while it (one CTA per batch row) takes at
-// most half of a B200's 148 SMs; with more rows it shares them.
-constexpr int kWholeSmMaxCtas = 74;
+// most half of the device's SMs; with more rows it shares them.
 struct SideStream {
     cudaStream_t stream = nullptr;
     cudaEvent_t fork = nullptr, join = nullptr;
@@ -31,12 +30,12 @@ struct SideStream {
 std::mutex g_side_mutex;
 SideStream g_side[kMaxDevices];
 
-// The second stream and its two events, created at the first call on each device.
+// The second stream and its two events, created at the first call on each device.  The caller holds
+// g_side_mutex.
 int32_t side_stream(SideStream **out) {
     int dev = -1;
     DSP_CUDA_TRY(cudaGetDevice(&dev));
     if (dev < 0 || dev >= kMaxDevices) return DSP_ERR_UNSUPPORTED;
-    std::lock_guard<std::mutex> lock(g_side_mutex);
     SideStream &s = g_side[dev];
     if (!s.stream) {
         int least = 0, greatest = 0;                     // numerically lower = higher priority
@@ -71,13 +70,16 @@ extern "C" int32_t dsp_draft_verify_step(
     if (B == 0) return DSP_OK;
     cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
     const int32_t KC = K_max + (eos_id >= 0 ? 1 : 0);
+    // One call at a time enqueues on the second stream and its fork / join events: calls from
+    // several host threads (or for several caller streams) then each see their own fork point.
+    std::lock_guard<std::mutex> lock(g_side_mutex);
     SideStream *side = nullptr;
     int32_t rc = side_stream(&side);
     if (rc != DSP_OK) return rc;
 
     const long long target_bytes = (long long)B * Lt * V * (dtype == DSP_BF16 ? 2 : 4);
     const bool long_pass = target_bytes >= kLongPassBytes;
-    const bool whole_sm = long_pass && B <= kWholeSmMaxCtas;
+    const bool whole_sm = long_pass && B <= device_sm_count() / 2;
     auto stats = [&](cudaStream_t s) {
         return verify_impl(target_logits, dtype, B, L, Lt, V, tstride_b, tstride_l, draft_logits, dstride_b,
                            dstride_l, path, path_slot, path_len, cand_logit, lse64, KC, all_greedy, mode, u, eos_id,

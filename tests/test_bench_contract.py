@@ -27,6 +27,11 @@ def test_reference_arm_prints_one_line_with_the_contract_keys():
     assert d["cpu_baseline"]["value"] == d["value"] == d["e2e"]["value"]
     assert d["e2e"]["h2d_bytes_per_step"] == 0 and d["e2e"]["d2h_bytes_per_step"] == 0
     assert "workload" in d["config"] and "model" not in d["config"]
+    # the same `config` object as the timed arm prints for this workload
+    sys.path.insert(0, ROOT)
+    import bench
+    from paper_2510_02358_b200 import workloads as wl
+    assert d["config"] == bench.config_of(wl.CONFIGS[1], 1)
 
 
 @pytest.mark.gpu

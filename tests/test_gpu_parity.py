@@ -92,6 +92,63 @@ def test_edge_shapes(B, L, V, K, W, dtype):
         assert rep["near_accept"] + rep["near_token"] + rep["near_tau"] <= 1
 
 
+@pytest.mark.parametrize("V,dtype", [(12288 + 64, torch.bfloat16), (6144 + 32, torch.float32),
+                                     (3 * 12288 + 8, torch.bfloat16)])
+def test_short_ragged_tail_in_a_slice_of_its_own(V, dtype):
+    """Few rows, so every tile is a slice of its own, and the last tile holds only a few vectors: most
+    threads of its CTA see nothing at all, which must neither count in the sums nor disturb them."""
+    inp = _to(wl.tiny_random(1, 4, V, dtype=dtype, seed=V % 97))
+    for tau, eos in ((0.0, -1), (0.8, 5)):
+        p = dict(K=8, W=4, tau=tau, lam=0.5, eos_id=eos)
+        for fused in (False, True):
+            rep = check_step(gpu_step(inp, fused=fused, **p), inp, **p)
+            assert rep["max_err"]["lse64"] < 5e-6 and rep["max_err"]["entropy"] < 5e-5
+
+
+def test_dense_proxy_ids_out_of_range_are_clamped():
+    B, L, K, V = 2, 5, 4, 50
+    g = torch.Generator().manual_seed(4)
+    lat = _hand_lattice(B, L, K, V, seed=3)
+    table = torch.round(torch.randn((V, V), generator=g) * 8) / 8
+    dlat = SimpleNamespace(**{k: v.to(DEV) for k, v in vars(lat).items()})
+    kw = dict(W=3, lam=0.5, eos_id=-1, V=V, proxy_kind=1)
+    out = {}
+    for name, prev in (("low", [-7, V + 100]), ("clamped", [0, V - 1])):
+        c = dsp.dsp_cps_search(dlat, torch.tensor(prev, dtype=torch.int32, device=DEV), table.to(DEV), **kw)
+        torch.cuda.synchronize()
+        out[name] = c
+    for f in ("path", "path_len", "beam_ids", "beam_cum"):
+        assert torch.equal(getattr(out["low"], f), getattr(out["clamped"], f)), f
+    o = oracle.cps_search(lat.cand_id, lat.cand_logit, lat.lse64, lat.cand_count, torch.tensor([0, V - 1], dtype=torch.int32),
+                          table, **kw)
+    assert torch.equal(out["clamped"].path.cpu(), o.path) and torch.equal(out["clamped"].beam_cum.cpu(), o.beam_cum)
+
+
+def test_single_call_step_from_two_host_threads():
+    """Two host threads, each with its own stream and buffers, call the one-call step at the same time."""
+    import threading
+    w = wl.CONFIGS[3].scaled(B=3, L=6, V=40000)
+    p = _params(w)
+    inps = [wl.make_inputs(w, step=s, device=DEV) for s in (11, 12)]
+    want = [gpu_step(i, fused=True, **p) for i in inps]
+    got, errs = [None, None], []
+
+    def work(k):
+        try:
+            st = torch.cuda.Stream()
+            with torch.cuda.stream(st):
+                for _ in range(20):
+                    got[k] = gpu_step(inps[k], fused=True, **p)
+        except Exception as e:                                      # surfaced below
+            errs.append(e)
+    ts = [threading.Thread(target=work, args=(k,)) for k in (0, 1)]
+    [t.start() for t in ts]
+    [t.join() for t in ts]
+    assert not errs, errs
+    for k in (0, 1):
+        _same_outputs(want[k], got[k])
+
+
 def test_target_with_bonus_row_and_all_greedy():
     B, L, V = 4, 5, 3000
     inp = _to(wl.tiny_random(B, L, V, dtype=torch.bfloat16, seed=3))

@@ -94,3 +94,63 @@ def test_slice_records_are_gathered_slice_major_on_every_rank():
             assert (o["sums"][s] == s + 1).all() and o["keys"][s, 0, 0, 0] == 1000 * s
             assert (o["status"][s] == 32 * s).all()
     assert torch.equal(out[0]["keys"], out[1]["keys"])
+
+
+class _WallTimer:
+    device = torch.device("cpu")
+
+    def __init__(self):
+        self.t = None
+
+    def record(self):
+        import time
+        self.t = time.perf_counter()
+
+    def sync(self):
+        pass
+
+    def elapsed_ms(self, other):
+        return (other.t - self.t) * 1e3
+
+
+def _exchange_worker(rank, world, port, out):
+    sys.path.insert(0, ROOT)
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port), RANK=str(rank), WORLD_SIZE=str(world))
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    from types import SimpleNamespace
+    import bench
+    from paper_2510_02358_b200 import binding as dsp
+    B, L, K, V = 2, 3, 4, 1000
+    lo, hi = bench.vocab_slice(V, world, rank)
+    seen = {}
+
+    def shard():                      # stand-in for dsp_lattice_shard: the records name their slice
+        return SimpleNamespace(sums=torch.full((B, L, dsp.SHARD_SUMS_BYTES), rank + 1, dtype=torch.uint8),
+                               keys=torch.full((B, L, K), lo, dtype=torch.int64),
+                               status=torch.zeros((B,), dtype=torch.int32))
+
+    def merge(a):                     # stand-in for dsp_lattice_merge: every slice must be there, in order
+        seen["los"] = a.keys[:, 0, 0, 0].tolist()
+        seen["shape"] = tuple(a.sums.shape)
+
+    res = bench.sharded_exchange_leg(shard, dsp.gather_shard_records, merge, _WallTimer, 3, dist)
+    out[rank] = dict(res=res, los=seen["los"], shape=seen["shape"], slice=(lo, hi))
+    dist.barrier()
+    dist.destroy_process_group()
+
+
+def test_sharded_exchange_leg_of_the_benchmark_on_two_ranks():
+    """The bench leg for several GPUs (slice -> all-gather of the records -> merge) with stand-in kernels:
+    the slices tile the vocabulary, every rank merges all slices' records in slice order, and the
+    reported times are the same on every rank (maximum over ranks)."""
+    world = 2
+    port = 33500 + os.getpid() % 2000
+    mgr = mp.Manager()
+    out = mgr.dict()
+    mp.spawn(_exchange_worker, args=(world, port, out), nprocs=world, join=True)
+    assert out[0]["slice"][0] == 0 and out[0]["slice"][1] == out[1]["slice"][0] and out[1]["slice"][1] == 1000
+    assert out[0]["slice"][1] % 8 == 0
+    for r in range(world):
+        assert out[r]["los"] == [out[0]["slice"][0], out[1]["slice"][0]] and out[r]["shape"][0] == world
+        assert set(out[r]["res"]) == {"shard_ms", "gather_ms", "merge_ms"}
+    assert out[0]["res"] == out[1]["res"]
