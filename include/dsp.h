@@ -305,11 +305,10 @@ int32_t dsp_verify(const void *target_logits, int32_t dtype,
  * results of the three calls (KC = K_max + (eos_id >= 0 ? 1 : 0); row_status is
  * overwritten by the lattice part and OR-ed into by the others; every output of
  * the three calls is written, nullable ones as there).  The one call lets the
- * statistics of the target rows, which need only the target logits, run beside
- * the lattice's finish and the path search, one side on `stream` and the other
- * on a second stream of the library (of the highest priority the device has;
- * on large inputs it carries the finish and the search, whose CTAs then keep
- * their SMs to themselves, otherwise the target statistics); the
+ * pass over the target logits, which needs only those, run beside the lattice
+ * build and the path search, one side on `stream` and the other on a second
+ * stream of the library (of the highest priority the device has; on large
+ * inputs it carries the build and the search, otherwise the target pass); the
  * decisions wait for both.  All work is ordered after what was enqueued on
  * `stream` before the call, and work enqueued on `stream` after it is ordered
  * after all of it.

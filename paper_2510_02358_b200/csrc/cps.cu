@@ -20,7 +20,6 @@ namespace dsp {
 
 constexpr int kMaxKC = DSP_MAX_K + 1;
 constexpr int kStepBudgetBytes = 48 * 1024;        // shared memory for one window of depths
-constexpr size_t kWholeSmBytes = 180 * 1024;       // dynamic shared memory that leaves no room for a streaming CTA
 
 struct CpsArgs {
     const int32_t *cand_id;
@@ -397,7 +396,7 @@ int32_t dsp::cps_search_impl(const int32_t *cand_id, const float *cand_logit,
                                   int32_t *path, int32_t *path_slot, int32_t *path_len,
                                   float *path_score,
                                   int32_t *beam_ids, float *beam_score, float *beam_cum,
-                                  uint32_t *row_status, cudaStream_t stream, bool whole_sm) {
+                                  uint32_t *row_status, cudaStream_t stream) {
     if (B < 0 || L < 1 || KC < 1 || V < 1) return DSP_ERR_INVALID_ARG;
     if (W < 1 || W > DSP_MAX_W || KC > DSP_MAX_K + 1 || L > DSP_MAX_L) return DSP_ERR_UNSUPPORTED;
     if (proxy_kind < 0 || proxy_kind > 3) return DSP_ERR_UNSUPPORTED;
@@ -420,11 +419,7 @@ int32_t dsp::cps_search_impl(const int32_t *cand_id, const float *cand_logit,
     const bool tri = proxy_kind == 3;
     a.SW = tri ? KC : KC * KC;
     a.D = cps_window_depths(L, KC, a.SW);
-    size_t dyn = cps_smem_bytes(L, W, KC, a.D, a.SW);
-    // `whole_sm`: ask for so much shared memory that no CTA of a streaming kernel fits beside this
-    // one on its SM (the search is a chain of shared-memory round trips and barriers, which take
-    // several times longer while a streaming kernel keeps the SM's memory pipeline full)
-    if (whole_sm && dyn < kWholeSmBytes) dyn = kWholeSmBytes;
+    const size_t dyn = cps_smem_bytes(L, W, KC, a.D, a.SW);
     {
         // raise the kernels' dynamic shared memory limit once per device (the attribute is per device)
         static bool done[64] = {};
@@ -435,7 +430,6 @@ int32_t dsp::cps_search_impl(const int32_t *cand_id, const float *cand_logit,
             // window (a window's arrays fill the budget up to one depth's worth of rounding)
             int most = (int)(align_up((size_t)3 * DSP_MAX_L * DSP_MAX_W, 16) + kStepBudgetBytes +
                              (size_t)kMaxKC * 8 + 64);
-            if (most < (int)kWholeSmBytes) most = (int)kWholeSmBytes;
             DSP_CUDA_TRY(cudaFuncSetAttribute(cps_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, most));
             DSP_CUDA_TRY(cudaFuncSetAttribute(cps_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, most));
             if (dev >= 0 && dev < 64) done[dev] = true;
@@ -459,6 +453,5 @@ extern "C" int32_t dsp_cps_search(const int32_t *cand_id, const float *cand_logi
                                   uint32_t *row_status, dsp_stream_t stream) {
     return cps_search_impl(cand_id, cand_logit, lse64, cand_count, B, L, KC, prev_token, proxy_kind, proxy_table,
                            table_log2, hash_seed, V, W, lambda, eos_id, path, path_slot, path_len, path_score,
-                           beam_ids, beam_score, beam_cum, row_status, reinterpret_cast<cudaStream_t>(stream),
-                           false);
+                           beam_ids, beam_score, beam_cum, row_status, reinterpret_cast<cudaStream_t>(stream));
 }

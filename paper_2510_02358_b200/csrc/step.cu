@@ -21,8 +21,6 @@ constexpr int kMaxDevices = 64;
 // Target logits from which the pass over them counts as long: its grid is then several times
 // what the SMs hold at once, and a kernel launched behind it waits for most of the pass.
 constexpr long long kLongPassBytes = 400ll << 20;
-// Beside a long pass the search keeps its SMs to itself while it (one CTA per batch row) takes at
-// most half of the device's SMs; with more rows it shares them.
 struct SideStream {
     cudaStream_t stream = nullptr;
     cudaEvent_t fork = nullptr, join = nullptr;
@@ -79,7 +77,6 @@ extern "C" int32_t dsp_draft_verify_step(
 
     const long long target_bytes = (long long)B * Lt * V * (dtype == DSP_BF16 ? 2 : 4);
     const bool long_pass = target_bytes >= kLongPassBytes;
-    const bool whole_sm = long_pass && B <= device_sm_count() / 2;
     auto stats = [&](cudaStream_t s) {
         return verify_impl(target_logits, dtype, B, L, Lt, V, tstride_b, tstride_l, draft_logits, dstride_b,
                            dstride_l, path, path_slot, path_len, cand_logit, lse64, KC, all_greedy, mode, u, eos_id,
@@ -89,7 +86,7 @@ extern "C" int32_t dsp_draft_verify_step(
     auto search = [&](cudaStream_t s) {
         return cps_search_impl(cand_id, cand_logit, lse64, cand_count, B, L, KC, prev_token, proxy_kind,
                                proxy_table, table_log2, hash_seed, V, W, lambda, eos_id, path, path_slot, path_len,
-                               path_score, beam_ids, beam_score, beam_cum, row_status, s, whole_sm);
+                               path_score, beam_ids, beam_score, beam_cum, row_status, s);
     };
     int32_t rc2 = DSP_OK;
     // The two sides start together: the second stream takes up where the caller's stream stands.
