@@ -63,7 +63,7 @@ __device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, volati
 }
 // Bulk copy global -> this CTA's shared memory; both addresses and the size are multiples of 16.
 // The logits are read once: their L2 lines are marked "evict first", so that streaming them does
-// not push out what pass 1 writes for pass 2 (the table of tile maxima and the sums).
+// not push out what the kernels of a step hand to one another (measured: faster than no hint).
 __device__ __forceinline__ void bulk_load(void *dst, const void *src, uint32_t bytes, uint64_t *bar) {
     uint64_t policy;
     asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(policy));
