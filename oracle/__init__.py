@@ -272,3 +272,35 @@ class Adl:
         k_min, k_max, delta, rho, gran = self.p
         return int(lib().orc_adl_update(C.byref(self.st), _p(a), _p(g), int(a.size), k_min, k_max,
                                         C.c_double(delta), C.c_double(rho), gran))
+
+
+class _BreadthState(C.Structure):
+    _fields_ = [("ema_entropy", C.c_double), ("ema_shortfall", C.c_double), ("K", C.c_int32), ("W", C.c_int32),
+                ("steps", C.c_int32)]
+
+
+class Breadth:
+    """Breadth controller state (the reading of the paper's future work iii): ``K`` / ``W`` for the next step."""
+
+    def __init__(self, K_min=1, K_max=16, W_min=1, W_max=16, rho=0.5):
+        self.p = (int(K_min), int(K_max), int(W_min), int(W_max), float(rho))
+        self.st = _BreadthState()
+        lib().orc_breadth_init(C.byref(self.st), int(K_max), int(W_max))
+
+    K = property(lambda self: int(self.st.K))
+    W = property(lambda self: int(self.st.W))
+    ema_entropy = property(lambda self: float(self.st.ema_entropy))
+    ema_shortfall = property(lambda self: float(self.st.ema_shortfall))
+
+    def update(self, entropy, accepted_len, gen_len):
+        e = _np(entropy, np.float32)
+        a = _np(accepted_len, np.int32).reshape(-1)
+        g = _np(gen_len, np.int32).reshape(-1)
+        B, L = e.shape
+        assert a.size == g.size == B
+        K_min, K_max, W_min, W_max, rho = self.p
+        rc = lib().orc_breadth_update(C.byref(self.st), _p(e), _p(a), _p(g), B, L, K_min, K_max, W_min, W_max,
+                                      C.c_double(rho))
+        if rc != 0:
+            raise ValueError("orc_breadth_update: bad arguments")
+        return self.K, self.W

@@ -778,3 +778,62 @@ int orc_adl_update(orc_adl_state *st, const int32_t *accepted_len, const int32_t
     st->steps += 1;
     return st->k;
 }
+
+/*
+ * Joint control of the search breadth (Sec. 6, future work iii, names it without a rule; the
+ * reading taken, stated in the design doc: the controller of Eq. 10-11 with two more signals).
+ * Per step, batch means:
+ *   H = mean over batch rows b and positions i < max(1, gen_len[b]) of entropy[b,i]   (nats)
+ *   s = mean over b of max(0, gen_len[b] - accepted_len[b]) / max(1, gen_len[b])       (shortfall)
+ *   ema = (1-rho) * ema + rho * signal                  (the form of Eq. 10, both start at 0)
+ *   K' = clip( ceil( exp(ema_H) ), K_min, K_max )       (the drafter's perplexity: how many
+ *                                                        candidates carry its mass)
+ *   W' = clip( ceil( W_min + (W_max - W_min) * ema_s ), W_min, W_max )
+ *                                                       (wider beams while verification cuts
+ *                                                        drafts short)
+ * Init: K = K_max, W = W_max (as Alg. 1 starts the draft length at k_max).
+ */
+typedef struct {
+    double ema_entropy;
+    double ema_shortfall;
+    int32_t K, W;
+    int32_t steps;
+} orc_breadth_state;
+
+void orc_breadth_init(orc_breadth_state *st, int K_max, int W_max)
+{
+    st->ema_entropy = 0.0;
+    st->ema_shortfall = 0.0;
+    st->K = K_max;
+    st->W = W_max;
+    st->steps = 0;
+}
+
+int orc_breadth_update(orc_breadth_state *st, const float *entropy, const int32_t *accepted_len,
+                       const int32_t *gen_len, int B, int L, int K_min, int K_max, int W_min, int W_max,
+                       double rho)
+{
+    if (B < 1 || L < 1) return -1;
+    double Hsum = 0.0, ssum = 0.0;
+    int64_t npos = 0;
+    for (int b = 0; b < B; ++b) {
+        int g = gen_len[b] < 1 ? 1 : (gen_len[b] > L ? L : gen_len[b]);
+        for (int i = 0; i < g; ++i) Hsum += (double)entropy[(int64_t)b * L + i];
+        npos += g;
+        int short_by = gen_len[b] - accepted_len[b];
+        if (short_by < 0) short_by = 0;
+        ssum += (double)short_by / (double)(gen_len[b] < 1 ? 1 : gen_len[b]);
+    }
+    st->ema_entropy = (1.0 - rho) * st->ema_entropy + rho * (Hsum / (double)npos);
+    st->ema_shortfall = (1.0 - rho) * st->ema_shortfall + rho * (ssum / (double)B);
+    double k = ceil(exp(st->ema_entropy));
+    double w = ceil((double)W_min + (double)(W_max - W_min) * st->ema_shortfall);
+    if (k < K_min) k = K_min;
+    if (k > K_max) k = K_max;
+    if (w < W_min) w = W_min;
+    if (w > W_max) w = W_max;
+    st->K = (int32_t)k;
+    st->W = (int32_t)w;
+    st->steps += 1;
+    return 0;
+}
