@@ -594,6 +594,42 @@ int32_t dsp_adl_update(dsp_adl_state *state, const dsp_adl_params *params,
                        const int32_t *accepted_len, const int32_t *gen_len, int32_t B,
                        int32_t *next_L /* host, out, nullable */);
 
+/* -------------------------------------------------------------------------
+ * Breadth controller, host side  (Sec. 6, future work iii: joint control of
+ * draft length and search / pruning breadth; the paper gives no rule, this
+ * is the library's: the moving averages of Eq. 10 on two more signals)
+ *
+ * Per step, from the lattice build's entropy output and the two lengths that
+ * dsp_adl_update takes (batch means; all pointers are HOST pointers):
+ *   H = mean over batch rows b and positions i < max(1, gen_len[b]) of
+ *       entropy[b,i]                                             (nats)
+ *   s = mean over b of max(0, gen_len[b] - accepted_len[b]) / max(1, gen_len[b])
+ *   ema = (1-rho) * ema + rho * signal            (both start at 0)
+ *   K' = clip( ceil( exp(ema_H) ), K_min, K_max )  candidates per position for
+ *        the next step (the drafter's perplexity)
+ *   W' = clip( ceil( W_min + (W_max - W_min) * ema_s ), W_min, W_max )  beam width
+ * dsp_breadth_init: averages 0, K = K_max, W = W_max.  All arithmetic in double.
+ * entropy: float [B,L] (a host copy of dsp_lattice_build's output).
+ * Errors : INVALID_ARG (null pointer, B < 1, L < 1, K_min < 1, K_min > K_max,
+ *          K_max > DSP_MAX_K, W likewise with DSP_MAX_W, rho outside (0,1]).
+ */
+typedef struct dsp_breadth_params {
+    int32_t K_min, K_max, W_min, W_max;
+    double rho;
+} dsp_breadth_params;
+
+typedef struct dsp_breadth_state {
+    double ema_entropy, ema_shortfall;
+    int32_t K, W;     /* candidate cap and beam width for the next step */
+    int32_t steps;    /* updates so far */
+} dsp_breadth_state;
+
+int32_t dsp_breadth_init(dsp_breadth_state *state, const dsp_breadth_params *params);
+int32_t dsp_breadth_update(dsp_breadth_state *state, const dsp_breadth_params *params,
+                           const float *entropy, const int32_t *accepted_len, const int32_t *gen_len,
+                           int32_t B, int32_t L,
+                           int32_t *next_K /* host, out, nullable */, int32_t *next_W /* host, out, nullable */);
+
 #ifdef __cplusplus
 }
 #endif

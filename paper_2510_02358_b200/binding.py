@@ -34,7 +34,7 @@ EXPORTS = ["dsp_strerror", "dsp_last_cuda_error", "dsp_version", "dsp_profile_ev
            "dsp_target_shard", "dsp_verify_merge_workspace_bytes", "dsp_verify_merge",
            "dsp_residual_sample_workspace_bytes", "dsp_residual_sample",
            "dsp_beam_tree", "dsp_verify_tree_workspace_bytes", "dsp_verify_tree",
-           "dsp_adl_init", "dsp_adl_update"]
+           "dsp_adl_init", "dsp_adl_update", "dsp_breadth_init", "dsp_breadth_update"]
 
 
 class DspError(RuntimeError):
@@ -565,3 +565,35 @@ def dsp_adl_update(state: AdlState, params: AdlParams, accepted_len, gen_len) ->
         C.byref(state), C.byref(params), C.c_void_p(a.data_ptr()), C.c_void_p(g.data_ptr()),
         a.numel(), C.byref(nxt)))
     return nxt.value
+
+
+class BreadthParams(C.Structure):
+    _fields_ = [("K_min", C.c_int32), ("K_max", C.c_int32), ("W_min", C.c_int32), ("W_max", C.c_int32),
+                ("rho", C.c_double)]
+
+
+class BreadthState(C.Structure):
+    _fields_ = [("ema_entropy", C.c_double), ("ema_shortfall", C.c_double), ("K", C.c_int32), ("W", C.c_int32),
+                ("steps", C.c_int32)]
+
+
+def dsp_breadth_init(K_min=1, K_max=16, W_min=1, W_max=16, rho=0.5):
+    """Returns (state, params) for dsp_breadth_update."""
+    p = BreadthParams(int(K_min), int(K_max), int(W_min), int(W_max), float(rho))
+    st = BreadthState()
+    _check("dsp_breadth_init", lib().dsp_breadth_init(C.byref(st), C.byref(p)))
+    return st, p
+
+
+def dsp_breadth_update(state: BreadthState, params: BreadthParams, entropy, accepted_len, gen_len):
+    """entropy: host float32 [B,L]; accepted_len / gen_len: host int32 [B].  Returns (K, W) for the next step."""
+    e = torch.as_tensor(entropy, dtype=torch.float32, device="cpu").contiguous()
+    a = torch.as_tensor(accepted_len, dtype=torch.int32, device="cpu").contiguous().view(-1)
+    g = torch.as_tensor(gen_len, dtype=torch.int32, device="cpu").contiguous().view(-1)
+    if e.dim() != 2 or a.numel() != e.shape[0] or g.numel() != e.shape[0]:
+        raise ValueError("entropy must be [B, L] and the two lengths [B]")
+    K, W = C.c_int32(0), C.c_int32(0)
+    _check("dsp_breadth_update", lib().dsp_breadth_update(
+        C.byref(state), C.byref(params), C.c_void_p(e.data_ptr()), C.c_void_p(a.data_ptr()), C.c_void_p(g.data_ptr()),
+        e.shape[0], e.shape[1], C.byref(K), C.byref(W)))
+    return K.value, W.value

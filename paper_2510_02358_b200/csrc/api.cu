@@ -106,3 +106,51 @@ extern "C" int32_t dsp_adl_update(dsp_adl_state *state, const dsp_adl_params *pa
     if (next_L) *next_L = state->k;
     return DSP_OK;
 }
+
+// ---- breadth controller (host): candidate cap from the drafter's perplexity, beam width from
+// the acceptance shortfall, both through moving averages of Eq. 10's form ----
+static bool breadth_params_ok(const dsp_breadth_params *p) {
+    return p && p->K_min >= 1 && p->K_min <= p->K_max && p->K_max <= DSP_MAX_K && p->W_min >= 1 &&
+           p->W_min <= p->W_max && p->W_max <= DSP_MAX_W && p->rho > 0.0 && p->rho <= 1.0;
+}
+
+extern "C" int32_t dsp_breadth_init(dsp_breadth_state *state, const dsp_breadth_params *params) {
+    if (!state || !breadth_params_ok(params)) return DSP_ERR_INVALID_ARG;
+    state->ema_entropy = 0.0;
+    state->ema_shortfall = 0.0;
+    state->K = params->K_max;
+    state->W = params->W_max;
+    state->steps = 0;
+    return DSP_OK;
+}
+
+extern "C" int32_t dsp_breadth_update(dsp_breadth_state *state, const dsp_breadth_params *params,
+                                      const float *entropy, const int32_t *accepted_len, const int32_t *gen_len,
+                                      int32_t B, int32_t L, int32_t *next_K, int32_t *next_W) {
+    if (!state || !breadth_params_ok(params) || !entropy || !accepted_len || !gen_len || B < 1 || L < 1)
+        return DSP_ERR_INVALID_ARG;
+    double h_sum = 0.0, s_sum = 0.0;
+    long long positions = 0;
+    for (int32_t b = 0; b < B; ++b) {
+        const int32_t g = gen_len[b];
+        const int32_t take = g < 1 ? 1 : (g > L ? L : g);           // drafted positions of this row
+        const float *row = entropy + (size_t)b * L;
+        for (int32_t i = 0; i < take; ++i) h_sum += (double)row[i];
+        positions += take;
+        const int32_t cut = g > accepted_len[b] ? g - accepted_len[b] : 0;
+        s_sum += (double)cut / (double)(g < 1 ? 1 : g);
+    }
+    const double rho = params->rho;
+    state->ema_entropy = (1.0 - rho) * state->ema_entropy + rho * (h_sum / (double)positions);
+    state->ema_shortfall = (1.0 - rho) * state->ema_shortfall + rho * (s_sum / (double)B);
+    double k = ceil(exp(state->ema_entropy));
+    double w = ceil((double)params->W_min + (double)(params->W_max - params->W_min) * state->ema_shortfall);
+    k = k < params->K_min ? params->K_min : (k > params->K_max ? params->K_max : k);
+    w = w < params->W_min ? params->W_min : (w > params->W_max ? params->W_max : w);
+    state->K = (int32_t)k;
+    state->W = (int32_t)w;
+    state->steps += 1;
+    if (next_K) *next_K = state->K;
+    if (next_W) *next_W = state->W;
+    return DSP_OK;
+}

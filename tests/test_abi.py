@@ -97,3 +97,31 @@ def test_adl_host_entry_points_follow_the_golden_trajectories():
         dsp.dsp_adl_init(k_min=10, k_max=5)
     with pytest.raises(dsp.DspError):
         dsp.dsp_adl_init(rho=0.0)
+
+
+def test_breadth_host_entry_points_follow_the_hand_computed_steps_and_the_oracle():
+    import torch
+    import oracle
+    st, prm = dsp.dsp_breadth_init(2, 16, 1, 9, 0.5)
+    assert (st.K, st.W) == (16, 9)
+    # the hand-computed steps of tests/test_oracle_breadth.py
+    assert dsp.dsp_breadth_update(st, prm, torch.full((1, 4), 2.0), [1], [4]) == (3, 4)
+    assert dsp.dsp_breadth_update(st, prm, torch.tensor([[4.0, 2.0, 9.0, 9.0]]), [2], [2]) == (8, 3)
+    assert dsp.dsp_breadth_update(st, prm, torch.tensor([[0.5, 7.0, 7.0, 7.0], [1.0, 1.0, 1.0, 1.5]]), [0, 5], [0, 4]) == (5, 2)
+    assert st.ema_entropy == 1.5 and st.ema_shortfall == 0.09375 and st.steps == 3
+    # a random trajectory against the oracle, state for state
+    g = torch.Generator().manual_seed(1)
+    st, prm = dsp.dsp_breadth_init(3, 15, 2, 8, 0.3)
+    ref = oracle.Breadth(3, 15, 2, 8, 0.3)
+    for _ in range(100):
+        B, L = int(torch.randint(1, 5, (1,), generator=g)), int(torch.randint(1, 9, (1,), generator=g))
+        e = 6.0 * torch.rand((B, L), generator=g)
+        acc, gen = torch.randint(0, L + 2, (B,), generator=g), torch.randint(0, L + 1, (B,), generator=g)
+        assert dsp.dsp_breadth_update(st, prm, e, acc, gen) == ref.update(e, acc, gen)
+        assert st.ema_entropy == ref.ema_entropy and st.ema_shortfall == ref.ema_shortfall
+    # argument errors
+    import ctypes as C
+    bad = dsp.BreadthParams(4, 2, 1, 8, 0.5)
+    assert dsp.lib().dsp_breadth_init(C.byref(dsp.BreadthState()), C.byref(bad)) == dsp.DSP_ERR_INVALID_ARG
+    bad = dsp.BreadthParams(1, 64, 1, 8, 0.5)                      # beyond DSP_MAX_K
+    assert dsp.lib().dsp_breadth_init(C.byref(dsp.BreadthState()), C.byref(bad)) == dsp.DSP_ERR_INVALID_ARG

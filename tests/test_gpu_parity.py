@@ -268,6 +268,27 @@ def test_paper_default_settings(B):
         assert abs(st.ema_gen - ref.ema_gen) < 1e-12 and abs(st.ema_acc - ref.ema_acc) < 1e-12
 
 
+def test_breadth_closed_loop_matches_oracle():
+    """Every step's candidate cap and beam width come from the breadth controller fed with the step before."""
+    w0 = wl.CONFIGS[4].scaled(B=4, L=8, V=40000)
+    prm_kw = dict(K_min=2, K_max=16, W_min=2, W_max=12, rho=0.5)
+    st, prm = dsp.dsp_breadth_init(**prm_kw)
+    ref = oracle.Breadth(**prm_kw)
+    seen = set()
+    for t in range(6):
+        K, W = st.K, st.W
+        assert (K, W) == (ref.K, ref.W)
+        seen.add((K, W))
+        w = w0.scaled(K=K, W=W)
+        inp = wl.make_inputs(w, step=t, device=DEV)
+        g = gpu_step(inp, fused=bool(t & 1), **_params(w))
+        check_step(g, inp, **_params(w))
+        nxt = dsp.dsp_breadth_update(st, prm, g.lat.entropy, g.ver.accepted_len, g.lat.gen_len)
+        assert nxt == ref.update(g.lat.entropy, g.ver.accepted_len, g.lat.gen_len)
+        assert st.ema_entropy == ref.ema_entropy and st.ema_shortfall == ref.ema_shortfall
+    assert len(seen) >= 2
+
+
 # ---- the path search alone, on lattices made by hand (sizes and ties the scans rarely give) ----
 def _hand_lattice(B, L, KC, V, seed, *, flat=False, counts=None):
     g = torch.Generator().manual_seed(seed)
