@@ -304,3 +304,22 @@ class Breadth:
         if rc != 0:
             raise ValueError("orc_breadth_update: bad arguments")
         return self.K, self.W
+
+
+def verify_tree_stochastic(target: torch.Tensor, draft: torch.Tensor, tree: SimpleNamespace, u):
+    """Stochastic verification of the tree; target [B, 1 + N, V], draft [B, L, V], u [B, N + 1]."""
+    target, draft = target.contiguous(), draft.contiguous()
+    B, N1, V = target.shape
+    N, L = N1 - 1, draft.shape[1]
+    assert draft.dtype == target.dtype and draft.shape[0] == B and draft.shape[2] == V
+    u_np = _np(u, np.float32)
+    assert u_np.shape == (B, N + 1)
+    o = SimpleNamespace(accepted_len=np.empty((B,), np.int32), accepted_node=np.empty((B, L), np.int32),
+                        next_token=np.empty((B,), np.int32), row_status=np.zeros((B,), np.uint32))
+    rc = lib().orc_verify_tree_stochastic(
+        _logits_ptr(target), _logits_ptr(draft), _dtype_code(target), B, N, L, C.c_int64(V),
+        _p(_np(tree.node_token, np.int32)), _p(_np(tree.node_parent, np.int32)), _p(_np(tree.n_nodes, np.int32)),
+        _p(u_np), _p(o.accepted_len), _p(o.accepted_node), _p(o.next_token), _p(o.row_status))
+    if rc != 0:
+        raise ValueError("orc_verify_tree_stochastic: bad arguments")
+    return SimpleNamespace(**{k: torch.from_numpy(v) for k, v in vars(o).items()})

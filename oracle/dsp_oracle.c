@@ -837,3 +837,114 @@ int orc_breadth_update(orc_breadth_state *st, const float *entropy, const int32_
     st->steps += 1;
     return 0;
 }
+
+/*
+ * Stochastic verification of a token tree (Sec. 2 names tree-based parallel verification and
+ * cites it; the rule is the multi-branch form of Eq. 1 with residual resampling: the siblings
+ * of a node are tried one after the other, and every rejection replaces the target
+ * distribution by the normalised residual before the next sibling is tried).
+ *
+ * target [B, 1+N, V]: row 0 after the prefix, row 1+n after node n.  draft [B, L, V]: row i is
+ * the drafter's distribution q_i of every node at depth i (one refinement step: the left-to-right
+ * proxy of Eq. 6 is the draft row itself).  u [B, N+1]: u[b,n] is the draw used if node n is
+ * tried, u[b,N] the draw of the emitted token.
+ *
+ * Walk from the root (depth i = 0, f = softmax(target row 0)):
+ *   the children of the current node, in node order: child n with token x is accepted iff
+ *   u[b,n] < f(x) / q_i(x) (f(x) > 0 = q_i(x) accepts, f(x) = 0 rejects); accepted: the walk
+ *   moves to n, i += 1, f = softmax(target row 1+n).  Rejected: f <- [f - q_i]_+ / R with
+ *   R = sum_v [f(v) - q_i(v)]_+, and the next sibling is tried against the new f.
+ *   When no child is left (all rejected, a leaf, or i = L): next_token = smallest v with
+ *   f(v) > 0 and sum_{w<=v} f(w) >= u[b,N] * sum_w f(w).
+ *   R = 0 (not a number either): next_token = argmax of the current node's target row,
+ *   ORC_ZERO_RESIDUAL.
+ * accepted_len = nodes walked, accepted_node[b,i] = the i-th of them (-1 beyond).
+ * An existing target row or a used draft row with NaN / +inf or no finite logit flags the batch row.
+ */
+int orc_verify_tree_stochastic(const void *target, const void *draft, int dtype, int B, int N, int L, int64_t V,
+                               const int32_t *node_token, const int32_t *node_parent, const int32_t *n_nodes,
+                               const float *u, int32_t *accepted_len, int32_t *accepted_node,
+                               int32_t *next_token, uint32_t *row_status)
+{
+    if (B < 0 || N < 1 || V < 1 || L < 1) return -1;
+    const size_t es = dtype == 0 ? 4 : 2;
+    #pragma omp parallel for schedule(dynamic)
+    for (int b = 0; b < B; ++b) {
+        const int32_t *tok = node_token + (int64_t)b * N, *par = node_parent + (int64_t)b * N;
+        const int nn = n_nodes[b] < 0 ? 0 : (n_nodes[b] > N ? N : n_nodes[b]);
+        uint32_t status = 0;
+        double *f = (double *)malloc(sizeof(double) * (size_t)V);
+        double *q = (double *)malloc(sizeof(double) * (size_t)V);
+        for (int i = 0; i < L; ++i) accepted_node[(int64_t)b * L + i] = -1;
+        for (int r = 0; r <= nn; ++r) {                 /* every existing row is checked */
+            const char *row = (const char *)target + ((size_t)b * (size_t)(1 + N) + (size_t)r) * (size_t)V * es;
+            if (row_stats(row, dtype, V, NULL, NULL, NULL)) status |= ORC_NONFINITE_INPUT;
+        }
+        int ctx = -1, acc = 0;
+        int64_t token = -1;
+        for (;;) {
+            const char *trow = (const char *)target + ((size_t)b * (size_t)(1 + N) + (size_t)(1 + ctx)) * (size_t)V * es;
+            double lse_t;
+            int64_t am;
+            row_stats(trow, dtype, V, &lse_t, NULL, &am);
+            for (int64_t v = 0; v < V; ++v) f[v] = exp(logit_at(trow, dtype, v) - lse_t);
+            int moved = 0, dead = 0, have_q = 0;
+            for (int n = 0; n < nn && acc < L && !moved && !dead; ++n) {
+                if (par[n] != ctx) continue;
+                if (!have_q) {
+                    const char *drow = (const char *)draft + ((size_t)b * L + (size_t)acc) * (size_t)V * es;
+                    double lse_d;
+                    if (row_stats(drow, dtype, V, &lse_d, NULL, NULL)) status |= ORC_NONFINITE_INPUT;
+                    for (int64_t v = 0; v < V; ++v) q[v] = exp(logit_at(drow, dtype, v) - lse_d);
+                    have_q = 1;
+                }
+                const int32_t x = tok[n];
+                const double fx = f[x], qx = q[x];
+                int ok;
+                if (qx > 0.0) ok = (double)u[(int64_t)b * (N + 1) + n] < fx / qx;
+                else ok = fx > 0.0;
+                if (ok) {
+                    accepted_node[(int64_t)b * L + acc] = n;
+                    ++acc;
+                    ctx = n;
+                    moved = 1;
+                } else {
+                    double R = 0.0;
+                    for (int64_t v = 0; v < V; ++v) {
+                        double r = f[v] - q[v];
+                        f[v] = r > 0.0 ? r : 0.0;
+                        R += f[v];
+                    }
+                    if (!(R > 0.0)) { dead = 1; token = am; status |= ORC_ZERO_RESIDUAL; }
+                    else for (int64_t v = 0; v < V; ++v) f[v] /= R;
+                }
+            }
+            if (moved) continue;
+            if (!dead) {
+                double R = 0.0;
+                for (int64_t v = 0; v < V; ++v) R += f[v];
+                if (!(R > 0.0)) { token = am; status |= ORC_ZERO_RESIDUAL; }
+                else {
+                    const double thr = (double)u[(int64_t)b * (N + 1) + N] * R;
+                    double cum = 0.0;
+                    int64_t last_pos = -1;
+                    for (int64_t v = 0; v < V; ++v) {
+                        cum += f[v];
+                        if (f[v] > 0.0) {
+                            last_pos = v;
+                            if (cum >= thr) { token = v; break; }
+                        }
+                    }
+                    if (token < 0) token = last_pos;    /* rounding at the very top of the CDF */
+                }
+            }
+            break;
+        }
+        accepted_len[b] = acc;
+        next_token[b] = (int32_t)token;
+        if (row_status) row_status[b] = status;
+        free(f);
+        free(q);
+    }
+    return 0;
+}
