@@ -462,7 +462,18 @@ int32_t dsp_residual_sample(const void *target_rows, const void *draft_rows, int
  * walk ended (correction, or bonus after a leaf), tgt_argmax int32 [B,1+N]
  * (-1 for unused rows), row_status (written): DSP_ROW_NONFINITE_INPUT if an
  * existing row holds NaN / +inf or no finite logit, DSP_ROW_TIMEOUT.
- * Stochastic tree verification is not provided.
+ * dsp_verify_tree_stochastic is the stochastic rule along the same tree (Sec. 2:
+ * Eq. 1 with residual resampling, in its multi-branch form): the children of the
+ * current node are tried in node order; child n with token x is accepted iff
+ * u[b,n] < f(x) / q_i(x), where f is the node's current target distribution
+ * (softmax of its target row at first) and q_i the softmax of draft row i, i the
+ * node's depth (f(x) > 0 = q_i(x) accepts, f(x) = 0 rejects); a rejection replaces
+ * f by [f - q_i]_+ / R (R its mass) before the next sibling is tried.  When no
+ * child is left (all rejected, a leaf, depth L) next_token is the smallest v with
+ * f(v) > 0 and sum_{w<=v} f(w) >= u[b,N] * sum_w f(w); R = 0 gives the argmax of
+ * the node's target row and DSP_ROW_ZERO_RESIDUAL.  draft_logits [B,L,V];
+ * u float [B,N+1] in [0,1).  At most DSP_MAX_W children of one node are tried (a
+ * tree of dsp_beam_tree has no more).  Sums run in double in a fixed order.
  * workspace: dsp_verify_tree_workspace_bytes(B, N, V, dtype), 256-byte aligned.
  * Errors : INVALID_ARG, UNSUPPORTED (W > DSP_MAX_W, L > DSP_MAX_L,
  *          N + 1 > DSP_MAX_L, dtype), WORKSPACE, CUDA.
@@ -472,6 +483,14 @@ int32_t dsp_beam_tree(const int32_t *beam_ids, const int32_t *path_len, int32_t 
                       int32_t *beam_node, int32_t *n_nodes, dsp_stream_t stream);
 int32_t dsp_verify_tree_workspace_bytes(int32_t B, int32_t N, int32_t V, int32_t dtype,
                                         size_t *bytes /* host, out */);
+int32_t dsp_verify_tree_stochastic(const void *target_logits, const void *draft_logits, int32_t dtype,
+                                   int32_t B, int32_t N, int32_t L, int32_t V,
+                                   int64_t tstride_b, int64_t tstride_l, int64_t dstride_b, int64_t dstride_l,
+                                   const int32_t *node_token, const int32_t *node_parent, const int32_t *n_nodes,
+                                   const float *u,
+                                   int32_t *accepted_len, int32_t *accepted_node, int32_t *next_token,
+                                   int32_t *tgt_argmax, uint32_t *row_status,
+                                   void *workspace, size_t workspace_bytes, dsp_stream_t stream);
 int32_t dsp_verify_tree(const void *target_logits, int32_t dtype, int32_t B, int32_t N, int32_t V,
                         int64_t stride_b, int64_t stride_l,
                         const int32_t *node_token, const int32_t *node_parent, const int32_t *n_nodes,

@@ -33,7 +33,7 @@ EXPORTS = ["dsp_strerror", "dsp_last_cuda_error", "dsp_version", "dsp_profile_ev
            "dsp_shard_workspace_bytes", "dsp_lattice_shard", "dsp_merge_workspace_bytes", "dsp_lattice_merge",
            "dsp_target_shard", "dsp_verify_merge_workspace_bytes", "dsp_verify_merge",
            "dsp_residual_sample_workspace_bytes", "dsp_residual_sample",
-           "dsp_beam_tree", "dsp_verify_tree_workspace_bytes", "dsp_verify_tree",
+           "dsp_beam_tree", "dsp_verify_tree_workspace_bytes", "dsp_verify_tree", "dsp_verify_tree_stochastic",
            "dsp_adl_init", "dsp_adl_update", "dsp_breadth_init", "dsp_breadth_update"]
 
 
@@ -499,6 +499,33 @@ def dsp_verify_tree(target: torch.Tensor, tree: SimpleNamespace, L: int, *,
         _ptr(tree.n_nodes), L, _ptr(out.accepted_len), _ptr(out.accepted_node), _ptr(out.next_token),
         _ptr(out.tgt_argmax), _ptr(out.row_status), _ptr(workspace), C.c_size_t(workspace.numel()),
         _stream(stream)))
+    return out
+
+
+def dsp_verify_tree_stochastic(target: torch.Tensor, draft: torch.Tensor, tree: SimpleNamespace, u: torch.Tensor, *,
+                               workspace: Optional[torch.Tensor] = None, stream=None) -> SimpleNamespace:
+    """Stochastic verification of the token tree; ``target`` [B, 1 + N, V], ``draft`` [B, L, V], ``u`` fp32 [B, N + 1]."""
+    B, N1, V, tsb, tsl = _logits3(target, "target")
+    Bd, L, Vd, dsb, dsl = _logits3(draft, "draft")
+    N = N1 - 1
+    if tuple(tree.node_token.shape) != (B, N) or (Bd, Vd) != (B, V) or draft.dtype != target.dtype:
+        raise ValueError("target must have one row per node slot plus one, draft the same batch, vocabulary and dtype")
+    if u.dtype != torch.float32 or tuple(u.shape) != (B, N + 1) or not u.is_contiguous() or u.device != target.device:
+        raise ValueError("u must be a contiguous fp32 [B, N + 1] tensor on the logits' device")
+    dev = target.device
+    dt = _dtype(target)
+    e = lambda shape: torch.empty(shape, dtype=torch.int32, device=dev)
+    out = SimpleNamespace(accepted_len=e((B,)), accepted_node=e((B, L)), next_token=e((B,)),
+                          tgt_argmax=e((B, N1)), row_status=e((B,)))
+    n = C.c_size_t(0)
+    _check("dsp_verify_tree_workspace_bytes", lib().dsp_verify_tree_workspace_bytes(B, N, V, dt, C.byref(n)))
+    if workspace is None:
+        workspace = alloc_workspace(n.value, dev)
+    _check("dsp_verify_tree_stochastic", lib().dsp_verify_tree_stochastic(
+        _ptr(target), _ptr(draft), dt, B, N, L, V, C.c_int64(tsb), C.c_int64(tsl), C.c_int64(dsb), C.c_int64(dsl),
+        _ptr(tree.node_token), _ptr(tree.node_parent), _ptr(tree.n_nodes), _ptr(u),
+        _ptr(out.accepted_len), _ptr(out.accepted_node), _ptr(out.next_token), _ptr(out.tgt_argmax),
+        _ptr(out.row_status), _ptr(workspace), C.c_size_t(workspace.numel()), _stream(stream)))
     return out
 
 

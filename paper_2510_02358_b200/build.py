@@ -8,7 +8,7 @@ PKG = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(PKG)
 CSRC = os.path.join(PKG, "csrc")
 LIB = os.path.join(PKG, "libdsp.so")
-SOURCES = ["api.cu", "lattice.cu", "cps.cu", "verify.cu", "step.cu", "step_graph.cu", "unmask.cu", "shard.cu", "tree.cu"]
+SOURCES = ["api.cu", "lattice.cu", "cps.cu", "verify.cu", "step.cu", "step_graph.cu", "unmask.cu", "shard.cu", "tree.cu", "tree_stochastic.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "-shared"]
 

@@ -43,4 +43,10 @@ int32_t unmask_impl(const void *logits, int32_t dtype, int32_t B, int32_t L, int
                     int32_t *n_left, uint32_t *row_status,
                     void *workspace, size_t workspace_bytes, cudaStream_t st);
 
+// First half of the tree verifications: the argmax of every existing target row of the tree and
+// the batch rows' status; workspace as dsp_verify_tree_workspace_bytes says.
+int32_t tree_row_stats(const void *target_logits, int32_t dtype, int32_t B, int32_t N, int32_t V,
+                       int64_t stride_b, int64_t stride_l, const int32_t *n_nodes, int32_t *tgt_argmax,
+                       uint32_t *row_status, void *workspace, size_t workspace_bytes, cudaStream_t st);
+
 }  // namespace dsp

@@ -146,6 +146,29 @@ static TreeWs tree_ws_layout(int64_t B, int64_t rows, size_t unmask_bytes) {
 
 using namespace dsp;
 
+// Argmax of every existing row of a tree's target logits (row 0 and the rows of the nodes; -1 for
+// unused slots) and the batch rows' status (NaN / +inf, time-outs), by the streaming kernels of the
+// refinement step: nothing is revealed (n_update = 0), so its `tokens` argument is never written.
+int32_t dsp::tree_row_stats(const void *target_logits, int32_t dtype, int32_t B, int32_t N, int32_t V,
+                            int64_t stride_b, int64_t stride_l, const int32_t *n_nodes, int32_t *tgt_argmax,
+                            uint32_t *row_status, void *workspace, size_t workspace_bytes, cudaStream_t st) {
+    if ((reinterpret_cast<uintptr_t>(workspace) & 255) != 0) return DSP_ERR_INVALID_ARG;
+    size_t un = 0;
+    const int32_t rc = dsp_unmask_workspace_bytes(B, N + 1, V, dtype, &un);
+    if (rc != DSP_OK) return rc;
+    const TreeWs w = tree_ws_layout(B, N + 1, un);
+    if (workspace_bytes < w.total) return DSP_ERR_WORKSPACE;
+    unsigned char *ws = static_cast<unsigned char *>(workspace);
+    uint8_t *masked = ws + w.off_masked;
+    float *conf = reinterpret_cast<float *>(ws + w.off_conf);
+    int32_t *left = reinterpret_cast<int32_t *>(ws + w.off_left);
+    const long long cells = (long long)B * (1 + N);
+    tree_rows_kernel<<<(unsigned)((cells + 255) / 256), 256, 0, st>>>(B, N, n_nodes, masked);
+    DSP_CUDA_TRY(cudaGetLastError());
+    return unmask_impl(target_logits, dtype, B, N + 1, V, stride_b, stride_l, 0, tgt_argmax, masked, tgt_argmax, conf,
+                       left, row_status, ws + w.off_unmask, un, st);
+}
+
 extern "C" int32_t dsp_beam_tree(const int32_t *beam_ids, const int32_t *path_len, int32_t B, int32_t W, int32_t L,
                                  int32_t *node_token, int32_t *node_parent, int32_t *node_depth,
                                  int32_t *beam_node, int32_t *n_nodes, dsp_stream_t stream) {
@@ -187,23 +210,9 @@ extern "C" int32_t dsp_verify_tree(const void *target_logits, int32_t dtype, int
     if (!target_logits || !node_token || !node_parent || !n_nodes || !accepted_len || !accepted_node || !next_token ||
         !tgt_argmax || !row_status || !workspace)
         return DSP_ERR_INVALID_ARG;
-    if ((reinterpret_cast<uintptr_t>(workspace) & 255) != 0) return DSP_ERR_INVALID_ARG;
-    size_t un = 0;
-    int32_t rc = dsp_unmask_workspace_bytes(B, N + 1, V, dtype, &un);
-    if (rc != DSP_OK) return rc;
-    const TreeWs w = tree_ws_layout(B, N + 1, un);
-    if (workspace_bytes < w.total) return DSP_ERR_WORKSPACE;
     cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
-    unsigned char *ws = static_cast<unsigned char *>(workspace);
-    uint8_t *masked = ws + w.off_masked;
-    float *conf = reinterpret_cast<float *>(ws + w.off_conf);
-    int32_t *left = reinterpret_cast<int32_t *>(ws + w.off_left);
-    const long long cells = (long long)B * (1 + N);
-    tree_rows_kernel<<<(unsigned)((cells + 255) / 256), 256, 0, st>>>(B, N, n_nodes, masked);
-    DSP_CUDA_TRY(cudaGetLastError());
-    // row statistics of the existing rows only; nothing is revealed (n_update = 0), so `tokens` is never written
-    rc = unmask_impl(target_logits, dtype, B, N + 1, V, stride_b, stride_l, 0, tgt_argmax, masked, tgt_argmax, conf,
-                     left, row_status, ws + w.off_unmask, un, st);
+    const int32_t rc = tree_row_stats(target_logits, dtype, B, N, V, stride_b, stride_l, n_nodes, tgt_argmax, row_status,
+                                      workspace, workspace_bytes, st);
     if (rc != DSP_OK) return rc;
     WalkArgs k;
     k.B = B; k.N = N; k.L = L;

@@ -600,6 +600,52 @@ def test_beam_tree_and_its_greedy_verification(B, L, V, K, W, dtype):
     assert (out.row_status.cpu() != 0).tolist() == (o.row_status != 0).tolist() == [True] + [False] * (B - 1)
 
 
+@pytest.mark.parametrize("B,L,V,K,W,dtype,sigma", [
+    (4, 5, 3000, 4, 6, torch.float32, 0.7),
+    (3, 6, 20000, 4, 8, torch.bfloat16, 0.3),     # target close to the draft: deep walks
+    (3, 4, 5003, 3, 4, torch.bfloat16, 1.5),      # rows that are not 16-byte aligned; many rejections
+    (2, 8, 1000, 2, 1, torch.float32, 0.5),       # one beam: the single-path rule
+])
+def test_stochastic_tree_verification_matches_oracle(B, L, V, K, W, dtype, sigma):
+    inp = _to(wl.tiny_random(B, L, V, dtype=dtype, seed=L * 3 + W))
+    lat = dsp.dsp_lattice_build(inp["draft"], K)
+    cps = dsp.dsp_cps_search(lat, inp["prev_token"], inp["table"], W=W, lam=0.5, table_log2=inp["table_log2"],
+                             hash_seed=inp["hash_seed"], V=V)
+    tree = dsp.dsp_beam_tree(cps)
+    torch.cuda.synchronize()
+    ot = oracle.beam_tree(cps.beam_ids.cpu(), cps.path_len.cpu())
+    N = W * L
+    g = torch.Generator().manual_seed(B + W)
+    draft = inp["draft"].cpu()
+    # a causal target: the row after a node is the draft row of the next depth plus noise (row 0: depth 0)
+    target = torch.zeros((B, 1 + N, V))
+    for b in range(B):
+        for r in range(1 + int(ot.n_nodes[b])):
+            depth = 0 if r == 0 else int(ot.node_depth[b, r - 1]) + 1
+            base = draft[b, min(depth, L - 1)].float()
+            target[b, r] = base + sigma * torch.randn(V, generator=g)
+        target[b, 1 + int(ot.n_nodes[b]):] = float("nan")    # rows of unused slots must not matter
+    target = target.to(dtype)
+    u = torch.rand((B, N + 1), generator=g)
+    o = oracle.verify_tree_stochastic(target, draft, ot, u)
+    out = dsp.dsp_verify_tree_stochastic(target.to(DEV), inp["draft"], tree, u.to(DEV))
+    torch.cuda.synchronize()
+    assert (o.row_status == 0).all() and (out.row_status.cpu() == 0).all()
+    for name in ("accepted_len", "accepted_node", "next_token"):
+        assert torch.equal(getattr(out, name).cpu(), getattr(o, name)), name
+    assert (out.next_token >= 0).all()
+    if W > 1:                                                # one path alone would have done no better
+        single = oracle.verify_tree_stochastic(target, draft, SimpleNamespace(
+            node_token=ot.node_token, node_parent=ot.node_parent, n_nodes=cps.path_len.cpu()), u)
+        assert (o.accepted_len >= single.accepted_len).all()
+    bad = target.clone()
+    bad[0, 1, 3] = float("nan")                              # an existing row goes bad: the batch row is flagged
+    out = dsp.dsp_verify_tree_stochastic(bad.to(DEV), inp["draft"], tree, u.to(DEV))
+    torch.cuda.synchronize()
+    ob = oracle.verify_tree_stochastic(bad, draft, ot, u)
+    assert ((out.row_status.cpu() & dsp.ROW_NONFINITE_INPUT) != 0).tolist() == ((ob.row_status & oracle.NONFINITE_INPUT) != 0).tolist()
+
+
 # ---- the drafter's refinement step (Eq. 5) ----
 def _check_unmask(x, tokens, masked, n, ws=None):
     """One step on both sides from the same state; returns the new state (the GPU's)."""
