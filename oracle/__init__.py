@@ -119,7 +119,7 @@ def lattice_build(draft: torch.Tensor, K_max: int, tau: float = 0.0, eos_id: int
 
 def cps_search(cand_id, cand_logit, lse64, cand_count, prev_token, table, *, W: int, lam: float,
                eos_id: int = -1, proxy_kind: int = 0, table_log2: int = 0, hash_seed: int = 0,
-               V: int = 0):
+               V: int = 0, ver_score=None, mu: float = 0.0):
     cand_id = _np(cand_id, np.int32)
     cand_logit = _np(cand_logit, np.float32)
     lse64 = _np(lse64, np.float64)
@@ -132,10 +132,12 @@ def cps_search(cand_id, cand_logit, lse64, cand_count, prev_token, table, *, W: 
         path_len=np.empty((B,), np.int32), path_score=np.empty((B,), np.float32),
         beam_ids=np.empty((B, W, L), np.int32), beam_score=np.empty((B, W), np.float32),
         beam_cum=np.empty((B, W), np.float32), row_status=np.zeros((B,), np.uint32))
-    rc = lib().orc_cps_search(
+    ver = _np(ver_score, np.float32)
+    assert ver is None or ver.shape == (B, L, KC)
+    rc = lib().orc_cps_search_biased(
         _p(cand_id), _p(cand_logit), _p(lse64), _p(cand_count), B, L, KC, _p(prev_token),
         proxy_kind, _p(table), table_log2, C.c_uint32(hash_seed & 0xFFFFFFFF), C.c_int64(V), W,
-        C.c_float(lam), eos_id, _p(o.path), _p(o.path_slot), _p(o.path_len), _p(o.path_score),
+        C.c_float(lam), eos_id, _p(ver) if ver is not None else None, C.c_float(mu), _p(o.path), _p(o.path_slot), _p(o.path_len), _p(o.path_score),
         _p(o.beam_ids), _p(o.beam_score), _p(o.beam_cum), _p(o.row_status))
     if rc != 0:
         raise ValueError("orc_cps_search: bad arguments")

@@ -324,12 +324,17 @@ static int exp_before(const expansion *a, const expansion *b)
  * double from cand_logit - lse64, beam_ids[B,W,L], beam_score[B,W] (Eq. 8 per
  * beam, -inf where no beam), beam_cum[B,W] (the fp32 ranking quantity).
  * beam_* may be NULL.
+ *
+ * Verifier-aware scoring (Sec. 6, future work ii, names it without a rule; the reading taken):
+ * a third term mu * l^ver in Eq. 8, with l^ver a per-candidate log-score from the verifier's
+ * side that the caller supplies slot by slot, ver_score[B,L,KC] (NULL or mu = 0: Eq. 8 as it is):
+ *   step = fp32( fp32( fp32(lambda*g) + fp32((1-lambda)*n) ) + fp32(mu * v) ).
  */
-int orc_cps_search(const int32_t *cand_id, const float *cand_logit, const double *lse64,
+int orc_cps_search_biased(const int32_t *cand_id, const float *cand_logit, const double *lse64,
                    const int32_t *cand_count, int B, int L, int KC,
                    const int32_t *prev_token, int proxy_kind, const float *table,
                    int table_log2, uint32_t hash_seed, int64_t V,
-                   int W, float lambda, int eos_id,
+                   int W, float lambda, int eos_id, const float *ver_score, float mu,
                    int32_t *path, int32_t *path_slot, int32_t *path_len, float *path_score,
                    int32_t *beam_ids, float *beam_score, float *beam_cum,
                    uint32_t *row_status)
@@ -364,6 +369,10 @@ int orc_cps_search(const int32_t *cand_id, const float *cand_logit, const double
                     volatile float a = lambda * g;
                     volatile float c = oml * ng;
                     volatile float step = a + c;
+                    if (ver_score) {
+                        volatile float v = mu * ver_score[r * KC + k];
+                        step = step + v;
+                    }
                     volatile float s = cum[w] + step;
                     ex[n].cum = s;
                     ex[n].tok = tok;
@@ -414,6 +423,7 @@ int orc_cps_search(const int32_t *cand_id, const float *cand_logit, const double
                                                   b, L, KC, i, slots[w * L + i], ids[w * L + i],
                                                   ids + w * L, slots + w * L);
                     s += (double)lambda * ldlm + (double)oml * lng;
+                    if (ver_score) s += (double)mu * (double)ver_score[r * KC + slots[w * L + i]];
                 }
             }
             if (w == 0) path_score[b] = (float)s;
@@ -427,6 +437,21 @@ int orc_cps_search(const int32_t *cand_id, const float *cand_logit, const double
         free(ids); free(slots); free(nids); free(nslots); free(cum); free(ncum); free(ex);
     }
     return 0;
+}
+
+/* Eq. 8 as the paper has it: no verifier-side term. */
+int orc_cps_search(const int32_t *cand_id, const float *cand_logit, const double *lse64,
+                   const int32_t *cand_count, int B, int L, int KC,
+                   const int32_t *prev_token, int proxy_kind, const float *table,
+                   int table_log2, uint32_t hash_seed, int64_t V,
+                   int W, float lambda, int eos_id,
+                   int32_t *path, int32_t *path_slot, int32_t *path_len, float *path_score,
+                   int32_t *beam_ids, float *beam_score, float *beam_cum,
+                   uint32_t *row_status)
+{
+    return orc_cps_search_biased(cand_id, cand_logit, lse64, cand_count, B, L, KC, prev_token, proxy_kind, table,
+                                 table_log2, hash_seed, V, W, lambda, eos_id, NULL, 0.0f, path, path_slot, path_len,
+                                 path_score, beam_ids, beam_score, beam_cum, row_status);
 }
 
 /*

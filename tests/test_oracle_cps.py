@@ -304,3 +304,45 @@ def test_tensor_proxy_built_from_the_dense_table_gives_the_dense_search():
                             proxy_kind=2, V=V)
     for k in ("path", "path_slot", "path_len", "beam_ids", "beam_cum", "path_score", "beam_score"):
         assert torch.equal(getattr(out, k), getattr(dense, k)), k
+
+
+# ---- verifier-aware scoring: a third term mu * l^ver(position, slot) in Eq. 8 ----
+@pytest.mark.parametrize("L,K,seed,mu", [(3, 4, 10, 0.7), (4, 3, 11, 1.5), (5, 2, 12, 0.25)])
+def test_verifier_term_wide_beam_equals_brute_force(L, K, seed, mu):
+    V, lam = 12, 0.5
+    _, lat, table, prev = _lattice(L, V, K, seed)
+    g = torch.Generator().manual_seed(seed + 100)
+    ver = -5.0 * torch.rand((1, L, K), generator=g)
+    W = K ** (L - 1)
+    out = oracle.cps_search(lat.cand_id, lat.cand_logit, lat.lse64, lat.cand_count, prev, table, W=W, lam=lam,
+                            proxy_kind=1, V=V, ver_score=ver, mu=mu)
+    scored = []
+    for slots in itertools.product(*[range(c) for c in lat.cand_count[0].tolist()]):
+        ids = [int(lat.cand_id[0, i, k]) for i, k in enumerate(slots)]
+        s = _eq8(lat, table, prev, 0, ids, slots, lam) + mu * sum(float(ver[0, i, k]) for i, k in enumerate(slots))
+        scored.append((s, ids))
+    scored.sort(key=lambda t: -t[0])
+    assert abs(out.path_score.item() - scored[0][0]) < 1e-4
+    if scored[0][0] - scored[1][0] > 1e-4:
+        assert out.path[0].tolist() == scored[0][1]
+    nb = min(W, len(scored))
+    assert np.allclose(out.beam_score[0, :nb].double().numpy(), np.array([s for s, _ in scored[:nb]]), atol=1e-4)
+
+
+def test_verifier_term_limits():
+    V, L, K, lam = 20, 6, 4, 0.5
+    _, lat, table, prev = _lattice(L, V, K, 21, B=3)
+    g = torch.Generator().manual_seed(5)
+    ver = -4.0 * torch.rand((3, L, K), generator=g)
+    kw = dict(W=3, lam=lam, proxy_kind=1, V=V)
+    base = oracle.cps_search(lat.cand_id, lat.cand_logit, lat.lse64, lat.cand_count, prev, table, **kw)
+    zero = oracle.cps_search(lat.cand_id, lat.cand_logit, lat.lse64, lat.cand_count, prev, table, ver_score=ver, mu=0.0, **kw)
+    for f in ("path", "path_len", "beam_ids", "beam_cum", "path_score"):       # mu = 0: Eq. 8 as it is, bit for bit
+        assert torch.equal(getattr(base, f), getattr(zero, f)), f
+    big = oracle.cps_search(lat.cand_id, lat.cand_logit, lat.lse64, lat.cand_count, prev, table, ver_score=ver, mu=1e4, **kw)
+    want = torch.gather(lat.cand_id, 2, ver.argmax(dim=2, keepdim=True)).squeeze(2)   # the verifier's favourite everywhere
+    assert torch.equal(big.path, want)
+    const = oracle.cps_search(lat.cand_id, lat.cand_logit, lat.lse64, lat.cand_count, prev, table,
+                              ver_score=torch.full((3, L, K), -2.0), mu=0.5, **kw)
+    assert torch.equal(const.path, base.path)                                   # a constant shifts every path alike
+    assert torch.allclose(const.path_score, base.path_score - 0.5 * 2.0 * L, atol=1e-4)
