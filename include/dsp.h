@@ -249,6 +249,40 @@ int32_t dsp_cps_search(const int32_t *cand_id, const float *cand_logit,
                        uint32_t *row_status, dsp_stream_t stream);
 
 /* -------------------------------------------------------------------------
+ * Path search with a verifier-side term  (Sec. 6, future work ii: a scoring
+ * that takes the verifier into account; the paper gives no rule, this is the
+ * reading taken)
+ *
+ * dsp_cps_search with a third term in the path score,
+ *   S(pi) = sum_i [ lambda * l^dlm_i(pi_i) + (1-lambda) * l^ng(pi_{i-1}, pi_i)
+ *                   + mu * l^ver_i(pi_i) ],
+ * where l^ver is a log-score of each lattice candidate from the verifier's
+ * side (a distilled head, a cached verifier row, a unigram of the verifier:
+ * the caller's choice), given slot by slot:
+ *   ver_score float [B,L,KC] (device; nullable): entry [b,i,k] scores candidate
+ *             slot k of position i; slots at or beyond cand_count are not read.
+ *   mu        float: its weight (finite; any sign).
+ * The ranking step becomes  step = fl( fl( fl(lambda*g) + fl((1-lambda)*n) )
+ * + fl(mu * v) );  path_score and beam_score include the term.  With
+ * ver_score null the call is dsp_cps_search bit for bit (mu is then ignored).
+ * Everything else (arguments, outputs, order of ties, early stop, errors) is as
+ * for dsp_cps_search; INVALID_ARG also for a NaN or infinite mu.
+ * dsp_draft_verify_step and the step graph search without the term: a caller
+ * that wants it makes the three calls.
+ */
+int32_t dsp_cps_search_biased(const int32_t *cand_id, const float *cand_logit,
+                              const double *lse64, const int32_t *cand_count,
+                              int32_t B, int32_t L, int32_t KC,
+                              const int32_t *prev_token,
+                              int32_t proxy_kind, const float *proxy_table, int32_t table_log2,
+                              uint32_t hash_seed, int32_t V,
+                              int32_t W, float lambda, int32_t eos_id,
+                              const float *ver_score, float mu,
+                              int32_t *path, int32_t *path_slot, int32_t *path_len, float *path_score,
+                              int32_t *beam_ids, float *beam_score, float *beam_cum,
+                              uint32_t *row_status, dsp_stream_t stream);
+
+/* -------------------------------------------------------------------------
  * Verification  (Sec. 2: acceptance rule Eq. 1, residual resampling, accepted
  *                length Eq. 2; Sec. 4: greedy = temperature 0; Alg. 1 stage 3;
  *                the drafter probability q is the draft row's own softmax, the

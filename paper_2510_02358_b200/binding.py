@@ -27,7 +27,7 @@ ROW_TIMEOUT = 32
 DSP_MAX_K, DSP_MAX_W, DSP_MAX_L = 32, 32, 1024
 
 EXPORTS = ["dsp_strerror", "dsp_last_cuda_error", "dsp_version", "dsp_profile_events", "dsp_read_probe", "dsp_lattice_workspace_bytes",
-           "dsp_lattice_build", "dsp_lattice_build_static", "dsp_cps_search", "dsp_verify_workspace_bytes", "dsp_verify", "dsp_draft_verify_step",
+           "dsp_lattice_build", "dsp_lattice_build_static", "dsp_cps_search", "dsp_cps_search_biased", "dsp_verify_workspace_bytes", "dsp_verify", "dsp_draft_verify_step",
            "dsp_step_graph_create", "dsp_step_graph_launch", "dsp_step_graph_destroy",
            "dsp_unmask_workspace_bytes", "dsp_unmask_step",
            "dsp_shard_workspace_bytes", "dsp_lattice_shard", "dsp_merge_workspace_bytes", "dsp_lattice_merge",
@@ -211,6 +211,26 @@ def dsp_cps_search(lat: SimpleNamespace, prev_token: torch.Tensor, table: torch.
         W, C.c_float(lam), eos_id, _ptr(out.path), _ptr(out.path_slot), _ptr(out.path_len),
         _ptr(out.path_score), _ptr(out.beam_ids), _ptr(out.beam_score), _ptr(out.beam_cum),
         _ptr(row_status), _stream(stream)))
+    return out
+
+
+def dsp_cps_search_biased(lat: SimpleNamespace, prev_token: torch.Tensor, table: torch.Tensor, *, W: int,
+                          lam: float, ver_score: Optional[torch.Tensor], mu: float, eos_id: int = -1,
+                          proxy_kind: int = 0, table_log2: int = 0, hash_seed: int = 0, V: int = 1,
+                          out: Optional[SimpleNamespace] = None, row_status: Optional[torch.Tensor] = None,
+                          beams: bool = True, stream=None) -> SimpleNamespace:
+    B, L, KC = lat.cand_id.shape
+    if ver_score is not None and (ver_score.dtype != torch.float32 or tuple(ver_score.shape) != (B, L, KC)
+                                  or not ver_score.is_contiguous()):
+        raise ValueError("ver_score must be a contiguous float32 [B, L, KC] tensor")
+    if out is None:
+        out = cps_outputs(B, L, W, lat.cand_id.device, beams)
+    _check("dsp_cps_search_biased", lib().dsp_cps_search_biased(
+        _ptr(lat.cand_id), _ptr(lat.cand_logit), _ptr(lat.lse64), _ptr(lat.cand_count), B, L, KC,
+        _ptr(prev_token), proxy_kind, _ptr(table), table_log2, C.c_uint32(hash_seed & 0xFFFFFFFF), V,
+        W, C.c_float(lam), eos_id, _ptr(ver_score), C.c_float(mu), _ptr(out.path), _ptr(out.path_slot),
+        _ptr(out.path_len), _ptr(out.path_score), _ptr(out.beam_ids), _ptr(out.beam_score),
+        _ptr(out.beam_cum), _ptr(row_status), _stream(stream)))
     return out
 
 

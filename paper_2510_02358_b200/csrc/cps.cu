@@ -2,6 +2,7 @@
 //
 // One CTA per batch row walks the lattice left to right.  The step score of a candidate,
 //   step = fl( fl(lambda * (x - x_top1)) + fl((1 - lambda) * l^ng(prev, cur)) ),
+// (with a verifier-side score per candidate slot, dsp_cps_search_biased: fl(step + fl(mu * l^ver)))
 // depends on the previous position's candidate slot and on its own slot but not on the beam, so
 // for a window of depths all (depth, previous slot, slot) steps are gathered and computed in
 // parallel before the depths of the window are walked; the sequential part of a depth is then
@@ -36,6 +37,8 @@ struct CpsArgs {
     int W;
     float lambda;
     int eos_id;
+    const float *ver_score;      // [B,L,KC] or null: the verifier-side term of the step score
+    float mu;
     int32_t *path, *path_slot, *path_len;
     float *path_score;
     int32_t *beam_ids;
@@ -175,7 +178,7 @@ __global__ void __launch_bounds__(kThreads) cps_kernel(const CpsArgs a) {
         if constexpr (!TRI) {
             const int total = nd * KK;
             for (int x0 = tid; x0 < total; x0 += kThreads * kGatherBatch) {
-                float ng[kGatherBatch];
+                float ng[kGatherBatch], vs[kGatherBatch];
                 int at[kGatherBatch];                           // d * KC + k of a live entry, else -1
 #pragma unroll
                 for (int u = 0; u < kGatherBatch; ++u) {        // no branches: the gathers of a batch overlap
@@ -188,13 +191,16 @@ __global__ void __launch_bounds__(kThreads) cps_kernel(const CpsArgs a) {
                         ng[u] = __ldg(&a.table[(row0 + i0) * KK + (ok ? x : 0)]);
                     else
                         ng[u] = proxy_score(a, ok ? cid[d * KC + p] : 0, ok ? cid[(d + 1) * KC + k] : 0);
+                    vs[u] = a.ver_score ? __ldg(&a.ver_score[(row0 + i0) * KC + (ok ? d * KC + k : 0)]) : 0.f;
                 }
 #pragma unroll
                 for (int u = 0; u < kGatherBatch; ++u) {
                     if (at[u] >= 0) {
                         const int d = div_by(at[u], mKC);
                         const float g = __fsub_rn(clg[at[u]], clg[d * KC]);
-                        step[x0 + u * kThreads] = __fadd_rn(__fmul_rn(lam, g), __fmul_rn(oml, ng[u]));
+                        float st = __fadd_rn(__fmul_rn(lam, g), __fmul_rn(oml, ng[u]));
+                        if (a.ver_score) st = __fadd_rn(st, __fmul_rn(a.mu, vs[u]));
+                        step[x0 + u * kThreads] = st;
                     }
                 }
             }
@@ -244,7 +250,9 @@ __global__ void __launch_bounds__(kThreads) cps_kernel(const CpsArgs a) {
                     const int w = (int)(((unsigned)e * inv) >> 16), k = e - w * cnt;
                     const float ng = trigram_score(a, btok2[cur][w], btok[cur][w], cid[(d + 1) * KC + k]);
                     const float g = __fsub_rn(clg[d * KC + k], clg[d * KC]);       // the drafter's part: x - x_top1
-                    const float cum = __fadd_rn(bcum[cur][w], __fadd_rn(__fmul_rn(lam, g), __fmul_rn(oml, ng)));
+                    float st = __fadd_rn(__fmul_rn(lam, g), __fmul_rn(oml, ng));
+                    if (a.ver_score) st = __fadd_rn(st, __fmul_rn(a.mu, __ldg(&a.ver_score[(row0 + i) * KC + k])));
+                    const float cum = __fadd_rn(bcum[cur][w], st);
                     const uint32_t ob = ord_bits(cum);
                     atomicMax(&tbest[cur][w], ob);
                     tkeys[e] = ((unsigned long long)ob << 32) | ((unsigned long long)(255 - trank[d * KC + k]) << 24) |
@@ -332,6 +340,7 @@ __global__ void __launch_bounds__(kThreads) cps_kernel(const CpsArgs a) {
 
     // ---- outputs ----
     // common term of Eq. 8 dropped from the ranking: lambda * sum_i (lse_i - x_top1,i), in double
+    // (the verifier-side term, where given, is part of the ranking quantity already)
     __shared__ double s_off[kWarps];
     double off = 0.0;
     for (int i = tid; i < m; i += kThreads) off += a.lse64[row0 + i] - (double)a.cand_logit[(row0 + i) * KC];
@@ -393,6 +402,7 @@ int32_t dsp::cps_search_impl(const int32_t *cand_id, const float *cand_logit,
                                   int32_t proxy_kind, const float *proxy_table, int32_t table_log2,
                                   uint32_t hash_seed, int32_t V,
                                   int32_t W, float lambda, int32_t eos_id,
+                                  const float *ver_score, float mu,
                                   int32_t *path, int32_t *path_slot, int32_t *path_len,
                                   float *path_score,
                                   int32_t *beam_ids, float *beam_score, float *beam_cum,
@@ -402,6 +412,7 @@ int32_t dsp::cps_search_impl(const int32_t *cand_id, const float *cand_logit,
     if (proxy_kind < 0 || proxy_kind > 3) return DSP_ERR_UNSUPPORTED;
     if ((proxy_kind == 0 || proxy_kind == 3) && (table_log2 < 1 || table_log2 > 31)) return DSP_ERR_INVALID_ARG;
     if (!(lambda >= 0.f && lambda <= 1.f)) return DSP_ERR_INVALID_ARG;
+    if (ver_score && !(fabsf(mu) <= 3.0e38f)) return DSP_ERR_INVALID_ARG;      // NaN or infinite weight
     if (B == 0) return DSP_OK;
     if (!cand_id || !cand_logit || !lse64 || !cand_count || !prev_token || !proxy_table || !path ||
         !path_slot || !path_len || !path_score)
@@ -413,6 +424,7 @@ int32_t dsp::cps_search_impl(const int32_t *cand_id, const float *cand_logit,
     a.prev_token = prev_token;
     a.proxy_kind = proxy_kind; a.table = proxy_table; a.table_log2 = table_log2;
     a.hash_seed = hash_seed; a.V = V; a.W = W; a.lambda = lambda; a.eos_id = eos_id;
+    a.ver_score = ver_score; a.mu = mu;
     a.path = path; a.path_slot = path_slot; a.path_len = path_len; a.path_score = path_score;
     a.beam_ids = beam_ids; a.beam_score = beam_score; a.beam_cum = beam_cum;
     a.row_status = row_status;
@@ -452,6 +464,25 @@ extern "C" int32_t dsp_cps_search(const int32_t *cand_id, const float *cand_logi
                                   int32_t *beam_ids, float *beam_score, float *beam_cum,
                                   uint32_t *row_status, dsp_stream_t stream) {
     return cps_search_impl(cand_id, cand_logit, lse64, cand_count, B, L, KC, prev_token, proxy_kind, proxy_table,
-                           table_log2, hash_seed, V, W, lambda, eos_id, path, path_slot, path_len, path_score,
-                           beam_ids, beam_score, beam_cum, row_status, reinterpret_cast<cudaStream_t>(stream));
+                           table_log2, hash_seed, V, W, lambda, eos_id, nullptr, 0.f, path, path_slot, path_len,
+                           path_score, beam_ids, beam_score, beam_cum, row_status,
+                           reinterpret_cast<cudaStream_t>(stream));
+}
+
+extern "C" int32_t dsp_cps_search_biased(const int32_t *cand_id, const float *cand_logit,
+                                         const double *lse64, const int32_t *cand_count,
+                                         int32_t B, int32_t L, int32_t KC,
+                                         const int32_t *prev_token,
+                                         int32_t proxy_kind, const float *proxy_table, int32_t table_log2,
+                                         uint32_t hash_seed, int32_t V,
+                                         int32_t W, float lambda, int32_t eos_id,
+                                         const float *ver_score, float mu,
+                                         int32_t *path, int32_t *path_slot, int32_t *path_len,
+                                         float *path_score,
+                                         int32_t *beam_ids, float *beam_score, float *beam_cum,
+                                         uint32_t *row_status, dsp_stream_t stream) {
+    return cps_search_impl(cand_id, cand_logit, lse64, cand_count, B, L, KC, prev_token, proxy_kind, proxy_table,
+                           table_log2, hash_seed, V, W, lambda, eos_id, ver_score, mu, path, path_slot, path_len,
+                           path_score, beam_ids, beam_score, beam_cum, row_status,
+                           reinterpret_cast<cudaStream_t>(stream));
 }

@@ -31,7 +31,8 @@ int32_t lattice_build_impl(const void *draft_logits, int32_t dtype, int32_t B, i
 int32_t cps_search_impl(const int32_t *cand_id, const float *cand_logit, const double *lse64,
                         const int32_t *cand_count, int32_t B, int32_t L, int32_t KC, const int32_t *prev_token,
                         int32_t proxy_kind, const float *proxy_table, int32_t table_log2, uint32_t hash_seed,
-                        int32_t V, int32_t W, float lambda, int32_t eos_id, int32_t *path, int32_t *path_slot,
+                        int32_t V, int32_t W, float lambda, int32_t eos_id, const float *ver_score, float mu,
+                        int32_t *path, int32_t *path_slot,
                         int32_t *path_len, float *path_score, int32_t *beam_ids, float *beam_score,
                         float *beam_cum, uint32_t *row_status, cudaStream_t stream);
 

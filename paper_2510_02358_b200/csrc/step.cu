@@ -85,8 +85,8 @@ extern "C" int32_t dsp_draft_verify_step(
     };
     auto search = [&](cudaStream_t s) {
         return cps_search_impl(cand_id, cand_logit, lse64, cand_count, B, L, KC, prev_token, proxy_kind,
-                               proxy_table, table_log2, hash_seed, V, W, lambda, eos_id, path, path_slot, path_len,
-                               path_score, beam_ids, beam_score, beam_cum, row_status, s);
+                               proxy_table, table_log2, hash_seed, V, W, lambda, eos_id, nullptr, 0.f, path, path_slot,
+                               path_len, path_score, beam_ids, beam_score, beam_cum, row_status, s);
     };
     int32_t rc2 = DSP_OK;
     // The two sides start together: the second stream takes up where the caller's stream stands.

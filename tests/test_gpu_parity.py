@@ -349,6 +349,57 @@ def test_path_search_on_hand_made_lattices(B, L, K, W, eos, lam, flat, case, kin
         assert o.path_len[1] == 1 and o.path_len[2] == L and (o.row_status[1:3] & oracle.EOS_STOPPED).all()
 
 
+@pytest.mark.parametrize("kind", [0, 2, 3])
+@pytest.mark.parametrize("B,L,K,W,eos,lam,mu", [
+    (3, 128, 32, 32, True, 0.5, 0.75),      # largest K and W, several windows
+    (5, 33, 5, 7, False, 0.3, -1.25),       # odd sizes, a negative weight
+    (4, 24, 8, 8, True, 0.5, 0.0),          # weight 0 with a tensor given
+])
+def test_path_search_with_a_verifier_side_term(B, L, K, W, eos, lam, mu, kind):
+    V = 5000
+    KC = K + (1 if eos else 0)
+    eos_id = 17 if eos else -1
+    lat = _hand_lattice(B, L, KC, V, seed=L * 11 + K)
+    g = torch.Generator().manual_seed(123)
+    tshape = (B, L, KC, KC) if kind == 2 else (1 << 12,)
+    table = torch.round(torch.randn(tshape, generator=g) * 8) / 8 - 3.0
+    ver = torch.round(torch.randn((B, L, KC), generator=g) * 8) / 8 - 2.0     # eighths: many equal sums
+    prev = torch.randint(0, V, (B, 2) if kind == 3 else (B,), generator=g).int()
+    kw = dict(W=W, lam=lam, eos_id=eos_id, table_log2=12, hash_seed=5, V=V, proxy_kind=kind)
+    o = oracle.cps_search(lat.cand_id, lat.cand_logit, lat.lse64, lat.cand_count, prev, table, ver_score=ver, mu=mu, **kw)
+    plain = oracle.cps_search(lat.cand_id, lat.cand_logit, lat.lse64, lat.cand_count, prev, table, **kw)
+    if mu != 0.0:
+        assert not torch.equal(o.path, plain.path)         # the case does exercise the term
+    dlat = SimpleNamespace(**{k: v.to(DEV) for k, v in vars(lat).items()})
+    status = torch.zeros(B, dtype=torch.int32, device=DEV)
+    c = dsp.dsp_cps_search_biased(dlat, prev.to(DEV), table.to(DEV), ver_score=ver.to(DEV), mu=mu,
+                                  row_status=status, **kw)
+    torch.cuda.synchronize()
+    for name in ("path", "path_slot", "path_len", "beam_ids", "beam_cum"):
+        assert torch.equal(getattr(c, name).cpu(), getattr(o, name)), f"{name} differs"
+    assert torch.allclose(c.beam_score.cpu(), o.beam_score, atol=1e-3, rtol=1e-5, equal_nan=True)
+    assert torch.allclose(c.path_score.cpu(), o.path_score, atol=1e-3, rtol=1e-5)
+    assert torch.equal((status.cpu() & dsp.ROW_EOS_STOPPED) != 0, (o.row_status & oracle.EOS_STOPPED) != 0)
+    # no tensor: the plain search bit for bit, whatever the weight
+    n = dsp.dsp_cps_search_biased(dlat, prev.to(DEV), table.to(DEV), ver_score=None, mu=3.0, **kw)
+    q = dsp.dsp_cps_search(dlat, prev.to(DEV), table.to(DEV), **kw)
+    torch.cuda.synchronize()
+    for name in ("path", "path_slot", "path_len", "path_score", "beam_ids", "beam_cum", "beam_score"):
+        assert torch.equal(getattr(n, name), getattr(q, name)), f"no tensor: {name} differs"
+    assert torch.equal(q.path.cpu(), plain.path)
+
+
+def test_verifier_side_term_rejects_a_non_finite_weight():
+    lat = _hand_lattice(1, 4, 3, 100, seed=1)
+    dlat = SimpleNamespace(**{k: v.to(DEV) for k, v in vars(lat).items()})
+    prev = torch.zeros(1, dtype=torch.int32, device=DEV)
+    table = torch.zeros(1 << 4, device=DEV)
+    ver = torch.zeros((1, 4, 3), device=DEV)
+    for bad in (float("nan"), float("inf")):
+        with pytest.raises(dsp.DspError):
+            dsp.dsp_cps_search_biased(dlat, prev, table, ver_score=ver, mu=bad, W=2, lam=0.5, table_log2=4, V=100)
+
+
 # ---- the step recorded as a CUDA graph ----
 def _same_outputs(a, b, w=None):
     for s in ("lat", "cps", "ver"):
