@@ -311,6 +311,10 @@ def _hand_lattice(B, L, KC, V, seed, *, flat=False, counts=None):
     (6, 32, 16, 16, True, 0.5, False, "eos"),      # the best beam meets EOS and stops
     (5, 33, 5, 7, False, 0.3, False, "odd"),       # W > K, odd sizes
     (2, 1024, 3, 32, True, 0.5, False, "long"),    # the longest draft the library takes
+    (4, 40, 8, 8, True, 0.0, True, "flat"),        # small beams (one warp walks the depths): all ties,
+    (6, 32, 8, 8, True, 0.5, False, "eos"),        # the early stop,
+    (2, 1024, 2, 8, True, 0.5, False, "long"),     # several windows
+    (3, 20, 1, 1, False, 0.5, False, "odd"),       # and a single candidate and beam
 ])
 def test_path_search_on_hand_made_lattices(B, L, K, W, eos, lam, flat, case, kind):
     V = 5000
