@@ -22,7 +22,8 @@ struct SampleJob {
     int trow;        // target row index b*Lt + i, or -1: no job
     int drow;        // draft row index b*L + i, or -1: draw from p itself (bonus token)
     float u;
-    int fallback;    // target argmax of that row (used when the residual mass is 0)
+    int fallback;    // target argmax of that row (used when the residual mass is 0); jobs of the
+                     // acceptance scan leave it unset: their kernel reads the row's argmax itself
 };
 
 struct VerifyArgs {
@@ -83,8 +84,15 @@ template <typename DT>
 __device__ SampleJob accept_row(const VerifyArgs &a, int b, bool write) {
     const int lane = threadIdx.x & 31;
     const int L = a.L, Lt = a.Lt;
-    const int m = max(0, min(__ldcg(&a.path_len[b]), L));
+    const int m_raw = __ldcg(&a.path_len[b]);
     const bool stoch = !a.all_greedy && a.mode[b] != 0;
+    // the first 32 positions' path entries are fetched beside the path length, not after it
+    int y_first = -1, slot_first = 0;
+    if (lane < L) {
+        y_first = __ldcg(&a.path[(long long)b * L + lane]);
+        if (stoch) slot_first = __ldcg(&a.path_slot[(long long)b * L + lane]);
+    }
+    const int m = max(0, min(m_raw, L));
     int acc = m;
     bool eos_seen_before_acc = false;
     for (int i0 = 0; i0 < L; i0 += 32) {
@@ -92,11 +100,11 @@ __device__ SampleJob accept_row(const VerifyArgs &a, int b, bool write) {
         bool rej = false;
         float rt_out = -1.f;
         if (i < m) {
-            const int y = __ldcg(&a.path[(long long)b * L + i]);
+            const int y = i0 == 0 ? y_first : __ldcg(&a.path[(long long)b * L + i]);
             if (!stoch) {
                 rej = y != __ldcg(&a.argmax[(long long)b * Lt + i]);
             } else {
-                const int slot = __ldcg(&a.path_slot[(long long)b * L + i]);
+                const int slot = i0 == 0 ? slot_first : __ldcg(&a.path_slot[(long long)b * L + i]);
                 const double xt = a.xt_probe ? (double)__ldcg(&a.xt_probe[(long long)b * Lt + i])
                                              : (double)Elem<DT>::load1(trow_ptr<DT>(a, (long long)b * Lt + i) + y);
                 const double xd = (double)__ldcg(&a.cand_logit[((long long)b * L + i) * a.KC + slot]);
@@ -126,14 +134,12 @@ __device__ SampleJob accept_row(const VerifyArgs &a, int b, bool write) {
         int nt = -1;
         const int at = acc < m ? acc : m;              // row the next token comes from
         if (acc < m || m < Lt) {
-            const int am = __ldcg(&a.argmax[(long long)b * Lt + at]);
             if (!stoch) {
-                nt = am;
-            } else {
+                nt = __ldcg(&a.argmax[(long long)b * Lt + at]);
+            } else {                                   // the fallback (the row's argmax) is read where it is needed
                 job.trow = b * Lt + at;
                 job.drow = acc < m ? b * L + at : -1;
                 job.u = a.u[(long long)b * (L + 1) + L];
-                job.fallback = am;
             }
         } else {
             status |= DSP_ROW_NO_BONUS_ROW;
@@ -328,15 +334,12 @@ __global__ void __launch_bounds__(kThreads, 4) residual_kernel(const VerifyArgs 
     const DT *tp = trow_ptr<DT>(a, job.trow);
     const DT *dp = has_q ? drow_ptr<DT>(a, job.drow) : tp;
     const bool aligned = ((reinterpret_cast<uintptr_t>(tp) | reinterpret_cast<uintptr_t>(dp)) & 15) == 0;
-    const RowProb pt = row_prob(a.tlse64[job.trow]);
-    const RowProb pd = has_q ? row_prob(a.draft_lse64[job.drow]) : pt;
     double *sums = a.chunk_sums + (long long)b * a.nchunks;
     const int V = a.V;
-
     const int c0 = rs * a.chunks_per_slice, c1 = min(a.nchunks, c0 + a.chunks_per_slice);
     constexpr int kChunkBatch = 4;              // chunks whose loads a warp has in flight together
-    for (int ch0 = c0 + warp; ch0 < c1; ch0 += kWarps * kChunkBatch) {
-        uint4 vt[kChunkBatch], vd[kChunkBatch];
+    uint4 vt[kChunkBatch], vd[kChunkBatch];
+    auto load_batch = [&](int ch0) {
 #pragma unroll
         for (int u = 0; u < kChunkBatch; ++u) {
             const int ch = ch0 + u * kWarps;
@@ -346,6 +349,15 @@ __global__ void __launch_bounds__(kThreads, 4) residual_kernel(const VerifyArgs 
                 vd[u] = has_q ? load_vec<DT>(dp, e0, V, aligned) : vt[u];
             }
         }
+    };
+    load_batch(c0 + warp);                      // in flight while the rows' constants are fetched and formed
+    const double tl = __ldcg(&a.tlse64[job.trow]);
+    const double dl = has_q ? __ldcg(&a.draft_lse64[job.drow]) : 0.0;
+    const RowProb pt = row_prob(tl);
+    const RowProb pd = has_q ? row_prob(dl) : pt;
+
+    for (int ch0 = c0 + warp; ch0 < c1; ch0 += kWarps * kChunkBatch) {
+        if (ch0 != c0 + warp) load_batch(ch0);
 #pragma unroll
         for (int u = 0; u < kChunkBatch; ++u) {
             const int ch = ch0 + u * kWarps;
@@ -369,8 +381,14 @@ __global__ void __launch_bounds__(kThreads, 4) residual_kernel(const VerifyArgs 
     // ---- last CTA of this job: invert the CDF ----
     const int per = (a.nchunks + kThreads - 1) / kThreads;     // consecutive chunks per thread
     const int k0 = min(a.nchunks, tid * per), k1 = min(a.nchunks, k0 + per);
+    constexpr int kKept = 4;                    // chunk sums a thread keeps in registers for its second look
+    double kept[kKept];
+#pragma unroll
+    for (int j = 0; j < kKept; ++j) kept[j] = k0 + j < k1 ? __ldcg(&sums[k0 + j]) : 0.0;
     double mine = 0.0;
-    for (int k = k0; k < k1; ++k) mine += __ldcg(&sums[k]);
+#pragma unroll
+    for (int j = 0; j < kKept; ++j) mine += kept[j];            // k0 + j >= k1: + 0.0, which changes nothing
+    for (int k = k0 + kKept; k < k1; ++k) mine += __ldcg(&sums[k]);
     if (tid == 0) s_found = 0x7FFFFFFF;
     // exclusive prefix of the 256 thread sums, in a fixed order: inside each warp, then over the warps
     double tincl = mine;
@@ -390,23 +408,43 @@ __global__ void __launch_bounds__(kThreads, 4) residual_kernel(const VerifyArgs 
     const double R = s_total;
     if (!(R > 0.0)) {
         if (tid == 0) {
-            a.next_token[b] = job.fallback;
+            a.next_token[b] = ACCEPT ? __ldcg(&a.argmax[job.trow]) : job.fallback;
             atomicOr(&a.row_status[b], DSP_ROW_ZERO_RESIDUAL);
         }
         return;
     }
     const double thr = (double)job.u * R;
     {
+        // The first chunk at which the running sum reaches the threshold; the thread that finds it
+        // leaves the sum of everything before that chunk in its slot of s_scan.
         double run = s_scan[tid];
-        for (int k = k0; k < k1; ++k) {
+        bool found = false;
+#pragma unroll
+        for (int j = 0; j < kKept; ++j) {
+            if (!found && k0 + j < k1) {
+                const double cs = kept[j];
+                if (cs > 0.0 && run + cs >= thr) {
+                    atomicMin(&s_found, k0 + j);
+                    s_scan[tid] = run;
+                    found = true;
+                }
+                run += cs;
+            }
+        }
+        for (int k = k0 + kKept; k < k1 && !found; ++k) {
             const double cs = __ldcg(&sums[k]);
+            if (cs > 0.0 && run + cs >= thr) {
+                atomicMin(&s_found, k);
+                s_scan[tid] = run;
+                found = true;
+            }
             run += cs;
-            if (cs > 0.0 && run >= thr) { atomicMin(&s_found, k); break; }
         }
     }
     __syncthreads();
     int ch = s_found;
-    if (ch == 0x7FFFFFFF) {                     // rounding at the very top: last chunk with mass
+    const bool at_top = ch == 0x7FFFFFFF;
+    if (at_top) {                               // rounding at the very top: last chunk with mass
         if (tid == 0) {
             int last = -1;
             for (int k = a.nchunks - 1; k >= 0; --k)
@@ -417,21 +455,22 @@ __global__ void __launch_bounds__(kThreads, 4) residual_kernel(const VerifyArgs 
         ch = s_found;
     }
     if (warp != 0) return;
-    // prefix of everything before chunk ch, in the same association as above
+    // prefix of everything before chunk ch: as its finder left it, else added up the same way
     double before = 0.0;
     {
         const int owner = min(kThreads - 1, ch / per);
         before = s_scan[owner];
-        for (int k = owner * per; k < ch; ++k) before += __ldcg(&sums[k]);
+        if (at_top)
+            for (int k = owner * per; k < ch; ++k) before += __ldcg(&sums[k]);
     }
     const int e0 = ch * CE + lane * N;
-    const uint4 vt = load_vec<DT>(tp, e0, V, aligned);
-    const uint4 vd = has_q ? load_vec<DT>(dp, e0, V, aligned) : vt;
+    const uint4 ct = load_vec<DT>(tp, e0, V, aligned);
+    const uint4 cd = has_q ? load_vec<DT>(dp, e0, V, aligned) : ct;
     float r[N];
     float s = 0.f;
 #pragma unroll
     for (int e = 0; e < N; ++e) {
-        r[e] = residual(Elem<DT>::get(vt, e), Elem<DT>::get(vd, e), pt, pd, has_q);
+        r[e] = residual(Elem<DT>::get(ct, e), Elem<DT>::get(cd, e), pt, pd, has_q);
         s = __fadd_rn(s, r[e]);
     }
     // exclusive prefix over lanes (double)
@@ -457,7 +496,8 @@ __global__ void __launch_bounds__(kThreads, 4) residual_kernel(const VerifyArgs 
         tok = __shfl_sync(0xFFFFFFFFu, hit, __ffs(bal) - 1);
     } else {
         const unsigned bl = __ballot_sync(0xFFFFFFFFu, lastpos >= 0);
-        tok = bl ? __shfl_sync(0xFFFFFFFFu, lastpos, 31 - __clz(bl)) : job.fallback;
+        tok = bl ? __shfl_sync(0xFFFFFFFFu, lastpos, 31 - __clz(bl))
+                 : (ACCEPT ? __ldcg(&a.argmax[job.trow]) : job.fallback);
     }
     if (lane == 0) a.next_token[b] = tok;
 }
