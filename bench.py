@@ -293,16 +293,19 @@ def time_proxies(w, st, sets, device, reps=50):
     g = torch.Generator(device=device).manual_seed(3)
     tensor = -6.0 * torch.rand((w.B, w.L, KC, KC), generator=g, device=device)
     prev2 = torch.stack([inp["prev_token"], inp["prev_token"]], dim=1).contiguous()
-    cases = {"hashed_bigram": (0, inp["table"], inp["prev_token"]), "tensor": (2, tensor, inp["prev_token"]),
-             "hashed_trigram": (3, inp["table"], prev2)}
+    ver = -4.0 * torch.rand((w.B, w.L, KC), generator=g, device=device)     # a verifier-side score per candidate slot
+    cases = {"hashed_bigram": (0, inp["table"], inp["prev_token"], None), "tensor": (2, tensor, inp["prev_token"], None),
+             "hashed_trigram": (3, inp["table"], prev2, None),
+             "hashed_bigram_with_verifier_term": (0, inp["table"], inp["prev_token"], ver)}
     out = {}
-    for name, (kind, table, prev) in cases.items():
+    for name, (kind, table, prev, vs) in cases.items():
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         for r in range(reps + 3):
             if r == 3:
                 e0.record()
-            dsp.dsp_cps_search(st.lat, prev, table, W=w.W, lam=w.lam, eos_id=w.eos_id, proxy_kind=kind,
-                               table_log2=inp["table_log2"], hash_seed=inp["hash_seed"], V=w.V, out=st.cps)
+            dsp.dsp_cps_search_biased(st.lat, prev, table, W=w.W, lam=w.lam, ver_score=vs, mu=0.5, eos_id=w.eos_id,
+                                      proxy_kind=kind, table_log2=inp["table_log2"], hash_seed=inp["hash_seed"], V=w.V,
+                                      out=st.cps)
         e1.record()
         torch.cuda.synchronize()
         out[name] = e0.elapsed_time(e1) / reps
