@@ -65,7 +65,8 @@ extern "C" int32_t dsp_step_graph_create(
         return cuda_fail(e);
     }
     cudaGraphExec_t exec = nullptr;
-    e = cudaGraphInstantiate(&exec, graph, 0);
+    // the kernels recorded from the step's second stream keep that stream's priority in the replay
+    e = cudaGraphInstantiateWithFlags(&exec, graph, cudaGraphInstantiateFlagUseNodePriority);
     if (e != cudaSuccess) {
         cudaGraphDestroy(graph);
         return cuda_fail(e);
