@@ -565,7 +565,7 @@ int32_t dsp::cps_search_impl(const int32_t *cand_id, const float *cand_logit,
                               : epl == 3 ? cps_kernel<false, 3>
                                          : cps_kernel<false, 0>;
     DSP_CUDA_TRY(launch_dependent(kernel, (unsigned)B, kThreads, dyn, stream, a,
-                                  short_kernel_follows_early(stream, (long long)B * L)));
+                                  true));
     return DSP_OK;
 }
 

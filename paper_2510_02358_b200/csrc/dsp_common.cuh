@@ -68,22 +68,8 @@ inline cudaError_t launch_dependent(void (*kernel)(Arg), unsigned grid, unsigned
     return cudaLaunchKernelEx(&cfg, kernel, a);
 }
 
-// Where the early placement pays (measured on a B200).  Between the short kernels of a call it
-// saves 1 to 2 us per launch.  In a captured graph the programmatic edges pay only on large
-// problems (small ones replay 2 us slower with them).
-constexpr long long kDependentGraphRows = 1024;           // fewest logits rows for programmatic edges in a graph
-inline bool stream_is_capturing(cudaStream_t st) {
-    cudaStreamCaptureStatus cs = cudaStreamCaptureStatusNone;
-    if (cudaStreamIsCapturing(st, &cs) != cudaSuccess) {
-        (void)cudaGetLastError();
-        return true;                                       // unknown: take the ordinary launch
-    }
-    return cs != cudaStreamCaptureStatusNone;
-}
-// A short kernel behind another short kernel, in a call over `nrows` rows of logits.
-inline bool short_kernel_follows_early(cudaStream_t st, long long nrows) {
-    return nrows >= kDependentGraphRows || !stream_is_capturing(st);
-}
+// The early placement saves 1 to 2 us per launch between the short kernels of a call, in a stream
+// and in a captured graph alike.
 
 // ---- order-preserving 64-bit keys: larger key = better under (logit desc, id asc) ----
 __device__ __forceinline__ uint32_t ord_bits(float x) {

@@ -240,7 +240,7 @@ static int32_t launch_lattice(LatticeArgs &a, void *workspace, size_t workspace_
         if (pe.start) DSP_CUDA_TRY(cudaEventRecord(pe.start, st));
         // the streaming kernel may start beside the preparation: it waits for it after its rows are streamed
         DSP_CUDA_TRY(launch_dependent(lattice_scan_kernel<DT>, (unsigned)nblocks, kThreads, (size_t)a.nstages * kTileBytes, st, a,
-                                      !pe.start && short_kernel_follows_early(st, nrows)));
+                                      !pe.start));
         if (pe.stop) DSP_CUDA_TRY(cudaEventRecord(pe.stop, st));
     } else {
         lattice_kernel<DT><<<(unsigned)nblocks, kThreads, 0, st>>>(a);

@@ -220,7 +220,7 @@ static int32_t launch_shard(ShardArgs &a, void *workspace, size_t workspace_byte
         DSP_CUDA_TRY(allow_ring_smem(shard_scan_kernel<DT>, smem_done));
         a.nstages = ring_stages(nblocks);
         DSP_CUDA_TRY(launch_dependent(shard_scan_kernel<DT>, (unsigned)nblocks, kThreads, (size_t)a.nstages * kTileBytes, st, a,
-                                      short_kernel_follows_early(st, nrows)));
+                                      true));
     } else {
         shard_rows_kernel<DT><<<(unsigned)((nrows + kWarps - 1) / kWarps), kThreads, 0, st>>>(a);
     }

@@ -208,7 +208,7 @@ static int32_t launch_unmask(UnmaskArgs &a, void *workspace, size_t workspace_by
         DSP_CUDA_TRY(allow_ring_smem(unmask_scan_kernel<DT>, smem_done));
         a.nstages = ring_stages(nblocks);
         DSP_CUDA_TRY(launch_dependent(unmask_scan_kernel<DT>, (unsigned)nblocks, kThreads, (size_t)a.nstages * kTileBytes, st, a,
-                                      short_kernel_follows_early(st, nrows)));
+                                      true));
     } else {
         unmask_rows_kernel<DT><<<(unsigned)((nrows + kWarps - 1) / kWarps), kThreads, 0, st>>>(a);
     }

@@ -584,7 +584,7 @@ static int32_t launch_verify(VerifyArgs &a, void *workspace, size_t workspace_by
         if (pe.start) DSP_CUDA_TRY(cudaEventRecord(pe.start, st));
         // the streaming kernel may start beside the preparation: it waits for it after its rows are streamed
         DSP_CUDA_TRY(launch_dependent(target_scan_kernel<DT>, (unsigned)nblocks, kThreads, (size_t)a.nstages * kTileBytes, st, a,
-                                      !pe.start && short_kernel_follows_early(st, nrows)));
+                                      !pe.start));
         if (pe.stop) DSP_CUDA_TRY(cudaEventRecord(pe.stop, st));
     } else {
         target_kernel<DT><<<(unsigned)nblocks, kThreads, 0, st>>>(a);
@@ -592,7 +592,7 @@ static int32_t launch_verify(VerifyArgs &a, void *workspace, size_t workspace_by
     DSP_CUDA_TRY(cudaGetLastError());
     }
     if (phases & kVerifyDecide) {
-        const bool early = short_kernel_follows_early(st, nrows);
+        const bool early = true;
         if (a.all_greedy)
             DSP_CUDA_TRY(launch_dependent(accept_kernel<DT>, (unsigned)((a.B + kWarps - 1) / kWarps), kThreads, 0, st, a, early));
         else           // the acceptance scan runs inside the residual kernel
