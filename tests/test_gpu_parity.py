@@ -3,6 +3,7 @@ import math
 from types import SimpleNamespace
 
 import pytest
+import numpy as np
 import torch
 
 import oracle
@@ -402,6 +403,46 @@ def test_verifier_side_term_rejects_a_non_finite_weight():
     for bad in (float("nan"), float("inf")):
         with pytest.raises(dsp.DspError):
             dsp.dsp_cps_search_biased(dlat, prev, table, ver_score=ver, mu=bad, W=2, lam=0.5, table_log2=4, V=100)
+
+
+@pytest.mark.parametrize("seed", range(8))
+def test_path_search_on_random_shapes(seed):
+    """Seeded random shapes across both forms of the walk (one warp for small beams, the whole CTA for
+    large ones), with quantised scores (ties), ragged counts, EOS among the candidates and all proxies."""
+    rng = np.random.default_rng(1000 + seed)
+    for case in range(6):
+        B = int(rng.integers(1, 5))
+        L = int(rng.integers(1, 70))
+        K = int(rng.choice([1, 2, 3, 5, 8, 11, 16, 32]))
+        W = int(rng.choice([1, 2, 3, 4, 8, 12, 16, 32]))
+        eos = bool(rng.integers(0, 2))
+        kind = int(rng.choice([0, 1, 2, 3]))
+        lam = float(rng.choice([0.0, 0.25, 0.5, 1.0]))
+        V = 300 if kind == 1 else 5000
+        KC = K + (1 if eos else 0)
+        eos_id = 17 if eos else -1
+        lat = _hand_lattice(B, L, KC, V, seed=seed * 100 + case)
+        if eos and L > 2:                                  # EOS somewhere among the candidates of one row
+            lat.cand_id[0, int(rng.integers(0, L)), int(rng.integers(0, KC))] = eos_id
+        if case % 3 == 2 and L > 3:
+            lat.cand_count[B - 1, int(rng.integers(1, L))] = 0     # a hole ends that lattice
+        g = torch.Generator().manual_seed(seed * 7 + case)
+        tshape = {0: (1 << 10,), 1: (V, V), 2: (B, L, KC, KC), 3: (1 << 10,)}[kind]
+        table = torch.round(torch.randn(tshape, generator=g) * 4) / 4 - 3.0
+        prev = torch.randint(0, V, (B, 2) if kind == 3 else (B,), generator=g).int()
+        ver = torch.round(torch.randn((B, L, KC), generator=g) * 4) / 4 if case % 2 else None
+        kw = dict(W=W, lam=lam, eos_id=eos_id, table_log2=10, hash_seed=seed, V=V, proxy_kind=kind)
+        o = oracle.cps_search(lat.cand_id, lat.cand_logit, lat.lse64, lat.cand_count, prev, table, ver_score=ver, mu=0.75, **kw)
+        dlat = SimpleNamespace(**{k: v.to(DEV) for k, v in vars(lat).items()})
+        status = torch.zeros(B, dtype=torch.int32, device=DEV)
+        c = dsp.dsp_cps_search_biased(dlat, prev.to(DEV), table.to(DEV), ver_score=None if ver is None else ver.to(DEV),
+                                      mu=0.75, row_status=status, **kw)
+        torch.cuda.synchronize()
+        what = f"seed {seed} case {case}: B={B} L={L} K={K} W={W} eos={eos} kind={kind} lam={lam}"
+        for name in ("path", "path_slot", "path_len", "beam_ids", "beam_cum"):
+            assert torch.equal(getattr(c, name).cpu(), getattr(o, name)), f"{what}: {name} differs"
+        assert torch.allclose(c.beam_score.cpu(), o.beam_score, atol=1e-3, rtol=1e-5, equal_nan=True), what
+        assert torch.equal((status.cpu() & dsp.ROW_EOS_STOPPED) != 0, (o.row_status & oracle.EOS_STOPPED) != 0), what
 
 
 # ---- the step recorded as a CUDA graph ----
