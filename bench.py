@@ -453,6 +453,47 @@ def time_unmask(w, device, reps=40):
     return res
 
 
+def time_tree(w, device, reps=30):
+    """The beams of the path search verified as one token tree in a single target pass (dsp_beam_tree,
+    then dsp_verify_tree for the greedy rule or dsp_verify_tree_stochastic for the sampling rule) on a
+    batch of 8 rows of the headline workload's vocabulary: draft length 16, 8 candidates, 4 beams,
+    64 node slots per batch row.  The target rows are synthetic: the draft row of the node's depth plus noise."""
+    from paper_2510_02358_b200 import binding as dsp
+    tw = w.scaled(B=8, L=16, K=8, W=4, tau=0.0, name="tree_B8_L16_W4")
+    inp = wl.make_inputs(tw, step=11, device=device)
+    lat = dsp.dsp_lattice_build(inp["draft"], tw.K)
+    cps = dsp.dsp_cps_search(lat, inp["prev_token"], inp["table"], W=tw.W, lam=tw.lam, table_log2=inp["table_log2"],
+                             hash_seed=inp["hash_seed"], V=tw.V)
+    tree = dsp.dsp_beam_tree(cps)
+    N = tw.W * tw.L
+    g = torch.Generator(device=device).manual_seed(5)
+    depth = torch.cat([torch.zeros((tw.B, 1), dtype=torch.long, device=device),
+                       (tree.node_depth.long() + 1).clamp_(0, tw.L - 1)], dim=1)          # row 0: after the prefix
+    target = torch.empty((tw.B, 1 + N, tw.V), dtype=tw.dtype, device=device)
+    for b in range(tw.B):
+        target[b] = (inp["draft"][b, depth[b]].float() +
+                     0.5 * torch.randn((1 + N, tw.V), generator=g, device=device)).to(tw.dtype)
+    u = torch.rand((tw.B, N + 1), generator=g, device=device)
+    res = {"workload": tw.name, "node_slots": N, "nodes_mean": float(tree.n_nodes.float().mean().item()),
+           "target_bytes": target.numel() * target.element_size()}
+    calls = {"beam_tree": lambda: dsp.dsp_beam_tree(cps),
+             "verify_tree_greedy": lambda: dsp.dsp_verify_tree(target, tree, tw.L),
+             "verify_tree_stochastic": lambda: dsp.dsp_verify_tree_stochastic(target, inp["draft"], tree, u)}
+    for name, call in calls.items():
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        out = None
+        for r in range(reps + 3):
+            if r == 3:
+                e0.record()
+            out = call()
+        e1.record()
+        torch.cuda.synchronize()
+        res[name + "_ms"] = e0.elapsed_time(e1) / reps
+        if name != "beam_tree":
+            res[name + "_mean_accepted_len"] = float(out.accepted_len.float().mean().item())
+    return res
+
+
 def time_e2e(w, st, sets, device, steps):
     """Same step through the public calls with HOST buffers: pinned logits are copied to the
     device inside the timed region and the step's results are read back every step."""
@@ -802,6 +843,7 @@ def main():
         line["workloads"] = extras
         line["adl_closed_loop_c2"] = time_adl_loop(device)
         line["unmask_step"] = time_unmask(w, device)
+        line["tree_verification"] = time_tree(w, device)
         line["vocab_sharded_lattice"] = time_sharded(w, device)
     print(json.dumps(line))
     if dist is not None:

@@ -317,11 +317,12 @@ def verify_tree_stochastic(target: torch.Tensor, draft: torch.Tensor, tree: Simp
     u_np = _np(u, np.float32)
     assert u_np.shape == (B, N + 1)
     o = SimpleNamespace(accepted_len=np.empty((B,), np.int32), accepted_node=np.empty((B, L), np.int32),
-                        next_token=np.empty((B,), np.int32), row_status=np.zeros((B,), np.uint32))
+                        next_token=np.empty((B,), np.int32), row_status=np.zeros((B,), np.uint32),
+                        margin=np.empty((B,), np.float64))
     rc = lib().orc_verify_tree_stochastic(
         _logits_ptr(target), _logits_ptr(draft), _dtype_code(target), B, N, L, C.c_int64(V),
         _p(_np(tree.node_token, np.int32)), _p(_np(tree.node_parent, np.int32)), _p(_np(tree.n_nodes, np.int32)),
-        _p(u_np), _p(o.accepted_len), _p(o.accepted_node), _p(o.next_token), _p(o.row_status))
+        _p(u_np), _p(o.accepted_len), _p(o.accepted_node), _p(o.next_token), _p(o.row_status), _p(o.margin))
     if rc != 0:
         raise ValueError("orc_verify_tree_stochastic: bad arguments")
     return SimpleNamespace(**{k: torch.from_numpy(v) for k, v in vars(o).items()})

@@ -885,11 +885,17 @@ int orc_breadth_update(orc_breadth_state *st, const float *entropy, const int32_
  *   ORC_ZERO_RESIDUAL.
  * accepted_len = nodes walked, accepted_node[b,i] = the i-th of them (-1 beyond).
  * An existing target row or a used draft row with NaN / +inf or no finite logit flags the batch row.
+ *
+ * margin [B] (may be NULL; a diagnostic, no part of the rule): how far the batch row's closest
+ * decision was from going the other way: over the acceptance tests |u - f(x)/q(x)| relative to
+ * the larger of the two, and for the emitted token the distance of u * sum f from the two ends of
+ * that token's step of the cumulative sum, relative to sum f.  A comparison against arithmetic of
+ * lower precision can tell a rounding difference from a wrong result with it.
  */
 int orc_verify_tree_stochastic(const void *target, const void *draft, int dtype, int B, int N, int L, int64_t V,
                                const int32_t *node_token, const int32_t *node_parent, const int32_t *n_nodes,
                                const float *u, int32_t *accepted_len, int32_t *accepted_node,
-                               int32_t *next_token, uint32_t *row_status)
+                               int32_t *next_token, uint32_t *row_status, double *margin)
 {
     if (B < 0 || N < 1 || V < 1 || L < 1) return -1;
     const size_t es = dtype == 0 ? 4 : 2;
@@ -898,6 +904,7 @@ int orc_verify_tree_stochastic(const void *target, const void *draft, int dtype,
         const int32_t *tok = node_token + (int64_t)b * N, *par = node_parent + (int64_t)b * N;
         const int nn = n_nodes[b] < 0 ? 0 : (n_nodes[b] > N ? N : n_nodes[b]);
         uint32_t status = 0;
+        double closest = INFINITY;
         double *f = (double *)malloc(sizeof(double) * (size_t)V);
         double *q = (double *)malloc(sizeof(double) * (size_t)V);
         for (int i = 0; i < L; ++i) accepted_node[(int64_t)b * L + i] = -1;
@@ -926,8 +933,13 @@ int orc_verify_tree_stochastic(const void *target, const void *draft, int dtype,
                 const int32_t x = tok[n];
                 const double fx = f[x], qx = q[x];
                 int ok;
-                if (qx > 0.0) ok = (double)u[(int64_t)b * (N + 1) + n] < fx / qx;
-                else ok = fx > 0.0;
+                if (qx > 0.0) {
+                    const double uu = (double)u[(int64_t)b * (N + 1) + n], ratio = fx / qx;
+                    ok = uu < ratio;
+                    const double big = uu > ratio ? uu : ratio;
+                    const double m = big > 0.0 ? fabs(uu - ratio) / big : 0.0;
+                    if (m < closest) closest = m;
+                } else ok = fx > 0.0;
                 if (ok) {
                     accepted_node[(int64_t)b * L + acc] = n;
                     ++acc;
@@ -957,7 +969,13 @@ int orc_verify_tree_stochastic(const void *target, const void *draft, int dtype,
                         cum += f[v];
                         if (f[v] > 0.0) {
                             last_pos = v;
-                            if (cum >= thr) { token = v; break; }
+                            if (cum >= thr) {
+                                token = v;
+                                const double up = (cum - thr) / R, down = (thr - (cum - f[v])) / R;
+                                const double m = up < down ? up : down;
+                                if (m < closest) closest = m;
+                                break;
+                            }
                         }
                     }
                     if (token < 0) token = last_pos;    /* rounding at the very top of the CDF */
@@ -968,6 +986,7 @@ int orc_verify_tree_stochastic(const void *target, const void *draft, int dtype,
         accepted_len[b] = acc;
         next_token[b] = (int32_t)token;
         if (row_status) row_status[b] = status;
+        if (margin) margin[b] = closest;
         free(f);
         free(q);
     }

@@ -112,3 +112,16 @@ def test_flags_and_depth_limit():
     assert oracle.verify_tree_stochastic(bad, drf, tree, u).row_status.item() & oracle.NONFINITE_INPUT
     o = oracle.verify_tree_stochastic(tgt, drf[:, :1], tree, u)   # L = 1: the walk stops after one node
     assert o.accepted_len.item() == 1 and o.accepted_node.tolist() == [[0]]
+
+
+def test_margin_of_the_closest_decision_by_hand():
+    p, q = [0.5, 0.3, 0.2], [0.2, 0.7, 0.1]
+    # one acceptance test at ratio 3/7 with u = 0.42, then the bonus draw from (0.25, 0.25, 0.5) at u = 0.6:
+    # token 2's step of the cumulative sum is (0.5, 1.0], so the draw is 0.1 from its lower end
+    o = _two_siblings(p, q, [1, 0], 0.42, 0.0, 0.6)
+    r = 3.0 / 7.0
+    assert o.margin.item() == pytest.approx(min((r - 0.42) / r, 0.1), rel=1e-5)
+    # rejected at 0.43 (margin (0.43 - 3/7) / 0.43), second child accepted far from its ratio (3.75 against
+    # 0.999), bonus draw at 0.1 from (0.25, 0.25, 0.5): 0.1 from the lower end of token 0's step
+    o = _two_siblings(p, q, [1, 0], 0.43, 0.999, 0.1)
+    assert o.margin.item() == pytest.approx((0.43 - r) / 0.43, rel=1e-4)
