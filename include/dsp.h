@@ -507,8 +507,15 @@ int32_t dsp_residual_sample(const void *target_rows, const void *draft_rows, int
  * f(v) > 0 and sum_{w<=v} f(w) >= u[b,N] * sum_w f(w); R = 0 gives the argmax of
  * the node's target row and DSP_ROW_ZERO_RESIDUAL.  draft_logits [B,L,V];
  * u float [B,N+1] in [0,1).  At most DSP_MAX_W children of one node are tried (a
- * tree of dsp_beam_tree has no more).  Sums run in double in a fixed order.
- * workspace: dsp_verify_tree_workspace_bytes(B, N, V, dtype), 256-byte aligned.
+ * tree of dsp_beam_tree has no more).  The acceptance test is evaluated in double
+ * from the two logits, the rows' log-sum-exp and the residual masses; the sums over
+ * a row (log-sum-exp, residual mass, the cumulative sum of the emitted token) add
+ * fp32 terms in double in a fixed order: a decision closer than about 1e-6
+ * (relative) to going the other way may differ from exact arithmetic.  The draft
+ * rows 0 .. min(L, N+1)-1 are read once more than the walk needs them (their
+ * log-sum-exp is formed for all batch rows up front).
+ * workspace: dsp_verify_tree_workspace_bytes(B, N, V, dtype), 256-byte aligned
+ * (one size for both rules).
  * Errors : INVALID_ARG, UNSUPPORTED (W > DSP_MAX_W, L > DSP_MAX_L,
  *          N + 1 > DSP_MAX_L, dtype), WORKSPACE, CUDA.
  */

@@ -152,6 +152,22 @@ template <> struct Elem<float> {
                      fmaxf(__uint_as_float(v.z), __uint_as_float(v.w)));
     }
 };
+// p(v) = 2^(x*kLog2e - c2) with c2 = lse*log2(e) split as hi + lo (lo folded into `corr`).
+struct RowProb {
+    float nchi;     // -c2_hi
+    float corr;     // 2^(-c2_lo)
+};
+__device__ __forceinline__ RowProb row_prob(double lse) {
+    const double c2 = lse / kLn2;
+    RowProb r;
+    const float hi = (float)c2;
+    r.nchi = -hi;
+    r.corr = (float)exp2(-(c2 - (double)hi));
+    return r;
+}
+__device__ __forceinline__ float prob(float x, const RowProb &r) {
+    return __fmul_rn(ex2_approx(fmaf(x, kLog2e, r.nchi)), r.corr);
+}
 constexpr int kVpt = 6;                         // vectors per thread per tile
 
 template <typename DT> __host__ __device__ constexpr int tile_elems() { return kThreads * kVpt * Elem<DT>::N; }

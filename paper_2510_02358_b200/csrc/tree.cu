@@ -12,6 +12,7 @@
 // carries that token.
 #include "dsp_common.cuh"
 #include "dsp_internal.h"
+#include "stream_core.cuh"
 
 namespace dsp {
 
@@ -128,18 +129,41 @@ __global__ void __launch_bounds__(kThreads) tree_walk_kernel(const WalkArgs a) {
     }
 }
 
-struct TreeWs {
-    size_t off_masked, off_conf, off_left, off_unmask, total;
-};
-static TreeWs tree_ws_layout(int64_t B, int64_t rows, size_t unmask_bytes) {
+TreeWs tree_ws_layout(int64_t B, int64_t rows, int V, int dtype, size_t unmask_bytes) {
     TreeWs w;
     size_t o = 0;
-    w.off_masked = o; o += align_up((size_t)(B * rows), 256);
-    w.off_conf = o;   o += align_up((size_t)(B * rows) * 4, 256);
-    w.off_left = o;   o += align_up((size_t)B * 4, 256);
-    w.off_unmask = o; o += align_up(unmask_bytes, 256);
+    w.off_masked = o;  o += align_up((size_t)(B * rows), 256);
+    w.off_conf = o;    o += align_up((size_t)(B * rows) * 4, 256);
+    w.off_left = o;    o += align_up((size_t)B * 4, 256);
+    w.off_unmask = o;  o += align_up(unmask_bytes, 256);
+    // the stochastic rule only: log-sum-exp of the target and the draft rows, scratch outputs of the
+    // pass over the draft rows, chunk sums of each batch row's latest pass
+    w.nchunks = (V + tree_chunk_elems(dtype) - 1) / tree_chunk_elems(dtype);
+    w.off_tlse = o;    o += align_up((size_t)(B * rows) * 8, 256);
+    w.off_dlse = o;    o += align_up((size_t)(B * rows) * 8, 256);
+    w.off_dargmax = o; o += align_up((size_t)(B * rows) * 4, 256);
+    w.off_dstatus = o; o += align_up((size_t)B * 4, 256);
+    w.off_chunks = o;  o += align_up((size_t)B * w.nchunks * 8, 256);
     w.total = o;
     return w;
+}
+
+// Scratch of the row-statistics kernels for any number of rows per batch row up to N + 1 (the
+// target rows are N + 1, the draft rows fewer, and fewer rows are cut into more slices).
+int32_t tree_unmask_bytes(int32_t B, int32_t N, int32_t V, int32_t dtype, size_t *bytes) {
+    // From one slice per row on (B * rows at least the number of CTAs wanted) the size grows with the
+    // rows: only the counts below that and the largest count need a look.
+    size_t most = 0;
+    const long long few = slice_target_ctas() / (B > 0 ? B : 1) + 1;
+    for (int32_t rows = 1; rows <= N + 1; ++rows) {
+        if (rows > few && rows < N + 1) rows = N + 1;
+        size_t n = 0;
+        const int32_t rc = dsp_unmask_workspace_bytes(B, rows, V, dtype, &n);
+        if (rc != DSP_OK) return rc;
+        most = n > most ? n : most;
+    }
+    *bytes = most;
+    return DSP_OK;
 }
 
 }  // namespace dsp
@@ -151,12 +175,13 @@ using namespace dsp;
 // refinement step: nothing is revealed (n_update = 0), so its `tokens` argument is never written.
 int32_t dsp::tree_row_stats(const void *target_logits, int32_t dtype, int32_t B, int32_t N, int32_t V,
                             int64_t stride_b, int64_t stride_l, const int32_t *n_nodes, int32_t *tgt_argmax,
-                            uint32_t *row_status, void *workspace, size_t workspace_bytes, cudaStream_t st) {
+                            bool with_lse, uint32_t *row_status, void *workspace, size_t workspace_bytes,
+                            cudaStream_t st) {
     if ((reinterpret_cast<uintptr_t>(workspace) & 255) != 0) return DSP_ERR_INVALID_ARG;
     size_t un = 0;
-    const int32_t rc = dsp_unmask_workspace_bytes(B, N + 1, V, dtype, &un);
+    const int32_t rc = tree_unmask_bytes(B, N, V, dtype, &un);
     if (rc != DSP_OK) return rc;
-    const TreeWs w = tree_ws_layout(B, N + 1, un);
+    const TreeWs w = tree_ws_layout(B, N + 1, V, dtype, un);
     if (workspace_bytes < w.total) return DSP_ERR_WORKSPACE;
     unsigned char *ws = static_cast<unsigned char *>(workspace);
     uint8_t *masked = ws + w.off_masked;
@@ -166,7 +191,29 @@ int32_t dsp::tree_row_stats(const void *target_logits, int32_t dtype, int32_t B,
     tree_rows_kernel<<<(unsigned)((cells + 255) / 256), 256, 0, st>>>(B, N, n_nodes, masked);
     DSP_CUDA_TRY(cudaGetLastError());
     return unmask_impl(target_logits, dtype, B, N + 1, V, stride_b, stride_l, 0, tgt_argmax, masked, tgt_argmax, conf,
-                       left, row_status, ws + w.off_unmask, un, st);
+                       with_lse ? reinterpret_cast<double *>(ws + w.off_tlse) : nullptr, left, row_status,
+                       ws + w.off_unmask, un, st);
+}
+
+// Log-sum-exp of the first Ld draft rows of every batch row into the workspace (NaN for a row with
+// NaN / +inf or no finite logit: the walk flags the batch row if it uses such a row), by the same
+// kernels; to be called after tree_row_stats, whose scratch it takes over.
+int32_t dsp::tree_draft_stats(const void *draft_logits, int32_t dtype, int32_t B, int32_t N, int32_t Ld, int32_t V,
+                              int64_t stride_b, int64_t stride_l, void *workspace, size_t workspace_bytes,
+                              cudaStream_t st) {
+    size_t un = 0;
+    const int32_t rc = tree_unmask_bytes(B, N, V, dtype, &un);
+    if (rc != DSP_OK) return rc;
+    const TreeWs w = tree_ws_layout(B, N + 1, V, dtype, un);
+    if (workspace_bytes < w.total || Ld < 1 || Ld > N + 1) return DSP_ERR_WORKSPACE;
+    unsigned char *ws = static_cast<unsigned char *>(workspace);
+    uint8_t *masked = ws + w.off_masked;
+    DSP_CUDA_TRY(cudaMemsetAsync(masked, 1, (size_t)B * Ld, st));                  // every row is read
+    int32_t *dargmax = reinterpret_cast<int32_t *>(ws + w.off_dargmax);
+    return unmask_impl(draft_logits, dtype, B, Ld, V, stride_b, stride_l, 0, dargmax, masked, dargmax,
+                       reinterpret_cast<float *>(ws + w.off_conf), reinterpret_cast<double *>(ws + w.off_dlse),
+                       reinterpret_cast<int32_t *>(ws + w.off_left), reinterpret_cast<uint32_t *>(ws + w.off_dstatus),
+                       ws + w.off_unmask, un, st);
 }
 
 extern "C" int32_t dsp_beam_tree(const int32_t *beam_ids, const int32_t *path_len, int32_t B, int32_t W, int32_t L,
@@ -191,9 +238,9 @@ extern "C" int32_t dsp_verify_tree_workspace_bytes(int32_t B, int32_t N, int32_t
     if (!bytes || B < 0 || N < 1 || V < 1) return DSP_ERR_INVALID_ARG;
     if (N + 1 > DSP_MAX_L) return DSP_ERR_UNSUPPORTED;
     size_t un = 0;
-    const int32_t rc = dsp_unmask_workspace_bytes(B, N + 1, V, dtype, &un);
+    const int32_t rc = tree_unmask_bytes(B, N, V, dtype, &un);
     if (rc != DSP_OK) return rc;
-    *bytes = tree_ws_layout(B > 0 ? B : 1, N + 1, un).total;
+    *bytes = tree_ws_layout(B > 0 ? B : 1, N + 1, V, dtype, un).total;
     return DSP_OK;
 }
 
@@ -211,8 +258,8 @@ extern "C" int32_t dsp_verify_tree(const void *target_logits, int32_t dtype, int
         !tgt_argmax || !row_status || !workspace)
         return DSP_ERR_INVALID_ARG;
     cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
-    const int32_t rc = tree_row_stats(target_logits, dtype, B, N, V, stride_b, stride_l, n_nodes, tgt_argmax, row_status,
-                                      workspace, workspace_bytes, st);
+    const int32_t rc = tree_row_stats(target_logits, dtype, B, N, V, stride_b, stride_l, n_nodes, tgt_argmax, false,
+                                      row_status, workspace, workspace_bytes, st);
     if (rc != DSP_OK) return rc;
     WalkArgs k;
     k.B = B; k.N = N; k.L = L;

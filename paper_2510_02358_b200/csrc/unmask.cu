@@ -23,6 +23,7 @@ struct UnmaskArgs {
     uint8_t *masked;
     int32_t *argmax;
     float *confidence;
+    double *lse64;            // [B*L] or null: the rows' log-sum-exp (NaN: not computed or not finite)
     int32_t *n_left;
     uint32_t *row_status;
     int nslices, slice_elems, ntiles_row, nstages;
@@ -86,10 +87,11 @@ __device__ bool warp_row_stats_elementwise(const DT *__restrict__ row, int V, in
 
 // One row is done (am / conf: its argmax and confidence, -1 / -inf for a row that was not masked);
 // the warp arriving last for a batch row reveals the best n_update masked positions.  One warp.
-__device__ void unmask_row_done(const UnmaskArgs &a, long long row, int b, int am, float conf, int lane) {
+__device__ void unmask_row_done(const UnmaskArgs &a, long long row, int b, int am, float conf, double lse, int lane) {
     if (lane == 0) {
         a.argmax[row] = am;
         a.confidence[row] = conf;
+        if (a.lse64) a.lse64[row] = lse;
     }
     // ---- last row of this batch row: rank the masked positions and reveal the best ----
     __threadfence();
@@ -145,7 +147,7 @@ __global__ void __launch_bounds__(kThreads, 3) unmask_scan_kernel(const UnmaskAr
     const int lane = threadIdx.x & 31;
     if (!a.masked[row]) {                                // whole CTA alike
         grid_dependency_wait();                          // the tickets are prepared by the kernel before
-        if (slice == 0 && threadIdx.x < 32) unmask_row_done(a, row, b, -1, -CUDART_INF_F, lane);
+        if (slice == 0 && threadIdx.x < 32) unmask_row_done(a, row, b, -1, -CUDART_INF_F, CUDART_NAN, lane);
         return;
     }
     const DT *rowp = reinterpret_cast<const DT *>(a.logits) + b * a.stride_b + l * a.stride_l;
@@ -161,7 +163,7 @@ __global__ void __launch_bounds__(kThreads, 3) unmask_scan_kernel(const UnmaskAr
     float conf = -CUDART_INF_F;
     if (ok) conf = (float)((double)key_value(best) - lse);
     else if (lane == 0) atomicOr(&a.b_status[b], DSP_ROW_NONFINITE_INPUT);
-    unmask_row_done(a, row, b, am, conf, lane);
+    unmask_row_done(a, row, b, am, conf, ok ? lse : CUDART_NAN, lane);
 }
 
 // Layouts that cannot be streamed: one warp per row, element by element.
@@ -174,13 +176,16 @@ __global__ void __launch_bounds__(kThreads) unmask_rows_kernel(const UnmaskArgs 
     const DT *rowp = reinterpret_cast<const DT *>(a.logits) + b * a.stride_b + l * a.stride_l;
     int am = -1;
     float conf = -CUDART_INF_F;
+    double lse_out = CUDART_NAN;
     if (a.masked[row]) {                                 // read before anyone's update: updates follow the last ticket
         float xmax = 0.f;
         double lse = 0.0;
-        if (warp_row_stats_elementwise<DT>(rowp, a.V, lane, am, xmax, lse)) conf = (float)((double)xmax - lse);
-        else if (lane == 0) atomicOr(&a.b_status[b], DSP_ROW_NONFINITE_INPUT);
+        if (warp_row_stats_elementwise<DT>(rowp, a.V, lane, am, xmax, lse)) {
+            conf = (float)((double)xmax - lse);
+            lse_out = lse;
+        } else if (lane == 0) atomicOr(&a.b_status[b], DSP_ROW_NONFINITE_INPUT);
     }
-    unmask_row_done(a, row, b, am, conf, lane);
+    unmask_row_done(a, row, b, am, conf, lse_out, lane);
 }
 
 template <typename DT>
@@ -244,7 +249,7 @@ extern "C" int32_t dsp_unmask_workspace_bytes(int32_t B, int32_t L, int32_t V, i
 
 int32_t dsp::unmask_impl(const void *logits, int32_t dtype, int32_t B, int32_t L, int32_t V,
                          int64_t stride_b, int64_t stride_l, int32_t n_update,
-                         int32_t *tokens, uint8_t *masked, int32_t *argmax, float *confidence,
+                         int32_t *tokens, uint8_t *masked, int32_t *argmax, float *confidence, double *lse64,
                          int32_t *n_left, uint32_t *row_status,
                          void *workspace, size_t workspace_bytes, cudaStream_t st) {
     const int32_t rc = check_unmask_shape(B, L, V, dtype);
@@ -263,7 +268,7 @@ int32_t dsp::unmask_impl(const void *logits, int32_t dtype, int32_t B, int32_t L
     a.B = B; a.L = L; a.V = V;
     a.stride_b = stride_b; a.stride_l = stride_l;
     a.n_update = n_update;
-    a.tokens = tokens; a.masked = masked; a.argmax = argmax; a.confidence = confidence;
+    a.tokens = tokens; a.masked = masked; a.argmax = argmax; a.confidence = confidence; a.lse64 = lse64;
     a.n_left = n_left; a.row_status = row_status;
     return dtype == DSP_BF16 ? launch_unmask<__nv_bfloat16>(a, workspace, workspace_bytes, st)
                              : launch_unmask<float>(a, workspace, workspace_bytes, st);
@@ -275,6 +280,6 @@ extern "C" int32_t dsp_unmask_step(const void *logits, int32_t dtype, int32_t B,
                                    int32_t *n_left, uint32_t *row_status,
                                    void *workspace, size_t workspace_bytes, dsp_stream_t stream) {
     if (n_update < 1) return DSP_ERR_INVALID_ARG;
-    return unmask_impl(logits, dtype, B, L, V, stride_b, stride_l, n_update, tokens, masked, argmax, confidence,
+    return unmask_impl(logits, dtype, B, L, V, stride_b, stride_l, n_update, tokens, masked, argmax, confidence, nullptr,
                        n_left, row_status, workspace, workspace_bytes, reinterpret_cast<cudaStream_t>(stream));
 }

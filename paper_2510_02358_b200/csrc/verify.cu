@@ -280,22 +280,6 @@ __global__ void __launch_bounds__(kThreads) accept_kernel(const VerifyArgs a) {
 
 // ---- residual / bonus sampling -------------------------------------------------------------
 
-// p(v) = 2^(x*kLog2e - c2) with c2 = lse*log2(e) split as hi + lo (lo folded into `corr`).
-struct RowProb {
-    float nchi;     // -c2_hi
-    float corr;     // 2^(-c2_lo)
-};
-__device__ __forceinline__ RowProb row_prob(double lse) {
-    const double c2 = lse / kLn2;
-    RowProb r;
-    const float hi = (float)c2;
-    r.nchi = -hi;
-    r.corr = (float)exp2(-(c2 - (double)hi));
-    return r;
-}
-__device__ __forceinline__ float prob(float x, const RowProb &r) {
-    return __fmul_rn(ex2_approx(fmaf(x, kLog2e, r.nchi)), r.corr);
-}
 __device__ __forceinline__ float residual(float xt, float xd, const RowProb &pt, const RowProb &pd, bool has_q) {
     const float p = prob(xt, pt);
     const float q = has_q ? prob(xd, pd) : 0.f;

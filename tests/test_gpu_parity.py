@@ -701,6 +701,9 @@ def test_beam_tree_and_its_greedy_verification(B, L, V, K, W, dtype):
     (3, 6, 20000, 4, 8, torch.bfloat16, 0.3),     # target close to the draft: deep walks
     (3, 4, 5003, 3, 4, torch.bfloat16, 1.5),      # rows that are not 16-byte aligned; many rejections
     (2, 8, 1000, 2, 1, torch.float32, 0.5),       # one beam: the single-path rule
+    (2, 3, 300000, 3, 2, torch.bfloat16, 1.0),    # more chunks than threads: several chunks per thread in the draw
+    (2, 4, 152064, 4, 4, torch.bfloat16, 2.5),    # a target far from the draft: chains of rejections
+    (3, 5, 40001, 3, 3, torch.float32, 0.1),      # fp32 rows that are not 16-byte aligned; long accepted walks
 ])
 def test_stochastic_tree_verification_matches_oracle(B, L, V, K, W, dtype, sigma):
     inp = _to(wl.tiny_random(B, L, V, dtype=dtype, seed=L * 3 + W))
@@ -727,8 +730,16 @@ def test_stochastic_tree_verification_matches_oracle(B, L, V, K, W, dtype, sigma
     out = dsp.dsp_verify_tree_stochastic(target.to(DEV), inp["draft"], tree, u.to(DEV))
     torch.cuda.synchronize()
     assert (o.row_status == 0).all() and (out.row_status.cpu() == 0).all()
-    for name in ("accepted_len", "accepted_node", "next_token"):
-        assert torch.equal(getattr(out, name).cpu(), getattr(o, name)), name
+    # The walk's row sums are fp32 terms added up in double, the oracle's are double throughout: a batch
+    # row may differ only if its closest decision (acceptance ratio against u, or the emitted token's step
+    # of the cumulative sum against u) was within 1e-5 of going the other way, and that is rare.
+    near = 0
+    for b in range(B):
+        same = all(torch.equal(getattr(out, name).cpu()[b], getattr(o, name)[b])
+                   for name in ("accepted_len", "accepted_node", "next_token"))
+        assert same or o.margin[b] < 1e-5, f"batch row {b} differs with margin {o.margin[b]:.3g}"
+        near += 0 if same else 1
+    assert near <= 1
     assert (out.next_token >= 0).all()
     if W > 1:                                                # one path alone would have done no better
         single = oracle.verify_tree_stochastic(target, draft, SimpleNamespace(
