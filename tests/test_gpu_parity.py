@@ -704,6 +704,8 @@ def test_beam_tree_and_its_greedy_verification(B, L, V, K, W, dtype):
     (2, 3, 300000, 3, 2, torch.bfloat16, 1.0),    # more chunks than threads: several chunks per thread in the draw
     (2, 4, 152064, 4, 4, torch.bfloat16, 2.5),    # a target far from the draft: chains of rejections
     (3, 5, 40001, 3, 3, torch.float32, 0.1),      # fp32 rows that are not 16-byte aligned; long accepted walks
+    (2, 16, 20000, 4, 4, torch.bfloat16, 0.4),    # few draft rows beside many target rows: the draft rows' statistics
+                                                  # cut their rows into more slices than the target rows' (workspace sizing)
 ])
 def test_stochastic_tree_verification_matches_oracle(B, L, V, K, W, dtype, sigma):
     inp = _to(wl.tiny_random(B, L, V, dtype=dtype, seed=L * 3 + W))
