@@ -93,6 +93,30 @@ def test_edge_shapes(B, L, V, K, W, dtype):
         assert rep["near_accept"] + rep["near_token"] + rep["near_tau"] <= 1
 
 
+@pytest.mark.parametrize("seed", range(6))
+def test_whole_step_on_random_shapes(seed):
+    """Seeded random shapes through the three calls and through the single call: both dtypes, aligned and
+    unaligned vocabularies, one to several tiles, pruning on and off, EOS, greedy / mixed batches."""
+    rng = np.random.default_rng(500 + seed)
+    near = 0
+    for case in range(4):
+        B = int(rng.integers(1, 6))
+        L = int(rng.integers(1, 20))
+        V = int(rng.choice([7, 100, 1000, 4096, 6151, 12288, 20000, 33000]))
+        K = int(rng.choice([1, 3, 8, 16, 32]))
+        W = int(rng.choice([1, 2, 4, 8, 16]))
+        dtype = torch.bfloat16 if rng.integers(0, 2) else torch.float32
+        tau = float(rng.choice([0.0, 0.5, 0.8, 0.95]))
+        eos = int(V - 1) if rng.integers(0, 2) else -1
+        greedy = bool(rng.integers(0, 3) == 0)
+        inp = _to(wl.tiny_random(B, L, V, dtype=dtype, seed=seed * 10 + case, sigma_t=float(rng.choice([0.2, 0.7, 1.5]))))
+        p = dict(K=K, W=W, tau=tau, lam=float(rng.choice([0.25, 0.5, 0.75])), eos_id=eos, all_greedy=greedy)
+        for fused in (False, True):
+            rep = check_step(gpu_step(inp, fused=fused, **p), inp, **p)
+            near += rep["near_accept"] + rep["near_token"] + rep["near_tau"]
+    assert near <= 4
+
+
 @pytest.mark.parametrize("V,dtype", [(12288 + 64, torch.bfloat16), (6144 + 32, torch.float32),
                                      (3 * 12288 + 8, torch.bfloat16)])
 def test_short_ragged_tail_in_a_slice_of_its_own(V, dtype):
