@@ -230,7 +230,7 @@ def time_workload(w, device, steps, warmup, dist=None, stages=True, seed_base=0,
 
     e0.record()
     for i in range(steps):
-        if stages and i % 8 == 0:                        # every 8th timed step carries the events
+        if stages and i % 16 == 0:                       # every 16th timed step carries the events
             profiled_step(sets[i % len(sets)])
         else:
             st.step(sets[i % len(sets)])
