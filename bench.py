@@ -48,6 +48,11 @@ HEADLINE = 4
 NCU_TRAFFIC_BYTES = {4: 640_400_000 + 626_800_000}
 
 
+# The streaming kernels' own time is sampled inside the timed region on one step in this many
+# (the events on both streams cost such a step 20 us or more), and on 32 steps right after it.
+PROFILE_EVERY = 16
+
+
 def measured_peak():
     p = os.path.join(ROOT, "MEASURED_PEAKS.json")
     try:
@@ -230,7 +235,7 @@ def time_workload(w, device, steps, warmup, dist=None, stages=True, seed_base=0,
 
     e0.record()
     for i in range(steps):
-        if stages and i % 16 == 0:                       # every 16th timed step carries the events
+        if stages and i % PROFILE_EVERY == 0:            # one timed step in PROFILE_EVERY carries the events
             profiled_step(sets[i % len(sets)])
         else:
             st.step(sets[i % len(sets)])
