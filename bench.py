@@ -276,7 +276,7 @@ def time_workload(w, device, steps, warmup, dist=None, stages=True, seed_base=0,
         for i in range(min(warmup, 2 * len(graphs))):
             graphs[i % len(graphs)].launch()
         torch.cuda.synchronize()
-        n = min(steps, 500)
+        n = steps                                        # as many replays as timed steps: the same load on the power limit
         g0, g1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         g0.record()
         for i in range(n):
